@@ -1,0 +1,365 @@
+// Decode / tree-verify attention over one shared prompt KV segment plus one private segment per stream
+// (Sec. 3.4, App. A.1: a stream's rows see the prefill segment and their own segment only) with the DS2D
+// tree-ancestor mask on the rows being verified (Sec. 3.5, App. A.2).  No mask tensor exists: stream
+// isolation is the addressing, the tree mask is one 64-bit word per row.
+//
+// Split-K online softmax: the key range is cut into chunks; a CTA takes (kv head, chunk, block of 64 query
+// rows) and produces un-normalised partial outputs with their running max and sum; a merge kernel combines
+// the chunks of a row by log-sum-exp.  A shared-prefix chunk is loaded once and used by the rows of ALL
+// streams and all query heads of the kv head; an own-segment chunk is used by that stream's rows.
+// QK^T and PV run on the tensor cores (mma.sync m16n8k16, fp32 accumulate), K/V tiles are staged through
+// shared memory with a two-stage cp.async pipeline.
+#include "common.cuh"
+
+namespace mlora {
+
+constexpr int ATT_WARPS = 4;
+constexpr int ATT_THREADS = ATT_WARPS * 32;
+constexpr int ATT_ROWS = ATT_WARPS * 16;   // query rows per CTA
+constexpr int ATT_KEYS = 64;               // keys per pipeline tile
+
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+  const uint32_t sa = (uint32_t)__cvta_generic_to_shared(smem);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(gmem));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N)); }
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* smem) {
+  const uint32_t sa = (uint32_t)__cvta_generic_to_shared(smem);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(sa));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* smem) {
+  const uint32_t sa = (uint32_t)__cvta_generic_to_shared(smem);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(sa));
+}
+
+struct AttnItem {
+  int is_own, s, chunk, row_block;
+};
+
+__device__ __forceinline__ AttnItem decode_item(const AttnArgs& p, int item, int rb_all, int rb_own) {
+  AttnItem it;
+  const int n_prefix_items = p.n_prefix_chunks * rb_all;
+  if (item < n_prefix_items) {
+    it.is_own = 0; it.s = 0;
+    it.chunk = item / rb_all;
+    it.row_block = item % rb_all;
+  } else {
+    item -= n_prefix_items;
+    it.is_own = 1;
+    it.row_block = item % rb_own;
+    item /= rb_own;
+    it.chunk = item % p.n_own_chunks;
+    it.s = item / p.n_own_chunks;
+  }
+  return it;
+}
+
+template <int HD>
+__global__ void __launch_bounds__(ATT_THREADS) attn_partial_kernel(const AttnArgs p, const int rb_all, const int rb_own,
+                                                                  const float scale_log2) {
+  constexpr int STRIDE = HD + 8;                      // halves per shared-memory row
+  constexpr int KSTEPS = HD / 16;
+  constexpr int DT = HD / 8;                          // output n8-tiles
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __half* Qs = reinterpret_cast<__half*>(smem_raw);                   // [ATT_ROWS][STRIDE]
+  __half* Ks = Qs + ATT_ROWS * STRIDE;                                // [2][ATT_KEYS][STRIDE]
+  __half* Vs = Ks + 2 * ATT_KEYS * STRIDE;                            // [2][ATT_KEYS][STRIDE]
+
+  const int kh = blockIdx.y;
+  const int g_heads = p.Hq / p.Hkv;
+  const AttnItem it = decode_item(p, blockIdx.x, rb_all, rb_own);
+  const int rows_per_stream = p.T * g_heads;
+  const int R_all = p.n * rows_per_stream;
+
+  int key_begin, key_end, S = 0;
+  const __half *kbase, *vbase;
+  int row_lo, row_hi;                                                  // virtual rows [row_lo, row_hi) within the kv head
+  if (!it.is_own) {
+    key_begin = it.chunk * p.prefix_chunk;
+    key_end = min(p.P, key_begin + p.prefix_chunk);
+    kbase = p.prefix_k + (size_t)kh * p.prefix_head_stride;
+    vbase = p.prefix_v + (size_t)kh * p.prefix_head_stride;
+    row_lo = it.row_block * ATT_ROWS;
+    row_hi = min(R_all, row_lo + ATT_ROWS);
+  } else {
+    S = p.suffix_len[it.s];
+    key_begin = it.chunk * p.own_chunk;
+    key_end = min(S + p.T, key_begin + p.own_chunk);
+    kbase = p.own_k + (size_t)it.s * p.own_stream_stride + (size_t)kh * p.own_head_stride;
+    vbase = p.own_v + (size_t)it.s * p.own_stream_stride + (size_t)kh * p.own_head_stride;
+    row_lo = it.s * rows_per_stream + it.row_block * ATT_ROWS;
+    row_hi = min((it.s + 1) * rows_per_stream, row_lo + ATT_ROWS);
+  }
+  if (key_begin >= key_end) return;                                    // nothing here (merge skips this slot too)
+  const int slot = it.is_own ? p.n_prefix_chunks + it.chunk : it.chunk;
+  const int slots = p.n_prefix_chunks + p.n_own_chunks;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int n_tiles = (key_end - key_begin + ATT_KEYS - 1) / ATT_KEYS;
+
+  auto load_kv_tile = [&](int tile, int stage) {
+    const int k0 = key_begin + tile * ATT_KEYS;
+    __half* kd = Ks + (size_t)stage * ATT_KEYS * STRIDE;
+    __half* vd = Vs + (size_t)stage * ATT_KEYS * STRIDE;
+    constexpr int VPR = HD / 8;                                        // 16-byte pieces per row
+    for (int i = threadIdx.x; i < ATT_KEYS * VPR; i += ATT_THREADS) {
+      const int r = i / VPR, c = (i % VPR) * 8;
+      const int key = min(k0 + r, key_end - 1);                        // rows past the end repeat the last valid key
+      cp_async16(kd + (size_t)r * STRIDE + c, kbase + (size_t)key * HD + c);
+      cp_async16(vd + (size_t)r * STRIDE + c, vbase + (size_t)key * HD + c);
+    }
+  };
+
+  load_kv_tile(0, 0);
+  cp_async_commit();
+
+  // query rows of this block -> shared memory (zero beyond the block's rows)
+  {
+    constexpr int VPR = HD / 8;
+    for (int i = threadIdx.x; i < ATT_ROWS * VPR; i += ATT_THREADS) {
+      const int r = i / VPR, c = (i % VPR) * 8;
+      const int v = row_lo + r;
+      uint4 val = make_uint4(0, 0, 0, 0);
+      if (v < row_hi) {
+        const int m = v / g_heads, j = v % g_heads;
+        val = *reinterpret_cast<const uint4*>(p.q + ((size_t)m * p.Hq + kh * g_heads + j) * HD + c);
+      }
+      *reinterpret_cast<uint4*>(Qs + (size_t)r * STRIDE + c) = val;
+    }
+  }
+  __syncthreads();
+
+  const bool warp_active = (row_lo + warp * 16) < row_hi;
+  uint32_t qf[KSTEPS][4];
+  if (warp_active) {
+#pragma unroll
+    for (int ks = 0; ks < KSTEPS; ++ks) {
+      const int mi = lane >> 3, r = lane & 7;
+      ldmatrix_x4(qf[ks], Qs + (size_t)(warp * 16 + (mi & 1) * 8 + r) * STRIDE + ks * 16 + (mi >> 1) * 8);
+    }
+  }
+
+  // per-row tree masks (own segment only): rows g and g+8 of the warp's tile
+  unsigned long long anc0 = ~0ull, anc1 = ~0ull;
+  if (it.is_own) {
+    const int v0 = row_lo + warp * 16 + g, v1 = v0 + 8;
+    anc0 = (v0 < row_hi) ? p.anc[v0 / g_heads] : 0ull;                 // v / g_heads = global row m = s*T + t
+    anc1 = (v1 < row_hi) ? p.anc[v1 / g_heads] : 0ull;
+  }
+
+  float o[DT][4];
+#pragma unroll
+  for (int i = 0; i < DT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+  float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
+
+  for (int tile = 0; tile < n_tiles; ++tile) {
+    const int stage = tile & 1;
+    if (tile + 1 < n_tiles) {
+      load_kv_tile(tile + 1, stage ^ 1);
+      cp_async_commit();
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
+    }
+    __syncthreads();
+    if (warp_active) {
+      const __half* kt = Ks + (size_t)stage * ATT_KEYS * STRIDE;
+      const __half* vt = Vs + (size_t)stage * ATT_KEYS * STRIDE;
+      float sacc[ATT_KEYS / 8][4];
+#pragma unroll
+      for (int nt = 0; nt < ATT_KEYS / 8; ++nt) {
+        sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ks += 2) {
+          uint32_t kb[4];
+          const int mi = lane >> 3, r = lane & 7;
+          ldmatrix_x4(kb, kt + (size_t)(nt * 8 + r) * STRIDE + ks * 16 + mi * 8);
+          mma_16816(sacc[nt], qf[ks], kb[0], kb[1]);
+          mma_16816(sacc[nt], qf[ks + 1], kb[2], kb[3]);
+        }
+      }
+      // scale, mask, running max
+      const int k0 = key_begin + tile * ATT_KEYS;
+      float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+      for (int nt = 0; nt < ATT_KEYS / 8; ++nt) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int key = k0 + nt * 8 + 2 * t + (e & 1);
+          bool ok = key < key_end;
+          if (it.is_own && key >= S) {
+            const unsigned long long a = (e & 2) ? anc1 : anc0;
+            ok = ok && ((a >> (key - S)) & 1ull);
+          }
+          const float v = ok ? sacc[nt][e] * scale_log2 : -INFINITY;
+          sacc[nt][e] = v;
+          mx[e >> 1] = fmaxf(mx[e >> 1], v);
+        }
+      }
+      float corr[2], msafe[2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+        mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
+        const float mnew = fmaxf(mrow[h], mx[h]);
+        msafe[h] = (mnew == -INFINITY) ? 0.f : mnew;
+        corr[h] = exp2f(mrow[h] - msafe[h]);                           // mrow = -inf -> 0
+        mrow[h] = mnew;
+      }
+      float ls[2] = {0.f, 0.f};
+      uint32_t pf[ATT_KEYS / 16][4];
+#pragma unroll
+      for (int nt = 0; nt < ATT_KEYS / 8; ++nt) {
+        const float p0 = exp2f(sacc[nt][0] - msafe[0]), p1 = exp2f(sacc[nt][1] - msafe[0]);
+        const float p2 = exp2f(sacc[nt][2] - msafe[1]), p3 = exp2f(sacc[nt][3] - msafe[1]);
+        ls[0] += p0 + p1;
+        ls[1] += p2 + p3;
+        pf[nt >> 1][(nt & 1) * 2 + 0] = h2_as_u32(__floats2half2_rn(p0, p1));
+        pf[nt >> 1][(nt & 1) * 2 + 1] = h2_as_u32(__floats2half2_rn(p2, p3));
+      }
+#pragma unroll
+      for (int h = 0; h < 2; ++h) lrow[h] = lrow[h] * corr[h] + ls[h];
+#pragma unroll
+      for (int dt = 0; dt < DT; ++dt) {
+        o[dt][0] *= corr[0]; o[dt][1] *= corr[0];
+        o[dt][2] *= corr[1]; o[dt][3] *= corr[1];
+      }
+#pragma unroll
+      for (int kk = 0; kk < ATT_KEYS / 16; ++kk) {
+#pragma unroll
+        for (int dt = 0; dt < DT; dt += 2) {
+          uint32_t vb[4];
+          const int mi = lane >> 3, r = lane & 7;
+          ldmatrix_x4_trans(vb, vt + (size_t)(kk * 16 + (mi & 1) * 8 + r) * STRIDE + (dt + (mi >> 1)) * 8);
+          mma_16816(o[dt], pf[kk], vb[0], vb[1]);
+          mma_16816(o[dt + 1], pf[kk], vb[2], vb[3]);
+        }
+      }
+    }
+    __syncthreads();                                                   // stage may be overwritten next iteration
+  }
+
+  if (!warp_active) return;
+  // partial results: un-normalised output, running max (log2 domain) and the lane-group's partial sum
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    lrow[h] += __shfl_xor_sync(0xffffffffu, lrow[h], 1);
+    lrow[h] += __shfl_xor_sync(0xffffffffu, lrow[h], 2);
+  }
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int v = row_lo + warp * 16 + g + 8 * h;
+    if (v >= row_hi) continue;
+    const size_t idx = ((size_t)kh * R_all + v) * slots + slot;
+    float* po = p.part_o + idx * HD;
+#pragma unroll
+    for (int dt = 0; dt < DT; ++dt)
+      *reinterpret_cast<float2*>(po + dt * 8 + 2 * t) = make_float2(o[dt][2 * h], o[dt][2 * h + 1]);
+    if (t == 0) *reinterpret_cast<float2*>(p.part_ml + idx * 2) = make_float2(mrow[h], lrow[h]);
+  }
+}
+
+// One warp per (row, query head): log-sum-exp merge of the row's chunks, output in fp16.
+__global__ void attn_merge_kernel(const AttnArgs p) {
+  const int w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  const int M = p.n * p.T;
+  if (w >= M * p.Hq) return;
+  const int m = w / p.Hq, hq = w % p.Hq;
+  const int g_heads = p.Hq / p.Hkv;
+  const int kh = hq / g_heads;
+  const int v = m * g_heads + hq % g_heads;
+  const int s = m / p.T;
+  const int R_all = M * g_heads;
+  const int slots = p.n_prefix_chunks + p.n_own_chunks;
+  const int own_valid = min(p.n_own_chunks, (p.suffix_len[s] + p.T + p.own_chunk - 1) / p.own_chunk);
+  const size_t base = ((size_t)kh * R_all + v) * slots;
+  float mmax = -INFINITY;
+  for (int i = 0; i < p.n_prefix_chunks + own_valid; ++i) mmax = fmaxf(mmax, p.part_ml[(base + i) * 2]);
+  const int hd = p.hd;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  float L = 0.f;
+  for (int i = 0; i < p.n_prefix_chunks + own_valid; ++i) {
+    const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + (base + i) * 2);
+    const float wgt = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - mmax);
+    L += wgt * ml.y;
+    const float* po = p.part_o + (base + i) * hd;
+    for (int e = 0; e * 32 + lane < hd; ++e) acc[e] = fmaf(wgt, po[e * 32 + lane], acc[e]);
+  }
+  const float inv = 1.f / L;
+  __half* out = p.out + ((size_t)m * p.Hq + hq) * hd;
+  for (int e = 0; e * 32 + lane < hd; ++e) out[e * 32 + lane] = __float2half_rn(acc[e] * inv);
+}
+
+void attn_plan(AttnArgs& a, int sm_count) {
+  const int g_heads = a.Hq / a.Hkv;
+  const int R_all = a.n * a.T * g_heads;
+  const int rb_all = (R_all + ATT_ROWS - 1) / ATT_ROWS;
+  const int rb_own = (a.T * g_heads + ATT_ROWS - 1) / ATT_ROWS;
+  const int target = 2 * sm_count;
+  // shared prefix: as many key chunks as it takes to fill the machine, at least 64 keys each
+  int want = target / (a.Hkv * rb_all);
+  if (want < 1) want = 1;
+  int tiles = (a.P + ATT_KEYS - 1) / ATT_KEYS;
+  if (tiles < 1) tiles = 1;
+  if (want > tiles) want = tiles;
+  int tiles_per_chunk = (tiles + want - 1) / want;
+  a.prefix_chunk = tiles_per_chunk * ATT_KEYS;
+  a.n_prefix_chunks = a.P > 0 ? (a.P + a.prefix_chunk - 1) / a.prefix_chunk : 0;
+  // own segments: there are already n * Hkv * rb_own CTAs per chunk
+  const int own_keys = a.suffix_bound + a.T;
+  want = target / (a.Hkv * a.n * rb_own);
+  if (want < 1) want = 1;
+  tiles = (own_keys + ATT_KEYS - 1) / ATT_KEYS;
+  if (want > tiles) want = tiles;
+  tiles_per_chunk = (tiles + want - 1) / want;
+  a.own_chunk = tiles_per_chunk * ATT_KEYS;
+  a.n_own_chunks = (own_keys + a.own_chunk - 1) / a.own_chunk;
+}
+
+size_t attn_workspace_floats(const AttnArgs& a) {
+  const int g_heads = a.Hq / a.Hkv;
+  const size_t R_all = (size_t)a.n * a.T * g_heads;
+  const size_t slots = a.n_prefix_chunks + a.n_own_chunks;
+  return (size_t)a.Hkv * R_all * slots * (a.hd + 2);
+}
+
+template <int HD>
+static cudaError_t launch_attn_hd(const AttnArgs& a, cudaStream_t st) {
+  const size_t smem = (size_t)(ATT_ROWS + 4 * ATT_KEYS) * (HD + 8) * sizeof(__half);
+  const int g_heads = a.Hq / a.Hkv;
+  const int rb_all = (a.n * a.T * g_heads + ATT_ROWS - 1) / ATT_ROWS;
+  const int rb_own = (a.T * g_heads + ATT_ROWS - 1) / ATT_ROWS;
+  const int items = a.n_prefix_chunks * rb_all + a.n * a.n_own_chunks * rb_own;
+  dim3 grid(items, a.Hkv);
+  const float scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
+  attn_partial_kernel<HD><<<grid, ATT_THREADS, smem, st>>>(a, rb_all, rb_own, scale_log2);
+  return cudaGetLastError();
+}
+
+cudaError_t init_attention() {
+  cudaError_t e = cudaFuncSetAttribute(attn_partial_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)((ATT_ROWS + 4 * ATT_KEYS) * (64 + 8) * sizeof(__half)));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attn_partial_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)((ATT_ROWS + 4 * ATT_KEYS) * (128 + 8) * sizeof(__half)));
+}
+
+cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st) {
+  if (a.hd == 64) return launch_attn_hd<64>(a, st);
+  if (a.hd == 128) return launch_attn_hd<128>(a, st);
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_attention_merge(const AttnArgs& a, cudaStream_t st) {
+  const int warps = a.n * a.T * a.Hq;
+  attn_merge_kernel<<<(warps + 3) / 4, 128, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace mlora

@@ -1,0 +1,175 @@
+// Shared device helpers and the kernel-launch interface between the translation units.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mlora {
+
+// ----------------------------------------------------------------------------- layout constants
+// Private weight layout ("fragment-major"): the [K][N] INT4 matrix is cut into tiles of 16 output
+// features x 64 input features.  A tile is 32 lanes x 16 bytes: lane (g = lane/4, t = lane%4) owns the
+// 16 consecutive input features k0+16t .. k0+16t+15 of output features n0+g and n0+g+8, so that one
+// 128-bit load per lane feeds four m16n8k16 tensor-core steps (the weights are the 16-wide operand).
+// Tiles are stored [n_tile][k_tile][lane] -- a warp streaming along K reads one contiguous run.
+// Word j (0..3) of the lane's uint4 holds input features k0+16t+4j+{0,1,2,3}:
+//   nibble 0/4: feature +0/+1 of row g      nibble 1/5: feature +0/+1 of row g+8
+//   nibble 2/6: feature +2/+3 of row g      nibble 3/7: feature +2/+3 of row g+8
+// Scales: uint32 [K/G][n_tile][8] -- entry g packs fp16 scale of row n0+g (low) and n0+g+8 (high).
+constexpr int TILE_N = 16;
+constexpr int TILE_K = 64;
+
+// GEMM CTA shape
+constexpr int GEMM_WARPS = 4;
+constexpr int GEMM_THREADS = GEMM_WARPS * 32;
+constexpr int GEMM_NB = GEMM_WARPS * TILE_N;   // output features per CTA
+constexpr int GEMM_PF = 8;                     // weight tiles in flight per lane
+constexpr int GEMM_MAX_MT = 16;                // m-tiles of 8 rows per CTA (128 rows)
+
+enum GemmMode { MODE_PLAIN = 0, MODE_QKV = 1, MODE_GATEUP = 2 };
+enum GemmEpi { EPI_F32 = 0, EPI_RESID = 1, EPI_SWIGLU = 2 };
+
+struct LoraSeg {
+  int proj_index;   // index into the adapter pointer tables (layer*7 + proj), or the plain table index 0
+  int n;            // logical output width of the segment
+};
+
+struct LoraArgs {
+  const int32_t* adapter_idx;     // dev: adapter of stream (row / rows_per_stream); nullptr => no LoRA
+  int rows_per_stream;
+  const __half* const* tabA;      // dev [n_slots][tab_stride]
+  const __half* const* tabB;
+  const float* scale;             // dev [n_slots]
+  int tab_stride;
+  int n_slots;
+  int rank;
+  int nseg;
+  LoraSeg seg[3];
+  float* T;                       // dev fp32 [M][nseg][rank], already multiplied by the adapter scale
+};
+
+struct GemmArgs {
+  const uint4* wq;
+  const uint32_t* sc;
+  int K, N, G;                    // N = physical (fused) width
+  const __half* h;                // [M][K]
+  int M;
+  int mode, epi;
+  int seg_n0, seg_n1;             // MODE_QKV: widths of the first two segments
+  float* out_f32; int ldo;        // EPI_F32
+  float* resid;                   // EPI_RESID: [M][N] in place
+  __half* out_f16;                // EPI_SWIGLU: [M][N/2]
+  float* partial;                 // split-K scratch [ksplit][M][N]
+  size_t partial_capacity;        // floats
+  unsigned* counters;             // zeroed, >= n_blocks * m_blocks entries
+  LoraArgs lora;
+};
+
+struct ShrinkArgs {
+  const float* x_f32;             // NORM mode: residual stream [M][K]
+  const __half* gain;             // NORM mode: RMSNorm gain
+  float eps;
+  const __half* h_in;             // PLAIN mode: fp16 input [M][K]
+  __half* h_out;                  // NORM mode: normalised fp16 rows written here
+  int M, K;
+  LoraArgs lora;                  // adapter_idx == nullptr: only the norm is done
+};
+
+struct AttnArgs {
+  const __half* q;                // [rows][Hq][hd]
+  const __half* prefix_k; const __half* prefix_v; size_t prefix_head_stride; int P;
+  const __half* own_k; const __half* own_v; size_t own_stream_stride, own_head_stride;
+  const int32_t* suffix_len;      // dev [n]
+  int suffix_bound;               // host upper bound on suffix_len
+  const unsigned long long* anc;  // dev [n][T] ancestor-or-self bit masks
+  int n, T, Hq, Hkv, hd;
+  __half* out;                    // [rows][Hq][hd]
+  float* part_o; float* part_ml;  // scratch
+  int n_prefix_chunks, prefix_chunk; // keys per prefix chunk (multiple of 64)
+  int n_own_chunks, own_chunk;
+};
+
+// ----------------------------------------------------------------------------- launchers
+cudaError_t init_gemm();        // opt-in shared-memory sizes; call once per process before the first launch
+cudaError_t init_shrink();
+cudaError_t init_attention();
+cudaError_t launch_repack(const uint8_t* qweight, const __half* scales, int K, int N, int G, uint4* wq,
+                          uint32_t* sc, int dst_tile_off, int dst_tile_stride, int dst_tiles, cudaStream_t st);
+cudaError_t launch_dequant(const uint4* wq, const uint32_t* sc, int K, int N, int G, int tile_off,
+                           int tile_stride, int tiles_phys, __half* out, cudaStream_t st);
+int gemm_pick_split(int K, int N, int M, size_t partial_capacity);
+cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
+cudaError_t launch_shrink(const ShrinkArgs& a, cudaStream_t st);
+cudaError_t launch_embed(const int32_t* tokens, const __half* embed, const __half* hidden_in, float* X, int M,
+                         int d, int vocab, int* status, cudaStream_t st);
+cudaError_t launch_tree_prep(const int32_t* parent, int n, int T, unsigned long long* anc, int32_t* depth,
+                             int* status, cudaStream_t st);
+cudaError_t launch_rope_kv(const float* qkv, int M, int T, int Hq, int Hkv, int hd, const float2* cs_table,
+                           int pos_base, const int32_t* suffix_len, const int32_t* depth, __half* q_out,
+                           __half* k_dst, __half* v_dst, size_t stream_stride, size_t head_stride, cudaStream_t st);
+void attn_plan(AttnArgs& a, int sm_count);
+size_t attn_workspace_floats(const AttnArgs& a);
+cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st);
+cudaError_t launch_attention_merge(const AttnArgs& a, cudaStream_t st);
+cudaError_t launch_argmax(const float* logits, int M, int V, int32_t* out, cudaStream_t st);
+cudaError_t launch_accept(const int32_t* tokens, const int32_t* parent, const int32_t* argmax, int n, int T,
+                          int32_t* acc_len, int32_t* acc_idx, int32_t* next, cudaStream_t st);
+cudaError_t launch_compact(__half* own_k, __half* own_v, size_t layer_stride, size_t stream_stride,
+                           size_t head_stride, int L, int n, int Hkv, int hd, const int32_t* suffix_len,
+                           const int32_t* acc_len, const int32_t* acc_idx, int T, cudaStream_t st);
+cudaError_t launch_advance(int32_t* suffix_len, const int32_t* acc_len, int n, int fixed, cudaStream_t st);
+cudaError_t launch_copy_rows_f32(const float* src, float* dst, size_t count, cudaStream_t st);
+
+// ----------------------------------------------------------------------------- device helpers
+#ifdef __CUDACC__
+__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint32_t ldg_nc_u32(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t h2_as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
+__device__ __forceinline__ __half2 u32_as_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
+
+// Eight INT4 weights -> four fp16x2 registers in m16n8k16 A-fragment order.  Each stored nibble u = q + 8
+// is placed into the mantissa of 1024.0 (giving 1024+u, or 1024+16u for the nibbles one hex digit up),
+// q = u - 8 is recovered exactly by one subtract / fused multiply-add, and the dequantised weight is the
+// single correctly-rounded fp16 product q * scale.
+__device__ __forceinline__ void dequant8(uint32_t w, __half2 s_lo, __half2 s_hi, uint32_t (&a)[4]) {
+  const uint32_t MAGIC = 0x64006400u;                       // (1024.0, 1024.0)
+  const __half2 k1032 = u32_as_h2(0x64086408u);             // 1032.0
+  const __half2 k16th = u32_as_h2(0x2C002C00u);             // 1/16
+  const __half2 km72 = u32_as_h2(0xD480D480u);              // -72.0
+  const uint32_t w8 = w >> 8;
+  const __half2 x0 = u32_as_h2((w & 0x000F000Fu) | MAGIC);
+  const __half2 x1 = u32_as_h2((w & 0x00F000F0u) | MAGIC);
+  const __half2 x2 = u32_as_h2((w8 & 0x000F000Fu) | MAGIC);
+  const __half2 x3 = u32_as_h2((w8 & 0x00F000F0u) | MAGIC);
+  a[0] = h2_as_u32(__hmul2(__hsub2(x0, k1032), s_lo));
+  a[1] = h2_as_u32(__hmul2(__hfma2(x1, k16th, km72), s_hi));
+  a[2] = h2_as_u32(__hmul2(__hsub2(x2, k1032), s_lo));
+  a[3] = h2_as_u32(__hmul2(__hfma2(x3, k16th, km72), s_hi));
+}
+__device__ __forceinline__ void split_scales(uint32_t sw, __half2& s_lo, __half2& s_hi) {
+  s_lo = u32_as_h2(__byte_perm(sw, sw, 0x1010));
+  s_hi = u32_as_h2(__byte_perm(sw, sw, 0x3232));
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+#endif
+
+}  // namespace mlora

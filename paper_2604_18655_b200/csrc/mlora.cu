@@ -1,0 +1,975 @@
+// Host side of the C ABI: context, weight repacking, the launch sequence of one decode / verify pass,
+// CUDA-graph replay of steps, per-family event timing.  Every step of the path runs in the kernels of
+// this library; there is no CPU or library fallback.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <unordered_map>
+#include <vector>
+
+#include "../../include/mlora.h"
+#include "common.cuh"
+
+using namespace mlora;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+struct PackedWeight {
+  uint4* wq = nullptr;
+  uint32_t* sc = nullptr;
+  int K = 0, N = 0, G = 0;   // N = physical width (all fused segments)
+};
+
+cudaError_t alloc_packed(PackedWeight& w, int K, int N, int G) {
+  w.K = K; w.N = N; w.G = G;
+  cudaError_t e = cudaMalloc(&w.wq, (size_t)K * N / 2);
+  if (e != cudaSuccess) return e;
+  return cudaMalloc(&w.sc, (size_t)(K / G) * N * sizeof(__half));
+}
+void free_packed(PackedWeight& w) {
+  if (w.wq) cudaFree(w.wq);
+  if (w.sc) cudaFree(w.sc);
+  w.wq = nullptr; w.sc = nullptr;
+}
+
+struct GraphKey {
+  int kind, n, T, prefix_chunk, n_prefix_chunks, own_chunk, n_own_chunks, flags;
+  const void* p[8];
+  bool operator==(const GraphKey& o) const { return std::memcmp(this, &o, sizeof(GraphKey)) == 0; }
+};
+struct GraphKeyHash {
+  size_t operator()(const GraphKey& k) const {
+    const unsigned char* b = reinterpret_cast<const unsigned char*>(&k);
+    size_t h = 1469598103934665603ull;
+    for (size_t i = 0; i < sizeof(GraphKey); ++i) { h ^= b[i]; h *= 1099511628211ull; }
+    return h;
+  }
+};
+struct GraphEntry { cudaGraphExec_t exec; int nodes; };
+
+}  // namespace
+
+struct mlora_weight {
+  PackedWeight w;
+  cudaStream_t stream;
+};
+
+struct mlora_ctx {
+  mlora_model_desc d;
+  cudaStream_t stream = nullptr;
+  int sm_count = 148;
+  int L = 0, Nq = 0, Nkv = 0, Nqkv = 0, cap = 0, Mmax = 0;
+  std::vector<PackedWeight> w_qkv, w_o, w_gateup, w_down;
+  PackedWeight w_lm;
+  std::vector<const __half*> rms_attn, rms_ffn;
+  // KV caches
+  __half *prefix_k = nullptr, *prefix_v = nullptr;   // [L][Hkv][max_prefix][hd]
+  __half *own_k = nullptr, *own_v = nullptr;         // [L][n][Hkv][cap][hd]
+  size_t prefix_layer_stride = 0, prefix_head_stride = 0;
+  size_t own_layer_stride = 0, own_stream_stride = 0, own_head_stride = 0;
+  // scratch
+  float *X = nullptr, *qkv = nullptr, *logits = nullptr, *T = nullptr, *partial = nullptr, *att_ws = nullptr;
+  __half *h = nullptr, *q16 = nullptr, *attn16 = nullptr, *act16 = nullptr;
+  size_t partial_floats = 0, att_ws_floats = 0;
+  unsigned* counters = nullptr;
+  unsigned long long* anc = nullptr;
+  int32_t *depth = nullptr, *argmax = nullptr, *suffix_len = nullptr, *zero_len = nullptr, *chain_parent = nullptr,
+          *root_parent = nullptr;
+  int* status = nullptr;
+  float2* cs_table = nullptr;
+  // adapters
+  const __half** tabA = nullptr;
+  const __half** tabB = nullptr;
+  float* ad_scale = nullptr;
+  const __half** stageA = nullptr;   // pinned host staging [max_adapters][L*7]
+  const __half** stageB = nullptr;
+  float* stage_scale = nullptr;
+  // host state
+  int P = 0;
+  bool prefilled = false;
+  int suffix_bound = 0;
+  int32_t* snap = nullptr;           // pinned copy of suffix_len
+  cudaEvent_t snap_event = nullptr;
+  bool snap_pending = false;
+  int snap_inc = 0;
+  int dbg_skip_compact = 0, dbg_no_graph = 0;
+  // graphs
+  std::unordered_map<GraphKey, GraphEntry, GraphKeyHash> graphs;
+  bool capturing = false;
+  // profiling
+  bool profiling = false;
+  struct Ev { cudaEvent_t a, b; int fam; };
+  std::vector<Ev> evs;
+  std::vector<cudaEvent_t> ev_pool;
+  int64_t launches = 0;
+  int captured_nodes = 0;
+};
+
+namespace {
+
+int fail(int code, const std::string& msg) {
+  g_last_error = msg;
+  return code;
+}
+#define CK(call)                                                                                   \
+  do {                                                                                             \
+    cudaError_t e__ = (call);                                                                      \
+    if (e__ != cudaSuccess)                                                                        \
+      return fail(MLORA_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e__));            \
+  } while (0)
+
+// wraps one kernel launch: counts it and, when profiling, brackets it with an event pair
+template <class F>
+cudaError_t run(mlora_ctx* c, int fam, F&& f) {
+  if (c->capturing) c->captured_nodes++;
+  else c->launches++;
+  if (!c->profiling) return f();
+  mlora_ctx::Ev ev;
+  for (cudaEvent_t* e : {&ev.a, &ev.b}) {
+    if (!c->ev_pool.empty()) { *e = c->ev_pool.back(); c->ev_pool.pop_back(); }
+    else { cudaError_t r = cudaEventCreate(e); if (r != cudaSuccess) return r; }
+  }
+  ev.fam = fam;
+  cudaEventRecord(ev.a, c->stream);
+  cudaError_t r = f();
+  cudaEventRecord(ev.b, c->stream);
+  c->evs.push_back(ev);
+  return r;
+}
+
+struct PassIO {
+  int n = 0, T = 1;
+  const int32_t* tokens = nullptr;
+  const __half* hidden_in = nullptr;
+  const int32_t* adapter_idx = nullptr;   // nullptr: base weights for every row
+  const int32_t* parent = nullptr;        // dev [n][T]
+  bool prefill = false;
+  int pos_base = 0;                        // length of the shared segment the rows attend to
+  const int32_t* suffix_len = nullptr;
+  int suffix_bound = 0;
+  float* logits = nullptr;                 // [M][vocab] destination, nullptr: skip lm_head
+  AttnArgs plan;                           // chunking, filled by plan_pass
+};
+
+LoraArgs lora_args(mlora_ctx* c, const PassIO& io, int l, int nseg, const int* projs, const int* widths) {
+  LoraArgs la{};
+  int mask = 0;
+  for (int i = 0; i < nseg; ++i) mask |= (1 << projs[i]);
+  if (io.adapter_idx == nullptr || !(c->d.lora_targets & mask) || c->d.lora_rank <= 0) return la;
+  la.adapter_idx = io.adapter_idx;
+  la.rows_per_stream = io.T;
+  la.tabA = c->tabA;
+  la.tabB = c->tabB;
+  la.scale = c->ad_scale;
+  la.tab_stride = c->L * 7;
+  la.n_slots = c->d.max_adapters;
+  la.rank = c->d.lora_rank;
+  la.nseg = nseg;
+  for (int i = 0; i < nseg; ++i) { la.seg[i].proj_index = l * 7 + projs[i]; la.seg[i].n = widths[i]; }
+  la.T = c->T;
+  return la;
+}
+
+void plan_pass(mlora_ctx* c, PassIO& io) {
+  AttnArgs& a = io.plan;
+  a = AttnArgs{};
+  a.P = io.pos_base;
+  a.n = io.n; a.T = io.T; a.Hq = c->d.n_q_heads; a.Hkv = c->d.n_kv_heads; a.hd = c->d.head_dim;
+  a.suffix_bound = (io.suffix_bound + 63) / 64 * 64;   // coarse, so the launch shape changes rarely
+  attn_plan(a, c->sm_count);
+}
+
+// the launch sequence of one pass over M = n*T rows (Sec. 3.1 decoder, Eq. 1-4 projections)
+int forward(mlora_ctx* c, const PassIO& io) {
+  const mlora_model_desc& d = c->d;
+  cudaStream_t st = c->stream;
+  const int M = io.n * io.T;
+  const int dm = d.d_model, F = d.d_ffn, hd = d.head_dim;
+  CK(run(c, MLORA_PROF_MISC, [&] { return launch_embed(io.tokens, (const __half*)d.embed, io.hidden_in, c->X, M, dm, d.vocab, c->status, st); }));
+  CK(run(c, MLORA_PROF_MISC, [&] { return launch_tree_prep(io.parent, io.n, io.T, c->anc, c->depth, c->status, st); }));
+  for (int l = 0; l < c->L; ++l) {
+    // attention block
+    {
+      const int projs[3] = {0, 1, 2}, widths[3] = {c->Nq, c->Nkv, c->Nkv};
+      ShrinkArgs s{};
+      s.x_f32 = c->X; s.gain = c->rms_attn[l]; s.eps = d.rms_eps; s.h_out = c->h; s.M = M; s.K = dm;
+      s.lora = lora_args(c, io, l, 3, projs, widths);
+      CK(run(c, MLORA_PROF_SHRINK, [&] { return launch_shrink(s, st); }));
+      GemmArgs g{};
+      const PackedWeight& w = c->w_qkv[l];
+      g.wq = w.wq; g.sc = w.sc; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->h; g.M = M;
+      g.mode = MODE_QKV; g.epi = EPI_F32; g.seg_n0 = c->Nq; g.seg_n1 = c->Nkv;
+      g.out_f32 = c->qkv; g.ldo = c->Nqkv;
+      g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
+      g.lora = s.lora;
+      CK(run(c, MLORA_PROF_GEMM, [&] { return launch_gemm(g, st); }));
+    }
+    __half *kd, *vd;
+    size_t sstride, hstride;
+    if (io.prefill) {
+      kd = c->prefix_k + (size_t)l * c->prefix_layer_stride + (size_t)io.pos_base * hd;
+      vd = c->prefix_v + (size_t)l * c->prefix_layer_stride + (size_t)io.pos_base * hd;
+      sstride = 0; hstride = c->prefix_head_stride;
+    } else {
+      kd = c->own_k + (size_t)l * c->own_layer_stride;
+      vd = c->own_v + (size_t)l * c->own_layer_stride;
+      sstride = c->own_stream_stride; hstride = c->own_head_stride;
+    }
+    CK(run(c, MLORA_PROF_ROPE_KV, [&] {
+      return launch_rope_kv(c->qkv, M, io.T, d.n_q_heads, d.n_kv_heads, hd, c->cs_table, io.pos_base, io.suffix_len,
+                            c->depth, c->q16, kd, vd, sstride, hstride, st);
+    }));
+    {
+      AttnArgs a = io.plan;
+      a.q = c->q16;
+      a.prefix_k = c->prefix_k + (size_t)l * c->prefix_layer_stride;
+      a.prefix_v = c->prefix_v + (size_t)l * c->prefix_layer_stride;
+      a.prefix_head_stride = c->prefix_head_stride;
+      a.own_k = kd; a.own_v = vd; a.own_stream_stride = sstride; a.own_head_stride = hstride;
+      a.suffix_len = io.suffix_len; a.anc = c->anc;
+      a.out = c->attn16;
+      if (attn_workspace_floats(a) > c->att_ws_floats) return fail(MLORA_ERR_CAPACITY, "attention scratch too small");
+      a.part_o = c->att_ws;
+      a.part_ml = c->att_ws + (attn_workspace_floats(a) / (a.hd + 2)) * a.hd;
+      CK(run(c, MLORA_PROF_ATTN, [&] { return launch_attention(a, st); }));
+      CK(run(c, MLORA_PROF_ATTN_MERGE, [&] { return launch_attention_merge(a, st); }));
+    }
+    {
+      const int projs[1] = {3}, widths[1] = {dm};
+      LoraArgs la = lora_args(c, io, l, 1, projs, widths);
+      if (la.adapter_idx) {
+        ShrinkArgs s{};
+        s.h_in = c->attn16; s.M = M; s.K = c->Nq; s.lora = la;
+        CK(run(c, MLORA_PROF_SHRINK, [&] { return launch_shrink(s, st); }));
+      }
+      GemmArgs g{};
+      const PackedWeight& w = c->w_o[l];
+      g.wq = w.wq; g.sc = w.sc; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->attn16; g.M = M;
+      g.mode = MODE_PLAIN; g.epi = EPI_RESID; g.resid = c->X;
+      g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
+      g.lora = la;
+      CK(run(c, MLORA_PROF_GEMM, [&] { return launch_gemm(g, st); }));
+    }
+    // MLP block
+    {
+      const int projs[2] = {4, 5}, widths[2] = {F, F};
+      ShrinkArgs s{};
+      s.x_f32 = c->X; s.gain = c->rms_ffn[l]; s.eps = d.rms_eps; s.h_out = c->h; s.M = M; s.K = dm;
+      s.lora = lora_args(c, io, l, 2, projs, widths);
+      CK(run(c, MLORA_PROF_SHRINK, [&] { return launch_shrink(s, st); }));
+      GemmArgs g{};
+      const PackedWeight& w = c->w_gateup[l];
+      g.wq = w.wq; g.sc = w.sc; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->h; g.M = M;
+      g.mode = MODE_GATEUP; g.epi = EPI_SWIGLU; g.out_f16 = c->act16;
+      g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
+      g.lora = s.lora;
+      CK(run(c, MLORA_PROF_GEMM, [&] { return launch_gemm(g, st); }));
+    }
+    {
+      const int projs[1] = {6}, widths[1] = {dm};
+      LoraArgs la = lora_args(c, io, l, 1, projs, widths);
+      if (la.adapter_idx) {
+        ShrinkArgs s{};
+        s.h_in = c->act16; s.M = M; s.K = F; s.lora = la;
+        CK(run(c, MLORA_PROF_SHRINK, [&] { return launch_shrink(s, st); }));
+      }
+      GemmArgs g{};
+      const PackedWeight& w = c->w_down[l];
+      g.wq = w.wq; g.sc = w.sc; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->act16; g.M = M;
+      g.mode = MODE_PLAIN; g.epi = EPI_RESID; g.resid = c->X;
+      g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
+      g.lora = la;
+      CK(run(c, MLORA_PROF_GEMM, [&] { return launch_gemm(g, st); }));
+    }
+  }
+  if (d.vocab > 0 && io.logits != nullptr) {
+    ShrinkArgs s{};
+    s.x_f32 = c->X; s.gain = (const __half*)d.rms_final; s.eps = d.rms_eps; s.h_out = c->h; s.M = M; s.K = dm;
+    CK(run(c, MLORA_PROF_SHRINK, [&] { return launch_shrink(s, st); }));
+    GemmArgs g{};
+    const PackedWeight& w = c->w_lm;
+    g.wq = w.wq; g.sc = w.sc; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->h; g.M = M;
+    g.mode = MODE_PLAIN; g.epi = EPI_F32; g.out_f32 = io.logits; g.ldo = d.vocab;
+    g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
+    CK(run(c, MLORA_PROF_GEMM, [&] { return launch_gemm(g, st); }));
+  }
+  return MLORA_OK;
+}
+
+// runs `body` directly, or captures it once into a CUDA graph and replays it
+template <class F>
+int replay_or_run(mlora_ctx* c, const GraphKey& key, F&& body) {
+  if (c->dbg_no_graph || c->profiling) return body();
+  auto it = c->graphs.find(key);
+  if (it == c->graphs.end()) {
+    cudaGraph_t graph = nullptr;
+    c->capturing = true;
+    c->captured_nodes = 0;
+    cudaError_t e = cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal);
+    if (e != cudaSuccess) { c->capturing = false; return fail(MLORA_ERR_CUDA, std::string("begin capture: ") + cudaGetErrorString(e)); }
+    int rc = body();
+    e = cudaStreamEndCapture(c->stream, &graph);
+    c->capturing = false;
+    if (rc != MLORA_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+    if (e != cudaSuccess) return fail(MLORA_ERR_CUDA, std::string("end capture: ") + cudaGetErrorString(e));
+    GraphEntry ent{};
+    e = cudaGraphInstantiate(&ent.exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) return fail(MLORA_ERR_CUDA, std::string("graph instantiate: ") + cudaGetErrorString(e));
+    ent.nodes = c->captured_nodes;
+    if (c->graphs.size() > 256) {                      // bound the cache
+      for (auto& kv : c->graphs) cudaGraphExecDestroy(kv.second.exec);
+      c->graphs.clear();
+    }
+    it = c->graphs.emplace(key, ent).first;
+  }
+  CK(cudaGraphLaunch(it->second.exec, c->stream));
+  c->launches += it->second.nodes;
+  return MLORA_OK;
+}
+
+// refreshes the host's upper bound on the suffix lengths from the last finished snapshot
+void poll_snapshot(mlora_ctx* c) {
+  if (c->snap_pending && cudaEventQuery(c->snap_event) == cudaSuccess) {
+    int mx = 0;
+    for (int s = 0; s < c->d.max_streams; ++s) mx = c->snap[s] > mx ? c->snap[s] : mx;
+    c->suffix_bound = mx + c->snap_inc;
+    c->snap_pending = false;
+  }
+}
+int ensure_capacity(mlora_ctx* c, int T) {
+  poll_snapshot(c);
+  if (c->suffix_bound + T <= c->cap) return MLORA_OK;
+  // the bound is pessimistic after verify rounds: read the true lengths once
+  CK(cudaStreamSynchronize(c->stream));
+  CK(cudaMemcpy(c->snap, c->suffix_len, sizeof(int32_t) * c->d.max_streams, cudaMemcpyDeviceToHost));
+  int mx = 0;
+  for (int s = 0; s < c->d.max_streams; ++s) mx = c->snap[s] > mx ? c->snap[s] : mx;
+  c->suffix_bound = mx;
+  c->snap_pending = false;
+  if (mx + T > c->cap) return fail(MLORA_ERR_CAPACITY, "own KV segment full");
+  return MLORA_OK;
+}
+
+int init_kernels() {
+  static bool done = false;
+  if (done) return MLORA_OK;
+  CK(init_gemm());
+  CK(init_shrink());
+  CK(init_attention());
+  done = true;
+  return MLORA_OK;
+}
+
+int check_ctx(mlora_ctx* c) { return c ? MLORA_OK : fail(MLORA_ERR_ARG, "null context"); }
+
+int prefill_impl(mlora_ctx* c, const int32_t* ids, const __half* hidden, int n, float* out_last) {
+  if (n <= 0) return fail(MLORA_ERR_ARG, "prefill needs at least one position");
+  if (n > c->d.max_prefix) return fail(MLORA_ERR_CAPACITY, "prompt longer than max_prefix");
+  const int chunk = 64;
+  const int dm = c->d.d_model;
+  for (int p0 = 0; p0 < n; p0 += chunk) {
+    PassIO io;
+    io.n = 1;
+    io.T = (n - p0 < chunk) ? (n - p0) : chunk;
+    io.tokens = ids ? ids + p0 : nullptr;
+    io.hidden_in = hidden ? hidden + (size_t)p0 * dm : nullptr;
+    io.parent = c->chain_parent;
+    io.prefill = true;
+    io.pos_base = p0;
+    io.suffix_len = c->zero_len;
+    io.suffix_bound = 0;
+    const bool last = (p0 + io.T >= n);
+    io.logits = (last && c->d.vocab > 0 && out_last) ? c->logits : nullptr;
+    plan_pass(c, io);
+    int rc = forward(c, io);
+    if (rc != MLORA_OK) return rc;
+    if (last && out_last) {
+      const float* src = c->d.vocab > 0 ? c->logits + (size_t)(io.T - 1) * c->d.vocab : c->X + (size_t)(io.T - 1) * dm;
+      const size_t cnt = c->d.vocab > 0 ? (size_t)c->d.vocab : (size_t)dm;
+      CK(run(c, MLORA_PROF_MISC, [&] { return launch_copy_rows_f32(src, out_last, cnt, c->stream); }));
+    }
+  }
+  CK(cudaMemsetAsync(c->suffix_len, 0, sizeof(int32_t) * c->d.max_streams, c->stream));
+  c->P = n;
+  c->prefilled = true;
+  c->suffix_bound = 0;
+  c->snap_pending = false;
+  return MLORA_OK;
+}
+
+int step_common_checks(mlora_ctx* c, int n_streams, const void* adapter_idx, int T) {
+  if (!c->prefilled) return fail(MLORA_ERR_STATE, "no shared prefill yet");
+  if (n_streams <= 0 || n_streams > c->d.max_streams) return fail(MLORA_ERR_ARG, "n_streams out of range");
+  if (adapter_idx == nullptr) return fail(MLORA_ERR_ARG, "adapter_idx is null");
+  if (T < 1 || T > c->d.max_tree) return fail(MLORA_ERR_CAPACITY, "tree larger than max_tree");
+  return ensure_capacity(c, T);
+}
+
+}  // namespace
+
+// ============================================================================= C ABI
+extern "C" {
+
+const char* mlora_last_error(mlora_ctx*) { return g_last_error.c_str(); }
+
+int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
+  if (!desc || !out) return fail(MLORA_ERR_ARG, "null argument");
+  const mlora_model_desc& d = *desc;
+  if (d.n_layers <= 0 || d.d_model <= 0 || d.n_q_heads <= 0 || d.n_kv_heads <= 0 || d.d_ffn <= 0 || d.vocab < 0)
+    return fail(MLORA_ERR_ARG, "non-positive model dimension");
+  if (!d.qweight || !d.scales || !d.rms_attn || !d.rms_ffn) return fail(MLORA_ERR_ARG, "null weight table");
+  if (d.vocab > 0 && (!d.embed || !d.rms_final)) return fail(MLORA_ERR_ARG, "vocab > 0 needs embed and rms_final");
+  if (d.head_dim != 64 && d.head_dim != 128) return fail(MLORA_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+  if (d.n_q_heads % d.n_kv_heads) return fail(MLORA_ERR_ARG, "n_q_heads must be a multiple of n_kv_heads");
+  if (d.group_size <= 0 || d.group_size % 64) return fail(MLORA_ERR_UNSUPPORTED, "group_size must be a multiple of 64");
+  const int Nq = d.n_q_heads * d.head_dim, Nkv = d.n_kv_heads * d.head_dim;
+  for (int K : {d.d_model, Nq, d.d_ffn})
+    if (K % 64 || K % d.group_size) return fail(MLORA_ERR_UNSUPPORTED, "every input width must be a multiple of 64 and of group_size");
+  for (int N : {d.d_model, Nq, Nkv, d.d_ffn, d.vocab})
+    if (N % 16) return fail(MLORA_ERR_UNSUPPORTED, "every output width must be a multiple of 16");
+  if (d.max_tree < 1 || d.max_tree > 64) return fail(MLORA_ERR_ARG, "max_tree must be in 1..64");
+  if (d.max_streams < 1 || d.max_prefix < 1 || d.max_suffix < 1 || d.max_adapters < 0 || d.lora_rank < 0)
+    return fail(MLORA_ERR_ARG, "bad capacity");
+
+  if (init_kernels() != MLORA_OK) return MLORA_ERR_CUDA;
+  mlora_ctx* c = new mlora_ctx();
+  c->d = d;
+  c->stream = (cudaStream_t)d.cuda_stream;
+  c->L = d.n_layers; c->Nq = Nq; c->Nkv = Nkv; c->Nqkv = Nq + 2 * Nkv;
+  c->cap = d.max_suffix + d.max_tree;
+  c->Mmax = d.max_streams * d.max_tree;
+  if (c->Mmax < 64) c->Mmax = 64;
+#define CKC(call)                                                                                  \
+  do {                                                                                             \
+    cudaError_t e__ = (call);                                                                      \
+    if (e__ != cudaSuccess) {                                                                      \
+      fail(MLORA_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e__));                   \
+      mlora_destroy(c);                                                                            \
+      return MLORA_ERR_CUDA;                                                                       \
+    }                                                                                              \
+  } while (0)
+  int dev = 0;
+  CKC(cudaGetDevice(&dev));
+  CKC(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev));
+  cudaStream_t st = c->stream;
+  const int L = c->L, dm = d.d_model, F = d.d_ffn, G = d.group_size, hd = d.head_dim;
+  // ---- weights: repack into fused fragment-major matrices
+  c->w_qkv.resize(L); c->w_o.resize(L); c->w_gateup.resize(L); c->w_down.resize(L);
+  c->rms_attn.resize(L); c->rms_ffn.resize(L);
+  for (int l = 0; l < L; ++l) {
+    const void* const* qw = d.qweight + (size_t)l * 7;
+    const void* const* sc = d.scales + (size_t)l * 7;
+    for (int p = 0; p < 7; ++p)
+      if (!qw[p] || !sc[p]) { fail(MLORA_ERR_ARG, "null weight pointer"); mlora_destroy(c); return MLORA_ERR_ARG; }
+    if (!d.rms_attn[l] || !d.rms_ffn[l]) { fail(MLORA_ERR_ARG, "null norm gain"); mlora_destroy(c); return MLORA_ERR_ARG; }
+    c->rms_attn[l] = (const __half*)d.rms_attn[l];
+    c->rms_ffn[l] = (const __half*)d.rms_ffn[l];
+    PackedWeight& wqkv = c->w_qkv[l];
+    CKC(alloc_packed(wqkv, dm, c->Nqkv, G));
+    const int tp = c->Nqkv / 16;
+    CKC(launch_repack((const uint8_t*)qw[0], (const __half*)sc[0], dm, Nq, G, wqkv.wq, wqkv.sc, 0, 1, tp, st));
+    CKC(launch_repack((const uint8_t*)qw[1], (const __half*)sc[1], dm, Nkv, G, wqkv.wq, wqkv.sc, Nq / 16, 1, tp, st));
+    CKC(launch_repack((const uint8_t*)qw[2], (const __half*)sc[2], dm, Nkv, G, wqkv.wq, wqkv.sc, (Nq + Nkv) / 16, 1, tp, st));
+    CKC(alloc_packed(c->w_o[l], Nq, dm, G));
+    CKC(launch_repack((const uint8_t*)qw[3], (const __half*)sc[3], Nq, dm, G, c->w_o[l].wq, c->w_o[l].sc, 0, 1, dm / 16, st));
+    PackedWeight& wgu = c->w_gateup[l];
+    CKC(alloc_packed(wgu, dm, 2 * F, G));
+    CKC(launch_repack((const uint8_t*)qw[4], (const __half*)sc[4], dm, F, G, wgu.wq, wgu.sc, 0, 2, 2 * F / 16, st));
+    CKC(launch_repack((const uint8_t*)qw[5], (const __half*)sc[5], dm, F, G, wgu.wq, wgu.sc, 1, 2, 2 * F / 16, st));
+    CKC(alloc_packed(c->w_down[l], F, dm, G));
+    CKC(launch_repack((const uint8_t*)qw[6], (const __half*)sc[6], F, dm, G, c->w_down[l].wq, c->w_down[l].sc, 0, 1, dm / 16, st));
+  }
+  if (d.vocab > 0) {
+    const void* qw = d.qweight[(size_t)L * 7];
+    const void* sc = d.scales[(size_t)L * 7];
+    if (!qw || !sc) { fail(MLORA_ERR_ARG, "null lm_head pointer"); mlora_destroy(c); return MLORA_ERR_ARG; }
+    CKC(alloc_packed(c->w_lm, dm, d.vocab, G));
+    CKC(launch_repack((const uint8_t*)qw, (const __half*)sc, dm, d.vocab, G, c->w_lm.wq, c->w_lm.sc, 0, 1, d.vocab / 16, st));
+  }
+  // ---- KV caches
+  c->prefix_head_stride = (size_t)d.max_prefix * hd;
+  c->prefix_layer_stride = c->prefix_head_stride * d.n_kv_heads;
+  c->own_head_stride = (size_t)c->cap * hd;
+  c->own_stream_stride = c->own_head_stride * d.n_kv_heads;
+  c->own_layer_stride = c->own_stream_stride * d.max_streams;
+  CKC(cudaMalloc(&c->prefix_k, c->prefix_layer_stride * L * sizeof(__half)));
+  CKC(cudaMalloc(&c->prefix_v, c->prefix_layer_stride * L * sizeof(__half)));
+  CKC(cudaMalloc(&c->own_k, c->own_layer_stride * L * sizeof(__half)));
+  CKC(cudaMalloc(&c->own_v, c->own_layer_stride * L * sizeof(__half)));
+  // ---- scratch
+  const size_t Mm = c->Mmax;
+  size_t maxK = dm; if ((size_t)F > maxK) maxK = F; if ((size_t)Nq > maxK) maxK = Nq;
+  CKC(cudaMalloc(&c->X, Mm * dm * sizeof(float)));
+  CKC(cudaMalloc(&c->qkv, Mm * c->Nqkv * sizeof(float)));
+  CKC(cudaMalloc(&c->h, Mm * maxK * sizeof(__half)));
+  CKC(cudaMalloc(&c->q16, Mm * Nq * sizeof(__half)));
+  CKC(cudaMalloc(&c->attn16, Mm * Nq * sizeof(__half)));
+  CKC(cudaMalloc(&c->act16, Mm * F * sizeof(__half)));
+  if (d.vocab > 0) CKC(cudaMalloc(&c->logits, Mm * d.vocab * sizeof(float)));
+  CKC(cudaMalloc(&c->T, Mm * 3 * (d.lora_rank > 0 ? d.lora_rank : 1) * sizeof(float)));
+  c->partial_floats = (size_t)16 << 20;               // 64 MB of split-K scratch
+  CKC(cudaMalloc(&c->partial, c->partial_floats * sizeof(float)));
+  CKC(cudaMalloc(&c->counters, 4096 * sizeof(unsigned)));
+  CKC(cudaMemsetAsync(c->counters, 0, 4096 * sizeof(unsigned), st));
+  {
+    // attention scratch: rows x chunks never exceeds (rows of one launch) + 64 x (CTAs the planner aims for),
+    // once for the shared-prefix chunks and once for the own-segment chunks
+    const size_t g_heads = d.n_q_heads / d.n_kv_heads;
+    const size_t R_all = Mm * g_heads;
+    c->att_ws_floats = ((size_t)d.n_kv_heads * R_all * 2 + (size_t)256 * c->sm_count + 4096) * (hd + 2);
+    CKC(cudaMalloc(&c->att_ws, c->att_ws_floats * sizeof(float)));
+  }
+  CKC(cudaMalloc(&c->anc, Mm * sizeof(unsigned long long)));
+  CKC(cudaMalloc(&c->depth, Mm * sizeof(int32_t)));
+  CKC(cudaMalloc(&c->argmax, Mm * sizeof(int32_t)));
+  CKC(cudaMalloc(&c->suffix_len, d.max_streams * sizeof(int32_t)));
+  CKC(cudaMalloc(&c->zero_len, d.max_streams * sizeof(int32_t)));
+  CKC(cudaMemsetAsync(c->suffix_len, 0, d.max_streams * sizeof(int32_t), st));
+  CKC(cudaMemsetAsync(c->zero_len, 0, d.max_streams * sizeof(int32_t), st));
+  CKC(cudaMalloc(&c->status, sizeof(int)));
+  CKC(cudaMemsetAsync(c->status, 0, sizeof(int), st));
+  {
+    std::vector<int32_t> chain(64), root(d.max_streams, -1);
+    for (int i = 0; i < 64; ++i) chain[i] = i - 1;
+    CKC(cudaMalloc(&c->chain_parent, 64 * sizeof(int32_t)));
+    CKC(cudaMalloc(&c->root_parent, d.max_streams * sizeof(int32_t)));
+    CKC(cudaMemcpyAsync(c->chain_parent, chain.data(), 64 * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    CKC(cudaMemcpyAsync(c->root_parent, root.data(), d.max_streams * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    CKC(cudaStreamSynchronize(st));
+  }
+  {
+    // cos/sin of pos * theta^(-2i/hd), evaluated in double
+    const int maxpos = d.max_prefix + c->cap + 1;
+    const int half = hd / 2;
+    std::vector<float2> tab((size_t)maxpos * half);
+    for (int i = 0; i < half; ++i) {
+      const double inv = std::pow((double)d.rope_theta, -2.0 * i / hd);
+      for (int p = 0; p < maxpos; ++p) {
+        const double ang = (double)p * inv;
+        tab[(size_t)p * half + i] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+      }
+    }
+    CKC(cudaMalloc(&c->cs_table, tab.size() * sizeof(float2)));
+    CKC(cudaMemcpyAsync(c->cs_table, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice, st));
+    CKC(cudaStreamSynchronize(st));
+  }
+  // ---- adapter tables
+  if (d.max_adapters > 0) {
+    const size_t ents = (size_t)d.max_adapters * L * 7;
+    CKC(cudaMalloc(&c->tabA, ents * sizeof(void*)));
+    CKC(cudaMalloc(&c->tabB, ents * sizeof(void*)));
+    CKC(cudaMalloc(&c->ad_scale, d.max_adapters * sizeof(float)));
+    CKC(cudaMemsetAsync(c->tabA, 0, ents * sizeof(void*), st));
+    CKC(cudaMemsetAsync(c->tabB, 0, ents * sizeof(void*), st));
+    CKC(cudaMemsetAsync(c->ad_scale, 0, d.max_adapters * sizeof(float), st));
+    CKC(cudaMallocHost(&c->stageA, ents * sizeof(void*)));
+    CKC(cudaMallocHost(&c->stageB, ents * sizeof(void*)));
+    CKC(cudaMallocHost(&c->stage_scale, d.max_adapters * sizeof(float)));
+  }
+  CKC(cudaMallocHost(&c->snap, d.max_streams * sizeof(int32_t)));
+  CKC(cudaEventCreateWithFlags(&c->snap_event, cudaEventDisableTiming));
+  CKC(cudaStreamSynchronize(st));
+#undef CKC
+  *out = c;
+  return MLORA_OK;
+}
+
+int mlora_destroy(mlora_ctx* c) {
+  if (!c) return MLORA_OK;
+  cudaStreamSynchronize(c->stream);
+  for (auto& kv : c->graphs) cudaGraphExecDestroy(kv.second.exec);
+  for (auto& w : c->w_qkv) free_packed(w);
+  for (auto& w : c->w_o) free_packed(w);
+  for (auto& w : c->w_gateup) free_packed(w);
+  for (auto& w : c->w_down) free_packed(w);
+  free_packed(c->w_lm);
+  void* dev_ptrs[] = {c->prefix_k, c->prefix_v, c->own_k, c->own_v, c->X, c->qkv, c->logits, c->T, c->partial, c->att_ws,
+                      c->h, c->q16, c->attn16, c->act16, c->counters, c->anc, c->depth, c->argmax, c->suffix_len,
+                      c->zero_len, c->chain_parent, c->root_parent, c->status, c->cs_table, (void*)c->tabA,
+                      (void*)c->tabB, c->ad_scale};
+  for (void* p : dev_ptrs) if (p) cudaFree(p);
+  if (c->stageA) cudaFreeHost((void*)c->stageA);
+  if (c->stageB) cudaFreeHost((void*)c->stageB);
+  if (c->stage_scale) cudaFreeHost(c->stage_scale);
+  if (c->snap) cudaFreeHost(c->snap);
+  if (c->snap_event) cudaEventDestroy(c->snap_event);
+  for (auto& e : c->evs) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+  for (auto& e : c->ev_pool) cudaEventDestroy(e);
+  delete c;
+  return MLORA_OK;
+}
+
+int mlora_set_adapter(mlora_ctx* c, int32_t slot, const void* const* A, const void* const* B, float alpha) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (slot < 0 || slot >= c->d.max_adapters) return fail(MLORA_ERR_ARG, "adapter slot out of range");
+  if ((A == nullptr) != (B == nullptr)) return fail(MLORA_ERR_ARG, "A and B must both be given or both be NULL");
+  if (c->d.lora_rank <= 0) return fail(MLORA_ERR_STATE, "context was created with lora_rank 0");
+  const size_t per = (size_t)c->L * 7;
+  // the staging row of this slot may still be in flight from an earlier call on the same slot
+  CK(cudaStreamSynchronize(c->stream));
+  for (size_t i = 0; A != nullptr && i < per; ++i)
+    if ((c->d.lora_targets & (1 << (int)(i % 7))) && (A[i] == nullptr || B[i] == nullptr))
+      return fail(MLORA_ERR_ARG, "null adapter tensor for a targeted projection");
+  for (size_t i = 0; i < per; ++i) {
+    const int p = (int)(i % 7);
+    const bool on = A != nullptr && (c->d.lora_targets & (1 << p));
+    c->stageA[slot * per + i] = on ? (const __half*)A[i] : nullptr;
+    c->stageB[slot * per + i] = on ? (const __half*)B[i] : nullptr;
+  }
+  c->stage_scale[slot] = A ? alpha / (float)c->d.lora_rank : 0.f;
+  CK(cudaMemcpyAsync(c->tabA + slot * per, c->stageA + slot * per, per * sizeof(void*), cudaMemcpyHostToDevice, c->stream));
+  CK(cudaMemcpyAsync(c->tabB + slot * per, c->stageB + slot * per, per * sizeof(void*), cudaMemcpyHostToDevice, c->stream));
+  CK(cudaMemcpyAsync(c->ad_scale + slot, c->stage_scale + slot, sizeof(float), cudaMemcpyHostToDevice, c->stream));
+  return MLORA_OK;
+}
+
+int mlora_prefill_shared(mlora_ctx* c, const int32_t* prompt_ids, int32_t n, float* out_last_logits) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (c->d.vocab == 0) return fail(MLORA_ERR_STATE, "context has no vocabulary: use mlora_prefill_shared_h");
+  if (!prompt_ids) return fail(MLORA_ERR_ARG, "prompt_ids is null");
+  return prefill_impl(c, prompt_ids, nullptr, n, out_last_logits);
+}
+
+int mlora_prefill_shared_h(mlora_ctx* c, const void* hidden, int32_t n, float* out_last_hidden) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (!hidden) return fail(MLORA_ERR_ARG, "hidden is null");
+  return prefill_impl(c, nullptr, (const __half*)hidden, n, out_last_hidden);
+}
+
+static int decode_impl(mlora_ctx* c, int n, const int32_t* adapter_idx, const int32_t* tokens, const __half* hidden,
+                       int32_t* out_next, float* out_logits, float* hidden_out) {
+  int rc = step_common_checks(c, n, adapter_idx, 1);
+  if (rc != MLORA_OK) return rc;
+  PassIO io;
+  io.n = n; io.T = 1; io.tokens = tokens; io.hidden_in = hidden; io.adapter_idx = adapter_idx;
+  io.parent = c->root_parent; io.pos_base = c->P; io.suffix_len = c->suffix_len; io.suffix_bound = c->suffix_bound;
+  io.logits = c->d.vocab > 0 ? (out_logits ? out_logits : c->logits) : nullptr;
+  plan_pass(c, io);
+  GraphKey key{};
+  key.kind = hidden ? 2 : 1; key.n = n; key.T = 1;
+  key.prefix_chunk = io.plan.prefix_chunk; key.n_prefix_chunks = io.plan.n_prefix_chunks;
+  key.own_chunk = io.plan.own_chunk; key.n_own_chunks = io.plan.n_own_chunks;
+  key.flags = c->P;
+  key.p[0] = adapter_idx; key.p[1] = tokens; key.p[2] = hidden; key.p[3] = out_next; key.p[4] = out_logits; key.p[5] = hidden_out;
+  rc = replay_or_run(c, key, [&]() -> int {
+    int r = forward(c, io);
+    if (r != MLORA_OK) return r;
+    if (c->d.vocab > 0) {
+      CK(run(c, MLORA_PROF_MISC, [&] { return launch_argmax(io.logits, n, c->d.vocab, out_next, c->stream); }));
+    } else {
+      CK(run(c, MLORA_PROF_MISC, [&] { return launch_copy_rows_f32(c->X, hidden_out, (size_t)n * c->d.d_model, c->stream); }));
+    }
+    CK(run(c, MLORA_PROF_MISC, [&] { return launch_advance(c->suffix_len, nullptr, n, 1, c->stream); }));
+    return MLORA_OK;
+  });
+  if (rc != MLORA_OK) return rc;
+  c->suffix_bound += 1;
+  if (c->snap_pending) c->snap_inc += 1;
+  return MLORA_OK;
+}
+
+int mlora_decode_step(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_idx, const int32_t* tokens,
+                      int32_t* out_next, float* out_logits) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (c->d.vocab == 0) return fail(MLORA_ERR_STATE, "context has no vocabulary: use mlora_decode_step_h");
+  if (!tokens || !out_next) return fail(MLORA_ERR_ARG, "tokens/out_next is null");
+  return decode_impl(c, n_streams, adapter_idx, tokens, nullptr, out_next, out_logits, nullptr);
+}
+
+int mlora_decode_step_h(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_idx, const void* hidden_in,
+                        float* hidden_out) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (!hidden_in || !hidden_out) return fail(MLORA_ERR_ARG, "hidden_in/hidden_out is null");
+  if (c->d.vocab != 0) return fail(MLORA_ERR_STATE, "context has a vocabulary: use mlora_decode_step");
+  return decode_impl(c, n_streams, adapter_idx, nullptr, (const __half*)hidden_in, nullptr, nullptr, hidden_out);
+}
+
+int mlora_verify_tree(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_idx, int32_t n_nodes,
+                      const int32_t* tree_tokens, const int32_t* tree_parent, int32_t* out_accept_len,
+                      int32_t* out_accept_idx, int32_t* out_next, float* out_logits) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (c->d.vocab == 0) return fail(MLORA_ERR_STATE, "verification needs logits: context has no vocabulary");
+  if (!tree_tokens || !tree_parent || !out_accept_len || !out_accept_idx || !out_next)
+    return fail(MLORA_ERR_ARG, "null argument");
+  int rc = step_common_checks(c, n_streams, adapter_idx, n_nodes);
+  if (rc != MLORA_OK) return rc;
+  const int n = n_streams, T = n_nodes;
+  PassIO io;
+  io.n = n; io.T = T; io.tokens = tree_tokens; io.adapter_idx = adapter_idx; io.parent = tree_parent;
+  io.pos_base = c->P; io.suffix_len = c->suffix_len; io.suffix_bound = c->suffix_bound;
+  io.logits = out_logits ? out_logits : c->logits;
+  plan_pass(c, io);
+  GraphKey key{};
+  key.kind = 3; key.n = n; key.T = T;
+  key.prefix_chunk = io.plan.prefix_chunk; key.n_prefix_chunks = io.plan.n_prefix_chunks;
+  key.own_chunk = io.plan.own_chunk; key.n_own_chunks = io.plan.n_own_chunks;
+  key.flags = c->P * 2 + c->dbg_skip_compact;
+  key.p[0] = adapter_idx; key.p[1] = tree_tokens; key.p[2] = tree_parent; key.p[3] = out_accept_len;
+  key.p[4] = out_accept_idx; key.p[5] = out_next; key.p[6] = out_logits;
+  rc = replay_or_run(c, key, [&]() -> int {
+    int r = forward(c, io);
+    if (r != MLORA_OK) return r;
+    cudaStream_t st = c->stream;
+    CK(run(c, MLORA_PROF_MISC, [&] { return launch_argmax(io.logits, n * T, c->d.vocab, c->argmax, st); }));
+    CK(run(c, MLORA_PROF_MISC, [&] { return launch_accept(tree_tokens, tree_parent, c->argmax, n, T, out_accept_len, out_accept_idx, out_next, st); }));
+    if (!c->dbg_skip_compact) {
+      CK(run(c, MLORA_PROF_MISC, [&] {
+        return launch_compact(c->own_k, c->own_v, c->own_layer_stride, c->own_stream_stride, c->own_head_stride, c->L, n,
+                              c->d.n_kv_heads, c->d.head_dim, c->suffix_len, out_accept_len, out_accept_idx, T, st);
+      }));
+      CK(run(c, MLORA_PROF_MISC, [&] { return launch_advance(c->suffix_len, out_accept_len, n, 0, st); }));
+    }
+    return MLORA_OK;
+  });
+  if (rc != MLORA_OK) return rc;
+  if (!c->dbg_skip_compact) {
+    c->suffix_bound += T;
+    if (c->snap_pending) c->snap_inc += T;
+    else if (!c->profiling) {
+      // ask for the true lengths so that the pessimistic bound can be tightened a few rounds later
+      CK(cudaMemcpyAsync(c->snap, c->suffix_len, sizeof(int32_t) * c->d.max_streams, cudaMemcpyDeviceToHost, c->stream));
+      CK(cudaEventRecord(c->snap_event, c->stream));
+      c->snap_pending = true;
+      c->snap_inc = 0;
+    }
+  }
+  return MLORA_OK;
+}
+
+int mlora_reset_streams(mlora_ctx* c) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  CK(cudaMemsetAsync(c->suffix_len, 0, sizeof(int32_t) * c->d.max_streams, c->stream));
+  c->suffix_bound = 0;
+  c->snap_pending = false;
+  return MLORA_OK;
+}
+
+int mlora_sync_status(mlora_ctx* c) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  CK(cudaStreamSynchronize(c->stream));
+  int st = 0;
+  CK(cudaMemcpy(&st, c->status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (st != 0) {
+    CK(cudaMemset(c->status, 0, sizeof(int)));
+    return fail(st, "device status: malformed tree or token id out of range");
+  }
+  return MLORA_OK;
+}
+
+int mlora_export_kv(mlora_ctx* c, int32_t layer, int32_t stream, int32_t first, int32_t count, int32_t* suffix_len,
+                    void* k_out, void* v_out) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (layer < 0 || layer >= c->L || stream < -1 || stream >= c->d.max_streams || first < 0 || count < 0)
+    return fail(MLORA_ERR_ARG, "export_kv: index out of range");
+  CK(cudaStreamSynchronize(c->stream));
+  const int hd = c->d.head_dim, Hkv = c->d.n_kv_heads;
+  const __half *ks, *vs;
+  size_t head_stride;
+  int limit;
+  if (stream < 0) {
+    ks = c->prefix_k + (size_t)layer * c->prefix_layer_stride;
+    vs = c->prefix_v + (size_t)layer * c->prefix_layer_stride;
+    head_stride = c->prefix_head_stride; limit = c->d.max_prefix;
+    if (suffix_len) *suffix_len = c->P;
+  } else {
+    ks = c->own_k + (size_t)layer * c->own_layer_stride + (size_t)stream * c->own_stream_stride;
+    vs = c->own_v + (size_t)layer * c->own_layer_stride + (size_t)stream * c->own_stream_stride;
+    head_stride = c->own_head_stride; limit = c->cap;
+    if (suffix_len) CK(cudaMemcpy(suffix_len, c->suffix_len + stream, sizeof(int32_t), cudaMemcpyDeviceToHost));
+  }
+  if (first + count > limit) return fail(MLORA_ERR_ARG, "export_kv: rows beyond the segment");
+  if (count == 0) return MLORA_OK;
+  if (!k_out || !v_out) return fail(MLORA_ERR_ARG, "export_kv: null output");
+  for (int kh = 0; kh < Hkv; ++kh) {
+    CK(cudaMemcpy2DAsync((__half*)k_out + (size_t)kh * hd, (size_t)Hkv * hd * 2, ks + kh * head_stride + (size_t)first * hd,
+                         (size_t)hd * 2, (size_t)hd * 2, count, cudaMemcpyDeviceToDevice, c->stream));
+    CK(cudaMemcpy2DAsync((__half*)v_out + (size_t)kh * hd, (size_t)Hkv * hd * 2, vs + kh * head_stride + (size_t)first * hd,
+                         (size_t)hd * 2, (size_t)hd * 2, count, cudaMemcpyDeviceToDevice, c->stream));
+  }
+  CK(cudaStreamSynchronize(c->stream));
+  return MLORA_OK;
+}
+
+int mlora_debug_dequant(mlora_ctx* c, int32_t layer, int32_t proj, void* out_fp16) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (!out_fp16) return fail(MLORA_ERR_ARG, "null output");
+  const PackedWeight* w = nullptr;
+  int N = 0, off = 0, stride = 1;
+  const int F = c->d.d_ffn;
+  if (layer == c->L && proj == 0 && c->d.vocab > 0) { w = &c->w_lm; N = c->d.vocab; }
+  else if (layer >= 0 && layer < c->L && proj >= 0 && proj < 7) {
+    switch (proj) {
+      case 0: w = &c->w_qkv[layer]; N = c->Nq; break;
+      case 1: w = &c->w_qkv[layer]; N = c->Nkv; off = c->Nq / 16; break;
+      case 2: w = &c->w_qkv[layer]; N = c->Nkv; off = (c->Nq + c->Nkv) / 16; break;
+      case 3: w = &c->w_o[layer]; N = c->d.d_model; break;
+      case 4: w = &c->w_gateup[layer]; N = F; stride = 2; break;
+      case 5: w = &c->w_gateup[layer]; N = F; off = 1; stride = 2; break;
+      default: w = &c->w_down[layer]; N = c->d.d_model; break;
+    }
+  } else return fail(MLORA_ERR_ARG, "debug_dequant: no such projection");
+  CK(launch_dequant(w->wq, w->sc, w->K, N, w->G, off, stride, w->N / 16, (__half*)out_fp16, c->stream));
+  c->launches++;
+  return MLORA_OK;
+}
+
+int mlora_debug_set(mlora_ctx* c, int32_t key, int32_t value) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (key == 1) c->dbg_skip_compact = value ? 1 : 0;
+  else if (key == 2) c->dbg_no_graph = value ? 1 : 0;
+  else return fail(MLORA_ERR_ARG, "unknown debug key");
+  return MLORA_OK;
+}
+
+int mlora_profile_begin(mlora_ctx* c) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  CK(cudaStreamSynchronize(c->stream));
+  c->profiling = true;
+  return MLORA_OK;
+}
+
+int mlora_profile_end(mlora_ctx* c, float* ms, int32_t* launches) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  CK(cudaStreamSynchronize(c->stream));
+  c->profiling = false;
+  for (int i = 0; i < MLORA_PROF_FAMILIES; ++i) { if (ms) ms[i] = 0.f; if (launches) launches[i] = 0; }
+  for (auto& e : c->evs) {
+    float t = 0.f;
+    cudaEventElapsedTime(&t, e.a, e.b);
+    if (ms) ms[e.fam] += t;
+    if (launches) launches[e.fam] += 1;
+    c->ev_pool.push_back(e.a);
+    c->ev_pool.push_back(e.b);
+  }
+  c->evs.clear();
+  return MLORA_OK;
+}
+
+int64_t mlora_launch_count(mlora_ctx* c) { return c ? c->launches : 0; }
+
+// ----------------------------------------------------------------------------- kernel-level calls
+int mlora_weight_create(const void* qweight, const void* scales, int32_t K, int32_t N, int32_t G, void* cuda_stream,
+                        mlora_weight** out) {
+  if (!qweight || !scales || !out) return fail(MLORA_ERR_ARG, "null argument");
+  if (init_kernels() != MLORA_OK) return MLORA_ERR_CUDA;
+  if (K <= 0 || N <= 0 || G <= 0 || K % 64 || N % 16 || G % 64 || K % G) return fail(MLORA_ERR_UNSUPPORTED, "need K%64==0, N%16==0, G%64==0, K%G==0");
+  mlora_weight* w = new mlora_weight();
+  w->stream = (cudaStream_t)cuda_stream;
+  cudaError_t e = alloc_packed(w->w, K, N, G);
+  if (e == cudaSuccess) e = launch_repack((const uint8_t*)qweight, (const __half*)scales, K, N, G, w->w.wq, w->w.sc, 0, 1, N / 16, w->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(w->stream);
+  if (e != cudaSuccess) { free_packed(w->w); delete w; return fail(MLORA_ERR_CUDA, cudaGetErrorString(e)); }
+  *out = w;
+  return MLORA_OK;
+}
+
+int mlora_weight_destroy(mlora_weight* w) {
+  if (!w) return MLORA_OK;
+  cudaStreamSynchronize(w->stream);
+  free_packed(w->w);
+  delete w;
+  return MLORA_OK;
+}
+
+int mlora_weight_dequant(mlora_weight* w, void* out_fp16) {
+  if (!w || !out_fp16) return fail(MLORA_ERR_ARG, "null argument");
+  CK(launch_dequant(w->w.wq, w->w.sc, w->w.K, w->w.N, w->w.G, 0, 1, w->w.N / 16, (__half*)out_fp16, w->stream));
+  return MLORA_OK;
+}
+
+static const size_t LIN_COUNTER_BYTES = 4096 * sizeof(unsigned);
+static size_t lin_T_bytes(int M, int rank) { return (((size_t)M * (rank > 0 ? rank : 1) * sizeof(float)) + 255) / 256 * 256; }
+
+size_t mlora_linear_workspace_bytes(const mlora_weight* w, int32_t M, int32_t rank) {
+  if (!w || M <= 0) return 0;
+  // counters + T + split-K partials for up to 8 splits (the planner uses fewer when this does not fit)
+  return LIN_COUNTER_BYTES + lin_T_bytes(M, rank) + (size_t)8 * M * w->w.N * sizeof(float);
+}
+
+int mlora_linear(mlora_weight* w, const void* x, int32_t M, const int32_t* row_adapter, const void* const* A,
+                 const void* const* B, const float* scale, int32_t n_adapters, int32_t rank, float* y, void* workspace,
+                 size_t workspace_bytes) {
+  if (!w || !x || !y || !workspace) return fail(MLORA_ERR_ARG, "null argument");
+  if (M <= 0 || M > 4096) return fail(MLORA_ERR_UNSUPPORTED, "M must be in 1..4096");
+  const bool lora = row_adapter != nullptr;
+  if (lora && (!A || !B || !scale || n_adapters <= 0 || rank <= 0)) return fail(MLORA_ERR_ARG, "incomplete adapter arguments");
+  const size_t fixed = LIN_COUNTER_BYTES + lin_T_bytes(M, rank);
+  if (workspace_bytes < fixed + (size_t)M * w->w.N * sizeof(float)) return fail(MLORA_ERR_CAPACITY, "workspace too small");
+  const int m_blocks = (M + GEMM_MAX_MT * 8 - 1) / (GEMM_MAX_MT * 8);
+  if ((size_t)((w->w.N + GEMM_NB - 1) / GEMM_NB) * m_blocks > 4096) return fail(MLORA_ERR_UNSUPPORTED, "too many output blocks");
+  unsigned char* ws = (unsigned char*)workspace;
+  LoraArgs la{};
+  if (lora) {
+    la.adapter_idx = row_adapter; la.rows_per_stream = 1;
+    la.tabA = (const __half* const*)A; la.tabB = (const __half* const*)B; la.scale = scale;
+    la.tab_stride = 1; la.n_slots = n_adapters; la.rank = rank; la.nseg = 1;
+    la.seg[0].proj_index = 0; la.seg[0].n = w->w.N;
+    la.T = (float*)(ws + LIN_COUNTER_BYTES);
+    ShrinkArgs s{};
+    s.h_in = (const __half*)x; s.M = M; s.K = w->w.K; s.lora = la;
+    CK(launch_shrink(s, w->stream));
+  }
+  GemmArgs g{};
+  g.wq = w->w.wq; g.sc = w->w.sc; g.K = w->w.K; g.N = w->w.N; g.G = w->w.G; g.h = (const __half*)x; g.M = M;
+  g.mode = MODE_PLAIN; g.epi = EPI_F32; g.out_f32 = y; g.ldo = w->w.N;
+  g.partial = (float*)(ws + fixed); g.partial_capacity = (workspace_bytes - fixed) / sizeof(float);
+  g.counters = (unsigned*)ws;
+  g.lora = la;
+  CK(launch_gemm(g, w->stream));
+  return MLORA_OK;
+}
+
+static void attn_fill(AttnArgs& a, int n, int T, int Hq, int Hkv, int hd, int P, int suffix_bound) {
+  a = AttnArgs{};
+  a.P = P; a.n = n; a.T = T; a.Hq = Hq; a.Hkv = Hkv; a.hd = hd;
+  a.suffix_bound = suffix_bound;
+  attn_plan(a, 148);
+}
+
+size_t mlora_attention_workspace_bytes(int32_t n, int32_t T, int32_t Hq, int32_t Hkv, int32_t hd, int32_t P,
+                                       int32_t own_capacity) {
+  if (n <= 0 || T <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv) return 0;
+  AttnArgs a;
+  attn_fill(a, n, T, Hq, Hkv, hd, P, own_capacity > T ? own_capacity - T : 0);
+  const size_t rows = (size_t)n * T;
+  return rows * (sizeof(unsigned long long) + sizeof(int32_t)) + 256 + attn_workspace_floats(a) * sizeof(float);
+}
+
+int mlora_attention(const void* q, const void* prefix_k, const void* prefix_v, int32_t P, const void* own_k,
+                    const void* own_v, int32_t own_capacity, const int32_t* suffix_len, int32_t suffix_bound,
+                    const int32_t* tree_parent, int32_t n, int32_t T, int32_t Hq, int32_t Hkv, int32_t hd, void* out,
+                    void* workspace, size_t workspace_bytes, int32_t* status, void* cuda_stream) {
+  if (!q || !own_k || !own_v || !suffix_len || !tree_parent || !out || !workspace || !status)
+    return fail(MLORA_ERR_ARG, "null argument");
+  if (P > 0 && (!prefix_k || !prefix_v)) return fail(MLORA_ERR_ARG, "null prefix");
+  if (n <= 0 || T <= 0 || T > 64 || Hq <= 0 || Hkv <= 0 || Hq % Hkv || P < 0) return fail(MLORA_ERR_ARG, "bad shape");
+  if (hd != 64 && hd != 128) return fail(MLORA_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+  if (suffix_bound < 0 || suffix_bound + T > own_capacity) return fail(MLORA_ERR_CAPACITY, "suffix_bound + n_nodes exceeds own_capacity");
+  if (init_kernels() != MLORA_OK) return MLORA_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  AttnArgs a;
+  attn_fill(a, n, T, Hq, Hkv, hd, P, suffix_bound);
+  const size_t rows = (size_t)n * T;
+  const size_t head = (rows * (sizeof(unsigned long long) + sizeof(int32_t)) + 255) / 256 * 256;
+  if (workspace_bytes < head + attn_workspace_floats(a) * sizeof(float)) return fail(MLORA_ERR_CAPACITY, "workspace too small");
+  unsigned char* ws = (unsigned char*)workspace;
+  unsigned long long* anc = (unsigned long long*)ws;
+  int32_t* depth = (int32_t*)(ws + rows * sizeof(unsigned long long));
+  CK(launch_tree_prep(tree_parent, n, T, anc, depth, status, st));
+  a.q = (const __half*)q;
+  a.prefix_k = (const __half*)prefix_k; a.prefix_v = (const __half*)prefix_v; a.prefix_head_stride = (size_t)P * hd;
+  a.own_k = (const __half*)own_k; a.own_v = (const __half*)own_v;
+  a.own_head_stride = (size_t)own_capacity * hd; a.own_stream_stride = a.own_head_stride * Hkv;
+  a.suffix_len = suffix_len; a.anc = anc; a.out = (__half*)out;
+  a.part_o = (float*)(ws + head);
+  a.part_ml = a.part_o + (attn_workspace_floats(a) / (hd + 2)) * hd;
+  CK(launch_attention(a, st));
+  CK(launch_attention_merge(a, st));
+  return MLORA_OK;
+}
+
+}  // extern "C"

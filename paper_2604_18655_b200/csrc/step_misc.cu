@@ -1,0 +1,255 @@
+// Small kernels around the projections: embedding gather, draft-tree preparation (ancestor masks and
+// depths, Sec. 3.5 / App. A.2), RoPE + KV append (Sec. 3.1), row argmax, the greedy longest-accepted-path
+// walk and the KV compaction that follows it (Sec. 3.5).
+#include "common.cuh"
+
+namespace mlora {
+
+// ----------------------------------------------------------------------------- embedding / hidden input
+__global__ void embed_kernel(const int32_t* __restrict__ tokens, const __half* __restrict__ embed,
+                             const __half* __restrict__ hidden_in, float* __restrict__ X, int d, int vocab,
+                             int* __restrict__ status) {
+  const int m = blockIdx.x;
+  const __half* src;
+  if (hidden_in != nullptr) {
+    src = hidden_in + (size_t)m * d;
+  } else {
+    int tok = tokens[m];
+    if (tok < 0 || tok >= vocab) {           // keep the access in bounds, report through the status word
+      if (threadIdx.x == 0) atomicCAS(status, 0, -1);
+      tok = 0;
+    }
+    src = embed + (size_t)tok * d;
+  }
+  for (int k = threadIdx.x * 2; k < d; k += blockDim.x * 2) {
+    const float2 v = __half22float2(*reinterpret_cast<const __half2*>(src + k));
+    *reinterpret_cast<float2*>(X + (size_t)m * d + k) = v;
+  }
+}
+
+cudaError_t launch_embed(const int32_t* tokens, const __half* embed, const __half* hidden_in, float* X, int M, int d,
+                         int vocab, int* status, cudaStream_t st) {
+  embed_kernel<<<M, 256, 0, st>>>(tokens, embed, hidden_in, X, d, vocab, status);
+  return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------- tree preparation
+// One thread per (stream, node): walks to the root, collecting the ancestor-or-self bit mask and the depth.
+// A parent outside [0, i) (or a non-root node 0) sets the status word and is treated as the root's child,
+// which keeps every later access in bounds.
+__global__ void tree_prep_kernel(const int32_t* __restrict__ parent, int n, int T, unsigned long long* __restrict__ anc,
+                                 int32_t* __restrict__ depth, int* __restrict__ status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n * T) return;
+  const int s = i / T, t = i % T;
+  const int32_t* par = parent + (size_t)s * T;
+  unsigned long long mask = 0ull;
+  int d = 0, c = t;
+  bool bad = (par[0] != -1);
+  for (int it = 0; it < 64 && c > 0; ++it) {
+    mask |= 1ull << c;
+    int pc = par[c];
+    if (pc < 0 || pc >= c) { bad = true; pc = 0; }
+    c = pc;
+    ++d;
+  }
+  mask |= 1ull;
+  anc[i] = mask;
+  depth[i] = d;
+  if (bad) atomicCAS(status, 0, -1);
+}
+
+cudaError_t launch_tree_prep(const int32_t* parent, int n, int T, unsigned long long* anc, int32_t* depth, int* status,
+                             cudaStream_t st) {
+  const int total = n * T;
+  tree_prep_kernel<<<(total + 127) / 128, 128, 0, st>>>(parent, n, T, anc, depth, status);
+  return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------- RoPE + KV append
+// Row m = s*T + t sits at position pos_base + suffix_len[s] + depth[m]; q and k rotate in (i, i + hd/2) pairs.
+// q goes to fp16 [M][Hq][hd]; k and v go to slot suffix_len[s] + t of the stream's own segment.
+__global__ void rope_kv_kernel(const float* __restrict__ qkv, int T, int Hq, int Hkv, int hd,
+                               const float2* __restrict__ cs_table, int pos_base, const int32_t* __restrict__ suffix_len,
+                               const int32_t* __restrict__ depth, __half* __restrict__ q_out, __half* __restrict__ k_dst,
+                               __half* __restrict__ v_dst, size_t stream_stride, size_t head_stride) {
+  const int m = blockIdx.x;
+  const int s = m / T, t = m % T;
+  const int S = suffix_len[s];
+  const int pos = pos_base + S + depth[m];
+  const int half = hd >> 1;
+  const int Nq = Hq * hd, Nkv = Hkv * hd;
+  const float* row = qkv + (size_t)m * (Nq + 2 * Nkv);
+  const float2* cs = cs_table + (size_t)pos * half;
+  // q heads and k heads: one thread per rotation pair
+  for (int i = threadIdx.x; i < (Hq + Hkv) * half; i += blockDim.x) {
+    const int head = i / half, e = i % half;
+    const float2 c = cs[e];
+    const float* src = row + (size_t)head * hd;      // k heads follow the q heads in the fused row
+    const float x1 = src[e], x2 = src[e + half];
+    const __half o1 = __float2half_rn(x1 * c.x - x2 * c.y);
+    const __half o2 = __float2half_rn(x2 * c.x + x1 * c.y);
+    __half* dst;
+    if (head < Hq) dst = q_out + ((size_t)m * Hq + head) * hd;
+    else dst = k_dst + (size_t)s * stream_stride + (size_t)(head - Hq) * head_stride + (size_t)(S + t) * hd;
+    dst[e] = o1;
+    dst[e + half] = o2;
+  }
+  for (int i = threadIdx.x; i < Nkv; i += blockDim.x) {
+    const int head = i / hd, e = i % hd;
+    v_dst[(size_t)s * stream_stride + (size_t)head * head_stride + (size_t)(S + t) * hd + e] =
+        __float2half_rn(row[Nq + Nkv + i]);
+  }
+}
+
+cudaError_t launch_rope_kv(const float* qkv, int M, int T, int Hq, int Hkv, int hd, const float2* cs_table,
+                           int pos_base, const int32_t* suffix_len, const int32_t* depth, __half* q_out, __half* k_dst,
+                           __half* v_dst, size_t stream_stride, size_t head_stride, cudaStream_t st) {
+  rope_kv_kernel<<<M, 256, 0, st>>>(qkv, T, Hq, Hkv, hd, cs_table, pos_base, suffix_len, depth, q_out, k_dst, v_dst,
+                                   stream_stride, head_stride);
+  return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------- argmax (lowest index on ties)
+__global__ void argmax_kernel(const float* __restrict__ logits, int V, int32_t* __restrict__ out) {
+  const int m = blockIdx.x;
+  const float* row = logits + (size_t)m * V;
+  float best = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int i = threadIdx.x; i < V; i += blockDim.x) {
+    const float v = row[i];
+    if (v > best || (v == best && i < bi)) { best = v; bi = i; }
+  }
+  __shared__ float sb[32];
+  __shared__ int si[32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) { sb[warp] = best; si[warp] = bi; }
+  __syncthreads();
+  if (warp == 0) {
+    const int nw = blockDim.x >> 5;
+    best = lane < nw ? sb[lane] : -INFINITY;
+    bi = lane < nw ? si[lane] : 0x7fffffff;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+    }
+    if (lane == 0) out[m] = (bi == 0x7fffffff) ? 0 : bi;
+  }
+}
+
+cudaError_t launch_argmax(const float* logits, int M, int V, int32_t* out, cudaStream_t st) {
+  argmax_kernel<<<M, 1024, 0, st>>>(logits, V, out);
+  return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------- greedy longest accepted path
+// One warp per stream.  From the root: g = argmax at the current node; the lanes test the candidate
+// children in parallel and the lowest matching node index wins; stop when no child carries g.
+__global__ void accept_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
+                              const int32_t* __restrict__ argmax, int T, int32_t* __restrict__ acc_len,
+                              int32_t* __restrict__ acc_idx, int32_t* __restrict__ next) {
+  const int s = blockIdx.x;
+  const int lane = threadIdx.x;
+  const int32_t* tok = tokens + (size_t)s * T;
+  const int32_t* par = parent + (size_t)s * T;
+  const int32_t* am = argmax + (size_t)s * T;
+  int32_t* idx = acc_idx + (size_t)s * T;
+  for (int i = lane; i < T; i += 32) idx[i] = -1;
+  __syncwarp();
+  int c = 0, len = 1;
+  if (lane == 0) idx[0] = 0;
+  for (int it = 0; it < T; ++it) {
+    const int g = am[c];
+    int found = -1;
+    for (int base = c + 1; base < T && found < 0; base += 32) {
+      const int u = base + lane;
+      const bool hit = (u < T) && (par[u] == c) && (tok[u] == g);
+      const unsigned b = __ballot_sync(0xffffffffu, hit);
+      if (b) found = base + __ffs(b) - 1;
+    }
+    if (found < 0) break;
+    c = found;
+    if (lane == 0) idx[len] = c;
+    ++len;
+  }
+  if (lane == 0) {
+    acc_len[s] = len;
+    next[s] = am[c];
+  }
+}
+
+cudaError_t launch_accept(const int32_t* tokens, const int32_t* parent, const int32_t* argmax, int n, int T,
+                          int32_t* acc_len, int32_t* acc_idx, int32_t* next, cudaStream_t st) {
+  accept_kernel<<<n, 32, 0, st>>>(tokens, parent, argmax, T, acc_len, acc_idx, next);
+  return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------- KV compaction
+// For (layer, stream, kv head): row suffix+acc_idx[j] moves to row suffix+j, j ascending.  Path indices are
+// strictly increasing with acc_idx[j] >= j, so a destination never covers a source that is still to be read.
+__global__ void compact_kernel(__half* __restrict__ own_k, __half* __restrict__ own_v, size_t layer_stride,
+                               size_t stream_stride, size_t head_stride, int hd, const int32_t* __restrict__ suffix_len,
+                               const int32_t* __restrict__ acc_len, const int32_t* __restrict__ acc_idx, int T) {
+  const int l = blockIdx.z, s = blockIdx.y, kh = blockIdx.x;
+  const int len = acc_len[s], S = suffix_len[s];
+  const size_t base = (size_t)l * layer_stride + (size_t)s * stream_stride + (size_t)kh * head_stride;
+  const int vecs = hd / 8;                                   // 16-byte pieces per row
+  for (int j = 1; j < len; ++j) {
+    const int src = acc_idx[(size_t)s * T + j];
+    if (src != j) {
+      uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
+      if ((int)threadIdx.x < vecs) {
+        kv = *reinterpret_cast<const uint4*>(own_k + base + (size_t)(S + src) * hd + threadIdx.x * 8);
+        vv = *reinterpret_cast<const uint4*>(own_v + base + (size_t)(S + src) * hd + threadIdx.x * 8);
+      }
+      __syncthreads();
+      if ((int)threadIdx.x < vecs) {
+        *reinterpret_cast<uint4*>(own_k + base + (size_t)(S + j) * hd + threadIdx.x * 8) = kv;
+        *reinterpret_cast<uint4*>(own_v + base + (size_t)(S + j) * hd + threadIdx.x * 8) = vv;
+      }
+      __syncthreads();
+    }
+  }
+}
+
+cudaError_t launch_compact(__half* own_k, __half* own_v, size_t layer_stride, size_t stream_stride, size_t head_stride,
+                           int L, int n, int Hkv, int hd, const int32_t* suffix_len, const int32_t* acc_len,
+                           const int32_t* acc_idx, int T, cudaStream_t st) {
+  dim3 grid(Hkv, n, L);
+  compact_kernel<<<grid, 32, 0, st>>>(own_k, own_v, layer_stride, stream_stride, head_stride, hd, suffix_len, acc_len,
+                                      acc_idx, T);
+  return cudaGetLastError();
+}
+
+__global__ void advance_kernel(int32_t* __restrict__ suffix_len, const int32_t* __restrict__ acc_len, int n, int fixed) {
+  const int s = threadIdx.x;
+  if (s < n) suffix_len[s] += (acc_len != nullptr) ? acc_len[s] : fixed;
+}
+
+cudaError_t launch_advance(int32_t* suffix_len, const int32_t* acc_len, int n, int fixed, cudaStream_t st) {
+  advance_kernel<<<1, 256, 0, st>>>(suffix_len, acc_len, n, fixed);
+  return cudaGetLastError();
+}
+
+__global__ void copy_f32_kernel(const float* __restrict__ src, float* __restrict__ dst, size_t count) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = src[i];
+}
+
+cudaError_t launch_copy_rows_f32(const float* src, float* dst, size_t count, cudaStream_t st) {
+  int blocks = (int)((count + 255) / 256);
+  if (blocks > 1024) blocks = 1024;
+  if (blocks < 1) blocks = 1;
+  copy_f32_kernel<<<blocks, 256, 0, st>>>(src, dst, count);
+  return cudaGetLastError();
+}
+
+}  // namespace mlora

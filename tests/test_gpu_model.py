@@ -1,0 +1,289 @@
+"""End-to-end parity of the decode / verify path on small models, through the C ABI, against the oracle."""
+import numpy as np
+import pytest
+
+import gen
+from oracle import ref
+from tests.helpers import compare, check_argmax
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+# small model with a vocabulary: 2 layers, GQA 4/2 heads of 64, adapters on all seven projections
+TINYV = gen.ModelCfg("tinyv", 2, 128, 4, 2, 64, 192, 160, 64, 4, 127, 3, 3, 70, b_std=0.05)
+
+
+@pytest.fixture(scope="module")
+def GpuModel():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from tests.helpers import GpuModel as G
+    return G
+
+
+def make_pair(GpuModel, cfg, seed=0, **kw):
+    m = gen.make_model(cfg, seed)
+    orc = ref.OracleModel.from_synth(m)
+    gm = GpuModel(m, **kw)
+    for a in range(cfg.n_adapters):
+        A, B = gen.make_adapter(cfg, a, seed)
+        orc.set_adapter(a, A, B, cfg.alpha)
+        gm.set_adapter(a, A, B, cfg.alpha)
+    return m, orc, gm
+
+
+def compare_kv(gm, orc, cfg, n_streams):
+    from paper_2604_18655_b200 import binding as mb
+    for l in range(cfg.n_layers):
+        for s in range(n_streams):
+            S = orc.suffix_len(s)
+            got_s, k, v = gm.export_kv(l, s, 0, S)
+            assert got_s == S
+            if S:
+                compare(k, orc.suf_k[l][s], f"suffix K l{l} s{s}")
+                compare(v, orc.suf_v[l][s], f"suffix V l{l} s{s}")
+    mb.mlora_sync_status(gm.ctx)
+
+
+def test_cfg0_hidden_state_decode(GpuModel):
+    cfg = gen.CFG0
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=8)
+    prompt = gen.make_hidden(cfg, cfg.prompt_len, 0, 0)
+    want_last = orc.prefill_shared(hidden=prompt)
+    got_last = gm.prefill_h(prompt)
+    compare(got_last, want_last, "prefill last hidden")
+    # shared segment KV
+    _, pk, pv = gm.export_kv(0, -1, 0, cfg.prompt_len)
+    compare(pk, orc.prefix_k[0], "prefix K")
+    compare(pv, orc.prefix_v[0], "prefix V")
+    ad = list(range(cfg.n_streams))
+    for step in range(3):
+        x = gen.make_hidden(cfg, cfg.n_streams, 0, 1 + step)
+        want = orc.decode_step(ad, hidden=x)["hidden"]
+        got = gm.decode_h(ad, x)
+        compare(got, want, f"decode hidden step {step}")
+    compare_kv(gm, orc, cfg, cfg.n_streams)
+    gm.close()
+
+
+def test_prefill_logits_and_follow_mode_decode(GpuModel):
+    cfg = TINYV
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=32)
+    ids = gen.make_prompt_ids(cfg, 0)
+    compare(gm.prefill(ids), orc.prefill_shared(ids), "prefill logits")
+    ad = [0, 2, -1]
+    toks = np.array([3, 50, 7], dtype=np.int32)
+    ties = 0
+    for step in range(8):
+        nxt, logits = gm.decode(ad, toks)
+        r = orc.decode_step(ad, tokens=toks)
+        compare(logits, r["logits"], f"decode logits step {step}")
+        ties += check_argmax(nxt, r["logits"], f"step {step}")
+        assert np.array_equal(nxt, np.argmax(logits, axis=1))            # the GPU's argmax of its own logits
+        toks = nxt                                                        # follow the GPU's tokens
+    compare_kv(gm, orc, cfg, 3)
+    gm.close()
+
+
+def test_adapter_switch_without_recreate(GpuModel):
+    """Adapters are run-time inputs: swapping a slot's tensors changes the next step, clearing gives the base."""
+    cfg = TINYV
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=32)
+    ids = gen.make_prompt_ids(cfg, 0)
+    gm.prefill(ids)
+    orc.prefill_shared(ids)
+    A9, B9 = gen.make_adapter(cfg, 9, 0)
+    gm.set_adapter(1, A9, B9, 8.0)
+    orc.set_adapter(1, A9, B9, 8.0)
+    gm.set_adapter(2, None, None, 0)
+    orc.set_adapter(2, None, None, 0)
+    _, logits = gm.decode([1, 2, -1], [5, 5, 5])
+    r = orc.decode_step([1, 2, -1], tokens=[5, 5, 5])
+    compare(logits, r["logits"], "after adapter switch")
+    assert np.abs(logits[0] - logits[2]).max() > 1e-3                     # adapter visible
+    compare(logits[1], logits[2], "cleared slot equals base")
+    gm.close()
+
+
+def planted_tree_tokens(rng, cfg, parent, last, truth):
+    """Random drafts with the true continuation planted along one branch (deepest-first children)."""
+    n, T = len(last), len(parent)
+    toks = rng.integers(0, cfg.vocab, size=(n, T)).astype(np.int32)
+    toks[:, 0] = last
+    dep = gen.tree_depths(parent)
+    for s in range(n):
+        node = 0
+        for d in range(len(truth[s])):
+            kids = [u for u in range(T) if parent[u] == node]
+            if not kids:
+                break
+            node = kids[-1]                                              # the last child carries the match
+            toks[s, node] = truth[s][d]
+    return toks
+
+
+def test_verify_tree_follow_mode_accept_and_kv(GpuModel):
+    cfg = TINYV
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=64, max_tree=16)
+    ids = gen.make_prompt_ids(cfg, 0)
+    gm.prefill(ids)
+    orc.prefill_shared(ids)
+    ad = [1, 0, 2]
+    # plain greedy continuation from the oracle, used as the planted truth
+    o2 = ref.OracleModel.from_synth(m)
+    for a in range(cfg.n_adapters):
+        A, B = gen.make_adapter(cfg, a, 0)
+        o2.set_adapter(a, A, B, cfg.alpha)
+    o2.prefill_shared(ids)
+    first = np.array([11, 12, 13], dtype=np.int32)
+    cur, truth = first.copy(), [[] for _ in ad]
+    for _ in range(20):
+        cur = o2.decode_step(ad, tokens=cur)["next"]
+        for s in range(3):
+            truth[s].append(int(cur[s]))
+    parent = gen.build_tree((4, 2, 2), 16)
+    rng = np.random.default_rng(4)
+    last = first.copy()
+    emitted = [[] for _ in ad]
+    total_accept = 0
+    for rnd in range(5):
+        plant = [truth[s][len(emitted[s]):len(emitted[s]) + 2] for s in range(3)]
+        toks = planted_tree_tokens(rng, cfg, parent, last, plant)
+        par = np.stack([parent] * 3)
+        g = gm.verify(ad, toks, par)
+        gpu_argmax = np.argmax(g["logits"], axis=1).reshape(3, 16)
+        r = orc.verify_tree(ad, par, toks, follow_argmax=gpu_argmax)
+        compare(g["logits"], r["logits"], f"verify logits round {rnd}")
+        check_argmax(gpu_argmax.reshape(-1), r["logits"], f"round {rnd}")
+        # integer outputs are bit-exact against the oracle's walk on the same argmax
+        assert np.array_equal(g["accept_len"], r["accept_len"])
+        assert np.array_equal(g["accept_idx"], r["accept_idx"])
+        assert np.array_equal(g["next"], r["next"])
+        for s in range(3):
+            L = int(g["accept_len"][s])
+            acc = [int(toks[s, i]) for i in g["accept_idx"][s, 1:L]] + [int(g["next"][s])]
+            emitted[s].extend(acc)
+            last[s] = acc[-1]
+            total_accept += L
+    assert total_accept > 15                                             # drafts were accepted (more than 1/round)
+    for s in range(3):
+        assert orc.suffix_len(s) == gm.suffix_len(s)
+    compare_kv(gm, orc, cfg, 3)
+    gm.close()
+
+
+def test_compaction_is_a_bit_exact_copy(GpuModel):
+    """Same verify pass twice from the same state: once with compaction skipped.  Row suffix+j of the
+    compacted cache must equal, bit for bit, tree row accept_idx[j] of the uncompacted one."""
+    from paper_2604_18655_b200 import binding as mb
+    cfg = TINYV
+    ids = gen.make_prompt_ids(cfg, 0)
+    parent = gen.build_tree((2, 2, 2), 12)
+    par = np.stack([parent] * 2)
+    outs = []
+    for skip in (1, 0):
+        m, orc, gm = make_pair(GpuModel, cfg, max_suffix=32, max_tree=12)
+        gm.prefill(ids)
+        nxt, _ = gm.decode([0, 1], [4, 5])
+        toks = np.zeros((2, 12), dtype=np.int32)
+        toks[:, 0] = nxt
+        # make every node match the argmax of its parent: chain of accepts down the first-child path
+        g0 = gm.decode([0, 1], nxt)[0]
+        mb.mlora_reset_streams(gm.ctx)
+        gm.decode([0, 1], [4, 5])
+        toks[:, 1] = g0
+        toks[:, 2] = g0                                                   # duplicate sibling: lowest index must win
+        mb.mlora_debug_set(gm.ctx, 1, skip)
+        g = gm.verify([0, 1], toks, par)
+        S0 = 1
+        rows = [gm.export_kv(l, s, 0, S0 + 12)[1:] for l in range(cfg.n_layers) for s in range(2)]
+        outs.append((g, rows, gm.suffix_len(0)))
+        gm.close()
+    (g_skip, rows_skip, s_skip), (g_cmp, rows_cmp, s_cmp) = outs
+    assert np.array_equal(g_skip["accept_idx"], g_cmp["accept_idx"])
+    assert s_skip == 1 and s_cmp == 1 + int(g_cmp["accept_len"][0])
+    assert int(g_cmp["accept_len"][0]) >= 2 and g_cmp["accept_idx"][0, 1] == 1
+    i = 0
+    for l in range(cfg.n_layers):
+        for s in range(2):
+            L = int(g_cmp["accept_len"][s])
+            for j in range(L):
+                src = int(g_cmp["accept_idx"][s, j])
+                for t in (0, 1):
+                    assert np.array_equal(rows_cmp[i][t][1 + j].view(np.uint16), rows_skip[i][t][1 + src].view(np.uint16))
+            i += 1
+
+
+def test_stream_isolation_on_gpu(GpuModel):
+    cfg = TINYV
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+    ids = gen.make_prompt_ids(cfg, 0)
+    gm.prefill(ids)
+    _, multi = gm.decode([0, 1, 2], [9, 9, 9])
+    for s in range(3):
+        m1, o1, g1 = make_pair(GpuModel, cfg, max_suffix=16, max_streams=1)
+        g1.prefill(ids)
+        _, single = g1.decode([s], [9])
+        compare(multi[s], single[0], f"stream {s} alone")
+        g1.close()
+    gm.close()
+
+
+def test_error_paths(GpuModel):
+    from paper_2604_18655_b200 import binding as mb
+    cfg = TINYV
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=2, max_tree=4)
+    with pytest.raises(mb.MloraError) as e:
+        gm.decode([0], [1])
+    assert e.value.code == -2                                            # no prefill yet
+    with pytest.raises(mb.MloraError) as e:
+        gm.prefill(np.zeros(cfg.prompt_len + 1, dtype=np.int32))
+    assert e.value.code == -3
+    gm.prefill(gen.make_prompt_ids(cfg, 0))
+    with pytest.raises(mb.MloraError) as e:
+        gm.decode([0, 0, 0, 0], [1, 1, 1, 1])
+    assert e.value.code == -1                                            # more streams than max_streams
+    with pytest.raises(mb.MloraError) as e:
+        gm.verify([0], np.zeros((1, 5), dtype=np.int32), np.array([[-1, 0, 0, 0, 0]], dtype=np.int32))
+    assert e.value.code == -3                                            # tree larger than max_tree
+    with pytest.raises(mb.MloraError):
+        gm.set_adapter(99, *gen.make_adapter(cfg, 0, 0), 16.0)
+    # malformed tree: reported through the device status word, context stays usable
+    gm.verify([0], np.zeros((1, 4), dtype=np.int32), np.array([[-1, 0, 2, 1]], dtype=np.int32))
+    with pytest.raises(mb.MloraError) as e:
+        mb.mlora_sync_status(gm.ctx)
+    assert e.value.code == -1
+    mb.mlora_sync_status(gm.ctx)                                          # cleared
+    # own segment capacity: max_suffix 2 (+ max_tree 4 rows of slack for tree rows)
+    mb.mlora_reset_streams(gm.ctx)
+    for _ in range(6):
+        gm.decode([0], [1])
+    with pytest.raises(mb.MloraError) as e:
+        gm.decode([0], [1])
+    assert e.value.code == -3
+    gm.close()
+
+
+def test_graph_replay_matches_direct_launches(GpuModel):
+    """Steps replayed from a CUDA graph give bit-identical logits to directly launched ones."""
+    from paper_2604_18655_b200 import binding as mb
+    cfg = TINYV
+    res = []
+    for no_graph in (1, 0):
+        m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+        mb.mlora_debug_set(gm.ctx, 2, no_graph)
+        gm.prefill(gen.make_prompt_ids(cfg, 0))
+        dev = torch.device("cuda")
+        ad = torch.tensor([0, 1, 2], dtype=torch.int32, device=dev)
+        tok = torch.tensor([1, 2, 3], dtype=torch.int32, device=dev)
+        nxt = torch.empty(3, dtype=torch.int32, device=dev)
+        logits = torch.empty(3, cfg.vocab, dtype=torch.float32, device=dev)
+        hist = []
+        for _ in range(5):
+            mb.mlora_decode_step(gm.ctx, ad, tok, nxt, logits)
+            tok.copy_(nxt)
+            hist.append(logits.cpu().numpy().copy())
+        res.append(np.stack(hist))
+        assert mb.mlora_launch_count(gm.ctx) > 50
+        gm.close()
+    assert np.array_equal(res[0].view(np.uint32), res[1].view(np.uint32))
