@@ -302,7 +302,8 @@ int forward(mlora_ctx* c, const PassIO& io) {
 // runs `body` directly, or captures it once into a CUDA graph and replays it
 template <class F>
 int replay_or_run(mlora_ctx* c, const GraphKey& key, F&& body) {
-  if (c->dbg_no_graph || c->profiling) return body();
+  // the legacy default stream cannot be captured: launch directly there
+  if (c->dbg_no_graph || c->profiling || c->stream == nullptr) return body();
   auto it = c->graphs.find(key);
   if (it == c->graphs.end()) {
     cudaGraph_t graph = nullptr;

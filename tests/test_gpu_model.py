@@ -269,21 +269,25 @@ def test_graph_replay_matches_direct_launches(GpuModel):
     from paper_2604_18655_b200 import binding as mb
     cfg = TINYV
     res = []
+    side = torch.cuda.Stream()                                            # the default stream cannot be captured
     for no_graph in (1, 0):
-        m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
-        mb.mlora_debug_set(gm.ctx, 2, no_graph)
-        gm.prefill(gen.make_prompt_ids(cfg, 0))
-        dev = torch.device("cuda")
-        ad = torch.tensor([0, 1, 2], dtype=torch.int32, device=dev)
-        tok = torch.tensor([1, 2, 3], dtype=torch.int32, device=dev)
-        nxt = torch.empty(3, dtype=torch.int32, device=dev)
-        logits = torch.empty(3, cfg.vocab, dtype=torch.float32, device=dev)
-        hist = []
-        for _ in range(5):
-            mb.mlora_decode_step(gm.ctx, ad, tok, nxt, logits)
-            tok.copy_(nxt)
-            hist.append(logits.cpu().numpy().copy())
-        res.append(np.stack(hist))
-        assert mb.mlora_launch_count(gm.ctx) > 50
-        gm.close()
+        with torch.cuda.stream(side):
+            m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+            mb.mlora_debug_set(gm.ctx, 2, no_graph)
+            gm.prefill(gen.make_prompt_ids(cfg, 0))
+            dev = torch.device("cuda")
+            ad = torch.tensor([0, 1, 2], dtype=torch.int32, device=dev)
+            tok = torch.tensor([1, 2, 3], dtype=torch.int32, device=dev)
+            nxt = torch.empty(3, dtype=torch.int32, device=dev)
+            logits = torch.empty(3, cfg.vocab, dtype=torch.float32, device=dev)
+            hist = []
+            before = mb.mlora_launch_count(gm.ctx)
+            for _ in range(5):
+                mb.mlora_decode_step(gm.ctx, ad, tok, nxt, logits)
+                tok.copy_(nxt)
+                side.synchronize()
+                hist.append(logits.cpu().numpy().copy())
+            res.append(np.stack(hist))
+            assert mb.mlora_launch_count(gm.ctx) - before > 50
+            gm.close()
     assert np.array_equal(res[0].view(np.uint32), res[1].view(np.uint32))
