@@ -7,17 +7,56 @@
 namespace mlora {
 
 // ----------------------------------------------------------------------------- layout constants
-// Private weight layout ("fragment-major"): the [K][N] INT4 matrix is cut into tiles of 16 output
+// Private weight layout ("fragment-major, chunked"): the [K][N] INT4 matrix is cut into tiles of 16 output
 // features x 64 input features.  A tile is 32 lanes x 16 bytes: lane (g = lane/4, t = lane%4) owns the
 // 16 consecutive input features k0+16t .. k0+16t+15 of output features n0+g and n0+g+8, so that one
 // 128-bit load per lane feeds four m16n8k16 tensor-core steps (the weights are the 16-wide operand).
-// Tiles are stored [n_tile][k_tile][lane] -- a warp streaming along K reads one contiguous run.
 // Word j (0..3) of the lane's uint4 holds input features k0+16t+4j+{0,1,2,3}:
 //   nibble 0/4: feature +0/+1 of row g      nibble 1/5: feature +0/+1 of row g+8
 //   nibble 2/6: feature +2/+3 of row g      nibble 3/7: feature +2/+3 of row g+8
-// Scales: uint32 [K/G][n_tile][8] -- entry g packs fp16 scale of row n0+g (low) and n0+g+8 (high).
+// The tiles of one n-tile (16 output features, all of K) form one contiguous "unit", cut into chunks of
+// CHUNK_KT k-tiles.  A chunk is self-contained -- its weight tiles followed by the scales of the groups it
+// covers (32 bytes per group: entry g packs the fp16 scale of row n0+g (low) and n0+g+8 (high)) -- so that
+// one bulk copy brings everything a CTA needs for 512 input features of 16 outputs:
+//   unit  = [chunk 0][chunk 1]...            chunk = [kc tiles x 512 B][groups x 32 B]
+// Chunks start on group boundaries: G divides 512 or is a multiple of 512.
 constexpr int TILE_N = 16;
 constexpr int TILE_K = 64;
+constexpr int CHUNK_KT = 8;                    // k-tiles per chunk (512 input features)
+
+struct WLayout {
+  int K, N, G, KT, NT, nchunks, kc_last, gpc, g_last;
+  uint32_t chunk_full, chunk_last;             // bytes
+  size_t unit_bytes;
+};
+__host__ __device__ inline WLayout make_wlayout(int K, int N, int G) {
+  WLayout L;
+  L.K = K; L.N = N; L.G = G;
+  L.KT = K / TILE_K; L.NT = N / TILE_N;
+  L.nchunks = (L.KT + CHUNK_KT - 1) / CHUNK_KT;
+  L.kc_last = L.KT - (L.nchunks - 1) * CHUNK_KT;
+  const int ck = CHUNK_KT * TILE_K;
+  L.gpc = G >= ck ? 1 : ck / G;
+  L.g_last = G >= ck ? 1 : (L.kc_last * TILE_K + G - 1) / G;
+  L.chunk_full = CHUNK_KT * 512 + L.gpc * 32;
+  L.chunk_last = L.kc_last * 512 + L.g_last * 32;
+  L.unit_bytes = (size_t)(L.nchunks - 1) * L.chunk_full + L.chunk_last;
+  return L;
+}
+__host__ __device__ inline bool wlayout_group_ok(int G) {
+  const int ck = CHUNK_KT * TILE_K;
+  return G > 0 && G % TILE_K == 0 && (ck % G == 0 || G % ck == 0);
+}
+// byte offset, inside a unit, of k-tile kt's weights and of the scale entry of its group
+__host__ __device__ inline size_t wl_tile_off(const WLayout& L, int kt) {
+  return (size_t)(kt / CHUNK_KT) * L.chunk_full + (size_t)(kt % CHUNK_KT) * 512;
+}
+__host__ __device__ inline size_t wl_scale_off(const WLayout& L, int kt) {
+  const int c = kt / CHUNK_KT;
+  const int kc = (c == L.nchunks - 1) ? L.kc_last : CHUNK_KT;
+  const int gi = (L.G >= CHUNK_KT * TILE_K) ? 0 : ((kt % CHUNK_KT) * TILE_K) / L.G;
+  return (size_t)c * L.chunk_full + (size_t)kc * 512 + (size_t)gi * 32;
+}
 
 // GEMM CTA shape
 constexpr int GEMM_WARPS = 4;
@@ -49,8 +88,7 @@ struct LoraArgs {
 };
 
 struct GemmArgs {
-  const uint4* wq;
-  const uint32_t* sc;
+  const unsigned char* w;         // packed weights (chunked fragment-major layout)
   int K, N, G;                    // N = physical (fused) width
   const __half* h;                // [M][K]
   int M;
@@ -89,14 +127,61 @@ struct AttnArgs {
   int n_own_chunks, own_chunk;
 };
 
+// ----------------------------------------------------------------------------- persistent projection chain
+// A "phase" is one fused projection group of the decoder (q,k,v | o | gate,up | down | lm_head) over at most
+// 8 rows.  The chain kernel runs a range of phases back to back with a grid barrier between them.
+enum ChainIn { IN_NORM = 0, IN_F16 = 1 };
+struct ChainPhase {
+  const unsigned char* w;         // packed weights
+  int K, N, G;                    // N = physical (fused) width
+  int mode, epi, in_kind;
+  int seg_n0, seg_n1;             // MODE_QKV: widths of the first two segments
+  const float* x_f32;             // IN_NORM: residual stream [M][K]
+  const __half* gain;             // IN_NORM: RMSNorm gain [K]
+  const __half* h_in;             // IN_F16: [M][K]
+  float* out_f32; int ldo;        // EPI_F32 (nullptr: the call's logits destination)
+  float* resid;                   // EPI_RESID: [M][N] in place
+  __half* out_f16;                // EPI_SWIGLU: [M][N/2]
+  int lora_nseg;                  // 0: no LoRA on this group
+  int lora_proj[3];               // index into the adapter pointer tables per segment
+  int lora_n[3];                  // logical output width per segment
+};
+struct ChainArgs {
+  const ChainPhase* phases;       // dev
+  int p0, p1;                     // phase range [p0, p1)
+  int M;
+  float eps;
+  float* logits;                  // destination of a phase whose out_f32 is nullptr
+  const __half* h_in;             // input of an IN_F16 phase whose h_in is nullptr
+  const int32_t* adapter_idx;     // dev; nullptr: base weights only
+  int rows_per_stream;
+  const __half* const* tabA;
+  const __half* const* tabB;
+  const float* scale;
+  int tab_stride, n_slots, rank;
+  float* T;                       // dev fp32 [M][3][rank] scratch
+  unsigned long long* sync;       // dev [4]: grid-barrier arrivals, shrink arrivals, abort flag, spare
+  int* status;                    // dev status word
+  int nstages;                    // ring stages
+  int kmax;                       // largest K of the phases in range (sizes the activation buffer)
+};
+constexpr int CHAIN_MAX_ROWS = 8;
+constexpr int CHAIN_MAX_RANK = 64;
+cudaError_t init_chain();
+// shared memory the chain kernel needs for the given largest K and rank with `nstages` ring stages; 0 if it cannot fit
+size_t chain_smem_bytes(int kmax, int rank, int nstages);
+int chain_pick_stages(int kmax, int rank);      // most stages that fit (0: not eligible)
+cudaError_t launch_chain(const ChainArgs& a, int sm_count, cudaStream_t st);
+
 // ----------------------------------------------------------------------------- launchers
 cudaError_t init_gemm();        // opt-in shared-memory sizes; call once per process before the first launch
 cudaError_t init_shrink();
 cudaError_t init_attention();
-cudaError_t launch_repack(const uint8_t* qweight, const __half* scales, int K, int N, int G, uint4* wq,
-                          uint32_t* sc, int dst_tile_off, int dst_tile_stride, int dst_tiles, cudaStream_t st);
-cudaError_t launch_dequant(const uint4* wq, const uint32_t* sc, int K, int N, int G, int tile_off,
-                           int tile_stride, int tiles_phys, __half* out, cudaStream_t st);
+// repack: logical n-tile nt of the canonical [K][N] matrix goes to physical unit dst_tile_off + nt*dst_tile_stride
+cudaError_t launch_repack(const uint8_t* qweight, const __half* scales, int K, int N, int G, unsigned char* w,
+                          int dst_tile_off, int dst_tile_stride, cudaStream_t st);
+cudaError_t launch_dequant(const unsigned char* w, int K, int N, int G, int tile_off, int tile_stride,
+                           __half* out, cudaStream_t st);
 int gemm_pick_split(int K, int N, int M, size_t partial_capacity);
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
 cudaError_t launch_shrink(const ShrinkArgs& a, cudaStream_t st);

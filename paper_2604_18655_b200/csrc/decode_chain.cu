@@ -1,0 +1,720 @@
+// Persistent projection chain for decode-sized batches (at most 8 rows): a range of fused projection groups
+// of the decoder (Sec. 3.1; LoRA term of Eq. 1-4 with the adapter picked per row, Sec. 3.2 (c); INT4 weights,
+// Sec. 3.3) runs inside ONE cooperative kernel, one CTA per SM, with a grid barrier between groups.
+//
+// Why: at these sizes a projection moves a few MB -- about a microsecond of HBM time -- so a kernel per
+// projection is bound by launch and ramp-up latency.  Here a producer warp streams the CTA's share of the
+// packed INT4 weights of ALL phases through a shared-memory ring with bulk asynchronous copies
+// (cp.async.bulk + mbarrier transaction counts).  Weights do not depend on activations, so the ring keeps
+// filling while the consumer warps sit in a grid barrier or in a prologue: HBM never idles across phase
+// boundaries.  Eight consumer warps split K inside a chunk, dequantise in registers and multiply on the tensor
+// cores (mma.sync m16n8k16: weights are the 16-wide operand, the rows the 8-wide one), reduce across warps in
+// shared memory in a fixed order, and run the epilogue (LoRA expand, residual add, SwiGLU, fp32 store).
+//
+// The LoRA shrink T = (alpha/r) h A^T is spread over all CTAs at the start of a phase (the rows of A come
+// through the same ring, so they are already in shared memory when the phase starts); a counter tells every
+// CTA when all of T is in global memory; the expand happens in the epilogue from slices of B that also came
+// through the ring.
+//
+// Every wait (mbarrier, grid barrier, shrink counter) is bounded by a clock limit.  When one runs out the CTA
+// raises a global abort flag and the status word MLORA_ERR_TIMEOUT; from then on every wait returns at once
+// and the kernel runs its (data-independent) control flow to the end, so no CTA is left in a barrier.
+#include "../../include/mlora.h"
+#include "common.cuh"
+
+namespace mlora {
+
+constexpr int CH_CWARPS = 8;                       // consumer warps
+constexpr int CH_CTHREADS = CH_CWARPS * 32;
+constexpr int CH_THREADS = CH_CTHREADS + 32;       // + one producer warp
+constexpr int CH_STAGE_BYTES = 4480;               // >= CHUNK_KT*512 + 8*32, multiple of 128
+constexpr int CH_MAX_STAGES = 40;
+constexpr int CH_MAX_ITEMS = 16;                   // shrink items per CTA per phase
+constexpr int CH_RED_BYTES = 16 * 1024;            // partial sums of a group of tiles
+constexpr int CH_BS_BYTES = 24 * 1024;             // LoRA-B slices of a group of tiles: [tile][row][j][16] fp16
+constexpr int CH_MAX_GROUP_TILES = 16;
+constexpr long long CH_WAIT_CYCLES = 4000000000ll; // ~2 s at 2 GHz
+
+static_assert(CH_STAGE_BYTES >= CHUNK_KT * 512 + 8 * 32, "stage too small for a chunk");
+
+// ----------------------------------------------------------------------------- shared-memory carve-up
+struct ChainSmem {
+  size_t bars, red, bs, ts, hs, ring, total;
+};
+__host__ __device__ inline ChainSmem chain_carve(int kmax, int rank, int nstages) {
+  ChainSmem s;
+  size_t o = 0;
+  s.bars = o; o += 1024;                                                   // mbarriers
+  s.red = o; o += (size_t)CH_RED_BYTES;                                    // partial sums [tile][slot][lane]
+  s.bs = o; o += (size_t)(rank > 0 ? CH_BS_BYTES : 0);                     // LoRA-B slices of a group
+  s.ts = o; o += (size_t)CHAIN_MAX_ROWS * 3 * (rank > 0 ? rank : 1) * 4;   // T of the phase
+  o = (o + 127) / 128 * 128;
+  s.hs = o; o += (size_t)CHAIN_MAX_ROWS * (kmax + 8) * 2;                  // activations fp16 [8][K+8]
+  o = (o + 127) / 128 * 128;
+  s.ring = o; o += (size_t)nstages * CH_STAGE_BYTES;
+  s.total = o;
+  return s;
+}
+
+size_t chain_smem_bytes(int kmax, int rank, int nstages) { return chain_carve(kmax, rank, nstages).total; }
+
+int chain_pick_stages(int kmax, int rank) {
+  if (rank > CHAIN_MAX_RANK || kmax % TILE_K) return 0;
+  const size_t limit = 227 * 1024 - 2048;        // static shared memory of the kernel comes on top
+  const size_t base = chain_carve(kmax, rank, 0).total;
+  if (base >= limit) return 0;
+  int n = (int)((limit - base) / CH_STAGE_BYTES);
+  if (n > CH_MAX_STAGES) n = CH_MAX_STAGES;
+  if (rank > 0 && CH_BS_BYTES / (CHAIN_MAX_ROWS * rank * 32) < 2) return 0;   // a gate/up pair must fit the B buffer
+  return n >= 8 ? n : 0;
+}
+
+// ----------------------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void cp_async16_ca(void* smem, const void* gmem) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem)), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit_wait_all() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(CH_CTHREADS) : "memory"); }
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void red_release_add_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ uint4 ldg_nc_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+// ----------------------------------------------------------------------------- bounded waits
+struct WaitCtx {
+  volatile int* s_abort;            // shared: this CTA has given up waiting
+  unsigned long long* sync;         // global: [0] barrier, [1] shrink, [2] abort
+  int* status;
+};
+__device__ __noinline__ void raise_abort(const WaitCtx& w) {
+  *w.s_abort = 1;
+  atomicCAS(w.status, 0, MLORA_ERR_TIMEOUT);
+  atomicExch(w.sync + 2, 1ull);
+}
+// mbarrier wait; false when the CTA is (or goes) in abort mode
+__device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const WaitCtx& w) {
+  if (mbar_try_wait(bar, parity)) return true;
+  if (*w.s_abort) return false;
+  const long long t0 = clock64();
+  for (int it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255) == 255) {
+      if (*w.s_abort) return false;
+      if (ld_acquire_u64(w.sync + 2) != 0ull) { *w.s_abort = 1; return false; }
+      if (clock64() - t0 > CH_WAIT_CYCLES) { raise_abort(w); return false; }
+    }
+  }
+}
+// one thread spins until *ctr >= target
+__device__ __forceinline__ void wait_counter(const unsigned long long* ctr, unsigned long long target, const WaitCtx& w) {
+  if (*w.s_abort) return;
+  const long long t0 = clock64();
+  for (int it = 0;; ++it) {
+    if (ld_acquire_u64(ctr) >= target) return;
+    if ((it & 63) == 63) {
+      if (ld_acquire_u64(w.sync + 2) != 0ull) { *w.s_abort = 1; return; }
+      if (clock64() - t0 > CH_WAIT_CYCLES) { raise_abort(w); return; }
+    }
+  }
+}
+
+// physical column -> (segment, logical column)
+__device__ __forceinline__ void chain_map_col(int mode, int c, int n0, int n1, int& seg, int& col) {
+  if (mode == MODE_PLAIN) { seg = 0; col = c; }
+  else if (mode == MODE_QKV) {
+    if (c < n0) { seg = 0; col = c; }
+    else if (c < n0 + n1) { seg = 1; col = c - n0; }
+    else { seg = 2; col = c - n0 - n1; }
+  } else {                         // gate/up interleaved by 16-column tiles
+    const int tile = c >> 4;
+    seg = tile & 1;
+    col = ((tile >> 1) << 4) | (c & 15);
+  }
+}
+
+// ----------------------------------------------------------------------------- optional timeline (trace builds only)
+// With -DCHAIN_TRACE thread 0 of the first and the last CTA stamp the global nanosecond timer at the section
+// boundaries of every phase; mlora_trace_read copies the stamps out.  Compiled out otherwise.
+#ifdef CHAIN_TRACE
+constexpr int TR_PER_PHASE = 64, TR_PHASES = 160;
+__device__ long long g_trace[2 * TR_PHASES * TR_PER_PHASE * 3];
+#define STAMP(id)                                                                                          \
+  do {                                                                                                     \
+    if (tid == 0 && tr_slot >= 0 && tr_n < TR_PER_PHASE && p < TR_PHASES) {                                \
+      long long tns;                                                                                       \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tns));                                              \
+      long long* e = g_trace + (((size_t)tr_slot * TR_PHASES + p) * TR_PER_PHASE + tr_n) * 3;              \
+      e[0] = (id); e[1] = tns; e[2] = clock64(); ++tr_n;                                                   \
+    }                                                                                                      \
+  } while (0)
+#else
+#define STAMP(id) do { } while (0)
+#endif
+
+// ----------------------------------------------------------------------------- the ring schedule
+// Everything immutable that a CTA needs flows through the ring in one fixed order, known to the producer and
+// to the consumers alike.  Per phase:
+//   1. for each shrink item of the CTA (row m, segment, rank index j) whose row has an adapter: the row j of
+//      A in pieces of CH_A_PIECE halves, one stage per piece;
+//   2. for each unit of the CTA, per tile, the weight chunks.
+// The 32-byte slices B[j][16 columns of a tile] of the rows' adapters are too small for bulk copies; the
+// consumer threads fetch them with cp.async into their own buffer at the start of a phase, where the
+// activation prologue hides the latency.
+constexpr int CH_A_PIECE = 2048;                   // halves of an A row per stage
+
+struct Ring {
+  int stage;
+  uint32_t parity;
+  int nstages;
+  __device__ __forceinline__ void advance() { if (++stage == nstages) { stage = 0; parity ^= 1; } }
+};
+
+// ----------------------------------------------------------------------------- the kernel
+__global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const ChainArgs a) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ ChainPhase s_ph[2];
+  __shared__ const __half* s_pA[2][3][CHAIN_MAX_ROWS];
+  __shared__ const __half* s_pB[2][3][CHAIN_MAX_ROWS];
+  __shared__ float s_scale[CHAIN_MAX_ROWS];
+  __shared__ int s_adapter[CHAIN_MAX_ROWS];
+  __shared__ int s_abort_word;
+  __shared__ unsigned long long s_base[2];
+  __shared__ unsigned s_shr_cnt;                      // warps of this CTA that finished their shrink items
+
+  const int nstages = a.nstages;
+  const ChainSmem cs = chain_carve(a.kmax, a.rank, nstages);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + cs.bars);
+  uint64_t* empty_bar = full_bar + CH_MAX_STAGES;
+  float4* red = reinterpret_cast<float4*>(smem + cs.red);
+  __half* Bs = reinterpret_cast<__half*>(smem + cs.bs);
+  float* Ts = reinterpret_cast<float*>(smem + cs.ts);
+  __half* hs = reinterpret_cast<__half*>(smem + cs.hs);
+  unsigned char* ring = smem + cs.ring;
+
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5, lane = tid & 31;
+  const unsigned G = gridDim.x;
+  const int M = a.M;
+  const int r = a.rank;
+  const bool lora_on = a.adapter_idx != nullptr && a.rank > 0;
+  WaitCtx wc{&s_abort_word, a.sync, a.status};
+
+  // ---- set-up: barriers, first phase descriptor, adapters of the rows, counter bases
+  if (tid == 0) {
+    for (int s = 0; s < nstages; ++s) {
+      mbar_init(smem_u32(full_bar + s), 1);
+      mbar_init(smem_u32(empty_bar + s), 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_abort_word = (ld_acquire_u64(a.sync + 2) != 0ull) ? 1 : 0;
+    s_shr_cnt = 0u;
+    // arrivals of earlier launches are whole multiples of the grid size; arrivals of this launch that are
+    // already counted are fewer than one grid
+    s_base[0] = ld_acquire_u64(a.sync + 0) / G * G;
+    s_base[1] = ld_acquire_u64(a.sync + 1) / G * G;
+  }
+  if (tid < CHAIN_MAX_ROWS) {
+    int ad = -1;
+    float sc = 0.f;
+    if (lora_on && tid < M) {
+      ad = a.adapter_idx[tid / a.rows_per_stream];
+      if (ad < 0 || ad >= a.n_slots) ad = -1;
+      else sc = a.scale[ad];
+    }
+    s_adapter[tid] = ad;
+    s_scale[tid] = sc;
+  }
+  __syncthreads();
+
+  // loads phase descriptor p and the rows' adapter pointers into slot (p - p0) & 1 (one warp)
+  auto prep_phase = [&](int p) {
+    const int slot = (p - a.p0) & 1;
+    const int* src = reinterpret_cast<const int*>(a.phases + p);
+    int* dst = reinterpret_cast<int*>(&s_ph[slot]);
+    for (int i = lane; i < (int)(sizeof(ChainPhase) / 4); i += 32) dst[i] = __ldg(src + i);
+    __syncwarp();
+    if (lane < 3 * CHAIN_MAX_ROWS) {
+      const int seg = lane / CHAIN_MAX_ROWS, m = lane % CHAIN_MAX_ROWS;
+      const __half *pa = nullptr, *pb = nullptr;
+      const int ad = s_adapter[m];
+      if (lora_on && seg < s_ph[slot].lora_nseg && ad >= 0) {
+        const size_t e = (size_t)ad * a.tab_stride + s_ph[slot].lora_proj[seg];
+        pa = a.tabA[e];
+        pb = a.tabB[e];
+        if (pa == nullptr || pb == nullptr) { pa = nullptr; pb = nullptr; }
+      }
+      s_pA[slot][seg][m] = pa;
+      s_pB[slot][seg][m] = pb;
+    }
+  };
+  if (warp == 0) prep_phase(a.p0);
+  __syncthreads();
+
+  // =========================================================================== producer warp
+  if (warp == CH_CWARPS) {
+    const uint64_t policy = policy_evict_first();
+    Ring rg{0, 1u, nstages};                         // a fresh "empty" barrier passes a wait on parity 1
+    long long issued = 0;
+    bool alive = true;
+    // lane 0 waits for the stage to be free; every lane learns the outcome
+    auto acquire = [&]() -> bool {
+      int ok = 1;
+      if (lane == 0) ok = wait_mbar(smem_u32(empty_bar + rg.stage), rg.parity, wc) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      return ok != 0;
+    };
+    for (int p = a.p0; p < a.p1 && alive; ++p) {
+      const ChainPhase* ph = a.phases + p;           // immutable: read the descriptor from global
+      const unsigned char* wbase = ph->w;
+      const int mode = ph->mode, K = ph->K;
+      const WLayout L = make_wlayout(K, ph->N, ph->G);
+      const int nseg = lora_on ? ph->lora_nseg : 0;
+      // adapter matrices of the rows for this phase: lane (seg, m)
+      const __half* myA = nullptr;
+      if (nseg > 0 && lane < 3 * CHAIN_MAX_ROWS) {
+        const int seg = lane / CHAIN_MAX_ROWS, m = lane % CHAIN_MAX_ROWS;
+        const int ad = s_adapter[m];
+        if (seg < nseg && ad >= 0) {
+          const size_t e = (size_t)ad * a.tab_stride + ph->lora_proj[seg];
+          myA = a.tabA[e];
+          if (myA == nullptr || a.tabB[e] == nullptr) myA = nullptr;
+        }
+      }
+      // ---- 1. rows of A for the CTA's shrink items
+      if (nseg > 0) {
+        const int n_items = M * nseg * r;
+        int my = 0;
+        for (int i = blockIdx.x; i < n_items && my < CH_MAX_ITEMS && alive; i += G, ++my) {
+          const int j = i % r, seg = (i / r) % nseg, m = i / (r * nseg);
+          const __half* A = reinterpret_cast<const __half*>(
+              __shfl_sync(0xffffffffu, (unsigned long long)myA, seg * CHAIN_MAX_ROWS + m));
+          if (A == nullptr) continue;
+          for (int k0 = 0; k0 < K; k0 += CH_A_PIECE) {
+            if (!acquire()) { alive = false; break; }
+            if (lane == 0) {
+              const uint32_t bytes = (uint32_t)min(CH_A_PIECE, K - k0) * 2;
+              const uint32_t fb = smem_u32(full_bar + rg.stage);
+              mbar_expect_tx(fb, bytes);
+              bulk_g2s(smem_u32(ring + (size_t)rg.stage * CH_STAGE_BYTES), A + (size_t)j * K + k0, bytes, fb, policy);
+            }
+            ++issued;
+            rg.advance();
+          }
+        }
+      }
+      // ---- 2. units: B slices, then weight chunks
+      const int tpu = (mode == MODE_GATEUP) ? 2 : 1;
+      const int n_units = L.NT / tpu;
+      for (int u = blockIdx.x; u < n_units && alive; u += G) {
+        for (int tu = 0; tu < tpu && alive; ++tu) {
+          const unsigned char* unit = wbase + (size_t)(u * tpu + tu) * L.unit_bytes;
+          for (int c = 0; c < L.nchunks; ++c) {
+            if (!acquire()) { alive = false; break; }
+            if (lane == 0) {
+              const uint32_t bytes = (c == L.nchunks - 1) ? L.chunk_last : L.chunk_full;
+              const uint32_t fb = smem_u32(full_bar + rg.stage);
+              mbar_expect_tx(fb, bytes);
+              bulk_g2s(smem_u32(ring + (size_t)rg.stage * CH_STAGE_BYTES), unit + (size_t)c * L.chunk_full, bytes, fb, policy);
+            }
+            ++issued;
+            rg.advance();
+          }
+        }
+      }
+    }
+    if (!alive && lane == 0) {
+      // abort: the copies already issued still land; wait (bounded) for the stages that may be in flight
+      const long long t0 = clock64();
+      const long long inflight = issued < nstages ? issued : nstages;
+      for (long long k = 1; k <= inflight; ++k) {
+        const long long idx = issued - k;            // k-th last stage filled
+        const int st = (int)(idx % nstages);
+        const uint32_t par = (uint32_t)((idx / nstages) & 1);
+        while (!mbar_try_wait(smem_u32(full_bar + st), par)) {
+          if (clock64() - t0 > CH_WAIT_CYCLES) break;
+        }
+      }
+    }
+    return;                                           // consumers use a named barrier; nothing below is for this warp
+  }
+
+  // =========================================================================== consumer warps
+  // The CTA's stages of a phase form one list (see "the ring schedule").  Every warp walks the list; a stage
+  // is waited for, read and released by its owner warp only:
+  //   shrink item k        -> warp k % 8 (all pieces of the row)
+  //   weight chunk ci      -> warp (ci + items) % 8, ci counting the CTA's chunks of the phase; a warp keeps the
+  //                           partial sums of its chunks of one tile in registers and parks them in
+  //                           red[tile][c % 8] -- the epilogue adds the slots in index order
+  //   LoRA-B stages        -> read by the epilogue threads, released by thread 0 afterwards
+  // Tiles are handled in groups of as many as the partial-sum buffer holds; one epilogue pass per group.
+  const int g = lane >> 2, t = lane & 3;
+  Ring rg{0, 0u, nstages};
+  unsigned long long n_bar = 0;                       // barriers passed in this launch
+  unsigned n_shr = 0;                                 // LoRA phases passed in this launch
+  float* redf = reinterpret_cast<float*>(red);
+#ifdef CHAIN_TRACE
+  const int tr_slot = blockIdx.x == 0 ? 0 : (blockIdx.x == G - 1 ? 1 : -1);
+#endif
+  for (int p = a.p0; p < a.p1; ++p) {
+    const int slot = (p - a.p0) & 1;
+    const ChainPhase& ph = s_ph[slot];
+    const int K = ph.K;
+    const int hs_stride = K + 8;
+    const WLayout L = make_wlayout(K, ph.N, ph.G);
+    const int nseg = lora_on ? ph.lora_nseg : 0;
+#ifdef CHAIN_TRACE
+    int tr_n = 0;
+#endif
+    STAMP(0);
+    const int tpu = (ph.mode == MODE_GATEUP) ? 2 : 1;
+    const int n_units = L.NT / tpu;
+    const int ns = L.nchunks < CH_CWARPS ? L.nchunks : CH_CWARPS;    // partial-sum slots per tile
+    int tiles_per_group = CH_RED_BYTES / (ns * 512);
+    if (tiles_per_group > CH_MAX_GROUP_TILES) tiles_per_group = CH_MAX_GROUP_TILES;
+    if (nseg > 0 && tiles_per_group > CH_BS_BYTES / (CHAIN_MAX_ROWS * r * 32)) tiles_per_group = CH_BS_BYTES / (CHAIN_MAX_ROWS * r * 32);
+    const int units_per_group = tiles_per_group / tpu;
+    // LoRA-B slices of the group starting at unit u0 -> Bs[tile][m][j][16]; immutable, so no need to wait for activations
+    auto issue_b = [&](int u0) {
+      const int per_tile = CHAIN_MAX_ROWS * r * 2;                     // 16-byte pieces
+      for (int ug = 0; ug < units_per_group; ++ug) {
+        const int u = u0 + ug * (int)G;
+        if (u >= n_units) break;
+        for (int i = tid; i < tpu * per_tile; i += CH_CTHREADS) {
+          const int tu = i / per_tile, rem = i % per_tile;
+          const int m = rem / (r * 2), j = (rem >> 1) % r, h16 = rem & 1;
+          int seg, col;
+          chain_map_col(ph.mode, (u * tpu + tu) * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
+          const __half* B = (m < M && seg < nseg) ? s_pB[slot][seg][m] : nullptr;
+          if (B != nullptr)
+            cp_async16_ca(Bs + (((size_t)(ug * tpu + tu) * CHAIN_MAX_ROWS + m) * r + j) * 16 + h16 * 8,
+                          B + (size_t)j * ph.lora_n[seg] + col + h16 * 8);
+        }
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    if (nseg > 0 && (int)blockIdx.x < n_units) issue_b(blockIdx.x);
+
+    // ---- 1. activations of the phase -> shared memory, fp16 [8][K+8]
+    if (ph.in_kind == IN_NORM) {
+      // RMSNorm (Sec. 3.1): warp m owns row m; the row was written by other CTAs: read it through L2
+      const int m = warp;
+      if (m < M) {
+        __half* dst = hs + (size_t)m * hs_stride;
+        const float* x = ph.x_f32 + (size_t)m * K;
+        constexpr int NV = 24;                         // rows up to 3072 wide stay in registers: one pass
+        if (K <= NV * 128) {
+          float4 xv[NV];
+          uint2 gv[NV];
+          float ss = 0.f;
+#pragma unroll
+          for (int i = 0; i < NV; ++i) {
+            const int k = lane * 4 + i * 128;
+            xv[i] = (k < K) ? __ldcg(reinterpret_cast<const float4*>(x + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            gv[i] = (k < K) ? __ldg(reinterpret_cast<const uint2*>(ph.gain + k)) : make_uint2(0, 0);
+          }
+#pragma unroll
+          for (int i = 0; i < NV; ++i) ss += xv[i].x * xv[i].x + xv[i].y * xv[i].y + xv[i].z * xv[i].z + xv[i].w * xv[i].w;
+          ss = warp_sum(ss);
+          const float inv = rsqrtf(ss / (float)K + a.eps);
+#pragma unroll
+          for (int i = 0; i < NV; ++i) {
+            const int k = lane * 4 + i * 128;
+            if (k < K) {
+              const float2 g01 = __half22float2(u32_as_h2(gv[i].x)), g23 = __half22float2(u32_as_h2(gv[i].y));
+              const __half2 o01 = __floats2half2_rn(xv[i].x * inv * g01.x, xv[i].y * inv * g01.y);
+              const __half2 o23 = __floats2half2_rn(xv[i].z * inv * g23.x, xv[i].w * inv * g23.y);
+              *reinterpret_cast<uint2*>(dst + k) = make_uint2(h2_as_u32(o01), h2_as_u32(o23));
+            }
+          }
+        } else {
+          float ss = 0.f;
+          for (int k = lane * 4; k < K; k += 128) {
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(x + k));
+            ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+          }
+          ss = warp_sum(ss);
+          const float inv = rsqrtf(ss / (float)K + a.eps);
+          for (int k = lane * 4; k < K; k += 128) {
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(x + k));
+            const uint2 gv = __ldg(reinterpret_cast<const uint2*>(ph.gain + k));
+            const float2 g01 = __half22float2(u32_as_h2(gv.x)), g23 = __half22float2(u32_as_h2(gv.y));
+            const __half2 o01 = __floats2half2_rn(v.x * inv * g01.x, v.y * inv * g01.y);
+            const __half2 o23 = __floats2half2_rn(v.z * inv * g23.x, v.w * inv * g23.y);
+            *reinterpret_cast<uint2*>(dst + k) = make_uint2(h2_as_u32(o01), h2_as_u32(o23));
+          }
+        }
+      }
+    } else {
+      const int vec_per_row = K / 8;
+      const __half* h_in = ph.h_in != nullptr ? ph.h_in : a.h_in;
+      for (int i = tid; i < M * vec_per_row; i += CH_CTHREADS) {
+        const int m = i / vec_per_row, k = (i % vec_per_row) * 8;
+        *reinterpret_cast<uint4*>(hs + (size_t)m * hs_stride + k) =
+            __ldcg(reinterpret_cast<const uint4*>(h_in + (size_t)m * K + k));
+      }
+    }
+    consumer_sync();
+    STAMP(1);
+
+    // ---- 2. next phase's descriptor and adapter pointers (immutable) while this phase runs
+    if (warp == CH_CWARPS - 1 && p + 1 < a.p1) prep_phase(p + 1);
+
+    // ---- 3. LoRA shrink (first factor of the low-rank term of Eq. 1-4): items (row, segment, rank index)
+    // are dealt round-robin to the CTAs; item k of the CTA belongs to warp k % 8
+    int n_my = 0;
+    if (nseg > 0) {
+      const int n_items = M * nseg * r;
+      const int np = (K + CH_A_PIECE - 1) / CH_A_PIECE;
+      for (int i = blockIdx.x; i < n_items && n_my < CH_MAX_ITEMS; i += G, ++n_my) {
+        const int seg = (i / r) % nseg, m = i / (r * nseg);
+        if (s_pA[slot][seg][m] == nullptr) continue;
+        if ((n_my & (CH_CWARPS - 1)) != warp) {
+          for (int q = 0; q < np; ++q) rg.advance();
+          continue;
+        }
+        const __half* hrow = hs + (size_t)m * hs_stride;
+        float acc = 0.f;
+        for (int k0 = 0; k0 < K; k0 += CH_A_PIECE) {
+          const bool ok = wait_mbar(smem_u32(full_bar + rg.stage), rg.parity, wc);
+          const unsigned char* sb = ring + (size_t)rg.stage * CH_STAGE_BYTES;
+          if (ok) {
+#pragma unroll
+            for (int q = 0; q < CH_A_PIECE / 256; ++q) {
+              const int off = q * 256 + lane * 8;            // halves inside the piece
+              if (k0 + off < K) {
+                const uint4 av = *reinterpret_cast<const uint4*>(sb + off * 2);
+                const uint4 hv = *reinterpret_cast<const uint4*>(hrow + k0 + off);
+                const uint32_t aw[4] = {av.x, av.y, av.z, av.w};
+                const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const float2 af = __half22float2(u32_as_h2(aw[e])), hf = __half22float2(u32_as_h2(hw[e]));
+                  acc = fmaf(af.x, hf.x, acc);
+                  acc = fmaf(af.y, hf.y, acc);
+                }
+              }
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(empty_bar + rg.stage));
+          rg.advance();
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) __stcg(a.T + i, acc * s_scale[m]);
+      }
+      // the last warp of the CTA to get here tells the grid that this CTA's share of T is written
+      ++n_shr;
+      if (lane == 0) {
+        __threadfence();
+        const unsigned old = atomicAdd(&s_shr_cnt, 1u);
+        if (old == n_shr * CH_CWARPS - 1) red_release_add_u64(a.sync + 1, 1ull);
+      }
+    }
+    STAMP(2);
+
+    // ---- 4. the CTA's units: one n-tile (or a gate/up pair of n-tiles), all of K
+    bool t_loaded = false;
+    int ci = n_my;                                     // chunk ownership continues after the shrink items
+    for (int u0 = blockIdx.x; u0 < n_units; u0 += G * units_per_group) {
+      int ng = 0;
+      if (nseg > 0 && u0 != (int)blockIdx.x) issue_b(u0);              // the first group's went out before the prologue
+      for (int ug = 0; ug < units_per_group; ++ug) {
+        const int u = u0 + ug * (int)G;
+        if (u >= n_units) break;
+        ++ng;
+        for (int tu = 0; tu < tpu; ++tu) {
+          float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
+          int my_slot = -1;
+          for (int c = 0; c < L.nchunks; ++c, ++ci) {
+            if ((ci & (CH_CWARPS - 1)) == warp) {
+              my_slot = c & (CH_CWARPS - 1);
+              const int kc = (c == L.nchunks - 1) ? L.kc_last : CHUNK_KT;
+              const bool ok = wait_mbar(smem_u32(full_bar + rg.stage), rg.parity, wc);
+              if (ok) {
+                const unsigned char* sb = ring + (size_t)rg.stage * CH_STAGE_BYTES;
+                const __half* hbase = hs + (size_t)g * hs_stride + (size_t)c * CHUNK_KT * TILE_K + 16 * t;
+#pragma unroll
+                for (int kt = 0; kt < CHUNK_KT; ++kt) {
+                  if (kt < kc) {
+                    const uint4 wv = *reinterpret_cast<const uint4*>(sb + kt * 512 + lane * 16);
+                    const int gi = (L.G >= CHUNK_KT * TILE_K) ? 0 : (kt * TILE_K) / L.G;
+                    const uint32_t sw = *reinterpret_cast<const uint32_t*>(sb + kc * 512 + gi * 32 + g * 4);
+                    const uint4 b01 = *reinterpret_cast<const uint4*>(hbase + kt * TILE_K);
+                    const uint4 b23 = *reinterpret_cast<const uint4*>(hbase + kt * TILE_K + 8);
+                    __half2 s_lo, s_hi;
+                    split_scales(sw, s_lo, s_hi);
+                    uint32_t af[4][4];
+                    dequant8(wv.x, s_lo, s_hi, af[0]);
+                    dequant8(wv.y, s_lo, s_hi, af[1]);
+                    dequant8(wv.z, s_lo, s_hi, af[2]);
+                    dequant8(wv.w, s_lo, s_hi, af[3]);
+                    mma_16816(acc0, af[0], b01.x, b01.y);
+                    mma_16816(acc1, af[1], b01.z, b01.w);
+                    mma_16816(acc0, af[2], b23.x, b23.y);
+                    mma_16816(acc1, af[3], b23.z, b23.w);
+                  }
+                }
+              }
+              __syncwarp();
+              if (lane == 0) mbar_arrive(smem_u32(empty_bar + rg.stage));
+            }
+            rg.advance();
+          }
+          if (my_slot >= 0)
+            red[((size_t)(ug * tpu + tu) * ns + my_slot) * 32 + lane] =
+                make_float4(acc0[0] + acc1[0], acc0[1] + acc1[1], acc0[2] + acc1[2], acc0[3] + acc1[3]);
+        }
+      }
+      STAMP(3);
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      consumer_sync();
+      if (nseg > 0 && !t_loaded) {
+        // all of T must be in global memory before the first expand of the phase
+        if (tid == 0) wait_counter(a.sync + 1, s_base[1] + (unsigned long long)n_shr * G, wc);
+        consumer_sync();
+        for (int i = tid; i < M * nseg * r; i += CH_CTHREADS) Ts[i] = __ldcg(a.T + i);
+        consumer_sync();
+        t_loaded = true;
+        STAMP(4);
+      }
+      STAMP(5);
+      // ---- epilogue of the group: one thread per (unit, row, column)
+      for (int o = tid; o < ng * CHAIN_MAX_ROWS * TILE_N; o += CH_CTHREADS) {
+        const int ug = o >> 7, m = (o >> 4) & 7, col16 = o & 15;
+        if (m >= M) continue;
+        const int u = u0 + ug * (int)G;
+        // accumulator layout of m16n8k16: lane (g,t) holds (out g, row 2t), (g, 2t+1), (g+8, 2t), (g+8, 2t+1)
+        const int src_lane = (col16 & 7) * 4 + (m >> 1);
+        const int e = (col16 >> 3) * 2 + (m & 1);
+        float yv[2] = {0.f, 0.f};
+        int colv[2] = {0, 0};
+#pragma unroll
+        for (int tu = 0; tu < 2; ++tu) {
+          if (tu < tpu) {
+            const int nt = u * tpu + tu;
+            const float* rp = redf + ((size_t)(ug * tpu + tu) * ns * 32 + src_lane) * 4 + e;
+            float y = 0.f;
+            for (int sl = 0; sl < ns; ++sl) y += rp[(size_t)sl * 128];
+            int seg, col;
+            chain_map_col(ph.mode, nt * TILE_N + col16, ph.seg_n0, ph.seg_n1, seg, col);
+            if (nseg > 0 && seg < nseg && s_pB[slot][seg][m] != nullptr) {
+              // LoRA expand (second factor of the low-rank term of Eq. 1-4): slice (m, j) sits at slot m*r + j
+              const float* Tm = Ts + ((size_t)m * nseg + seg) * r;
+              const __half* bp = Bs + (((size_t)(ug * tpu + tu) * CHAIN_MAX_ROWS + m) * r) * 16 + col16;
+              float s0 = 0.f, s1 = 0.f;
+              for (int j = 0; j < r; j += 2) {
+                s0 = fmaf(Tm[j], __half2float(bp[(size_t)j * 16]), s0);
+                if (j + 1 < r) s1 = fmaf(Tm[j + 1], __half2float(bp[(size_t)(j + 1) * 16]), s1);
+              }
+              y += s0 + s1;
+            }
+            yv[tu] = y;
+            colv[tu] = col;
+          }
+        }
+        const int nt0 = u * tpu;
+        if (ph.epi == EPI_F32) {
+          float* out = ph.out_f32 != nullptr ? ph.out_f32 : a.logits;
+          __stcg(out + (size_t)m * ph.ldo + nt0 * TILE_N + col16, yv[0]);
+        } else if (ph.epi == EPI_RESID) {
+          float* xp = ph.resid + (size_t)m * ph.N + nt0 * TILE_N + col16;
+          __stcg(xp, __ldcg(xp) + yv[0]);
+        } else {                                       // EPI_SWIGLU: even tile = gate, odd tile = up
+          const float v = yv[0] / (1.f + __expf(-yv[0])) * yv[1];
+          ph.out_f16[(size_t)m * (ph.N / 2) + colv[1]] = __float2half_rn(v);
+        }
+      }
+      consumer_sync();                                 // red and the B stages may be reused
+      STAMP(6);
+    }
+
+    // ---- 5. grid barrier: the next phase reads what every CTA wrote
+    STAMP(7);
+    if (p + 1 < a.p1) {
+      ++n_bar;
+      if (tid == 0) {
+        __threadfence();
+        red_release_add_u64(a.sync + 0, 1ull);
+        wait_counter(a.sync + 0, s_base[0] + n_bar * G, wc);
+        __threadfence();
+      }
+      consumer_sync();
+    }
+    STAMP(8);
+  }
+}
+
+#ifdef CHAIN_TRACE
+extern "C" int mlora_trace_read(long long* host_out, int n_longs) {
+  const size_t total = sizeof(g_trace) / sizeof(long long);
+  const size_t n = (size_t)n_longs < total ? (size_t)n_longs : total;
+  return (int)cudaMemcpyFromSymbol(host_out, g_trace, n * sizeof(long long));
+}
+extern "C" int mlora_trace_clear() {
+  void* p = nullptr;
+  cudaError_t e = cudaGetSymbolAddress(&p, g_trace);
+  if (e != cudaSuccess) return (int)e;
+  return (int)cudaMemset(p, 0, sizeof(g_trace));
+}
+#endif
+
+// ----------------------------------------------------------------------------- host side
+cudaError_t init_chain() {
+  return cudaFuncSetAttribute(decode_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048);
+}
+
+cudaError_t launch_chain(const ChainArgs& a, int sm_count, cudaStream_t st) {
+  if (a.M < 1 || a.M > CHAIN_MAX_ROWS || a.nstages < 2 || a.nstages > CH_MAX_STAGES) return cudaErrorInvalidValue;
+  const size_t smem = chain_smem_bytes(a.kmax, a.rank, a.nstages);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)sm_count);
+  cfg.blockDim = dim3(CH_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;          // all CTAs resident: the grid barrier needs it
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, decode_chain_kernel, a);
+}
+
+}  // namespace mlora

@@ -18,21 +18,18 @@ namespace {
 thread_local std::string g_last_error;
 
 struct PackedWeight {
-  uint4* wq = nullptr;
-  uint32_t* sc = nullptr;
-  int K = 0, N = 0, G = 0;   // N = physical width (all fused segments)
+  unsigned char* data = nullptr;   // chunked fragment-major layout: nibbles and scales interleaved per chunk
+  int K = 0, N = 0, G = 0;         // N = physical width (all fused segments)
 };
 
 cudaError_t alloc_packed(PackedWeight& w, int K, int N, int G) {
   w.K = K; w.N = N; w.G = G;
-  cudaError_t e = cudaMalloc(&w.wq, (size_t)K * N / 2);
-  if (e != cudaSuccess) return e;
-  return cudaMalloc(&w.sc, (size_t)(K / G) * N * sizeof(__half));
+  const WLayout L = make_wlayout(K, N, G);
+  return cudaMalloc(&w.data, (size_t)L.NT * L.unit_bytes);
 }
 void free_packed(PackedWeight& w) {
-  if (w.wq) cudaFree(w.wq);
-  if (w.sc) cudaFree(w.sc);
-  w.wq = nullptr; w.sc = nullptr;
+  if (w.data) cudaFree(w.data);
+  w.data = nullptr;
 }
 
 struct GraphKey {
@@ -55,6 +52,8 @@ struct GraphEntry { cudaGraphExec_t exec; int nodes; };
 struct mlora_weight {
   PackedWeight w;
   cudaStream_t stream;
+  ChainPhase* phase = nullptr;     // dev: descriptor of this projection for the persistent kernel
+  int sm_count = 0;
 };
 
 struct mlora_ctx {
@@ -95,7 +94,12 @@ struct mlora_ctx {
   cudaEvent_t snap_event = nullptr;
   bool snap_pending = false;
   int snap_inc = 0;
-  int dbg_skip_compact = 0, dbg_no_graph = 0;
+  int dbg_skip_compact = 0, dbg_no_graph = 0, dbg_no_chain = 0;
+  // persistent projection chain (rows <= 8)
+  ChainPhase* phases = nullptr;      // dev [4*L (+1)]: qkv, o, gate/up, down per layer; then lm_head
+  int n_phases = 0;
+  unsigned long long* chain_sync = nullptr;   // dev [4]
+  int chain_stages = 0, chain_kmax = 0;
   // graphs
   std::unordered_map<GraphKey, GraphEntry, GraphKeyHash> graphs;
   bool capturing = false;
@@ -182,12 +186,89 @@ void plan_pass(mlora_ctx* c, PassIO& io) {
   attn_plan(a, c->sm_count);
 }
 
-// the launch sequence of one pass over M = n*T rows (Sec. 3.1 decoder, Eq. 1-4 projections)
-int forward(mlora_ctx* c, const PassIO& io) {
+// where a pass writes the K/V of its rows
+void kv_destination(mlora_ctx* c, const PassIO& io, int l, __half*& kd, __half*& vd, size_t& sstride, size_t& hstride) {
+  const int hd = c->d.head_dim;
+  if (io.prefill) {
+    kd = c->prefix_k + (size_t)l * c->prefix_layer_stride + (size_t)io.pos_base * hd;
+    vd = c->prefix_v + (size_t)l * c->prefix_layer_stride + (size_t)io.pos_base * hd;
+    sstride = 0; hstride = c->prefix_head_stride;
+  } else {
+    kd = c->own_k + (size_t)l * c->own_layer_stride;
+    vd = c->own_v + (size_t)l * c->own_layer_stride;
+    sstride = c->own_stream_stride; hstride = c->own_head_stride;
+  }
+}
+
+int launch_attention_block(mlora_ctx* c, const PassIO& io, int l) {
+  const mlora_model_desc& d = c->d;
+  cudaStream_t st = c->stream;
+  const int M = io.n * io.T, hd = d.head_dim;
+  __half *kd, *vd;
+  size_t sstride, hstride;
+  kv_destination(c, io, l, kd, vd, sstride, hstride);
+  CK(run(c, MLORA_PROF_ROPE_KV, [&] {
+    return launch_rope_kv(c->qkv, M, io.T, d.n_q_heads, d.n_kv_heads, hd, c->cs_table, io.pos_base, io.suffix_len,
+                          c->depth, c->q16, kd, vd, sstride, hstride, st);
+  }));
+  AttnArgs a = io.plan;
+  a.q = c->q16;
+  a.prefix_k = c->prefix_k + (size_t)l * c->prefix_layer_stride;
+  a.prefix_v = c->prefix_v + (size_t)l * c->prefix_layer_stride;
+  a.prefix_head_stride = c->prefix_head_stride;
+  a.own_k = kd; a.own_v = vd; a.own_stream_stride = sstride; a.own_head_stride = hstride;
+  a.suffix_len = io.suffix_len; a.anc = c->anc;
+  a.out = c->attn16;
+  if (attn_workspace_floats(a) > c->att_ws_floats) return fail(MLORA_ERR_CAPACITY, "attention scratch too small");
+  a.part_o = c->att_ws;
+  a.part_ml = c->att_ws + (attn_workspace_floats(a) / (a.hd + 2)) * a.hd;
+  CK(run(c, MLORA_PROF_ATTN, [&] { return launch_attention(a, st); }));
+  CK(run(c, MLORA_PROF_ATTN_MERGE, [&] { return launch_attention_merge(a, st); }));
+  return MLORA_OK;
+}
+
+bool chain_eligible(const mlora_ctx* c, const PassIO& io) {
+  return c->chain_stages > 0 && !c->dbg_no_chain && !io.prefill && io.n * io.T <= CHAIN_MAX_ROWS;
+}
+
+// decode-sized pass: the projections of a layer run as one persistent kernel between the attention blocks
+int forward_chain(mlora_ctx* c, const PassIO& io) {
   const mlora_model_desc& d = c->d;
   cudaStream_t st = c->stream;
   const int M = io.n * io.T;
-  const int dm = d.d_model, F = d.d_ffn, hd = d.head_dim;
+  CK(run(c, MLORA_PROF_MISC, [&] { return launch_embed(io.tokens, (const __half*)d.embed, io.hidden_in, c->X, M, d.d_model, d.vocab, c->status, st); }));
+  CK(run(c, MLORA_PROF_MISC, [&] { return launch_tree_prep(io.parent, io.n, io.T, c->anc, c->depth, c->status, st); }));
+  ChainArgs a{};
+  a.phases = c->phases;
+  a.M = M; a.eps = d.rms_eps; a.logits = io.logits;
+  if (io.adapter_idx != nullptr && d.lora_rank > 0 && d.max_adapters > 0 && d.lora_targets != 0) {
+    a.adapter_idx = io.adapter_idx; a.rows_per_stream = io.T;
+    a.tabA = c->tabA; a.tabB = c->tabB; a.scale = c->ad_scale;
+    a.tab_stride = c->L * 7; a.n_slots = d.max_adapters;
+  }
+  a.rank = d.lora_rank;
+  a.T = c->T; a.sync = c->chain_sync; a.status = c->status;
+  a.nstages = c->chain_stages; a.kmax = c->chain_kmax;
+  const int last = 4 * c->L + ((d.vocab > 0 && io.logits != nullptr) ? 1 : 0);
+  a.p0 = 0; a.p1 = 1;
+  CK(run(c, MLORA_PROF_GEMM, [&] { return launch_chain(a, c->sm_count, st); }));
+  for (int l = 0; l < c->L; ++l) {
+    int rc = launch_attention_block(c, io, l);
+    if (rc != MLORA_OK) return rc;
+    a.p0 = 4 * l + 1;
+    a.p1 = (l + 1 < c->L) ? 4 * l + 5 : last;
+    CK(run(c, MLORA_PROF_GEMM, [&] { return launch_chain(a, c->sm_count, st); }));
+  }
+  return MLORA_OK;
+}
+
+// the launch sequence of one pass over M = n*T rows (Sec. 3.1 decoder, Eq. 1-4 projections)
+int forward(mlora_ctx* c, const PassIO& io) {
+  if (chain_eligible(c, io)) return forward_chain(c, io);
+  const mlora_model_desc& d = c->d;
+  cudaStream_t st = c->stream;
+  const int M = io.n * io.T;
+  const int dm = d.d_model, F = d.d_ffn;
   CK(run(c, MLORA_PROF_MISC, [&] { return launch_embed(io.tokens, (const __half*)d.embed, io.hidden_in, c->X, M, dm, d.vocab, c->status, st); }));
   CK(run(c, MLORA_PROF_MISC, [&] { return launch_tree_prep(io.parent, io.n, io.T, c->anc, c->depth, c->status, st); }));
   for (int l = 0; l < c->L; ++l) {
@@ -200,42 +281,16 @@ int forward(mlora_ctx* c, const PassIO& io) {
       CK(run(c, MLORA_PROF_SHRINK, [&] { return launch_shrink(s, st); }));
       GemmArgs g{};
       const PackedWeight& w = c->w_qkv[l];
-      g.wq = w.wq; g.sc = w.sc; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->h; g.M = M;
+      g.w = w.data; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->h; g.M = M;
       g.mode = MODE_QKV; g.epi = EPI_F32; g.seg_n0 = c->Nq; g.seg_n1 = c->Nkv;
       g.out_f32 = c->qkv; g.ldo = c->Nqkv;
       g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
       g.lora = s.lora;
       CK(run(c, MLORA_PROF_GEMM, [&] { return launch_gemm(g, st); }));
     }
-    __half *kd, *vd;
-    size_t sstride, hstride;
-    if (io.prefill) {
-      kd = c->prefix_k + (size_t)l * c->prefix_layer_stride + (size_t)io.pos_base * hd;
-      vd = c->prefix_v + (size_t)l * c->prefix_layer_stride + (size_t)io.pos_base * hd;
-      sstride = 0; hstride = c->prefix_head_stride;
-    } else {
-      kd = c->own_k + (size_t)l * c->own_layer_stride;
-      vd = c->own_v + (size_t)l * c->own_layer_stride;
-      sstride = c->own_stream_stride; hstride = c->own_head_stride;
-    }
-    CK(run(c, MLORA_PROF_ROPE_KV, [&] {
-      return launch_rope_kv(c->qkv, M, io.T, d.n_q_heads, d.n_kv_heads, hd, c->cs_table, io.pos_base, io.suffix_len,
-                            c->depth, c->q16, kd, vd, sstride, hstride, st);
-    }));
     {
-      AttnArgs a = io.plan;
-      a.q = c->q16;
-      a.prefix_k = c->prefix_k + (size_t)l * c->prefix_layer_stride;
-      a.prefix_v = c->prefix_v + (size_t)l * c->prefix_layer_stride;
-      a.prefix_head_stride = c->prefix_head_stride;
-      a.own_k = kd; a.own_v = vd; a.own_stream_stride = sstride; a.own_head_stride = hstride;
-      a.suffix_len = io.suffix_len; a.anc = c->anc;
-      a.out = c->attn16;
-      if (attn_workspace_floats(a) > c->att_ws_floats) return fail(MLORA_ERR_CAPACITY, "attention scratch too small");
-      a.part_o = c->att_ws;
-      a.part_ml = c->att_ws + (attn_workspace_floats(a) / (a.hd + 2)) * a.hd;
-      CK(run(c, MLORA_PROF_ATTN, [&] { return launch_attention(a, st); }));
-      CK(run(c, MLORA_PROF_ATTN_MERGE, [&] { return launch_attention_merge(a, st); }));
+      int rc = launch_attention_block(c, io, l);
+      if (rc != MLORA_OK) return rc;
     }
     {
       const int projs[1] = {3}, widths[1] = {dm};
@@ -247,7 +302,7 @@ int forward(mlora_ctx* c, const PassIO& io) {
       }
       GemmArgs g{};
       const PackedWeight& w = c->w_o[l];
-      g.wq = w.wq; g.sc = w.sc; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->attn16; g.M = M;
+      g.w = w.data; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->attn16; g.M = M;
       g.mode = MODE_PLAIN; g.epi = EPI_RESID; g.resid = c->X;
       g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
       g.lora = la;
@@ -262,7 +317,7 @@ int forward(mlora_ctx* c, const PassIO& io) {
       CK(run(c, MLORA_PROF_SHRINK, [&] { return launch_shrink(s, st); }));
       GemmArgs g{};
       const PackedWeight& w = c->w_gateup[l];
-      g.wq = w.wq; g.sc = w.sc; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->h; g.M = M;
+      g.w = w.data; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->h; g.M = M;
       g.mode = MODE_GATEUP; g.epi = EPI_SWIGLU; g.out_f16 = c->act16;
       g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
       g.lora = s.lora;
@@ -278,7 +333,7 @@ int forward(mlora_ctx* c, const PassIO& io) {
       }
       GemmArgs g{};
       const PackedWeight& w = c->w_down[l];
-      g.wq = w.wq; g.sc = w.sc; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->act16; g.M = M;
+      g.w = w.data; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->act16; g.M = M;
       g.mode = MODE_PLAIN; g.epi = EPI_RESID; g.resid = c->X;
       g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
       g.lora = la;
@@ -291,7 +346,7 @@ int forward(mlora_ctx* c, const PassIO& io) {
     CK(run(c, MLORA_PROF_SHRINK, [&] { return launch_shrink(s, st); }));
     GemmArgs g{};
     const PackedWeight& w = c->w_lm;
-    g.wq = w.wq; g.sc = w.sc; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->h; g.M = M;
+    g.w = w.data; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->h; g.M = M;
     g.mode = MODE_PLAIN; g.epi = EPI_F32; g.out_f32 = io.logits; g.ldo = d.vocab;
     g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
     CK(run(c, MLORA_PROF_GEMM, [&] { return launch_gemm(g, st); }));
@@ -361,6 +416,7 @@ int init_kernels() {
   CK(init_gemm());
   CK(init_shrink());
   CK(init_attention());
+  CK(init_chain());
   done = true;
   return MLORA_OK;
 }
@@ -426,7 +482,8 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
   if (d.vocab > 0 && (!d.embed || !d.rms_final)) return fail(MLORA_ERR_ARG, "vocab > 0 needs embed and rms_final");
   if (d.head_dim != 64 && d.head_dim != 128) return fail(MLORA_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
   if (d.n_q_heads % d.n_kv_heads) return fail(MLORA_ERR_ARG, "n_q_heads must be a multiple of n_kv_heads");
-  if (d.group_size <= 0 || d.group_size % 64) return fail(MLORA_ERR_UNSUPPORTED, "group_size must be a multiple of 64");
+  if (!wlayout_group_ok(d.group_size))
+    return fail(MLORA_ERR_UNSUPPORTED, "group_size must be 64, 128, 256 or a multiple of 512");
   const int Nq = d.n_q_heads * d.head_dim, Nkv = d.n_kv_heads * d.head_dim;
   for (int K : {d.d_model, Nq, d.d_ffn})
     if (K % 64 || K % d.group_size) return fail(MLORA_ERR_UNSUPPORTED, "every input width must be a multiple of 64 and of group_size");
@@ -471,25 +528,24 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
     c->rms_ffn[l] = (const __half*)d.rms_ffn[l];
     PackedWeight& wqkv = c->w_qkv[l];
     CKC(alloc_packed(wqkv, dm, c->Nqkv, G));
-    const int tp = c->Nqkv / 16;
-    CKC(launch_repack((const uint8_t*)qw[0], (const __half*)sc[0], dm, Nq, G, wqkv.wq, wqkv.sc, 0, 1, tp, st));
-    CKC(launch_repack((const uint8_t*)qw[1], (const __half*)sc[1], dm, Nkv, G, wqkv.wq, wqkv.sc, Nq / 16, 1, tp, st));
-    CKC(launch_repack((const uint8_t*)qw[2], (const __half*)sc[2], dm, Nkv, G, wqkv.wq, wqkv.sc, (Nq + Nkv) / 16, 1, tp, st));
+    CKC(launch_repack((const uint8_t*)qw[0], (const __half*)sc[0], dm, Nq, G, wqkv.data, 0, 1, st));
+    CKC(launch_repack((const uint8_t*)qw[1], (const __half*)sc[1], dm, Nkv, G, wqkv.data, Nq / 16, 1, st));
+    CKC(launch_repack((const uint8_t*)qw[2], (const __half*)sc[2], dm, Nkv, G, wqkv.data, (Nq + Nkv) / 16, 1, st));
     CKC(alloc_packed(c->w_o[l], Nq, dm, G));
-    CKC(launch_repack((const uint8_t*)qw[3], (const __half*)sc[3], Nq, dm, G, c->w_o[l].wq, c->w_o[l].sc, 0, 1, dm / 16, st));
+    CKC(launch_repack((const uint8_t*)qw[3], (const __half*)sc[3], Nq, dm, G, c->w_o[l].data, 0, 1, st));
     PackedWeight& wgu = c->w_gateup[l];
     CKC(alloc_packed(wgu, dm, 2 * F, G));
-    CKC(launch_repack((const uint8_t*)qw[4], (const __half*)sc[4], dm, F, G, wgu.wq, wgu.sc, 0, 2, 2 * F / 16, st));
-    CKC(launch_repack((const uint8_t*)qw[5], (const __half*)sc[5], dm, F, G, wgu.wq, wgu.sc, 1, 2, 2 * F / 16, st));
+    CKC(launch_repack((const uint8_t*)qw[4], (const __half*)sc[4], dm, F, G, wgu.data, 0, 2, st));
+    CKC(launch_repack((const uint8_t*)qw[5], (const __half*)sc[5], dm, F, G, wgu.data, 1, 2, st));
     CKC(alloc_packed(c->w_down[l], F, dm, G));
-    CKC(launch_repack((const uint8_t*)qw[6], (const __half*)sc[6], F, dm, G, c->w_down[l].wq, c->w_down[l].sc, 0, 1, dm / 16, st));
+    CKC(launch_repack((const uint8_t*)qw[6], (const __half*)sc[6], F, dm, G, c->w_down[l].data, 0, 1, st));
   }
   if (d.vocab > 0) {
     const void* qw = d.qweight[(size_t)L * 7];
     const void* sc = d.scales[(size_t)L * 7];
     if (!qw || !sc) { fail(MLORA_ERR_ARG, "null lm_head pointer"); mlora_destroy(c); return MLORA_ERR_ARG; }
     CKC(alloc_packed(c->w_lm, dm, d.vocab, G));
-    CKC(launch_repack((const uint8_t*)qw, (const __half*)sc, dm, d.vocab, G, c->w_lm.wq, c->w_lm.sc, 0, 1, d.vocab / 16, st));
+    CKC(launch_repack((const uint8_t*)qw, (const __half*)sc, dm, d.vocab, G, c->w_lm.data, 0, 1, st));
   }
   // ---- KV caches
   c->prefix_head_stride = (size_t)d.max_prefix * hd;
@@ -571,6 +627,55 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
     CKC(cudaMallocHost(&c->stageB, ents * sizeof(void*)));
     CKC(cudaMallocHost(&c->stage_scale, d.max_adapters * sizeof(float)));
   }
+  // ---- phase descriptors of the persistent projection chain
+  {
+    size_t kmax = dm; if ((size_t)F > kmax) kmax = F; if ((size_t)Nq > kmax) kmax = Nq;
+    c->chain_kmax = (int)kmax;
+    c->chain_stages = chain_pick_stages(c->chain_kmax, d.lora_rank);
+    // every CTA must be able to hold its share of the shrink items of a phase
+    if ((CHAIN_MAX_ROWS * 3 * (d.lora_rank > 0 ? d.lora_rank : 1) + c->sm_count - 1) / c->sm_count > 16) c->chain_stages = 0;
+    std::vector<ChainPhase> ph;
+    const int tg = d.lora_rank > 0 && d.max_adapters > 0 ? d.lora_targets : 0;
+    for (int l = 0; l < L; ++l) {
+      ChainPhase q{};
+      q.w = c->w_qkv[l].data; q.K = dm; q.N = c->Nqkv; q.G = G; q.mode = MODE_QKV; q.epi = EPI_F32; q.in_kind = IN_NORM;
+      q.seg_n0 = Nq; q.seg_n1 = Nkv; q.x_f32 = c->X; q.gain = c->rms_attn[l]; q.out_f32 = c->qkv; q.ldo = c->Nqkv;
+      if (tg & (MLORA_Q | MLORA_K | MLORA_V)) {
+        q.lora_nseg = 3;
+        for (int i = 0; i < 3; ++i) q.lora_proj[i] = l * 7 + i;
+        q.lora_n[0] = Nq; q.lora_n[1] = Nkv; q.lora_n[2] = Nkv;
+      }
+      ph.push_back(q);
+      ChainPhase o{};
+      o.w = c->w_o[l].data; o.K = Nq; o.N = dm; o.G = G; o.mode = MODE_PLAIN; o.epi = EPI_RESID; o.in_kind = IN_F16;
+      o.h_in = c->attn16; o.resid = c->X;
+      if (tg & MLORA_O) { o.lora_nseg = 1; o.lora_proj[0] = l * 7 + 3; o.lora_n[0] = dm; }
+      ph.push_back(o);
+      ChainPhase gu{};
+      gu.w = c->w_gateup[l].data; gu.K = dm; gu.N = 2 * F; gu.G = G; gu.mode = MODE_GATEUP; gu.epi = EPI_SWIGLU;
+      gu.in_kind = IN_NORM; gu.x_f32 = c->X; gu.gain = c->rms_ffn[l]; gu.out_f16 = c->act16;
+      if (tg & (MLORA_GATE | MLORA_UP)) {
+        gu.lora_nseg = 2; gu.lora_proj[0] = l * 7 + 4; gu.lora_proj[1] = l * 7 + 5; gu.lora_n[0] = F; gu.lora_n[1] = F;
+      }
+      ph.push_back(gu);
+      ChainPhase dn{};
+      dn.w = c->w_down[l].data; dn.K = F; dn.N = dm; dn.G = G; dn.mode = MODE_PLAIN; dn.epi = EPI_RESID; dn.in_kind = IN_F16;
+      dn.h_in = c->act16; dn.resid = c->X;
+      if (tg & MLORA_DOWN) { dn.lora_nseg = 1; dn.lora_proj[0] = l * 7 + 6; dn.lora_n[0] = dm; }
+      ph.push_back(dn);
+    }
+    if (d.vocab > 0) {
+      ChainPhase lm{};
+      lm.w = c->w_lm.data; lm.K = dm; lm.N = d.vocab; lm.G = G; lm.mode = MODE_PLAIN; lm.epi = EPI_F32; lm.in_kind = IN_NORM;
+      lm.x_f32 = c->X; lm.gain = (const __half*)d.rms_final; lm.out_f32 = nullptr; lm.ldo = d.vocab;
+      ph.push_back(lm);
+    }
+    c->n_phases = (int)ph.size();
+    CKC(cudaMalloc(&c->phases, ph.size() * sizeof(ChainPhase)));
+    CKC(cudaMemcpy(c->phases, ph.data(), ph.size() * sizeof(ChainPhase), cudaMemcpyHostToDevice));
+    CKC(cudaMalloc(&c->chain_sync, 4 * sizeof(unsigned long long)));
+    CKC(cudaMemsetAsync(c->chain_sync, 0, 4 * sizeof(unsigned long long), st));
+  }
   CKC(cudaMallocHost(&c->snap, d.max_streams * sizeof(int32_t)));
   CKC(cudaEventCreateWithFlags(&c->snap_event, cudaEventDisableTiming));
   CKC(cudaStreamSynchronize(st));
@@ -591,7 +696,7 @@ int mlora_destroy(mlora_ctx* c) {
   void* dev_ptrs[] = {c->prefix_k, c->prefix_v, c->own_k, c->own_v, c->X, c->qkv, c->logits, c->T, c->partial, c->att_ws,
                       c->h, c->q16, c->attn16, c->act16, c->counters, c->anc, c->depth, c->argmax, c->suffix_len,
                       c->zero_len, c->chain_parent, c->root_parent, c->status, c->cs_table, (void*)c->tabA,
-                      (void*)c->tabB, c->ad_scale};
+                      (void*)c->tabB, c->ad_scale, c->phases, c->chain_sync};
   for (void* p : dev_ptrs) if (p) cudaFree(p);
   if (c->stageA) cudaFreeHost((void*)c->stageA);
   if (c->stageB) cudaFreeHost((void*)c->stageB);
@@ -615,6 +720,9 @@ int mlora_set_adapter(mlora_ctx* c, int32_t slot, const void* const* A, const vo
   for (size_t i = 0; A != nullptr && i < per; ++i)
     if ((c->d.lora_targets & (1 << (int)(i % 7))) && (A[i] == nullptr || B[i] == nullptr))
       return fail(MLORA_ERR_ARG, "null adapter tensor for a targeted projection");
+  for (size_t i = 0; A != nullptr && i < per; ++i)
+    if ((c->d.lora_targets & (1 << (int)(i % 7))) && (((uintptr_t)A[i] | (uintptr_t)B[i]) & 15))
+      return fail(MLORA_ERR_ARG, "adapter tensors must be 16-byte aligned");
   for (size_t i = 0; i < per; ++i) {
     const int p = (int)(i % 7);
     const bool on = A != nullptr && (c->d.lora_targets & (1 << p));
@@ -654,7 +762,7 @@ static int decode_impl(mlora_ctx* c, int n, const int32_t* adapter_idx, const in
   key.kind = hidden ? 2 : 1; key.n = n; key.T = 1;
   key.prefix_chunk = io.plan.prefix_chunk; key.n_prefix_chunks = io.plan.n_prefix_chunks;
   key.own_chunk = io.plan.own_chunk; key.n_own_chunks = io.plan.n_own_chunks;
-  key.flags = c->P;
+  key.flags = c->P * 2 + c->dbg_no_chain;
   key.p[0] = adapter_idx; key.p[1] = tokens; key.p[2] = hidden; key.p[3] = out_next; key.p[4] = out_logits; key.p[5] = hidden_out;
   rc = replay_or_run(c, key, [&]() -> int {
     int r = forward(c, io);
@@ -708,7 +816,7 @@ int mlora_verify_tree(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_id
   key.kind = 3; key.n = n; key.T = T;
   key.prefix_chunk = io.plan.prefix_chunk; key.n_prefix_chunks = io.plan.n_prefix_chunks;
   key.own_chunk = io.plan.own_chunk; key.n_own_chunks = io.plan.n_own_chunks;
-  key.flags = c->P * 2 + c->dbg_skip_compact;
+  key.flags = c->P * 4 + c->dbg_skip_compact * 2 + c->dbg_no_chain;
   key.p[0] = adapter_idx; key.p[1] = tree_tokens; key.p[2] = tree_parent; key.p[3] = out_accept_len;
   key.p[4] = out_accept_idx; key.p[5] = out_next; key.p[6] = out_logits;
   rc = replay_or_run(c, key, [&]() -> int {
@@ -756,7 +864,10 @@ int mlora_sync_status(mlora_ctx* c) {
   CK(cudaMemcpy(&st, c->status, sizeof(int), cudaMemcpyDeviceToHost));
   if (st != 0) {
     CK(cudaMemset(c->status, 0, sizeof(int)));
-    return fail(st, "device status: malformed tree or token id out of range");
+    // a wait that ran out leaves the barrier counters of the persistent kernel mid-count: start them afresh
+    CK(cudaMemset(c->chain_sync, 0, 4 * sizeof(unsigned long long)));
+    return fail(st, st == MLORA_ERR_TIMEOUT ? "device status: a bounded wait ran out"
+                                            : "device status: malformed tree or token id out of range");
   }
   return MLORA_OK;
 }
@@ -813,7 +924,7 @@ int mlora_debug_dequant(mlora_ctx* c, int32_t layer, int32_t proj, void* out_fp1
       default: w = &c->w_down[layer]; N = c->d.d_model; break;
     }
   } else return fail(MLORA_ERR_ARG, "debug_dequant: no such projection");
-  CK(launch_dequant(w->wq, w->sc, w->K, N, w->G, off, stride, w->N / 16, (__half*)out_fp16, c->stream));
+  CK(launch_dequant(w->data, w->K, N, w->G, off, stride, (__half*)out_fp16, c->stream));
   c->launches++;
   return MLORA_OK;
 }
@@ -822,6 +933,7 @@ int mlora_debug_set(mlora_ctx* c, int32_t key, int32_t value) {
   if (check_ctx(c)) return MLORA_ERR_ARG;
   if (key == 1) c->dbg_skip_compact = value ? 1 : 0;
   else if (key == 2) c->dbg_no_graph = value ? 1 : 0;
+  else if (key == 3) c->dbg_no_chain = value ? 1 : 0;
   else return fail(MLORA_ERR_ARG, "unknown debug key");
   return MLORA_OK;
 }
@@ -857,13 +969,31 @@ int mlora_weight_create(const void* qweight, const void* scales, int32_t K, int3
                         mlora_weight** out) {
   if (!qweight || !scales || !out) return fail(MLORA_ERR_ARG, "null argument");
   if (init_kernels() != MLORA_OK) return MLORA_ERR_CUDA;
-  if (K <= 0 || N <= 0 || G <= 0 || K % 64 || N % 16 || G % 64 || K % G) return fail(MLORA_ERR_UNSUPPORTED, "need K%64==0, N%16==0, G%64==0, K%G==0");
+  if (K <= 0 || N <= 0 || G <= 0 || K % 64 || N % 16 || K % G || !wlayout_group_ok(G))
+    return fail(MLORA_ERR_UNSUPPORTED, "need K%64==0, N%16==0, K%G==0, G in {64,128,256} or a multiple of 512");
   mlora_weight* w = new mlora_weight();
   w->stream = (cudaStream_t)cuda_stream;
   cudaError_t e = alloc_packed(w->w, K, N, G);
-  if (e == cudaSuccess) e = launch_repack((const uint8_t*)qweight, (const __half*)scales, K, N, G, w->w.wq, w->w.sc, 0, 1, N / 16, w->stream);
+  if (e == cudaSuccess) e = launch_repack((const uint8_t*)qweight, (const __half*)scales, K, N, G, w->w.data, 0, 1, w->stream);
+  if (e == cudaSuccess) {
+    int dev = 0;
+    e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&w->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  }
+  if (e == cudaSuccess) e = cudaMalloc(&w->phase, sizeof(ChainPhase));
+  if (e == cudaSuccess) {
+    ChainPhase ph{};                    // input and output pointers come with each call
+    ph.w = w->w.data; ph.K = K; ph.N = N; ph.G = G; ph.mode = MODE_PLAIN; ph.epi = EPI_F32; ph.in_kind = IN_F16;
+    ph.ldo = N; ph.lora_nseg = 1; ph.lora_proj[0] = 0; ph.lora_n[0] = N;
+    e = cudaMemcpy(w->phase, &ph, sizeof(ph), cudaMemcpyHostToDevice);
+  }
   if (e == cudaSuccess) e = cudaStreamSynchronize(w->stream);
-  if (e != cudaSuccess) { free_packed(w->w); delete w; return fail(MLORA_ERR_CUDA, cudaGetErrorString(e)); }
+  if (e != cudaSuccess) {
+    free_packed(w->w);
+    if (w->phase) cudaFree(w->phase);
+    delete w;
+    return fail(MLORA_ERR_CUDA, cudaGetErrorString(e));
+  }
   *out = w;
   return MLORA_OK;
 }
@@ -872,17 +1002,20 @@ int mlora_weight_destroy(mlora_weight* w) {
   if (!w) return MLORA_OK;
   cudaStreamSynchronize(w->stream);
   free_packed(w->w);
+  if (w->phase) cudaFree(w->phase);
   delete w;
   return MLORA_OK;
 }
 
 int mlora_weight_dequant(mlora_weight* w, void* out_fp16) {
   if (!w || !out_fp16) return fail(MLORA_ERR_ARG, "null argument");
-  CK(launch_dequant(w->w.wq, w->w.sc, w->w.K, w->w.N, w->w.G, 0, 1, w->w.N / 16, (__half*)out_fp16, w->stream));
+  CK(launch_dequant(w->w.data, w->w.K, w->w.N, w->w.G, 0, 1, (__half*)out_fp16, w->stream));
   return MLORA_OK;
 }
 
-static const size_t LIN_COUNTER_BYTES = 4096 * sizeof(unsigned);
+// workspace head: 64 bytes of barrier words for the persistent kernel, then the split-K arrival counters
+static const size_t LIN_SYNC_BYTES = 64;
+static const size_t LIN_COUNTER_BYTES = 16640;
 static size_t lin_T_bytes(int M, int rank) { return (((size_t)M * (rank > 0 ? rank : 1) * sizeof(float)) + 255) / 256 * 256; }
 
 size_t mlora_linear_workspace_bytes(const mlora_weight* w, int32_t M, int32_t rank) {
@@ -903,6 +1036,26 @@ int mlora_linear(mlora_weight* w, const void* x, int32_t M, const int32_t* row_a
   const int m_blocks = (M + GEMM_MAX_MT * 8 - 1) / (GEMM_MAX_MT * 8);
   if ((size_t)((w->w.N + GEMM_NB - 1) / GEMM_NB) * m_blocks > 4096) return fail(MLORA_ERR_UNSUPPORTED, "too many output blocks");
   unsigned char* ws = (unsigned char*)workspace;
+  if (M <= CHAIN_MAX_ROWS) {
+    // few rows: one persistent kernel does shrink, GEMM and expand
+    const int stages = chain_pick_stages(w->w.K, lora ? rank : 0);
+    const bool items_fit = !lora || (CHAIN_MAX_ROWS * rank + w->sm_count - 1) / w->sm_count <= 16;
+    if (stages > 0 && items_fit) {
+      ChainArgs a{};
+      a.phases = w->phase; a.p0 = 0; a.p1 = 1; a.M = M; a.logits = y; a.h_in = (const __half*)x;
+      if (lora) {
+        a.adapter_idx = row_adapter; a.rows_per_stream = 1;
+        a.tabA = (const __half* const*)A; a.tabB = (const __half* const*)B; a.scale = scale;
+        a.tab_stride = 1; a.n_slots = n_adapters; a.rank = rank;
+      }
+      a.T = (float*)(ws + LIN_COUNTER_BYTES);
+      a.sync = (unsigned long long*)ws;
+      a.status = (int*)(ws + 32);
+      a.nstages = stages; a.kmax = w->w.K;
+      CK(launch_chain(a, w->sm_count, w->stream));
+      return MLORA_OK;
+    }
+  }
   LoraArgs la{};
   if (lora) {
     la.adapter_idx = row_adapter; la.rows_per_stream = 1;
@@ -915,10 +1068,10 @@ int mlora_linear(mlora_weight* w, const void* x, int32_t M, const int32_t* row_a
     CK(launch_shrink(s, w->stream));
   }
   GemmArgs g{};
-  g.wq = w->w.wq; g.sc = w->w.sc; g.K = w->w.K; g.N = w->w.N; g.G = w->w.G; g.h = (const __half*)x; g.M = M;
+  g.w = w->w.data; g.K = w->w.K; g.N = w->w.N; g.G = w->w.G; g.h = (const __half*)x; g.M = M;
   g.mode = MODE_PLAIN; g.epi = EPI_F32; g.out_f32 = y; g.ldo = w->w.N;
   g.partial = (float*)(ws + fixed); g.partial_capacity = (workspace_bytes - fixed) / sizeof(float);
-  g.counters = (unsigned*)ws;
+  g.counters = (unsigned*)(ws + LIN_SYNC_BYTES);
   g.lora = la;
   CK(launch_gemm(g, w->stream));
   return MLORA_OK;

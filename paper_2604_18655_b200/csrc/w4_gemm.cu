@@ -10,10 +10,10 @@ namespace mlora {
 
 // ----------------------------------------------------------------------------- repack (create time)
 // One thread per (tile, lane): builds the lane's 16 bytes from the canonical nibbles.
-__global__ void repack_kernel(const uint8_t* __restrict__ qw, const __half* __restrict__ scales, int K, int N, int G,
-                              uint4* __restrict__ wq, uint32_t* __restrict__ sc, int tile_off, int tile_stride,
-                              int tiles_phys) {
-  const int KT = K / TILE_K, NT = N / TILE_N;
+__global__ void repack_kernel(const uint8_t* __restrict__ qw, const __half* __restrict__ scales, const WLayout L,
+                              unsigned char* __restrict__ w, int tile_off, int tile_stride) {
+  const int K = L.K, N = L.N, G = L.G;
+  const int KT = L.KT, NT = L.NT;
   const long long total = (long long)NT * KT * 32;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
@@ -24,7 +24,7 @@ __global__ void repack_kernel(const uint8_t* __restrict__ qw, const __half* __re
     uint32_t words[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      uint32_t w = 0;
+      uint32_t wd = 0;
 #pragma unroll
       for (int nib = 0; nib < 8; ++nib) {
         const int a = nib & 3, hi = nib >> 2;
@@ -32,14 +32,15 @@ __global__ void repack_kernel(const uint8_t* __restrict__ qw, const __half* __re
         const int k = kt * TILE_K + 16 * t + 4 * j + 2 * (a >> 1) + hi;
         const uint8_t byte = qw[(size_t)k * (N / 2) + (n >> 1)];
         const uint32_t u = (n & 1) ? (byte >> 4) : (byte & 0xF);
-        w |= u << (4 * nib);
+        wd |= u << (4 * nib);
       }
-      words[j] = w;
+      words[j] = wd;
     }
     const int pt = tile_off + nt * tile_stride;
-    wq[((size_t)pt * KT + kt) * 32 + lane] = make_uint4(words[0], words[1], words[2], words[3]);
+    unsigned char* unit = w + (size_t)pt * L.unit_bytes;
+    *reinterpret_cast<uint4*>(unit + wl_tile_off(L, kt) + lane * 16) = make_uint4(words[0], words[1], words[2], words[3]);
   }
-  // scales
+  // scales: one entry per (n-tile, group, g); a group lies inside one chunk
   const int KG = K / G;
   const long long stotal = (long long)KG * NT * 8;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < stotal;
@@ -51,24 +52,31 @@ __global__ void repack_kernel(const uint8_t* __restrict__ qw, const __half* __re
     const __half hi = scales[(size_t)kg * N + nt * TILE_N + g + 8];
     const uint32_t v = (uint32_t)__half_as_ushort(lo) | ((uint32_t)__half_as_ushort(hi) << 16);
     const int pt = tile_off + nt * tile_stride;
-    sc[((size_t)kg * tiles_phys + pt) * 8 + g] = v;
+    unsigned char* unit = w + (size_t)pt * L.unit_bytes;
+    // every chunk the group covers gets a copy (a group longer than a chunk spans several chunks)
+    const int kt_first = (kg * G) / TILE_K, kt_last = ((kg + 1) * G) / TILE_K - 1;
+    for (int c = kt_first / CHUNK_KT; c <= kt_last / CHUNK_KT; ++c) {
+      const int kt = max(kt_first, c * CHUNK_KT);
+      *reinterpret_cast<uint32_t*>(unit + wl_scale_off(L, kt) + g * 4) = v;
+    }
   }
 }
 
-cudaError_t launch_repack(const uint8_t* qweight, const __half* scales, int K, int N, int G, uint4* wq,
-                          uint32_t* sc, int dst_tile_off, int dst_tile_stride, int dst_tiles, cudaStream_t st) {
-  const long long total = (long long)(N / TILE_N) * (K / TILE_K) * 32;
+cudaError_t launch_repack(const uint8_t* qweight, const __half* scales, int K, int N, int G, unsigned char* w,
+                          int dst_tile_off, int dst_tile_stride, cudaStream_t st) {
+  const WLayout L = make_wlayout(K, N, G);
+  const long long total = (long long)L.NT * L.KT * 32;
   int blocks = (int)((total + 255) / 256);
   if (blocks > 148 * 16) blocks = 148 * 16;
-  repack_kernel<<<blocks, 256, 0, st>>>(qweight, scales, K, N, G, wq, sc, dst_tile_off, dst_tile_stride, dst_tiles);
+  repack_kernel<<<blocks, 256, 0, st>>>(qweight, scales, L, w, dst_tile_off, dst_tile_stride);
   return cudaGetLastError();
 }
 
 // ----------------------------------------------------------------------------- dequant through the GEMM's unpack path
 // One warp per tile: same loads, same dequant8() as the GEMM; writes fp16 [K][N] of the logical matrix.
-__global__ void dequant_kernel(const uint4* __restrict__ wq, const uint32_t* __restrict__ sc, int K, int N, int G,
-                               int tile_off, int tile_stride, int tiles_phys, __half* __restrict__ out) {
-  const int KT = K / TILE_K, NT = N / TILE_N;
+__global__ void dequant_kernel(const unsigned char* __restrict__ w, const WLayout L, int tile_off, int tile_stride,
+                               __half* __restrict__ out) {
+  const int KT = L.KT, NT = L.NT, N = L.N;
   const int lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
   const long long warps = (long long)gridDim.x * (blockDim.x >> 5);
@@ -76,12 +84,12 @@ __global__ void dequant_kernel(const uint4* __restrict__ wq, const uint32_t* __r
        tile += warps) {
     const int kt = (int)(tile % KT), nt = (int)(tile / KT);
     const int pt = tile_off + nt * tile_stride;
-    const uint4 w = ldg_stream(wq + ((size_t)pt * KT + kt) * 32 + lane);
-    const int kg = (kt * TILE_K) / G;
-    const uint32_t sw = ldg_nc_u32(sc + ((size_t)kg * tiles_phys + pt) * 8 + g);
+    const unsigned char* unit = w + (size_t)pt * L.unit_bytes;
+    const uint4 wv = ldg_stream(reinterpret_cast<const uint4*>(unit + wl_tile_off(L, kt)) + lane);
+    const uint32_t sw = ldg_nc_u32(reinterpret_cast<const uint32_t*>(unit + wl_scale_off(L, kt)) + g);
     __half2 s_lo, s_hi;
     split_scales(sw, s_lo, s_hi);
-    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+    const uint32_t words[4] = {wv.x, wv.y, wv.z, wv.w};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       uint32_t a[4];
@@ -101,12 +109,14 @@ __global__ void dequant_kernel(const uint4* __restrict__ wq, const uint32_t* __r
   }
 }
 
-cudaError_t launch_dequant(const uint4* wq, const uint32_t* sc, int K, int N, int G, int tile_off, int tile_stride,
-                           int tiles_phys, __half* out, cudaStream_t st) {
-  const long long tiles = (long long)(N / TILE_N) * (K / TILE_K);
+// K, N: logical shape of the projection being written out; the physical matrix may hold other projections too
+cudaError_t launch_dequant(const unsigned char* w, int K, int N, int G, int tile_off, int tile_stride, __half* out,
+                           cudaStream_t st) {
+  const WLayout L = make_wlayout(K, N, G);
+  const long long tiles = (long long)L.NT * L.KT;
   int blocks = (int)((tiles + 7) / 8);
   if (blocks > 148 * 8) blocks = 148 * 8;
-  dequant_kernel<<<blocks, 256, 0, st>>>(wq, sc, K, N, G, tile_off, tile_stride, tiles_phys, out);
+  dequant_kernel<<<blocks, 256, 0, st>>>(w, L, tile_off, tile_stride, out);
   return cudaGetLastError();
 }
 
@@ -160,16 +170,17 @@ __global__ void __launch_bounds__(GEMM_THREADS) w4_gemm_kernel(const GemmArgs p,
   for (int i = 0; i < MT; ++i) { acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f; }
 
   // weight / scale prefetch ring (independent of the activations)
-  const uint4* wp = p.wq + ((size_t)(active ? nt : 0) * KT + kt_begin) * 32 + lane;
-  const uint32_t* sp = p.sc + (size_t)(active ? nt : 0) * 8 + g;
-  const size_t sc_group_stride = (size_t)NTILES * 8;
+  const WLayout L = make_wlayout(p.K, p.N, p.G);
+  const unsigned char* unit = p.w + (size_t)(active ? nt : 0) * L.unit_bytes;
+  auto w_at = [&](int kt) { return ldg_stream(reinterpret_cast<const uint4*>(unit + wl_tile_off(L, kt)) + lane); };
+  auto s_at = [&](int kt) { return ldg_nc_u32(reinterpret_cast<const uint32_t*>(unit + wl_scale_off(L, kt)) + g); };
   uint4 wr[GEMM_PF];
   uint32_t sr[GEMM_PF];
 #pragma unroll
   for (int i = 0; i < GEMM_PF; ++i) {
     if (active && i < nk) {
-      wr[i] = ldg_stream(wp + (size_t)i * 32);
-      sr[i] = ldg_nc_u32(sp + (size_t)(((kt_begin + i) * TILE_K) / p.G) * sc_group_stride);
+      wr[i] = w_at(kt_begin + i);
+      sr[i] = s_at(kt_begin + i);
     } else {
       wr[i] = make_uint4(0, 0, 0, 0);
       sr[i] = 0;
@@ -201,8 +212,8 @@ __global__ void __launch_bounds__(GEMM_THREADS) w4_gemm_kernel(const GemmArgs p,
           split_scales(sr[i], s_lo, s_hi);
           const int nxt = k0 + i + GEMM_PF;
           if (nxt < nk) {
-            wr[i] = ldg_stream(wp + (size_t)nxt * 32);
-            sr[i] = ldg_nc_u32(sp + (size_t)(((kt_begin + nxt) * TILE_K) / p.G) * sc_group_stride);
+            wr[i] = w_at(kt_begin + nxt);
+            sr[i] = s_at(kt_begin + nxt);
           }
           uint32_t a[4][4];
           dequant8(w.x, s_lo, s_hi, a[0]);
