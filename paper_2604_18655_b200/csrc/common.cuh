@@ -171,6 +171,8 @@ cudaError_t init_chain();
 // shared memory the chain kernel needs for the given largest K and rank with `nstages` ring stages; 0 if it cannot fit
 size_t chain_smem_bytes(int kmax, int rank, int nstages);
 int chain_pick_stages(int kmax, int rank);      // most stages that fit (0: not eligible)
+// whether one projection group (K inputs, nseg LoRA segments) can run in the chain kernel with that many stages
+bool chain_phase_fits(int K, int mode, int nseg, int rank, int nstages, int sm_count);
 cudaError_t launch_chain(const ChainArgs& a, int sm_count, cudaStream_t st);
 
 // ----------------------------------------------------------------------------- launchers

@@ -4,38 +4,44 @@
 //
 // Why: at these sizes a projection moves a few MB -- about a microsecond of HBM time -- so a kernel per
 // projection is bound by launch and ramp-up latency.  Here a producer warp streams the CTA's share of the
-// packed INT4 weights of ALL phases through a shared-memory ring with bulk asynchronous copies
-// (cp.async.bulk + mbarrier transaction counts).  Weights do not depend on activations, so the ring keeps
-// filling while the consumer warps sit in a grid barrier or in a prologue: HBM never idles across phase
-// boundaries.  Eight consumer warps split K inside a chunk, dequantise in registers and multiply on the tensor
-// cores (mma.sync m16n8k16: weights are the 16-wide operand, the rows the 8-wide one), reduce across warps in
-// shared memory in a fixed order, and run the epilogue (LoRA expand, residual add, SwiGLU, fp32 store).
+// packed INT4 weights (and of the LoRA-A rows) of ALL phases through a shared-memory ring with bulk
+// asynchronous copies (cp.async.bulk + mbarrier transaction counts).  They do not depend on activations, so
+// the ring keeps filling while the consumer warps sit in a grid barrier or in a prologue: HBM never idles
+// across phase boundaries.  Sixteen consumer warps (four per scheduler, to hide latency) work in teams: a team
+// takes one n-tile (or gate/up pair) at a time, its warps split K, dequantise in registers and multiply on the
+// tensor cores (mma.sync m16n8k16: weights are the 16-wide operand, the rows the 8-wide one), add their
+// partial sums through shared memory in a fixed order and run the epilogue (LoRA expand, residual add, SwiGLU,
+// fp32 store) on their own, behind a named barrier of the team.
 //
-// The LoRA shrink T = (alpha/r) h A^T is spread over all CTAs at the start of a phase (the rows of A come
-// through the same ring, so they are already in shared memory when the phase starts); a counter tells every
-// CTA when all of T is in global memory; the expand happens in the epilogue from slices of B that also came
-// through the ring.
+// The LoRA shrink T = (alpha/r) h A^T is spread over all CTAs at the start of a phase; a counter tells every
+// CTA when all of T is in global memory; the expand happens in the epilogue from 32-byte slices of B that the
+// team fetched with cp.async before the phase's prologue.
 //
 // Every wait (mbarrier, grid barrier, shrink counter) is bounded by a clock limit.  When one runs out the CTA
-// raises a global abort flag and the status word MLORA_ERR_TIMEOUT; from then on every wait returns at once
-// and the kernel runs its (data-independent) control flow to the end, so no CTA is left in a barrier.
+// raises a global abort flag and the status word MLORA_ERR_TIMEOUT and records which wait it was; from then on
+// every wait returns at once and the kernel runs its (data-independent) control flow to the end, so no CTA is
+// left in a barrier.
 #include "../../include/mlora.h"
 #include "common.cuh"
 
 namespace mlora {
 
-constexpr int CH_CWARPS = 8;                       // consumer warps
+constexpr int CH_CWARPS = 16;                      // consumer warps
 constexpr int CH_CTHREADS = CH_CWARPS * 32;
 constexpr int CH_THREADS = CH_CTHREADS + 32;       // + one producer warp
 constexpr int CH_STAGE_BYTES = 4480;               // >= CHUNK_KT*512 + 8*32, multiple of 128
 constexpr int CH_MAX_STAGES = 40;
 constexpr int CH_MAX_ITEMS = 16;                   // shrink items per CTA per phase
-constexpr int CH_RED_BYTES = 16 * 1024;            // partial sums of a group of tiles
-constexpr int CH_BS_BYTES = 24 * 1024;             // LoRA-B slices of a group of tiles: [tile][row][j][16] fp16
-constexpr int CH_MAX_GROUP_TILES = 16;
+constexpr int CH_ITEM_KT = 2;                      // k-tiles per GEMM work item
+constexpr int CH_ITEMS_PER_CHUNK = CHUNK_KT / CH_ITEM_KT;   // = arrivals that free a ring stage
+constexpr int CH_A_PIECE = 2048;                   // halves of a LoRA-A row per ring stage
+constexpr int CH_RED_BYTES = 2 * CH_CWARPS * 512;  // partial sums: one slot per consumer warp and tile of a pair
+constexpr int CH_BS_BYTES = 24 * 1024;             // LoRA-B slices of the teams' units: [team][tile][row][j][16] fp16
+constexpr int CH_MAX_TEAMS = 8;
 constexpr long long CH_WAIT_CYCLES = 4000000000ll; // ~2 s at 2 GHz
 
 static_assert(CH_STAGE_BYTES >= CHUNK_KT * 512 + 8 * 32, "stage too small for a chunk");
+static_assert(CH_STAGE_BYTES >= CH_A_PIECE * 2, "stage too small for an A piece");
 
 // ----------------------------------------------------------------------------- shared-memory carve-up
 struct ChainSmem {
@@ -45,8 +51,8 @@ __host__ __device__ inline ChainSmem chain_carve(int kmax, int rank, int nstages
   ChainSmem s;
   size_t o = 0;
   s.bars = o; o += 1024;                                                   // mbarriers
-  s.red = o; o += (size_t)CH_RED_BYTES;                                    // partial sums [tile][slot][lane]
-  s.bs = o; o += (size_t)(rank > 0 ? CH_BS_BYTES : 0);                     // LoRA-B slices of a group
+  s.red = o; o += (size_t)CH_RED_BYTES;                                    // partial sums [tile of pair][warp][lane]
+  s.bs = o; o += (size_t)(rank > 0 ? CH_BS_BYTES : 0);                     // LoRA-B slices
   s.ts = o; o += (size_t)CHAIN_MAX_ROWS * 3 * (rank > 0 ? rank : 1) * 4;   // T of the phase
   o = (o + 127) / 128 * 128;
   s.hs = o; o += (size_t)CHAIN_MAX_ROWS * (kmax + 8) * 2;                  // activations fp16 [8][K+8]
@@ -54,6 +60,21 @@ __host__ __device__ inline ChainSmem chain_carve(int kmax, int rank, int nstages
   s.ring = o; o += (size_t)nstages * CH_STAGE_BYTES;
   s.total = o;
   return s;
+}
+
+// A consumer may never wait a whole ring lap ahead of the fill front (mbarrier parities repeat every two laps):
+// one unit's chunks, and the A rows of a CTA's shrink items, must fit the ring.
+bool chain_phase_fits(int K, int mode, int nseg, int rank, int nstages, int sm_count) {
+  const WLayout L = make_wlayout(K, TILE_N, TILE_K);
+  const int tpu = (mode == MODE_GATEUP) ? 2 : 1;
+  if (tpu * L.nchunks > nstages) return false;
+  if (nseg > 0 && rank > 0) {
+    const int items = (CHAIN_MAX_ROWS * nseg * rank + sm_count - 1) / sm_count;
+    const int np = (K + CH_A_PIECE - 1) / CH_A_PIECE;
+    if (items > CH_MAX_ITEMS || items * np > nstages) return false;
+    if (CH_BS_BYTES / (tpu * CHAIN_MAX_ROWS * rank * 32) < 1) return false;     // one unit's B slices must fit
+  }
+  return true;
 }
 
 size_t chain_smem_bytes(int kmax, int rank, int nstages) { return chain_carve(kmax, rank, nstages).total; }
@@ -65,7 +86,6 @@ int chain_pick_stages(int kmax, int rank) {
   if (base >= limit) return 0;
   int n = (int)((limit - base) / CH_STAGE_BYTES);
   if (n > CH_MAX_STAGES) n = CH_MAX_STAGES;
-  if (rank > 0 && CH_BS_BYTES / (CHAIN_MAX_ROWS * rank * 32) < 2) return 0;   // a gate/up pair must fit the B buffer
   return n >= 8 ? n : 0;
 }
 
@@ -100,9 +120,6 @@ __device__ __forceinline__ uint64_t policy_evict_first() {
 __device__ __forceinline__ void cp_async16_ca(void* smem, const void* gmem) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem)), "l"(gmem) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit_wait_all() {
-  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-}
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(CH_CTHREADS) : "memory"); }
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
   unsigned long long v;
@@ -112,25 +129,26 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 __device__ __forceinline__ void red_release_add_u64(unsigned long long* p, unsigned long long v) {
   asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
-__device__ __forceinline__ uint4 ldg_nc_v4(const void* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
+// the ring is addressed by the running stage count since the start of the launch
+__device__ __forceinline__ int pos_stage(int pos, int nstages) { return pos % nstages; }
+__device__ __forceinline__ uint32_t pos_parity(int pos, int nstages) { return (uint32_t)((pos / nstages) & 1); }
 
 // ----------------------------------------------------------------------------- bounded waits
 struct WaitCtx {
   volatile int* s_abort;            // shared: this CTA has given up waiting
-  unsigned long long* sync;         // global: [0] barrier, [1] shrink, [2] abort
+  unsigned long long* sync;         // global: [0] barrier, [1] shrink, [2] abort, [3] where the first wait gave up
   int* status;
 };
-__device__ __noinline__ void raise_abort(const WaitCtx& w) {
+// where codes: 1 producer/free stage, 2 shrink/A piece, 3 GEMM/weight chunk, 4 T counter, 5 grid barrier
+__device__ __noinline__ void raise_abort(const WaitCtx& w, int where, int phase) {
   *w.s_abort = 1;
   atomicCAS(w.status, 0, MLORA_ERR_TIMEOUT);
+  atomicCAS(w.sync + 3, 0ull, ((unsigned long long)where << 48) | ((unsigned long long)(phase & 0xffff) << 32) |
+                                  ((unsigned long long)(blockIdx.x & 0xffff) << 16) | (unsigned long long)(threadIdx.x & 0xffff));
   atomicExch(w.sync + 2, 1ull);
 }
 // mbarrier wait; false when the CTA is (or goes) in abort mode
-__device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const WaitCtx& w) {
+__device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const WaitCtx& w, int where, int phase) {
   if (mbar_try_wait(bar, parity)) return true;
   if (*w.s_abort) return false;
   const long long t0 = clock64();
@@ -139,19 +157,20 @@ __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const W
     if ((it & 255) == 255) {
       if (*w.s_abort) return false;
       if (ld_acquire_u64(w.sync + 2) != 0ull) { *w.s_abort = 1; return false; }
-      if (clock64() - t0 > CH_WAIT_CYCLES) { raise_abort(w); return false; }
+      if (clock64() - t0 > CH_WAIT_CYCLES) { raise_abort(w, where, phase); return false; }
     }
   }
 }
 // one thread spins until *ctr >= target
-__device__ __forceinline__ void wait_counter(const unsigned long long* ctr, unsigned long long target, const WaitCtx& w) {
+__device__ __forceinline__ void wait_counter(const unsigned long long* ctr, unsigned long long target, const WaitCtx& w,
+                                             int where, int phase) {
   if (*w.s_abort) return;
   const long long t0 = clock64();
   for (int it = 0;; ++it) {
     if (ld_acquire_u64(ctr) >= target) return;
     if ((it & 63) == 63) {
       if (ld_acquire_u64(w.sync + 2) != 0ull) { *w.s_abort = 1; return; }
-      if (clock64() - t0 > CH_WAIT_CYCLES) { raise_abort(w); return; }
+      if (clock64() - t0 > CH_WAIT_CYCLES) { raise_abort(w, where, phase); return; }
     }
   }
 }
@@ -181,8 +200,8 @@ __device__ long long g_trace[2 * TR_PHASES * TR_PER_PHASE * 3];
     if (tid == 0 && tr_slot >= 0 && tr_n < TR_PER_PHASE && p < TR_PHASES) {                                \
       long long tns;                                                                                       \
       asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tns));                                              \
-      long long* e = g_trace + (((size_t)tr_slot * TR_PHASES + p) * TR_PER_PHASE + tr_n) * 3;              \
-      e[0] = (id); e[1] = tns; e[2] = clock64(); ++tr_n;                                                   \
+      long long* e_ = g_trace + (((size_t)tr_slot * TR_PHASES + p) * TR_PER_PHASE + tr_n) * 3;             \
+      e_[0] = (id); e_[1] = tns; e_[2] = clock64(); ++tr_n;                                                \
     }                                                                                                      \
   } while (0)
 #else
@@ -190,22 +209,75 @@ __device__ long long g_trace[2 * TR_PHASES * TR_PER_PHASE * 3];
 #endif
 
 // ----------------------------------------------------------------------------- the ring schedule
-// Everything immutable that a CTA needs flows through the ring in one fixed order, known to the producer and
-// to the consumers alike.  Per phase:
+// Everything immutable and bulky that a CTA needs flows through the ring in one fixed order, known to the
+// producer and to the consumers alike.  Per phase:
 //   1. for each shrink item of the CTA (row m, segment, rank index j) whose row has an adapter: the row j of
 //      A in pieces of CH_A_PIECE halves, one stage per piece;
 //   2. for each unit of the CTA, per tile, the weight chunks.
-// The 32-byte slices B[j][16 columns of a tile] of the rows' adapters are too small for bulk copies; the
-// consumer threads fetch them with cp.async into their own buffer at the start of a phase, where the
-// activation prologue hides the latency.
-constexpr int CH_A_PIECE = 2048;                   // halves of an A row per stage
-
 struct Ring {
   int stage;
   uint32_t parity;
   int nstages;
   __device__ __forceinline__ void advance() { if (++stage == nstages) { stage = 0; parity ^= 1; } }
 };
+
+// RMSNorm (Sec. 3.1) of up to 8 rows by all consumer threads: thread `tid` owns the float4 columns
+// tid + i*CH_CTHREADS (i < NVR) of EVERY row, so the gain is loaded once per thread and the rows stay in
+// registers between the sum of squares and the scaling.  The rows were written by other CTAs: read through L2.
+template <int NVR>
+__device__ __forceinline__ void norm_rows(const float* __restrict__ x, const __half* __restrict__ gain, int K, int M,
+                                          float eps, __half* hs, int hs_stride, float* s_ssw, float* s_inv, int tid) {
+  const int warp = tid >> 5, lane = tid & 31;
+  const int nvec = K >> 2;
+  float4 xv[NVR][CHAIN_MAX_ROWS];
+  uint2 gv[NVR];
+  float ss[CHAIN_MAX_ROWS];
+#pragma unroll
+  for (int m = 0; m < CHAIN_MAX_ROWS; ++m) ss[m] = 0.f;
+#pragma unroll
+  for (int i = 0; i < NVR; ++i) {
+    const int v = tid + i * CH_CTHREADS;
+    const bool in = v < nvec;
+    gv[i] = in ? __ldg(reinterpret_cast<const uint2*>(gain) + v) : make_uint2(0, 0);
+#pragma unroll
+    for (int m = 0; m < CHAIN_MAX_ROWS; ++m)
+      xv[i][m] = (in && m < M) ? __ldcg(reinterpret_cast<const float4*>(x + (size_t)m * K) + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+#pragma unroll
+  for (int i = 0; i < NVR; ++i)
+#pragma unroll
+    for (int m = 0; m < CHAIN_MAX_ROWS; ++m)
+      ss[m] += xv[i][m].x * xv[i][m].x + xv[i][m].y * xv[i][m].y + xv[i][m].z * xv[i][m].z + xv[i][m].w * xv[i][m].w;
+#pragma unroll
+  for (int m = 0; m < CHAIN_MAX_ROWS; ++m) {
+    ss[m] = warp_sum(ss[m]);
+    if (lane == 0) s_ssw[warp * CHAIN_MAX_ROWS + m] = ss[m];
+  }
+  consumer_sync();
+  if (tid < CHAIN_MAX_ROWS) {
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < CH_CWARPS; ++w) tot += s_ssw[w * CHAIN_MAX_ROWS + tid];
+    s_inv[tid] = rsqrtf(tot / (float)K + eps);
+  }
+  consumer_sync();
+#pragma unroll
+  for (int i = 0; i < NVR; ++i) {
+    const int v = tid + i * CH_CTHREADS;
+    if (v < nvec) {
+      const float2 g01 = __half22float2(u32_as_h2(gv[i].x)), g23 = __half22float2(u32_as_h2(gv[i].y));
+#pragma unroll
+      for (int m = 0; m < CHAIN_MAX_ROWS; ++m) {
+        if (m < M) {
+          const float inv = s_inv[m];
+          const __half2 o01 = __floats2half2_rn(xv[i][m].x * inv * g01.x, xv[i][m].y * inv * g01.y);
+          const __half2 o23 = __floats2half2_rn(xv[i][m].z * inv * g23.x, xv[i][m].w * inv * g23.y);
+          *reinterpret_cast<uint2*>(hs + (size_t)m * hs_stride + 4 * v) = make_uint2(h2_as_u32(o01), h2_as_u32(o23));
+        }
+      }
+    }
+  }
+}
 
 // ----------------------------------------------------------------------------- the kernel
 __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const ChainArgs a) {
@@ -218,6 +290,8 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
   __shared__ int s_abort_word;
   __shared__ unsigned long long s_base[2];
   __shared__ unsigned s_shr_cnt;                      // warps of this CTA that finished their shrink items
+  __shared__ float s_ssw[CH_CWARPS * CHAIN_MAX_ROWS];  // RMSNorm: per-warp sums of squares of every row
+  __shared__ float s_inv[CHAIN_MAX_ROWS];
 
   const int nstages = a.nstages;
   const ChainSmem cs = chain_carve(a.kmax, a.rank, nstages);
@@ -241,7 +315,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
   if (tid == 0) {
     for (int s = 0; s < nstages; ++s) {
       mbar_init(smem_u32(full_bar + s), 1);
-      mbar_init(smem_u32(empty_bar + s), 1);
+      mbar_init(smem_u32(empty_bar + s), CH_ITEMS_PER_CHUNK);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     s_abort_word = (ld_acquire_u64(a.sync + 2) != 0ull) ? 1 : 0;
@@ -294,20 +368,22 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     Ring rg{0, 1u, nstages};                         // a fresh "empty" barrier passes a wait on parity 1
     long long issued = 0;
     bool alive = true;
+    int cur_phase = a.p0;
     // lane 0 waits for the stage to be free; every lane learns the outcome
     auto acquire = [&]() -> bool {
       int ok = 1;
-      if (lane == 0) ok = wait_mbar(smem_u32(empty_bar + rg.stage), rg.parity, wc) ? 1 : 0;
+      if (lane == 0) ok = wait_mbar(smem_u32(empty_bar + rg.stage), rg.parity, wc, 1, cur_phase) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
       return ok != 0;
     };
     for (int p = a.p0; p < a.p1 && alive; ++p) {
+      cur_phase = p;
       const ChainPhase* ph = a.phases + p;           // immutable: read the descriptor from global
       const unsigned char* wbase = ph->w;
       const int mode = ph->mode, K = ph->K;
       const WLayout L = make_wlayout(K, ph->N, ph->G);
       const int nseg = lora_on ? ph->lora_nseg : 0;
-      // adapter matrices of the rows for this phase: lane (seg, m)
+      // LoRA-A matrices of the rows for this phase: lane (seg, m)
       const __half* myA = nullptr;
       if (nseg > 0 && lane < 3 * CHAIN_MAX_ROWS) {
         const int seg = lane / CHAIN_MAX_ROWS, m = lane % CHAIN_MAX_ROWS;
@@ -340,7 +416,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
           }
         }
       }
-      // ---- 2. units: B slices, then weight chunks
+      // ---- 2. units: weight chunks
       const int tpu = (mode == MODE_GATEUP) ? 2 : 1;
       const int n_units = L.NT / tpu;
       for (int u = blockIdx.x; u < n_units && alive; u += G) {
@@ -373,20 +449,20 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
         }
       }
     }
-    return;                                           // consumers use a named barrier; nothing below is for this warp
+    return;                                           // consumers use named barriers; nothing below is for this warp
   }
 
   // =========================================================================== consumer warps
-  // The CTA's stages of a phase form one list (see "the ring schedule").  Every warp walks the list; a stage
-  // is waited for, read and released by its owner warp only:
-  //   shrink item k        -> warp k % 8 (all pieces of the row)
-  //   weight chunk ci      -> warp (ci + items) % 8, ci counting the CTA's chunks of the phase; a warp keeps the
-  //                           partial sums of its chunks of one tile in registers and parks them in
-  //                           red[tile][c % 8] -- the epilogue adds the slots in index order
-  //   LoRA-B stages        -> read by the epilogue threads, released by thread 0 afterwards
-  // Tiles are handled in groups of as many as the partial-sum buffer holds; one epilogue pass per group.
+  // The CTA's stages of a phase form one list (see "the ring schedule"); a consumer finds a stage by its
+  // running count since the start of the launch.
+  //   shrink item k   -> warp k % 16 reads all pieces of the row and frees each stage on its own
+  //   weight chunks   -> warps work in teams; team tm takes the CTA's units tm, tm + teams, ...; inside a unit
+  //                      every tile's k-tiles are cut into items of CH_ITEM_KT k-tiles and each member warp owns a
+  //                      contiguous run of them, keeps their partial sums in registers and parks them in its own
+  //                      slot; the team adds the slots in member order (fixed summation order) and runs the
+  //                      epilogue.  A stage is free again after CH_ITEMS_PER_CHUNK arrivals, one per item.
   const int g = lane >> 2, t = lane & 3;
-  Ring rg{0, 0u, nstages};
+  int pos = 0;                                        // stages of this CTA consumed (or skipped) so far
   unsigned long long n_bar = 0;                       // barriers passed in this launch
   unsigned n_shr = 0;                                 // LoRA phases passed in this launch
   float* redf = reinterpret_cast<float*>(red);
@@ -406,76 +482,66 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     STAMP(0);
     const int tpu = (ph.mode == MODE_GATEUP) ? 2 : 1;
     const int n_units = L.NT / tpu;
-    const int ns = L.nchunks < CH_CWARPS ? L.nchunks : CH_CWARPS;    // partial-sum slots per tile
-    int tiles_per_group = CH_RED_BYTES / (ns * 512);
-    if (tiles_per_group > CH_MAX_GROUP_TILES) tiles_per_group = CH_MAX_GROUP_TILES;
-    if (nseg > 0 && tiles_per_group > CH_BS_BYTES / (CHAIN_MAX_ROWS * r * 32)) tiles_per_group = CH_BS_BYTES / (CHAIN_MAX_ROWS * r * 32);
-    const int units_per_group = tiles_per_group / tpu;
-    // LoRA-B slices of the group starting at unit u0 -> Bs[tile][m][j][16]; immutable, so no need to wait for activations
-    auto issue_b = [&](int u0) {
+    const int ipt = (L.KT + CH_ITEM_KT - 1) / CH_ITEM_KT;             // items per tile
+    const int gshift = (L.G >= CHUNK_KT * TILE_K) ? 31 : (31 - __clz(L.G / TILE_K));   // k-tile -> scale group of its chunk
+    // teams: as many units in flight as the CTA has, as the ring can hold at once (a wait must never be a whole
+    // lap ahead of the fill front: mbarrier parities repeat every two laps) and as the B buffer has room for
+    const int my_units = (n_units > (int)blockIdx.x) ? (n_units - 1 - (int)blockIdx.x) / (int)G + 1 : 0;
+    int teams = my_units < CH_MAX_TEAMS ? my_units : CH_MAX_TEAMS;
+    if (teams > nstages / (tpu * L.nchunks)) teams = nstages / (tpu * L.nchunks);
+    if (nseg > 0 && teams > CH_BS_BYTES / (tpu * CHAIN_MAX_ROWS * r * 32)) teams = CH_BS_BYTES / (tpu * CHAIN_MAX_ROWS * r * 32);
+    if (teams < 1) teams = 1;
+    const int wpt = CH_CWARPS / teams;                                // warps per team
+    const int tm = warp / wpt, member = warp - tm * wpt;
+    const bool in_team = tm < teams;
+    const int team_threads = wpt * 32, tt = member * 32 + lane;
+    __half* Bs_team = Bs + (size_t)tm * tpu * CHAIN_MAX_ROWS * r * 16;
+    auto team_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(2 + tm), "r"(team_threads) : "memory"); };
+    // LoRA-B slices of unit u -> Bs_team[tile][m][j][16]; immutable, so no need to wait for activations
+    auto issue_b = [&](int u) {
       const int per_tile = CHAIN_MAX_ROWS * r * 2;                     // 16-byte pieces
-      for (int ug = 0; ug < units_per_group; ++ug) {
-        const int u = u0 + ug * (int)G;
-        if (u >= n_units) break;
-        for (int i = tid; i < tpu * per_tile; i += CH_CTHREADS) {
-          const int tu = i / per_tile, rem = i % per_tile;
-          const int m = rem / (r * 2), j = (rem >> 1) % r, h16 = rem & 1;
-          int seg, col;
-          chain_map_col(ph.mode, (u * tpu + tu) * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
-          const __half* B = (m < M && seg < nseg) ? s_pB[slot][seg][m] : nullptr;
-          if (B != nullptr)
-            cp_async16_ca(Bs + (((size_t)(ug * tpu + tu) * CHAIN_MAX_ROWS + m) * r + j) * 16 + h16 * 8,
-                          B + (size_t)j * ph.lora_n[seg] + col + h16 * 8);
-        }
+      for (int i = tt; i < tpu * per_tile; i += team_threads) {
+        const int tu = i / per_tile, rem = i % per_tile;
+        const int m = rem / (r * 2), j = (rem >> 1) % r, h16 = rem & 1;
+        int seg, col;
+        chain_map_col(ph.mode, (u * tpu + tu) * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
+        const __half* B = (m < M && seg < nseg) ? s_pB[slot][seg][m] : nullptr;
+        if (B != nullptr)
+          cp_async16_ca(Bs_team + (((size_t)tu * CHAIN_MAX_ROWS + m) * r + j) * 16 + h16 * 8,
+                        B + (size_t)j * ph.lora_n[seg] + col + h16 * 8);
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    if (nseg > 0 && (int)blockIdx.x < n_units) issue_b(blockIdx.x);
+    if (nseg > 0 && in_team && tm < my_units) issue_b(blockIdx.x + tm * (int)G);
 
     // ---- 1. activations of the phase -> shared memory, fp16 [8][K+8]
     if (ph.in_kind == IN_NORM) {
-      // RMSNorm (Sec. 3.1): warp m owns row m; the row was written by other CTAs: read it through L2
-      const int m = warp;
-      if (m < M) {
-        __half* dst = hs + (size_t)m * hs_stride;
-        const float* x = ph.x_f32 + (size_t)m * K;
-        constexpr int NV = 24;                         // rows up to 3072 wide stay in registers: one pass
-        if (K <= NV * 128) {
-          float4 xv[NV];
-          uint2 gv[NV];
-          float ss = 0.f;
-#pragma unroll
-          for (int i = 0; i < NV; ++i) {
-            const int k = lane * 4 + i * 128;
-            xv[i] = (k < K) ? __ldcg(reinterpret_cast<const float4*>(x + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
-            gv[i] = (k < K) ? __ldg(reinterpret_cast<const uint2*>(ph.gain + k)) : make_uint2(0, 0);
-          }
-#pragma unroll
-          for (int i = 0; i < NV; ++i) ss += xv[i].x * xv[i].x + xv[i].y * xv[i].y + xv[i].z * xv[i].z + xv[i].w * xv[i].w;
-          ss = warp_sum(ss);
-          const float inv = rsqrtf(ss / (float)K + a.eps);
-#pragma unroll
-          for (int i = 0; i < NV; ++i) {
-            const int k = lane * 4 + i * 128;
-            if (k < K) {
-              const float2 g01 = __half22float2(u32_as_h2(gv[i].x)), g23 = __half22float2(u32_as_h2(gv[i].y));
-              const __half2 o01 = __floats2half2_rn(xv[i].x * inv * g01.x, xv[i].y * inv * g01.y);
-              const __half2 o23 = __floats2half2_rn(xv[i].z * inv * g23.x, xv[i].w * inv * g23.y);
-              *reinterpret_cast<uint2*>(dst + k) = make_uint2(h2_as_u32(o01), h2_as_u32(o23));
-            }
-          }
-        } else {
-          float ss = 0.f;
-          for (int k = lane * 4; k < K; k += 128) {
+      const int nvec = K >> 2;
+      if (nvec <= CH_CTHREADS) norm_rows<1>(ph.x_f32, ph.gain, K, M, a.eps, hs, hs_stride, s_ssw, s_inv, tid);
+      else if (nvec <= 2 * CH_CTHREADS) norm_rows<2>(ph.x_f32, ph.gain, K, M, a.eps, hs, hs_stride, s_ssw, s_inv, tid);
+      else {
+        // wide rows: two passes, warps 2m and 2m+1 own the halves of row m
+        const int m = warp >> 1, hf = warp & 1;
+        const int kh = K / 2;
+        const float* x = ph.x_f32 + (size_t)m * K + hf * kh;
+        const __half* gp = ph.gain + hf * kh;
+        float ss = 0.f;
+        if (m < M) {
+          for (int k = lane * 4; k < kh; k += 128) {
             const float4 v = __ldcg(reinterpret_cast<const float4*>(x + k));
             ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
           }
           ss = warp_sum(ss);
-          const float inv = rsqrtf(ss / (float)K + a.eps);
-          for (int k = lane * 4; k < K; k += 128) {
+        }
+        if (lane == 0) s_ssw[warp] = ss;
+        consumer_sync();
+        if (m < M) {
+          const float inv = rsqrtf((s_ssw[2 * m] + s_ssw[2 * m + 1]) / (float)K + a.eps);
+          __half* dst = hs + (size_t)m * hs_stride + hf * kh;
+          for (int k = lane * 4; k < kh; k += 128) {
             const float4 v = __ldcg(reinterpret_cast<const float4*>(x + k));
-            const uint2 gv = __ldg(reinterpret_cast<const uint2*>(ph.gain + k));
-            const float2 g01 = __half22float2(u32_as_h2(gv.x)), g23 = __half22float2(u32_as_h2(gv.y));
+            const uint2 gw = __ldg(reinterpret_cast<const uint2*>(gp + k));
+            const float2 g01 = __half22float2(u32_as_h2(gw.x)), g23 = __half22float2(u32_as_h2(gw.y));
             const __half2 o01 = __floats2half2_rn(v.x * inv * g01.x, v.y * inv * g01.y);
             const __half2 o23 = __floats2half2_rn(v.z * inv * g23.x, v.w * inv * g23.y);
             *reinterpret_cast<uint2*>(dst + k) = make_uint2(h2_as_u32(o01), h2_as_u32(o23));
@@ -498,52 +564,55 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     if (warp == CH_CWARPS - 1 && p + 1 < a.p1) prep_phase(p + 1);
 
     // ---- 3. LoRA shrink (first factor of the low-rank term of Eq. 1-4): items (row, segment, rank index)
-    // are dealt round-robin to the CTAs; item k of the CTA belongs to warp k % 8
-    int n_my = 0;
+    // are dealt round-robin to the CTAs; item k of the CTA belongs to warp k % 16
     if (nseg > 0) {
       const int n_items = M * nseg * r;
       const int np = (K + CH_A_PIECE - 1) / CH_A_PIECE;
+      int n_my = 0;
+      bool wrote = false;
       for (int i = blockIdx.x; i < n_items && n_my < CH_MAX_ITEMS; i += G, ++n_my) {
         const int seg = (i / r) % nseg, m = i / (r * nseg);
         if (s_pA[slot][seg][m] == nullptr) continue;
-        if ((n_my & (CH_CWARPS - 1)) != warp) {
-          for (int q = 0; q < np; ++q) rg.advance();
-          continue;
-        }
-        const __half* hrow = hs + (size_t)m * hs_stride;
-        float acc = 0.f;
-        for (int k0 = 0; k0 < K; k0 += CH_A_PIECE) {
-          const bool ok = wait_mbar(smem_u32(full_bar + rg.stage), rg.parity, wc);
-          const unsigned char* sb = ring + (size_t)rg.stage * CH_STAGE_BYTES;
-          if (ok) {
+        if (n_my % CH_CWARPS == warp) {
+          const __half* hrow = hs + (size_t)m * hs_stride;
+          float acc = 0.f;
+          for (int q = 0; q < np; ++q) {
+            const int k0 = q * CH_A_PIECE;
+            const int st = pos_stage(pos + q, nstages);
+            const bool ok = wait_mbar(smem_u32(full_bar + st), pos_parity(pos + q, nstages), wc, 2, p);
+            const unsigned char* sb = ring + (size_t)st * CH_STAGE_BYTES;
+            if (ok) {
 #pragma unroll
-            for (int q = 0; q < CH_A_PIECE / 256; ++q) {
-              const int off = q * 256 + lane * 8;            // halves inside the piece
-              if (k0 + off < K) {
-                const uint4 av = *reinterpret_cast<const uint4*>(sb + off * 2);
-                const uint4 hv = *reinterpret_cast<const uint4*>(hrow + k0 + off);
-                const uint32_t aw[4] = {av.x, av.y, av.z, av.w};
-                const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
+              for (int v = 0; v < CH_A_PIECE / 256; ++v) {
+                const int off = v * 256 + lane * 8;            // halves inside the piece
+                if (k0 + off < K) {
+                  const uint4 av = *reinterpret_cast<const uint4*>(sb + off * 2);
+                  const uint4 hv = *reinterpret_cast<const uint4*>(hrow + k0 + off);
+                  const uint32_t aw[4] = {av.x, av.y, av.z, av.w};
+                  const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  const float2 af = __half22float2(u32_as_h2(aw[e])), hf = __half22float2(u32_as_h2(hw[e]));
-                  acc = fmaf(af.x, hf.x, acc);
-                  acc = fmaf(af.y, hf.y, acc);
+                  for (int e = 0; e < 4; ++e) {
+                    const float2 af = __half22float2(u32_as_h2(aw[e])), hf2 = __half22float2(u32_as_h2(hw[e]));
+                    acc = fmaf(af.x, hf2.x, acc);
+                    acc = fmaf(af.y, hf2.y, acc);
+                  }
                 }
               }
             }
+            __syncwarp();
+            if (lane < CH_ITEMS_PER_CHUNK) mbar_arrive(smem_u32(empty_bar + st));
           }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(empty_bar + rg.stage));
-          rg.advance();
+          acc = warp_sum(acc);
+          if (lane == 0) __stcg(a.T + i, acc * s_scale[m]);
+          wrote = true;
         }
-        acc = warp_sum(acc);
-        if (lane == 0) __stcg(a.T + i, acc * s_scale[m]);
+        pos += np;
       }
-      // the last warp of the CTA to get here tells the grid that this CTA's share of T is written
+      // the last warp of the CTA to get here tells the grid that this CTA's share of T is written; a warp that
+      // stored part of T makes it visible device-wide before it counts itself in
       ++n_shr;
       if (lane == 0) {
-        __threadfence();
+        if (wrote) __threadfence();
         const unsigned old = atomicAdd(&s_shr_cnt, 1u);
         if (old == n_shr * CH_CWARPS - 1) red_release_add_u64(a.sync + 1, 1ull);
       }
@@ -551,129 +620,134 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     STAMP(2);
 
     // ---- 4. the CTA's units: one n-tile (or a gate/up pair of n-tiles), all of K
-    bool t_loaded = false;
-    int ci = n_my;                                     // chunk ownership continues after the shrink items
-    for (int u0 = blockIdx.x; u0 < n_units; u0 += G * units_per_group) {
-      int ng = 0;
-      if (nseg > 0 && u0 != (int)blockIdx.x) issue_b(u0);              // the first group's went out before the prologue
-      for (int ug = 0; ug < units_per_group; ++ug) {
-        const int u = u0 + ug * (int)G;
-        if (u >= n_units) break;
-        ++ng;
+    if (in_team) {
+      bool t_loaded = false;
+      const int it_lo = (member * ipt) / wpt, it_hi = ((member + 1) * ipt) / wpt;   // this warp's items of a tile
+      for (int k = tm; k < my_units; k += teams) {
+        const int u = blockIdx.x + k * (int)G;
+        if (nseg > 0 && k != tm) issue_b(u);                              // the first unit's went out before the prologue
+        const int ubase = pos + k * tpu * L.nchunks;                      // first stage of the unit
         for (int tu = 0; tu < tpu; ++tu) {
           float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
-          int my_slot = -1;
-          for (int c = 0; c < L.nchunks; ++c, ++ci) {
-            if ((ci & (CH_CWARPS - 1)) == warp) {
-              my_slot = c & (CH_CWARPS - 1);
-              const int kc = (c == L.nchunks - 1) ? L.kc_last : CHUNK_KT;
-              const bool ok = wait_mbar(smem_u32(full_bar + rg.stage), rg.parity, wc);
-              if (ok) {
-                const unsigned char* sb = ring + (size_t)rg.stage * CH_STAGE_BYTES;
-                const __half* hbase = hs + (size_t)g * hs_stride + (size_t)c * CHUNK_KT * TILE_K + 16 * t;
+          int waited = -1;
+          for (int it = it_lo; it < it_hi; ++it) {
+            const int c = it / CH_ITEMS_PER_CHUNK;
+            const int kc = (c == L.nchunks - 1) ? L.kc_last : CHUNK_KT;
+            const int P = ubase + tu * L.nchunks + c;
+            const int st = pos_stage(P, nstages);
+            bool ok = true;
+            if (P != waited) {
+              ok = wait_mbar(smem_u32(full_bar + st), pos_parity(P, nstages), wc, 3, p);
+              waited = P;
+            }
+            const int itl = it - c * CH_ITEMS_PER_CHUNK;                  // item inside its chunk
+            const int ktl = itl * CH_ITEM_KT;                             // its first k-tile inside the chunk
+            if (ok) {
+              const unsigned char* sb = ring + (size_t)st * CH_STAGE_BYTES;
+              const __half* hbase = hs + (size_t)g * hs_stride + (size_t)(c * CHUNK_KT + ktl) * TILE_K + 16 * t;
 #pragma unroll
-                for (int kt = 0; kt < CHUNK_KT; ++kt) {
-                  if (kt < kc) {
-                    const uint4 wv = *reinterpret_cast<const uint4*>(sb + kt * 512 + lane * 16);
-                    const int gi = (L.G >= CHUNK_KT * TILE_K) ? 0 : (kt * TILE_K) / L.G;
-                    const uint32_t sw = *reinterpret_cast<const uint32_t*>(sb + kc * 512 + gi * 32 + g * 4);
-                    const uint4 b01 = *reinterpret_cast<const uint4*>(hbase + kt * TILE_K);
-                    const uint4 b23 = *reinterpret_cast<const uint4*>(hbase + kt * TILE_K + 8);
-                    __half2 s_lo, s_hi;
-                    split_scales(sw, s_lo, s_hi);
-                    uint32_t af[4][4];
-                    dequant8(wv.x, s_lo, s_hi, af[0]);
-                    dequant8(wv.y, s_lo, s_hi, af[1]);
-                    dequant8(wv.z, s_lo, s_hi, af[2]);
-                    dequant8(wv.w, s_lo, s_hi, af[3]);
-                    mma_16816(acc0, af[0], b01.x, b01.y);
-                    mma_16816(acc1, af[1], b01.z, b01.w);
-                    mma_16816(acc0, af[2], b23.x, b23.y);
-                    mma_16816(acc1, af[3], b23.z, b23.w);
-                  }
+              for (int q = 0; q < CH_ITEM_KT; ++q) {
+                if (ktl + q < kc) {
+                  const uint4 wv = *reinterpret_cast<const uint4*>(sb + (ktl + q) * 512 + lane * 16);
+                  const uint32_t sw = *reinterpret_cast<const uint32_t*>(sb + kc * 512 + ((ktl + q) >> gshift) * 32 + g * 4);
+                  const uint4 b01 = *reinterpret_cast<const uint4*>(hbase + q * TILE_K);
+                  const uint4 b23 = *reinterpret_cast<const uint4*>(hbase + q * TILE_K + 8);
+                  __half2 s_lo, s_hi;
+                  split_scales(sw, s_lo, s_hi);
+                  uint32_t af[4][4];
+                  dequant8(wv.x, s_lo, s_hi, af[0]);
+                  dequant8(wv.y, s_lo, s_hi, af[1]);
+                  dequant8(wv.z, s_lo, s_hi, af[2]);
+                  dequant8(wv.w, s_lo, s_hi, af[3]);
+                  mma_16816(acc0, af[0], b01.x, b01.y);
+                  mma_16816(acc1, af[1], b01.z, b01.w);
+                  mma_16816(acc0, af[2], b23.x, b23.y);
+                  mma_16816(acc1, af[3], b23.z, b23.w);
                 }
               }
-              __syncwarp();
-              if (lane == 0) mbar_arrive(smem_u32(empty_bar + rg.stage));
             }
-            rg.advance();
+            __syncwarp();
+            // one arrival per item; the last item of a ragged chunk also arrives for the items the chunk lacks
+            const int items_here = (kc + CH_ITEM_KT - 1) / CH_ITEM_KT;
+            const int arrivals = (itl == items_here - 1) ? CH_ITEMS_PER_CHUNK - items_here + 1 : 1;
+            if (lane < arrivals) mbar_arrive(smem_u32(empty_bar + st));
           }
-          if (my_slot >= 0)
-            red[((size_t)(ug * tpu + tu) * ns + my_slot) * 32 + lane] =
-                make_float4(acc0[0] + acc1[0], acc0[1] + acc1[1], acc0[2] + acc1[2], acc0[3] + acc1[3]);
+          red[(size_t)(tu * CH_CWARPS + warp) * 32 + lane] =
+              make_float4(acc0[0] + acc1[0], acc0[1] + acc1[1], acc0[2] + acc1[2], acc0[3] + acc1[3]);
         }
-      }
-      STAMP(3);
-      asm volatile("cp.async.wait_group 0;" ::: "memory");
-      consumer_sync();
-      if (nseg > 0 && !t_loaded) {
-        // all of T must be in global memory before the first expand of the phase
-        if (tid == 0) wait_counter(a.sync + 1, s_base[1] + (unsigned long long)n_shr * G, wc);
-        consumer_sync();
-        for (int i = tid; i < M * nseg * r; i += CH_CTHREADS) Ts[i] = __ldcg(a.T + i);
-        consumer_sync();
-        t_loaded = true;
-        STAMP(4);
-      }
-      STAMP(5);
-      // ---- epilogue of the group: one thread per (unit, row, column)
-      for (int o = tid; o < ng * CHAIN_MAX_ROWS * TILE_N; o += CH_CTHREADS) {
-        const int ug = o >> 7, m = (o >> 4) & 7, col16 = o & 15;
-        if (m >= M) continue;
-        const int u = u0 + ug * (int)G;
-        // accumulator layout of m16n8k16: lane (g,t) holds (out g, row 2t), (g, 2t+1), (g+8, 2t), (g+8, 2t+1)
-        const int src_lane = (col16 & 7) * 4 + (m >> 1);
-        const int e = (col16 >> 3) * 2 + (m & 1);
-        float yv[2] = {0.f, 0.f};
-        int colv[2] = {0, 0};
+        STAMP(3);
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        team_sync();
+        if (nseg > 0 && !t_loaded) {
+          // all of T must be in global memory before the first expand; every team fetches the same values
+          if (tt == 0) wait_counter(a.sync + 1, s_base[1] + (unsigned long long)n_shr * G, wc, 4, p);
+          team_sync();
+          for (int i = tt; i < M * nseg * r; i += team_threads) Ts[i] = __ldcg(a.T + i);
+          team_sync();
+          t_loaded = true;
+          STAMP(4);
+        }
+        // ---- epilogue of the unit: one thread per (row, column)
+        for (int o = tt; o < CHAIN_MAX_ROWS * TILE_N; o += team_threads) {
+          const int m = o >> 4, col16 = o & 15;
+          if (m >= M) continue;
+          // accumulator layout of m16n8k16: lane (g,t) holds (out g, row 2t), (g, 2t+1), (g+8, 2t), (g+8, 2t+1)
+          const int src_lane = (col16 & 7) * 4 + (m >> 1);
+          const int e = (col16 >> 3) * 2 + (m & 1);
+          float yv[2] = {0.f, 0.f};
+          int colv[2] = {0, 0};
 #pragma unroll
-        for (int tu = 0; tu < 2; ++tu) {
-          if (tu < tpu) {
-            const int nt = u * tpu + tu;
-            const float* rp = redf + ((size_t)(ug * tpu + tu) * ns * 32 + src_lane) * 4 + e;
-            float y = 0.f;
-            for (int sl = 0; sl < ns; ++sl) y += rp[(size_t)sl * 128];
-            int seg, col;
-            chain_map_col(ph.mode, nt * TILE_N + col16, ph.seg_n0, ph.seg_n1, seg, col);
-            if (nseg > 0 && seg < nseg && s_pB[slot][seg][m] != nullptr) {
-              // LoRA expand (second factor of the low-rank term of Eq. 1-4): slice (m, j) sits at slot m*r + j
-              const float* Tm = Ts + ((size_t)m * nseg + seg) * r;
-              const __half* bp = Bs + (((size_t)(ug * tpu + tu) * CHAIN_MAX_ROWS + m) * r) * 16 + col16;
-              float s0 = 0.f, s1 = 0.f;
-              for (int j = 0; j < r; j += 2) {
-                s0 = fmaf(Tm[j], __half2float(bp[(size_t)j * 16]), s0);
-                if (j + 1 < r) s1 = fmaf(Tm[j + 1], __half2float(bp[(size_t)(j + 1) * 16]), s1);
+          for (int tu = 0; tu < 2; ++tu) {
+            if (tu < tpu) {
+              const int nt = u * tpu + tu;
+              float y = 0.f;
+              for (int j = 0; j < wpt; ++j)                               // fixed order: member 0, 1, ...
+                y += redf[((size_t)(tu * CH_CWARPS + tm * wpt + j) * 32 + src_lane) * 4 + e];
+              int seg, col;
+              chain_map_col(ph.mode, nt * TILE_N + col16, ph.seg_n0, ph.seg_n1, seg, col);
+              if (nseg > 0 && seg < nseg && s_pB[slot][seg][m] != nullptr) {
+                // LoRA expand (second factor of the low-rank term of Eq. 1-4)
+                const float* Tm = Ts + ((size_t)m * nseg + seg) * r;
+                const __half* bp = Bs_team + (((size_t)tu * CHAIN_MAX_ROWS + m) * r) * 16 + col16;
+                float s0 = 0.f, s1 = 0.f;
+                for (int j = 0; j < r; j += 2) {
+                  s0 = fmaf(Tm[j], __half2float(bp[(size_t)j * 16]), s0);
+                  if (j + 1 < r) s1 = fmaf(Tm[j + 1], __half2float(bp[(size_t)(j + 1) * 16]), s1);
+                }
+                y += s0 + s1;
               }
-              y += s0 + s1;
+              yv[tu] = y;
+              colv[tu] = col;
             }
-            yv[tu] = y;
-            colv[tu] = col;
+          }
+          const int nt0 = u * tpu;
+          if (ph.epi == EPI_F32) {
+            float* out = ph.out_f32 != nullptr ? ph.out_f32 : a.logits;
+            __stcg(out + (size_t)m * ph.ldo + nt0 * TILE_N + col16, yv[0]);
+          } else if (ph.epi == EPI_RESID) {
+            float* xp = ph.resid + (size_t)m * ph.N + nt0 * TILE_N + col16;
+            __stcg(xp, __ldcg(xp) + yv[0]);
+          } else {                                     // EPI_SWIGLU: even tile = gate, odd tile = up
+            const float v = yv[0] / (1.f + __expf(-yv[0])) * yv[1];
+            ph.out_f16[(size_t)m * (ph.N / 2) + colv[1]] = __float2half_rn(v);
           }
         }
-        const int nt0 = u * tpu;
-        if (ph.epi == EPI_F32) {
-          float* out = ph.out_f32 != nullptr ? ph.out_f32 : a.logits;
-          __stcg(out + (size_t)m * ph.ldo + nt0 * TILE_N + col16, yv[0]);
-        } else if (ph.epi == EPI_RESID) {
-          float* xp = ph.resid + (size_t)m * ph.N + nt0 * TILE_N + col16;
-          __stcg(xp, __ldcg(xp) + yv[0]);
-        } else {                                       // EPI_SWIGLU: even tile = gate, odd tile = up
-          const float v = yv[0] / (1.f + __expf(-yv[0])) * yv[1];
-          ph.out_f16[(size_t)m * (ph.N / 2) + colv[1]] = __float2half_rn(v);
-        }
+        STAMP(5);
+        team_sync();                                   // the team's partial sums and B slices may be rewritten
       }
-      consumer_sync();                                 // red and the B stages may be reused
-      STAMP(6);
     }
+    pos += my_units * tpu * L.nchunks;
+    STAMP(6);
 
     // ---- 5. grid barrier: the next phase reads what every CTA wrote
-    STAMP(7);
     if (p + 1 < a.p1) {
       ++n_bar;
+      consumer_sync();
+      STAMP(7);
       if (tid == 0) {
         __threadfence();
         red_release_add_u64(a.sync + 0, 1ull);
-        wait_counter(a.sync + 0, s_base[0] + n_bar * G, wc);
+        wait_counter(a.sync + 0, s_base[0] + n_bar * G, wc, 5, p);
         __threadfence();
       }
       consumer_sync();
@@ -689,10 +763,10 @@ extern "C" int mlora_trace_read(long long* host_out, int n_longs) {
   return (int)cudaMemcpyFromSymbol(host_out, g_trace, n * sizeof(long long));
 }
 extern "C" int mlora_trace_clear() {
-  void* p = nullptr;
-  cudaError_t e = cudaGetSymbolAddress(&p, g_trace);
+  void* ptr = nullptr;
+  cudaError_t e = cudaGetSymbolAddress(&ptr, g_trace);
   if (e != cudaSuccess) return (int)e;
-  return (int)cudaMemset(p, 0, sizeof(g_trace));
+  return (int)cudaMemset(ptr, 0, sizeof(g_trace));
 }
 #endif
 

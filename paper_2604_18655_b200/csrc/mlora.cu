@@ -632,8 +632,6 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
     size_t kmax = dm; if ((size_t)F > kmax) kmax = F; if ((size_t)Nq > kmax) kmax = Nq;
     c->chain_kmax = (int)kmax;
     c->chain_stages = chain_pick_stages(c->chain_kmax, d.lora_rank);
-    // every CTA must be able to hold its share of the shrink items of a phase
-    if ((CHAIN_MAX_ROWS * 3 * (d.lora_rank > 0 ? d.lora_rank : 1) + c->sm_count - 1) / c->sm_count > 16) c->chain_stages = 0;
     std::vector<ChainPhase> ph;
     const int tg = d.lora_rank > 0 && d.max_adapters > 0 ? d.lora_targets : 0;
     for (int l = 0; l < L; ++l) {
@@ -670,6 +668,9 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
       lm.x_f32 = c->X; lm.gain = (const __half*)d.rms_final; lm.out_f32 = nullptr; lm.ldo = d.vocab;
       ph.push_back(lm);
     }
+    for (const ChainPhase& q : ph)
+      if (c->chain_stages > 0 && !chain_phase_fits(q.K, q.mode, q.lora_nseg, d.lora_rank, c->chain_stages, c->sm_count))
+        c->chain_stages = 0;
     c->n_phases = (int)ph.size();
     CKC(cudaMalloc(&c->phases, ph.size() * sizeof(ChainPhase)));
     CKC(cudaMemcpy(c->phases, ph.data(), ph.size() * sizeof(ChainPhase), cudaMemcpyHostToDevice));
@@ -864,10 +865,17 @@ int mlora_sync_status(mlora_ctx* c) {
   CK(cudaMemcpy(&st, c->status, sizeof(int), cudaMemcpyDeviceToHost));
   if (st != 0) {
     CK(cudaMemset(c->status, 0, sizeof(int)));
+    unsigned long long where = 0;
+    CK(cudaMemcpy(&where, c->chain_sync + 3, sizeof(where), cudaMemcpyDeviceToHost));
     // a wait that ran out leaves the barrier counters of the persistent kernel mid-count: start them afresh
     CK(cudaMemset(c->chain_sync, 0, 4 * sizeof(unsigned long long)));
-    return fail(st, st == MLORA_ERR_TIMEOUT ? "device status: a bounded wait ran out"
-                                            : "device status: malformed tree or token id out of range");
+    if (st == MLORA_ERR_TIMEOUT) {
+      char buf[160];
+      std::snprintf(buf, sizeof(buf), "device status: a bounded wait ran out (wait kind %d, phase %d, block %d, thread %d)",
+                    (int)(where >> 48), (int)((where >> 32) & 0xffff), (int)((where >> 16) & 0xffff), (int)(where & 0xffff));
+      return fail(st, buf);
+    }
+    return fail(st, "device status: malformed tree or token id out of range");
   }
   return MLORA_OK;
 }
@@ -1039,8 +1047,7 @@ int mlora_linear(mlora_weight* w, const void* x, int32_t M, const int32_t* row_a
   if (M <= CHAIN_MAX_ROWS) {
     // few rows: one persistent kernel does shrink, GEMM and expand
     const int stages = chain_pick_stages(w->w.K, lora ? rank : 0);
-    const bool items_fit = !lora || (CHAIN_MAX_ROWS * rank + w->sm_count - 1) / w->sm_count <= 16;
-    if (stages > 0 && items_fit) {
+    if (stages > 0 && chain_phase_fits(w->w.K, MODE_PLAIN, lora ? 1 : 0, rank, stages, w->sm_count)) {
       ChainArgs a{};
       a.phases = w->phase; a.p0 = 0; a.p1 = 1; a.M = M; a.logits = y; a.h_in = (const __half*)x;
       if (lora) {

@@ -85,6 +85,28 @@ def test_prefill_logits_and_follow_mode_decode(GpuModel):
     gm.close()
 
 
+def test_decode_long_weight_streams(GpuModel):
+    """A vocabulary and an FFN wide enough that one CTA's weight chunks of a projection wrap the shared-memory
+    ring of the persistent kernel several times (the tiny models never do), 8 streams, rank-16 adapters."""
+    from paper_2604_18655_b200 import binding as mb
+    cfg = gen.ModelCfg("widev", 1, 256, 4, 2, 64, 2816, 32000, 128, 16, 127, 8, 8, 40, b_std=0.05)
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+    ids = gen.make_prompt_ids(cfg, 0)
+    gm.prefill(ids)
+    orc.prefill_shared(ids)
+    ad = [0, 1, 2, 3, 4, 5, 6, -1]
+    toks = np.arange(8, dtype=np.int32) * 101 + 7
+    for step in range(3):
+        nxt, logits = gm.decode(ad, toks)
+        r = orc.decode_step(ad, tokens=toks)
+        compare(logits, r["logits"], f"wide decode logits step {step}")
+        check_argmax(nxt, r["logits"], f"wide step {step}")
+        toks = nxt
+    mb.mlora_sync_status(gm.ctx)
+    compare_kv(gm, orc, cfg, 8)
+    gm.close()
+
+
 def test_adapter_switch_without_recreate(GpuModel):
     """Adapters are run-time inputs: swapping a slot's tensors changes the next step, clearing gives the base."""
     cfg = TINYV
