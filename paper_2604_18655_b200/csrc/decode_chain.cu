@@ -465,6 +465,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
   int pos = 0;                                        // stages of this CTA consumed (or skipped) so far
   unsigned long long n_bar = 0;                       // barriers passed in this launch
   unsigned n_shr = 0;                                 // LoRA phases passed in this launch
+  unsigned shr_target = 0;                          // count-ins of shrink warps in the phases before this one
   float* redf = reinterpret_cast<float*>(red);
 #ifdef CHAIN_TRACE
   const int tr_slot = blockIdx.x == 0 ? 0 : (blockIdx.x == G - 1 ? 1 : -1);
@@ -491,9 +492,21 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     if (teams > nstages / (tpu * L.nchunks)) teams = nstages / (tpu * L.nchunks);
     if (nseg > 0 && teams > CH_BS_BYTES / (tpu * CHAIN_MAX_ROWS * r * 32)) teams = CH_BS_BYTES / (tpu * CHAIN_MAX_ROWS * r * 32);
     if (teams < 1) teams = 1;
-    const int wpt = CH_CWARPS / teams;                                // warps per team
+    // LoRA phases: the CTA's shrink items (row, segment, rank index) run on the last shr_warps warps, off the
+    // critical path of the GEMM teams, which share the other warps
+    int n_my_items = 0;
+    if (nseg > 0) {
+      const int n_items = M * nseg * r;
+      n_my_items = (n_items > (int)blockIdx.x) ? (n_items - 1 - (int)blockIdx.x) / (int)G + 1 : 0;
+      if (n_my_items > CH_MAX_ITEMS) n_my_items = CH_MAX_ITEMS;
+    }
+    const int shr_warps = nseg > 0 ? (n_my_items < 4 ? (n_my_items > 0 ? n_my_items : 1) : 4) : 0;
+    const int gemm_warps = CH_CWARPS - shr_warps;
+    if (teams > gemm_warps) teams = gemm_warps;
+    const int wpt = gemm_warps / teams;                               // warps per team
     const int tm = warp / wpt, member = warp - tm * wpt;
     const bool in_team = tm < teams;
+    const int shr_id = warp - gemm_warps;                             // >= 0: this warp is shrink warp shr_id
     const int team_threads = wpt * 32, tt = member * 32 + lane;
     __half* Bs_team = Bs + (size_t)tm * tpu * CHAIN_MAX_ROWS * r * 16;
     auto team_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(2 + tm), "r"(team_threads) : "memory"); };
@@ -564,18 +577,16 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     if (warp == CH_CWARPS - 1 && p + 1 < a.p1) prep_phase(p + 1);
 
     // ---- 3. LoRA shrink (first factor of the low-rank term of Eq. 1-4): items (row, segment, rank index)
-    // are dealt round-robin to the CTAs; item k of the CTA belongs to warp k % 16
+    // are dealt round-robin to the CTAs; item k of the CTA belongs to shrink warp k % shr_warps
     if (nseg > 0) {
-      const int n_items = M * nseg * r;
       const int np = (K + CH_A_PIECE - 1) / CH_A_PIECE;
-      int n_my = 0;
-      bool wrote = false;
-      for (int i = blockIdx.x; i < n_items && n_my < CH_MAX_ITEMS; i += G, ++n_my) {
+      for (int k = 0; k < n_my_items; ++k) {
+        const int i = blockIdx.x + k * (int)G;
         const int seg = (i / r) % nseg, m = i / (r * nseg);
         if (s_pA[slot][seg][m] == nullptr) continue;
-        if (n_my % CH_CWARPS == warp) {
+        if (shr_id >= 0 && k % shr_warps == shr_id) {
           const __half* hrow = hs + (size_t)m * hs_stride;
-          float acc = 0.f;
+          float acc4[4] = {0.f, 0.f, 0.f, 0.f};
           for (int q = 0; q < np; ++q) {
             const int k0 = q * CH_A_PIECE;
             const int st = pos_stage(pos + q, nstages);
@@ -593,8 +604,8 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
 #pragma unroll
                   for (int e = 0; e < 4; ++e) {
                     const float2 af = __half22float2(u32_as_h2(aw[e])), hf2 = __half22float2(u32_as_h2(hw[e]));
-                    acc = fmaf(af.x, hf2.x, acc);
-                    acc = fmaf(af.y, hf2.y, acc);
+                    acc4[e] = fmaf(af.x, hf2.x, acc4[e]);
+                    acc4[e] = fmaf(af.y, hf2.y, acc4[e]);
                   }
                 }
               }
@@ -602,20 +613,20 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
             __syncwarp();
             if (lane < CH_ITEMS_PER_CHUNK) mbar_arrive(smem_u32(empty_bar + st));
           }
-          acc = warp_sum(acc);
+          const float acc = warp_sum((acc4[0] + acc4[1]) + (acc4[2] + acc4[3]));
           if (lane == 0) __stcg(a.T + i, acc * s_scale[m]);
-          wrote = true;
         }
         pos += np;
       }
-      // the last warp of the CTA to get here tells the grid that this CTA's share of T is written; a warp that
-      // stored part of T makes it visible device-wide before it counts itself in
+      // the last shrink warp of the CTA to get here tells the grid that this CTA's share of T is written: its
+      // release is cumulative over the stores the other shrink warps ordered before their own count-in
       ++n_shr;
-      if (lane == 0) {
-        if (wrote) __threadfence();
+      if (shr_id >= 0 && lane == 0) {
+        __threadfence_block();
         const unsigned old = atomicAdd(&s_shr_cnt, 1u);
-        if (old == n_shr * CH_CWARPS - 1) red_release_add_u64(a.sync + 1, 1ull);
+        if (old == shr_target + (unsigned)shr_warps - 1u) red_release_add_u64(a.sync + 1, 1ull);
       }
+      shr_target += (unsigned)shr_warps;
     }
     STAMP(2);
 
@@ -745,10 +756,10 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
       consumer_sync();
       STAMP(7);
       if (tid == 0) {
-        __threadfence();
+        // the release is cumulative over what the CTA's threads wrote before the named barrier above; the
+        // acquire load inside wait_counter orders the next phase's reads after the other CTAs' writes
         red_release_add_u64(a.sync + 0, 1ull);
         wait_counter(a.sync + 0, s_base[0] + n_bar * G, wc, 5, p);
-        __threadfence();
       }
       consumer_sync();
     }
