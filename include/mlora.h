@@ -168,6 +168,23 @@ int mlora_linear(mlora_weight* w, const void* x, int32_t M, const int32_t* row_a
                  const void* const* B, const float* scale, int32_t n_adapters, int32_t rank, float* y,
                  void* workspace, size_t workspace_bytes);
 
+/* Allocation-free variant of mlora_linear for at most 8 rows (the paper has no counterpart: this is a
+ * convenience of this library).  It is meant for callers that must not allocate device memory when they
+ * issue work: a serving loop whose memory was reserved up front and that cannot afford the device-wide
+ * synchronisation an allocation may cause, or code that holds no allocator at all at that point.  Same
+ * operation, arguments and result as mlora_linear, but the kernel's scratch (its barrier words and the LoRA
+ * intermediate) is a 4096-byte array built into the library, present on every GPU that loads it; the call
+ * itself makes no cudaMalloc/cudaFree and calls no allocating routine.  (mlora_weight_create, done once
+ * beforehand, does allocate.)
+ * Limits: 1 <= M <= 8, rank <= 64, and an input width K small enough for the single-kernel path (K <= 8192
+ * on a B200); anything beyond returns MLORA_ERR_CAPACITY and runs nothing -- use mlora_linear there.
+ * The first call on a device looks up the array's device address; make that call outside any stream capture.
+ * All calls on a device share the one array: two calls that overlap on the GPU (different streams) race;
+ * calls on the weight's own stream, or otherwise ordered, are fine.
+ * Errors: ARG, CAPACITY, UNSUPPORTED, CUDA. */
+int mlora_linear_noalloc(mlora_weight* w, const void* x, int32_t M, const int32_t* row_adapter, const void* const* A,
+                         const void* const* B, const float* scale, int32_t n_adapters, int32_t rank, float* y);
+
 /* Bytes of scratch for mlora_attention. */
 size_t mlora_attention_workspace_bytes(int32_t n_streams, int32_t n_nodes, int32_t n_q_heads, int32_t n_kv_heads,
                                        int32_t head_dim, int32_t prefix_len, int32_t own_capacity);

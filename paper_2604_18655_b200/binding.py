@@ -65,6 +65,8 @@ _SIGS = {
     "mlora_linear_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int32, C.c_int32]),
     "mlora_linear": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_size_t]),
+    "mlora_linear_noalloc": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                       C.c_int32, C.c_int32, C.c_void_p]),
     "mlora_attention_workspace_bytes": (C.c_size_t, [C.c_int32] * 7),
     "mlora_attention": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
                                   C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
@@ -231,6 +233,13 @@ def mlora_linear(w, x, y, workspace, row_adapter=None, A_ptrs=None, B_ptrs=None,
     n_ad = 0 if A_ptrs is None else A_ptrs.numel()
     _check(lib().mlora_linear(w, _ptr(x), x.shape[0], _ptr(row_adapter), _ptr(A_ptrs), _ptr(B_ptrs), _ptr(scale),
                               n_ad, rank, _ptr(y), _ptr(workspace), workspace.numel() * workspace.element_size()))
+
+
+def mlora_linear_noalloc(w, x, y, row_adapter=None, A_ptrs=None, B_ptrs=None, scale=None, rank=0):
+    """mlora_linear for at most 8 rows with the scratch built into the library: the call allocates nothing."""
+    n_ad = 0 if A_ptrs is None else A_ptrs.numel()
+    _check(lib().mlora_linear_noalloc(w, _ptr(x), x.shape[0], _ptr(row_adapter), _ptr(A_ptrs), _ptr(B_ptrs),
+                                      _ptr(scale), n_ad, rank, _ptr(y)))
 
 
 def mlora_attention_workspace_bytes(n, T, Hq, Hkv, hd, P, own_capacity):

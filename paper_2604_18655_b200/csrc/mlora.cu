@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <string>
 #include <unordered_map>
 #include <vector>
@@ -1081,6 +1082,61 @@ int mlora_linear(mlora_weight* w, const void* x, int32_t M, const int32_t* row_a
   g.counters = (unsigned*)(ws + LIN_SYNC_BYTES);
   g.lora = la;
   CK(launch_gemm(g, w->stream));
+  return MLORA_OK;
+}
+
+// ----------------------------------------------------------------------------- allocation-free projection
+// Scratch of mlora_linear_noalloc: the persistent kernel's barrier words and status (first 64 bytes) and the
+// LoRA intermediate T (8 rows x rank 64 floats at most).  Lives in every GPU that loads the library.
+static const size_t NOALLOC_SCRATCH_BYTES = 4096;
+static const size_t NOALLOC_HEAD_BYTES = 64;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
+static const int NOALLOC_MAX_DEVICES = 64;
+static void* g_noalloc_ptr[NOALLOC_MAX_DEVICES];      // device address of the array on each device, once asked for
+static std::mutex g_noalloc_mutex;
+
+int mlora_linear_noalloc(mlora_weight* w, const void* x, int32_t M, const int32_t* row_adapter, const void* const* A,
+                         const void* const* B, const float* scale, int32_t n_adapters, int32_t rank, float* y) {
+  if (!w || !x || !y) return fail(MLORA_ERR_ARG, "null argument");
+  const bool lora = row_adapter != nullptr;
+  if (lora && (!A || !B || !scale || n_adapters <= 0 || rank <= 0)) return fail(MLORA_ERR_ARG, "incomplete adapter arguments");
+  if (M < 1 || M > CHAIN_MAX_ROWS) return fail(MLORA_ERR_CAPACITY, "mlora_linear_noalloc takes 1..8 rows");
+  if (lora && rank > CHAIN_MAX_RANK) return fail(MLORA_ERR_CAPACITY, "mlora_linear_noalloc takes LoRA ranks up to 64");
+  if (NOALLOC_HEAD_BYTES + (size_t)M * (lora ? rank : 1) * sizeof(float) > NOALLOC_SCRATCH_BYTES)
+    return fail(MLORA_ERR_CAPACITY, "rows x rank exceeds the built-in scratch");
+  const int stages = chain_pick_stages(w->w.K, lora ? rank : 0);
+  if (stages <= 0 || !chain_phase_fits(w->w.K, MODE_PLAIN, lora ? 1 : 0, rank, stages, w->sm_count))
+    return fail(MLORA_ERR_CAPACITY, "input width too large for the built-in scratch path: use mlora_linear");
+  int dev = 0;
+  CK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return fail(MLORA_ERR_UNSUPPORTED, "device ordinal out of range");
+  void* scratch = nullptr;
+  {
+    // the array's name is only a host-side handle: ask the runtime, once per device and with that device
+    // current, where the array lives on the device
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (g_noalloc_ptr[dev] == nullptr) {
+      void* ptr = nullptr;
+      CK(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+      g_noalloc_ptr[dev] = ptr;
+    }
+    scratch = g_noalloc_ptr[dev];
+  }
+  // barrier words, abort flag and status start from zero on every call (the array keeps the last call's contents)
+  CK(cudaMemsetAsync(scratch, 0, NOALLOC_HEAD_BYTES, w->stream));
+  unsigned char* ws = (unsigned char*)scratch;
+  ChainArgs a{};
+  a.phases = w->phase; a.p0 = 0; a.p1 = 1; a.M = M; a.logits = y; a.h_in = (const __half*)x;
+  if (lora) {
+    a.adapter_idx = row_adapter; a.rows_per_stream = 1;
+    a.tabA = (const __half* const*)A; a.tabB = (const __half* const*)B; a.scale = scale;
+    a.tab_stride = 1; a.n_slots = n_adapters; a.rank = rank;
+  }
+  a.T = (float*)(ws + NOALLOC_HEAD_BYTES);
+  a.sync = (unsigned long long*)ws;
+  a.status = (int*)(ws + 32);
+  a.nstages = stages; a.kmax = w->w.K;
+  CK(launch_chain(a, w->sm_count, w->stream));
   return MLORA_OK;
 }
 
