@@ -26,9 +26,9 @@ sys.path.insert(0, ROOT)
 
 GEN_STEPS = 128          # decode steps per generation (per stream) before the streams are reset
 ORACLE_PREFIX = 64       # prompt length used for the CPU-baseline sample (the 512-token prefill is not timed work)
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the GEMM kernel, from the ncu capture summarised in
-# profiles/ (None until captured)
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of decode_chain_kernel, averaged over the 17 launches of
+# a full-model step, from the ncu capture summarised in profiles/decode_chain_kernel_llama1b_cut4L_8streams.md
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = 32.8e6
 
 
 def parse_args():
@@ -39,6 +39,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="cfg1", choices=["cfg0", "cfg1"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="profiling aid: cut the model to this many layers (small ncu captures); not a bench result")
     return ap.parse_args()
 
 
@@ -208,6 +210,8 @@ def main():
     args = parse_args()
     import gen
     cfg = {"cfg0": gen.CFG0, "cfg1": gen.CFG1}[args.config]
+    if args.layers is not None:
+        cfg = cfg.small(n_layers=args.layers, name=f"{cfg.name}-cut{args.layers}L")
     if args.impl == "reference":
         run_reference(args, cfg)
         return
