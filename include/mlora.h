@@ -136,13 +136,15 @@ int mlora_export_kv(mlora_ctx* ctx, int32_t layer, int32_t stream, int32_t first
 int mlora_debug_dequant(mlora_ctx* ctx, int32_t layer, int32_t proj, void* out_fp16);
 /* Debug switches: key 1 = skip KV compaction and suffix growth in mlora_verify_tree (tree rows stay where
  * the pass wrote them: rows suffix_len .. suffix_len + n_nodes - 1 of the own segment).
- * key 2 = 1 disables CUDA-graph replay of steps (every kernel launched directly). */
+ * key 2 = 1 disables CUDA-graph replay of steps (every kernel launched directly).
+ * key 3 = 1 runs decode-sized passes through the one-kernel-per-projection path instead of the persistent kernel. */
 int mlora_debug_set(mlora_ctx* ctx, int32_t key, int32_t value);
 /* Per-kernel-family device time of the NEXT steps, measured with CUDA events on the context's stream.
  * mlora_profile_begin switches to direct launches with an event pair around every kernel; mlora_profile_end
  * synchronises, switches back, and fills ms[family] / launches[family] (host arrays of MLORA_PROF_FAMILIES). */
 enum { MLORA_PROF_GEMM = 0, MLORA_PROF_SHRINK = 1, MLORA_PROF_ATTN = 2, MLORA_PROF_ATTN_MERGE = 3,
-       MLORA_PROF_ROPE_KV = 4, MLORA_PROF_MISC = 5, MLORA_PROF_FAMILIES = 6 };
+       MLORA_PROF_ROPE_KV = 4 /* unused: RoPE and the KV append run inside the attention kernel */, MLORA_PROF_MISC = 5,
+       MLORA_PROF_FAMILIES = 6 };
 int mlora_profile_begin(mlora_ctx* ctx);
 int mlora_profile_end(mlora_ctx* ctx, float* ms, int32_t* launches);
 /* Kernels launched by this context since creation (direct launches plus graph-replayed nodes). */

@@ -36,6 +36,32 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(sa));
 }
 
+// eight consecutive elements c..c+7 of one head of a projection row, rotated (pairs (i, i + hd/2), Sec. 3.1) or not.
+// All loads are issued before the first use; the row was written by another kernel or CTA: read through L2.
+__device__ __forceinline__ uint4 head_piece_f16(const float* __restrict__ head, int c, int hd, const float2* __restrict__ cs) {
+  const float4 x0 = __ldcg(reinterpret_cast<const float4*>(head + c));
+  const float4 x1 = __ldcg(reinterpret_cast<const float4*>(head + c + 4));
+  float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+  if (cs != nullptr) {
+    const int half = hd >> 1;
+    const bool lo = c < half;                          // a piece never straddles the middle: c and hd/2 are multiples of 8
+    const int pc = lo ? c + half : c - half;           // the partner piece
+    const float4 y0 = __ldcg(reinterpret_cast<const float4*>(head + pc));
+    const float4 y1 = __ldcg(reinterpret_cast<const float4*>(head + pc + 4));
+    const float4* t4 = reinterpret_cast<const float4*>(cs + (lo ? c : pc));
+    const float4 t0 = __ldg(t4), t1 = __ldg(t4 + 1), t2 = __ldg(t4 + 2), t3 = __ldg(t4 + 3);
+    const float y[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
+    const float co[8] = {t0.x, t0.z, t1.x, t1.z, t2.x, t2.z, t3.x, t3.z};
+    const float si[8] = {t0.y, t0.w, t1.y, t1.w, t2.y, t2.w, t3.y, t3.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = lo ? v[i] * co[i] - y[i] * si[i] : v[i] * co[i] + y[i] * si[i];
+  }
+  __half2 o[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) o[i] = __halves2half2(__float2half_rn(v[2 * i]), __float2half_rn(v[2 * i + 1]));
+  return make_uint4(h2_as_u32(o[0]), h2_as_u32(o[1]), h2_as_u32(o[2]), h2_as_u32(o[3]));
+}
+
 struct AttnItem {
   int is_own, s, chunk, row_block;
 };
@@ -59,8 +85,8 @@ __device__ __forceinline__ AttnItem decode_item(const AttnArgs& p, int item, int
 }
 
 template <int HD>
-__global__ void __launch_bounds__(ATT_THREADS) attn_partial_kernel(const AttnArgs p, const int rb_all, const int rb_own,
-                                                                  const float scale_log2) {
+__device__ __forceinline__ void attn_partial_body(const AttnArgs& p, const int rb_all, const int rb_own,
+                                                  const float scale_log2) {
   constexpr int STRIDE = HD + 8;                      // halves per shared-memory row
   constexpr int KSTEPS = HD / 16;
   constexpr int DT = HD / 8;                          // output n8-tiles
@@ -71,6 +97,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_partial_kernel(const AttnArg
 
   const int kh = blockIdx.y;
   const int g_heads = p.Hq / p.Hkv;
+  const bool fused = p.qkv_f32 != nullptr;
   const AttnItem it = decode_item(p, blockIdx.x, rb_all, rb_own);
   const int rows_per_stream = p.T * g_heads;
   const int R_all = p.n * rows_per_stream;
@@ -109,9 +136,29 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_partial_kernel(const AttnArg
     constexpr int VPR = HD / 8;                                        // 16-byte pieces per row
     for (int i = threadIdx.x; i < ATT_KEYS * VPR; i += ATT_THREADS) {
       const int r = i / VPR, c = (i % VPR) * 8;
-      const int key = min(k0 + r, key_end - 1);                        // rows past the end repeat the last valid key
-      cp_async16(kd + (size_t)r * STRIDE + c, kbase + (size_t)key * HD + c);
-      cp_async16(vd + (size_t)r * STRIDE + c, vbase + (size_t)key * HD + c);
+      const int key = k0 + r;
+      if (key >= key_end) {
+        // rows past the end of the chunk: zeros (their scores are masked; a zero V row keeps 0 * v finite)
+        *reinterpret_cast<uint4*>(kd + (size_t)r * STRIDE + c) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(vd + (size_t)r * STRIDE + c) = make_uint4(0, 0, 0, 0);
+      } else if (fused && it.is_own && key >= S) {
+        // a row of this pass: not in the cache yet -- build it from the projections (k rotated), use it, and let
+        // the first row block of the chunk append it to the stream's own segment
+        const int m = it.s * p.T + (key - S);
+        const float* row = p.qkv_f32 + (size_t)m * (size_t)((p.Hq + 2 * p.Hkv) * HD);
+        const float2* cs = p.cs_table + (size_t)(p.pos_base + S + p.depth[m]) * (HD / 2);
+        const uint4 kv8 = head_piece_f16(row + (size_t)(p.Hq + kh) * HD, c, HD, cs);
+        const uint4 vv8 = head_piece_f16(row + (size_t)(p.Hq + p.Hkv + kh) * HD, c, HD, nullptr);
+        *reinterpret_cast<uint4*>(kd + (size_t)r * STRIDE + c) = kv8;
+        *reinterpret_cast<uint4*>(vd + (size_t)r * STRIDE + c) = vv8;
+        if (it.row_block == 0) {
+          *reinterpret_cast<uint4*>(const_cast<__half*>(kbase) + (size_t)key * HD + c) = kv8;
+          *reinterpret_cast<uint4*>(const_cast<__half*>(vbase) + (size_t)key * HD + c) = vv8;
+        }
+      } else {
+        cp_async16(kd + (size_t)r * STRIDE + c, kbase + (size_t)key * HD + c);
+        cp_async16(vd + (size_t)r * STRIDE + c, vbase + (size_t)key * HD + c);
+      }
     }
   };
 
@@ -127,7 +174,13 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_partial_kernel(const AttnArg
       uint4 val = make_uint4(0, 0, 0, 0);
       if (v < row_hi) {
         const int m = v / g_heads, j = v % g_heads;
-        val = *reinterpret_cast<const uint4*>(p.q + ((size_t)m * p.Hq + kh * g_heads + j) * HD + c);
+        if (fused) {
+          const float* row = p.qkv_f32 + (size_t)m * (size_t)((p.Hq + 2 * p.Hkv) * HD);
+          const float2* cs = p.cs_table + (size_t)(p.pos_base + p.suffix_len[m / p.T] + p.depth[m]) * (HD / 2);
+          val = head_piece_f16(row + (size_t)(kh * g_heads + j) * HD, c, HD, cs);
+        } else {
+          val = *reinterpret_cast<const uint4*>(p.q + ((size_t)m * p.Hq + kh * g_heads + j) * HD + c);
+        }
       }
       *reinterpret_cast<uint4*>(Qs + (size_t)r * STRIDE + c) = val;
     }
@@ -264,6 +317,86 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_partial_kernel(const AttnArg
   }
 }
 
+// log-sum-exp merge of the chunks of virtual row v (row m, query head hq) of kv head kh by one warp.  The lanes
+// take the chunks' (max, sum) pairs side by side; the weighted sum over chunks runs in chunk order with
+// independent loads.
+__device__ __forceinline__ void merge_row(const AttnArgs& p, int kh, int v, int m, int hq, int lane) {
+  const int g_heads = p.Hq / p.Hkv;
+  const int R_all = p.n * p.T * g_heads;
+  const int slots = p.n_prefix_chunks + p.n_own_chunks;
+  const int s = m / p.T;
+  const int own_valid = min(p.n_own_chunks, (p.suffix_len[s] + p.T + p.own_chunk - 1) / p.own_chunk);
+  const int n_valid = p.n_prefix_chunks + own_valid;
+  const size_t base = ((size_t)kh * R_all + v) * slots;
+  const int hd = p.hd;
+  __half* out = p.out + ((size_t)m * p.Hq + hq) * hd;
+  constexpr int FAST = 12;                             // chunks whose partial outputs fit in registers
+  if (n_valid <= FAST && hd <= 128) {
+    // one round trip: every load is issued before the first use
+    float2 ml = make_float2(-INFINITY, 0.f);
+    if (lane < n_valid) ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (base + lane) * 2));
+    float po[FAST][4];
+#pragma unroll
+    for (int i = 0; i < FAST; ++i)
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        po[i][e] = (i < n_valid && e * 32 + lane < hd) ? __ldcg(p.part_o + (base + i) * hd + e * 32 + lane) : 0.f;
+    float mmax = ml.x;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, o));
+    const float wgt = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - mmax);
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float L = 0.f;
+#pragma unroll
+    for (int i = 0; i < FAST; ++i) {                                     // fixed order: chunk 0, 1, ...
+      const float wi = __shfl_sync(0xffffffffu, wgt, i);
+      L = fmaf(wi, __shfl_sync(0xffffffffu, ml.y, i), L);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[e] = fmaf(wi, po[i][e], acc[e]);
+    }
+    const float inv = 1.f / L;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (e * 32 + lane < hd) out[e * 32 + lane] = __float2half_rn(acc[e] * inv);
+    return;
+  }
+  float mmax = -INFINITY;
+  for (int i = lane; i < n_valid; i += 32) mmax = fmaxf(mmax, __ldcg(p.part_ml + (base + i) * 2));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, o));
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  float L = 0.f;
+  for (int i0 = 0; i0 < n_valid; i0 += 32) {
+    // lane i0 + lane holds the weight and the sum of its chunk
+    float wgt = 0.f, lsum = 0.f;
+    if (i0 + lane < n_valid) {
+      const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (base + i0 + lane) * 2));
+      wgt = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - mmax);
+      lsum = ml.y;
+    }
+    const int cnt = min(32, n_valid - i0);
+#pragma unroll 4
+    for (int i = 0; i < cnt; ++i) {                                      // fixed order: chunk 0, 1, ...
+      const float wi = __shfl_sync(0xffffffffu, wgt, i);
+      L = fmaf(wi, __shfl_sync(0xffffffffu, lsum, i), L);
+      const float* po = p.part_o + (base + i0 + i) * hd;
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (e * 32 + lane < hd) acc[e] = fmaf(wi, __ldcg(po + e * 32 + lane), acc[e]);
+    }
+  }
+  const float inv = 1.f / L;
+#pragma unroll
+  for (int e = 0; e < 4; ++e)
+    if (e * 32 + lane < hd) out[e * 32 + lane] = __float2half_rn(acc[e] * inv);
+}
+
+template <int HD>
+__global__ void __launch_bounds__(ATT_THREADS) attn_partial_kernel(const AttnArgs p, const int rb_all, const int rb_own,
+                                                                  const float scale_log2) {
+  attn_partial_body<HD>(p, rb_all, rb_own, scale_log2);
+}
+
 // One warp per (row, query head): log-sum-exp merge of the row's chunks, output in fp16.
 __global__ void attn_merge_kernel(const AttnArgs p) {
   const int w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -272,28 +405,7 @@ __global__ void attn_merge_kernel(const AttnArgs p) {
   if (w >= M * p.Hq) return;
   const int m = w / p.Hq, hq = w % p.Hq;
   const int g_heads = p.Hq / p.Hkv;
-  const int kh = hq / g_heads;
-  const int v = m * g_heads + hq % g_heads;
-  const int s = m / p.T;
-  const int R_all = M * g_heads;
-  const int slots = p.n_prefix_chunks + p.n_own_chunks;
-  const int own_valid = min(p.n_own_chunks, (p.suffix_len[s] + p.T + p.own_chunk - 1) / p.own_chunk);
-  const size_t base = ((size_t)kh * R_all + v) * slots;
-  float mmax = -INFINITY;
-  for (int i = 0; i < p.n_prefix_chunks + own_valid; ++i) mmax = fmaxf(mmax, p.part_ml[(base + i) * 2]);
-  const int hd = p.hd;
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  float L = 0.f;
-  for (int i = 0; i < p.n_prefix_chunks + own_valid; ++i) {
-    const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + (base + i) * 2);
-    const float wgt = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - mmax);
-    L += wgt * ml.y;
-    const float* po = p.part_o + (base + i) * hd;
-    for (int e = 0; e * 32 + lane < hd; ++e) acc[e] = fmaf(wgt, po[e * 32 + lane], acc[e]);
-  }
-  const float inv = 1.f / L;
-  __half* out = p.out + ((size_t)m * p.Hq + hq) * hd;
-  for (int e = 0; e * 32 + lane < hd; ++e) out[e * 32 + lane] = __float2half_rn(acc[e] * inv);
+  merge_row(p, hq / g_heads, m * g_heads + hq % g_heads, m, hq, lane);
 }
 
 void attn_plan(AttnArgs& a, int sm_count) {

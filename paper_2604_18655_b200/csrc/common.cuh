@@ -125,6 +125,12 @@ struct AttnArgs {
   float* part_o; float* part_ml;  // scratch
   int n_prefix_chunks, prefix_chunk; // keys per prefix chunk (multiple of 64)
   int n_own_chunks, own_chunk;
+  // fused mode (qkv_f32 != nullptr): q and the pass's new k rows are rotated here (RoPE, Sec. 3.1) and the new K/V
+  // rows are written to the own segment by the CTA that owns their chunk; q is not read
+  const float* qkv_f32;           // [rows][(Hq + 2 Hkv) * hd] fp32 projections
+  const float2* cs_table;         // cos/sin of pos * theta^(-2i/hd): [pos][hd/2]
+  int pos_base;                   // position of a row = pos_base + suffix_len[s] + depth[row]
+  const int32_t* depth;           // dev [rows]
 };
 
 // ----------------------------------------------------------------------------- persistent projection chain
@@ -191,9 +197,6 @@ cudaError_t launch_embed(const int32_t* tokens, const __half* embed, const __hal
                          int d, int vocab, int* status, cudaStream_t st);
 cudaError_t launch_tree_prep(const int32_t* parent, int n, int T, unsigned long long* anc, int32_t* depth,
                              int* status, cudaStream_t st);
-cudaError_t launch_rope_kv(const float* qkv, int M, int T, int Hq, int Hkv, int hd, const float2* cs_table,
-                           int pos_base, const int32_t* suffix_len, const int32_t* depth, __half* q_out,
-                           __half* k_dst, __half* v_dst, size_t stream_stride, size_t head_stride, cudaStream_t st);
 void attn_plan(AttnArgs& a, int sm_count);
 size_t attn_workspace_floats(const AttnArgs& a);
 cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st);

@@ -72,7 +72,7 @@ struct mlora_ctx {
   size_t own_layer_stride = 0, own_stream_stride = 0, own_head_stride = 0;
   // scratch
   float *X = nullptr, *qkv = nullptr, *logits = nullptr, *T = nullptr, *partial = nullptr, *att_ws = nullptr;
-  __half *h = nullptr, *q16 = nullptr, *attn16 = nullptr, *act16 = nullptr;
+  __half *h = nullptr, *attn16 = nullptr, *act16 = nullptr;
   size_t partial_floats = 0, att_ws_floats = 0;
   unsigned* counters = nullptr;
   unsigned long long* anc = nullptr;
@@ -202,18 +202,13 @@ void kv_destination(mlora_ctx* c, const PassIO& io, int l, __half*& kd, __half*&
 }
 
 int launch_attention_block(mlora_ctx* c, const PassIO& io, int l) {
-  const mlora_model_desc& d = c->d;
   cudaStream_t st = c->stream;
-  const int M = io.n * io.T, hd = d.head_dim;
   __half *kd, *vd;
   size_t sstride, hstride;
   kv_destination(c, io, l, kd, vd, sstride, hstride);
-  CK(run(c, MLORA_PROF_ROPE_KV, [&] {
-    return launch_rope_kv(c->qkv, M, io.T, d.n_q_heads, d.n_kv_heads, hd, c->cs_table, io.pos_base, io.suffix_len,
-                          c->depth, c->q16, kd, vd, sstride, hstride, st);
-  }));
   AttnArgs a = io.plan;
-  a.q = c->q16;
+  // q and the new k rows are rotated on load, the new K/V rows appended by the attention kernel itself
+  a.qkv_f32 = c->qkv; a.cs_table = c->cs_table; a.pos_base = io.pos_base; a.depth = c->depth;
   a.prefix_k = c->prefix_k + (size_t)l * c->prefix_layer_stride;
   a.prefix_v = c->prefix_v + (size_t)l * c->prefix_layer_stride;
   a.prefix_head_stride = c->prefix_head_stride;
@@ -564,7 +559,6 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
   CKC(cudaMalloc(&c->X, Mm * dm * sizeof(float)));
   CKC(cudaMalloc(&c->qkv, Mm * c->Nqkv * sizeof(float)));
   CKC(cudaMalloc(&c->h, Mm * maxK * sizeof(__half)));
-  CKC(cudaMalloc(&c->q16, Mm * Nq * sizeof(__half)));
   CKC(cudaMalloc(&c->attn16, Mm * Nq * sizeof(__half)));
   CKC(cudaMalloc(&c->act16, Mm * F * sizeof(__half)));
   if (d.vocab > 0) CKC(cudaMalloc(&c->logits, Mm * d.vocab * sizeof(float)));
@@ -696,7 +690,7 @@ int mlora_destroy(mlora_ctx* c) {
   for (auto& w : c->w_down) free_packed(w);
   free_packed(c->w_lm);
   void* dev_ptrs[] = {c->prefix_k, c->prefix_v, c->own_k, c->own_v, c->X, c->qkv, c->logits, c->T, c->partial, c->att_ws,
-                      c->h, c->q16, c->attn16, c->act16, c->counters, c->anc, c->depth, c->argmax, c->suffix_len,
+                      c->h, c->attn16, c->act16, c->counters, c->anc, c->depth, c->argmax, c->suffix_len,
                       c->zero_len, c->chain_parent, c->root_parent, c->status, c->cs_table, (void*)c->tabA,
                       (void*)c->tabB, c->ad_scale, c->phases, c->chain_sync};
   for (void* p : dev_ptrs) if (p) cudaFree(p);

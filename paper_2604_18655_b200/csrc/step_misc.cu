@@ -1,6 +1,6 @@
 // Small kernels around the projections: embedding gather, draft-tree preparation (ancestor masks and
-// depths, Sec. 3.5 / App. A.2), RoPE + KV append (Sec. 3.1), row argmax, the greedy longest-accepted-path
-// walk and the KV compaction that follows it (Sec. 3.5).
+// depths, Sec. 3.5 / App. A.2), row argmax, the greedy longest-accepted-path walk and the KV compaction that
+// follows it (Sec. 3.5).  (RoPE and the KV append of a pass happen inside the attention kernel.)
 #include "common.cuh"
 
 namespace mlora {
@@ -63,50 +63,6 @@ cudaError_t launch_tree_prep(const int32_t* parent, int n, int T, unsigned long 
                              cudaStream_t st) {
   const int total = n * T;
   tree_prep_kernel<<<(total + 127) / 128, 128, 0, st>>>(parent, n, T, anc, depth, status);
-  return cudaGetLastError();
-}
-
-// ----------------------------------------------------------------------------- RoPE + KV append
-// Row m = s*T + t sits at position pos_base + suffix_len[s] + depth[m]; q and k rotate in (i, i + hd/2) pairs.
-// q goes to fp16 [M][Hq][hd]; k and v go to slot suffix_len[s] + t of the stream's own segment.
-__global__ void rope_kv_kernel(const float* __restrict__ qkv, int T, int Hq, int Hkv, int hd,
-                               const float2* __restrict__ cs_table, int pos_base, const int32_t* __restrict__ suffix_len,
-                               const int32_t* __restrict__ depth, __half* __restrict__ q_out, __half* __restrict__ k_dst,
-                               __half* __restrict__ v_dst, size_t stream_stride, size_t head_stride) {
-  const int m = blockIdx.x;
-  const int s = m / T, t = m % T;
-  const int S = suffix_len[s];
-  const int pos = pos_base + S + depth[m];
-  const int half = hd >> 1;
-  const int Nq = Hq * hd, Nkv = Hkv * hd;
-  const float* row = qkv + (size_t)m * (Nq + 2 * Nkv);
-  const float2* cs = cs_table + (size_t)pos * half;
-  // q heads and k heads: one thread per rotation pair
-  for (int i = threadIdx.x; i < (Hq + Hkv) * half; i += blockDim.x) {
-    const int head = i / half, e = i % half;
-    const float2 c = cs[e];
-    const float* src = row + (size_t)head * hd;      // k heads follow the q heads in the fused row
-    const float x1 = src[e], x2 = src[e + half];
-    const __half o1 = __float2half_rn(x1 * c.x - x2 * c.y);
-    const __half o2 = __float2half_rn(x2 * c.x + x1 * c.y);
-    __half* dst;
-    if (head < Hq) dst = q_out + ((size_t)m * Hq + head) * hd;
-    else dst = k_dst + (size_t)s * stream_stride + (size_t)(head - Hq) * head_stride + (size_t)(S + t) * hd;
-    dst[e] = o1;
-    dst[e + half] = o2;
-  }
-  for (int i = threadIdx.x; i < Nkv; i += blockDim.x) {
-    const int head = i / hd, e = i % hd;
-    v_dst[(size_t)s * stream_stride + (size_t)head * head_stride + (size_t)(S + t) * hd + e] =
-        __float2half_rn(row[Nq + Nkv + i]);
-  }
-}
-
-cudaError_t launch_rope_kv(const float* qkv, int M, int T, int Hq, int Hkv, int hd, const float2* cs_table,
-                           int pos_base, const int32_t* suffix_len, const int32_t* depth, __half* q_out, __half* k_dst,
-                           __half* v_dst, size_t stream_stride, size_t head_stride, cudaStream_t st) {
-  rope_kv_kernel<<<M, 256, 0, st>>>(qkv, T, Hq, Hkv, hd, cs_table, pos_base, suffix_len, depth, q_out, k_dst, v_dst,
-                                   stream_stride, head_stride);
   return cudaGetLastError();
 }
 
