@@ -380,7 +380,7 @@ def main():
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "decode_chain_kernel (persistent INT4 GEMM + LoRA shrink/expand + norm), all launches of a step",
                      "achieved": achieved, "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH,
+                     "frac": achieved / peak, "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH if args.config == "cfg1" and args.layers is None else None,
                      "bytes_per_launch": gemm_bytes_step / gemm_per_step, "launches_per_step": gemm_per_step,
                      "us_per_launch": 1e3 * gemm_ms / max(gemm_launches, 1)},
         "step_roofline": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_bytes / (ms_step / 1e3) / 1e9,
