@@ -456,7 +456,8 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
   // The CTA's stages of a phase form one list (see "the ring schedule"); a consumer finds a stage by its
   // running count since the start of the launch.
   //   shrink item k   -> warp k % 16 reads all pieces of the row and frees each stage on its own
-  //   weight chunks   -> warps work in teams; team tm takes the CTA's units tm, tm + teams, ...; inside a unit
+  //   weight chunks   -> warps work in teams, formed anew for every round of units: in a round team tm takes the
+  //                      CTA's next unit number tm; inside a unit
   //                      every tile's k-tiles are cut into items of CH_ITEM_KT k-tiles and each member warp owns a
   //                      contiguous run of them, keeps their partial sums in registers and parks them in its own
   //                      slot; the team adds the slots in member order (fixed summation order) and runs the
@@ -503,12 +504,24 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     const int shr_warps = nseg > 0 ? (n_my_items < 4 ? (n_my_items > 0 ? n_my_items : 1) : 4) : 0;
     const int gemm_warps = CH_CWARPS - shr_warps;
     if (teams > gemm_warps) teams = gemm_warps;
-    const int wpt = gemm_warps / teams;                               // warps per team
-    const int tm = warp / wpt, member = warp - tm * wpt;
-    const bool in_team = tm < teams;
+    // the teams are formed anew for every round of units: the last round may have fewer units than teams, and
+    // then all GEMM warps share what is left
+    int teams_r = 0, wpt = 1, tm = 0, member = 0, team_threads = 32, tt = 0;
+    bool in_team = false;
+    __half* Bs_team = Bs;
+    auto form_teams = [&](int units_left) {
+      teams_r = units_left < teams ? units_left : teams;
+      if (teams_r < 1) teams_r = 1;
+      wpt = gemm_warps / teams_r;                                     // warps per team
+      tm = warp / wpt;
+      member = warp - tm * wpt;
+      in_team = tm < teams_r;
+      team_threads = wpt * 32;
+      tt = member * 32 + lane;
+      Bs_team = Bs + (size_t)tm * tpu * CHAIN_MAX_ROWS * r * 16;
+    };
+    form_teams(my_units);
     const int shr_id = warp - gemm_warps;                             // >= 0: this warp is shrink warp shr_id
-    const int team_threads = wpt * 32, tt = member * 32 + lane;
-    __half* Bs_team = Bs + (size_t)tm * tpu * CHAIN_MAX_ROWS * r * 16;
     auto team_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(2 + tm), "r"(team_threads) : "memory"); };
     // LoRA-B slices of unit u -> Bs_team[tile][m][j][16]; immutable, so no need to wait for activations
     auto issue_b = [&](int u) {
@@ -631,12 +644,19 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     STAMP(2);
 
     // ---- 4. the CTA's units: one n-tile (or a gate/up pair of n-tiles), all of K
-    if (in_team) {
-      bool t_loaded = false;
-      const int it_lo = (member * ipt) / wpt, it_hi = ((member + 1) * ipt) / wpt;   // this warp's items of a tile
-      for (int k = tm; k < my_units; k += teams) {
+    bool t_loaded = false;
+    for (int k0 = 0; k0 < my_units && warp < gemm_warps; k0 += teams_r) {
+      if (k0 > 0) {
+        // next round: every GEMM warp is done with the last one (partial sums, B slices and T are settled)
+        asm volatile("bar.sync 10, %0;" ::"r"(gemm_warps * 32) : "memory");
+        form_teams(my_units - k0);
+        t_loaded = true;
+      }
+      if (in_team) {
+        const int it_lo = (member * ipt) / wpt, it_hi = ((member + 1) * ipt) / wpt;   // this warp's items of a tile
+        const int k = k0 + tm;
         const int u = blockIdx.x + k * (int)G;
-        if (nseg > 0 && k != tm) issue_b(u);                              // the first unit's went out before the prologue
+        if (nseg > 0 && k0 > 0) issue_b(u);                               // the first round's went out before the prologue
         const int ubase = pos + k * tpu * L.nchunks;                      // first stage of the unit
         for (int tu = 0; tu < tpu; ++tu) {
           float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
