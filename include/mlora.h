@@ -103,6 +103,12 @@ int mlora_prefill_shared_h(mlora_ctx* ctx, const void* hidden, int32_t n, float*
  * Errors: ARG, STATE (no prefill yet), CAPACITY (own segment full). */
 int mlora_decode_step(mlora_ctx* ctx, int32_t n_streams, const int32_t* adapter_idx, const int32_t* tokens,
                       int32_t* out_next, float* out_logits);
+/* The same step for a caller that holds HOST arrays (Sec. 3.4; the application side of the paper's flow): copies
+ * adapter_idx and tokens (host int32 [n_streams], pinned or pageable) to the device on the context's stream,
+ * runs the step, copies the greedy next tokens back to out_next_host and synchronises the stream before
+ * returning.  Errors: as mlora_decode_step. */
+int mlora_decode_step_host(mlora_ctx* ctx, int32_t n_streams, const int32_t* adapter_idx_host,
+                           const int32_t* tokens_host, int32_t* out_next_host);
 /* Hidden-state variant: hidden_in dev fp16 [n_streams][d_model]; hidden_out dev fp32 [n_streams][d_model]
  * (residual stream after the last layer). */
 int mlora_decode_step_h(mlora_ctx* ctx, int32_t n_streams, const int32_t* adapter_idx, const void* hidden_in,

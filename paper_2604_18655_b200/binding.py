@@ -45,6 +45,7 @@ _SIGS = {
     "mlora_prefill_shared": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]),
     "mlora_prefill_shared_h": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]),
     "mlora_decode_step": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "mlora_decode_step_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "mlora_decode_step_h": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "mlora_verify_tree": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                     C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -159,6 +160,14 @@ def mlora_prefill_shared_h(ctx, hidden, out_last_hidden=None):
 def mlora_decode_step(ctx, adapter_idx, tokens, out_next, out_logits=None):
     _check(lib().mlora_decode_step(ctx, adapter_idx.numel(), _ptr(adapter_idx), _ptr(tokens), _ptr(out_next),
                                    _ptr(out_logits)))
+
+
+def mlora_decode_step_host(ctx, adapter_idx, tokens, out_next):
+    """Host-buffer form: the three arguments are CPU int32 tensors (pinned for asynchronous copies)."""
+    for t in (adapter_idx, tokens, out_next):
+        assert not t.is_cuda and t.is_contiguous() and t.dtype == torch.int32
+    _check(lib().mlora_decode_step_host(ctx, adapter_idx.numel(), C.c_void_p(adapter_idx.data_ptr()),
+                                        C.c_void_p(tokens.data_ptr()), C.c_void_p(out_next.data_ptr())))
 
 
 def mlora_decode_step_h(ctx, adapter_idx, hidden_in, hidden_out):

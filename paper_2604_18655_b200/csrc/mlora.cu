@@ -96,6 +96,7 @@ struct mlora_ctx {
   bool snap_pending = false;
   int snap_inc = 0;
   int dbg_skip_compact = 0, dbg_no_graph = 0, dbg_no_chain = 0;
+  int32_t* host_io = nullptr;        // dev [3][max_streams]: adapter_idx, tokens, next of the host-buffer step
   // persistent projection chain (rows <= 8)
   ChainPhase* phases = nullptr;      // dev [4*L (+1)]: qkv, o, gate/up, down per layer; then lm_head
   int n_phases = 0;
@@ -575,6 +576,7 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
     c->att_ws_floats = ((size_t)d.n_kv_heads * R_all * 2 + (size_t)256 * c->sm_count + 4096) * (hd + 2);
     CKC(cudaMalloc(&c->att_ws, c->att_ws_floats * sizeof(float)));
   }
+  CKC(cudaMalloc(&c->host_io, 3 * (size_t)d.max_streams * sizeof(int32_t)));
   CKC(cudaMalloc(&c->anc, Mm * sizeof(unsigned long long)));
   CKC(cudaMalloc(&c->depth, Mm * sizeof(int32_t)));
   CKC(cudaMalloc(&c->argmax, Mm * sizeof(int32_t)));
@@ -692,7 +694,7 @@ int mlora_destroy(mlora_ctx* c) {
   void* dev_ptrs[] = {c->prefix_k, c->prefix_v, c->own_k, c->own_v, c->X, c->qkv, c->logits, c->T, c->partial, c->att_ws,
                       c->h, c->attn16, c->act16, c->counters, c->anc, c->depth, c->argmax, c->suffix_len,
                       c->zero_len, c->chain_parent, c->root_parent, c->status, c->cs_table, (void*)c->tabA,
-                      (void*)c->tabB, c->ad_scale, c->phases, c->chain_sync};
+                      (void*)c->tabB, c->ad_scale, c->phases, c->chain_sync, c->host_io};
   for (void* p : dev_ptrs) if (p) cudaFree(p);
   if (c->stageA) cudaFreeHost((void*)c->stageA);
   if (c->stageB) cudaFreeHost((void*)c->stageB);
@@ -783,6 +785,25 @@ int mlora_decode_step(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_id
   if (c->d.vocab == 0) return fail(MLORA_ERR_STATE, "context has no vocabulary: use mlora_decode_step_h");
   if (!tokens || !out_next) return fail(MLORA_ERR_ARG, "tokens/out_next is null");
   return decode_impl(c, n_streams, adapter_idx, tokens, nullptr, out_next, out_logits, nullptr);
+}
+
+int mlora_decode_step_host(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_idx_host, const int32_t* tokens_host,
+                           int32_t* out_next_host) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (c->d.vocab == 0) return fail(MLORA_ERR_STATE, "context has no vocabulary");
+  if (!adapter_idx_host || !tokens_host || !out_next_host) return fail(MLORA_ERR_ARG, "null host buffer");
+  if (n_streams <= 0 || n_streams > c->d.max_streams) return fail(MLORA_ERR_ARG, "n_streams out of range");
+  int32_t* d_ad = c->host_io;
+  int32_t* d_tok = c->host_io + c->d.max_streams;
+  int32_t* d_next = c->host_io + 2 * (size_t)c->d.max_streams;
+  const size_t bytes = (size_t)n_streams * sizeof(int32_t);
+  CK(cudaMemcpyAsync(d_ad, adapter_idx_host, bytes, cudaMemcpyHostToDevice, c->stream));
+  CK(cudaMemcpyAsync(d_tok, tokens_host, bytes, cudaMemcpyHostToDevice, c->stream));
+  int rc = decode_impl(c, n_streams, d_ad, d_tok, nullptr, d_next, nullptr, nullptr);
+  if (rc != MLORA_OK) return rc;
+  CK(cudaMemcpyAsync(out_next_host, d_next, bytes, cudaMemcpyDeviceToHost, c->stream));
+  CK(cudaStreamSynchronize(c->stream));
+  return MLORA_OK;
 }
 
 int mlora_decode_step_h(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_idx, const void* hidden_in,

@@ -337,3 +337,29 @@ def test_decode_paths_agree(GpuModel):
     compare(res[1][0], res[0][0], "logits across paths")
     compare(res[1][1], res[0][1], "K across paths")
     compare(res[1][2], res[0][2], "V across paths")
+
+
+def test_host_buffer_step_matches_device_step(GpuModel):
+    """mlora_decode_step_host (host arrays in and out) gives the tokens of mlora_decode_step."""
+    from paper_2604_18655_b200 import binding as mb
+    cfg = TINYV
+    outs = []
+    for host in (False, True):
+        m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+        gm.prefill(gen.make_prompt_ids(cfg, 0))
+        toks = np.array([4, 9, 11], dtype=np.int32)
+        hist = []
+        for _ in range(4):
+            if host:
+                h_ad = torch.tensor([0, 1, -1], dtype=torch.int32).pin_memory()
+                h_tok = torch.from_numpy(toks.copy()).pin_memory()
+                h_next = torch.empty(3, dtype=torch.int32).pin_memory()
+                mb.mlora_decode_step_host(gm.ctx, h_ad, h_tok, h_next)
+                toks = h_next.numpy().copy()
+            else:
+                toks, _ = gm.decode([0, 1, -1], toks, want_logits=False)
+            hist.append(toks.copy())
+        outs.append(np.stack(hist))
+        mb.mlora_sync_status(gm.ctx)
+        gm.close()
+    assert np.array_equal(outs[0], outs[1])
