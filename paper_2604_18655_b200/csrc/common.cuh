@@ -192,6 +192,10 @@ cudaError_t launch_dequant(const unsigned char* w, int K, int N, int G, int tile
                            __half* out, cudaStream_t st);
 int gemm_pick_split(int K, int N, int M, size_t partial_capacity);
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
+// tcgen05 path for passes with 32 rows or more: partial sums on the tensor cores, then an epilogue kernel
+cudaError_t init_gemm_tc();
+bool gemm_tc_eligible(const GemmArgs& a);
+cudaError_t launch_gemm_tc(const GemmArgs& a, int sm_count, int* status, cudaStream_t st);
 cudaError_t launch_shrink(const ShrinkArgs& a, cudaStream_t st);
 cudaError_t launch_embed(const int32_t* tokens, const __half* embed, const __half* hidden_in, float* X, int M,
                          int d, int vocab, int* status, cudaStream_t st);

@@ -95,7 +95,7 @@ struct mlora_ctx {
   cudaEvent_t snap_event = nullptr;
   bool snap_pending = false;
   int snap_inc = 0;
-  int dbg_skip_compact = 0, dbg_no_graph = 0, dbg_no_chain = 0;
+  int dbg_skip_compact = 0, dbg_no_graph = 0, dbg_no_chain = 0, dbg_no_tc = 0;
   int32_t* host_io = nullptr;        // dev [3][max_streams]: adapter_idx, tokens, next of the host-buffer step
   // persistent projection chain (rows <= 8)
   ChainPhase* phases = nullptr;      // dev [4*L (+1)]: qkv, o, gate/up, down per layer; then lm_head
@@ -259,6 +259,12 @@ int forward_chain(mlora_ctx* c, const PassIO& io) {
   return MLORA_OK;
 }
 
+// one projection of a pass with more than 8 rows: tensor-core path from 32 rows up, split-K mma.sync below
+cudaError_t launch_projection(mlora_ctx* c, const GemmArgs& g, cudaStream_t st) {
+  if (!c->dbg_no_tc && gemm_tc_eligible(g)) return launch_gemm_tc(g, c->sm_count, c->status, st);
+  return launch_gemm(g, st);
+}
+
 // the launch sequence of one pass over M = n*T rows (Sec. 3.1 decoder, Eq. 1-4 projections)
 int forward(mlora_ctx* c, const PassIO& io) {
   if (chain_eligible(c, io)) return forward_chain(c, io);
@@ -283,7 +289,7 @@ int forward(mlora_ctx* c, const PassIO& io) {
       g.out_f32 = c->qkv; g.ldo = c->Nqkv;
       g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
       g.lora = s.lora;
-      CK(run(c, MLORA_PROF_GEMM, [&] { return launch_gemm(g, st); }));
+      CK(run(c, MLORA_PROF_GEMM, [&] { return launch_projection(c, g, st); }));
     }
     {
       int rc = launch_attention_block(c, io, l);
@@ -303,7 +309,7 @@ int forward(mlora_ctx* c, const PassIO& io) {
       g.mode = MODE_PLAIN; g.epi = EPI_RESID; g.resid = c->X;
       g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
       g.lora = la;
-      CK(run(c, MLORA_PROF_GEMM, [&] { return launch_gemm(g, st); }));
+      CK(run(c, MLORA_PROF_GEMM, [&] { return launch_projection(c, g, st); }));
     }
     // MLP block
     {
@@ -318,7 +324,7 @@ int forward(mlora_ctx* c, const PassIO& io) {
       g.mode = MODE_GATEUP; g.epi = EPI_SWIGLU; g.out_f16 = c->act16;
       g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
       g.lora = s.lora;
-      CK(run(c, MLORA_PROF_GEMM, [&] { return launch_gemm(g, st); }));
+      CK(run(c, MLORA_PROF_GEMM, [&] { return launch_projection(c, g, st); }));
     }
     {
       const int projs[1] = {6}, widths[1] = {dm};
@@ -334,7 +340,7 @@ int forward(mlora_ctx* c, const PassIO& io) {
       g.mode = MODE_PLAIN; g.epi = EPI_RESID; g.resid = c->X;
       g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
       g.lora = la;
-      CK(run(c, MLORA_PROF_GEMM, [&] { return launch_gemm(g, st); }));
+      CK(run(c, MLORA_PROF_GEMM, [&] { return launch_projection(c, g, st); }));
     }
   }
   if (d.vocab > 0 && io.logits != nullptr) {
@@ -346,7 +352,7 @@ int forward(mlora_ctx* c, const PassIO& io) {
     g.w = w.data; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->h; g.M = M;
     g.mode = MODE_PLAIN; g.epi = EPI_F32; g.out_f32 = io.logits; g.ldo = d.vocab;
     g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
-    CK(run(c, MLORA_PROF_GEMM, [&] { return launch_gemm(g, st); }));
+    CK(run(c, MLORA_PROF_GEMM, [&] { return launch_projection(c, g, st); }));
   }
   return MLORA_OK;
 }
@@ -414,6 +420,7 @@ int init_kernels() {
   CK(init_shrink());
   CK(init_attention());
   CK(init_chain());
+  CK(init_gemm_tc());
   done = true;
   return MLORA_OK;
 }
@@ -833,7 +840,7 @@ int mlora_verify_tree(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_id
   key.kind = 3; key.n = n; key.T = T;
   key.prefix_chunk = io.plan.prefix_chunk; key.n_prefix_chunks = io.plan.n_prefix_chunks;
   key.own_chunk = io.plan.own_chunk; key.n_own_chunks = io.plan.n_own_chunks;
-  key.flags = c->P * 4 + c->dbg_skip_compact * 2 + c->dbg_no_chain;
+  key.flags = c->P * 8 + c->dbg_no_tc * 4 + c->dbg_skip_compact * 2 + c->dbg_no_chain;
   key.p[0] = adapter_idx; key.p[1] = tree_tokens; key.p[2] = tree_parent; key.p[3] = out_accept_len;
   key.p[4] = out_accept_idx; key.p[5] = out_next; key.p[6] = out_logits;
   rc = replay_or_run(c, key, [&]() -> int {
@@ -958,6 +965,7 @@ int mlora_debug_set(mlora_ctx* c, int32_t key, int32_t value) {
   if (key == 1) c->dbg_skip_compact = value ? 1 : 0;
   else if (key == 2) c->dbg_no_graph = value ? 1 : 0;
   else if (key == 3) c->dbg_no_chain = value ? 1 : 0;
+  else if (key == 4) c->dbg_no_tc = value ? 1 : 0;
   else return fail(MLORA_ERR_ARG, "unknown debug key");
   return MLORA_OK;
 }
@@ -1096,7 +1104,8 @@ int mlora_linear(mlora_weight* w, const void* x, int32_t M, const int32_t* row_a
   g.partial = (float*)(ws + fixed); g.partial_capacity = (workspace_bytes - fixed) / sizeof(float);
   g.counters = (unsigned*)(ws + LIN_SYNC_BYTES);
   g.lora = la;
-  CK(launch_gemm(g, w->stream));
+  if (gemm_tc_eligible(g)) CK(launch_gemm_tc(g, w->sm_count, (int*)(ws + 32), w->stream));
+  else CK(launch_gemm(g, w->stream));
   return MLORA_OK;
 }
 

@@ -1,0 +1,311 @@
+// INT4 group-quantised GEMM on the 5th-generation tensor cores for passes with many rows (DS2D verify passes
+// of 128-256 rows, prefill chunks): Y^T[n][m] = sum_k Wdeq[k][n] h[m][k]  (Sec. 3.1 projections with the INT4
+// weights of Sec. 3.3; "swap-AB": the 128 output features of a CTA are the UMMA M dimension, the rows the N
+// dimension).  Per 64 input features a CTA
+//   - dequantises its 128 x 64 weight tile from the packed INT4 layout in registers (the same dequant8() as every
+//     other path: exactly fp16(q * scale)) and writes it to shared memory as a K-major tile in the 128-byte
+//     swizzled layout the tensor core reads,
+//   - copies the rows' 64 activations into a second swizzled K-major tile,
+//   - lets one thread issue four tcgen05.mma (M 128, N = rows, K 16, fp16 in, fp32 accumulate in tensor memory).
+// The MMAs run asynchronously; a tcgen05.commit per stage tells the threads when a stage's buffers may be
+// overwritten, so dequantisation of the next stages overlaps the tensor core.  The accumulator is read back with
+// tcgen05.ld and written as fp32 partial sums [split][M][N]; gemm_tc_epilogue_kernel adds the K splits in a fixed
+// order, adds the LoRA expand term (Eq. 1-4) and applies the projection's epilogue.
+// Every mbarrier wait is bounded; a wait that runs out sets the status word and the CTA winds down (it still waits,
+// bounded, for its MMAs and frees its tensor memory).
+#include "../../include/mlora.h"
+#include "common.cuh"
+
+namespace mlora {
+
+constexpr int TC_BM = 128;                 // output features per CTA (UMMA M)
+constexpr int TC_BK = 64;                  // input features per stage: one 128-byte swizzle row of fp16
+constexpr int TC_STAGES = 3;
+constexpr int TC_THREADS = 256;
+constexpr long long TC_WAIT_CYCLES = 4000000000ll;
+
+__device__ __forceinline__ uint32_t tc_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool tc_wait(uint32_t bar, uint32_t parity, int* status) {
+  const long long t0 = clock64();
+  for (int it = 0;; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
+    if ((it & 255) == 255 && clock64() - t0 > TC_WAIT_CYCLES) {
+      if (status != nullptr) atomicCAS(status, 0, MLORA_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+// byte offset of the 16-byte piece `chunk` (8 fp16) of row `r` in a K-major tile with 128-byte rows, 128B swizzle:
+// 8-row groups of 1024 bytes, the piece index XORed with the row inside the group
+__device__ __forceinline__ uint32_t sw128_off(int r, int chunk) {
+  return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((chunk ^ (r & 7)) << 4));
+}
+// shared-memory matrix descriptor: K-major, 128B swizzle, 1024 bytes between 8-row groups (descriptor version 1)
+__device__ __forceinline__ uint64_t tc_desc(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+         ((uint64_t)2 << 61);
+}
+
+template <int NROWS>
+__global__ void __launch_bounds__(TC_THREADS, 1) w4_gemm_tc_kernel(const GemmArgs p, const int kts_per_split,
+                                                                 int* status) {
+  extern __shared__ __align__(1024) unsigned char tc_smem_raw[];
+  // 1024-byte aligned stage buffers (the swizzle pattern is tied to address bits 7..9)
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
+  constexpr uint32_t A_BYTES = TC_BM * TC_BK * 2, B_BYTES = NROWS * TC_BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+  __shared__ __align__(8) uint64_t stage_free[TC_STAGES];
+  __shared__ __align__(8) uint64_t done_bar;
+  __shared__ uint32_t tmem_base_s;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int slab = blockIdx.x, split = blockIdx.y, m0 = blockIdx.z * NROWS;
+  const WLayout L = make_wlayout(p.K, p.N, p.G);
+  const int kt_begin = split * kts_per_split;
+  const int kt_end = min(L.KT, kt_begin + kts_per_split);
+  const int nk = kt_end - kt_begin;
+  const int rows = min(NROWS, p.M - m0);
+
+  if (tid == 0) {
+    for (int s = 0; s < TC_STAGES; ++s)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(tc_smem_u32(stage_free + s)) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(tc_smem_u32(&done_bar)) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    // tensor memory for the accumulator: NROWS columns of 128 lanes x fp32
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem_u32(&tmem_base_s)), "r"((uint32_t)NROWS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = tmem_base_s;
+
+  // instruction descriptor: D fp32, A and B fp16, both K-major, N = NROWS, M = 128
+  constexpr uint32_t IDESC = (1u << 4) | ((uint32_t)(NROWS >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+  const int nt = slab * (TC_BM / TILE_N) + warp;          // this warp's n-tile (16 output features) of the slab
+  const bool nt_ok = nt < L.NT;
+  const unsigned char* unit = p.w + (size_t)(nt_ok ? nt : 0) * L.unit_bytes;
+  bool alive = true;
+
+  for (int i = 0; i < nk; ++i) {
+    const int s = i % TC_STAGES;
+    const int kt = kt_begin + i;
+    if (i >= TC_STAGES && alive) alive = tc_wait(tc_smem_u32(stage_free + s), (uint32_t)((i / TC_STAGES - 1) & 1), status);
+    unsigned char* As = base + (size_t)s * STAGE_BYTES;
+    unsigned char* Bs = As + A_BYTES;
+    // ---- weights: warp w dequantises n-tile w of the slab (rows 16w + g and 16w + g + 8 of the A tile)
+    {
+      uint4 wv = make_uint4(0x88888888u, 0x88888888u, 0x88888888u, 0x88888888u);   // nibble 8 = weight 0
+      uint32_t sw = 0;
+      if (nt_ok) {
+        wv = ldg_stream(reinterpret_cast<const uint4*>(unit + wl_tile_off(L, kt)) + lane);
+        sw = ldg_nc_u32(reinterpret_cast<const uint32_t*>(unit + wl_scale_off(L, kt)) + g);
+      }
+      __half2 s_lo, s_hi;
+      split_scales(sw, s_lo, s_hi);
+      uint32_t a[4][4];
+      dequant8(wv.x, s_lo, s_hi, a[0]);
+      dequant8(wv.y, s_lo, s_hi, a[1]);
+      dequant8(wv.z, s_lo, s_hi, a[2]);
+      dequant8(wv.w, s_lo, s_hi, a[3]);
+      // a[j][0] / a[j][2]: features 16t+4j+{0,1} / {2,3} of row g;  a[j][1] / a[j][3]: the same of row g+8
+      const int r0 = warp * 16 + g, r1 = r0 + 8;
+      *reinterpret_cast<uint4*>(As + sw128_off(r0, 2 * t)) = make_uint4(a[0][0], a[0][2], a[1][0], a[1][2]);
+      *reinterpret_cast<uint4*>(As + sw128_off(r0, 2 * t + 1)) = make_uint4(a[2][0], a[2][2], a[3][0], a[3][2]);
+      *reinterpret_cast<uint4*>(As + sw128_off(r1, 2 * t)) = make_uint4(a[0][1], a[0][3], a[1][1], a[1][3]);
+      *reinterpret_cast<uint4*>(As + sw128_off(r1, 2 * t + 1)) = make_uint4(a[2][1], a[2][3], a[3][1], a[3][3]);
+    }
+    // ---- activations: 64 features of every row of the block (zero beyond the valid rows)
+    for (int q = tid; q < NROWS * 8; q += TC_THREADS) {
+      const int r = q >> 3, c = q & 7;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (r < rows) v = *reinterpret_cast<const uint4*>(p.h + (size_t)(m0 + r) * p.K + (size_t)kt * TC_BK + c * 8);
+      *reinterpret_cast<uint4*>(Bs + sw128_off(r, c)) = v;
+    }
+    // the tensor core reads shared memory through the async proxy: order the writes above before it
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+    if (tid == 0 && alive) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint64_t adesc = tc_desc(tc_smem_u32(As)), bdesc = tc_desc(tc_smem_u32(Bs));
+#pragma unroll
+      for (int kk = 0; kk < TC_BK / 16; ++kk) {
+        const uint32_t acc = (i > 0 || kk > 0) ? 1u : 0u;
+        // 16 features further along K: 32 bytes inside the swizzled 128-byte row (address field in 16-byte units)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(tmem), "l"(adesc + (uint64_t)(kk * 2)), "l"(bdesc + (uint64_t)(kk * 2)), "r"(IDESC), "r"(acc) : "memory");
+      }
+      // arrives on the stage's barrier when the MMAs issued so far have finished reading the stage
+      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(stage_free + s)) : "memory");
+    }
+  }
+  if (tid == 0) asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(&done_bar)) : "memory");
+  // all MMAs done (also when a stage wait gave up earlier: wait, bounded, before touching or freeing anything)
+  const bool done = tc_wait(tc_smem_u32(&done_bar), 0u, status);
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+
+  // ---- accumulator -> fp32 partial sums [split][M][N]: lane = output feature, columns = rows
+  if (done && alive && nk > 0) {
+    const int lane_grp = warp & 3, col_half = warp >> 2;       // warps w and w+4 share the lanes, split the columns
+    const int n = slab * TC_BM + lane_grp * 32 + lane;
+    float* dst = p.partial + (size_t)split * p.M * p.N;
+    for (int c0 = col_half * (NROWS / 2); c0 < (col_half + 1) * (NROWS / 2); c0 += 32) {
+      uint32_t v[32];
+      const uint32_t taddr = tmem + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)c0;
+      asm volatile(
+          "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+          "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+          "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+          : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+            "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+            "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+            "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+          : "r"(taddr) : "memory");
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      if (n < p.N) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const int m = m0 + c0 + j;
+          if (m < p.M) dst[(size_t)m * p.N + n] = __uint_as_float(v[j]);
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)NROWS) : "memory");
+}
+
+// physical column -> (segment, logical column)
+__device__ __forceinline__ void tc_map_col(int mode, int c, int n0, int n1, int& seg, int& col) {
+  if (mode == MODE_PLAIN) { seg = 0; col = c; }
+  else if (mode == MODE_QKV) {
+    if (c < n0) { seg = 0; col = c; }
+    else if (c < n0 + n1) { seg = 1; col = c - n0; }
+    else { seg = 2; col = c - n0 - n1; }
+  } else {                         // gate/up interleaved by 16-column tiles
+    const int tile = c >> 4;
+    seg = tile & 1;
+    col = ((tile >> 1) << 4) | (c & 15);
+  }
+}
+
+// sum of the K splits (fixed order) plus the LoRA expand term of four consecutive physical columns of row m
+__device__ __forceinline__ float4 tc_row_quad(const GemmArgs& p, int ksplit, int m, int c) {
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int sp = 0; sp < ksplit; ++sp) {
+    const float4 v = __ldcg(reinterpret_cast<const float4*>(p.partial + ((size_t)sp * p.M + m) * p.N + c));
+    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+  }
+  if (p.lora.adapter_idx != nullptr) {
+    const int a = p.lora.adapter_idx[m / p.lora.rows_per_stream];
+    if (a >= 0 && a < p.lora.n_slots) {
+      int seg, col;
+      tc_map_col(p.mode, c, p.seg_n0, p.seg_n1, seg, col);
+      const __half* B = p.lora.tabB[(size_t)a * p.lora.tab_stride + p.lora.seg[seg].proj_index];
+      if (B != nullptr) {
+        const int r = p.lora.rank, ldb = p.lora.seg[seg].n;
+        const float* T = p.lora.T + ((size_t)m * p.lora.nseg + seg) * r;
+        for (int j = 0; j < r; ++j) {
+          const float tj = T[j];
+          const uint2 bv = *reinterpret_cast<const uint2*>(B + (size_t)j * ldb + col);
+          const float2 b01 = __half22float2(u32_as_h2(bv.x)), b23 = __half22float2(u32_as_h2(bv.y));
+          s.x = fmaf(tj, b01.x, s.x); s.y = fmaf(tj, b01.y, s.y);
+          s.z = fmaf(tj, b23.x, s.z); s.w = fmaf(tj, b23.y, s.w);
+        }
+      }
+    }
+  }
+  return s;
+}
+
+// One thread per (row, 4 physical columns): split sum, LoRA expand (Eq. 1-4, second factor), projection epilogue.
+__global__ void gemm_tc_epilogue_kernel(const GemmArgs p, const int ksplit) {
+  const int quads = p.N / 4;
+  const long long total = (long long)p.M * quads;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const int m = (int)(i / quads), c = (int)(i % quads) * 4;
+    if (p.epi == EPI_SWIGLU) {
+      if ((c >> 4) & 1) continue;                              // the gate quad's thread also takes the up quad
+      const float4 gq = tc_row_quad(p, ksplit, m, c), uq = tc_row_quad(p, ksplit, m, c + 16);
+      const float gv[4] = {gq.x, gq.y, gq.z, gq.w}, uv[4] = {uq.x, uq.y, uq.z, uq.w};
+      float v[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) v[e] = gv[e] / (1.f + __expf(-gv[e])) * uv[e];
+      const int f = ((c >> 5) << 4) | (c & 15);
+      const __half2 o01 = __floats2half2_rn(v[0], v[1]), o23 = __floats2half2_rn(v[2], v[3]);
+      *reinterpret_cast<uint2*>(p.out_f16 + (size_t)m * (p.N / 2) + f) = make_uint2(h2_as_u32(o01), h2_as_u32(o23));
+    } else {
+      const float4 s = tc_row_quad(p, ksplit, m, c);
+      if (p.epi == EPI_F32) {
+        *reinterpret_cast<float4*>(p.out_f32 + (size_t)m * p.ldo + c) = s;
+      } else {
+        float4* xp = reinterpret_cast<float4*>(p.resid + (size_t)m * p.N + c);
+        float4 x = *xp;
+        x.x += s.x; x.y += s.y; x.z += s.z; x.w += s.w;
+        *xp = x;
+      }
+    }
+  }
+}
+
+template <int NROWS>
+static cudaError_t tc_launch(const GemmArgs& a, int slabs, int ksplit, int kts_per_split, int* status, cudaStream_t st) {
+  const size_t smem = (size_t)TC_STAGES * (TC_BM * TC_BK * 2 + NROWS * TC_BK * 2) + 1024;
+  dim3 grid(slabs, ksplit, (a.M + NROWS - 1) / NROWS);
+  w4_gemm_tc_kernel<NROWS><<<grid, TC_THREADS, smem, st>>>(a, kts_per_split, status);
+  return cudaGetLastError();
+}
+
+cudaError_t init_gemm_tc() {
+  cudaError_t e;
+  e = cudaFuncSetAttribute(w4_gemm_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_STAGES * (16384 + 64 * 128) + 1024);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(w4_gemm_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_STAGES * (16384 + 128 * 128) + 1024);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(w4_gemm_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_STAGES * (16384 + 256 * 128) + 1024);
+}
+
+bool gemm_tc_eligible(const GemmArgs& a) {
+  if (a.M < 32 || a.N % 16 || a.K % 64) return false;
+  const int nrows = a.M <= 64 ? 64 : (a.M <= 128 ? 128 : 256);
+  const size_t m_blocks = (a.M + nrows - 1) / nrows;
+  (void)m_blocks;
+  return (size_t)a.M * a.N <= a.partial_capacity;            // room for at least one split
+}
+
+// Tensor-core path: partial sums by w4_gemm_tc_kernel, then the epilogue kernel.  `status` may be nullptr.
+cudaError_t launch_gemm_tc(const GemmArgs& a, int sm_count, int* status, cudaStream_t st) {
+  const int nrows = a.M <= 64 ? 64 : (a.M <= 128 ? 128 : 256);
+  const int slabs = (a.N + TC_BM - 1) / TC_BM;
+  const int m_blocks = (a.M + nrows - 1) / nrows;
+  const int KT = a.K / TILE_K;
+  // enough CTAs to fill the machine, at least four k-tiles per split, partial sums must fit the scratch
+  int ksplit = sm_count / (slabs * m_blocks);
+  if (ksplit < 1) ksplit = 1;
+  if (ksplit > KT / 4) ksplit = KT / 4 > 0 ? KT / 4 : 1;
+  while (ksplit > 1 && (size_t)ksplit * a.M * a.N > a.partial_capacity) --ksplit;
+  const int kts_per_split = (KT + ksplit - 1) / ksplit;
+  ksplit = (KT + kts_per_split - 1) / kts_per_split;
+  cudaError_t e;
+  if (nrows == 64) e = tc_launch<64>(a, slabs, ksplit, kts_per_split, status, st);
+  else if (nrows == 128) e = tc_launch<128>(a, slabs, ksplit, kts_per_split, status, st);
+  else e = tc_launch<256>(a, slabs, ksplit, kts_per_split, status, st);
+  if (e != cudaSuccess) return e;
+  const long long total = (long long)a.M * (a.N / 4);
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > sm_count * 8) blocks = sm_count * 8;
+  gemm_tc_epilogue_kernel<<<blocks, 256, 0, st>>>(a, ksplit);
+  return cudaGetLastError();
+}
+
+}  // namespace mlora
