@@ -93,27 +93,56 @@ __global__ void __launch_bounds__(TC_THREADS, 1) w4_gemm_tc_kernel(const GemmArg
   const unsigned char* unit = p.w + (size_t)(nt_ok ? nt : 0) * L.unit_bytes;
   bool alive = true;
 
+  // software pipeline, one k-step ahead: the packed weights of step i+1 wait in registers and the activations of
+  // step i+1 are on their way into their stage (cp.async) while step i is dequantised and issued
+  auto load_w = [&](int kt, uint4& wv, uint32_t& sw) {
+    wv = make_uint4(0x88888888u, 0x88888888u, 0x88888888u, 0x88888888u);   // nibble 8 = weight 0
+    sw = 0;
+    if (nt_ok) {
+      wv = ldg_stream(reinterpret_cast<const uint4*>(unit + wl_tile_off(L, kt)) + lane);
+      sw = ldg_nc_u32(reinterpret_cast<const uint32_t*>(unit + wl_scale_off(L, kt)) + g);
+    }
+  };
+  auto issue_act = [&](int kt, unsigned char* Bs) {
+    // 64 features of every row of the block (zero beyond the valid rows)
+    for (int q = tid; q < NROWS * 8; q += TC_THREADS) {
+      const int r = q >> 3, c = q & 7;
+      unsigned char* dst = Bs + sw128_off(r, c);
+      if (r < rows)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(tc_smem_u32(dst)),
+                     "l"(p.h + (size_t)(m0 + r) * p.K + (size_t)kt * TC_BK + c * 8) : "memory");
+      else
+        *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  uint4 wv_cur, wv_next = make_uint4(0, 0, 0, 0);
+  uint32_t sw_cur, sw_next = 0;
+  if (nk > 0) {
+    load_w(kt_begin, wv_cur, sw_cur);
+    issue_act(kt_begin, base + A_BYTES);
+  }
   for (int i = 0; i < nk; ++i) {
     const int s = i % TC_STAGES;
-    const int kt = kt_begin + i;
-    if (i >= TC_STAGES && alive) alive = tc_wait(tc_smem_u32(stage_free + s), (uint32_t)((i / TC_STAGES - 1) & 1), status);
     unsigned char* As = base + (size_t)s * STAGE_BYTES;
     unsigned char* Bs = As + A_BYTES;
+    if (i + 1 < nk) {
+      const int s1 = (i + 1) % TC_STAGES;
+      // the MMAs that last read stage s1 (step i + 1 - TC_STAGES) must be done before it is refilled
+      if (i + 1 >= TC_STAGES && alive)
+        alive = tc_wait(tc_smem_u32(stage_free + s1), (uint32_t)(((i + 1) / TC_STAGES - 1) & 1), status);
+      load_w(kt_begin + i + 1, wv_next, sw_next);
+      issue_act(kt_begin + i + 1, base + (size_t)s1 * STAGE_BYTES + A_BYTES);
+    }
     // ---- weights: warp w dequantises n-tile w of the slab (rows 16w + g and 16w + g + 8 of the A tile)
     {
-      uint4 wv = make_uint4(0x88888888u, 0x88888888u, 0x88888888u, 0x88888888u);   // nibble 8 = weight 0
-      uint32_t sw = 0;
-      if (nt_ok) {
-        wv = ldg_stream(reinterpret_cast<const uint4*>(unit + wl_tile_off(L, kt)) + lane);
-        sw = ldg_nc_u32(reinterpret_cast<const uint32_t*>(unit + wl_scale_off(L, kt)) + g);
-      }
       __half2 s_lo, s_hi;
-      split_scales(sw, s_lo, s_hi);
+      split_scales(sw_cur, s_lo, s_hi);
       uint32_t a[4][4];
-      dequant8(wv.x, s_lo, s_hi, a[0]);
-      dequant8(wv.y, s_lo, s_hi, a[1]);
-      dequant8(wv.z, s_lo, s_hi, a[2]);
-      dequant8(wv.w, s_lo, s_hi, a[3]);
+      dequant8(wv_cur.x, s_lo, s_hi, a[0]);
+      dequant8(wv_cur.y, s_lo, s_hi, a[1]);
+      dequant8(wv_cur.z, s_lo, s_hi, a[2]);
+      dequant8(wv_cur.w, s_lo, s_hi, a[3]);
       // a[j][0] / a[j][2]: features 16t+4j+{0,1} / {2,3} of row g;  a[j][1] / a[j][3]: the same of row g+8
       const int r0 = warp * 16 + g, r1 = r0 + 8;
       *reinterpret_cast<uint4*>(As + sw128_off(r0, 2 * t)) = make_uint4(a[0][0], a[0][2], a[1][0], a[1][2]);
@@ -121,13 +150,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) w4_gemm_tc_kernel(const GemmArg
       *reinterpret_cast<uint4*>(As + sw128_off(r1, 2 * t)) = make_uint4(a[0][1], a[0][3], a[1][1], a[1][3]);
       *reinterpret_cast<uint4*>(As + sw128_off(r1, 2 * t + 1)) = make_uint4(a[2][1], a[2][3], a[3][1], a[3][3]);
     }
-    // ---- activations: 64 features of every row of the block (zero beyond the valid rows)
-    for (int q = tid; q < NROWS * 8; q += TC_THREADS) {
-      const int r = q >> 3, c = q & 7;
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (r < rows) v = *reinterpret_cast<const uint4*>(p.h + (size_t)(m0 + r) * p.K + (size_t)kt * TC_BK + c * 8);
-      *reinterpret_cast<uint4*>(Bs + sw128_off(r, c)) = v;
-    }
+    // the activations of this step have landed (those of the next may still be in flight)
+    if (i + 1 < nk) asm volatile("cp.async.wait_group 1;" ::: "memory");
+    else asm volatile("cp.async.wait_group 0;" ::: "memory");
     // the tensor core reads shared memory through the async proxy: order the writes above before it
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
@@ -146,6 +171,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) w4_gemm_tc_kernel(const GemmArg
       // arrives on the stage's barrier when the MMAs issued so far have finished reading the stage
       asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(stage_free + s)) : "memory");
     }
+    wv_cur = wv_next;
+    sw_cur = sw_next;
   }
   if (tid == 0) asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(&done_bar)) : "memory");
   // all MMAs done (also when a stage wait gave up earlier: wait, bounded, before touching or freeing anything)
