@@ -37,7 +37,8 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="cfg1", choices=["cfg0", "cfg1"])
+    ap.add_argument("--config", default="cfg1", choices=["cfg0", "cfg1", "cfg2", "cfg3"],
+                    help="cfg1 (default) is the benchmark workload; cfg2/cfg3 time DS2D verify rounds (side measurement)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=None,
                     help="profiling aid: cut the model to this many layers (small ncu captures); not a bench result")
@@ -200,6 +201,76 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def run_verify(args, cfg):
+    """Side measurement: DS2D verify rounds (8 streams x tree_nodes rows per pass, uniform-random draft ids, so about
+    one token is accepted per stream and round).  One JSON line: rows/s verified and tokens/s emitted."""
+    import torch
+    import gen
+    from paper_2604_18655_b200 import binding as mb
+    from paper_2604_18655_b200.runtime import MloraModel
+    K = args.steps if args.steps is not None else 64
+    W = max(args.warmup if args.warmup is not None else 8, 3)
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    side = torch.cuda.Stream()
+    synth, adapters = build_inputs(cfg)
+    n, T = cfg.n_streams, cfg.tree_nodes
+    with torch.cuda.stream(side):
+        model = MloraModel(synth, max_suffix=(K + W + 8) * 4 + 8, max_tree=T)
+        for a, (A, B) in enumerate(adapters):
+            model.set_adapter(a, A, B, cfg.alpha)
+        ctx = model.ctx
+        ids = torch.from_numpy(gen.make_prompt_ids(cfg, 0)).to(dev)
+        last = torch.empty(cfg.vocab, dtype=torch.float32, device=dev)
+        mb.mlora_prefill_shared(ctx, ids, last)
+        parent = torch.from_numpy(np.stack([gen.build_tree(cfg.branch, T)] * n).astype(np.int32)).to(dev)
+        cand = torch.from_numpy(gen.make_candidates(cfg, 64, n, T, 0)).to(dev)
+        tt = torch.empty(n, T, dtype=torch.int32, device=dev)
+        acc_len = torch.empty(n, dtype=torch.int32, device=dev)
+        acc_idx = torch.empty(n, T, dtype=torch.int32, device=dev)
+        nxt = torch.topk(last, n).indices.to(torch.int32)
+        ad = torch.arange(n, dtype=torch.int32, device=dev)
+        emitted = torch.zeros(1, dtype=torch.int64, device=dev)
+
+        def round_(i):
+            tt[:, 0] = nxt
+            tt[:, 1:] = cand[i % 64]
+            mb.mlora_verify_tree(ctx, ad, tt, parent, acc_len, acc_idx, nxt, None)
+            emitted.add_(acc_len.sum())
+
+        for i in range(W):
+            round_(i)
+        emitted.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        side.synchronize()
+        e0.record(side)
+        for i in range(K):
+            round_(W + i)
+        e1.record(side)
+        side.synchronize()
+        ms = e0.elapsed_time(e1) / K
+        tokens = int(emitted.item())
+        mb.mlora_profile_begin(ctx)
+        for i in range(4):
+            round_(W + K + i)
+        prof = mb.mlora_profile_end(ctx)
+        mb.mlora_sync_status(ctx)
+    params = sum(gen.proj_shape(cfg, p)[0] * gen.proj_shape(cfg, p)[1] for p in gen.PROJ_NAMES) * cfg.n_layers + \
+        cfg.d_model * cfg.vocab
+    line = {
+        "metric": "DS2D verify rows/s", "value": n * T / (ms / 1e3), "unit": "rows/s", "n_gpus": 1, "steps": K, "warmup": W,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
+        "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: {n} streams x {T}-node trees {cfg.branch}, prompt {cfg.prompt_len}, "
+                               f"rank-{cfg.lora_rank} LoRA, uniform-random drafts", "rows_per_pass": n * T},
+        "tokens_per_s": tokens / (ms * K / 1e3), "tokens_per_round": tokens / K,
+        "gemm_tflops": 2.0 * n * T * params / (ms / 1e3) / 1e12,
+        "family_us_per_step": {k: 1e3 * v[0] / 4 for k, v in prof.items()},
+    }
+    print(json.dumps(line), flush=True)
+    model.close()
+
+
 def workload_name(cfg):
     return (f"{cfg.name}: d{cfg.d_model} L{cfg.n_layers} {cfg.n_q_heads}q/{cfg.n_kv_heads}kv hd{cfg.head_dim} "
             f"ffn{cfg.d_ffn} vocab{cfg.vocab} int4-g{cfg.group_size}; {cfg.n_streams} streams x rank-{cfg.lora_rank} "
@@ -209,11 +280,14 @@ def workload_name(cfg):
 def main():
     args = parse_args()
     import gen
-    cfg = {"cfg0": gen.CFG0, "cfg1": gen.CFG1}[args.config]
+    cfg = {"cfg0": gen.CFG0, "cfg1": gen.CFG1, "cfg2": gen.CFG2, "cfg3": gen.CFG3}[args.config]
     if args.layers is not None:
         cfg = cfg.small(n_layers=args.layers, name=f"{cfg.name}-cut{args.layers}L")
     if args.impl == "reference":
         run_reference(args, cfg)
+        return
+    if cfg.tree_nodes > 1:
+        run_verify(args, cfg)
         return
     import torch
     from paper_2604_18655_b200 import binding as mb

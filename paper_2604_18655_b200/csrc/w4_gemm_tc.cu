@@ -242,7 +242,21 @@ __device__ __forceinline__ float4 tc_row_quad(const GemmArgs& p, int ksplit, int
       if (B != nullptr) {
         const int r = p.lora.rank, ldb = p.lora.seg[seg].n;
         const float* T = p.lora.T + ((size_t)m * p.lora.nseg + seg) * r;
-        for (int j = 0; j < r; ++j) {
+        int j = 0;
+        for (; (r & 3) == 0 && j + 4 <= r; j += 4) {            // loads of four rank indices in flight together
+          const float4 t4 = *reinterpret_cast<const float4*>(T + j);
+          uint2 bv[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) bv[e] = __ldg(reinterpret_cast<const uint2*>(B + (size_t)(j + e) * ldb + col));
+          const float tj[4] = {t4.x, t4.y, t4.z, t4.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 b01 = __half22float2(u32_as_h2(bv[e].x)), b23 = __half22float2(u32_as_h2(bv[e].y));
+            s.x = fmaf(tj[e], b01.x, s.x); s.y = fmaf(tj[e], b01.y, s.y);
+            s.z = fmaf(tj[e], b23.x, s.z); s.w = fmaf(tj[e], b23.y, s.w);
+          }
+        }
+        for (; j < r; ++j) {
           const float tj = T[j];
           const uint2 bv = *reinterpret_cast<const uint2*>(B + (size_t)j * ldb + col);
           const float2 b01 = __half22float2(u32_as_h2(bv.x)), b23 = __half22float2(u32_as_h2(bv.y));
