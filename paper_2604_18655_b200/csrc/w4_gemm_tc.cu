@@ -20,7 +20,8 @@ namespace mlora {
 
 constexpr int TC_BM = 128;                 // output features per CTA (UMMA M)
 constexpr int TC_BK = 64;                  // input features per stage: one 128-byte swizzle row of fp16
-constexpr int TC_STAGES = 3;
+constexpr int TC_STAGES = 3;                // 96 KB at 128 rows: two CTAs per SM hide each other's stalls
+constexpr int TC_AHEAD = 2;                // k-steps whose operands are in flight ahead of the one being issued
 constexpr int TC_THREADS = 256;
 constexpr long long TC_WAIT_CYCLES = 4000000000ll;
 
@@ -116,23 +117,26 @@ __global__ void __launch_bounds__(TC_THREADS, 1) w4_gemm_tc_kernel(const GemmArg
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
-  uint4 wv_cur, wv_next = make_uint4(0, 0, 0, 0);
-  uint32_t sw_cur, sw_next = 0;
-  if (nk > 0) {
-    load_w(kt_begin, wv_cur, sw_cur);
-    issue_act(kt_begin, base + A_BYTES);
-  }
+  uint4 wv_cur = make_uint4(0, 0, 0, 0), wv_n1 = make_uint4(0, 0, 0, 0), wv_n2 = make_uint4(0, 0, 0, 0);
+  uint32_t sw_cur = 0, sw_n1 = 0, sw_n2 = 0;
+  // prologue: the first TC_AHEAD steps (one cp.async group per step, empty if the step does not exist)
+  if (nk > 0) { load_w(kt_begin, wv_cur, sw_cur); issue_act(kt_begin, base + A_BYTES); }
+  else asm volatile("cp.async.commit_group;" ::: "memory");
+  if (nk > 1) { load_w(kt_begin + 1, wv_n1, sw_n1); issue_act(kt_begin + 1, base + STAGE_BYTES + A_BYTES); }
+  else asm volatile("cp.async.commit_group;" ::: "memory");
   for (int i = 0; i < nk; ++i) {
     const int s = i % TC_STAGES;
     unsigned char* As = base + (size_t)s * STAGE_BYTES;
     unsigned char* Bs = As + A_BYTES;
-    if (i + 1 < nk) {
-      const int s1 = (i + 1) % TC_STAGES;
-      // the MMAs that last read stage s1 (step i + 1 - TC_STAGES) must be done before it is refilled
-      if (i + 1 >= TC_STAGES && alive)
-        alive = tc_wait(tc_smem_u32(stage_free + s1), (uint32_t)(((i + 1) / TC_STAGES - 1) & 1), status);
-      load_w(kt_begin + i + 1, wv_next, sw_next);
-      issue_act(kt_begin + i + 1, base + (size_t)s1 * STAGE_BYTES + A_BYTES);
+    if (i + TC_AHEAD < nk) {
+      const int sa = (i + TC_AHEAD) % TC_STAGES;
+      // the MMAs that last read stage sa (step i + TC_AHEAD - TC_STAGES) must be done before it is refilled
+      if (i + TC_AHEAD >= TC_STAGES && alive)
+        alive = tc_wait(tc_smem_u32(stage_free + sa), (uint32_t)(((i + TC_AHEAD) / TC_STAGES - 1) & 1), status);
+      load_w(kt_begin + i + TC_AHEAD, wv_n2, sw_n2);
+      issue_act(kt_begin + i + TC_AHEAD, base + (size_t)sa * STAGE_BYTES + A_BYTES);
+    } else {
+      asm volatile("cp.async.commit_group;" ::: "memory");
     }
     // ---- weights: warp w dequantises n-tile w of the slab (rows 16w + g and 16w + g + 8 of the A tile)
     {
@@ -150,9 +154,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) w4_gemm_tc_kernel(const GemmArg
       *reinterpret_cast<uint4*>(As + sw128_off(r1, 2 * t)) = make_uint4(a[0][1], a[0][3], a[1][1], a[1][3]);
       *reinterpret_cast<uint4*>(As + sw128_off(r1, 2 * t + 1)) = make_uint4(a[2][1], a[2][3], a[3][1], a[3][3]);
     }
-    // the activations of this step have landed (those of the next may still be in flight)
-    if (i + 1 < nk) asm volatile("cp.async.wait_group 1;" ::: "memory");
-    else asm volatile("cp.async.wait_group 0;" ::: "memory");
+    // the activations of this step have landed (those of the next TC_AHEAD steps may still be in flight)
+    asm volatile("cp.async.wait_group %0;" ::"n"(TC_AHEAD) : "memory");
     // the tensor core reads shared memory through the async proxy: order the writes above before it
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
@@ -171,8 +174,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) w4_gemm_tc_kernel(const GemmArg
       // arrives on the stage's barrier when the MMAs issued so far have finished reading the stage
       asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(stage_free + s)) : "memory");
     }
-    wv_cur = wv_next;
-    sw_cur = sw_next;
+    wv_cur = wv_n1; sw_cur = sw_n1;
+    wv_n1 = wv_n2; sw_n1 = sw_n2;
   }
   if (tid == 0) asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(&done_bar)) : "memory");
   // all MMAs done (also when a stage wait gave up earlier: wait, bounded, before touching or freeing anything)
@@ -330,8 +333,8 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, int sm_count, int* status, cudaStr
   const int slabs = (a.N + TC_BM - 1) / TC_BM;
   const int m_blocks = (a.M + nrows - 1) / nrows;
   const int KT = a.K / TILE_K;
-  // enough CTAs to fill the machine, at least four k-tiles per split, partial sums must fit the scratch
-  int ksplit = sm_count / (slabs * m_blocks);
+  // enough CTAs for two per SM (up to 128 rows two fit), at least four k-tiles per split, partial sums must fit
+  int ksplit = (nrows <= 128 ? 2 * sm_count : sm_count) / (slabs * m_blocks);
   if (ksplit < 1) ksplit = 1;
   if (ksplit > KT / 4) ksplit = KT / 4 > 0 ? KT / 4 : 1;
   while (ksplit > 1 && (size_t)ksplit * a.M * a.N > a.partial_capacity) --ksplit;
