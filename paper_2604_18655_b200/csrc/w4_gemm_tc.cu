@@ -232,8 +232,18 @@ __device__ __forceinline__ void tc_map_col(int mode, int c, int n0, int n1, int&
 // sum of the K splits (fixed order) plus the LoRA expand term of four consecutive physical columns of row m
 __device__ __forceinline__ float4 tc_row_quad(const GemmArgs& p, int ksplit, int m, int c) {
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int sp = 0; sp < ksplit; ++sp) {
-    const float4 v = __ldcg(reinterpret_cast<const float4*>(p.partial + ((size_t)sp * p.M + m) * p.N + c));
+  const size_t sstride = (size_t)p.M * p.N;
+  const float* pp = p.partial + (size_t)m * p.N + c;
+  int sp = 0;
+  for (; sp + 4 <= ksplit; sp += 4) {                      // four splits' loads in flight; still added in split order
+    float4 v[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) v[e] = __ldcg(reinterpret_cast<const float4*>(pp + (size_t)(sp + e) * sstride));
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { s.x += v[e].x; s.y += v[e].y; s.z += v[e].z; s.w += v[e].w; }
+  }
+  for (; sp < ksplit; ++sp) {
+    const float4 v = __ldcg(reinterpret_cast<const float4*>(pp + (size_t)sp * sstride));
     s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
   }
   if (p.lora.adapter_idx != nullptr) {
