@@ -165,6 +165,22 @@ def oracle_sample(cfg, synth, adapters, n_steps, n_threads_note=None):
     return cfg.n_streams * n_steps / dt, dt, desc
 
 
+def max_over_ranks(ms, world, device):
+    """The job's time is the slowest rank's (replicas only: no collective on the data path, only this one)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(ms)], device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tokens_per_s(world, n_streams, steps, ms_total):
+    """Whole-job throughput of `world` independent replicas (weak scaling: every rank runs the full workload)."""
+    return world * n_streams * steps / (ms_total / 1e3)
+
+
 def cores_used():
     try:
         return len(os.sched_getaffinity(0))
@@ -365,11 +381,8 @@ def main():
         clocks = sampler.stop(t0, t1)
         ms_total = e0.elapsed_time(e1)
         launches = mb.mlora_launch_count(ctx) - l0
-        if world > 1:
-            t = torch.tensor([ms_total], device=dev)
-            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-            ms_total = float(t.item())
-        value = world * n * K / (ms_total / 1e3)
+        ms_total = max_over_ranks(ms_total, world, dev)
+        value = aggregate_tokens_per_s(world, n, K, ms_total)
 
         # ---- end to end through the C ABI with HOST buffers: H2D of the step's inputs, D2H of its result
         Ke = min(K, 512)
@@ -414,11 +427,8 @@ def main():
         e1.record(side)
         barrier()
         ms_e2e = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms_e2e], device=dev)
-            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-            ms_e2e = float(t.item())
-        e2e_value = world * n * Ke / (ms_e2e / 1e3)
+        ms_e2e = max_over_ranks(ms_e2e, world, dev)
+        e2e_value = aggregate_tokens_per_s(world, n, Ke, ms_e2e)
 
         # ---- per-family device time of the same steps (direct launches, an event pair around every kernel)
         mb.mlora_reset_streams(ctx)
