@@ -144,7 +144,11 @@ int mlora_debug_dequant(mlora_ctx* ctx, int32_t layer, int32_t proj, void* out_f
  * the pass wrote them: rows suffix_len .. suffix_len + n_nodes - 1 of the own segment).
  * key 2 = 1 disables CUDA-graph replay of steps (every kernel launched directly).
  * key 3 = 1 runs decode-sized passes through the one-kernel-per-projection path instead of the persistent kernel.
- * key 4 = 1 runs passes of 32 rows or more on the split-K mma.sync GEMM instead of the tcgen05 one. */
+ * key 4 = 1 runs passes of 32 rows or more on the split-K mma.sync GEMM instead of the tcgen05 one.
+ * key 5 = 1 (test hook for the bounded waits) makes the NEXT decode-sized pass wait, with a limit of about 0.1 s,
+ *         at a grid barrier for an arrival nobody makes: the pass ends with garbage outputs and the device status
+ *         MLORA_ERR_TIMEOUT; mlora_sync_status reports and clears it, after which the context works again
+ *         (run mlora_prefill_shared or mlora_reset_streams to drop the garbage rows). */
 int mlora_debug_set(mlora_ctx* ctx, int32_t key, int32_t value);
 /* Per-kernel-family device time of the NEXT steps, measured with CUDA events on the context's stream.
  * mlora_profile_begin switches to direct launches with an event pair around every kernel; mlora_profile_end

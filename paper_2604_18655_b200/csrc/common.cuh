@@ -168,6 +168,8 @@ struct ChainArgs {
   float* T;                       // dev fp32 [M][3][rank] scratch
   unsigned long long* sync;       // dev [4]: grid-barrier arrivals, shrink arrivals, abort flag, spare
   int* status;                    // dev status word
+  long long wait_cycles;          // clock limit of every wait (0: the default, about two seconds)
+  int inject_stall;               // test hook: the launch's first grid barrier waits for an arrival nobody makes
   int nstages;                    // ring stages
   int kmax;                       // largest K of the phases in range (sizes the activation buffer)
 };

@@ -135,6 +135,7 @@ __device__ __forceinline__ uint32_t pos_parity(int pos, int nstages) { return (u
 
 // ----------------------------------------------------------------------------- bounded waits
 struct WaitCtx {
+  long long limit;                  // clock cycles a wait may take
   volatile int* s_abort;            // shared: this CTA has given up waiting
   unsigned long long* sync;         // global: [0] barrier, [1] shrink, [2] abort, [3] where the first wait gave up
   int* status;
@@ -157,7 +158,7 @@ __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const W
     if ((it & 255) == 255) {
       if (*w.s_abort) return false;
       if (ld_acquire_u64(w.sync + 2) != 0ull) { *w.s_abort = 1; return false; }
-      if (clock64() - t0 > CH_WAIT_CYCLES) { raise_abort(w, where, phase); return false; }
+      if (clock64() - t0 > w.limit) { raise_abort(w, where, phase); return false; }
     }
   }
 }
@@ -170,7 +171,7 @@ __device__ __forceinline__ void wait_counter(const unsigned long long* ctr, unsi
     if (ld_acquire_u64(ctr) >= target) return;
     if ((it & 63) == 63) {
       if (ld_acquire_u64(w.sync + 2) != 0ull) { *w.s_abort = 1; return; }
-      if (clock64() - t0 > CH_WAIT_CYCLES) { raise_abort(w, where, phase); return; }
+      if (clock64() - t0 > w.limit) { raise_abort(w, where, phase); return; }
     }
   }
 }
@@ -309,7 +310,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
   const int M = a.M;
   const int r = a.rank;
   const bool lora_on = a.adapter_idx != nullptr && a.rank > 0;
-  WaitCtx wc{&s_abort_word, a.sync, a.status};
+  WaitCtx wc{a.wait_cycles > 0 ? a.wait_cycles : CH_WAIT_CYCLES, &s_abort_word, a.sync, a.status};
 
   // ---- set-up: barriers, first phase descriptor, adapters of the rows, counter bases
   if (tid == 0) {
@@ -445,7 +446,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
         const int st = (int)(idx % nstages);
         const uint32_t par = (uint32_t)((idx / nstages) & 1);
         while (!mbar_try_wait(smem_u32(full_bar + st), par)) {
-          if (clock64() - t0 > CH_WAIT_CYCLES) break;
+          if (clock64() - t0 > wc.limit) break;
         }
       }
     }
@@ -779,7 +780,8 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
         // the release is cumulative over what the CTA's threads wrote before the named barrier above; the
         // acquire load inside wait_counter orders the next phase's reads after the other CTAs' writes
         red_release_add_u64(a.sync + 0, 1ull);
-        wait_counter(a.sync + 0, s_base[0] + n_bar * G, wc, 5, p);
+        // (test hook: with inject_stall the first barrier of the launch waits for one arrival too many)
+        wait_counter(a.sync + 0, s_base[0] + n_bar * G + ((a.inject_stall && n_bar == 1) ? 1ull : 0ull), wc, 5, p);
       }
       consumer_sync();
     }

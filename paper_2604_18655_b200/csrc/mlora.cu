@@ -95,7 +95,7 @@ struct mlora_ctx {
   cudaEvent_t snap_event = nullptr;
   bool snap_pending = false;
   int snap_inc = 0;
-  int dbg_skip_compact = 0, dbg_no_graph = 0, dbg_no_chain = 0, dbg_no_tc = 0;
+  int dbg_skip_compact = 0, dbg_no_graph = 0, dbg_no_chain = 0, dbg_no_tc = 0, dbg_inject_stall = 0;
   int32_t* host_io = nullptr;        // dev [3][max_streams]: adapter_idx, tokens, next of the host-buffer step
   // persistent projection chain (rows <= 8)
   ChainPhase* phases = nullptr;      // dev [4*L (+1)]: qkv, o, gate/up, down per layer; then lm_head
@@ -246,6 +246,11 @@ int forward_chain(mlora_ctx* c, const PassIO& io) {
   a.rank = d.lora_rank;
   a.T = c->T; a.sync = c->chain_sync; a.status = c->status;
   a.nstages = c->chain_stages; a.kmax = c->chain_kmax;
+  if (c->dbg_inject_stall) {                           // one pass only: short waits, one barrier that cannot complete
+    a.wait_cycles = 200000000ll;                       // ~0.1 s
+    a.inject_stall = 1;
+    c->dbg_inject_stall = 0;
+  }
   const int last = 4 * c->L + ((d.vocab > 0 && io.logits != nullptr) ? 1 : 0);
   a.p0 = 0; a.p1 = 1;
   CK(run(c, MLORA_PROF_GEMM, [&] { return launch_chain(a, c->sm_count, st); }));
@@ -767,7 +772,7 @@ static int decode_impl(mlora_ctx* c, int n, const int32_t* adapter_idx, const in
   key.kind = hidden ? 2 : 1; key.n = n; key.T = 1;
   key.prefix_chunk = io.plan.prefix_chunk; key.n_prefix_chunks = io.plan.n_prefix_chunks;
   key.own_chunk = io.plan.own_chunk; key.n_own_chunks = io.plan.n_own_chunks;
-  key.flags = c->P * 2 + c->dbg_no_chain;
+  key.flags = c->P * 4 + c->dbg_inject_stall * 2 + c->dbg_no_chain;
   key.p[0] = adapter_idx; key.p[1] = tokens; key.p[2] = hidden; key.p[3] = out_next; key.p[4] = out_logits; key.p[5] = hidden_out;
   rc = replay_or_run(c, key, [&]() -> int {
     int r = forward(c, io);
@@ -966,6 +971,7 @@ int mlora_debug_set(mlora_ctx* c, int32_t key, int32_t value) {
   else if (key == 2) c->dbg_no_graph = value ? 1 : 0;
   else if (key == 3) c->dbg_no_chain = value ? 1 : 0;
   else if (key == 4) c->dbg_no_tc = value ? 1 : 0;
+  else if (key == 5) c->dbg_inject_stall = value ? 1 : 0;
   else return fail(MLORA_ERR_ARG, "unknown debug key");
   return MLORA_OK;
 }

@@ -363,3 +363,29 @@ def test_host_buffer_step_matches_device_step(GpuModel):
         mb.mlora_sync_status(gm.ctx)
         gm.close()
     assert np.array_equal(outs[0], outs[1])
+
+
+def test_bounded_wait_runs_out_and_context_recovers(GpuModel):
+    """Failure detection without a fault: a grid barrier of the persistent kernel is made to wait (limit ~0.1 s) for an
+    arrival nobody makes.  The kernel must return, the device status must say TIMEOUT and name the wait, and after
+    mlora_sync_status the same context must compute the same logits as before."""
+    from paper_2604_18655_b200 import binding as mb
+    cfg = TINYV
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+    ids = gen.make_prompt_ids(cfg, 0)
+    toks = np.array([1, 2, 3], dtype=np.int32)
+    gm.prefill(ids)
+    _, want = gm.decode([0, 1, -1], toks)
+    mb.mlora_sync_status(gm.ctx)
+    gm.prefill(ids)
+    mb.mlora_debug_set(gm.ctx, 5, 1)
+    gm.decode([0, 1, -1], toks)                        # returns (with garbage) instead of hanging
+    with pytest.raises(mb.MloraError) as e:
+        mb.mlora_sync_status(gm.ctx)
+    assert e.value.code == -5 and "wait kind 5" in str(e.value)
+    mb.mlora_sync_status(gm.ctx)                       # cleared
+    gm.prefill(ids)
+    _, got = gm.decode([0, 1, -1], toks)
+    mb.mlora_sync_status(gm.ctx)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    gm.close()
