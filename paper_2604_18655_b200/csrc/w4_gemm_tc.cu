@@ -5,7 +5,8 @@
 //   - dequantises its 128 x 64 weight tile from the packed INT4 layout in registers (the same dequant8() as every
 //     other path: exactly fp16(q * scale)) and writes it to shared memory as a K-major tile in the 128-byte
 //     swizzled layout the tensor core reads,
-//   - copies the rows' 64 activations into a second swizzled K-major tile,
+//   - has the rows' 64 activations copied into a second swizzled K-major tile by one TMA tile copy
+//     (cp.async.bulk.tensor, 128-byte swizzle, completion counted on an mbarrier; rows past M read as zero),
 //   - lets one thread issue four tcgen05.mma (M 128, N = rows, K 16, fp16 in, fp32 accumulate in tensor memory).
 // The MMAs run asynchronously; a tcgen05.commit per stage tells the threads when a stage's buffers may be
 // overwritten, so dequantisation of the next stages overlaps the tensor core.  The accumulator is read back with
@@ -13,6 +14,9 @@
 // order, adds the LoRA expand term (Eq. 1-4) and applies the projection's epilogue.
 // Every mbarrier wait is bounded; a wait that runs out sets the status word and the CTA winds down (it still waits,
 // bounded, for its MMAs and frees its tensor memory).
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
 #include "../../include/mlora.h"
 #include "common.cuh"
 
@@ -20,9 +24,18 @@ namespace mlora {
 
 constexpr int TC_BM = 128;                 // output features per CTA (UMMA M)
 constexpr int TC_BK = 64;                  // input features per stage: one 128-byte swizzle row of fp16
-constexpr int TC_STAGES = 3;                // 96 KB at 128 rows: two CTAs per SM hide each other's stalls
-constexpr int TC_AHEAD = 2;                // k-steps whose operands are in flight ahead of the one being issued
-constexpr int TC_THREADS = 256;
+constexpr int TC_DEQ_WARPS = 8, TC_DEQ_THREADS = TC_DEQ_WARPS * 32;   // one n-tile (16 features) per warp
+// dequantised-weight tiles / activation tiles / packed-weight ring depth per CTA.  Up to 128 rows two CTAs share an
+// SM (<= 106 KB each); at 256 rows one CTA takes 217 KB.
+__host__ __device__ constexpr int tc_nsta(int nrows) { return nrows == 256 ? 3 : 2; }
+__host__ __device__ constexpr int tc_nstb(int nrows) { return nrows == 256 ? 4 : (nrows == 128 ? 3 : 4); }
+__host__ __device__ constexpr int tc_wdepth(int nrows) { return nrows == 256 ? 8 : 5; }
+__host__ __device__ constexpr int tc_ctas_per_sm(int nrows) { return nrows == 256 ? 1 : 2; }
+__host__ __device__ constexpr size_t tc_smem_bytes(int nrows) {
+  return (size_t)tc_nsta(nrows) * TC_BM * TC_BK * 2 + (size_t)tc_nstb(nrows) * nrows * TC_BK * 2 +
+         (size_t)tc_wdepth(nrows) * TC_DEQ_THREADS * 20 + 1024;
+}
+constexpr int TC_THREADS = TC_DEQ_THREADS + 64;      // + one warp for the activation copies, one for the MMAs
 constexpr long long TC_WAIT_CYCLES = 4000000000ll;
 
 __device__ __forceinline__ uint32_t tc_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -52,13 +65,19 @@ __device__ __forceinline__ uint64_t tc_desc(uint32_t saddr) {
 }
 
 template <int NROWS>
-__global__ void __launch_bounds__(TC_THREADS, 1) w4_gemm_tc_kernel(const GemmArgs p, const int kts_per_split,
-                                                                 int* status) {
+__global__ void __launch_bounds__(TC_THREADS, tc_ctas_per_sm(NROWS))
+w4_gemm_tc_kernel(const GemmArgs p, const int kts_per_split, int* status, const __grid_constant__ CUtensorMap act_map) {
   extern __shared__ __align__(1024) unsigned char tc_smem_raw[];
-  // 1024-byte aligned stage buffers (the swizzle pattern is tied to address bits 7..9)
+  // 1024-byte aligned tiles (the swizzle pattern is tied to address bits 7..9): NSTA weight tiles, NSTB activation
+  // tiles, then the ring of packed weights (WD slots of 16 + 4 bytes per dequantising thread)
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~(uintptr_t)1023);
-  constexpr uint32_t A_BYTES = TC_BM * TC_BK * 2, B_BYTES = NROWS * TC_BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-  __shared__ __align__(8) uint64_t stage_free[TC_STAGES];
+  constexpr int NSTA = tc_nsta(NROWS), NSTB = tc_nstb(NROWS), WD = tc_wdepth(NROWS);
+  constexpr uint32_t A_BYTES = TC_BM * TC_BK * 2, B_BYTES = NROWS * TC_BK * 2;
+  unsigned char* const act_tiles = base + (size_t)NSTA * A_BYTES;
+  unsigned char* const wring = act_tiles + (size_t)NSTB * B_BYTES;
+  __shared__ __align__(8) uint64_t step_done[NSTB];   // step k arrives on slot k % NSTB when its MMAs have finished
+  __shared__ __align__(8) uint64_t act_full[NSTB];    // the activation tile of step k has landed in tile k % NSTB
+  __shared__ __align__(8) uint64_t a_full[NSTA];      // all dequantising warps have written weight tile k % NSTA
   __shared__ __align__(8) uint64_t done_bar;
   __shared__ uint32_t tmem_base_s;
 
@@ -69,11 +88,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) w4_gemm_tc_kernel(const GemmArg
   const int kt_begin = split * kts_per_split;
   const int kt_end = min(L.KT, kt_begin + kts_per_split);
   const int nk = kt_end - kt_begin;
-  const int rows = min(NROWS, p.M - m0);
 
   if (tid == 0) {
-    for (int s = 0; s < TC_STAGES; ++s)
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(tc_smem_u32(stage_free + s)) : "memory");
+    for (int s = 0; s < NSTB; ++s) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(tc_smem_u32(step_done + s)) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(tc_smem_u32(act_full + s)) : "memory");
+    }
+    for (int s = 0; s < NSTA; ++s)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(tc_smem_u32(a_full + s)), "n"(TC_DEQ_WARPS) : "memory");
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(tc_smem_u32(&done_bar)) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -86,104 +108,143 @@ __global__ void __launch_bounds__(TC_THREADS, 1) w4_gemm_tc_kernel(const GemmArg
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = tmem_base_s;
-
-  // instruction descriptor: D fp32, A and B fp16, both K-major, N = NROWS, M = 128
-  constexpr uint32_t IDESC = (1u << 4) | ((uint32_t)(NROWS >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
-  const int nt = slab * (TC_BM / TILE_N) + warp;          // this warp's n-tile (16 output features) of the slab
-  const bool nt_ok = nt < L.NT;
-  const unsigned char* unit = p.w + (size_t)(nt_ok ? nt : 0) * L.unit_bytes;
   bool alive = true;
+  auto wait_step = [&](int k) {                 // the MMAs of step k have finished reading their tiles
+    if (alive) alive = tc_wait(tc_smem_u32(step_done + k % NSTB), (uint32_t)((k / NSTB) & 1), status);
+  };
 
-  // software pipeline, one k-step ahead: the packed weights of step i+1 wait in registers and the activations of
-  // step i+1 are on their way into their stage (cp.async) while step i is dequantised and issued
-  auto load_w = [&](int kt, uint4& wv, uint32_t& sw) {
-    wv = make_uint4(0x88888888u, 0x88888888u, 0x88888888u, 0x88888888u);   // nibble 8 = weight 0
-    sw = 0;
-    if (nt_ok) {
-      wv = ldg_stream(reinterpret_cast<const uint4*>(unit + wl_tile_off(L, kt)) + lane);
-      sw = ldg_nc_u32(reinterpret_cast<const uint32_t*>(unit + wl_scale_off(L, kt)) + g);
-    }
-  };
-  auto issue_act = [&](int kt, unsigned char* Bs) {
-    // 64 features of every row of the block (zero beyond the valid rows)
-    for (int q = tid; q < NROWS * 8; q += TC_THREADS) {
-      const int r = q >> 3, c = q & 7;
-      unsigned char* dst = Bs + sw128_off(r, c);
-      if (r < rows)
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(tc_smem_u32(dst)),
-                     "l"(p.h + (size_t)(m0 + r) * p.K + (size_t)kt * TC_BK + c * 8) : "memory");
-      else
-        *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-  };
-  uint4 wv_cur = make_uint4(0, 0, 0, 0), wv_n1 = make_uint4(0, 0, 0, 0), wv_n2 = make_uint4(0, 0, 0, 0);
-  uint32_t sw_cur = 0, sw_n1 = 0, sw_n2 = 0;
-  // prologue: the first TC_AHEAD steps (one cp.async group per step, empty if the step does not exist)
-  if (nk > 0) { load_w(kt_begin, wv_cur, sw_cur); issue_act(kt_begin, base + A_BYTES); }
-  else asm volatile("cp.async.commit_group;" ::: "memory");
-  if (nk > 1) { load_w(kt_begin + 1, wv_n1, sw_n1); issue_act(kt_begin + 1, base + STAGE_BYTES + A_BYTES); }
-  else asm volatile("cp.async.commit_group;" ::: "memory");
-  for (int i = 0; i < nk; ++i) {
-    const int s = i % TC_STAGES;
-    unsigned char* As = base + (size_t)s * STAGE_BYTES;
-    unsigned char* Bs = As + A_BYTES;
-    if (i + TC_AHEAD < nk) {
-      const int sa = (i + TC_AHEAD) % TC_STAGES;
-      // the MMAs that last read stage sa (step i + TC_AHEAD - TC_STAGES) must be done before it is refilled
-      if (i + TC_AHEAD >= TC_STAGES && alive)
-        alive = tc_wait(tc_smem_u32(stage_free + sa), (uint32_t)(((i + TC_AHEAD) / TC_STAGES - 1) & 1), status);
-      load_w(kt_begin + i + TC_AHEAD, wv_n2, sw_n2);
-      issue_act(kt_begin + i + TC_AHEAD, base + (size_t)sa * STAGE_BYTES + A_BYTES);
-    } else {
-      asm volatile("cp.async.commit_group;" ::: "memory");
-    }
-    // ---- weights: warp w dequantises n-tile w of the slab (rows 16w + g and 16w + g + 8 of the A tile)
-    {
-      __half2 s_lo, s_hi;
-      split_scales(sw_cur, s_lo, s_hi);
-      uint32_t a[4][4];
-      dequant8(wv_cur.x, s_lo, s_hi, a[0]);
-      dequant8(wv_cur.y, s_lo, s_hi, a[1]);
-      dequant8(wv_cur.z, s_lo, s_hi, a[2]);
-      dequant8(wv_cur.w, s_lo, s_hi, a[3]);
-      // a[j][0] / a[j][2]: features 16t+4j+{0,1} / {2,3} of row g;  a[j][1] / a[j][3]: the same of row g+8
-      const int r0 = warp * 16 + g, r1 = r0 + 8;
-      *reinterpret_cast<uint4*>(As + sw128_off(r0, 2 * t)) = make_uint4(a[0][0], a[0][2], a[1][0], a[1][2]);
-      *reinterpret_cast<uint4*>(As + sw128_off(r0, 2 * t + 1)) = make_uint4(a[2][0], a[2][2], a[3][0], a[3][2]);
-      *reinterpret_cast<uint4*>(As + sw128_off(r1, 2 * t)) = make_uint4(a[0][1], a[0][3], a[1][1], a[1][3]);
-      *reinterpret_cast<uint4*>(As + sw128_off(r1, 2 * t + 1)) = make_uint4(a[2][1], a[2][3], a[3][1], a[3][3]);
-    }
-    // the activations of this step have landed (those of the next TC_AHEAD steps may still be in flight)
-    asm volatile("cp.async.wait_group %0;" ::"n"(TC_AHEAD) : "memory");
-    // the tensor core reads shared memory through the async proxy: order the writes above before it
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncthreads();
-    if (tid == 0 && alive) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint64_t adesc = tc_desc(tc_smem_u32(As)), bdesc = tc_desc(tc_smem_u32(Bs));
-#pragma unroll
-      for (int kk = 0; kk < TC_BK / 16; ++kk) {
-        const uint32_t acc = (i > 0 || kk > 0) ? 1u : 0u;
-        // 16 features further along K: 32 bytes inside the swizzled 128-byte row (address field in 16-byte units)
+  if (warp == TC_DEQ_WARPS) {
+    // ---- activation producer (one thread).  Step j's tile: 64 features (x = kt * 64 elements: a multiple of 128
+    // bytes) of NROWS rows from m0, rows >= M filled with zero; tile j % NSTB is refilled once step j - NSTB is done
+    if (lane == 0) {
+      int issued = 0;
+      for (int j = 0; j < nk; ++j) {
+        if (j >= NSTB) wait_step(j - NSTB);
+        if (!alive) break;
+        const uint32_t bar = tc_smem_u32(act_full + j % NSTB);
+        const uint32_t dst = tc_smem_u32(act_tiles + (size_t)(j % NSTB) * B_BYTES);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(B_BYTES) : "memory");
         asm volatile(
-            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-            ::"r"(tmem), "l"(adesc + (uint64_t)(kk * 2)), "l"(bdesc + (uint64_t)(kk * 2)), "r"(IDESC), "r"(acc) : "memory");
+            "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+            ::"r"(dst), "l"(reinterpret_cast<uint64_t>(&act_map)), "r"((kt_begin + j) * TC_BK), "r"(m0), "r"(bar) : "memory");
+        issued = j + 1;
       }
-      // arrives on the stage's barrier when the MMAs issued so far have finished reading the stage
-      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(stage_free + s)) : "memory");
+      // no copy may still be in flight when the CTA ends: the newest phase of every tile (passes at once unless a
+      // wait gave up somewhere)
+      for (int j = max(0, issued - NSTB); j < issued; ++j)
+        tc_wait(tc_smem_u32(act_full + j % NSTB), (uint32_t)((j / NSTB) & 1), status);
     }
-    wv_cur = wv_n1; sw_cur = sw_n1;
-    wv_n1 = wv_n2; sw_n1 = sw_n2;
+  } else if (warp == TC_DEQ_WARPS + 1) {
+    // ---- MMA issuer (one thread): per step, wait for the weight tile and the activation tile, issue, commit
+    if (lane == 0) {
+      // instruction descriptor: D fp32, A and B fp16, both K-major, N = NROWS, M = 128
+      constexpr uint32_t IDESC = (1u << 4) | ((uint32_t)(NROWS >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+      int sa = 0; uint32_t pa = 0;
+      int sb = 0; uint32_t pb = 0;
+      for (int i = 0; i < nk && alive; ++i) {
+        alive = tc_wait(tc_smem_u32(a_full + sa), pa, status);
+        if (alive) alive = tc_wait(tc_smem_u32(act_full + sb), pb, status);
+        if (!alive) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint64_t adesc = tc_desc(tc_smem_u32(base + (size_t)sa * A_BYTES));
+        const uint64_t bdesc = tc_desc(tc_smem_u32(act_tiles + (size_t)sb * B_BYTES));
+#pragma unroll
+        for (int kk = 0; kk < TC_BK / 16; ++kk) {
+          const uint32_t acc = (i > 0 || kk > 0) ? 1u : 0u;
+          // 16 features further along K: 32 bytes inside the swizzled 128-byte row (address field in 16-byte units)
+          asm volatile(
+              "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+              "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+              ::"r"(tmem), "l"(adesc + (uint64_t)(kk * 2)), "l"(bdesc + (uint64_t)(kk * 2)), "r"(IDESC), "r"(acc) : "memory");
+        }
+        // arrives on the step's barrier when the MMAs issued so far have finished reading their tiles
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(step_done + sb)) : "memory");
+        if (++sa == NSTA) { sa = 0; pa ^= 1u; }
+        if (++sb == NSTB) { sb = 0; pb ^= 1u; }
+      }
+      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(&done_bar)) : "memory");
+    }
+  } else {
+    // ---- dequantising warps: each runs on its own, up to NSTA weight tiles ahead of the tensor core
+    const int nt = slab * (TC_BM / TILE_N) + warp;        // this warp's n-tile (16 output features) of the slab
+    // past the last n-tile the warp reads tile 0 again: those accumulator lanes are never stored
+    const unsigned char* unit = p.w + (size_t)(nt < L.NT ? nt : 0) * L.unit_bytes;
+    // packed weights: each thread copies its own 16 bytes of nibbles and its scale word WD steps ahead
+    // (cp.async, one group per step) and later reads back only what it copied itself, so no barrier is involved
+    const uint32_t wslot0 = tc_smem_u32(wring) + (uint32_t)tid * 16, sslot0 = tc_smem_u32(wring) + TC_DEQ_THREADS * 16 + (uint32_t)tid * 4;
+    constexpr uint32_t WSLOT = TC_DEQ_THREADS * 20;
+    // The loop is a serial chain per warp with only two warps per scheduler to hide it, so everything that can be
+    // is kept as running state: k-tile of the next fetch, ring offsets, tile indices and barrier parities.
+    const int gshift = L.G == 64 ? 0 : (L.G == 128 ? 1 : (L.G == 256 ? 2 : 3));   // k-tiles per scale entry, log2
+    const unsigned char* wsrc = unit + (size_t)lane * 16;
+    const unsigned char* ssrc = unit + (size_t)g * 4;
+    int f_kt = kt_begin;                                  // k-tile of the next fetch
+    uint32_t f_off = 0;                                   // its slot's byte offset in the ring
+    auto fetch_w = [&]() {
+      if (f_kt < kt_end) {
+        const int c = f_kt >> 3, r = f_kt & 7;
+        const uint32_t cbase = (uint32_t)c * L.chunk_full;
+        const uint32_t kc = (c == L.nchunks - 1) ? (uint32_t)L.kc_last : (uint32_t)CHUNK_KT;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(wslot0 + f_off), "l"(wsrc + cbase + r * 512) : "memory");
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sslot0 + f_off),
+                     "l"(ssrc + cbase + kc * 512 + ((r >> gshift) << 5)) : "memory");
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      ++f_kt;
+      f_off = (f_off + WSLOT == WD * WSLOT) ? 0u : f_off + WSLOT;
+    };
+#pragma unroll 1
+    for (int j = 0; j < WD; ++j) fetch_w();
+
+    // this thread's four 16-byte pieces of the weight tile (rows 16w + g and 16w + g + 8, pieces 2t and 2t + 1)
+    const int r0 = warp * 16 + g, r1 = r0 + 8;
+    const uint32_t a_off0 = sw128_off(r0, 2 * t), a_off1 = sw128_off(r0, 2 * t + 1);
+    const uint32_t a_off2 = sw128_off(r1, 2 * t), a_off3 = sw128_off(r1, 2 * t + 1);
+    uint32_t c_off = 0;                                   // ring offset of the slot consumed next
+    int sa = 0;                                           // weight tile of step i
+    int sd = NSTB - 1; uint32_t pd = 1;                   // barrier slot of step i - NSTA and its parity (stepped from i = NSTA - 1 on)
+#pragma unroll 1
+    for (int i = 0; i < nk; ++i) {
+      unsigned char* As = base + (size_t)sa * A_BYTES;
+      if (i >= NSTA && alive) alive = tc_wait(tc_smem_u32(step_done + sd), pd, status);
+      asm volatile("cp.async.wait_group %0;" ::"n"(WD - 1) : "memory");
+      uint4 wv;
+      uint32_t sw;
+      asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(wv.x), "=r"(wv.y), "=r"(wv.z), "=r"(wv.w) : "r"(wslot0 + c_off) : "memory");
+      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(sw) : "r"(sslot0 + c_off) : "memory");
+      c_off = (c_off + WSLOT == WD * WSLOT) ? 0u : c_off + WSLOT;
+      // ---- weights: warp w dequantises n-tile w of the slab (rows 16w + g and 16w + g + 8 of the A tile)
+      {
+        __half2 s_lo, s_hi;
+        split_scales(sw, s_lo, s_hi);
+        uint32_t a[4][4];
+        dequant8(wv.x, s_lo, s_hi, a[0]);
+        dequant8(wv.y, s_lo, s_hi, a[1]);
+        dequant8(wv.z, s_lo, s_hi, a[2]);
+        dequant8(wv.w, s_lo, s_hi, a[3]);
+        // a[j][0] / a[j][2]: features 16t+4j+{0,1} / {2,3} of row g;  a[j][1] / a[j][3]: the same of row g+8
+        *reinterpret_cast<uint4*>(As + a_off0) = make_uint4(a[0][0], a[0][2], a[1][0], a[1][2]);
+        *reinterpret_cast<uint4*>(As + a_off1) = make_uint4(a[2][0], a[2][2], a[3][0], a[3][2]);
+        *reinterpret_cast<uint4*>(As + a_off2) = make_uint4(a[0][1], a[0][3], a[1][1], a[1][3]);
+        *reinterpret_cast<uint4*>(As + a_off3) = make_uint4(a[2][1], a[2][3], a[3][1], a[3][3]);
+      }
+      fetch_w();                                           // refills the slot just read
+      // the tensor core reads shared memory through the async proxy: order the writes above before it, then one
+      // arrival per warp on the tile's barrier
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tc_smem_u32(a_full + sa)) : "memory");
+      sa = (sa + 1 == NSTA) ? 0 : sa + 1;
+      if (i >= NSTA - 1 && ++sd == NSTB) { sd = 0; pd ^= 1u; }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
   }
-  if (tid == 0) asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(&done_bar)) : "memory");
   // all MMAs done (also when a stage wait gave up earlier: wait, bounded, before touching or freeing anything)
   const bool done = tc_wait(tc_smem_u32(&done_bar), 0u, status);
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
   // ---- accumulator -> fp32 partial sums [split][M][N]: lane = output feature, columns = rows
-  if (done && alive && nk > 0) {
+  if (done && alive && nk > 0 && warp < TC_DEQ_WARPS) {
     const int lane_grp = warp & 3, col_half = warp >> 2;       // warps w and w+4 share the lanes, split the columns
     const int n = slab * TC_BM + lane_grp * 32 + lane;
     float* dst = p.partial + (size_t)split * p.M * p.N;
@@ -312,25 +373,56 @@ __global__ void gemm_tc_epilogue_kernel(const GemmArgs p, const int ksplit) {
   }
 }
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point lookup (the library does not link libcuda)
+static PFN_cuTensorMapEncodeTiled_v12000 tensor_map_encoder() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = []() -> PFN_cuTensorMapEncodeTiled_v12000 {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    return reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(sym);
+  }();
+  return fn;
+}
+
+// rank-2 fp16 map over the activations h [M][K]: box = 64 features x nrows rows, 128-byte swizzle, zero fill
+static cudaError_t encode_act_map(const GemmArgs& a, int nrows, CUtensorMap* map) {
+  PFN_cuTensorMapEncodeTiled_v12000 enc = tensor_map_encoder();
+  if (enc == nullptr) return cudaErrorNotSupported;
+  const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.M};
+  const cuuint64_t strides[1] = {(cuuint64_t)a.K * sizeof(__half)};
+  const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)nrows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<__half*>(a.h), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 template <int NROWS>
 static cudaError_t tc_launch(const GemmArgs& a, int slabs, int ksplit, int kts_per_split, int* status, cudaStream_t st) {
-  const size_t smem = (size_t)TC_STAGES * (TC_BM * TC_BK * 2 + NROWS * TC_BK * 2) + 1024;
+  const size_t smem = tc_smem_bytes(NROWS);
   dim3 grid(slabs, ksplit, (a.M + NROWS - 1) / NROWS);
-  w4_gemm_tc_kernel<NROWS><<<grid, TC_THREADS, smem, st>>>(a, kts_per_split, status);
+  CUtensorMap map;
+  const cudaError_t e = encode_act_map(a, NROWS, &map);
+  if (e != cudaSuccess) return e;
+  w4_gemm_tc_kernel<NROWS><<<grid, TC_THREADS, smem, st>>>(a, kts_per_split, status, map);
   return cudaGetLastError();
 }
 
 cudaError_t init_gemm_tc() {
   cudaError_t e;
-  e = cudaFuncSetAttribute(w4_gemm_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_STAGES * (16384 + 64 * 128) + 1024);
+  e = cudaFuncSetAttribute(w4_gemm_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes(64));
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(w4_gemm_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_STAGES * (16384 + 128 * 128) + 1024);
+  e = cudaFuncSetAttribute(w4_gemm_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes(128));
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(w4_gemm_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_STAGES * (16384 + 256 * 128) + 1024);
+  return cudaFuncSetAttribute(w4_gemm_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes(256));
 }
 
 bool gemm_tc_eligible(const GemmArgs& a) {
   if (a.M < 32 || a.N % 16 || a.K % 64) return false;
+  if (reinterpret_cast<uintptr_t>(a.h) % 16 != 0 || tensor_map_encoder() == nullptr) return false;   // TMA needs both
   const int nrows = a.M <= 64 ? 64 : (a.M <= 128 ? 128 : 256);
   const size_t m_blocks = (a.M + nrows - 1) / nrows;
   (void)m_blocks;
