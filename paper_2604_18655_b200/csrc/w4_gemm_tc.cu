@@ -15,6 +15,7 @@
 // Every mbarrier wait is bounded; a wait that runs out sets the status word and the CTA winds down (it still waits,
 // bounded, for its MMAs and frees its tensor memory).
 #include <cuda.h>
+#include <type_traits>
 #include <cudaTypedefs.h>
 
 #include "../../include/mlora.h"
@@ -373,6 +374,130 @@ __global__ void gemm_tc_epilogue_kernel(const GemmArgs p, const int ksplit) {
   }
 }
 
+// The same epilogue for passes whose rows come in runs of 16 that share an adapter (rows_per_stream a multiple of
+// 16: DS2D trees of 16 or 32 nodes), or that have no adapter at all.  A warp takes 16 rows x 32 physical columns and
+// computes the LoRA expand term T B (Eq. 1-4, second factor) with mma.sync m16n8k16: T (fp32) enters as the sum of
+// two fp16 values (value and rounding remainder), so the product keeps fp32 accuracy; B is fp16 as stored.  The
+// adapter's B values are fetched once per 16 rows instead of once per row.
+template <bool SWIGLU>
+__global__ void __launch_bounds__(256) gemm_tc_epilogue_mma_kernel(const GemmArgs p, const int ksplit) {
+  const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int ctiles = (p.N + 31) / 32, rtiles = (p.M + 15) / 16;
+  const size_t sstride = (size_t)p.M * p.N;
+  for (int wt = blockIdx.x * 8 + (threadIdx.x >> 5); wt < ctiles * rtiles; wt += gridDim.x * 8) {
+    const int m0 = (wt / ctiles) * 16, c0 = (wt % ctiles) * 32;
+    const int mA = m0 + g, mB = mA + 8;
+    const bool okA = mA < p.M, okB = mB < p.M;
+    // accumulator fragment of n-tile nt: [0],[1] = row mA, columns c0 + 8 nt + 2t, +1;  [2],[3] = row mB
+    float acc[4][4];
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+    // the adapter of the tile's rows: its loads go out before the split sums need theirs
+    int a = -1;
+    if (p.lora.adapter_idx != nullptr) a = p.lora.adapter_idx[m0 / p.lora.rows_per_stream];
+    auto add_splits = [&](int sp, auto nsp_tag) {              // nsp splits' loads in flight, added in split order
+      constexpr int NSP = decltype(nsp_tag)::value;
+      float2 va[NSP][4], vb[NSP][4];
+#pragma unroll
+      for (int u = 0; u < NSP; ++u) {
+        const float* pp = p.partial + (size_t)(sp + u) * sstride + c0 + 2 * t;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+          const bool cok = c0 + nt * 8 < p.N;
+          va[u][nt] = (okA && cok) ? __ldcg(reinterpret_cast<const float2*>(pp + (size_t)mA * p.N + nt * 8)) : make_float2(0.f, 0.f);
+          vb[u][nt] = (okB && cok) ? __ldcg(reinterpret_cast<const float2*>(pp + (size_t)mB * p.N + nt * 8)) : make_float2(0.f, 0.f);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < NSP; ++u)
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+          acc[nt][0] += va[u][nt].x; acc[nt][1] += va[u][nt].y; acc[nt][2] += vb[u][nt].x; acc[nt][3] += vb[u][nt].y;
+        }
+    };
+    int sp = 0;
+    for (; sp + 4 <= ksplit; sp += 4) add_splits(sp, std::integral_constant<int, 4>());
+    for (; sp < ksplit; ++sp) add_splits(sp, std::integral_constant<int, 1>());
+    if (p.lora.adapter_idx != nullptr) {
+      if (a >= 0 && a < p.lora.n_slots) {
+        const int r = p.lora.rank;
+        int seg_of[4], col_of[4];
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) tc_map_col(p.mode, min(c0 + nt * 8, p.N - 8), p.seg_n0, p.seg_n1, seg_of[nt], col_of[nt]);
+        for (int seg = 0; seg < p.lora.nseg; ++seg) {
+          bool any = false;
+#pragma unroll
+          for (int nt = 0; nt < 4; ++nt) any = any || (seg_of[nt] == seg && c0 + nt * 8 < p.N);
+          const __half* B = p.lora.tabB[(size_t)a * p.lora.tab_stride + p.lora.seg[seg].proj_index];
+          if (!any || B == nullptr) continue;
+          const int ldb = p.lora.seg[seg].n;
+          const float* TA = p.lora.T + ((size_t)mA * p.lora.nseg + seg) * r;
+          const float* TB = p.lora.T + ((size_t)mB * p.lora.nseg + seg) * r;
+          for (int k0 = 0; k0 < r; k0 += 16) {
+            // A fragments of T: a0 = (row mA, k 2t, 2t+1), a1 = (row mB, same k), a2 / a3 = the same rows, k + 8
+            uint32_t ah[4], al[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float* Tr = (q & 1) ? TB : TA;
+              const bool rok = (q & 1) ? okB : okA;
+              const int k = k0 + 2 * t + (q >> 1) * 8;
+              const float x0 = (rok && k < r) ? Tr[k] : 0.f, x1 = (rok && k + 1 < r) ? Tr[k + 1] : 0.f;
+              const __half h0 = __float2half_rn(x0), h1 = __float2half_rn(x1);
+              ah[q] = h2_as_u32(__halves2half2(h0, h1));
+              al[q] = h2_as_u32(__floats2half2_rn(x0 - __half2float(h0), x1 - __half2float(h1)));
+            }
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+              if (seg_of[nt] != seg || c0 + nt * 8 >= p.N) continue;      // uniform over the warp
+              // B fragment: b0 = (k 2t, 2t+1; column g), b1 = (k + 8; column g)
+              const unsigned short* Bc = reinterpret_cast<const unsigned short*>(B) + col_of[nt] + g;
+              const int k = k0 + 2 * t;
+              const uint32_t e0 = k < r ? __ldg(Bc + (size_t)k * ldb) : 0u, e1 = k + 1 < r ? __ldg(Bc + (size_t)(k + 1) * ldb) : 0u;
+              const uint32_t e2 = k + 8 < r ? __ldg(Bc + (size_t)(k + 8) * ldb) : 0u, e3 = k + 9 < r ? __ldg(Bc + (size_t)(k + 9) * ldb) : 0u;
+              const uint32_t b0 = e0 | (e1 << 16), b1 = e2 | (e3 << 16);
+              mma_16816(acc[nt], ah, b0, b1);
+              mma_16816(acc[nt], al, b0, b1);
+            }
+          }
+        }
+      }
+    }
+    if (SWIGLU) {
+      // columns c0 .. c0+15 are a gate tile (n-tiles 0, 1), c0+16 .. c0+31 its up tile (n-tiles 2, 3)
+      if (c0 >= p.N) continue;
+      const int f0 = (c0 >> 5) << 4;
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        float v[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { const float gv = acc[nt][e]; v[e] = gv / (1.f + __expf(-gv)) * acc[nt + 2][e]; }
+        const int f = f0 + nt * 8 + 2 * t;
+        if (okA) *reinterpret_cast<__half2*>(p.out_f16 + (size_t)mA * (p.N / 2) + f) = __floats2half2_rn(v[0], v[1]);
+        if (okB) *reinterpret_cast<__half2*>(p.out_f16 + (size_t)mB * (p.N / 2) + f) = __floats2half2_rn(v[2], v[3]);
+      }
+    } else {
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+        const int c = c0 + nt * 8 + 2 * t;
+        if (c >= p.N) continue;
+        if (p.epi == EPI_F32) {
+          if (okA) *reinterpret_cast<float2*>(p.out_f32 + (size_t)mA * p.ldo + c) = make_float2(acc[nt][0], acc[nt][1]);
+          if (okB) *reinterpret_cast<float2*>(p.out_f32 + (size_t)mB * p.ldo + c) = make_float2(acc[nt][2], acc[nt][3]);
+        } else {
+          if (okA) {
+            float2* xp = reinterpret_cast<float2*>(p.resid + (size_t)mA * p.N + c);
+            float2 x = *xp; x.x += acc[nt][0]; x.y += acc[nt][1]; *xp = x;
+          }
+          if (okB) {
+            float2* xp = reinterpret_cast<float2*>(p.resid + (size_t)mB * p.N + c);
+            float2 x = *xp; x.x += acc[nt][2]; x.y += acc[nt][3]; *xp = x;
+          }
+        }
+      }
+    }
+  }
+}
+
 // cuTensorMapEncodeTiled through the runtime's driver entry point lookup (the library does not link libcuda)
 static PFN_cuTensorMapEncodeTiled_v12000 tensor_map_encoder() {
   static PFN_cuTensorMapEncodeTiled_v12000 fn = []() -> PFN_cuTensorMapEncodeTiled_v12000 {
@@ -447,6 +572,16 @@ cudaError_t launch_gemm_tc(const GemmArgs& a, int sm_count, int* status, cudaStr
   else if (nrows == 128) e = tc_launch<128>(a, slabs, ksplit, kts_per_split, status, st);
   else e = tc_launch<256>(a, slabs, ksplit, kts_per_split, status, st);
   if (e != cudaSuccess) return e;
+  const int wtiles = ((a.N + 31) / 32) * ((a.M + 15) / 16);
+  if ((a.lora.adapter_idx == nullptr || a.lora.rows_per_stream % 16 == 0) && a.ldo % 2 == 0 && wtiles >= 8 * sm_count) {
+    // rows come in runs of 16 with one adapter (or none) and there are enough 16 x 32 tiles to give every SM
+    // several warps: the expand term runs on mma.sync (below that size the thread-per-quad kernel hides its
+    // latencies better)
+    const int blocks = (wtiles + 7) / 8;
+    if (a.epi == EPI_SWIGLU) gemm_tc_epilogue_mma_kernel<true><<<blocks, 256, 0, st>>>(a, ksplit);
+    else gemm_tc_epilogue_mma_kernel<false><<<blocks, 256, 0, st>>>(a, ksplit);
+    return cudaGetLastError();
+  }
   const long long total = (long long)a.M * (a.N / 4);
   int blocks = (int)((total + 255) / 256);
   if (blocks > sm_count * 8) blocks = sm_count * 8;
