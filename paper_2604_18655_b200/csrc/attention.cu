@@ -408,6 +408,217 @@ __global__ void attn_merge_kernel(const AttnArgs p) {
   merge_row(p, hq / g_heads, m * g_heads + hq % g_heads, m, hq, lane);
 }
 
+// ----------------------------------------------------------------------------- single-pass decode attention
+// One decode row per stream (T = 1) and a short context: one CTA per (kv head, stream) does the whole softmax, so
+// there are no partial results in global memory and no merge kernel.  The shared prefix is re-read by every stream's
+// CTA, but from L2: HBM still sees it once.  The warps take 32-key tiles of (prefix ++ own segment) round-robin, each
+// with its own double-buffered K/V tiles (cp.async) and its own online softmax over the kv head's query heads (one
+// m16 tile, rows past the group zero); the warps' results are combined by log-sum-exp in shared memory.  The new
+// K/V row of the pass is built from the projections (k rotated), used, and appended to the cache by the warp whose
+// tile holds it.
+constexpr int DEC_KEYS = 32;
+__host__ __device__ constexpr int dec_warps(int hd) { return hd == 64 ? 8 : 4; }
+__host__ __device__ constexpr size_t dec_smem_bytes(int hd) {
+  return (size_t)16 * (hd + 8) * 2 + (size_t)dec_warps(hd) * 4 * DEC_KEYS * (hd + 8) * 2 +
+         (size_t)dec_warps(hd) * 16 * (hd + 2) * 4;
+}
+
+template <int HD>
+__global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const AttnArgs p, const float scale_log2) {
+  constexpr int W = dec_warps(HD), STRIDE = HD + 8, KSTEPS = HD / 16, DT = HD / 8, VPR = HD / 8;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __half* Qs = reinterpret_cast<__half*>(smem_raw);                       // [16][STRIDE]
+  __half* tiles = Qs + 16 * STRIDE;                                       // [W][2 buffers][K, V][DEC_KEYS][STRIDE]
+  float* part_o = reinterpret_cast<float*>(tiles + (size_t)W * 4 * DEC_KEYS * STRIDE);   // [W][16][HD]
+  float* part_ml = part_o + (size_t)W * 16 * HD;                          // [W][16][2]
+
+  const int kh = blockIdx.x, s = blockIdx.y;
+  const int g_heads = p.Hq / p.Hkv;
+  const bool fused = p.qkv_f32 != nullptr;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int n_ptiles = (p.P + DEC_KEYS - 1) / DEC_KEYS;
+  int S = 0, own_keys = 0, n_tiles = n_ptiles;                            // known once suffix_len has arrived
+  const __half* pk = p.prefix_k + (size_t)kh * p.prefix_head_stride;
+  const __half* pv = p.prefix_v + (size_t)kh * p.prefix_head_stride;
+  __half* ok = const_cast<__half*>(p.own_k) + (size_t)s * p.own_stream_stride + (size_t)kh * p.own_head_stride;
+  __half* ov = const_cast<__half*>(p.own_v) + (size_t)s * p.own_stream_stride + (size_t)kh * p.own_head_stride;
+  const int m = s;                                                        // the stream's row (T = 1)
+  const float* prow = fused ? p.qkv_f32 + (size_t)m * (size_t)((p.Hq + 2 * p.Hkv) * HD) : nullptr;
+  const float2* cs = nullptr;
+
+  __half* my_tiles = tiles + (size_t)warp * 4 * DEC_KEYS * STRIDE;
+  auto load_tile = [&](int ti, int buf) {
+    __half* kd = my_tiles + (size_t)buf * 2 * DEC_KEYS * STRIDE;
+    __half* vd = kd + DEC_KEYS * STRIDE;
+    const bool own = ti >= n_ptiles;
+    const int k0 = (own ? ti - n_ptiles : ti) * DEC_KEYS;
+    const int kend = own ? own_keys : p.P;
+    const __half* kb = own ? ok : pk;
+    const __half* vb = own ? ov : pv;
+    for (int i = lane; i < DEC_KEYS * VPR; i += 32) {
+      const int r = i / VPR, c = (i % VPR) * 8, key = k0 + r;
+      if (key >= kend) {
+        *reinterpret_cast<uint4*>(kd + (size_t)r * STRIDE + c) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(vd + (size_t)r * STRIDE + c) = make_uint4(0, 0, 0, 0);
+      } else if (fused && own && key == S) {
+        const uint4 kv8 = head_piece_f16(prow + (size_t)(p.Hq + kh) * HD, c, HD, cs);
+        const uint4 vv8 = head_piece_f16(prow + (size_t)(p.Hq + p.Hkv + kh) * HD, c, HD, nullptr);
+        *reinterpret_cast<uint4*>(kd + (size_t)r * STRIDE + c) = kv8;
+        *reinterpret_cast<uint4*>(vd + (size_t)r * STRIDE + c) = vv8;
+        *reinterpret_cast<uint4*>(ok + (size_t)key * HD + c) = kv8;
+        *reinterpret_cast<uint4*>(ov + (size_t)key * HD + c) = vv8;
+      } else {
+        cp_async16(kd + (size_t)r * STRIDE + c, kb + (size_t)key * HD + c);
+        cp_async16(vd + (size_t)r * STRIDE + c, vb + (size_t)key * HD + c);
+      }
+    }
+    cp_async_commit();
+  };
+  // a warp whose first tile lies in the shared prefix starts it before anything that depends on the stream
+  if (warp < n_ptiles) load_tile(warp, 0);
+  S = p.suffix_len[s];
+  own_keys = S + 1;                                                       // cached rows + this pass's row
+  n_tiles = n_ptiles + (own_keys + DEC_KEYS - 1) / DEC_KEYS;
+  if (fused) cs = p.cs_table + (size_t)(p.pos_base + S + p.depth[m]) * (HD / 2);
+  if (warp >= n_ptiles && warp < n_tiles) load_tile(warp, 0);
+  if (warp + W < n_tiles) load_tile(warp + W, 1);
+
+  // the group's query rows (rotated on load in fused mode), zero past the group
+  for (int i = threadIdx.x; i < 16 * VPR; i += W * 32) {
+    const int r = i / VPR, c = (i % VPR) * 8;
+    uint4 val = make_uint4(0, 0, 0, 0);
+    if (r < g_heads) {
+      if (fused) val = head_piece_f16(prow + (size_t)(kh * g_heads + r) * HD, c, HD, cs);
+      else val = *reinterpret_cast<const uint4*>(p.q + ((size_t)m * p.Hq + kh * g_heads + r) * HD + c);
+    }
+    *reinterpret_cast<uint4*>(Qs + (size_t)r * STRIDE + c) = val;
+  }
+  __syncthreads();
+  uint32_t qf[KSTEPS][4];
+#pragma unroll
+  for (int ks = 0; ks < KSTEPS; ++ks) {
+    const int mi = lane >> 3, r = lane & 7;
+    ldmatrix_x4(qf[ks], Qs + (size_t)((mi & 1) * 8 + r) * STRIDE + ks * 16 + (mi >> 1) * 8);
+  }
+
+  float o[DT][4];
+#pragma unroll
+  for (int i = 0; i < DT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+  float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
+
+  int buf = 0;
+  for (int ti = warp; ti < n_tiles; ti += W, buf ^= 1) {
+    if (ti + W < n_tiles) cp_async_wait<1>();              // the next tile may still be in flight
+    else cp_async_wait<0>();
+    __syncwarp();
+    const __half* kt = my_tiles + (size_t)buf * 2 * DEC_KEYS * STRIDE;
+    const __half* vt = kt + DEC_KEYS * STRIDE;
+    const bool own = ti >= n_ptiles;
+    const int k0 = (own ? ti - n_ptiles : ti) * DEC_KEYS, kend = own ? own_keys : p.P;
+    float sacc[DEC_KEYS / 8][4];
+#pragma unroll
+    for (int nt = 0; nt < DEC_KEYS / 8; ++nt) {
+      sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < KSTEPS; ks += 2) {
+        uint32_t kb[4];
+        const int mi = lane >> 3, r = lane & 7;
+        ldmatrix_x4(kb, kt + (size_t)(nt * 8 + r) * STRIDE + ks * 16 + mi * 8);
+        mma_16816(sacc[nt], qf[ks], kb[0], kb[1]);
+        mma_16816(sacc[nt], qf[ks + 1], kb[2], kb[3]);
+      }
+    }
+    float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int nt = 0; nt < DEC_KEYS / 8; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int key = k0 + nt * 8 + 2 * t + (e & 1);
+        const float v = key < kend ? sacc[nt][e] * scale_log2 : -INFINITY;
+        sacc[nt][e] = v;
+        mx[e >> 1] = fmaxf(mx[e >> 1], v);
+      }
+    }
+    float corr[2], msafe[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+      mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
+      const float mnew = fmaxf(mrow[h], mx[h]);
+      msafe[h] = (mnew == -INFINITY) ? 0.f : mnew;
+      corr[h] = exp2f(mrow[h] - msafe[h]);
+      mrow[h] = mnew;
+    }
+    float ls[2] = {0.f, 0.f};
+    uint32_t pf[DEC_KEYS / 16][4];
+#pragma unroll
+    for (int nt = 0; nt < DEC_KEYS / 8; ++nt) {
+      const float p0 = exp2f(sacc[nt][0] - msafe[0]), p1 = exp2f(sacc[nt][1] - msafe[0]);
+      const float p2 = exp2f(sacc[nt][2] - msafe[1]), p3 = exp2f(sacc[nt][3] - msafe[1]);
+      ls[0] += p0 + p1;
+      ls[1] += p2 + p3;
+      pf[nt >> 1][(nt & 1) * 2 + 0] = h2_as_u32(__floats2half2_rn(p0, p1));
+      pf[nt >> 1][(nt & 1) * 2 + 1] = h2_as_u32(__floats2half2_rn(p2, p3));
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) lrow[h] = lrow[h] * corr[h] + ls[h];
+#pragma unroll
+    for (int dt = 0; dt < DT; ++dt) {
+      o[dt][0] *= corr[0]; o[dt][1] *= corr[0];
+      o[dt][2] *= corr[1]; o[dt][3] *= corr[1];
+    }
+#pragma unroll
+    for (int kk = 0; kk < DEC_KEYS / 16; ++kk) {
+#pragma unroll
+      for (int dt = 0; dt < DT; dt += 2) {
+        uint32_t vb[4];
+        const int mi = lane >> 3, r = lane & 7;
+        ldmatrix_x4_trans(vb, vt + (size_t)(kk * 16 + (mi & 1) * 8 + r) * STRIDE + (dt + (mi >> 1)) * 8);
+        mma_16816(o[dt], pf[kk], vb[0], vb[1]);
+        mma_16816(o[dt + 1], pf[kk], vb[2], vb[3]);
+      }
+    }
+    __syncwarp();                                        // every lane is done with the buffer: refill it
+    if (ti + 2 * W < n_tiles) load_tile(ti + 2 * W, buf);
+  }
+
+  // this warp's un-normalised output, running max (log2 domain) and sum for the group's rows
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    lrow[h] += __shfl_xor_sync(0xffffffffu, lrow[h], 1);
+    lrow[h] += __shfl_xor_sync(0xffffffffu, lrow[h], 2);
+    const int r = g + 8 * h;
+    if (r >= g_heads) continue;
+    float* po = part_o + ((size_t)warp * 16 + r) * HD;
+#pragma unroll
+    for (int dt = 0; dt < DT; ++dt) *reinterpret_cast<float2*>(po + dt * 8 + 2 * t) = make_float2(o[dt][2 * h], o[dt][2 * h + 1]);
+    if (t == 0) *reinterpret_cast<float2*>(part_ml + ((size_t)warp * 16 + r) * 2) = make_float2(mrow[h], lrow[h]);
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < g_heads * HD; i += W * 32) {
+    const int r = i / HD, d = i % HD;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < W; ++w) M = fmaxf(M, part_ml[((size_t)w * 16 + r) * 2]);
+    float num = 0.f, den = 0.f;
+#pragma unroll
+    for (int w = 0; w < W; ++w) {                          // warp order: fixed
+      const float mw = part_ml[((size_t)w * 16 + r) * 2];
+      if (mw == -INFINITY) continue;                       // a warp without tiles
+      const float f = exp2f(mw - M);
+      num += f * part_o[((size_t)w * 16 + r) * HD + d];
+      den += f * part_ml[((size_t)w * 16 + r) * 2 + 1];
+    }
+    p.out[((size_t)m * p.Hq + kh * g_heads + r) * HD + d] = __float2half_rn(den > 0.f ? num / den : 0.f);
+  }
+}
+
+// one decode row per stream, a context short enough for one CTA per (kv head, stream), at most 16 query heads per
+// kv head
+bool attn_single_pass(const AttnArgs& a) {
+  return a.T == 1 && a.Hq / a.Hkv <= 16 && a.P + a.suffix_bound + 1 <= 2048 && (a.hd == 64 || a.hd == 128);
+}
+
 void attn_plan(AttnArgs& a, int sm_count) {
   const int g_heads = a.Hq / a.Hkv;
   const int R_all = a.n * a.T * g_heads;
@@ -458,17 +669,29 @@ cudaError_t init_attention() {
   cudaError_t e = cudaFuncSetAttribute(attn_partial_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)((ATT_ROWS + 4 * ATT_KEYS) * (64 + 8) * sizeof(__half)));
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attn_decode_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem_bytes(64));
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attn_decode_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem_bytes(128));
+  if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(attn_partial_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)((ATT_ROWS + 4 * ATT_KEYS) * (128 + 8) * sizeof(__half)));
 }
 
 cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st) {
+  if (attn_single_pass(a)) {
+    dim3 grid(a.Hkv, a.n);
+    const float scale_log2 = 1.4426950408889634f / sqrtf((float)a.hd);
+    if (a.hd == 64) attn_decode_kernel<64><<<grid, dec_warps(64) * 32, dec_smem_bytes(64), st>>>(a, scale_log2);
+    else attn_decode_kernel<128><<<grid, dec_warps(128) * 32, dec_smem_bytes(128), st>>>(a, scale_log2);
+    return cudaGetLastError();
+  }
   if (a.hd == 64) return launch_attn_hd<64>(a, st);
   if (a.hd == 128) return launch_attn_hd<128>(a, st);
   return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_attention_merge(const AttnArgs& a, cudaStream_t st) {
+  if (attn_single_pass(a)) return cudaSuccess;             // nothing to merge
   const int warps = a.n * a.T * a.Hq;
   attn_merge_kernel<<<(warps + 3) / 4, 128, 0, st>>>(a);
   return cudaGetLastError();

@@ -205,6 +205,7 @@ cudaError_t launch_tree_prep(const int32_t* parent, int n, int T, unsigned long 
                              int* status, cudaStream_t st);
 void attn_plan(AttnArgs& a, int sm_count);
 size_t attn_workspace_floats(const AttnArgs& a);
+bool attn_single_pass(const AttnArgs& a);          // one kernel does the whole softmax: no merge launch follows
 cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st);
 cudaError_t launch_attention_merge(const AttnArgs& a, cudaStream_t st);
 cudaError_t launch_argmax(const float* logits, int M, int V, int32_t* out, cudaStream_t st);

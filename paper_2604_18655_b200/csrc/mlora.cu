@@ -220,7 +220,7 @@ int launch_attention_block(mlora_ctx* c, const PassIO& io, int l) {
   a.part_o = c->att_ws;
   a.part_ml = c->att_ws + (attn_workspace_floats(a) / (a.hd + 2)) * a.hd;
   CK(run(c, MLORA_PROF_ATTN, [&] { return launch_attention(a, st); }));
-  CK(run(c, MLORA_PROF_ATTN_MERGE, [&] { return launch_attention_merge(a, st); }));
+  if (!attn_single_pass(a)) CK(run(c, MLORA_PROF_ATTN_MERGE, [&] { return launch_attention_merge(a, st); }));
   return MLORA_OK;
 }
 
