@@ -661,48 +661,57 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
         const int ubase = pos + k * tpu * L.nchunks;                      // first stage of the unit
         for (int tu = 0; tu < tpu; ++tu) {
           float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
-          int waited = -1;
-          for (int it = it_lo; it < it_hi; ++it) {
-            const int c = it / CH_ITEMS_PER_CHUNK;
+          // the warp's items it_lo .. it_hi-1 lie in consecutive chunks; stage and parity of a chunk are stepped,
+          // not divided out again (the loop is a serial chain per warp: every instruction in it counts)
+          int c = it_lo / CH_ITEMS_PER_CHUNK;
+          int st = 0;
+          uint32_t par = 0;
+          if (it_lo < it_hi) {
+            const int P0 = ubase + tu * L.nchunks + c;
+            st = pos_stage(P0, nstages);
+            par = pos_parity(P0, nstages);
+          }
+          const __half* hrow = hs + (size_t)g * hs_stride + 16 * t;
+          for (int it = it_lo; it < it_hi; ++c) {
             const int kc = (c == L.nchunks - 1) ? L.kc_last : CHUNK_KT;
-            const int P = ubase + tu * L.nchunks + c;
-            const int st = pos_stage(P, nstages);
-            bool ok = true;
-            if (P != waited) {
-              ok = wait_mbar(smem_u32(full_bar + st), pos_parity(P, nstages), wc, 3, p);
-              waited = P;
-            }
-            const int itl = it - c * CH_ITEMS_PER_CHUNK;                  // item inside its chunk
-            const int ktl = itl * CH_ITEM_KT;                             // its first k-tile inside the chunk
-            if (ok) {
-              const unsigned char* sb = ring + (size_t)st * CH_STAGE_BYTES;
-              const __half* hbase = hs + (size_t)g * hs_stride + (size_t)(c * CHUNK_KT + ktl) * TILE_K + 16 * t;
+            const int items_here = (kc + CH_ITEM_KT - 1) / CH_ITEM_KT;
+            const int it_end = min(it_hi, (c + 1) * CH_ITEMS_PER_CHUNK);
+            const bool ok = wait_mbar(smem_u32(full_bar + st), par, wc, 3, p);
+            const unsigned char* sb = ring + (size_t)st * CH_STAGE_BYTES;
+            const unsigned char* ssc = sb + kc * 512 + g * 4;
+            const uint32_t ebar = smem_u32(empty_bar + st);
+            for (; it < it_end; ++it) {
+              const int itl = it - c * CH_ITEMS_PER_CHUNK;                // item inside its chunk
+              const int ktl = itl * CH_ITEM_KT;                           // its first k-tile inside the chunk
+              if (ok) {
+                const __half* hbase = hrow + (size_t)(c * CHUNK_KT + ktl) * TILE_K;
 #pragma unroll
-              for (int q = 0; q < CH_ITEM_KT; ++q) {
-                if (ktl + q < kc) {
-                  const uint4 wv = *reinterpret_cast<const uint4*>(sb + (ktl + q) * 512 + lane * 16);
-                  const uint32_t sw = *reinterpret_cast<const uint32_t*>(sb + kc * 512 + ((ktl + q) >> gshift) * 32 + g * 4);
-                  const uint4 b01 = *reinterpret_cast<const uint4*>(hbase + q * TILE_K);
-                  const uint4 b23 = *reinterpret_cast<const uint4*>(hbase + q * TILE_K + 8);
-                  __half2 s_lo, s_hi;
-                  split_scales(sw, s_lo, s_hi);
-                  uint32_t af[4][4];
-                  dequant8(wv.x, s_lo, s_hi, af[0]);
-                  dequant8(wv.y, s_lo, s_hi, af[1]);
-                  dequant8(wv.z, s_lo, s_hi, af[2]);
-                  dequant8(wv.w, s_lo, s_hi, af[3]);
-                  mma_16816(acc0, af[0], b01.x, b01.y);
-                  mma_16816(acc1, af[1], b01.z, b01.w);
-                  mma_16816(acc0, af[2], b23.x, b23.y);
-                  mma_16816(acc1, af[3], b23.z, b23.w);
+                for (int q = 0; q < CH_ITEM_KT; ++q) {
+                  if (ktl + q < kc) {
+                    const uint4 wv = *reinterpret_cast<const uint4*>(sb + (ktl + q) * 512 + lane * 16);
+                    const uint32_t sw = *reinterpret_cast<const uint32_t*>(ssc + ((ktl + q) >> gshift) * 32);
+                    const uint4 b01 = *reinterpret_cast<const uint4*>(hbase + q * TILE_K);
+                    const uint4 b23 = *reinterpret_cast<const uint4*>(hbase + q * TILE_K + 8);
+                    __half2 s_lo, s_hi;
+                    split_scales(sw, s_lo, s_hi);
+                    uint32_t af[4][4];
+                    dequant8(wv.x, s_lo, s_hi, af[0]);
+                    dequant8(wv.y, s_lo, s_hi, af[1]);
+                    dequant8(wv.z, s_lo, s_hi, af[2]);
+                    dequant8(wv.w, s_lo, s_hi, af[3]);
+                    mma_16816(acc0, af[0], b01.x, b01.y);
+                    mma_16816(acc1, af[1], b01.z, b01.w);
+                    mma_16816(acc0, af[2], b23.x, b23.y);
+                    mma_16816(acc1, af[3], b23.z, b23.w);
+                  }
                 }
               }
+              __syncwarp();
+              // one arrival per item; the last item of a ragged chunk also arrives for the items the chunk lacks
+              const int arrivals = (itl == items_here - 1) ? CH_ITEMS_PER_CHUNK - items_here + 1 : 1;
+              if (lane < arrivals) mbar_arrive(ebar);
             }
-            __syncwarp();
-            // one arrival per item; the last item of a ragged chunk also arrives for the items the chunk lacks
-            const int items_here = (kc + CH_ITEM_KT - 1) / CH_ITEM_KT;
-            const int arrivals = (itl == items_here - 1) ? CH_ITEMS_PER_CHUNK - items_here + 1 : 1;
-            if (lane < arrivals) mbar_arrive(smem_u32(empty_bar + st));
+            if (++st == nstages) { st = 0; par ^= 1u; }
           }
           red[(size_t)(tu * CH_CWARPS + warp) * 32 + lane] =
               make_float4(acc0[0] + acc1[0], acc0[1] + acc1[1], acc0[2] + acc1[2], acc0[3] + acc1[3]);
