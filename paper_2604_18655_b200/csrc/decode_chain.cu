@@ -133,6 +133,13 @@ __device__ __forceinline__ void red_release_add_u64(unsigned long long* p, unsig
 __device__ __forceinline__ int pos_stage(int pos, int nstages) { return pos % nstages; }
 __device__ __forceinline__ uint32_t pos_parity(int pos, int nstages) { return (uint32_t)((pos / nstages) & 1); }
 
+// what every consumer thread needs of a phase beyond its descriptor; worked out once per phase by one thread (the
+// divisions in it would otherwise sit at the head of every thread's phase, ahead of its first loads)
+struct PhaseDerived {
+  WLayout L;
+  int tpu, n_units, ipt, gshift, my_units, teams, n_my_items, shr_warps, gemm_warps;
+};
+
 // ----------------------------------------------------------------------------- bounded waits
 struct WaitCtx {
   long long limit;                  // clock cycles a wait may take
@@ -284,6 +291,7 @@ __device__ __forceinline__ void norm_rows(const float* __restrict__ x, const __h
 __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const ChainArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ ChainPhase s_ph[2];
+  __shared__ PhaseDerived s_pd[2];
   __shared__ const __half* s_pA[2][3][CHAIN_MAX_ROWS];
   __shared__ const __half* s_pB[2][3][CHAIN_MAX_ROWS];
   __shared__ float s_scale[CHAIN_MAX_ROWS];
@@ -360,7 +368,45 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
       s_pB[slot][seg][m] = pb;
     }
   };
-  if (warp == 0) prep_phase(a.p0);
+  // the phase's derived values, by one thread, once its descriptor is in shared memory
+  auto derive_phase = [&](int p) {
+    const int slot = (p - a.p0) & 1;
+    {
+      const ChainPhase& ph = s_ph[slot];
+      PhaseDerived d;
+      d.L = make_wlayout(ph.K, ph.N, ph.G);
+      const int nseg = lora_on ? ph.lora_nseg : 0;
+      d.tpu = (ph.mode == MODE_GATEUP) ? 2 : 1;
+      d.n_units = d.L.NT / d.tpu;
+      d.ipt = (d.L.KT + CH_ITEM_KT - 1) / CH_ITEM_KT;                 // items per tile
+      d.gshift = (d.L.G >= CHUNK_KT * TILE_K) ? 31 : (31 - __clz(d.L.G / TILE_K));   // k-tile -> scale group of its chunk
+      // teams: as many units in flight as the CTA has, as the ring can hold at once (a wait must never be a whole
+      // lap ahead of the fill front: mbarrier parities repeat every two laps) and as the B buffer has room for
+      d.my_units = (d.n_units > (int)blockIdx.x) ? (d.n_units - 1 - (int)blockIdx.x) / (int)G + 1 : 0;
+      int teams = d.my_units < CH_MAX_TEAMS ? d.my_units : CH_MAX_TEAMS;
+      if (teams > nstages / (d.tpu * d.L.nchunks)) teams = nstages / (d.tpu * d.L.nchunks);
+      if (nseg > 0 && teams > CH_BS_BYTES / (d.tpu * CHAIN_MAX_ROWS * r * 32)) teams = CH_BS_BYTES / (d.tpu * CHAIN_MAX_ROWS * r * 32);
+      if (teams < 1) teams = 1;
+      // LoRA phases: the CTA's shrink items (row, segment, rank index) run on the last shr_warps warps, off the
+      // critical path of the GEMM teams, which share the other warps
+      d.n_my_items = 0;
+      if (nseg > 0) {
+        const int n_items = M * nseg * r;
+        d.n_my_items = (n_items > (int)blockIdx.x) ? (n_items - 1 - (int)blockIdx.x) / (int)G + 1 : 0;
+        if (d.n_my_items > CH_MAX_ITEMS) d.n_my_items = CH_MAX_ITEMS;
+      }
+      d.shr_warps = nseg > 0 ? (d.n_my_items < 4 ? (d.n_my_items > 0 ? d.n_my_items : 1) : 4) : 0;
+      d.gemm_warps = CH_CWARPS - d.shr_warps;
+      if (teams > d.gemm_warps) teams = d.gemm_warps;
+      d.teams = teams;
+      s_pd[slot] = d;
+    }
+  };
+  if (warp == 0) {
+    prep_phase(a.p0);
+    __syncwarp();
+    if (lane == 0) derive_phase(a.p0);
+  }
   __syncthreads();
 
   // =========================================================================== producer warp
@@ -477,34 +523,15 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     const ChainPhase& ph = s_ph[slot];
     const int K = ph.K;
     const int hs_stride = K + 8;
-    const WLayout L = make_wlayout(K, ph.N, ph.G);
+    const PhaseDerived& pd = s_pd[slot];
+    const WLayout L = pd.L;
     const int nseg = lora_on ? ph.lora_nseg : 0;
 #ifdef CHAIN_TRACE
     int tr_n = 0;
 #endif
     STAMP(0);
-    const int tpu = (ph.mode == MODE_GATEUP) ? 2 : 1;
-    const int n_units = L.NT / tpu;
-    const int ipt = (L.KT + CH_ITEM_KT - 1) / CH_ITEM_KT;             // items per tile
-    const int gshift = (L.G >= CHUNK_KT * TILE_K) ? 31 : (31 - __clz(L.G / TILE_K));   // k-tile -> scale group of its chunk
-    // teams: as many units in flight as the CTA has, as the ring can hold at once (a wait must never be a whole
-    // lap ahead of the fill front: mbarrier parities repeat every two laps) and as the B buffer has room for
-    const int my_units = (n_units > (int)blockIdx.x) ? (n_units - 1 - (int)blockIdx.x) / (int)G + 1 : 0;
-    int teams = my_units < CH_MAX_TEAMS ? my_units : CH_MAX_TEAMS;
-    if (teams > nstages / (tpu * L.nchunks)) teams = nstages / (tpu * L.nchunks);
-    if (nseg > 0 && teams > CH_BS_BYTES / (tpu * CHAIN_MAX_ROWS * r * 32)) teams = CH_BS_BYTES / (tpu * CHAIN_MAX_ROWS * r * 32);
-    if (teams < 1) teams = 1;
-    // LoRA phases: the CTA's shrink items (row, segment, rank index) run on the last shr_warps warps, off the
-    // critical path of the GEMM teams, which share the other warps
-    int n_my_items = 0;
-    if (nseg > 0) {
-      const int n_items = M * nseg * r;
-      n_my_items = (n_items > (int)blockIdx.x) ? (n_items - 1 - (int)blockIdx.x) / (int)G + 1 : 0;
-      if (n_my_items > CH_MAX_ITEMS) n_my_items = CH_MAX_ITEMS;
-    }
-    const int shr_warps = nseg > 0 ? (n_my_items < 4 ? (n_my_items > 0 ? n_my_items : 1) : 4) : 0;
-    const int gemm_warps = CH_CWARPS - shr_warps;
-    if (teams > gemm_warps) teams = gemm_warps;
+    const int tpu = pd.tpu, ipt = pd.ipt, gshift = pd.gshift, my_units = pd.my_units, teams = pd.teams;
+    const int n_my_items = pd.n_my_items, shr_warps = pd.shr_warps, gemm_warps = pd.gemm_warps;
     // the teams are formed anew for every round of units: the last round may have fewer units than teams, and
     // then all GEMM warps share what is left
     int teams_r = 0, wpt = 1, tm = 0, member = 0, team_threads = 32, tt = 0;
@@ -792,6 +819,9 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
         // (test hook: with inject_stall the first barrier of the launch waits for one arrival too many)
         wait_counter(a.sync + 0, s_base[0] + n_bar * G + ((a.inject_stall && n_bar == 1) ? 1ull : 0ull), wc, 5, p);
       }
+      // while thread 0 waits for the other CTAs: the next phase's derived values (its descriptor was loaded
+      // before the barrier above)
+      if (tid == 32) derive_phase(p + 1);
       consumer_sync();
     }
     STAMP(8);
