@@ -81,7 +81,7 @@ size_t chain_smem_bytes(int kmax, int rank, int nstages) { return chain_carve(km
 
 int chain_pick_stages(int kmax, int rank) {
   if (rank > CHAIN_MAX_RANK || kmax % TILE_K) return 0;
-  const size_t limit = 227 * 1024 - 2048;        // static shared memory of the kernel comes on top
+  const size_t limit = 227 * 1024 - 2560;        // static shared memory of the kernel comes on top
   const size_t base = chain_carve(kmax, rank, 0).total;
   if (base >= limit) return 0;
   int n = (int)((limit - base) / CH_STAGE_BYTES);
@@ -138,6 +138,9 @@ __device__ __forceinline__ uint32_t pos_parity(int pos, int nstages) { return (u
 struct PhaseDerived {
   WLayout L;
   int tpu, n_units, ipt, gshift, my_units, teams, n_my_items, shr_warps, gemm_warps;
+  int n_valid;                       // the CTA's shrink items whose row has an adapter, in item order
+  int item_i[CH_MAX_ITEMS];          // their index (row, segment, rank index) = position in T
+  int item_sm[CH_MAX_ITEMS];         // their segment | row << 8
 };
 
 // ----------------------------------------------------------------------------- bounded waits
@@ -317,6 +320,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
   const unsigned G = gridDim.x;
   const int M = a.M;
   const int r = a.rank;
+  const int r2_shift = (r > 0 && (r & (r - 1)) == 0) ? 32 - __clz(r) : -1;   // log2(2 r) for power-of-two ranks
   const bool lora_on = a.adapter_idx != nullptr && a.rank > 0;
   WaitCtx wc{a.wait_cycles > 0 ? a.wait_cycles : CH_WAIT_CYCLES, &s_abort_word, a.sync, a.status};
 
@@ -373,7 +377,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     const int slot = (p - a.p0) & 1;
     {
       const ChainPhase& ph = s_ph[slot];
-      PhaseDerived d;
+      PhaseDerived& d = s_pd[slot];
       d.L = make_wlayout(ph.K, ph.N, ph.G);
       const int nseg = lora_on ? ph.lora_nseg : 0;
       d.tpu = (ph.mode == MODE_GATEUP) ? 2 : 1;
@@ -395,11 +399,19 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
         d.n_my_items = (n_items > (int)blockIdx.x) ? (n_items - 1 - (int)blockIdx.x) / (int)G + 1 : 0;
         if (d.n_my_items > CH_MAX_ITEMS) d.n_my_items = CH_MAX_ITEMS;
       }
+      d.n_valid = 0;
+      for (int k = 0; k < d.n_my_items; ++k) {
+        const int i = blockIdx.x + k * (int)G;
+        const int seg = (i / r) % nseg, m = i / (r * nseg);
+        if (s_pA[slot][seg][m] == nullptr) continue;
+        d.item_i[d.n_valid] = i;
+        d.item_sm[d.n_valid] = seg | (m << 8);
+        ++d.n_valid;
+      }
       d.shr_warps = nseg > 0 ? (d.n_my_items < 4 ? (d.n_my_items > 0 ? d.n_my_items : 1) : 4) : 0;
       d.gemm_warps = CH_CWARPS - d.shr_warps;
       if (teams > d.gemm_warps) teams = d.gemm_warps;
       d.teams = teams;
-      s_pd[slot] = d;
     }
   };
   if (warp == 0) {
@@ -531,7 +543,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
 #endif
     STAMP(0);
     const int tpu = pd.tpu, ipt = pd.ipt, gshift = pd.gshift, my_units = pd.my_units, teams = pd.teams;
-    const int n_my_items = pd.n_my_items, shr_warps = pd.shr_warps, gemm_warps = pd.gemm_warps;
+    const int shr_warps = pd.shr_warps, gemm_warps = pd.gemm_warps;
     // the teams are formed anew for every round of units: the last round may have fewer units than teams, and
     // then all GEMM warps share what is left
     int teams_r = 0, wpt = 1, tm = 0, member = 0, team_threads = 32, tt = 0;
@@ -553,16 +565,20 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     auto team_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(2 + tm), "r"(team_threads) : "memory"); };
     // LoRA-B slices of unit u -> Bs_team[tile][m][j][16]; immutable, so no need to wait for activations
     auto issue_b = [&](int u) {
-      const int per_tile = CHAIN_MAX_ROWS * r * 2;                     // 16-byte pieces
-      for (int i = tt; i < tpu * per_tile; i += team_threads) {
-        const int tu = i / per_tile, rem = i % per_tile;
-        const int m = rem / (r * 2), j = (rem >> 1) % r, h16 = rem & 1;
+      const int r2 = r * 2;                                            // 16-byte pieces per row of a tile
+      for (int tu = 0; tu < tpu; ++tu) {
         int seg, col;
         chain_map_col(ph.mode, (u * tpu + tu) * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
-        const __half* B = (m < M && seg < nseg) ? s_pB[slot][seg][m] : nullptr;
-        if (B != nullptr)
-          cp_async16_ca(Bs_team + (((size_t)tu * CHAIN_MAX_ROWS + m) * r + j) * 16 + h16 * 8,
-                        B + (size_t)j * ph.lora_n[seg] + col + h16 * 8);
+        if (seg >= nseg) continue;
+        const int ldb = ph.lora_n[seg];
+        for (int idx = tt; idx < M * r2; idx += team_threads) {
+          const int m = r2_shift >= 0 ? idx >> r2_shift : idx / r2;
+          const int x = idx - m * r2, j = x >> 1, h16 = x & 1;
+          const __half* B = s_pB[slot][seg][m];
+          if (B != nullptr)
+            cp_async16_ca(Bs_team + (((size_t)tu * CHAIN_MAX_ROWS + m) * r + j) * 16 + h16 * 8,
+                          B + (size_t)j * ldb + col + h16 * 8);
+        }
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
@@ -621,17 +637,17 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     // are dealt round-robin to the CTAs; item k of the CTA belongs to shrink warp k % shr_warps
     if (nseg > 0) {
       const int np = (K + CH_A_PIECE - 1) / CH_A_PIECE;
-      for (int k = 0; k < n_my_items; ++k) {
-        const int i = blockIdx.x + k * (int)G;
-        const int seg = (i / r) % nseg, m = i / (r * nseg);
-        if (s_pA[slot][seg][m] == nullptr) continue;
-        if (shr_id >= 0 && k % shr_warps == shr_id) {
+      // the items with an adapter were listed when the phase was set up; only the shrink warps walk them
+      if (shr_id >= 0) {
+        for (int kk = shr_id; kk < pd.n_valid; kk += shr_warps) {
+          const int i = pd.item_i[kk], m = pd.item_sm[kk] >> 8;
           const __half* hrow = hs + (size_t)m * hs_stride;
           float acc4[4] = {0.f, 0.f, 0.f, 0.f};
+          int st = pos_stage(pos + kk * np, nstages);
+          uint32_t par = pos_parity(pos + kk * np, nstages);
           for (int q = 0; q < np; ++q) {
             const int k0 = q * CH_A_PIECE;
-            const int st = pos_stage(pos + q, nstages);
-            const bool ok = wait_mbar(smem_u32(full_bar + st), pos_parity(pos + q, nstages), wc, 2, p);
+            const bool ok = wait_mbar(smem_u32(full_bar + st), par, wc, 2, p);
             const unsigned char* sb = ring + (size_t)st * CH_STAGE_BYTES;
             if (ok) {
 #pragma unroll
@@ -653,12 +669,13 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
             }
             __syncwarp();
             if (lane < CH_ITEMS_PER_CHUNK) mbar_arrive(smem_u32(empty_bar + st));
+            if (++st == nstages) { st = 0; par ^= 1u; }
           }
           const float acc = warp_sum((acc4[0] + acc4[1]) + (acc4[2] + acc4[3]));
           if (lane == 0) __stcg(a.T + i, acc * s_scale[m]);
         }
-        pos += np;
       }
+      pos += np * pd.n_valid;
       // the last shrink warp of the CTA to get here tells the grid that this CTA's share of T is written: its
       // release is cumulative over the stores the other shrink warps ordered before their own count-in
       ++n_shr;
@@ -844,7 +861,7 @@ extern "C" int mlora_trace_clear() {
 
 // ----------------------------------------------------------------------------- host side
 cudaError_t init_chain() {
-  return cudaFuncSetAttribute(decode_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048);
+  return cudaFuncSetAttribute(decode_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2560);
 }
 
 cudaError_t launch_chain(const ChainArgs& a, int sm_count, cudaStream_t st) {
