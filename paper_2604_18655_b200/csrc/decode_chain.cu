@@ -71,7 +71,7 @@ bool chain_phase_fits(int K, int mode, int nseg, int rank, int nstages, int sm_c
   if (nseg > 0 && rank > 0) {
     const int items = (CHAIN_MAX_ROWS * nseg * rank + sm_count - 1) / sm_count;
     const int np = (K + CH_A_PIECE - 1) / CH_A_PIECE;
-    if (items > CH_MAX_ITEMS || items * np > nstages) return false;
+    if (items > CH_MAX_ITEMS || items * np > nstages || np > 8) return false;   // 2 np partial sums per item fit 16 slots
     if (CH_BS_BYTES / (tpu * CHAIN_MAX_ROWS * rank * 32) < 1) return false;     // one unit's B slices must fit
   }
   return true;
@@ -81,7 +81,7 @@ size_t chain_smem_bytes(int kmax, int rank, int nstages) { return chain_carve(km
 
 int chain_pick_stages(int kmax, int rank) {
   if (rank > CHAIN_MAX_RANK || kmax % TILE_K) return 0;
-  const size_t limit = 227 * 1024 - 2560;        // static shared memory of the kernel comes on top
+  const size_t limit = 227 * 1024 - 3584;        // static shared memory of the kernel comes on top
   const size_t base = chain_carve(kmax, rank, 0).total;
   if (base >= limit) return 0;
   int n = (int)((limit - base) / CH_STAGE_BYTES);
@@ -215,8 +215,19 @@ __device__ long long g_trace[2 * TR_PHASES * TR_PER_PHASE * 3];
       e_[0] = (id); e_[1] = tns; e_[2] = clock64(); ++tr_n;                                                \
     }                                                                                                      \
   } while (0)
+// the same from lane 0 of the first shrink warp (second half of the phase's record)
+#define STAMPS(id)                                                                                         \
+  do {                                                                                                     \
+    if (shr_id == 0 && lane == 0 && tr_slot >= 0 && tr_n2 < TR_PER_PHASE / 2 && p < TR_PHASES) {           \
+      long long tns;                                                                                       \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tns));                                              \
+      long long* e_ = g_trace + (((size_t)tr_slot * TR_PHASES + p) * TR_PER_PHASE + TR_PER_PHASE / 2 + tr_n2) * 3; \
+      e_[0] = (id); e_[1] = tns; e_[2] = clock64(); ++tr_n2;                                               \
+    }                                                                                                      \
+  } while (0)
 #else
 #define STAMP(id) do { } while (0)
+#define STAMPS(id) do { } while (0)
 #endif
 
 // ----------------------------------------------------------------------------- the ring schedule
@@ -301,7 +312,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
   __shared__ int s_adapter[CHAIN_MAX_ROWS];
   __shared__ int s_abort_word;
   __shared__ unsigned long long s_base[2];
-  __shared__ unsigned s_shr_cnt;                      // warps of this CTA that finished their shrink items
+  __shared__ float s_shr_part[CH_MAX_ITEMS][16];      // shrink: partial sums of an item's half pieces
   __shared__ float s_ssw[CH_CWARPS * CHAIN_MAX_ROWS];  // RMSNorm: per-warp sums of squares of every row
   __shared__ float s_inv[CHAIN_MAX_ROWS];
 
@@ -332,7 +343,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     s_abort_word = (ld_acquire_u64(a.sync + 2) != 0ull) ? 1 : 0;
-    s_shr_cnt = 0u;
     // arrivals of earlier launches are whole multiples of the grid size; arrivals of this launch that are
     // already counted are fewer than one grid
     s_base[0] = ld_acquire_u64(a.sync + 0) / G * G;
@@ -408,7 +418,11 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
         d.item_sm[d.n_valid] = seg | (m << 8);
         ++d.n_valid;
       }
-      d.shr_warps = nseg > 0 ? (d.n_my_items < 4 ? (d.n_my_items > 0 ? d.n_my_items : 1) : 4) : 0;
+      // one shrink warp per half piece of 1024 features, four at most
+      {
+        const int n_half = d.n_valid * 2 * ((ph.K + CH_A_PIECE - 1) / CH_A_PIECE);
+        d.shr_warps = nseg > 0 ? (n_half < 4 ? (n_half > 0 ? n_half : 1) : 4) : 0;
+      }
       d.gemm_warps = CH_CWARPS - d.shr_warps;
       if (teams > d.gemm_warps) teams = d.gemm_warps;
       d.teams = teams;
@@ -525,7 +539,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
   int pos = 0;                                        // stages of this CTA consumed (or skipped) so far
   unsigned long long n_bar = 0;                       // barriers passed in this launch
   unsigned n_shr = 0;                                 // LoRA phases passed in this launch
-  unsigned shr_target = 0;                          // count-ins of shrink warps in the phases before this one
   float* redf = reinterpret_cast<float*>(red);
 #ifdef CHAIN_TRACE
   const int tr_slot = blockIdx.x == 0 ? 0 : (blockIdx.x == G - 1 ? 1 : -1);
@@ -539,7 +552,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     const WLayout L = pd.L;
     const int nseg = lora_on ? ph.lora_nseg : 0;
 #ifdef CHAIN_TRACE
-    int tr_n = 0;
+    int tr_n = 0, tr_n2 = 0;
 #endif
     STAMP(0);
     const int tpu = pd.tpu, ipt = pd.ipt, gshift = pd.gshift, my_units = pd.my_units, teams = pd.teams;
@@ -637,54 +650,70 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     // are dealt round-robin to the CTAs; item k of the CTA belongs to shrink warp k % shr_warps
     if (nseg > 0) {
       const int np = (K + CH_A_PIECE - 1) / CH_A_PIECE;
-      // the items with an adapter were listed when the phase was set up; only the shrink warps walk them
+      // The items with an adapter were listed when the phase was set up; only the shrink warps walk them.  An item
+      // (one rank index of one row: a dot product over K) is cut into half pieces of 1024 features that are dealt
+      // to the shrink warps, so that a long row (K = 5632: six halves) does not sit on one warp; the partial sums
+      // are added in order by the first shrink warp, which also tells the grid that the CTA's share of T is written.
       if (shr_id >= 0) {
-        for (int kk = shr_id; kk < pd.n_valid; kk += shr_warps) {
-          const int i = pd.item_i[kk], m = pd.item_sm[kk] >> 8;
-          const __half* hrow = hs + (size_t)m * hs_stride;
+        STAMPS(10);
+        const int hp = 2 * np;                                            // half pieces per item
+        const int n_half = pd.n_valid * hp;
+        const int st0 = pos_stage(pos, nstages);
+        const uint32_t par0 = pos_parity(pos, nstages);
+        int kk = 0, hq = shr_id;                                          // item and half piece of unit un, stepped
+        for (int un = shr_id; un < n_half; un += shr_warps, hq += shr_warps) {
+          while (hq >= hp) { hq -= hp; ++kk; }
+          const int q = hq >> 1, hf = hq & 1;
+          const int m = pd.item_sm[kk] >> 8;
+          // the CTA's A pieces of a phase fit the ring (checked on the host): at most one wrap from the first
+          int st = st0 + kk * np + q;
+          uint32_t par = par0;
+          if (st >= nstages) { st -= nstages; par ^= 1u; }
+          const bool ok = wait_mbar(smem_u32(full_bar + st), par, wc, 2, p);
+          STAMPS(11);
+          const int k0 = q * CH_A_PIECE + hf * (CH_A_PIECE / 2);
+          const unsigned char* sb = ring + (size_t)st * CH_STAGE_BYTES + hf * CH_A_PIECE;   // bytes: half a piece
+          const __half* hrow = hs + (size_t)m * hs_stride + k0;
           float acc4[4] = {0.f, 0.f, 0.f, 0.f};
-          int st = pos_stage(pos + kk * np, nstages);
-          uint32_t par = pos_parity(pos + kk * np, nstages);
-          for (int q = 0; q < np; ++q) {
-            const int k0 = q * CH_A_PIECE;
-            const bool ok = wait_mbar(smem_u32(full_bar + st), par, wc, 2, p);
-            const unsigned char* sb = ring + (size_t)st * CH_STAGE_BYTES;
-            if (ok) {
+          if (ok) {
 #pragma unroll
-              for (int v = 0; v < CH_A_PIECE / 256; ++v) {
-                const int off = v * 256 + lane * 8;            // halves inside the piece
-                if (k0 + off < K) {
-                  const uint4 av = *reinterpret_cast<const uint4*>(sb + off * 2);
-                  const uint4 hv = *reinterpret_cast<const uint4*>(hrow + k0 + off);
-                  const uint32_t aw[4] = {av.x, av.y, av.z, av.w};
-                  const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
+            for (int v = 0; v < CH_A_PIECE / 512; ++v) {
+              const int off = v * 256 + lane * 8;                         // halves inside the half piece
+              if (k0 + off < K) {
+                const uint4 av = *reinterpret_cast<const uint4*>(sb + off * 2);
+                const uint4 hv = *reinterpret_cast<const uint4*>(hrow + off);
+                const uint32_t aw[4] = {av.x, av.y, av.z, av.w};
+                const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
 #pragma unroll
-                  for (int e = 0; e < 4; ++e) {
-                    const float2 af = __half22float2(u32_as_h2(aw[e])), hf2 = __half22float2(u32_as_h2(hw[e]));
-                    acc4[e] = fmaf(af.x, hf2.x, acc4[e]);
-                    acc4[e] = fmaf(af.y, hf2.y, acc4[e]);
-                  }
+                for (int e = 0; e < 4; ++e) {
+                  const float2 af = __half22float2(u32_as_h2(aw[e])), hf2 = __half22float2(u32_as_h2(hw[e]));
+                  acc4[e] = fmaf(af.x, hf2.x, acc4[e]);
+                  acc4[e] = fmaf(af.y, hf2.y, acc4[e]);
                 }
               }
             }
-            __syncwarp();
-            if (lane < CH_ITEMS_PER_CHUNK) mbar_arrive(smem_u32(empty_bar + st));
-            if (++st == nstages) { st = 0; par ^= 1u; }
           }
+          __syncwarp();
+          if (lane < CH_ITEMS_PER_CHUNK / 2) mbar_arrive(smem_u32(empty_bar + st));   // the two halves free the stage
           const float acc = warp_sum((acc4[0] + acc4[1]) + (acc4[2] + acc4[3]));
-          if (lane == 0) __stcg(a.T + i, acc * s_scale[m]);
+          if (lane == 0) s_shr_part[kk][hq] = acc;
+          STAMPS(12);
+        }
+        asm volatile("bar.sync 11, %0;" ::"r"(shr_warps * 32) : "memory");
+        if (shr_id == 0) {
+          if (lane < pd.n_valid) {
+            float tot = 0.f;
+            for (int hq = 0; hq < hp; ++hq) tot += s_shr_part[lane][hq];
+            __stcg(a.T + pd.item_i[lane], tot * s_scale[pd.item_sm[lane] >> 8]);
+          }
+          // the warp barrier orders the lanes' stores before lane 0's release, which is cumulative over them
+          __syncwarp();
+          if (lane == 0) red_release_add_u64(a.sync + 1, 1ull);
+          STAMPS(13);
         }
       }
       pos += np * pd.n_valid;
-      // the last shrink warp of the CTA to get here tells the grid that this CTA's share of T is written: its
-      // release is cumulative over the stores the other shrink warps ordered before their own count-in
       ++n_shr;
-      if (shr_id >= 0 && lane == 0) {
-        __threadfence_block();
-        const unsigned old = atomicAdd(&s_shr_cnt, 1u);
-        if (old == shr_target + (unsigned)shr_warps - 1u) red_release_add_u64(a.sync + 1, 1ull);
-      }
-      shr_target += (unsigned)shr_warps;
     }
     STAMP(2);
 
@@ -861,7 +890,7 @@ extern "C" int mlora_trace_clear() {
 
 // ----------------------------------------------------------------------------- host side
 cudaError_t init_chain() {
-  return cudaFuncSetAttribute(decode_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2560);
+  return cudaFuncSetAttribute(decode_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 3584);
 }
 
 cudaError_t launch_chain(const ChainArgs& a, int sm_count, cudaStream_t st) {
