@@ -135,6 +135,7 @@ __device__ __forceinline__ uint32_t pos_parity(int pos, int nstages) { return (u
 
 // what every consumer thread needs of a phase beyond its descriptor; worked out once per phase by one thread (the
 // divisions in it would otherwise sit at the head of every thread's phase, ahead of its first loads)
+static_assert(sizeof(ChainPhase) == 128, "a phase descriptor is loaded as one word per lane");
 struct PhaseDerived {
   WLayout L;
   int tpu, n_units, ipt, gshift, my_units, teams, n_my_items, shr_warps, gemm_warps;
@@ -418,10 +419,12 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
         d.item_sm[d.n_valid] = seg | (m << 8);
         ++d.n_valid;
       }
-      // one shrink warp per half piece of 1024 features, four at most
+      // one shrink warp per half piece of 1024 features, four at most for tile pairs
       {
         const int n_half = d.n_valid * 2 * ((ph.K + CH_A_PIECE - 1) / CH_A_PIECE);
-        d.shr_warps = nseg > 0 ? (n_half < 4 ? (n_half > 0 ? n_half : 1) : 4) : 0;
+        // (eight where a unit is a single tile: there the wait for T, not the GEMM, ends the phase)
+        const int cap = d.tpu == 1 ? 8 : 4;
+        d.shr_warps = nseg > 0 ? (n_half < cap ? (n_half > 0 ? n_half : 1) : cap) : 0;
       }
       d.gemm_warps = CH_CWARPS - d.shr_warps;
       if (teams > d.gemm_warps) teams = d.gemm_warps;
@@ -643,8 +646,13 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     consumer_sync();
     STAMP(1);
 
-    // ---- 2. next phase's descriptor and adapter pointers (immutable) while this phase runs
-    if (warp == CH_CWARPS - 1 && p + 1 < a.p1) prep_phase(p + 1);
+    // ---- 2. next phase's descriptor and adapter pointers (immutable) while this phase runs: warp 0 issues the
+    // loads here and stores what they return further down, so neither round trip holds anything up
+    const bool prep_next = warp == 0 && p + 1 < a.p1;
+    const int nslot = slot ^ 1;
+    int prep_word = 0;
+    const __half *prep_pa = nullptr, *prep_pb = nullptr;
+    if (prep_next) prep_word = __ldg(reinterpret_cast<const int*>(a.phases + p + 1) + lane);
 
     // ---- 3. LoRA shrink (first factor of the low-rank term of Eq. 1-4): items (row, segment, rank index)
     // are dealt round-robin to the CTAs; item k of the CTA belongs to shrink warp k % shr_warps
@@ -716,6 +724,19 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
       ++n_shr;
     }
     STAMP(2);
+    if (prep_next) {
+      reinterpret_cast<int*>(&s_ph[nslot])[lane] = prep_word;
+      __syncwarp();
+      if (lane < 3 * CHAIN_MAX_ROWS) {
+        const int seg = lane / CHAIN_MAX_ROWS, m = lane % CHAIN_MAX_ROWS;
+        const int ad = s_adapter[m];
+        if (lora_on && seg < s_ph[nslot].lora_nseg && ad >= 0) {
+          const size_t e = (size_t)ad * a.tab_stride + s_ph[nslot].lora_proj[seg];
+          prep_pa = a.tabA[e];
+          prep_pb = a.tabB[e];
+        }
+      }
+    }
 
     // ---- 4. the CTA's units: one n-tile (or a gate/up pair of n-tiles), all of K
     bool t_loaded = false;
@@ -851,6 +872,11 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
       }
     }
     pos += my_units * tpu * L.nchunks;
+    if (prep_next && lane < 3 * CHAIN_MAX_ROWS) {
+      if (prep_pa == nullptr || prep_pb == nullptr) { prep_pa = nullptr; prep_pb = nullptr; }
+      s_pA[nslot][lane / CHAIN_MAX_ROWS][lane % CHAIN_MAX_ROWS] = prep_pa;
+      s_pB[nslot][lane / CHAIN_MAX_ROWS][lane % CHAIN_MAX_ROWS] = prep_pb;
+    }
     STAMP(6);
 
     // ---- 5. grid barrier: the next phase reads what every CTA wrote
