@@ -455,6 +455,22 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
     const int kend = own ? own_keys : p.P;
     const __half* kb = own ? ok : pk;
     const __half* vb = own ? ov : pv;
+    if (k0 + DEC_KEYS <= kend && !(fused && own && S >= k0 && S < k0 + DEC_KEYS)) {
+      // a full tile of cached rows: straight copies, the addresses stepped
+      constexpr int RPI = 32 / VPR;                                       // rows covered by one pass of the warp
+      const int r0 = lane / VPR, c = (lane % VPR) * 8;
+      const __half* ks = kb + (size_t)(k0 + r0) * HD + c;
+      const __half* vs = vb + (size_t)(k0 + r0) * HD + c;
+      __half* kdp = kd + (size_t)r0 * STRIDE + c;
+      __half* vdp = vd + (size_t)r0 * STRIDE + c;
+#pragma unroll
+      for (int it = 0; it < DEC_KEYS / RPI; ++it) {
+        cp_async16(kdp + (size_t)it * RPI * STRIDE, ks + (size_t)it * RPI * HD);
+        cp_async16(vdp + (size_t)it * RPI * STRIDE, vs + (size_t)it * RPI * HD);
+      }
+      cp_async_commit();
+      return;
+    }
     for (int i = lane; i < DEC_KEYS * VPR; i += 32) {
       const int r = i / VPR, c = (i % VPR) * 8, key = k0 + r;
       if (key >= kend) {
@@ -482,6 +498,18 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   if (fused) cs = p.cs_table + (size_t)(p.pos_base + S + p.depth[m]) * (HD / 2);
   if (warp >= n_ptiles && warp < n_tiles) load_tile(warp, 0);
   if (warp + W < n_tiles) load_tile(warp + W, 1);
+  // the warp's later tiles: ask for them in L2 now, so that their copies two iterations on do not wait for HBM
+  if (lane == 0) {
+    for (int ti = warp + 2 * W; ti < n_tiles; ti += W) {
+      const bool own = ti >= n_ptiles;
+      const int k0 = (own ? ti - n_ptiles : ti) * DEC_KEYS;
+      const int rows = min(DEC_KEYS, (own ? S : p.P) - k0);               // cached rows only
+      if (rows <= 0) continue;
+      const uint32_t bytes = (uint32_t)rows * HD * 2;
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"((own ? ok : pk) + (size_t)k0 * HD), "r"(bytes) : "memory");
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"((own ? ov : pv) + (size_t)k0 * HD), "r"(bytes) : "memory");
+    }
+  }
 
   // the group's query rows (rotated on load in fused mode), zero past the group
   for (int i = threadIdx.x; i < 16 * VPR; i += W * 32) {
