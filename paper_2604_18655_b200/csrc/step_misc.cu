@@ -72,9 +72,23 @@ __global__ void argmax_kernel(const float* __restrict__ logits, int V, int32_t* 
   const float* row = logits + (size_t)m * V;
   float best = -INFINITY;
   int bi = 0x7fffffff;
-  for (int i = threadIdx.x; i < V; i += blockDim.x) {
-    const float v = row[i];
-    if (v > best || (v == best && i < bi)) { best = v; bi = i; }
+  auto take = [&](float v, int i) { if (v > best || (v == best && i < bi)) { best = v; bi = i; } };
+  if ((V & 3) == 0 && (reinterpret_cast<uintptr_t>(row) & 15) == 0) {
+    // four 16-byte loads per thread in flight (a scalar loop pays one L2 round trip per element)
+    const float4* row4 = reinterpret_cast<const float4*>(row);
+    const int nv = V >> 2, bd = blockDim.x;
+    for (int b = threadIdx.x; b < nv; b += 4 * bd) {
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v[u] = (b + u * bd < nv) ? __ldcs(row4 + b + u * bd) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = (b + u * bd) << 2;
+        if (b + u * bd < nv) { take(v[u].x, i); take(v[u].y, i + 1); take(v[u].z, i + 2); take(v[u].w, i + 3); }
+      }
+    }
+  } else {
+    for (int i = threadIdx.x; i < V; i += blockDim.x) take(row[i], i);
   }
   __shared__ float sb[32];
   __shared__ int si[32];
