@@ -152,6 +152,12 @@ struct ChainPhase {
   int lora_proj[3];               // index into the adapter pointer tables per segment
   int lora_n[3];                  // logical output width per segment
 };
+// a strided region of global memory that the kernel launched next will read (the next attention's K/V): the chain
+// kernel asks for it in L2 while its last phase runs
+struct ChainPrefetch {
+  const unsigned char* base;      // nullptr: nothing
+  unsigned n_outer, outer_stride, inner;   // n_outer runs of `inner` bytes, `outer_stride` bytes apart (multiples of 16)
+};
 struct ChainArgs {
   const ChainPhase* phases;       // dev
   int p0, p1;                     // phase range [p0, p1)
@@ -172,6 +178,7 @@ struct ChainArgs {
   int inject_stall;               // test hook: the launch's first grid barrier waits for an arrival nobody makes
   int nstages;                    // ring stages
   int kmax;                       // largest K of the phases in range (sizes the activation buffer)
+  ChainPrefetch pf[4];
 };
 constexpr int CHAIN_MAX_ROWS = 8;
 constexpr int CHAIN_MAX_RANK = 64;

@@ -454,6 +454,21 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     };
     for (int p = a.p0; p < a.p1 && alive; ++p) {
       cur_phase = p;
+      if (p == a.p1 - 1) {
+        // last phase of the launch: what the next kernel reads first (its K/V) is asked for in L2 now, in 4 KB
+        // pieces dealt over the CTAs and lanes
+#pragma unroll 1
+        for (int d = 0; d < 4; ++d) {
+          const ChainPrefetch f = a.pf[d];
+          if (f.base == nullptr || f.inner == 0u) continue;
+          const unsigned ppo = (f.inner + 4095u) / 4096u, total = f.n_outer * ppo;
+          for (unsigned i = blockIdx.x * 32u + lane; i < total; i += G * 32u) {
+            const unsigned o = i / ppo, off = (i - o * ppo) * 4096u;
+            const unsigned bytes = min(4096u, f.inner - off);
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(f.base + (size_t)o * f.outer_stride + off), "r"(bytes) : "memory");
+          }
+        }
+      }
       const ChainPhase* ph = a.phases + p;           // immutable: read the descriptor from global
       const unsigned char* wbase = ph->w;
       const int mode = ph->mode, K = ph->K;

@@ -252,13 +252,35 @@ int forward_chain(mlora_ctx* c, const PassIO& io) {
     c->dbg_inject_stall = 0;
   }
   const int last = 4 * c->L + ((d.vocab > 0 && io.logits != nullptr) ? 1 : 0);
+  // the K/V that the attention of layer l reads: prefetched into L2 by the chain launch before it
+  auto kv_prefetch = [&](int l) {
+    for (int i = 0; i < 4; ++i) a.pf[i] = ChainPrefetch{};
+    if (l >= c->L) return;
+    const unsigned hd2 = (unsigned)d.head_dim * 2u;
+    if (io.pos_base > 0) {
+      a.pf[0] = ChainPrefetch{(const unsigned char*)(c->prefix_k + (size_t)l * c->prefix_layer_stride), (unsigned)d.n_kv_heads,
+                              (unsigned)(c->prefix_head_stride * 2), (unsigned)io.pos_base * hd2};
+      a.pf[1] = a.pf[0];
+      a.pf[1].base = (const unsigned char*)(c->prefix_v + (size_t)l * c->prefix_layer_stride);
+    }
+    // (the same coarse bound on the suffix lengths as the attention's launch shape, so frozen graphs stay valid)
+    const size_t own_rows = std::min<size_t>((size_t)(io.suffix_bound + 63) / 64 * 64, c->own_head_stride / (size_t)d.head_dim);
+    if (own_rows > 0 && c->own_stream_stride == c->own_head_stride * (size_t)d.n_kv_heads) {
+      a.pf[2] = ChainPrefetch{(const unsigned char*)(c->own_k + (size_t)l * c->own_layer_stride), (unsigned)(io.n * d.n_kv_heads),
+                              (unsigned)(c->own_head_stride * 2), (unsigned)own_rows * hd2};
+      a.pf[3] = a.pf[2];
+      a.pf[3].base = (const unsigned char*)(c->own_v + (size_t)l * c->own_layer_stride);
+    }
+  };
   a.p0 = 0; a.p1 = 1;
+  kv_prefetch(0);
   CK(run(c, MLORA_PROF_GEMM, [&] { return launch_chain(a, c->sm_count, st); }));
   for (int l = 0; l < c->L; ++l) {
     int rc = launch_attention_block(c, io, l);
     if (rc != MLORA_OK) return rc;
     a.p0 = 4 * l + 1;
     a.p1 = (l + 1 < c->L) ? 4 * l + 5 : last;
+    kv_prefetch(l + 1);
     CK(run(c, MLORA_PROF_GEMM, [&] { return launch_chain(a, c->sm_count, st); }));
   }
   return MLORA_OK;
