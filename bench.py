@@ -28,7 +28,9 @@ GEN_STEPS = 128          # decode steps per generation (per stream) before the s
 ORACLE_PREFIX = 64       # prompt length used for the CPU-baseline sample (the 512-token prefill is not timed work)
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of decode_chain_kernel, averaged over the 17 launches of
 # a full-model step, from the ncu capture summarised in profiles/decode_chain_kernel_llama1b_cut4L_8streams.md
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = 32.8e6
+# (32.8 MB of weights, adapters and activations plus 2.1 MB of K/V that the kernel prefetches into L2 for the
+# attention kernel that follows it)
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = 34.8e6
 
 
 def parse_args():

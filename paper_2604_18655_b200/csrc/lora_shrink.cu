@@ -83,13 +83,13 @@ __global__ void __launch_bounds__(SHRINK_THREADS) norm_shrink_kernel(const Shrin
 }
 
 // LoRA shrink on mma.sync for passes whose rows come in runs of 16 that share an adapter (rows_per_stream a multiple
-// of 16: DS2D trees of 16 or 32 nodes).  One CTA per (16 rows, segment, 8 rank indices); its eight warps split K in
+// of 16: DS2D trees of 16 or 32 nodes).  One CTA per (16 rows, segment, 8 rank indices); its sixteen warps split K in
 // contiguous ranges and the partial fragments are added in warp order.  Per 16 features a thread loads 8 consecutive
 // features of an activation row (rows g and g+8 of the tile) and of an A row (rank index j0 + g): the two k16 steps
 // use features {0,1 | 2,3} and {4,5 | 6,7} of that piece for the fragment's (k 2t.. | k 2t+8..) slots -- any pairing of
 // slots with features is valid as long as both operands use the same one.  The activations are the fp16 rows the
 // GEMM reads (written by the norm pass before), so the A matrix of a stream is fetched once per 16 rows.
-constexpr int SHRINK_MMA_WARPS = 8;
+constexpr int SHRINK_MMA_WARPS = 16;
 __global__ void __launch_bounds__(SHRINK_MMA_WARPS * 32) shrink_mma_kernel(const ShrinkArgs p, const __half* __restrict__ h) {
   __shared__ float red[SHRINK_MMA_WARPS][32][4];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
