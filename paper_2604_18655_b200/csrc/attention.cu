@@ -199,10 +199,16 @@ __device__ __forceinline__ void attn_partial_body(const AttnArgs& p, const int r
 
   // per-row tree masks (own segment only): rows g and g+8 of the warp's tile
   unsigned long long anc0 = ~0ull, anc1 = ~0ull;
+  int tq0 = -1, tq1 = -1;                                              // causal passes: the rows' own indices
   if (it.is_own) {
     const int v0 = row_lo + warp * 16 + g, v1 = v0 + 8;
-    anc0 = (v0 < row_hi) ? p.anc[v0 / g_heads] : 0ull;                 // v / g_heads = global row m = s*T + t
-    anc1 = (v1 < row_hi) ? p.anc[v1 / g_heads] : 0ull;
+    if (p.causal) {
+      tq0 = (v0 < row_hi) ? (v0 / g_heads) % p.T : -1;
+      tq1 = (v1 < row_hi) ? (v1 / g_heads) % p.T : -1;
+    } else {
+      anc0 = (v0 < row_hi) ? p.anc[v0 / g_heads] : 0ull;               // v / g_heads = global row m = s*T + t
+      anc1 = (v1 < row_hi) ? p.anc[v1 / g_heads] : 0ull;
+    }
   }
 
   float o[DT][4];
@@ -246,8 +252,12 @@ __device__ __forceinline__ void attn_partial_body(const AttnArgs& p, const int r
           const int key = k0 + nt * 8 + 2 * t + (e & 1);
           bool ok = key < key_end;
           if (it.is_own && key >= S) {
-            const unsigned long long a = (e & 2) ? anc1 : anc0;
-            ok = ok && ((a >> (key - S)) & 1ull);
+            if (p.causal) {
+              ok = ok && (key - S) <= ((e & 2) ? tq1 : tq0);
+            } else {
+              const unsigned long long a = (e & 2) ? anc1 : anc0;
+              ok = ok && ((a >> (key - S)) & 1ull);
+            }
           }
           const float v = ok ? sacc[nt][e] * scale_log2 : -INFINITY;
           sacc[nt][e] = v;

@@ -120,6 +120,7 @@ struct AttnArgs {
   const int32_t* suffix_len;      // dev [n]
   int suffix_bound;               // host upper bound on suffix_len
   const unsigned long long* anc;  // dev [n][T] ancestor-or-self bit masks
+  int causal;                     // the pass's rows form a chain (prefill): row t sees new rows 0..t, anc is not read
   int n, T, Hq, Hkv, hd;
   __half* out;                    // [rows][Hq][hd]
   float* part_o; float* part_ml;  // scratch

@@ -214,7 +214,7 @@ int launch_attention_block(mlora_ctx* c, const PassIO& io, int l) {
   a.prefix_v = c->prefix_v + (size_t)l * c->prefix_layer_stride;
   a.prefix_head_stride = c->prefix_head_stride;
   a.own_k = kd; a.own_v = vd; a.own_stream_stride = sstride; a.own_head_stride = hstride;
-  a.suffix_len = io.suffix_len; a.anc = c->anc;
+  a.suffix_len = io.suffix_len; a.anc = c->anc; a.causal = io.prefill ? 1 : 0;
   a.out = c->attn16;
   if (attn_workspace_floats(a) > c->att_ws_floats) return fail(MLORA_ERR_CAPACITY, "attention scratch too small");
   a.part_o = c->att_ws;
@@ -457,7 +457,8 @@ int check_ctx(mlora_ctx* c) { return c ? MLORA_OK : fail(MLORA_ERR_ARG, "null co
 int prefill_impl(mlora_ctx* c, const int32_t* ids, const __half* hidden, int n, float* out_last) {
   if (n <= 0) return fail(MLORA_ERR_ARG, "prefill needs at least one position");
   if (n > c->d.max_prefix) return fail(MLORA_ERR_CAPACITY, "prompt longer than max_prefix");
-  const int chunk = 64;
+  // a chunk of the prompt is one causal pass: 256 rows keep the tensor-core GEMMs at their largest row block
+  const int chunk = c->Mmax >= 256 ? 256 : c->Mmax / 64 * 64;
   const int dm = c->d.d_model;
   for (int p0 = 0; p0 < n; p0 += chunk) {
     PassIO io;
@@ -465,7 +466,7 @@ int prefill_impl(mlora_ctx* c, const int32_t* ids, const __half* hidden, int n, 
     io.T = (n - p0 < chunk) ? (n - p0) : chunk;
     io.tokens = ids ? ids + p0 : nullptr;
     io.hidden_in = hidden ? hidden + (size_t)p0 * dm : nullptr;
-    io.parent = c->chain_parent;
+    io.parent = nullptr;                    // causal: the attention kernel compares row indices
     io.prefill = true;
     io.pos_base = p0;
     io.suffix_len = c->zero_len;
@@ -531,7 +532,7 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
   c->L = d.n_layers; c->Nq = Nq; c->Nkv = Nkv; c->Nqkv = Nq + 2 * Nkv;
   c->cap = d.max_suffix + d.max_tree;
   c->Mmax = d.max_streams * d.max_tree;
-  if (c->Mmax < 64) c->Mmax = 64;
+  if (c->Mmax < 256) c->Mmax = 256;        // prefill passes have up to 256 rows
 #define CKC(call)                                                                                  \
   do {                                                                                             \
     cudaError_t e__ = (call);                                                                      \

@@ -42,6 +42,11 @@ __global__ void tree_prep_kernel(const int32_t* __restrict__ parent, int n, int 
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n * T) return;
   const int s = i / T, t = i % T;
+  if (parent == nullptr) {                 // a chain of any length (prefill): no mask word, depth = index
+    anc[i] = ~0ull;
+    depth[i] = t;
+    return;
+  }
   const int32_t* par = parent + (size_t)s * T;
   unsigned long long mask = 0ull;
   int d = 0, c = t;

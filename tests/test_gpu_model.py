@@ -66,6 +66,21 @@ def test_cfg0_hidden_state_decode(GpuModel):
     gm.close()
 
 
+def test_prefill_ragged_causal_chunks(GpuModel):
+    """A prompt of 300 positions runs as one causal pass of 256 rows and one of 44 that also attends to the first:
+    last hidden row and every position's K/V against the oracle."""
+    cfg = gen.ModelCfg("tiny1L300", 1, 512, 8, 8, 64, 1408, 0, 64, 8, 15, 4, 4, 300)
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=8)
+    prompt = gen.make_hidden(cfg, cfg.prompt_len, 0, 0)
+    want_last = orc.prefill_shared(hidden=prompt)
+    got_last = gm.prefill_h(prompt)
+    compare(got_last, want_last, "prefill last hidden, 300 positions")
+    _, pk, pv = gm.export_kv(0, -1, 0, cfg.prompt_len)
+    compare(pk, orc.prefix_k[0], "prefix K")
+    compare(pv, orc.prefix_v[0], "prefix V")
+    gm.close()
+
+
 def test_prefill_logits_and_follow_mode_decode(GpuModel):
     cfg = TINYV
     m, orc, gm = make_pair(GpuModel, cfg, max_suffix=32)
