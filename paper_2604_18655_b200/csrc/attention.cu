@@ -419,18 +419,20 @@ __global__ void attn_merge_kernel(const AttnArgs p) {
 }
 
 // ----------------------------------------------------------------------------- single-pass decode attention
-// One decode row per stream (T = 1) and a short context: one CTA per (kv head, stream) does the whole softmax, so
-// there are no partial results in global memory and no merge kernel.  The shared prefix is re-read by every stream's
+// One decode row per stream (T = 1) and a short context: a cluster of two CTAs per (kv head, stream) does the whole
+// softmax (the CTAs take alternate tiles and the second hands its result to the first through distributed shared
+// memory), so there are no partial results in global memory and no merge kernel.  The shared prefix is re-read by every stream's
 // CTA, but from L2: HBM still sees it once.  The warps take 32-key tiles of (prefix ++ own segment) round-robin, each
 // with its own double-buffered K/V tiles (cp.async) and its own online softmax over the kv head's query heads (one
 // m16 tile, rows past the group zero); the warps' results are combined by log-sum-exp in shared memory.  The new
 // K/V row of the pass is built from the projections (k rotated), used, and appended to the cache by the warp whose
 // tile holds it.
 constexpr int DEC_KEYS = 32;
+constexpr int DEC_SPLIT = 2;                 // CTAs (one cluster) that share the tiles of a (kv head, stream)
 __host__ __device__ constexpr int dec_warps(int hd) { return hd == 64 ? 8 : 4; }
 __host__ __device__ constexpr size_t dec_smem_bytes(int hd) {
   return (size_t)16 * (hd + 8) * 2 + (size_t)dec_warps(hd) * 4 * DEC_KEYS * (hd + 8) * 2 +
-         (size_t)dec_warps(hd) * 16 * (hd + 2) * 4;
+         (size_t)dec_warps(hd) * 16 * (hd + 2) * 4 + (size_t)16 * (hd + 2) * 4;
 }
 
 template <int HD>
@@ -441,6 +443,9 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   __half* tiles = Qs + 16 * STRIDE;                                       // [W][2 buffers][K, V][DEC_KEYS][STRIDE]
   float* part_o = reinterpret_cast<float*>(tiles + (size_t)W * 4 * DEC_KEYS * STRIDE);   // [W][16][HD]
   float* part_ml = part_o + (size_t)W * 16 * HD;                          // [W][16][2]
+  float* xch = part_ml + (size_t)W * 16 * 2;                              // [16][HD + 2]: this CTA's result for its peer
+  const int rank = blockIdx.z;                                            // position in the cluster (1, 1, DEC_SPLIT)
+  auto tile_of = [&](int li) { return li * DEC_SPLIT + rank; };          // the CTA's li-th tile
 
   const int kh = blockIdx.x, s = blockIdx.y;
   const int g_heads = p.Hq / p.Hkv;
@@ -501,16 +506,17 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
     cp_async_commit();
   };
   // a warp whose first tile lies in the shared prefix starts it before anything that depends on the stream
-  if (warp < n_ptiles) load_tile(warp, 0);
+  if (tile_of(warp) < n_ptiles) load_tile(tile_of(warp), 0);
   S = p.suffix_len[s];
   own_keys = S + 1;                                                       // cached rows + this pass's row
   n_tiles = n_ptiles + (own_keys + DEC_KEYS - 1) / DEC_KEYS;
   if (fused) cs = p.cs_table + (size_t)(p.pos_base + S + p.depth[m]) * (HD / 2);
-  if (warp >= n_ptiles && warp < n_tiles) load_tile(warp, 0);
-  if (warp + W < n_tiles) load_tile(warp + W, 1);
+  if (tile_of(warp) >= n_ptiles && tile_of(warp) < n_tiles) load_tile(tile_of(warp), 0);
+  if (tile_of(warp + W) < n_tiles) load_tile(tile_of(warp + W), 1);
   // the warp's later tiles: ask for them in L2 now, so that their copies two iterations on do not wait for HBM
   if (lane == 0) {
-    for (int ti = warp + 2 * W; ti < n_tiles; ti += W) {
+    for (int li = warp + 2 * W; tile_of(li) < n_tiles; li += W) {
+      const int ti = tile_of(li);
       const bool own = ti >= n_ptiles;
       const int k0 = (own ? ti - n_ptiles : ti) * DEC_KEYS;
       const int rows = min(DEC_KEYS, (own ? S : p.P) - k0);               // cached rows only
@@ -545,8 +551,9 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
 
   int buf = 0;
-  for (int ti = warp; ti < n_tiles; ti += W, buf ^= 1) {
-    if (ti + W < n_tiles) cp_async_wait<1>();              // the next tile may still be in flight
+  for (int li = warp; tile_of(li) < n_tiles; li += W, buf ^= 1) {
+    const int ti = tile_of(li);
+    if (tile_of(li + W) < n_tiles) cp_async_wait<1>();     // the next tile may still be in flight
     else cp_async_wait<0>();
     __syncwarp();
     const __half* kt = my_tiles + (size_t)buf * 2 * DEC_KEYS * STRIDE;
@@ -617,7 +624,7 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
       }
     }
     __syncwarp();                                        // every lane is done with the buffer: refill it
-    if (ti + 2 * W < n_tiles) load_tile(ti + 2 * W, buf);
+    if (tile_of(li + 2 * W) < n_tiles) load_tile(tile_of(li + 2 * W), buf);
   }
 
   // this warp's un-normalised output, running max (log2 domain) and sum for the group's rows
@@ -633,22 +640,49 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
     if (t == 0) *reinterpret_cast<float2*>(part_ml + ((size_t)warp * 16 + r) * 2) = make_float2(mrow[h], lrow[h]);
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < g_heads * HD; i += W * 32) {
-    const int r = i / HD, d = i % HD;
-    float M = -INFINITY;
+  // the CTA's result per (row, feature): running max, numerator, denominator over its warps (warp order: fixed)
+  auto cta_result = [&](int r, int d, float& M, float& num, float& den) {
+    M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < W; ++w) M = fmaxf(M, part_ml[((size_t)w * 16 + r) * 2]);
-    float num = 0.f, den = 0.f;
+    num = 0.f; den = 0.f;
 #pragma unroll
-    for (int w = 0; w < W; ++w) {                          // warp order: fixed
+    for (int w = 0; w < W; ++w) {
       const float mw = part_ml[((size_t)w * 16 + r) * 2];
       if (mw == -INFINITY) continue;                       // a warp without tiles
       const float f = exp2f(mw - M);
       num += f * part_o[((size_t)w * 16 + r) * HD + d];
       den += f * part_ml[((size_t)w * 16 + r) * 2 + 1];
     }
-    p.out[((size_t)m * p.Hq + kh * g_heads + r) * HD + d] = __float2half_rn(den > 0.f ? num / den : 0.f);
+  };
+  if (rank != 0) {
+    for (int i = threadIdx.x; i < g_heads * HD; i += W * 32) {
+      const int r = i / HD, d = i % HD;
+      float M, num, den;
+      cta_result(r, d, M, num, den);
+      xch[r * (HD + 2) + d] = num;
+      if (d == 0) { xch[r * (HD + 2) + HD] = M; xch[r * (HD + 2) + HD + 1] = den; }
+    }
   }
+  // every thread of both CTAs gets here (no early exit above): the peer's result is complete and visible
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+  if (rank == 0) {
+    uint32_t peer;                                         // the peer's xch in the cluster's shared window
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(peer) : "r"((uint32_t)__cvta_generic_to_shared(xch)), "r"(1));
+    auto peer_f32 = [&](int idx) { float v; asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(peer + 4u * (uint32_t)idx) : "memory"); return v; };
+    for (int i = threadIdx.x; i < g_heads * HD; i += W * 32) {
+      const int r = i / HD, d = i % HD;
+      float M0, num0, den0;
+      cta_result(r, d, M0, num0, den0);
+      const float num1 = peer_f32(r * (HD + 2) + d), M1 = peer_f32(r * (HD + 2) + HD), den1 = peer_f32(r * (HD + 2) + HD + 1);
+      const float M = fmaxf(M0, M1);
+      const float f0 = (M0 == -INFINITY) ? 0.f : exp2f(M0 - M), f1 = (M1 == -INFINITY) ? 0.f : exp2f(M1 - M);
+      const float num = f0 * num0 + f1 * num1, den = f0 * den0 + f1 * den1;
+      p.out[((size_t)m * p.Hq + kh * g_heads + r) * HD + d] = __float2half_rn(den > 0.f ? num / den : 0.f);
+    }
+  }
+  // the peer's shared memory must outlive the reads above
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 // one decode row per stream, a context short enough for one CTA per (kv head, stream), at most 16 query heads per
@@ -717,11 +751,19 @@ cudaError_t init_attention() {
 
 cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st) {
   if (attn_single_pass(a)) {
-    dim3 grid(a.Hkv, a.n);
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)a.hd);
-    if (a.hd == 64) attn_decode_kernel<64><<<grid, dec_warps(64) * 32, dec_smem_bytes(64), st>>>(a, scale_log2);
-    else attn_decode_kernel<128><<<grid, dec_warps(128) * 32, dec_smem_bytes(128), st>>>(a, scale_log2);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)a.Hkv, (unsigned)a.n, DEC_SPLIT);
+    cfg.blockDim = dim3((unsigned)dec_warps(a.hd) * 32);
+    cfg.dynamicSmemBytes = dec_smem_bytes(a.hd);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;      // the DEC_SPLIT CTAs of a (kv head, stream) form a cluster
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = DEC_SPLIT;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (a.hd == 64) return cudaLaunchKernelEx(&cfg, attn_decode_kernel<64>, a, scale_log2);
+    return cudaLaunchKernelEx(&cfg, attn_decode_kernel<128>, a, scale_log2);
   }
   if (a.hd == 64) return launch_attn_hd<64>(a, st);
   if (a.hd == 128) return launch_attn_hd<128>(a, st);
