@@ -667,17 +667,25 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   // every thread of both CTAs gets here (no early exit above): the peer's result is complete and visible
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
   if (rank == 0) {
-    uint32_t peer;                                         // the peer's xch in the cluster's shared window
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(peer) : "r"((uint32_t)__cvta_generic_to_shared(xch)), "r"(1));
-    auto peer_f32 = [&](int idx) { float v; asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(peer + 4u * (uint32_t)idx) : "memory"); return v; };
+    const uint32_t mine = (uint32_t)__cvta_generic_to_shared(xch);
     for (int i = threadIdx.x; i < g_heads * HD; i += W * 32) {
       const int r = i / HD, d = i % HD;
-      float M0, num0, den0;
-      cta_result(r, d, M0, num0, den0);
-      const float num1 = peer_f32(r * (HD + 2) + d), M1 = peer_f32(r * (HD + 2) + HD), den1 = peer_f32(r * (HD + 2) + HD + 1);
-      const float M = fmaxf(M0, M1);
-      const float f0 = (M0 == -INFINITY) ? 0.f : exp2f(M0 - M), f1 = (M1 == -INFINITY) ? 0.f : exp2f(M1 - M);
-      const float num = f0 * num0 + f1 * num1, den = f0 * den0 + f1 * den1;
+      float M, num, den;
+      cta_result(r, d, M, num, den);
+      if (M == -INFINITY) { num = 0.f; den = 0.f; }
+#pragma unroll
+      for (int pr = 1; pr < DEC_SPLIT; ++pr) {             // peer order: fixed
+        uint32_t peer;                                     // the peer's xch in the cluster's shared window
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(peer) : "r"(mine), "r"(pr));
+        auto peer_f32 = [&](int idx) { float v; asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(peer + 4u * (uint32_t)idx) : "memory"); return v; };
+        const float num1 = peer_f32(r * (HD + 2) + d), M1 = peer_f32(r * (HD + 2) + HD), den1 = peer_f32(r * (HD + 2) + HD + 1);
+        if (M1 == -INFINITY) continue;                     // a peer without tiles
+        const float Mn = fmaxf(M, M1);
+        const float f0 = (M == -INFINITY) ? 0.f : exp2f(M - Mn), f1 = exp2f(M1 - Mn);
+        num = f0 * num + f1 * num1;
+        den = f0 * den + f1 * den1;
+        M = Mn;
+      }
       p.out[((size_t)m * p.Hq + kh * g_heads + r) * HD + d] = __float2half_rn(den > 0.f ? num / den : 0.f);
     }
   }
