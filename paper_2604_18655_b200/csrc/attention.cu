@@ -16,7 +16,7 @@ namespace mlora {
 constexpr int ATT_WARPS = 4;
 constexpr int ATT_THREADS = ATT_WARPS * 32;
 constexpr int ATT_ROWS = ATT_WARPS * 16;   // query rows per CTA
-constexpr int ATT_KEYS = 64;               // keys per pipeline tile
+constexpr int ATT_KEYS = 32;               // keys per pipeline tile
 
 __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
   const uint32_t sa = (uint32_t)__cvta_generic_to_shared(smem);
@@ -402,7 +402,7 @@ __device__ __forceinline__ void merge_row(const AttnArgs& p, int kh, int v, int 
 }
 
 template <int HD>
-__global__ void __launch_bounds__(ATT_THREADS) attn_partial_kernel(const AttnArgs p, const int rb_all, const int rb_own,
+__global__ void __launch_bounds__(ATT_THREADS, 3) attn_partial_kernel(const AttnArgs p, const int rb_all, const int rb_own,
                                                                   const float scale_log2) {
   attn_partial_body<HD>(p, rb_all, rb_own, scale_log2);
 }
