@@ -20,7 +20,7 @@ def declared_functions():
     return sorted(set(re.findall(r"\b(mlora_[a-z_0-9]+)\s*\(", text)))
 
 
-def test_header_declares_the_north_star_calls():
+def test_header_declares_the_main_calls():
     names = declared_functions()
     for f in ("mlora_create", "mlora_set_adapter", "mlora_prefill_shared", "mlora_decode_step", "mlora_verify_tree"):
         assert f in names
