@@ -103,6 +103,13 @@ def test_linear_lora_matches_oracle(mb, K, N, G, M, n_ad, rank):
     compare(got, want, f"linear lora K{K} N{N} M{M} ad{n_ad} r{rank}")
 
 
+def test_linear_base_wide_ragged_output(mb):
+    """Enough 16 x 32 output tiles for the warp-per-tile epilogue, with a width that is not a multiple of 32 and a row
+    count that is not a multiple of 16: the ragged last tiles of both directions."""
+    got, want = run_linear(mb, 256, 4112, 64, 168, 0, 0, seed=11)
+    compare(got, want, "linear base K256 N4112 M168")
+
+
 def test_linear_lora_visible_and_b_zero_is_base(mb):
     """The low-rank term changes the result, and adapter index -1 gives the base projection exactly."""
     got_l, _ = run_linear(mb, 512, 256, 128, 8, 4, 16, seed=5, with_base_rows=False)
