@@ -312,6 +312,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
   __shared__ float s_scale[CHAIN_MAX_ROWS];
   __shared__ int s_adapter[CHAIN_MAX_ROWS];
   __shared__ int s_abort_word;
+  __shared__ volatile unsigned s_t_ready;             // LoRA phases of this launch whose T is in shared memory
   __shared__ unsigned long long s_base[2];
   __shared__ float s_shr_part[CH_MAX_ITEMS][16];      // shrink: partial sums of an item's half pieces
   __shared__ float s_ssw[CH_CWARPS * CHAIN_MAX_ROWS];  // RMSNorm: per-warp sums of squares of every row
@@ -344,6 +345,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     s_abort_word = (ld_acquire_u64(a.sync + 2) != 0ull) ? 1 : 0;
+    s_t_ready = 0u;
     // arrivals of earlier launches are whole multiples of the grid size; arrivals of this launch that are
     // already counted are fewer than one grid
     s_base[0] = ld_acquire_u64(a.sync + 0) / G * G;
@@ -733,6 +735,15 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
           __syncwarp();
           if (lane == 0) red_release_add_u64(a.sync + 1, 1ull);
           STAMPS(13);
+          // This warp has nothing else to do in the phase: it watches for the other CTAs' shares and brings all of
+          // T into shared memory as soon as it is complete, so that the GEMM teams, when their main loop ends, find
+          // it there instead of paying a counter poll and a load round trip each.
+          if (lane == 0) wait_counter(a.sync + 1, s_base[1] + (unsigned long long)(n_shr + 1u) * G, wc, 4, p);
+          __syncwarp();
+          for (int i = lane; i < M * nseg * r; i += 32) Ts[i] = __ldcg(a.T + i);
+          __threadfence_block();
+          __syncwarp();
+          if (lane == 0) s_t_ready = n_shr + 1u;
         }
       }
       pos += np * pd.n_valid;
@@ -829,10 +840,16 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         team_sync();
         if (nseg > 0 && !t_loaded) {
-          // all of T must be in global memory before the first expand; every team fetches the same values
-          if (tt == 0) wait_counter(a.sync + 1, s_base[1] + (unsigned long long)n_shr * G, wc, 4, p);
-          team_sync();
-          for (int i = tt; i < M * nseg * r; i += team_threads) Ts[i] = __ldcg(a.T + i);
+          // all of T must be in shared memory before the first expand: the first shrink warp puts it there
+          if (tt == 0) {
+            const long long t0 = clock64();
+            for (int it = 0; s_t_ready < n_shr; ++it) {
+              if ((it & 255) == 255) {
+                if (*wc.s_abort) break;
+                if (clock64() - t0 > wc.limit) { raise_abort(wc, 4, p); break; }
+              }
+            }
+          }
           team_sync();
           t_loaded = true;
           STAMP(4);
