@@ -169,6 +169,9 @@ def run_attention(mb, n, T, Hq, Hkv, hd, P, suf, branch, seed, cap=None):
     (3, 16, (4, 2, 2), 300, [0, 63, 130]),
     (2, 64, (4, 4, 4), 65, [1, 40]),
     (2, 10, (3, 2), 0, [4, 0]),
+    (3, 1, (), 0, [0, 33, 64]),          # no shared prefix: one CTA of a decode cluster may have no tile at all
+    (2, 1, (), 31, [0, 1]),              # a prefix shorter than one tile
+    (2, 1, (), 1500, [100, 7]),          # the longest context the single-pass kernel takes
 ])
 def test_attention_matches_oracle(mb, hd, n, T, branch, P, suf):
     got, want = run_attention(mb, n, T, 8, 2, hd, P, suf, branch, seed=hd + n + T + P)
