@@ -143,7 +143,9 @@ int mlora_debug_dequant(mlora_ctx* ctx, int32_t layer, int32_t proj, void* out_f
 /* Debug switches: key 1 = skip KV compaction and suffix growth in mlora_verify_tree (tree rows stay where
  * the pass wrote them: rows suffix_len .. suffix_len + n_nodes - 1 of the own segment).
  * key 2 = 1 disables CUDA-graph replay of steps (every kernel launched directly).
- * key 3 = 1 runs decode-sized passes through the one-kernel-per-projection path instead of the persistent kernel.
+ * key 3 = 1 runs decode-sized passes through the one-kernel-per-projection path instead of the persistent kernels.
+ * key 6 = 1 runs decode steps through the per-layer persistent projection kernel plus attention kernels (replayed
+ *         from a CUDA graph) instead of the single kernel that does the whole step.
  * key 4 = 1 runs passes of 32 rows or more on the split-K mma.sync GEMM instead of the tcgen05 one.
  * key 5 = 1 (test hook for the bounded waits) makes the NEXT decode-sized pass wait, with a limit of about 0.1 s,
  *         at a grid barrier for an arrival nobody makes: the pass ends with garbage outputs and the device status

@@ -5,7 +5,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-SOURCES = ["w4_gemm.cu", "lora_shrink.cu", "step_misc.cu", "attention.cu", "decode_chain.cu", "w4_gemm_tc.cu", "mlora.cu"]
+SOURCES = ["w4_gemm.cu", "lora_shrink.cu", "step_misc.cu", "attention.cu", "decode_chain.cu", "decode_step.cu", "w4_gemm_tc.cu", "mlora.cu"]
 LIB = os.path.join(HERE, "libmlora.so")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]
@@ -20,7 +20,7 @@ def _newer(target, deps):
 
 def build(force=False, verbose=False):
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    headers = [os.path.join(CSRC, "common.cuh"), os.path.join(HERE, "..", "include", "mlora.h")]
+    headers = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "pipe.cuh"), os.path.join(HERE, "..", "include", "mlora.h")]
     objdir = os.path.join(HERE, "_build")
     os.makedirs(objdir, exist_ok=True)
     objs = []

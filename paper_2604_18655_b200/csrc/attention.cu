@@ -36,32 +36,6 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(sa));
 }
 
-// eight consecutive elements c..c+7 of one head of a projection row, rotated (pairs (i, i + hd/2), Sec. 3.1) or not.
-// All loads are issued before the first use; the row was written by another kernel or CTA: read through L2.
-__device__ __forceinline__ uint4 head_piece_f16(const float* __restrict__ head, int c, int hd, const float2* __restrict__ cs) {
-  const float4 x0 = __ldcg(reinterpret_cast<const float4*>(head + c));
-  const float4 x1 = __ldcg(reinterpret_cast<const float4*>(head + c + 4));
-  float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-  if (cs != nullptr) {
-    const int half = hd >> 1;
-    const bool lo = c < half;                          // a piece never straddles the middle: c and hd/2 are multiples of 8
-    const int pc = lo ? c + half : c - half;           // the partner piece
-    const float4 y0 = __ldcg(reinterpret_cast<const float4*>(head + pc));
-    const float4 y1 = __ldcg(reinterpret_cast<const float4*>(head + pc + 4));
-    const float4* t4 = reinterpret_cast<const float4*>(cs + (lo ? c : pc));
-    const float4 t0 = __ldg(t4), t1 = __ldg(t4 + 1), t2 = __ldg(t4 + 2), t3 = __ldg(t4 + 3);
-    const float y[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
-    const float co[8] = {t0.x, t0.z, t1.x, t1.z, t2.x, t2.z, t3.x, t3.z};
-    const float si[8] = {t0.y, t0.w, t1.y, t1.w, t2.y, t2.w, t3.y, t3.w};
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = lo ? v[i] * co[i] - y[i] * si[i] : v[i] * co[i] + y[i] * si[i];
-  }
-  __half2 o[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) o[i] = __halves2half2(__float2half_rn(v[2 * i]), __float2half_rn(v[2 * i + 1]));
-  return make_uint4(h2_as_u32(o[0]), h2_as_u32(o[1]), h2_as_u32(o[2]), h2_as_u32(o[3]));
-}
-
 struct AttnItem {
   int is_own, s, chunk, row_block;
 };

@@ -191,6 +191,75 @@ int chain_pick_stages(int kmax, int rank);      // most stages that fit (0: not 
 bool chain_phase_fits(int K, int mode, int nseg, int rank, int nstages, int sm_count);
 cudaError_t launch_chain(const ChainArgs& a, int sm_count, cudaStream_t st);
 
+// ----------------------------------------------------------------------------- whole decode step in one kernel
+// One decode step (one row per stream, at most 8 rows) as ONE persistent cooperative kernel: embedding, every
+// projection group, the attention of every layer, lm_head, row argmax and the suffix-length update are phases
+// separated by grid barriers.
+enum StepKind { SK_EMBED = 0, SK_GEMM = 1, SK_ATTN = 2, SK_FIN = 3 };
+struct StepPhase {
+  int kind, layer;
+  const unsigned char* w;         // SK_GEMM: packed weights
+  int K, N, G;                    // N = physical (fused) width; SK_EMBED: N = d_model
+  int mode, epi;
+  int seg_n0, seg_n1;             // MODE_QKV: widths of the first two segments
+  const __half* in16;             // SK_GEMM: input rows fp16 [8][K]
+  int norm_in;                    // index of the sums of squares that normalise the input rows (-1: used as they are)
+  int ldo;
+  float* out_f32;                 // EPI_F32 (nullptr: the call's logits destination)
+  __half* out16;                  // EPI_SWIGLU: [8][N/2]; EPI_RESID / SK_EMBED: x * gain_next [8][N]; SK_ATTN: [8][Hq*hd]
+  const __half* gain_next;        // EPI_RESID / SK_EMBED: gain of the RMSNorm that follows (nullptr: none)
+  int ssq_out;                    // where the sums of squares of the new residual rows are accumulated (-1: nowhere)
+  int lora_nseg;                  // 0: no LoRA on this group
+  int lora_proj[3];               // index into the adapter pointer tables per segment
+  int lora_n[3];                  // logical output width per segment
+  int t_in;                       // index of this group's accumulated shrink sums
+  int next_nseg;                  // LoRA segments of the group that consumes this phase's outputs (0: none)
+  int next_proj[3];
+  int next_ld;                    // row length of their A matrices (= that group's K)
+  int t_out;                      // where the partial shrink sums over this phase's outputs are accumulated
+  int last;                       // the residual rows this phase writes are the call's hidden-state output
+  int pad_;
+};
+struct StepArgs {
+  const StepPhase* phases;        // dev
+  int n_phases;
+  int M;                          // rows = streams
+  float eps;
+  const int32_t* tokens;          // dev [M] (nullptr: hidden-state input)
+  const __half* embed; int vocab;
+  const __half* hidden_in;        // dev fp16 [M][d_model]
+  const int32_t* adapter_idx;     // dev [M]; nullptr: base weights only
+  const __half* const* tabA;
+  const __half* const* tabB;
+  const float* scale;
+  int tab_stride, n_slots, rank;
+  // attention
+  int Hq, Hkv, hd, P;
+  const float* qkv;               // fp32 [8][(Hq + 2 Hkv) hd]: q,k,v projections of the layer
+  const __half* prefix_k; const __half* prefix_v; size_t prefix_layer_stride, prefix_head_stride;
+  __half* own_k; __half* own_v; size_t own_layer_stride, own_stream_stride, own_head_stride;
+  int32_t* suffix_len;            // dev [M]: read at the start, advanced by one at the end
+  const float2* cs_table;
+  // outputs
+  float* logits;                  // dev fp32 [M][vocab] or nullptr
+  int32_t* out_next;              // dev [M] greedy tokens (vocab > 0)
+  float* hidden_out;              // dev fp32 [M][d_model] (vocab == 0)
+  unsigned long long* amax;       // dev [grid][8]: per-CTA row maxima of the logits
+  // accumulators (64-bit fixed point, zero at launch; the kernel leaves them zero)
+  unsigned long long* tacc;       // [n_tacc][8][3][rank]
+  unsigned long long* ssq;        // [n_ssq][8]
+  int n_tacc, n_ssq;
+  unsigned long long* sync;       // dev [4]: grid-barrier arrivals, spare, abort flag, where the first wait gave up
+  int* status;
+  long long wait_cycles;
+  int inject_stall;
+  int nstages, own_tiles, as_bytes;
+};
+cudaError_t init_step();
+// ring stages the step kernel gets for this model on this device (0: the kernel cannot run it)
+int step_plan(int d_model, int d_ffn, int Nq, int Nkv, int hd, int rank, int lora_targets, int sm_count, int* own_tiles, int* as_bytes);
+cudaError_t launch_step(const StepArgs& a, int sm_count, cudaStream_t st);
+
 // ----------------------------------------------------------------------------- launchers
 cudaError_t init_gemm();        // opt-in shared-memory sizes; call once per process before the first launch
 cudaError_t init_shrink();
@@ -270,6 +339,45 @@ __device__ __forceinline__ void split_scales(uint32_t sw, __half2& s_lo, __half2
   s_lo = u32_as_h2(__byte_perm(sw, sw, 0x1010));
   s_hi = u32_as_h2(__byte_perm(sw, sw, 0x3232));
 }
+// physical column of a fused projection -> (segment, logical column)
+__device__ __forceinline__ void map_col(int mode, int c, int n0, int n1, int& seg, int& col) {
+  if (mode == MODE_PLAIN) { seg = 0; col = c; }
+  else if (mode == MODE_QKV) {
+    if (c < n0) { seg = 0; col = c; }
+    else if (c < n0 + n1) { seg = 1; col = c - n0; }
+    else { seg = 2; col = c - n0 - n1; }
+  } else {                         // gate/up interleaved by 16-column tiles
+    const int tile = c >> 4;
+    seg = tile & 1;
+    col = ((tile >> 1) << 4) | (c & 15);
+  }
+}
+// eight consecutive elements c..c+7 of one head of a projection row, rotated (pairs (i, i + hd/2), Sec. 3.1) or not.
+// All loads are issued before the first use; the row was written by another kernel or CTA: read through L2.
+__device__ __forceinline__ uint4 head_piece_f16(const float* __restrict__ head, int c, int hd, const float2* __restrict__ cs) {
+  const float4 x0 = __ldcg(reinterpret_cast<const float4*>(head + c));
+  const float4 x1 = __ldcg(reinterpret_cast<const float4*>(head + c + 4));
+  float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+  if (cs != nullptr) {
+    const int half = hd >> 1;
+    const bool lo = c < half;                          // a piece never straddles the middle: c and hd/2 are multiples of 8
+    const int pc = lo ? c + half : c - half;           // the partner piece
+    const float4 y0 = __ldcg(reinterpret_cast<const float4*>(head + pc));
+    const float4 y1 = __ldcg(reinterpret_cast<const float4*>(head + pc + 4));
+    const float4* t4 = reinterpret_cast<const float4*>(cs + (lo ? c : pc));
+    const float4 t0 = __ldg(t4), t1 = __ldg(t4 + 1), t2 = __ldg(t4 + 2), t3 = __ldg(t4 + 3);
+    const float y[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
+    const float co[8] = {t0.x, t0.z, t1.x, t1.z, t2.x, t2.z, t3.x, t3.z};
+    const float si[8] = {t0.y, t0.w, t1.y, t1.w, t2.y, t2.w, t3.y, t3.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = lo ? v[i] * co[i] - y[i] * si[i] : v[i] * co[i] + y[i] * si[i];
+  }
+  __half2 o[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) o[i] = __halves2half2(__float2half_rn(v[2 * i]), __float2half_rn(v[2 * i + 1]));
+  return make_uint4(h2_as_u32(o[0]), h2_as_u32(o[1]), h2_as_u32(o[2]), h2_as_u32(o[3]));
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

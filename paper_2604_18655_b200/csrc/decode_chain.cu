@@ -21,8 +21,7 @@
 // raises a global abort flag and the status word MLORA_ERR_TIMEOUT and records which wait it was; from then on
 // every wait returns at once and the kernel runs its (data-independent) control flow to the end, so no CTA is
 // left in a barrier.
-#include "../../include/mlora.h"
-#include "common.cuh"
+#include "pipe.cuh"
 
 namespace mlora {
 
@@ -38,10 +37,11 @@ constexpr int CH_A_PIECE = 2048;                   // halves of a LoRA-A row per
 constexpr int CH_RED_BYTES = 2 * CH_CWARPS * 512;  // partial sums: one slot per consumer warp and tile of a pair
 constexpr int CH_BS_BYTES = 24 * 1024;             // LoRA-B slices of the teams' units: [team][tile][row][j][16] fp16
 constexpr int CH_MAX_TEAMS = 8;
-constexpr long long CH_WAIT_CYCLES = 4000000000ll; // ~2 s at 2 GHz
 
 static_assert(CH_STAGE_BYTES >= CHUNK_KT * 512 + 8 * 32, "stage too small for a chunk");
 static_assert(CH_STAGE_BYTES >= CH_A_PIECE * 2, "stage too small for an A piece");
+
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(CH_CTHREADS) : "memory"); }
 
 // ----------------------------------------------------------------------------- shared-memory carve-up
 struct ChainSmem {
@@ -89,50 +89,6 @@ int chain_pick_stages(int kmax, int rank) {
   return n >= 8 ? n : 0;
 }
 
-// ----------------------------------------------------------------------------- PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok;
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
-}
-__device__ __forceinline__ uint64_t policy_evict_first() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ __forceinline__ void cp_async16_ca(void* smem, const void* gmem) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem)), "l"(gmem) : "memory");
-}
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(CH_CTHREADS) : "memory"); }
-__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
-  unsigned long long v;
-  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void red_release_add_u64(unsigned long long* p, unsigned long long v) {
-  asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-// the ring is addressed by the running stage count since the start of the launch
-__device__ __forceinline__ int pos_stage(int pos, int nstages) { return pos % nstages; }
-__device__ __forceinline__ uint32_t pos_parity(int pos, int nstages) { return (uint32_t)((pos / nstages) & 1); }
-
 // what every consumer thread needs of a phase beyond its descriptor; worked out once per phase by one thread (the
 // divisions in it would otherwise sit at the head of every thread's phase, ahead of its first loads)
 static_assert(sizeof(ChainPhase) == 128, "a phase descriptor is loaded as one word per lane");
@@ -143,63 +99,6 @@ struct PhaseDerived {
   int item_i[CH_MAX_ITEMS];          // their index (row, segment, rank index) = position in T
   int item_sm[CH_MAX_ITEMS];         // their segment | row << 8
 };
-
-// ----------------------------------------------------------------------------- bounded waits
-struct WaitCtx {
-  long long limit;                  // clock cycles a wait may take
-  volatile int* s_abort;            // shared: this CTA has given up waiting
-  unsigned long long* sync;         // global: [0] barrier, [1] shrink, [2] abort, [3] where the first wait gave up
-  int* status;
-};
-// where codes: 1 producer/free stage, 2 shrink/A piece, 3 GEMM/weight chunk, 4 T counter, 5 grid barrier
-__device__ __noinline__ void raise_abort(const WaitCtx& w, int where, int phase) {
-  *w.s_abort = 1;
-  atomicCAS(w.status, 0, MLORA_ERR_TIMEOUT);
-  atomicCAS(w.sync + 3, 0ull, ((unsigned long long)where << 48) | ((unsigned long long)(phase & 0xffff) << 32) |
-                                  ((unsigned long long)(blockIdx.x & 0xffff) << 16) | (unsigned long long)(threadIdx.x & 0xffff));
-  atomicExch(w.sync + 2, 1ull);
-}
-// mbarrier wait; false when the CTA is (or goes) in abort mode
-__device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const WaitCtx& w, int where, int phase) {
-  if (mbar_try_wait(bar, parity)) return true;
-  if (*w.s_abort) return false;
-  const long long t0 = clock64();
-  for (int it = 0;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255) == 255) {
-      if (*w.s_abort) return false;
-      if (ld_acquire_u64(w.sync + 2) != 0ull) { *w.s_abort = 1; return false; }
-      if (clock64() - t0 > w.limit) { raise_abort(w, where, phase); return false; }
-    }
-  }
-}
-// one thread spins until *ctr >= target
-__device__ __forceinline__ void wait_counter(const unsigned long long* ctr, unsigned long long target, const WaitCtx& w,
-                                             int where, int phase) {
-  if (*w.s_abort) return;
-  const long long t0 = clock64();
-  for (int it = 0;; ++it) {
-    if (ld_acquire_u64(ctr) >= target) return;
-    if ((it & 63) == 63) {
-      if (ld_acquire_u64(w.sync + 2) != 0ull) { *w.s_abort = 1; return; }
-      if (clock64() - t0 > w.limit) { raise_abort(w, where, phase); return; }
-    }
-  }
-}
-
-// physical column -> (segment, logical column)
-__device__ __forceinline__ void chain_map_col(int mode, int c, int n0, int n1, int& seg, int& col) {
-  if (mode == MODE_PLAIN) { seg = 0; col = c; }
-  else if (mode == MODE_QKV) {
-    if (c < n0) { seg = 0; col = c; }
-    else if (c < n0 + n1) { seg = 1; col = c - n0; }
-    else { seg = 2; col = c - n0 - n1; }
-  } else {                         // gate/up interleaved by 16-column tiles
-    const int tile = c >> 4;
-    seg = tile & 1;
-    col = ((tile >> 1) << 4) | (c & 15);
-  }
-}
 
 // ----------------------------------------------------------------------------- optional timeline (trace builds only)
 // With -DCHAIN_TRACE thread 0 of the first and the last CTA stamp the global nanosecond timer at the section
@@ -335,7 +234,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
   const int r = a.rank;
   const int r2_shift = (r > 0 && (r & (r - 1)) == 0) ? 32 - __clz(r) : -1;   // log2(2 r) for power-of-two ranks
   const bool lora_on = a.adapter_idx != nullptr && a.rank > 0;
-  WaitCtx wc{a.wait_cycles > 0 ? a.wait_cycles : CH_WAIT_CYCLES, &s_abort_word, a.sync, a.status};
+  WaitCtx wc{a.wait_cycles > 0 ? a.wait_cycles : PIPE_WAIT_CYCLES, &s_abort_word, a.sync, a.status};
 
   // ---- set-up: barriers, first phase descriptor, adapters of the rows, counter bases
   if (tid == 0) {
@@ -601,7 +500,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
       const int r2 = r * 2;                                            // 16-byte pieces per row of a tile
       for (int tu = 0; tu < tpu; ++tu) {
         int seg, col;
-        chain_map_col(ph.mode, (u * tpu + tu) * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
+        map_col(ph.mode, (u * tpu + tu) * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
         if (seg >= nseg) continue;
         const int ldb = ph.lora_n[seg];
         for (int idx = tt; idx < M * r2; idx += team_threads) {
@@ -871,7 +770,7 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
               for (int j = 0; j < wpt; ++j)                               // fixed order: member 0, 1, ...
                 y += redf[((size_t)(tu * CH_CWARPS + tm * wpt + j) * 32 + src_lane) * 4 + e];
               int seg, col;
-              chain_map_col(ph.mode, nt * TILE_N + col16, ph.seg_n0, ph.seg_n1, seg, col);
+              map_col(ph.mode, nt * TILE_N + col16, ph.seg_n0, ph.seg_n1, seg, col);
               if (nseg > 0 && seg < nseg && s_pB[slot][seg][m] != nullptr) {
                 // LoRA expand (second factor of the low-rank term of Eq. 1-4)
                 const float* Tm = Ts + ((size_t)m * nseg + seg) * r;

@@ -95,13 +95,19 @@ struct mlora_ctx {
   cudaEvent_t snap_event = nullptr;
   bool snap_pending = false;
   int snap_inc = 0;
-  int dbg_skip_compact = 0, dbg_no_graph = 0, dbg_no_chain = 0, dbg_no_tc = 0, dbg_inject_stall = 0;
+  int dbg_skip_compact = 0, dbg_no_graph = 0, dbg_no_chain = 0, dbg_no_tc = 0, dbg_inject_stall = 0, dbg_no_step = 0;
   int32_t* host_io = nullptr;        // dev [3][max_streams]: adapter_idx, tokens, next of the host-buffer step
   // persistent projection chain (rows <= 8)
   ChainPhase* phases = nullptr;      // dev [4*L (+1)]: qkv, o, gate/up, down per layer; then lm_head
   int n_phases = 0;
   unsigned long long* chain_sync = nullptr;   // dev [4]
   int chain_stages = 0, chain_kmax = 0;
+  // whole decode step in one kernel (one row per stream, rows <= 8)
+  StepPhase* step_phases = nullptr;  // dev [5*L + 3]: embed; qkv, attention, o, gate/up, down per layer; lm_head; end
+  int n_step_phases = 0, step_stages = 0, step_own_tiles = 0, step_as_bytes = 0;
+  __half *xg_attn = nullptr, *xg_ffn = nullptr;     // residual rows times the gain of the next RMSNorm, fp16 [8][d_model]
+  unsigned long long *step_tacc = nullptr, *step_ssq = nullptr, *step_amax = nullptr;
+  int n_tacc = 0, n_ssq = 0;
   // graphs
   std::unordered_map<GraphKey, GraphEntry, GraphKeyHash> graphs;
   bool capturing = false;
@@ -226,6 +232,43 @@ int launch_attention_block(mlora_ctx* c, const PassIO& io, int l) {
 
 bool chain_eligible(const mlora_ctx* c, const PassIO& io) {
   return c->chain_stages > 0 && !c->dbg_no_chain && !io.prefill && io.n * io.T <= CHAIN_MAX_ROWS;
+}
+
+// a decode step (one row per stream) that the single-kernel path can take
+bool step_eligible(const mlora_ctx* c, int n, int T) {
+  return c->step_stages > 0 && !c->dbg_no_chain && !c->dbg_no_step && T == 1 && n <= CHAIN_MAX_ROWS;
+}
+
+// one decode step as one persistent kernel: embedding to greedy token (or hidden state), suffix lengths advanced
+int forward_step(mlora_ctx* c, int n, const int32_t* adapter_idx, const int32_t* tokens, const __half* hidden,
+                 int32_t* out_next, float* out_logits, float* hidden_out) {
+  const mlora_model_desc& d = c->d;
+  StepArgs a{};
+  a.phases = c->step_phases; a.n_phases = c->n_step_phases; a.M = n; a.eps = d.rms_eps;
+  a.tokens = tokens; a.embed = (const __half*)d.embed; a.vocab = d.vocab; a.hidden_in = hidden;
+  if (adapter_idx != nullptr && d.lora_rank > 0 && d.max_adapters > 0 && d.lora_targets != 0) {
+    a.adapter_idx = adapter_idx; a.tabA = c->tabA; a.tabB = c->tabB; a.scale = c->ad_scale;
+    a.tab_stride = c->L * 7; a.n_slots = d.max_adapters;
+  }
+  a.rank = (d.max_adapters > 0 && d.lora_targets != 0) ? d.lora_rank : 0;
+  a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim; a.P = c->P;
+  a.qkv = c->qkv;
+  a.prefix_k = c->prefix_k; a.prefix_v = c->prefix_v;
+  a.prefix_layer_stride = c->prefix_layer_stride; a.prefix_head_stride = c->prefix_head_stride;
+  a.own_k = c->own_k; a.own_v = c->own_v;
+  a.own_layer_stride = c->own_layer_stride; a.own_stream_stride = c->own_stream_stride; a.own_head_stride = c->own_head_stride;
+  a.suffix_len = c->suffix_len; a.cs_table = c->cs_table;
+  a.logits = out_logits; a.out_next = out_next; a.hidden_out = hidden_out; a.amax = c->step_amax;
+  a.tacc = c->step_tacc; a.ssq = c->step_ssq; a.n_tacc = c->n_tacc; a.n_ssq = c->n_ssq;
+  a.sync = c->chain_sync; a.status = c->status;
+  if (c->dbg_inject_stall) {                           // one pass only: short waits, one barrier that cannot complete
+    a.wait_cycles = 200000000ll;                       // ~0.1 s
+    a.inject_stall = 1;
+    c->dbg_inject_stall = 0;
+  }
+  a.nstages = c->step_stages; a.own_tiles = c->step_own_tiles; a.as_bytes = c->step_as_bytes;
+  CK(run(c, MLORA_PROF_GEMM, [&] { return launch_step(a, c->sm_count, c->stream); }));
+  return MLORA_OK;
 }
 
 // decode-sized pass: the projections of a layer run as one persistent kernel between the attention blocks
@@ -447,6 +490,7 @@ int init_kernels() {
   CK(init_shrink());
   CK(init_attention());
   CK(init_chain());
+  CK(init_step());
   CK(init_gemm_tc());
   done = true;
   return MLORA_OK;
@@ -709,6 +753,93 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
     CKC(cudaMalloc(&c->chain_sync, 4 * sizeof(unsigned long long)));
     CKC(cudaMemsetAsync(c->chain_sync, 0, 4 * sizeof(unsigned long long), st));
   }
+  // ---- phase descriptors and scratch of the single-kernel decode step
+  {
+    const int tg = d.lora_rank > 0 && d.max_adapters > 0 ? d.lora_targets : 0;
+    c->step_stages = step_plan(dm, F, Nq, Nkv, hd, d.lora_rank, tg, c->sm_count, &c->step_own_tiles, &c->step_as_bytes);
+    if (d.max_streams > 0 && c->step_stages > 0) {
+      const int rr = tg ? d.lora_rank : 0;
+      c->n_tacc = 4 * L; c->n_ssq = 2 * L + 1;
+      CKC(cudaMalloc(&c->xg_attn, (size_t)CHAIN_MAX_ROWS * dm * sizeof(__half)));
+      CKC(cudaMalloc(&c->xg_ffn, (size_t)CHAIN_MAX_ROWS * dm * sizeof(__half)));
+      const size_t tacc_bytes = (size_t)c->n_tacc * CHAIN_MAX_ROWS * 3 * (rr > 0 ? rr : 1) * sizeof(unsigned long long);
+      CKC(cudaMalloc(&c->step_tacc, tacc_bytes));
+      CKC(cudaMemsetAsync(c->step_tacc, 0, tacc_bytes, st));
+      CKC(cudaMalloc(&c->step_ssq, (size_t)c->n_ssq * CHAIN_MAX_ROWS * sizeof(unsigned long long)));
+      CKC(cudaMemsetAsync(c->step_ssq, 0, (size_t)c->n_ssq * CHAIN_MAX_ROWS * sizeof(unsigned long long), st));
+      CKC(cudaMalloc(&c->step_amax, (size_t)c->sm_count * CHAIN_MAX_ROWS * sizeof(unsigned long long)));
+      CKC(cudaMemsetAsync(c->step_amax, 0, (size_t)c->sm_count * CHAIN_MAX_ROWS * sizeof(unsigned long long), st));
+      std::vector<StepPhase> sp;
+      auto next_qkv = [&](StepPhase& q, int l) {          // the consuming group is q,k,v of layer l
+        if (tg & (MLORA_Q | MLORA_K | MLORA_V)) {
+          q.next_nseg = 3;
+          for (int i = 0; i < 3; ++i) q.next_proj[i] = l * 7 + i;
+          q.next_ld = dm; q.t_out = 4 * l;
+        }
+      };
+      StepPhase e{};
+      e.kind = SK_EMBED; e.N = dm; e.out16 = c->xg_attn; e.gain_next = c->rms_attn[0]; e.ssq_out = 0; e.norm_in = -1;
+      next_qkv(e, 0);
+      sp.push_back(e);
+      for (int l = 0; l < L; ++l) {
+        StepPhase q{};
+        q.kind = SK_GEMM; q.layer = l; q.w = c->w_qkv[l].data; q.K = dm; q.N = c->Nqkv; q.G = G; q.mode = MODE_QKV; q.epi = EPI_F32;
+        q.seg_n0 = Nq; q.seg_n1 = Nkv; q.in16 = c->xg_attn; q.norm_in = 2 * l; q.out_f32 = c->qkv; q.ldo = c->Nqkv; q.ssq_out = -1;
+        if (tg & (MLORA_Q | MLORA_K | MLORA_V)) {
+          q.lora_nseg = 3;
+          for (int i = 0; i < 3; ++i) q.lora_proj[i] = l * 7 + i;
+          q.lora_n[0] = Nq; q.lora_n[1] = Nkv; q.lora_n[2] = Nkv; q.t_in = 4 * l;
+        }
+        sp.push_back(q);
+        StepPhase at{};
+        at.kind = SK_ATTN; at.layer = l; at.out16 = c->attn16; at.norm_in = -1; at.ssq_out = -1;
+        if (tg & MLORA_O) { at.next_nseg = 1; at.next_proj[0] = l * 7 + 3; at.next_ld = Nq; at.t_out = 4 * l + 1; }
+        sp.push_back(at);
+        StepPhase o{};
+        o.kind = SK_GEMM; o.layer = l; o.w = c->w_o[l].data; o.K = Nq; o.N = dm; o.G = G; o.mode = MODE_PLAIN; o.epi = EPI_RESID;
+        o.in16 = c->attn16; o.norm_in = -1; o.out16 = c->xg_ffn; o.gain_next = c->rms_ffn[l]; o.ssq_out = 2 * l + 1;
+        if (tg & MLORA_O) { o.lora_nseg = 1; o.lora_proj[0] = l * 7 + 3; o.lora_n[0] = dm; o.t_in = 4 * l + 1; }
+        if (tg & (MLORA_GATE | MLORA_UP)) {
+          o.next_nseg = 2; o.next_proj[0] = l * 7 + 4; o.next_proj[1] = l * 7 + 5; o.next_ld = dm; o.t_out = 4 * l + 2;
+        }
+        sp.push_back(o);
+        StepPhase gu{};
+        gu.kind = SK_GEMM; gu.layer = l; gu.w = c->w_gateup[l].data; gu.K = dm; gu.N = 2 * F; gu.G = G; gu.mode = MODE_GATEUP;
+        gu.epi = EPI_SWIGLU; gu.in16 = c->xg_ffn; gu.norm_in = 2 * l + 1; gu.out16 = c->act16; gu.ssq_out = -1;
+        if (tg & (MLORA_GATE | MLORA_UP)) {
+          gu.lora_nseg = 2; gu.lora_proj[0] = l * 7 + 4; gu.lora_proj[1] = l * 7 + 5; gu.lora_n[0] = F; gu.lora_n[1] = F;
+          gu.t_in = 4 * l + 2;
+        }
+        if (tg & MLORA_DOWN) { gu.next_nseg = 1; gu.next_proj[0] = l * 7 + 6; gu.next_ld = F; gu.t_out = 4 * l + 3; }
+        sp.push_back(gu);
+        StepPhase dn{};
+        dn.kind = SK_GEMM; dn.layer = l; dn.w = c->w_down[l].data; dn.K = F; dn.N = dm; dn.G = G; dn.mode = MODE_PLAIN;
+        dn.epi = EPI_RESID; dn.in16 = c->act16; dn.norm_in = -1; dn.ssq_out = -1;
+        if (tg & MLORA_DOWN) { dn.lora_nseg = 1; dn.lora_proj[0] = l * 7 + 6; dn.lora_n[0] = dm; dn.t_in = 4 * l + 3; }
+        if (l + 1 < L) {
+          dn.out16 = c->xg_attn; dn.gain_next = c->rms_attn[l + 1]; dn.ssq_out = 2 * (l + 1);
+          next_qkv(dn, l + 1);
+        } else if (d.vocab > 0) {
+          dn.out16 = c->xg_attn; dn.gain_next = (const __half*)d.rms_final; dn.ssq_out = 2 * L;
+        } else {
+          dn.last = 1;
+        }
+        sp.push_back(dn);
+      }
+      if (d.vocab > 0) {
+        StepPhase lm{};
+        lm.kind = SK_GEMM; lm.layer = L; lm.w = c->w_lm.data; lm.K = dm; lm.N = d.vocab; lm.G = G; lm.mode = MODE_PLAIN;
+        lm.epi = EPI_F32; lm.in16 = c->xg_attn; lm.norm_in = 2 * L; lm.out_f32 = nullptr; lm.ldo = d.vocab; lm.ssq_out = -1;
+        sp.push_back(lm);
+      }
+      StepPhase fin{};
+      fin.kind = SK_FIN; fin.norm_in = -1; fin.ssq_out = -1;
+      sp.push_back(fin);
+      c->n_step_phases = (int)sp.size();
+      CKC(cudaMalloc(&c->step_phases, sp.size() * sizeof(StepPhase)));
+      CKC(cudaMemcpy(c->step_phases, sp.data(), sp.size() * sizeof(StepPhase), cudaMemcpyHostToDevice));
+    }
+  }
   CKC(cudaMallocHost(&c->snap, d.max_streams * sizeof(int32_t)));
   CKC(cudaEventCreateWithFlags(&c->snap_event, cudaEventDisableTiming));
   CKC(cudaStreamSynchronize(st));
@@ -729,7 +860,8 @@ int mlora_destroy(mlora_ctx* c) {
   void* dev_ptrs[] = {c->prefix_k, c->prefix_v, c->own_k, c->own_v, c->X, c->qkv, c->logits, c->T, c->partial, c->att_ws,
                       c->h, c->attn16, c->act16, c->counters, c->anc, c->depth, c->argmax, c->suffix_len,
                       c->zero_len, c->chain_parent, c->root_parent, c->status, c->cs_table, (void*)c->tabA,
-                      (void*)c->tabB, c->ad_scale, c->phases, c->chain_sync, c->host_io};
+                      (void*)c->tabB, c->ad_scale, c->phases, c->chain_sync, c->host_io, c->step_phases, c->xg_attn, c->xg_ffn,
+                      c->step_tacc, c->step_ssq, c->step_amax};
   for (void* p : dev_ptrs) if (p) cudaFree(p);
   if (c->stageA) cudaFreeHost((void*)c->stageA);
   if (c->stageB) cudaFreeHost((void*)c->stageB);
@@ -786,6 +918,13 @@ static int decode_impl(mlora_ctx* c, int n, const int32_t* adapter_idx, const in
                        int32_t* out_next, float* out_logits, float* hidden_out) {
   int rc = step_common_checks(c, n, adapter_idx, 1);
   if (rc != MLORA_OK) return rc;
+  if (step_eligible(c, n, 1)) {
+    rc = forward_step(c, n, adapter_idx, tokens, hidden, out_next, out_logits, hidden_out);
+    if (rc != MLORA_OK) return rc;
+    c->suffix_bound += 1;
+    if (c->snap_pending) c->snap_inc += 1;
+    return MLORA_OK;
+  }
   PassIO io;
   io.n = n; io.T = 1; io.tokens = tokens; io.hidden_in = hidden; io.adapter_idx = adapter_idx;
   io.parent = c->root_parent; io.pos_base = c->P; io.suffix_len = c->suffix_len; io.suffix_bound = c->suffix_bound;
@@ -920,6 +1059,12 @@ int mlora_sync_status(mlora_ctx* c) {
     CK(cudaMemcpy(&where, c->chain_sync + 3, sizeof(where), cudaMemcpyDeviceToHost));
     // a wait that ran out leaves the barrier counters of the persistent kernel mid-count: start them afresh
     CK(cudaMemset(c->chain_sync, 0, 4 * sizeof(unsigned long long)));
+    // ... and the step kernel's accumulators part-filled
+    if (c->step_tacc) {
+      const int rr = c->d.lora_rank > 0 && c->d.max_adapters > 0 && c->d.lora_targets ? c->d.lora_rank : 1;
+      CK(cudaMemset(c->step_tacc, 0, (size_t)c->n_tacc * CHAIN_MAX_ROWS * 3 * rr * sizeof(unsigned long long)));
+      CK(cudaMemset(c->step_ssq, 0, (size_t)c->n_ssq * CHAIN_MAX_ROWS * sizeof(unsigned long long)));
+    }
     if (st == MLORA_ERR_TIMEOUT) {
       char buf[160];
       std::snprintf(buf, sizeof(buf), "device status: a bounded wait ran out (wait kind %d, phase %d, block %d, thread %d)",
@@ -995,6 +1140,7 @@ int mlora_debug_set(mlora_ctx* c, int32_t key, int32_t value) {
   else if (key == 3) c->dbg_no_chain = value ? 1 : 0;
   else if (key == 4) c->dbg_no_tc = value ? 1 : 0;
   else if (key == 5) c->dbg_inject_stall = value ? 1 : 0;
+  else if (key == 6) c->dbg_no_step = value ? 1 : 0;
   else return fail(MLORA_ERR_ARG, "unknown debug key");
   return MLORA_OK;
 }

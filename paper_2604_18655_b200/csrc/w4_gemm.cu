@@ -121,20 +121,6 @@ cudaError_t launch_dequant(const unsigned char* w, int K, int N, int G, int tile
 }
 
 // ----------------------------------------------------------------------------- GEMM
-// physical column -> (segment, logical column)
-__device__ __forceinline__ void map_col(int mode, int c, int n0, int n1, int& seg, int& col) {
-  if (mode == MODE_PLAIN) { seg = 0; col = c; }
-  else if (mode == MODE_QKV) {
-    if (c < n0) { seg = 0; col = c; }
-    else if (c < n0 + n1) { seg = 1; col = c - n0; }
-    else { seg = 2; col = c - n0 - n1; }
-  } else {                         // gate/up interleaved by 16-column tiles
-    const int tile = c >> 4;
-    seg = tile & 1;
-    col = ((tile >> 1) << 4) | (c & 15);
-  }
-}
-
 struct GemmPlan {
   int ksplit, kts_per_split, kc_tiles, m_blocks, n_blocks, mt;
   size_t smem;

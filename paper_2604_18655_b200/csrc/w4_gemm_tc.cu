@@ -277,20 +277,6 @@ w4_gemm_tc_kernel(const GemmArgs p, const int kts_per_split, int* status, const 
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)NROWS) : "memory");
 }
 
-// physical column -> (segment, logical column)
-__device__ __forceinline__ void tc_map_col(int mode, int c, int n0, int n1, int& seg, int& col) {
-  if (mode == MODE_PLAIN) { seg = 0; col = c; }
-  else if (mode == MODE_QKV) {
-    if (c < n0) { seg = 0; col = c; }
-    else if (c < n0 + n1) { seg = 1; col = c - n0; }
-    else { seg = 2; col = c - n0 - n1; }
-  } else {                         // gate/up interleaved by 16-column tiles
-    const int tile = c >> 4;
-    seg = tile & 1;
-    col = ((tile >> 1) << 4) | (c & 15);
-  }
-}
-
 // sum of the K splits (fixed order) plus the LoRA expand term of four consecutive physical columns of row m
 __device__ __forceinline__ float4 tc_row_quad(const GemmArgs& p, int ksplit, int m, int c) {
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -312,7 +298,7 @@ __device__ __forceinline__ float4 tc_row_quad(const GemmArgs& p, int ksplit, int
     const int a = p.lora.adapter_idx[m / p.lora.rows_per_stream];
     if (a >= 0 && a < p.lora.n_slots) {
       int seg, col;
-      tc_map_col(p.mode, c, p.seg_n0, p.seg_n1, seg, col);
+      map_col(p.mode, c, p.seg_n0, p.seg_n1, seg, col);
       const __half* B = p.lora.tabB[(size_t)a * p.lora.tab_stride + p.lora.seg[seg].proj_index];
       if (B != nullptr) {
         const int r = p.lora.rank, ldb = p.lora.seg[seg].n;
@@ -423,7 +409,7 @@ __global__ void __launch_bounds__(256) gemm_tc_epilogue_mma_kernel(const GemmArg
         const int r = p.lora.rank;
         int seg_of[4], col_of[4];
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) tc_map_col(p.mode, min(c0 + nt * 8, p.N - 8), p.seg_n0, p.seg_n1, seg_of[nt], col_of[nt]);
+        for (int nt = 0; nt < 4; ++nt) map_col(p.mode, min(c0 + nt * 8, p.N - 8), p.seg_n0, p.seg_n1, seg_of[nt], col_of[nt]);
         for (int seg = 0; seg < p.lora.nseg; ++seg) {
           bool any = false;
 #pragma unroll

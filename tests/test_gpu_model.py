@@ -302,7 +302,8 @@ def test_error_paths(GpuModel):
 
 
 def test_graph_replay_matches_direct_launches(GpuModel):
-    """Steps replayed from a CUDA graph give bit-identical logits to directly launched ones."""
+    """Steps of the multi-kernel path (debug switch 6: no single-kernel step) replayed from a CUDA graph give
+    bit-identical logits to directly launched ones."""
     from paper_2604_18655_b200 import binding as mb
     cfg = TINYV
     res = []
@@ -310,6 +311,7 @@ def test_graph_replay_matches_direct_launches(GpuModel):
     for no_graph in (1, 0):
         with torch.cuda.stream(side):
             m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+            mb.mlora_debug_set(gm.ctx, 6, 1)
             mb.mlora_debug_set(gm.ctx, 2, no_graph)
             gm.prefill(gen.make_prompt_ids(cfg, 0))
             dev = torch.device("cuda")
@@ -330,15 +332,38 @@ def test_graph_replay_matches_direct_launches(GpuModel):
     assert np.array_equal(res[0].view(np.uint32), res[1].view(np.uint32))
 
 
-def test_decode_paths_agree(GpuModel):
-    """The persistent projection kernel against the one-kernel-per-projection form of the same arithmetic (debug
-    switch 3): logits and KV within the parity tolerance."""
+def test_step_kernel_is_one_launch_and_bit_reproducible(GpuModel):
+    """A decode step is ONE kernel launch, and two runs of the same steps give bit-identical logits (the cross-CTA
+    sums of the kernel are integer atomics on fixed-point values: the order of arrival cannot change them)."""
     from paper_2604_18655_b200 import binding as mb
     cfg = TINYV
     res = []
-    for no_chain in (0, 1):
+    for rep in range(2):
         m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
-        mb.mlora_debug_set(gm.ctx, 3, no_chain)
+        gm.prefill(gen.make_prompt_ids(cfg, 0))
+        toks = np.array([1, 2, 3], dtype=np.int32)
+        hist = []
+        before = mb.mlora_launch_count(gm.ctx)
+        for _ in range(5):
+            toks, logits = gm.decode([0, 1, -1], toks)
+            hist.append(logits)
+        assert mb.mlora_launch_count(gm.ctx) - before == 5
+        res.append(np.stack(hist))
+        mb.mlora_sync_status(gm.ctx)
+        gm.close()
+    assert np.array_equal(res[0].view(np.uint32), res[1].view(np.uint32))
+
+
+def test_decode_paths_agree(GpuModel):
+    """The single-kernel step against the per-layer persistent projection kernel (debug switch 6) and the
+    one-kernel-per-projection form of the same arithmetic (debug switch 3): logits and KV within the parity tolerance."""
+    from paper_2604_18655_b200 import binding as mb
+    cfg = TINYV
+    res = []
+    for key in (0, 6, 3):
+        m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+        if key:
+            mb.mlora_debug_set(gm.ctx, key, 1)
         gm.prefill(gen.make_prompt_ids(cfg, 0))
         toks = np.array([1, 2, 3], dtype=np.int32)
         hist = []
@@ -349,9 +374,10 @@ def test_decode_paths_agree(GpuModel):
         res.append((np.stack(hist), k, v))
         mb.mlora_sync_status(gm.ctx)
         gm.close()
-    compare(res[1][0], res[0][0], "logits across paths")
-    compare(res[1][1], res[0][1], "K across paths")
-    compare(res[1][2], res[0][2], "V across paths")
+    for i in (0, 1):
+        compare(res[i][0], res[2][0], "logits across paths")
+        compare(res[i][1], res[2][1], "K across paths")
+        compare(res[i][2], res[2][2], "V across paths")
 
 
 def test_host_buffer_step_matches_device_step(GpuModel):
