@@ -42,6 +42,8 @@ def parse_args():
     ap.add_argument("--config", default="cfg1", choices=["cfg0", "cfg1", "cfg2", "cfg3"],
                     help="cfg1 (default) is the benchmark workload; cfg2/cfg3 time DS2D verify rounds (side measurement)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--timeline", action="store_true",
+                    help="profiling aid: print the phase timeline of one traced decode step (markdown) instead of the bench line")
     ap.add_argument("--layers", type=int, default=None,
                     help="profiling aid: cut the model to this many layers (small ncu captures); not a bench result")
     return ap.parse_args()
@@ -289,6 +291,36 @@ def run_verify(args, cfg):
     model.close()
 
 
+def print_timeline(tl, cfg):
+    """Markdown table of one traced decode step: per phase kind, mean microseconds between the stamps of CTA 0
+    (main loop / partial sums parked / epilogue / rest of the phase / wait for the CTA / grid barrier)."""
+    kinds = ["embed"] + ["qkv", "attention", "o", "gate_up", "down"] * cfg.n_layers + (["lm_head"] if cfg.vocab else []) + ["end"]
+    names = ["slices", "weights", "tile0", "main", "park", "epilogue", "rest", "cta_sync", "barrier"]
+    agg = {}
+    for cta in (0, 1):
+        for p, k in enumerate(kinds):
+            st = tl[cta][p]
+            if st[0] == 0:
+                continue
+            prev, row = st[0], []
+            for i in (7, 8, 9, 1, 2, 3, 4, 5, 6):
+                if st[i] == 0:
+                    row.append(0.0)
+                else:
+                    row.append((st[i] - prev) / 1e3)
+                    prev = st[i]
+            row.append((prev - st[0]) / 1e3)
+            agg.setdefault((cta, k), []).append(row)
+    print("| CTA | phase | n | " + " | ".join(names) + " | total us |")
+    print("|---|---|---|" + "---|" * (len(names) + 1))
+    for (cta, k), rows in agg.items():
+        m = np.mean(np.array(rows), axis=0)
+        print(f"| {'first' if cta == 0 else 'last'} | {k} | {len(rows)} | " + " | ".join(f"{v:.2f}" for v in m) + " |")
+    t0 = min(tl[0][0][0], tl[1][0][0] or tl[0][0][0])
+    t1 = max(max(tl[0][-1]), max(tl[1][-1]))
+    print(f"\nstep (first stamp to last stamp): {(t1 - t0) / 1e3:.1f} us")
+
+
 def workload_name(cfg):
     return (f"{cfg.name}: d{cfg.d_model} L{cfg.n_layers} {cfg.n_q_heads}q/{cfg.n_kv_heads}kv hd{cfg.head_dim} "
             f"ffn{cfg.d_ffn} vocab{cfg.vocab} int4-g{cfg.group_size}; {cfg.n_streams} streams x rank-{cfg.lora_rank} "
@@ -368,6 +400,12 @@ def main():
         # ---- device-resident timed region
         for i in range(W):
             generation_step(i)
+        if args.timeline:
+            mb.mlora_debug_set(ctx, 7, 1)
+            generation_step(W)
+            print_timeline(mb.mlora_step_timeline(ctx), cfg)
+            model.close()
+            return
         sampler = ClockSampler(local)
         sampler.start()
         barrier()

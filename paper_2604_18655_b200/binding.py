@@ -59,6 +59,7 @@ _SIGS = {
     "mlora_profile_begin": (C.c_int, [C.c_void_p]),
     "mlora_profile_end": (C.c_int, [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32)]),
     "mlora_launch_count": (C.c_int64, [C.c_void_p]),
+    "mlora_step_timeline": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64), C.c_int32, C.POINTER(C.c_int32)]),
     "mlora_weight_create": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
                                       C.POINTER(C.c_void_p)]),
     "mlora_weight_destroy": (C.c_int, [C.c_void_p]),
@@ -216,6 +217,17 @@ def mlora_profile_end(ctx):
 
 def mlora_launch_count(ctx):
     return int(lib().mlora_launch_count(ctx))
+
+
+def mlora_step_timeline(ctx):
+    """Stamps of the last traced decode step as a nested list [2][n_phases][12] of nanoseconds (0: no stamp)."""
+    n = C.c_int32(0)
+    lib().mlora_step_timeline(ctx, None, 0, C.byref(n))          # asks for the phase count only
+    cnt = n.value * 24
+    buf = (C.c_int64 * max(cnt, 1))()
+    _check(lib().mlora_step_timeline(ctx, buf, cnt, C.byref(n)))
+    vals = list(buf)
+    return [[vals[(c * n.value + p) * 12:(c * n.value + p) * 12 + 12] for p in range(n.value)] for c in range(2)]
 
 
 # ----------------------------------------------------------------------------- kernel-level calls

@@ -233,6 +233,8 @@ struct StepArgs {
   const __half* const* tabB;
   const float* scale;
   int tab_stride, n_slots, rank;
+  const unsigned char* tmapA;     // dev [n_slots][tab_stride] tensor maps (STEP_TMAP_BYTES each) over the A / B matrices:
+  const unsigned char* tmapB;     // boxes of 16 columns x rank rows
   // attention
   int Hq, Hkv, hd, P;
   const float* qkv;               // fp32 [8][(Hq + 2 Hkv) hd]: q,k,v projections of the layer
@@ -253,11 +255,15 @@ struct StepArgs {
   int* status;
   long long wait_cycles;
   int inject_stall;
-  int nstages, own_tiles, as_bytes;
+  int nstages, own_tiles;
+  long long* trace;               // dev [2][n_phases][12] nanosecond stamps of the first and the last CTA, or nullptr
 };
 cudaError_t init_step();
 // ring stages the step kernel gets for this model on this device (0: the kernel cannot run it)
-int step_plan(int d_model, int d_ffn, int Nq, int Nkv, int hd, int rank, int lora_targets, int sm_count, int* own_tiles, int* as_bytes);
+int step_plan(int d_model, int d_ffn, int Nq, int Nkv, int hd, int rank, int lora_targets, int sm_count, int* own_tiles);
+constexpr int STEP_TMAP_BYTES = 128;
+// tensor map (STEP_TMAP_BYTES, host memory) over one LoRA matrix fp16 [rank][width] for the step kernel's slice copies
+cudaError_t step_encode_slice_map(const void* base, int width, int rank, void* map_out);
 cudaError_t launch_step(const StepArgs& a, int sm_count, cudaStream_t st);
 
 // ----------------------------------------------------------------------------- launchers

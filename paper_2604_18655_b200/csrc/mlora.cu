@@ -104,9 +104,13 @@ struct mlora_ctx {
   int chain_stages = 0, chain_kmax = 0;
   // whole decode step in one kernel (one row per stream, rows <= 8)
   StepPhase* step_phases = nullptr;  // dev [5*L + 3]: embed; qkv, attention, o, gate/up, down per layer; lm_head; end
-  int n_step_phases = 0, step_stages = 0, step_own_tiles = 0, step_as_bytes = 0;
+  int n_step_phases = 0, step_stages = 0, step_own_tiles = 0;
+  unsigned char *tmapA = nullptr, *tmapB = nullptr;           // dev [max_adapters][L*7] tensor maps over the adapters' matrices
+  unsigned char *stage_tmA = nullptr, *stage_tmB = nullptr;   // pinned host staging of the same
   __half *xg_attn = nullptr, *xg_ffn = nullptr;     // residual rows times the gain of the next RMSNorm, fp16 [8][d_model]
   unsigned long long *step_tacc = nullptr, *step_ssq = nullptr, *step_amax = nullptr;
+  long long* step_trace = nullptr;   // dev [2][n_step_phases][8]
+  int dbg_trace = 0;
   int n_tacc = 0, n_ssq = 0;
   // graphs
   std::unordered_map<GraphKey, GraphEntry, GraphKeyHash> graphs;
@@ -249,6 +253,7 @@ int forward_step(mlora_ctx* c, int n, const int32_t* adapter_idx, const int32_t*
   if (adapter_idx != nullptr && d.lora_rank > 0 && d.max_adapters > 0 && d.lora_targets != 0) {
     a.adapter_idx = adapter_idx; a.tabA = c->tabA; a.tabB = c->tabB; a.scale = c->ad_scale;
     a.tab_stride = c->L * 7; a.n_slots = d.max_adapters;
+    a.tmapA = c->tmapA; a.tmapB = c->tmapB;
   }
   a.rank = (d.max_adapters > 0 && d.lora_targets != 0) ? d.lora_rank : 0;
   a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim; a.P = c->P;
@@ -266,7 +271,8 @@ int forward_step(mlora_ctx* c, int n, const int32_t* adapter_idx, const int32_t*
     a.inject_stall = 1;
     c->dbg_inject_stall = 0;
   }
-  a.nstages = c->step_stages; a.own_tiles = c->step_own_tiles; a.as_bytes = c->step_as_bytes;
+  a.nstages = c->step_stages; a.own_tiles = c->step_own_tiles;
+  a.trace = c->dbg_trace ? c->step_trace : nullptr;
   CK(run(c, MLORA_PROF_GEMM, [&] { return launch_step(a, c->sm_count, c->stream); }));
   return MLORA_OK;
 }
@@ -702,6 +708,12 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
     CKC(cudaMallocHost(&c->stageA, ents * sizeof(void*)));
     CKC(cudaMallocHost(&c->stageB, ents * sizeof(void*)));
     CKC(cudaMallocHost(&c->stage_scale, d.max_adapters * sizeof(float)));
+    CKC(cudaMalloc(&c->tmapA, ents * STEP_TMAP_BYTES));
+    CKC(cudaMalloc(&c->tmapB, ents * STEP_TMAP_BYTES));
+    CKC(cudaMemsetAsync(c->tmapA, 0, ents * STEP_TMAP_BYTES, st));
+    CKC(cudaMemsetAsync(c->tmapB, 0, ents * STEP_TMAP_BYTES, st));
+    CKC(cudaMallocHost(&c->stage_tmA, ents * STEP_TMAP_BYTES));
+    CKC(cudaMallocHost(&c->stage_tmB, ents * STEP_TMAP_BYTES));
   }
   // ---- phase descriptors of the persistent projection chain
   {
@@ -756,7 +768,7 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
   // ---- phase descriptors and scratch of the single-kernel decode step
   {
     const int tg = d.lora_rank > 0 && d.max_adapters > 0 ? d.lora_targets : 0;
-    c->step_stages = step_plan(dm, F, Nq, Nkv, hd, d.lora_rank, tg, c->sm_count, &c->step_own_tiles, &c->step_as_bytes);
+    c->step_stages = step_plan(dm, F, Nq, Nkv, hd, d.lora_rank, tg, c->sm_count, &c->step_own_tiles);
     if (d.max_streams > 0 && c->step_stages > 0) {
       const int rr = tg ? d.lora_rank : 0;
       c->n_tacc = 4 * L; c->n_ssq = 2 * L + 1;
@@ -836,6 +848,8 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
       fin.kind = SK_FIN; fin.norm_in = -1; fin.ssq_out = -1;
       sp.push_back(fin);
       c->n_step_phases = (int)sp.size();
+      CKC(cudaMalloc(&c->step_trace, sp.size() * 2 * 12 * sizeof(long long)));
+      CKC(cudaMemsetAsync(c->step_trace, 0, sp.size() * 2 * 12 * sizeof(long long), st));
       CKC(cudaMalloc(&c->step_phases, sp.size() * sizeof(StepPhase)));
       CKC(cudaMemcpy(c->step_phases, sp.data(), sp.size() * sizeof(StepPhase), cudaMemcpyHostToDevice));
     }
@@ -861,11 +875,13 @@ int mlora_destroy(mlora_ctx* c) {
                       c->h, c->attn16, c->act16, c->counters, c->anc, c->depth, c->argmax, c->suffix_len,
                       c->zero_len, c->chain_parent, c->root_parent, c->status, c->cs_table, (void*)c->tabA,
                       (void*)c->tabB, c->ad_scale, c->phases, c->chain_sync, c->host_io, c->step_phases, c->xg_attn, c->xg_ffn,
-                      c->step_tacc, c->step_ssq, c->step_amax};
+                      c->step_tacc, c->step_ssq, c->step_amax, c->step_trace, c->tmapA, c->tmapB};
   for (void* p : dev_ptrs) if (p) cudaFree(p);
   if (c->stageA) cudaFreeHost((void*)c->stageA);
   if (c->stageB) cudaFreeHost((void*)c->stageB);
   if (c->stage_scale) cudaFreeHost(c->stage_scale);
+  if (c->stage_tmA) cudaFreeHost(c->stage_tmA);
+  if (c->stage_tmB) cudaFreeHost(c->stage_tmB);
   if (c->snap) cudaFreeHost(c->snap);
   if (c->snap_event) cudaEventDestroy(c->snap_event);
   for (auto& e : c->evs) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
@@ -895,6 +911,29 @@ int mlora_set_adapter(mlora_ctx* c, int32_t slot, const void* const* A, const vo
     c->stageB[slot * per + i] = on ? (const __half*)B[i] : nullptr;
   }
   c->stage_scale[slot] = A ? alpha / (float)c->d.lora_rank : 0.f;
+  // tensor maps over the caller's matrices for the single-kernel decode step (its producer warp copies 16-column
+  // slices of them; nothing of the matrices themselves is copied or repacked here)
+  if (c->step_stages > 0) {
+    const mlora_model_desc& d = c->d;
+    const int widthK[7] = {d.d_model, d.d_model, d.d_model, c->Nq, d.d_model, d.d_model, d.d_ffn};
+    const int widthN[7] = {c->Nq, c->Nkv, c->Nkv, d.d_model, d.d_ffn, d.d_ffn, d.d_model};
+    for (size_t i = 0; i < per; ++i) {
+      const int p = (int)(i % 7);
+      unsigned char* ma = c->stage_tmA + (slot * per + i) * STEP_TMAP_BYTES;
+      unsigned char* mb = c->stage_tmB + (slot * per + i) * STEP_TMAP_BYTES;
+      if (c->stageA[slot * per + i] != nullptr) {
+        CK(step_encode_slice_map(c->stageA[slot * per + i], widthK[p], d.lora_rank, ma));
+        CK(step_encode_slice_map(c->stageB[slot * per + i], widthN[p], d.lora_rank, mb));
+      } else {
+        std::memset(ma, 0, STEP_TMAP_BYTES);
+        std::memset(mb, 0, STEP_TMAP_BYTES);
+      }
+    }
+    CK(cudaMemcpyAsync(c->tmapA + slot * per * STEP_TMAP_BYTES, c->stage_tmA + slot * per * STEP_TMAP_BYTES, per * STEP_TMAP_BYTES,
+                       cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(c->tmapB + slot * per * STEP_TMAP_BYTES, c->stage_tmB + slot * per * STEP_TMAP_BYTES, per * STEP_TMAP_BYTES,
+                       cudaMemcpyHostToDevice, c->stream));
+  }
   CK(cudaMemcpyAsync(c->tabA + slot * per, c->stageA + slot * per, per * sizeof(void*), cudaMemcpyHostToDevice, c->stream));
   CK(cudaMemcpyAsync(c->tabB + slot * per, c->stageB + slot * per, per * sizeof(void*), cudaMemcpyHostToDevice, c->stream));
   CK(cudaMemcpyAsync(c->ad_scale + slot, c->stage_scale + slot, sizeof(float), cudaMemcpyHostToDevice, c->stream));
@@ -1141,6 +1180,7 @@ int mlora_debug_set(mlora_ctx* c, int32_t key, int32_t value) {
   else if (key == 4) c->dbg_no_tc = value ? 1 : 0;
   else if (key == 5) c->dbg_inject_stall = value ? 1 : 0;
   else if (key == 6) c->dbg_no_step = value ? 1 : 0;
+  else if (key == 7) c->dbg_trace = value ? 1 : 0;
   else return fail(MLORA_ERR_ARG, "unknown debug key");
   return MLORA_OK;
 }
@@ -1170,6 +1210,18 @@ int mlora_profile_end(mlora_ctx* c, float* ms, int32_t* launches) {
 }
 
 int64_t mlora_launch_count(mlora_ctx* c) { return c ? c->launches : 0; }
+
+int mlora_step_timeline(mlora_ctx* c, int64_t* host_out, int32_t capacity, int32_t* n_phases) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (!n_phases) return fail(MLORA_ERR_ARG, "null argument");
+  *n_phases = c->n_step_phases;
+  if (c->step_trace == nullptr) return fail(MLORA_ERR_STATE, "this context has no single-kernel decode step");
+  const size_t n = (size_t)c->n_step_phases * 2 * 12;
+  if (!host_out || (size_t)capacity < n) return fail(MLORA_ERR_CAPACITY, "timeline needs 24 values per phase");
+  CK(cudaStreamSynchronize(c->stream));
+  CK(cudaMemcpy(host_out, c->step_trace, n * sizeof(long long), cudaMemcpyDeviceToHost));
+  return MLORA_OK;
+}
 
 // ----------------------------------------------------------------------------- kernel-level calls
 int mlora_weight_create(const void* qweight, const void* scales, int32_t K, int32_t N, int32_t G, void* cuda_stream,
