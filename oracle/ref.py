@@ -28,8 +28,10 @@ computation; base projection against numpy matmul; run-time LoRA against the mer
 and the one-hot-masked sum of Sec. 3.2 (approach b); stream isolation; tree rows against sequential
 decode of each root path; shared-prefix attention against plain causal attention over the
 concatenated sequence; RoPE/RMSNorm/SiLU closed forms; accept walk against brute force on every
-small tree; the (3,2) -> 9/10/30 node counts and the 32-row budgets of Table 7.
-Parity unpinned: absolute activation values of a forward pass (the paper prints none).
+small tree; the (3,2) -> 9/10/30 node counts and the 32-row budgets of Table 7; the wiring of a decoder block
+(norm placement, residuals, gate/up roles, final norm) against scalar loops written from the definitions
+(tests/test_oracle_wiring_pin.py).
+Parity unpinned by the paper: absolute activation values of a forward pass of ITS model (it prints none).
 """
 import numpy as np
 

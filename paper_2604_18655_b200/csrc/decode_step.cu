@@ -38,7 +38,7 @@ constexpr int DS_CTHREADS = DS_CWARPS * 32;
 constexpr int DS_THREADS = DS_CTHREADS + 32;       // + one producer warp
 constexpr int DS_STAGE_BYTES = 4480;               // >= CHUNK_KT*512 + 8*32, multiple of 128
 constexpr int DS_MAX_STAGES = 48;
-constexpr int DS_BT = 4;                           // output tiles whose partial sums are parked together
+constexpr int DS_BT = 6;                           // output tiles whose partial sums are parked together
 constexpr int DS_MAX_ITEMS = 6;                    // work items (one k-tile) per warp and tile: K <= 5760
 constexpr int DS_ITEM_KT = 1;
 constexpr int DS_ITEMS_PER_CHUNK = CHUNK_KT / DS_ITEM_KT;   // = arrivals that free a ring stage
@@ -99,7 +99,7 @@ int step_plan(int d_model, int d_ffn, int Nq, int Nkv, int hd, int rank, int lor
   // two tiles of the widest input with their slices must fit the ring (see the parity rule in the kernel)
   int maxK = d_model; if (Nq > maxK) maxK = Nq; if (d_ffn > maxK) maxK = d_ffn;
   const int nch = (maxK / TILE_K + CHUNK_KT - 1) / CHUNK_KT;
-  if (n < DS_MIN_STAGES || n < 2 * (nch + 4 * ds_stages_per_set(r))) return 0;
+  if (n < DS_MIN_STAGES || n < 2 * (nch + 4 * ds_stages_per_set(r))) return 0;   // ds_batch_tiles >= 2 for every group
   *own_tiles = ot;
   return n;
 }
@@ -140,6 +140,24 @@ __device__ __forceinline__ void ring_at(int st0, uint32_t par0, int off, int n, 
   par = par0;
   if (st >= n) { st -= n; par ^= 1u; }
 }
+// tiles per batch of a projection group: the batch's slice stages and weight chunks must fit the ring (a warp may be
+// a whole batch ahead of the slowest one, and a wait must never be a ring lap ahead of the fill front: mbarrier
+// parities repeat every two laps)
+__device__ __forceinline__ int ds_batch_tiles(int nstages, int nchunks, int spr, int nseg, int nnext, int tpu) {
+  const int per_tile = nchunks + (nseg > 0 ? spr : 0) + (nnext * spr + tpu - 1) / tpu;
+  int bt = nstages / per_tile;
+  if (bt > DS_BT) bt = DS_BT;
+  if (tpu == 2) bt &= ~1;
+  return bt;
+}
+__device__ __forceinline__ void ds_ldmatrix_x4(uint32_t (&r)[4], const void* smem) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(smem)));
+}
+__device__ __forceinline__ void ds_ldmatrix_x4_trans(uint32_t (&r)[4], const void* smem) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(smem)));
+}
 __device__ __forceinline__ void ds_stamp(const StepArgs& a, int p, int id) {
   if (a.trace != nullptr && threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1)) {
     long long tns;
@@ -160,8 +178,9 @@ struct GemmLoop {
 // The warp's NI work items (two k-tiles each) of every tile of the batch.  Its slice of the input rows (mma B
 // fragments: row g of the lane, features 16t..16t+15 of each k-tile, zero past M) is loaded from L2 into registers
 // first and serves every tile of the batch.
-template <int NI>
-__device__ __forceinline__ void gemm_tiles(const GemmLoop& q, const WaitCtx& wc) {
+// `early` runs right behind the issue of those loads (further loads the phase needs: one round trip for all).
+template <int NI, class Early>
+__device__ __forceinline__ void gemm_tiles(const GemmLoop& q, const WaitCtx& wc, Early early) {
   uint4 bfr[NI][DS_ITEM_KT][2];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
@@ -180,9 +199,11 @@ __device__ __forceinline__ void gemm_tiles(const GemmLoop& q, const WaitCtx& wc)
           bfr[qi][k2][1] = make_uint4(0, 0, 0, 0);
         }
       }
+    early();
   }
   int st_t = q.st_b;
   uint32_t par_t = q.par_b;
+#pragma unroll 1
   for (int tl = 0; tl < q.nb; ++tl) {
     float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
     int c_cur = -1, st = 0, kc = 0;
@@ -237,7 +258,7 @@ __device__ __forceinline__ void gemm_tiles(const GemmLoop& q, const WaitCtx& wc)
       q.tr[9] = tns + (long long)(acc0[0] != acc0[0] ? 1 : 0);
     }
     // park the tile's partial sums: [tile][warp][lane]
-    q.red[(size_t)(tl * DS_CWARPS + warp) * 32 + lane] =
+    q.red[(size_t)(tl * 16 + warp) * 32 + lane] =
         make_float4(acc0[0] + acc1[0], acc0[1] + acc1[1], acc0[2] + acc1[2], acc0[3] + acc1[3]);
     st_t += q.nchunks;
     if (st_t >= q.nstages) { st_t -= q.nstages; par_t ^= 1u; }
@@ -271,6 +292,7 @@ __device__ __forceinline__ void attn_phase(const StepArgs& a, const PhaseS& ps, 
   const int ocols = g_heads * HD;
   const int rps = ds_rows_per_stage(r), slot = ds_slot_bytes(r);
   const int n_ao = (ocols / TILE_N + rps - 1) / rps;                  // ring stages of the o projection's A slices
+#pragma unroll 1
   for (int u = bid; u < M * Hkv; u += G) {
     const int s = u / Hkv, h = u - s * Hkv;
     const int S = s_suffix[s];
@@ -344,6 +366,7 @@ __device__ __forceinline__ void attn_phase(const StepArgs& a, const PhaseS& ps, 
     for (int i = 0; i < 4; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
     float mrow = -INFINITY, lrow = 0.f;                               // of head g (the lane's row of QK^T)
     const int src_a = (2 * t) * 4 + t, src_b = (2 * t + 1) * 4 + t;   // lanes that hold heads 2t and 2t+1
+#pragma unroll 1
     for (int ti = warp; ti < n_tiles; ti += DS_CWARPS) {
       const bool own = ti >= nP;
       const int k0 = (own ? ti - nP : ti) << 4, kend = own ? S : a.P;
@@ -464,12 +487,14 @@ __device__ __forceinline__ void attn_phase(const StepArgs& a, const PhaseS& ps, 
     // (column block cb of 16 in slot cb of the unit's ring stages, [rank][16]) came through the ring
     if (ph.next_nseg > 0 && a.adapter_idx != nullptr && r > 0) {
       // (every stage is waited for before it is released, also when the row has no adapter and nothing was copied)
+#pragma unroll 1
       for (int k = 0; k < n_ao; ++k) {
         int st; uint32_t par;
         ring_at(pos.st, pos.par, k, nstages, st, par);
         wait_mbar(smem_u32(full_bar + st), par, wc, 2, p);
       }
       if (has_ao) {
+#pragma unroll 1
         for (int j = warp; j < r; j += DS_CWARPS) {
           float acc = 0.f;
           for (int c = lane; c < ocols; c += 32) {
@@ -587,6 +612,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
     };
     // the slices of up to 8 rows at column x of the matrices named by (tmaps, proj): lane m copies row m's slice
     auto issue_row_set = [&](int p, const unsigned char* tmaps, int proj, unsigned valid8, int x) -> bool {
+#pragma unroll 1
       for (int k = 0; k < spr; ++k) {
         if (!acquire(p)) return false;
         const unsigned here = (valid8 >> (k * rps)) & ((1u << rps) - 1u);
@@ -602,6 +628,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
       }
       return true;
     };
+#pragma unroll 1
     for (int p = 0; p < a.n_phases && alive; ++p) {
       const StepPhase* ph = a.phases + p;              // immutable: read from global
       const int kind = ph->kind;
@@ -617,6 +644,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
         vA = __ballot_sync(0xffffffffu, c);
       }
       if (kind == SK_ATTN) {
+#pragma unroll 1
         for (int u = bid; u < M * a.Hkv && alive; u += G) {
           const int s = u / a.Hkv, h = u - s * a.Hkv;
           // the K/V this unit will read: asked for in L2 well ahead of the phase
@@ -641,6 +669,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
             // the o projection's A slices of the row at the unit's columns: column block cb -> slot cb
             const int ocols = (a.Hq / a.Hkv) * a.hd, nbc = ocols / TILE_N;
             const bool ok_row = (vA >> s) & 1u;
+#pragma unroll 1
             for (int c0 = 0; c0 < nbc && alive; c0 += rps) {
               if (!acquire(p)) { alive = false; break; }
               const int here = min(rps, nbc - c0);
@@ -665,16 +694,16 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
         tpu = (ph->mode == MODE_GATEUP) ? 2 : 1;
         n_units = L.NT / tpu;
         nchunks = L.nchunks;
-        bt = nstages / (L.nchunks + 4 * spr);
-        if (bt > DS_BT) bt = DS_BT;
-        if (tpu == 2) bt &= ~1;
+        bt = ds_batch_tiles(nstages, L.nchunks, spr, nseg, ph->epi != EPI_F32 ? nnext : 0, tpu);
       }
       const int my_units = (n_units > bid) ? (n_units - 1 - bid) / G + 1 : 0;
       const int my_tiles = my_units * tpu;
       const bool a_next = nnext > 0 && (kind == SK_EMBED || ph->epi != EPI_F32);
+#pragma unroll 1
       for (int b0 = 0; b0 < my_tiles && alive; b0 += bt) {
         const int nb = min(bt, my_tiles - b0);
         // (1) LoRA-B slices of the batch's tiles
+#pragma unroll 1
         for (int tl = 0; tl < nb && nseg > 0 && alive; ++tl) {
           const int ti = b0 + tl;
           const int nt = (bid + (ti / tpu) * G) * tpu + (ti % tpu);
@@ -692,17 +721,21 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
         // (2) LoRA-A slices of the consuming group at the batch's output columns
         if (a_next) {
           const int n_un = nb / tpu;
+#pragma unroll 1
           for (int ul = 0; ul < n_un && alive; ++ul) {
             const int col = (bid + (b0 / tpu + ul) * G) * TILE_N;
+#pragma unroll 1
             for (int seg = 0; seg < nnext && alive; ++seg)
               if (!issue_row_set(p, a.tmapA, ph->next_proj[seg], (vA >> (seg * 8)) & 0xffu, col)) alive = false;
           }
         }
         // (3) weight chunks of the batch's tiles
+#pragma unroll 1
         for (int tl = 0; tl < nb && kind == SK_GEMM && alive; ++tl) {
           const int ti = b0 + tl;
           const int nt = (bid + (ti / tpu) * G) * tpu + (ti % tpu);
           const unsigned char* unit = ph->w + (size_t)nt * L.unit_bytes;
+#pragma unroll 1
           for (int c = 0; c < nchunks; ++c) {
             if (!acquire(p)) { alive = false; break; }
             if (lane == 0) {
@@ -761,13 +794,8 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
         ps.n_units = ps.L.NT / ps.tpu;
         ps.ipt = (ps.L.KT + DS_ITEM_KT - 1) / DS_ITEM_KT;
         ps.gshift = (ps.L.G >= CHUNK_KT * TILE_K) ? 31 : (31 - __clz(ps.L.G / TILE_K));
-        // a batch (its slices and its tiles' chunks) must fit the ring: a warp may be a whole batch ahead of the
-        // slowest one, and a wait must never be a ring lap ahead of the fill front (mbarrier parities repeat
-        // every two laps)
-        int bt = nstages / (ps.L.nchunks + 4 * spr);
-        if (bt > DS_BT) bt = DS_BT;
-        if (ps.tpu == 2) bt &= ~1;
-        ps.bt = bt;
+        ps.bt = ds_batch_tiles(nstages, ps.L.nchunks, spr, lora_on ? ph.lora_nseg : 0,
+                               (lora_on && ph.epi != EPI_F32) ? ph.next_nseg : 0, ps.tpu);
       } else if (ph.kind == SK_EMBED) {
         ps.n_units = ph.N / TILE_N;
       }
@@ -787,6 +815,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
   };
   // every thread waits for the n_sl slice stages of the batch (they arrived long ago: one test each)
   auto wait_slices = [&](int n_sl, int p) {
+#pragma unroll 1
     for (int k = 0; k < n_sl; ++k) {
       int st; uint32_t par;
       ring_at(pos.st, pos.par, k, nstages, st, par);
@@ -824,34 +853,43 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
       if (valid && c == 0) red_add_u64(a.ssq + (size_t)ph.ssq_out * CHAIN_MAX_ROWS + m, fix_of(sq));
     }
   };
-  // partial shrink sums of the consuming group over the batch's fresh outputs (Ys): one thread per (row, segment,
-  // rank index), added straight into the fixed-point accumulators; the A slices of (unit, segment) start a_off +
-  // (unit * nseg + segment) * spr stages past the batch's first stage
+  // partial shrink sums of the consuming group over the batch's fresh outputs (Ys, values exact in fp16), on the
+  // tensor cores: warp m takes row m; per segment and block of 16 rank indices D[16 j][8 rows] = Aslice[16 j][16 columns]
+  // * Y^T[16 columns][8 rows], accumulated over the batch's units; column m of D goes into the fixed-point accumulators.
+  // The A slices of (unit, segment) start a_off + (unit * nseg + segment) * spr stages past the batch's first stage.
   auto shrink_partial = [&](const PhaseS& ps, int n_un, int a_off) {
     const int nseg = lora_on ? ps.ph.next_nseg : 0;
-    if (nseg == 0) return;
-    const int per_row = nseg * r;
-    for (int o = tid; o < M * per_row; o += DS_CTHREADS) {
-      const int m = o / per_row, sj = o - m * per_row;
-      const int seg = sj / r, j = sj - seg * r;
+    if (nseg == 0 || warp >= M) return;
+    const int m = warp, g = lane >> 2, t = lane & 3;
+#pragma unroll 1
+    for (int seg = 0; seg < nseg; ++seg) {
       if (!((ps.vA >> (seg * 8 + m)) & 1u)) continue;
-      float acc = 0.f;
-      for (int ul = 0; ul < n_un; ++ul) {
-        const uint4* ap = reinterpret_cast<const uint4*>(slice_ptr(a_off + (ul * nseg + seg) * spr, m) + j * TILE_N);
-        const float4* yp = reinterpret_cast<const float4*>(Ys + (ul * CHAIN_MAX_ROWS + m) * TILE_N);
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-          const uint4 av = ap[hh];
-          const float4 y0 = yp[2 * hh], y1 = yp[2 * hh + 1];
-          const float2 f0 = __half22float2(u32_as_h2(av.x)), f1 = __half22float2(u32_as_h2(av.y));
-          const float2 f2 = __half22float2(u32_as_h2(av.z)), f3 = __half22float2(u32_as_h2(av.w));
-          acc += y0.x * f0.x + y0.y * f0.y + y0.z * f1.x + y0.w * f1.y + y1.x * f2.x + y1.y * f2.y + y1.z * f3.x + y1.w * f3.y;
+#pragma unroll 1
+      for (int j0 = 0; j0 < r; j0 += 16) {
+        float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+        for (int ul = 0; ul < n_un; ++ul) {
+          const unsigned char* sl = reinterpret_cast<const unsigned char*>(slice_ptr(a_off + (ul * nseg + seg) * spr, m));
+          uint32_t af[4];
+          {
+            const int i = lane >> 3;
+            const int row = min(j0 + 8 * (i & 1) + (lane & 7), r - 1);     // rows past the rank: a valid row, not used
+            ds_ldmatrix_x4(af, sl + (size_t)row * 32 + (i >> 1) * 16);
+          }
+          const float* yr = Ys + (ul * CHAIN_MAX_ROWS + g) * TILE_N;        // row g of the unit's outputs
+          const float2 y0 = *reinterpret_cast<const float2*>(yr + 2 * t), y1 = *reinterpret_cast<const float2*>(yr + 2 * t + 8);
+          mma_16816(d, af, h2_as_u32(__floats2half2_rn(y0.x, y0.y)), h2_as_u32(__floats2half2_rn(y1.x, y1.y)));
+        }
+        if (t == (m >> 1)) {                                               // the lanes that hold column m of D
+          unsigned long long* dst = a.tacc + ((size_t)ps.ph.t_out * CHAIN_MAX_ROWS + m) * 3 * r + seg * r;
+          if (j0 + g < r) red_add_u64(dst + j0 + g, fix_of(d[m & 1]));
+          if (j0 + 8 + g < r) red_add_u64(dst + j0 + 8 + g, fix_of(d[2 + (m & 1)]));
         }
       }
-      red_add_u64(a.tacc + ((size_t)ps.ph.t_out * CHAIN_MAX_ROWS + m) * 3 * r + sj, fix_of(acc));
     }
   };
 
+#pragma unroll 1
   for (int p = 0; p < a.n_phases; ++p) {
     const PhaseS& ps = s_ps[p & 1];
     const StepPhase& ph = ps.ph;
@@ -897,28 +935,87 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
       const int tpu = ps.tpu, my_tiles = ps.my_tiles, bt = ps.bt, gshift = ps.gshift;
       const int it_lo = (warp * ps.ipt) / DS_CWARPS, it_hi = ((warp + 1) * ps.ipt) / DS_CWARPS;
       const int n_it = it_hi - it_lo;
-      // ---- the norm factor of the rows and the accumulated shrink sums of this group: the loads are issued here,
-      // their values go to shared memory after the first batch's main loop (nothing waits for L2 ahead of the weights)
-      unsigned long long ssq_raw = 0ull, t_raw = 0ull;
-      if (tid < M && ph.norm_in >= 0) ssq_raw = __ldcg(a.ssq + (size_t)ph.norm_in * CHAIN_MAX_ROWS + tid);
-      if (nseg > 0 && tid < M * 3 * r && ((tid / r) % 3) < nseg) t_raw = __ldcg(a.tacc + (size_t)ph.t_in * CHAIN_MAX_ROWS * 3 * r + tid);
-      // T (times the adapter's scale: the norm factor is applied to the sum of both terms) and the norm factors
-      auto settle_inputs = [&]() {
-        if (tid < CHAIN_MAX_ROWS)
-          s_inv[tid] = (ph.norm_in >= 0 && tid < M) ? rsqrtf(unfix(ssq_raw) / (float)K + a.eps) : 1.f;
-        if (nseg > 0) {
-          if (tid < M * 3 * r) Ts[tid] = unfix(t_raw) * s_scale[tid / (3 * r)];
-          for (int i = tid + DS_CTHREADS; i < M * 3 * r; i += DS_CTHREADS)
-            Ts[i] = ((i / r) % 3) < nseg ? unfix(__ldcg(a.tacc + (size_t)ph.t_in * CHAIN_MAX_ROWS * 3 * r + i)) * s_scale[i / (3 * r)] : 0.f;
+      // ---- the phase's small inputs: the sums of squares of the rows (tid < M) and, per warp w < M, the accumulated
+      // shrink sums of row w.  Their loads are issued behind the input fragments' (see gemm_tiles); the values settle in
+      // shared memory later: T (times the adapter's scale; the norm factor is applied to the sum of both terms) in the
+      // warp's own part of Ts before its first expand, the norm factors before the epilogue.
+      int b0_cur = 0;                                                     // first tile of the running batch
+      unsigned long long ssq_raw = 0ull, t_raw[2] = {0ull, 0ull};
+      const unsigned long long* t_src = a.tacc + ((size_t)ph.t_in * CHAIN_MAX_ROWS + warp) * 3 * r;
+      auto early_loads = [&]() {
+        if (b0_cur > 0) return;                                           // first batch only
+        if (tid < M && ph.norm_in >= 0) ssq_raw = __ldcg(a.ssq + (size_t)ph.norm_in * CHAIN_MAX_ROWS + tid);
+        if (nseg > 0 && warp < M) {
+          if (lane < 3 * r) t_raw[0] = __ldcg(t_src + lane);
+          if (lane + 32 < 3 * r) t_raw[1] = __ldcg(t_src + lane + 32);
         }
+      };
+      bool t_settled = false;
+      auto settle_t = [&]() {                                             // (whole warp w < M)
+        float* Tw = Ts + (size_t)warp * 3 * r;
+        const float sc = s_scale[warp];
+        if (lane < 3 * r) Tw[lane] = unfix(t_raw[0]) * sc;
+        if (lane + 32 < 3 * r) Tw[lane + 32] = unfix(t_raw[1]) * sc;
+        for (int i = lane + 64; i < 3 * r; i += 32) Tw[i] = unfix(__ldcg(t_src + i)) * sc;
+        __syncwarp();
+        t_settled = true;
+      };
+      // LoRA expand of tile tl for row m = warp (second factor of the low-rank term of Eq. 1-4) on the tensor cores:
+      // D[16 columns][8 rows] = Bslice^T[16 columns][rank] * T[rank][8 rows], T zero outside column m.  T enters as fp16
+      // value + fp16 remainder.  Column m of D (the lanes and registers that hold it) is parked in the sixteenth slot of
+      // the tile's partial sums, beside the fifteen warps' slots: the warps of the 8 rows fill disjoint parts of it.
+      auto lora_expand = [&](int tl) {
+        if (nseg == 0 || warp >= CHAIN_MAX_ROWS) return;
+        const int m = warp;
+        const int g = lane >> 2, t = lane & 3;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        float* slot15 = redf + ((size_t)(tl * 16 + 15) * 32 + lane) * 4;
+        const int ti = b0_cur + tl;
+        const int nt = (bid + (ti / tpu) * G) * tpu + (ti % tpu);
+        int seg, col;
+        map_col(ph.mode, nt * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
+        if (m >= M || seg >= nseg || !((ps.vB >> (seg * 8 + m)) & 1u)) {
+          if (t == (m >> 1)) { slot15[m & 1] = 0.f; slot15[2 + (m & 1)] = 0.f; }
+          return;
+        }
+        if (!t_settled) settle_t();
+        int st; uint32_t par;
+        ring_at(pos.st, pos.par, tl * spr + m / rps, nstages, st, par);
+        wait_mbar(smem_u32(full_bar + st), par, wc, 2, p);
+        const unsigned char* sl = ring + (size_t)st * DS_STAGE_BYTES + (size_t)(m % rps) * slot;   // [rank][16] fp16
+        const float* Tm = Ts + ((size_t)m * 3 + seg) * r;
+#pragma unroll 1
+        for (int j0 = 0; j0 < r; j0 += 16) {
+          // A fragments: (column g | g+8, rank index j0 + 2t.. | j0 + 2t+8..) = transposed 8x8 blocks of the slice
+          uint32_t af[4];
+          {
+            const int i = lane >> 3;
+            const int row = min(j0 + 8 * (i >> 1) + (lane & 7), r - 1);   // rows past the rank: a valid row, times zero
+            ds_ldmatrix_x4_trans(af, sl + (size_t)row * 32 + (i & 1) * 16);
+          }
+          float tv[4] = {0.f, 0.f, 0.f, 0.f};
+          if (g == m) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int j = j0 + 2 * t + (e & 1) + (e >> 1) * 8;
+              if (j < r) tv[e] = Tm[j];
+            }
+          }
+          const __half2 h01 = __floats2half2_rn(tv[0], tv[1]), h23 = __floats2half2_rn(tv[2], tv[3]);
+          const float2 f01 = __half22float2(h01), f23 = __half22float2(h23);
+          const __half2 l01 = __floats2half2_rn(tv[0] - f01.x, tv[1] - f01.y), l23 = __floats2half2_rn(tv[2] - f23.x, tv[3] - f23.y);
+          mma_16816(acc, af, h2_as_u32(h01), h2_as_u32(h23));
+          mma_16816(acc, af, h2_as_u32(l01), h2_as_u32(l23));
+        }
+        if (t == (m >> 1)) { slot15[m & 1] = acc[m & 1]; slot15[2 + (m & 1)] = acc[2 + (m & 1)]; }
       };
       const bool track_max = (ph.epi == EPI_F32 && ph.out_f32 == nullptr);
 
-      // the batches of the CTA's tiles; NI = work items per warp and tile (the warp's slice of the input rows takes
-      // NI * 8 registers during a batch's main loop)
-      auto run_batches = [&](auto ni_tag) {
-      constexpr int NI = decltype(ni_tag)::value;
+      // the batches of the CTA's tiles
+      const int imax = (ps.ipt + DS_CWARPS - 1) / DS_CWARPS;              // work items per warp and tile, at most
+#pragma unroll 1
       for (int b0 = 0; b0 < my_tiles; b0 += bt) {
+        b0_cur = b0;
         const int nb = min(bt, my_tiles - b0);                            // tiles in this batch
         const int n_un = nb / tpu;
         const int nB = nseg > 0 ? nb * spr : 0;                           // slice stages of the batch: B sets, then A sets
@@ -937,16 +1034,22 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
                             nb, it_lo, n_it, M, p,
                             (a.trace != nullptr && tid == 0 && b0 == 0 && (bid == 0 || bid == G - 1))
                                 ? a.trace + ((size_t)(bid == 0 ? 0 : 1) * a.n_phases + p) * 12 : nullptr};
-          gemm_tiles<NI>(gl, wc);
+          // (the warp's slice of the input rows takes 8 registers per work item during the main loop)
+          if (imax <= 3) gemm_tiles<3>(gl, wc, early_loads);
+          else gemm_tiles<6>(gl, wc, early_loads);
+#pragma unroll 1
+          for (int tl = 0; tl < nb; ++tl) lora_expand(tl);
         }
         stamp(p, 1);
-        if (b0 == 0) settle_inputs();
+        if (b0 == 0 && tid < CHAIN_MAX_ROWS)
+          s_inv[tid] = (ph.norm_in >= 0 && tid < M) ? rsqrtf(unfix(ssq_raw) / (float)K + a.eps) : 1.f;
         wait_slices(nB + nA, p);
         ds_sync();
         stamp(p, 2);
 
         // ---- epilogue: one thread per (tile or pair, row, column)
         {
+#pragma unroll 1
           for (int o = tid; o < n_un * 128; o += DS_CTHREADS) {           // (whole warps: 128 outputs per unit)
           const int ul = o >> 7, m = (o >> 4) & 7, c = o & 15;            // unit of the batch, row, column
           const bool live = m < M;
@@ -963,25 +1066,8 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
                 float y = 0.f;
 #pragma unroll
                 for (int w = 0; w < DS_CWARPS; ++w)                       // fixed order
-                  y += redf[((size_t)(tl * DS_CWARPS + w) * 32 + src_lane) * 4 + e];
-                if (nseg > 0) {
-                  const int ti = b0 + tl;
-                  const int nt = (bid + (ti / tpu) * G) * tpu + (ti % tpu);
-                  int seg, col;
-                  map_col(ph.mode, nt * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
-                  if (seg < nseg && ((ps.vB >> (seg * 8 + m)) & 1u)) {
-                    // LoRA expand (second factor of the low-rank term of Eq. 1-4)
-                    const float* Tm = Ts + ((size_t)m * 3 + seg) * r;
-                    const __half* bp = slice_ptr(tl * spr, m) + c;
-                    float s0 = 0.f, s1 = 0.f;
-#pragma unroll 4
-                    for (int j = 0; j < r; j += 2) {
-                      s0 = fmaf(Tm[j], __half2float(bp[(size_t)j * 16]), s0);
-                      s1 = fmaf(Tm[j + 1], __half2float(bp[(size_t)(j + 1) * 16]), s1);
-                    }
-                    y += s0 + s1;
-                  }
-                }
+                  y += redf[((size_t)(tl * 16 + w) * 32 + src_lane) * 4 + e];
+                if (nseg > 0) y += redf[((size_t)(tl * 16 + 15) * 32 + src_lane) * 4 + e];   // the LoRA expand term
                 yv[tu] = y * inv;
               }
             }
@@ -1029,12 +1115,6 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
           while (adv >= nstages) { adv -= nstages; pos.par ^= 1u; }
           ring_at(pos.st, pos.par, adv, nstages, pos.st, pos.par);
         }
-      }
-      };
-      {
-        const int imax = (ps.ipt + DS_CWARPS - 1) / DS_CWARPS;            // items per warp and tile, at most
-        if (imax <= 3) run_batches(std::integral_constant<int, 3>{});
-        else run_batches(std::integral_constant<int, 6>{});
       }
       if (track_max) {
         // the CTA's best (logit, lowest index) per row -> its slot of the exchange array

@@ -67,9 +67,9 @@ static __device__ __noinline__ void raise_abort(const WaitCtx& w, int where, int
                                   ((unsigned long long)(blockIdx.x & 0xffff) << 16) | (unsigned long long)(threadIdx.x & 0xffff));
   atomicExch(w.sync + 2, 1ull);
 }
-// mbarrier wait; false when the CTA is (or goes) in abort mode
-__device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const WaitCtx& w, int where, int phase) {
-  if (mbar_try_wait(bar, parity)) return true;
+// mbarrier wait; false when the CTA is (or goes) in abort mode.  The slow path is a function of its own: the waits
+// sit in many places of the persistent kernels, whose code must stay small enough for the instruction cache.
+static __device__ __noinline__ bool wait_mbar_slow(uint32_t bar, uint32_t parity, const WaitCtx& w, int where, int phase) {
   if (*w.s_abort) return false;
   const long long t0 = clock64();
   for (int it = 0;; ++it) {
@@ -80,6 +80,10 @@ __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const W
       if (clock64() - t0 > w.limit) { raise_abort(w, where, phase); return false; }
     }
   }
+}
+__device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, const WaitCtx& w, int where, int phase) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return wait_mbar_slow(bar, parity, w, where, phase);
 }
 // one thread spins until *ctr >= target
 __device__ __forceinline__ void wait_counter(const unsigned long long* ctr, unsigned long long target, const WaitCtx& w,
