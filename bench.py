@@ -291,11 +291,11 @@ def run_verify(args, cfg):
     model.close()
 
 
-def print_timeline(tl, cfg):
-    """Markdown table of one traced decode step: per phase kind, mean microseconds between the stamps of CTA 0
-    (main loop / partial sums parked / epilogue / rest of the phase / wait for the CTA / grid barrier)."""
+def print_timeline(tl, cfg, sm_mhz):
+    """Markdown table of one traced decode step: per phase kind, mean microseconds between the stamps of a CTA
+    (cycle counts of its SM, converted at the sampled SM clock)."""
     kinds = ["embed"] + ["qkv", "attention", "o", "gate_up", "down"] * cfg.n_layers + (["lm_head"] if cfg.vocab else []) + ["end"]
-    names = ["slices", "weights", "tile0", "main", "park", "epilogue", "rest", "cta_sync", "barrier"]
+    names = ["setup", "weights", "tile0", "main", "park", "epilogue", "rest", "cta_sync", "barrier"]
     agg = {}
     for cta in (0, 1):
         for p, k in enumerate(kinds):
@@ -307,18 +307,17 @@ def print_timeline(tl, cfg):
                 if st[i] == 0:
                     row.append(0.0)
                 else:
-                    row.append((st[i] - prev) / 1e3)
+                    row.append((st[i] - prev) / sm_mhz)
                     prev = st[i]
-            row.append((prev - st[0]) / 1e3)
+            row.append((prev - st[0]) / sm_mhz)
             agg.setdefault((cta, k), []).append(row)
+    print(f"(cycle stamps converted at {sm_mhz:.0f} MHz)\n")
     print("| CTA | phase | n | " + " | ".join(names) + " | total us |")
     print("|---|---|---|" + "---|" * (len(names) + 1))
     for (cta, k), rows in agg.items():
         m = np.mean(np.array(rows), axis=0)
         print(f"| {'first' if cta == 0 else 'last'} | {k} | {len(rows)} | " + " | ".join(f"{v:.2f}" for v in m) + " |")
-    t0 = min(tl[0][0][0], tl[1][0][0] or tl[0][0][0])
-    t1 = max(max(tl[0][-1]), max(tl[1][-1]))
-    print(f"\nstep (first stamp to last stamp): {(t1 - t0) / 1e3:.1f} us")
+    print(f"\nstep (global timer, first CTA): {(tl[0][-1][11] - tl[0][0][11]) / 1e3:.1f} us")
 
 
 def workload_name(cfg):
@@ -403,7 +402,14 @@ def main():
         if args.timeline:
             mb.mlora_debug_set(ctx, 7, 1)
             generation_step(W)
-            print_timeline(mb.mlora_step_timeline(ctx), cfg)
+            side.synchronize()
+            mhz = float(subprocess.run(["nvidia-smi", f"--id={local}", "--query-gpu=clocks.sm", "--format=csv,noheader,nounits"],
+                                       capture_output=True, text=True).stdout.strip() or 1965.0)
+            for i in range(200):                     # (clock sampled under load: keep the GPU busy while asking)
+                generation_step(W + 1 + i)
+            mhz = float(subprocess.run(["nvidia-smi", f"--id={local}", "--query-gpu=clocks.sm", "--format=csv,noheader,nounits"],
+                                       capture_output=True, text=True).stdout.strip() or mhz)
+            print_timeline(mb.mlora_step_timeline(ctx), cfg, mhz)
             model.close()
             return
         sampler = ClockSampler(local)

@@ -155,11 +155,14 @@ int mlora_debug_dequant(mlora_ctx* ctx, int32_t layer, int32_t proj, void* out_f
 int mlora_debug_set(mlora_ctx* ctx, int32_t key, int32_t value);
 /* Timeline of the LAST decode step that ran with debug key 7 set (Sec. 3.1 decoder: the step's phases are the
  * embedding, then q,k,v projection / attention / o projection / gate,up projection / down projection per layer,
- * then lm_head and the closing phase).  host_out receives [2][n_phases][12] nanosecond stamps of the GPU's global
- * timer, taken by the first (index 0) and the last (index 1) CTA: 0 phase start, 1 main loop (attention: the row's
- * q,k,v in shared memory) done, 2 partial sums (attention: all key tiles) done, 3 epilogue done, 4 phase work done,
- * 5 CTA at the grid barrier, 6 barrier passed, 7 adapter slices requested, 8 first weights in shared memory, 9 first
- * tile multiplied; 0 where a point does not apply.  capacity = values host_out holds (>= 24 * n_phases); *n_phases receives the phase count.  Synchronises.  Errors: ARG, STATE, CAPACITY, CUDA. */
+ * then lm_head and the closing phase).  host_out receives [2][n_phases][12] values taken by thread 0 of the first
+ * (index 0) and of the last (index 1) CTA: slots 0..9 are readings of that SM's cycle counter (only differences
+ * within one CTA mean anything): 0 phase start, 7 phase set-up done, 8 first weights in shared memory, 9 first tile
+ * multiplied, 1 main loop (attention: the row's q,k,v in shared memory) done, 2 partial sums parked (attention: all
+ * key tiles done), 3 epilogue done, 4 phase work done, 5 CTA at the grid barrier, 6 barrier passed; 0 where a point
+ * does not apply.  Slot 11 of the first phase / of the last phase holds the GPU's global nanosecond timer at the
+ * step's start / end.  capacity = values host_out holds (>= 24 * n_phases); *n_phases receives the phase count.
+ * Synchronises.  Errors: ARG, STATE, CAPACITY, CUDA. */
 int mlora_step_timeline(mlora_ctx* ctx, int64_t* host_out, int32_t capacity, int32_t* n_phases);
 /* Per-kernel-family device time of the NEXT steps, measured with CUDA events on the context's stream.
  * mlora_profile_begin switches to direct launches with an event pair around every kernel; mlora_profile_end

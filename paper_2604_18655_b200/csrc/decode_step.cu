@@ -89,6 +89,9 @@ int step_plan(int d_model, int d_ffn, int Nq, int Nkv, int hd, int rank, int lor
     if (K % TILE_K || (K / TILE_K + DS_ITEM_KT - 1) / DS_ITEM_KT > DS_MAX_ITEMS * DS_CWARPS) return 0;
   const int ot = (d_model / TILE_N + sm_count - 1) / sm_count;
   if (ot > 3) return 0;                            // a residual phase's outputs take one pass of the epilogue threads
+  // inputs too wide for one pass of three k-tiles per warp: only the down projection, and only one tile per CTA
+  const int wide = 3 * DS_CWARPS * TILE_K;
+  if (d_model > wide || Nq > wide || (d_ffn > wide && ot > 1)) return 0;
   const int r = (rank > 0 && lora_targets != 0) ? rank : 0;
   if (r % 4) return 0;                             // a row's slice (rank x 32 bytes) is a TMA destination: 128-byte aligned
   const size_t limit = 227 * 1024 - 6144;          // the kernel's static shared memory comes on top
@@ -158,13 +161,25 @@ __device__ __forceinline__ void ds_ldmatrix_x4_trans(uint32_t (&r)[4], const voi
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(smem)));
 }
-__device__ __forceinline__ void ds_stamp(const StepArgs& a, int p, int id) {
+// timeline stamp: the SM's cycle counter (cheap to read); slot 11 of the first and of the last phase also get the
+// global nanosecond timer
+static __device__ __noinline__ void ds_stamp(const StepArgs& a, int p, int id) {
   if (a.trace != nullptr && threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1)) {
-    long long tns;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tns));
-    a.trace[((size_t)(blockIdx.x == 0 ? 0 : 1) * a.n_phases + p) * 12 + id] = tns;
+    long long* e = a.trace + ((size_t)(blockIdx.x == 0 ? 0 : 1) * a.n_phases + p) * 12;
+    e[id] = clock64();
+    if ((p == 0 && id == 0) || (p == a.n_phases - 1 && id == 6)) {
+      long long tns;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tns));
+      e[11] = tns;
+    }
   }
 }
+
+// (functions of their own, to keep the kernel's code small: it is executed once per phase, from a cold instruction cache)
+static __device__ __noinline__ uint4 ds_head_piece(const float* head, int c, int hd, const float2* cs) {
+  return head_piece_f16(head, c, hd, cs);
+}
+static __device__ __noinline__ WLayout ds_wlayout(int K, int N, int G) { return make_wlayout(K, N, G); }
 
 // ----------------------------------------------------------------------------- main loop of a projection group
 struct GemmLoop {
@@ -175,32 +190,47 @@ struct GemmLoop {
   int nb, it_lo, n_it, M, phase;
   long long* tr;                       // timeline slots of this phase for this thread, or nullptr
 };
-// The warp's NI work items (two k-tiles each) of every tile of the batch.  Its slice of the input rows (mma B
-// fragments: row g of the lane, features 16t..16t+15 of each k-tile, zero past M) is loaded from L2 into registers
-// first and serves every tile of the batch.
+constexpr int DS_PASS_ITEMS = 3;       // work items whose input fragments a warp holds in registers at a time
+// The warp's work items (one k-tile each) of every tile of the batch.  Its slice of the input rows (mma B fragments:
+// row g of the lane, features 16t..16t+15 of each k-tile, zero past M) is loaded from L2 into registers first and
+// serves every tile of the batch.  A warp with more than DS_PASS_ITEMS items (wide inputs; the batch is then a single
+// tile) works in two passes: the second pass's fragments wait, copied asynchronously, in the warp's own slots of the
+// parking area, which nothing else uses before the tile is parked.
 // `early` runs right behind the issue of those loads (further loads the phase needs: one round trip for all).
-template <int NI, class Early>
+template <class Early>
 __device__ __forceinline__ void gemm_tiles(const GemmLoop& q, const WaitCtx& wc, Early early) {
-  uint4 bfr[NI][DS_ITEM_KT][2];
+  uint4 bfr[DS_PASS_ITEMS][2];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, t = lane & 3;
-  {
-    const __half* hrow = q.in16 + (size_t)g * q.K + 16 * t;
+  const __half* hrow = q.in16 + (size_t)g * q.K + 16 * t;
+  const int n_pass = q.n_it > DS_PASS_ITEMS ? 2 : 1;
+  uint4* spare = reinterpret_cast<uint4*>(q.red) + (size_t)warp * 32 + lane;     // + k * 512: the warp's slot of tile k
 #pragma unroll
-    for (int qi = 0; qi < NI; ++qi)
-#pragma unroll
-      for (int k2 = 0; k2 < DS_ITEM_KT; ++k2) {
-        const int kt = (q.it_lo + qi) * DS_ITEM_KT + k2;
-        if (qi < q.n_it && kt < q.KT && g < q.M) {
-          bfr[qi][k2][0] = __ldcg(reinterpret_cast<const uint4*>(hrow + (size_t)kt * TILE_K));
-          bfr[qi][k2][1] = __ldcg(reinterpret_cast<const uint4*>(hrow + (size_t)kt * TILE_K + 8));
-        } else {
-          bfr[qi][k2][0] = make_uint4(0, 0, 0, 0);
-          bfr[qi][k2][1] = make_uint4(0, 0, 0, 0);
-        }
-      }
-    early();
+  for (int qi = 0; qi < DS_PASS_ITEMS; ++qi) {
+    const int kt = q.it_lo + qi;
+    if (qi < q.n_it && kt < q.KT && g < q.M) {
+      bfr[qi][0] = __ldcg(reinterpret_cast<const uint4*>(hrow + (size_t)kt * TILE_K));
+      bfr[qi][1] = __ldcg(reinterpret_cast<const uint4*>(hrow + (size_t)kt * TILE_K + 8));
+    } else {
+      bfr[qi][0] = make_uint4(0, 0, 0, 0);
+      bfr[qi][1] = make_uint4(0, 0, 0, 0);
+    }
   }
+  if (n_pass > 1) {
+#pragma unroll 1
+    for (int qi = DS_PASS_ITEMS; qi < 2 * DS_PASS_ITEMS; ++qi) {
+      const int kt = q.it_lo + qi;
+      const bool live = qi < q.n_it && kt < q.KT && g < q.M;
+      const __half* src = live ? hrow + (size_t)kt * TILE_K : q.in16;
+      const uint32_t bytes = live ? 16u : 0u;                             // 0: the destination is filled with zeros
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh)
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(spare + (size_t)((qi - DS_PASS_ITEMS) * 2 + hh) * 512)),
+                     "l"(src + hh * 8), "r"(bytes) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+  early();
   int st_t = q.st_b;
   uint32_t par_t = q.par_b;
 #pragma unroll 1
@@ -209,55 +239,60 @@ __device__ __forceinline__ void gemm_tiles(const GemmLoop& q, const WaitCtx& wc,
     int c_cur = -1, st = 0, kc = 0;
     bool ok = false;
     const unsigned char* sb = nullptr;
-#pragma unroll
-    for (int qi = 0; qi < NI; ++qi) {
-      if (qi < q.n_it) {
-        const int it = q.it_lo + qi;
-        const int c = it / DS_ITEMS_PER_CHUNK, itl = it - c * DS_ITEMS_PER_CHUNK;
-        if (c != c_cur) {
-          c_cur = c;
-          st = st_t + c;
-          uint32_t par = par_t;
-          if (st >= q.nstages) { st -= q.nstages; par ^= 1u; }
-          kc = (c == q.nchunks - 1) ? q.kc_last : CHUNK_KT;
-          ok = wait_mbar(smem_u32(q.full_bar + st), par, wc, 3, q.phase);
-          sb = q.ring + (size_t)st * DS_STAGE_BYTES;
-          if (q.tr != nullptr && tl == 0 && qi == 0) { long long tns; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tns)); q.tr[8] = tns; }
-        }
-        const int ktl = itl * DS_ITEM_KT;
-        if (ok) {
-#pragma unroll
-          for (int k2 = 0; k2 < DS_ITEM_KT; ++k2) {
-            if (ktl + k2 < kc) {
-              const uint4 wv = *reinterpret_cast<const uint4*>(sb + (ktl + k2) * 512 + lane * 16);
-              const uint32_t sw = *reinterpret_cast<const uint32_t*>(sb + kc * 512 + g * 4 + ((ktl + k2) >> q.gshift) * 32);
-              __half2 s_lo, s_hi;
-              split_scales(sw, s_lo, s_hi);
-              uint32_t af[4];
-              dequant8(wv.x, s_lo, s_hi, af);
-              mma_16816(acc0, af, bfr[qi][k2][0].x, bfr[qi][k2][0].y);
-              dequant8(wv.y, s_lo, s_hi, af);
-              mma_16816(acc1, af, bfr[qi][k2][0].z, bfr[qi][k2][0].w);
-              dequant8(wv.z, s_lo, s_hi, af);
-              mma_16816(acc0, af, bfr[qi][k2][1].x, bfr[qi][k2][1].y);
-              dequant8(wv.w, s_lo, s_hi, af);
-              mma_16816(acc1, af, bfr[qi][k2][1].z, bfr[qi][k2][1].w);
-            }
-          }
-        }
+#pragma unroll 1
+    for (int pass = 0; pass < n_pass; ++pass) {
+      const int it0 = q.it_lo + pass * DS_PASS_ITEMS, n_here = min(q.n_it - pass * DS_PASS_ITEMS, DS_PASS_ITEMS);
+      if (pass == 1) {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
         __syncwarp();
-        // one arrival per item; the last item of a ragged chunk also arrives for the items the chunk lacks
-        const int items_here = (kc + DS_ITEM_KT - 1) / DS_ITEM_KT;
-        const int arrivals = (itl == items_here - 1) ? DS_ITEMS_PER_CHUNK - items_here + 1 : 1;
-        if (lane < arrivals) mbar_arrive(smem_u32(q.empty_bar + st));
+#pragma unroll
+        for (int qi = 0; qi < DS_PASS_ITEMS; ++qi) {
+          bfr[qi][0] = spare[(size_t)(qi * 2) * 512];
+          bfr[qi][1] = spare[(size_t)(qi * 2 + 1) * 512];
+        }
+      }
+#pragma unroll
+      for (int qi = 0; qi < DS_PASS_ITEMS; ++qi) {
+        if (qi < n_here) {
+          const int it = it0 + qi;
+          const int c = it / DS_ITEMS_PER_CHUNK, itl = it - c * DS_ITEMS_PER_CHUNK;
+          if (c != c_cur) {
+            c_cur = c;
+            st = st_t + c;
+            uint32_t par = par_t;
+            if (st >= q.nstages) { st -= q.nstages; par ^= 1u; }
+            kc = (c == q.nchunks - 1) ? q.kc_last : CHUNK_KT;
+            ok = wait_mbar(smem_u32(q.full_bar + st), par, wc, 3, q.phase);
+            sb = q.ring + (size_t)st * DS_STAGE_BYTES;
+            if (q.tr != nullptr && tl == 0 && pass == 0 && qi == 0) q.tr[8] = clock64();
+          }
+          if (ok && itl < kc) {
+            const uint4 wv = *reinterpret_cast<const uint4*>(sb + itl * 512 + lane * 16);
+            const uint32_t sw = *reinterpret_cast<const uint32_t*>(sb + kc * 512 + g * 4 + (itl >> q.gshift) * 32);
+            __half2 s_lo, s_hi;
+            split_scales(sw, s_lo, s_hi);
+            uint32_t af[4];
+            dequant8(wv.x, s_lo, s_hi, af);
+            mma_16816(acc0, af, bfr[qi][0].x, bfr[qi][0].y);
+            dequant8(wv.y, s_lo, s_hi, af);
+            mma_16816(acc1, af, bfr[qi][0].z, bfr[qi][0].w);
+            dequant8(wv.z, s_lo, s_hi, af);
+            mma_16816(acc0, af, bfr[qi][1].x, bfr[qi][1].y);
+            dequant8(wv.w, s_lo, s_hi, af);
+            mma_16816(acc1, af, bfr[qi][1].z, bfr[qi][1].w);
+          }
+          __syncwarp();
+          // one arrival per item; the last item of a ragged chunk also arrives for the items the chunk lacks
+          const int arrivals = (itl == kc - 1) ? DS_ITEMS_PER_CHUNK - kc + 1 : 1;
+          if (lane < arrivals) mbar_arrive(smem_u32(q.empty_bar + st));
+        }
       }
     }
     if (q.tr != nullptr && tl == 0) {
       // (the accumulators are complete when this value is: it depends on them)
-      long long tns; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tns));
-      q.tr[9] = tns + (long long)(acc0[0] != acc0[0] ? 1 : 0);
+      q.tr[9] = clock64() + (long long)(acc0[0] != acc0[0] ? 1 : 0);
     }
-    // park the tile's partial sums: [tile][warp][lane]
+    // park the tile's partial sums: [tile][slot of the warp][lane]
     q.red[(size_t)(tl * 16 + warp) * 32 + lane] =
         make_float4(acc0[0] + acc1[0], acc0[1] + acc1[1], acc0[2] + acc1[2], acc0[3] + acc1[3]);
     st_t += q.nchunks;
@@ -311,15 +346,15 @@ __device__ __forceinline__ void attn_phase(const StepArgs& a, const PhaseS& ps, 
       const int nq = g_heads * (HD / 8);
       if (tid < nq) {
         const int hq = tid / (HD / 8), c = (tid % (HD / 8)) * 8;
-        *reinterpret_cast<uint4*>(Qs + hq * HD + c) = head_piece_f16(prow + (size_t)(h * g_heads + hq) * HD, c, HD, csr);
+        *reinterpret_cast<uint4*>(Qs + hq * HD + c) = ds_head_piece(prow + (size_t)(h * g_heads + hq) * HD, c, HD, csr);
       } else if (tid < nq + HD / 8) {
         const int c = (tid - nq) * 8;
-        const uint4 v8 = head_piece_f16(prow + (size_t)(a.Hq + h) * HD, c, HD, csr);
+        const uint4 v8 = ds_head_piece(prow + (size_t)(a.Hq + h) * HD, c, HD, csr);
         *reinterpret_cast<uint4*>(Kn + c) = v8;
         *reinterpret_cast<uint4*>(ok_ + (size_t)S * HD + c) = v8;
       } else if (tid < nq + 2 * (HD / 8)) {
         const int c = (tid - nq - HD / 8) * 8;
-        const uint4 v8 = head_piece_f16(prow + (size_t)(a.Hq + Hkv + h) * HD, c, HD, nullptr);
+        const uint4 v8 = ds_head_piece(prow + (size_t)(a.Hq + Hkv + h) * HD, c, HD, nullptr);
         *reinterpret_cast<uint4*>(Vn + c) = v8;
         *reinterpret_cast<uint4*>(ov_ + (size_t)S * HD + c) = v8;
       }
@@ -690,7 +725,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
       int tpu = 1, n_units = ph->N / TILE_N, nchunks = 0, bt = DS_BT;
       WLayout L{};
       if (kind == SK_GEMM) {
-        L = make_wlayout(ph->K, ph->N, ph->G);
+        L = ds_wlayout(ph->K, ph->N, ph->G);
         tpu = (ph->mode == MODE_GATEUP) ? 2 : 1;
         n_units = L.NT / tpu;
         nchunks = L.nchunks;
@@ -789,7 +824,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
       const StepPhase& ph = ps.ph;
       ps.tpu = 1; ps.n_units = 0; ps.ipt = 0; ps.gshift = 31; ps.bt = DS_BT;
       if (ph.kind == SK_GEMM) {
-        ps.L = make_wlayout(ph.K, ph.N, ph.G);
+        ps.L = ds_wlayout(ph.K, ph.N, ph.G);
         ps.tpu = (ph.mode == MODE_GATEUP) ? 2 : 1;
         ps.n_units = ps.L.NT / ps.tpu;
         ps.ipt = (ps.L.KT + DS_ITEM_KT - 1) / DS_ITEM_KT;
@@ -1012,7 +1047,6 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
       const bool track_max = (ph.epi == EPI_F32 && ph.out_f32 == nullptr);
 
       // the batches of the CTA's tiles
-      const int imax = (ps.ipt + DS_CWARPS - 1) / DS_CWARPS;              // work items per warp and tile, at most
 #pragma unroll 1
       for (int b0 = 0; b0 < my_tiles; b0 += bt) {
         b0_cur = b0;
@@ -1034,9 +1068,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
                             nb, it_lo, n_it, M, p,
                             (a.trace != nullptr && tid == 0 && b0 == 0 && (bid == 0 || bid == G - 1))
                                 ? a.trace + ((size_t)(bid == 0 ? 0 : 1) * a.n_phases + p) * 12 : nullptr};
-          // (the warp's slice of the input rows takes 8 registers per work item during the main loop)
-          if (imax <= 3) gemm_tiles<3>(gl, wc, early_loads);
-          else gemm_tiles<6>(gl, wc, early_loads);
+          gemm_tiles(gl, wc, early_loads);
 #pragma unroll 1
           for (int tl = 0; tl < nb; ++tl) lora_expand(tl);
         }
