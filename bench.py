@@ -295,7 +295,7 @@ def print_timeline(tl, cfg, sm_mhz):
     """Markdown table of one traced decode step: per phase kind, mean microseconds between the stamps of a CTA
     (cycle counts of its SM, converted at the sampled SM clock)."""
     kinds = ["embed"] + ["qkv", "attention", "o", "gate_up", "down"] * cfg.n_layers + (["lm_head"] if cfg.vocab else []) + ["end"]
-    names = ["setup", "weights", "tile0", "main", "park", "epilogue", "rest", "cta_sync", "barrier"]
+    names = ["setup", "weights", "tile0", "tiles", "expand", "park", "epilogue", "rest", "cta_sync", "barrier"]
     agg = {}
     for cta in (0, 1):
         for p, k in enumerate(kinds):
@@ -303,17 +303,18 @@ def print_timeline(tl, cfg, sm_mhz):
             if st[0] == 0:
                 continue
             prev, row = st[0], []
-            for i in (7, 8, 9, 1, 2, 3, 4, 5, 6):
+            for i in (7, 8, 9, 10, 1, 2, 3, 4, 5, 6):
                 if st[i] == 0:
                     row.append(0.0)
                 else:
                     row.append((st[i] - prev) / sm_mhz)
                     prev = st[i]
             row.append((prev - st[0]) / sm_mhz)
+            row.append((st[0] - st[11]) / sm_mhz if (st[11] and 0 < p < len(kinds) - 1) else 0.0)   # producer's lead
             agg.setdefault((cta, k), []).append(row)
     print(f"(cycle stamps converted at {sm_mhz:.0f} MHz)\n")
-    print("| CTA | phase | n | " + " | ".join(names) + " | total us |")
-    print("|---|---|---|" + "---|" * (len(names) + 1))
+    print("| CTA | phase | n | " + " | ".join(names) + " | total us | producer lead us |")
+    print("|---|---|---|" + "---|" * (len(names) + 2))
     for (cta, k), rows in agg.items():
         m = np.mean(np.array(rows), axis=0)
         print(f"| {'first' if cta == 0 else 'last'} | {k} | {len(rows)} | " + " | ".join(f"{v:.2f}" for v in m) + " |")

@@ -158,7 +158,7 @@ int mlora_debug_set(mlora_ctx* ctx, int32_t key, int32_t value);
  * then lm_head and the closing phase).  host_out receives [2][n_phases][12] values taken by thread 0 of the first
  * (index 0) and of the last (index 1) CTA: slots 0..9 are readings of that SM's cycle counter (only differences
  * within one CTA mean anything): 0 phase start, 7 phase set-up done, 8 first weights in shared memory, 9 first tile
- * multiplied, 1 main loop (attention: the row's q,k,v in shared memory) done, 2 partial sums parked (attention: all
+ * multiplied, 10 all tiles of the first batch multiplied, 1 main loop (attention: the row's q,k,v in shared memory) done, 2 partial sums parked (attention: all
  * key tiles done), 3 epilogue done, 4 phase work done, 5 CTA at the grid barrier, 6 barrier passed; 0 where a point
  * does not apply.  Slot 11 of the first phase / of the last phase holds the GPU's global nanosecond timer at the
  * step's start / end.  capacity = values host_out holds (>= 24 * n_phases); *n_phases receives the phase count.

@@ -625,9 +625,11 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
 
   // =========================================================================== producer warp
   // The ring schedule, known to the producer and to the consumers alike.  Per projection group, per batch of the CTA's
-  // tiles: (1) the LoRA-B slices of the batch's tiles (stages_per_set stages per tile), (2) the LoRA-A slices of the
-  // consuming group at the batch's output columns (per unit and segment), (3) the weight chunks of the tiles.
-  // Embedding: (2) only.  Attention: the o projection's A slices at the unit's columns.
+  // tiles: (1) the weight chunks of the tiles, (2) the LoRA-B slices of the batch's tiles (stages_per_set stages per
+  // tile), (3) the LoRA-A slices of the consuming group at the batch's output columns (per unit and segment).  The
+  // slices come last because their stages are held until the batch's epilogue is done: the producer, which refills
+  // the ring in order, can meanwhile run on through the weight stages that the main loop has freed.
+  // Embedding: (3) only.  Attention: the o projection's A slices at the unit's columns.
   if (warp == DS_CWARPS) {
     const uint64_t policy = policy_evict_first();
     int stage = 0;
@@ -722,6 +724,8 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
         }
         continue;
       }
+      if (a.trace != nullptr && lane == 0 && p > 0 && (bid == 0 || bid == G - 1))      // when the producer reached this phase
+        a.trace[((size_t)(bid == 0 ? 0 : 1) * a.n_phases + p) * 12 + 11] = clock64();
       int tpu = 1, n_units = ph->N / TILE_N, nchunks = 0, bt = DS_BT;
       WLayout L{};
       if (kind == SK_GEMM) {
@@ -737,34 +741,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
 #pragma unroll 1
       for (int b0 = 0; b0 < my_tiles && alive; b0 += bt) {
         const int nb = min(bt, my_tiles - b0);
-        // (1) LoRA-B slices of the batch's tiles
-#pragma unroll 1
-        for (int tl = 0; tl < nb && nseg > 0 && alive; ++tl) {
-          const int ti = b0 + tl;
-          const int nt = (bid + (ti / tpu) * G) * tpu + (ti % tpu);
-          int seg = 0, col = 0;
-          if (ph->mode == MODE_PLAIN) { seg = 0; col = nt * TILE_N; }
-          else if (ph->mode == MODE_QKV) {
-            const int c = nt * TILE_N;
-            if (c < ph->seg_n0) { seg = 0; col = c; }
-            else if (c < ph->seg_n0 + ph->seg_n1) { seg = 1; col = c - ph->seg_n0; }
-            else { seg = 2; col = c - ph->seg_n0 - ph->seg_n1; }
-          } else { seg = nt & 1; col = (nt >> 1) * TILE_N; }
-          const unsigned v8 = seg < nseg ? (vB >> (seg * 8)) & 0xffu : 0u;
-          if (!issue_row_set(p, a.tmapB, ph->lora_proj[seg < 3 ? seg : 0], v8, col)) alive = false;
-        }
-        // (2) LoRA-A slices of the consuming group at the batch's output columns
-        if (a_next) {
-          const int n_un = nb / tpu;
-#pragma unroll 1
-          for (int ul = 0; ul < n_un && alive; ++ul) {
-            const int col = (bid + (b0 / tpu + ul) * G) * TILE_N;
-#pragma unroll 1
-            for (int seg = 0; seg < nnext && alive; ++seg)
-              if (!issue_row_set(p, a.tmapA, ph->next_proj[seg], (vA >> (seg * 8)) & 0xffu, col)) alive = false;
-          }
-        }
-        // (3) weight chunks of the batch's tiles
+        // (1) weight chunks of the batch's tiles
 #pragma unroll 1
         for (int tl = 0; tl < nb && kind == SK_GEMM && alive; ++tl) {
           const int ti = b0 + tl;
@@ -780,6 +757,33 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
               bulk_g2s(smem_u32(ring + (size_t)stage * DS_STAGE_BYTES), unit + (size_t)c * L.chunk_full, bytes, fb, policy);
             }
             advance();
+          }
+        }
+        // (2) LoRA-B slices of the batch's tiles
+#pragma unroll 1
+        for (int tl = 0; tl < nb && nseg > 0 && alive; ++tl) {
+          const int ti = b0 + tl;
+          const int nt = (bid + (ti / tpu) * G) * tpu + (ti % tpu);
+          int seg = 0, col = 0;
+          if (ph->mode == MODE_PLAIN) { seg = 0; col = nt * TILE_N; }
+          else if (ph->mode == MODE_QKV) {
+            const int c = nt * TILE_N;
+            if (c < ph->seg_n0) { seg = 0; col = c; }
+            else if (c < ph->seg_n0 + ph->seg_n1) { seg = 1; col = c - ph->seg_n0; }
+            else { seg = 2; col = c - ph->seg_n0 - ph->seg_n1; }
+          } else { seg = nt & 1; col = (nt >> 1) * TILE_N; }
+          const unsigned v8 = seg < nseg ? (vB >> (seg * 8)) & 0xffu : 0u;
+          if (!issue_row_set(p, a.tmapB, ph->lora_proj[seg < 3 ? seg : 0], v8, col)) alive = false;
+        }
+        // (3) LoRA-A slices of the consuming group at the batch's output columns
+        if (a_next) {
+          const int n_un = nb / tpu;
+#pragma unroll 1
+          for (int ul = 0; ul < n_un && alive; ++ul) {
+            const int col = (bid + (b0 / tpu + ul) * G) * TILE_N;
+#pragma unroll 1
+            for (int seg = 0; seg < nnext && alive; ++seg)
+              if (!issue_row_set(p, a.tmapA, ph->next_proj[seg], (vA >> (seg * 8)) & 0xffu, col)) alive = false;
           }
         }
       }
@@ -843,9 +847,10 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
 
   auto stamp = [&](int p, int id) { ds_stamp(a, p, id); };
   // address of the slice of row m in the row set that starts `off` stages past the batch's first stage
+  int sl_base = 0;                                      // stages from the batch's first stage to its first slice stage
   auto slice_ptr = [&](int off, int m) -> const __half* {
     int st; uint32_t par;
-    ring_at(pos.st, pos.par, off + m / rps, nstages, st, par);
+    ring_at(pos.st, pos.par, sl_base + off + m / rps, nstages, st, par);
     return reinterpret_cast<const __half*>(ring + (size_t)st * DS_STAGE_BYTES + (size_t)(m % rps) * slot);
   };
   // every thread waits for the n_sl slice stages of the batch (they arrived long ago: one test each)
@@ -853,7 +858,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
 #pragma unroll 1
     for (int k = 0; k < n_sl; ++k) {
       int st; uint32_t par;
-      ring_at(pos.st, pos.par, k, nstages, st, par);
+      ring_at(pos.st, pos.par, sl_base + k, nstages, st, par);
       wait_mbar(smem_u32(full_bar + st), par, wc, 2, p);
     }
   };
@@ -861,7 +866,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
   auto release_slices = [&](int n_sl) {
     if (tid < n_sl * DS_ITEMS_PER_CHUNK) {
       int st; uint32_t par;
-      ring_at(pos.st, pos.par, tid / DS_ITEMS_PER_CHUNK, nstages, st, par);
+      ring_at(pos.st, pos.par, sl_base + tid / DS_ITEMS_PER_CHUNK, nstages, st, par);
       mbar_arrive(smem_u32(empty_bar + st));
     }
   };
@@ -936,6 +941,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
       const int my_tiles = ps.my_tiles;                                  // <= own_tiles <= 3: one batch
       const int nnext = lora_on ? ph.next_nseg : 0;
       const int n_sl = my_tiles * nnext * spr;
+      sl_base = 0;
       {
         const int tl = tid >> 7, m = (tid >> 4) & 7, c = tid & 15;
         if (tl < my_tiles) {
@@ -1015,7 +1021,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
         }
         if (!t_settled) settle_t();
         int st; uint32_t par;
-        ring_at(pos.st, pos.par, tl * spr + m / rps, nstages, st, par);
+        ring_at(pos.st, pos.par, sl_base + tl * spr + m / rps, nstages, st, par);
         wait_mbar(smem_u32(full_bar + st), par, wc, 2, p);
         const unsigned char* sl = ring + (size_t)st * DS_STAGE_BYTES + (size_t)(m % rps) * slot;   // [rank][16] fp16
         const float* Tm = Ts + ((size_t)m * 3 + seg) * r;
@@ -1054,6 +1060,7 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
         const int n_un = nb / tpu;
         const int nB = nseg > 0 ? nb * spr : 0;                           // slice stages of the batch: B sets, then A sets
         const int nA = nnext > 0 ? n_un * nnext * spr : 0;
+        sl_base = nb * L.nchunks;                                         // the weight chunks come first
         // the gain of the RMSNorm that follows, for this thread's output column (used in the epilogue)
         float gpre = 1.f;
         if (ph.epi == EPI_RESID && ph.gain_next != nullptr && (tid >> 7) < nb && ((tid >> 4) & 7) < M)
@@ -1062,13 +1069,12 @@ __global__ void __launch_bounds__(DS_THREADS, 1) decode_step_kernel(const __grid
         // ---- main loop: the warp's items of every tile of the batch; a tile's partial sums are parked at once
         if (b0 == 0) stamp(p, 7);
         {
-          int st_b; uint32_t par_b;                                       // the batch's first weight chunk
-          ring_at(pos.st, pos.par, nB + nA, nstages, st_b, par_b);
-          const GemmLoop gl{ring, full_bar, empty_bar, red, ph.in16, K, L.KT, L.nchunks, L.kc_last, gshift, nstages, st_b, par_b,
+          const GemmLoop gl{ring, full_bar, empty_bar, red, ph.in16, K, L.KT, L.nchunks, L.kc_last, gshift, nstages, pos.st, pos.par,
                             nb, it_lo, n_it, M, p,
                             (a.trace != nullptr && tid == 0 && b0 == 0 && (bid == 0 || bid == G - 1))
                                 ? a.trace + ((size_t)(bid == 0 ? 0 : 1) * a.n_phases + p) * 12 : nullptr};
           gemm_tiles(gl, wc, early_loads);
+          if (b0 == 0) stamp(p, 10);
 #pragma unroll 1
           for (int tl = 0; tl < nb; ++tl) lora_expand(tl);
         }
