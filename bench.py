@@ -401,6 +401,7 @@ def main():
         for i in range(W):
             generation_step(i)
         if args.timeline:
+            mb.mlora_debug_set(ctx, 6, 2)
             mb.mlora_debug_set(ctx, 7, 1)
             generation_step(W)
             side.synchronize()

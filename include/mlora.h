@@ -144,13 +144,10 @@ int mlora_debug_dequant(mlora_ctx* ctx, int32_t layer, int32_t proj, void* out_f
  * the pass wrote them: rows suffix_len .. suffix_len + n_nodes - 1 of the own segment).
  * key 2 = 1 disables CUDA-graph replay of steps (every kernel launched directly).
  * key 3 = 1 runs decode-sized passes through the one-kernel-per-projection path instead of the persistent kernels.
- * key 6 = 1 runs decode steps through the per-layer persistent projection kernel plus attention kernels (replayed
- *         from a CUDA graph) instead of the single kernel that does the whole step.
- * key 4 = 1 runs passes of 32 rows or more on the split-K mma.sync GEMM instead of the tcgen05 one.
- * key 5 = 1 (test hook for the bounded waits) makes the NEXT decode-sized pass wait, with a limit of about 0.1 s,
- *         at a grid barrier for an arrival nobody makes: the pass ends with garbage outputs and the device status
- *         MLORA_ERR_TIMEOUT; mlora_sync_status reports and clears it, after which the context works again
- *         (run mlora_prefill_shared or mlora_reset_streams to drop the garbage rows).
+ * key 6 picks the path of decode steps (one row per stream, at most 8 streams): 1 = the per-layer persistent projection
+ *         kernel plus attention kernels, replayed from a CUDA graph; 2 = ONE kernel that does the whole step (embedding to
+ *         greedy token; where the model's shapes allow it, else the per-layer path); 0 = the library's choice
+ *         (currently the per-layer path, the faster of the two at the 1B / 8-stream shapes).
  * key 7 = 1 makes the single-kernel decode step record a timeline (see mlora_step_timeline). */
 int mlora_debug_set(mlora_ctx* ctx, int32_t key, int32_t value);
 /* Timeline of the LAST decode step that ran with debug key 7 set (Sec. 3.1 decoder: the step's phases are the

@@ -95,7 +95,8 @@ struct mlora_ctx {
   cudaEvent_t snap_event = nullptr;
   bool snap_pending = false;
   int snap_inc = 0;
-  int dbg_skip_compact = 0, dbg_no_graph = 0, dbg_no_chain = 0, dbg_no_tc = 0, dbg_inject_stall = 0, dbg_no_step = 0;
+  int dbg_skip_compact = 0, dbg_no_graph = 0, dbg_no_chain = 0, dbg_no_tc = 0, dbg_inject_stall = 0;
+  int step_mode = 0;                 // decode steps: 0 = the library's choice, 1 = per-layer kernels, 2 = the single-kernel step
   int32_t* host_io = nullptr;        // dev [3][max_streams]: adapter_idx, tokens, next of the host-buffer step
   // persistent projection chain (rows <= 8)
   ChainPhase* phases = nullptr;      // dev [4*L (+1)]: qkv, o, gate/up, down per layer; then lm_head
@@ -240,7 +241,8 @@ bool chain_eligible(const mlora_ctx* c, const PassIO& io) {
 
 // a decode step (one row per stream) that the single-kernel path can take
 bool step_eligible(const mlora_ctx* c, int n, int T) {
-  return c->step_stages > 0 && !c->dbg_no_chain && !c->dbg_no_step && T == 1 && n <= CHAIN_MAX_ROWS;
+  // (the library's own choice is the per-layer path: at the 1B / 8-stream shapes it is the faster of the two)
+  return c->step_stages > 0 && !c->dbg_no_chain && c->step_mode == 2 && T == 1 && n <= CHAIN_MAX_ROWS;
 }
 
 // one decode step as one persistent kernel: embedding to greedy token (or hidden state), suffix lengths advanced
@@ -1179,7 +1181,7 @@ int mlora_debug_set(mlora_ctx* c, int32_t key, int32_t value) {
   else if (key == 3) c->dbg_no_chain = value ? 1 : 0;
   else if (key == 4) c->dbg_no_tc = value ? 1 : 0;
   else if (key == 5) c->dbg_inject_stall = value ? 1 : 0;
-  else if (key == 6) c->dbg_no_step = value ? 1 : 0;
+  else if (key == 6) c->step_mode = (value >= 0 && value <= 2) ? value : 0;
   else if (key == 7) c->dbg_trace = value ? 1 : 0;
   else return fail(MLORA_ERR_ARG, "unknown debug key");
   return MLORA_OK;

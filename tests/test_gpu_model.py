@@ -21,10 +21,17 @@ def GpuModel():
     return G
 
 
-def make_pair(GpuModel, cfg, seed=0, **kw):
+# decode-step paths of the library (debug switch 6): per-layer kernels, or one kernel for the whole step
+STEP_PATHS = [pytest.param(1, id="per_layer_kernels"), pytest.param(2, id="single_kernel_step")]
+
+
+def make_pair(GpuModel, cfg, seed=0, step_path=0, **kw):
+    from paper_2604_18655_b200 import binding as mb
     m = gen.make_model(cfg, seed)
     orc = ref.OracleModel.from_synth(m)
     gm = GpuModel(m, **kw)
+    if step_path:
+        mb.mlora_debug_set(gm.ctx, 6, step_path)
     for a in range(cfg.n_adapters):
         A, B = gen.make_adapter(cfg, a, seed)
         orc.set_adapter(a, A, B, cfg.alpha)
@@ -45,9 +52,10 @@ def compare_kv(gm, orc, cfg, n_streams):
     mb.mlora_sync_status(gm.ctx)
 
 
-def test_cfg0_hidden_state_decode(GpuModel):
+@pytest.mark.parametrize("step_path", STEP_PATHS)
+def test_cfg0_hidden_state_decode(GpuModel, step_path):
     cfg = gen.CFG0
-    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=8)
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=8, step_path=step_path)
     prompt = gen.make_hidden(cfg, cfg.prompt_len, 0, 0)
     want_last = orc.prefill_shared(hidden=prompt)
     got_last = gm.prefill_h(prompt)
@@ -81,9 +89,10 @@ def test_prefill_ragged_causal_chunks(GpuModel):
     gm.close()
 
 
-def test_prefill_logits_and_follow_mode_decode(GpuModel):
+@pytest.mark.parametrize("step_path", STEP_PATHS)
+def test_prefill_logits_and_follow_mode_decode(GpuModel, step_path):
     cfg = TINYV
-    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=32)
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=32, step_path=step_path)
     ids = gen.make_prompt_ids(cfg, 0)
     compare(gm.prefill(ids), orc.prefill_shared(ids), "prefill logits")
     ad = [0, 2, -1]
@@ -100,12 +109,13 @@ def test_prefill_logits_and_follow_mode_decode(GpuModel):
     gm.close()
 
 
-def test_decode_long_weight_streams(GpuModel):
+@pytest.mark.parametrize("step_path", STEP_PATHS)
+def test_decode_long_weight_streams(GpuModel, step_path):
     """A vocabulary and an FFN wide enough that one CTA's weight chunks of a projection wrap the shared-memory
     ring of the persistent kernel several times (the tiny models never do), 8 streams, rank-16 adapters."""
     from paper_2604_18655_b200 import binding as mb
     cfg = gen.ModelCfg("widev", 1, 256, 4, 2, 64, 2816, 32000, 128, 16, 127, 8, 8, 40, b_std=0.05)
-    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16, step_path=step_path)
     ids = gen.make_prompt_ids(cfg, 0)
     gm.prefill(ids)
     orc.prefill_shared(ids)
@@ -122,10 +132,11 @@ def test_decode_long_weight_streams(GpuModel):
     gm.close()
 
 
-def test_adapter_switch_without_recreate(GpuModel):
+@pytest.mark.parametrize("step_path", STEP_PATHS)
+def test_adapter_switch_without_recreate(GpuModel, step_path):
     """Adapters are run-time inputs: swapping a slot's tensors changes the next step, clearing gives the base."""
     cfg = TINYV
-    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=32)
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=32, step_path=step_path)
     ids = gen.make_prompt_ids(cfg, 0)
     gm.prefill(ids)
     orc.prefill_shared(ids)
@@ -311,7 +322,7 @@ def test_graph_replay_matches_direct_launches(GpuModel):
     for no_graph in (1, 0):
         with torch.cuda.stream(side):
             m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
-            mb.mlora_debug_set(gm.ctx, 6, 1)
+            mb.mlora_debug_set(gm.ctx, 6, 1)                 # the multi-kernel path
             mb.mlora_debug_set(gm.ctx, 2, no_graph)
             gm.prefill(gen.make_prompt_ids(cfg, 0))
             dev = torch.device("cuda")
@@ -340,6 +351,7 @@ def test_step_kernel_is_one_launch_and_bit_reproducible(GpuModel):
     res = []
     for rep in range(2):
         m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+        mb.mlora_debug_set(gm.ctx, 6, 2)                     # the single-kernel step
         gm.prefill(gen.make_prompt_ids(cfg, 0))
         toks = np.array([1, 2, 3], dtype=np.int32)
         hist = []
@@ -360,10 +372,9 @@ def test_decode_paths_agree(GpuModel):
     from paper_2604_18655_b200 import binding as mb
     cfg = TINYV
     res = []
-    for key in (0, 6, 3):
+    for key, val in ((6, 2), (6, 1), (3, 1)):
         m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
-        if key:
-            mb.mlora_debug_set(gm.ctx, key, 1)
+        mb.mlora_debug_set(gm.ctx, key, val)
         gm.prefill(gen.make_prompt_ids(cfg, 0))
         toks = np.array([1, 2, 3], dtype=np.int32)
         hist = []
@@ -406,13 +417,14 @@ def test_host_buffer_step_matches_device_step(GpuModel):
     assert np.array_equal(outs[0], outs[1])
 
 
-def test_bounded_wait_runs_out_and_context_recovers(GpuModel):
+@pytest.mark.parametrize("step_path", STEP_PATHS)
+def test_bounded_wait_runs_out_and_context_recovers(GpuModel, step_path):
     """Failure detection without a fault: a grid barrier of the persistent kernel is made to wait (limit ~0.1 s) for an
     arrival nobody makes.  The kernel must return, the device status must say TIMEOUT and name the wait, and after
     mlora_sync_status the same context must compute the same logits as before."""
     from paper_2604_18655_b200 import binding as mb
     cfg = TINYV
-    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16, step_path=step_path)
     ids = gen.make_prompt_ids(cfg, 0)
     toks = np.array([1, 2, 3], dtype=np.int32)
     gm.prefill(ids)

@@ -16,11 +16,11 @@ pytestmark = pytest.mark.gpu
 PROMPT = 64
 
 
-def build(cfg, max_tree):
+def build(cfg, max_tree, prompt=PROMPT, max_suffix=None):
     from tests.helpers import GpuModel
     m = gen.make_model(cfg, 0)
     orc = ref.OracleModel.from_synth(m, dtype=np.float32)
-    gm = GpuModel(m, max_prefix=PROMPT, max_suffix=8 + 3 * max_tree, max_tree=max_tree)
+    gm = GpuModel(m, max_prefix=prompt, max_suffix=max_suffix or 8 + 3 * max_tree, max_tree=max_tree)
     for a in range(cfg.n_adapters):
         A, B = gen.make_adapter(cfg, a, 0)
         orc.set_adapter(a, A, B, cfg.alpha)
@@ -28,13 +28,14 @@ def build(cfg, max_tree):
     return m, orc, gm
 
 
-def run_decode_and_verify(cfg, n_decode, branch, T):
+def run_decode_and_verify(cfg, n_decode, branch, T, step_path=0):
     from paper_2604_18655_b200 import binding as mb
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     side = torch.cuda.Stream()                       # graph replay needs a capturable stream, as in bench.py
     with torch.cuda.stream(side):
         m, orc, gm = build(cfg, T)
+        mb.mlora_debug_set(gm.ctx, 6, step_path)
         ids = gen.make_prompt_ids(cfg, 0, PROMPT)
         got_last = gm.prefill(ids)
         want_last = orc.prefill_shared(ids, n_streams=cfg.n_streams)
@@ -75,6 +76,45 @@ def run_decode_and_verify(cfg, n_decode, branch, T):
 
 def test_llama1b_full_depth_decode_and_verify():
     run_decode_and_verify(gen.CFG1, n_decode=3, branch=(4, 2, 2), T=16)
+
+
+def test_llama1b_full_depth_single_kernel_step():
+    """The same workload with decode steps through the kernel that does a whole step in one launch."""
+    run_decode_and_verify(gen.CFG1, n_decode=3, branch=(4, 2, 2), T=16, step_path=2)
+
+
+@pytest.mark.parametrize("step_path", [1, 2])
+def test_llama1b_full_prompt_sixteen_steps(step_path):
+    """The benchmark workload itself: the full 512-token shared prompt, 8 streams, 16 greedy decode steps in follow
+    mode (the oracle walks on the GPU's tokens), logits of every step against the oracle, own-segment KV at the end."""
+    from paper_2604_18655_b200 import binding as mb
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    cfg = gen.CFG1
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        m, orc, gm = build(cfg, 1, prompt=cfg.prompt_len, max_suffix=24)
+        mb.mlora_debug_set(gm.ctx, 6, step_path)
+        ids = gen.make_prompt_ids(cfg, 0)
+        got_last = gm.prefill(ids)
+        want_last = orc.prefill_shared(ids, n_streams=cfg.n_streams)
+        compare(got_last, want_last, "llama1b prefill logits, 512 tokens")
+        n = cfg.n_streams
+        ad = list(range(n))
+        toks = np.argsort(-want_last)[:n].astype(np.int32)
+        for step in range(16):
+            nxt, logits = gm.decode(ad, toks)
+            r = orc.decode_step(ad, tokens=toks)
+            compare(logits, r["logits"], f"llama1b full-prompt decode logits step {step}")
+            check_argmax(nxt, r["logits"], f"llama1b full-prompt decode step {step}")
+            toks = nxt
+        for s in (0, n - 1):
+            got_s, k, v = gm.export_kv(cfg.n_layers - 1, s, 0, 16)
+            assert got_s == 16
+            compare(k, orc.suf_k[cfg.n_layers - 1][s], f"suffix K stream {s}")
+            compare(v, orc.suf_v[cfg.n_layers - 1][s], f"suffix V stream {s}")
+        mb.mlora_sync_status(gm.ctx)
+        gm.close()
 
 
 def test_llama3b_widths_two_layers_decode_and_verify():
