@@ -7,6 +7,9 @@ decoding in generations of 128 steps per stream.  One "step" = one mlora_decode_
 (8 tokens).  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+  python bench.py --config cfg2|cfg3        DS2D verify rounds (8 streams x 16- or 32-node trees), same line shape
+  python bench.py --config cfg4 [--quick]   kernel-level sweep of the single projection and of tree attention
+  python bench.py --timeline                phase timeline of the single-kernel decode step (markdown)
 
 With N > 1 (torchrun) every rank runs an independent replica of the same job: the path has no exchange
 step, so there is no collective on the data path ("replicas only").
@@ -26,11 +29,10 @@ sys.path.insert(0, ROOT)
 
 GEN_STEPS = 128          # decode steps per generation (per stream) before the streams are reset
 ORACLE_PREFIX = 64       # prompt length used for the CPU-baseline sample (the 512-token prefill is not timed work)
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of decode_chain_kernel, averaged over the 17 launches of
-# a full-model step, from the ncu capture summarised in profiles/decode_chain_kernel_llama1b_cut4L_8streams.md
-# (32.8 MB of weights, adapters and activations plus 2.1 MB of K/V that the kernel prefetches into L2 for the
-# attention kernel that follows it)
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = 34.8e6
+L2_BYTES = 126e6
+# DRAM bytes (read + write counters of one ncu capture) per launch of the dominant kernel, by workload; None where
+# no capture of the kernel as it stands exists
+NCU_DRAM_BYTES_PER_LAUNCH = {"cfg1": None}
 
 
 def parse_args():
@@ -39,8 +41,11 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="cfg1", choices=["cfg0", "cfg1", "cfg2", "cfg3"],
-                    help="cfg1 (default) is the benchmark workload; cfg2/cfg3 time DS2D verify rounds (side measurement)")
+    ap.add_argument("--config", default="cfg1", choices=["cfg0", "cfg1", "cfg2", "cfg3", "cfg4"],
+                    help="cfg1 (default) is the benchmark workload; cfg2/cfg3 time DS2D verify rounds; cfg4 is the "
+                         "kernel-level sweep (one JSON line with a list of points; --markdown prints tables)")
+    ap.add_argument("--quick", action="store_true", help="cfg4: a small sub-grid")
+    ap.add_argument("--markdown", action="store_true", help="cfg4: markdown tables instead of the JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--timeline", action="store_true",
                     help="profiling aid: print the phase timeline of one traced decode step (markdown) instead of the bench line")
@@ -49,15 +54,16 @@ def parse_args():
     return ap.parse_args()
 
 
-def peaks():
+def peaks(key="hbm_gbs"):
+    """(peak, "measured" | "fallback") for hbm_gbs (GB/s), bf16_tflops or bf16_tflops_sustained (TFLOP/s)."""
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         try:
             j = json.load(open(p))
-            return float(j["hbm_gbs"]), "measured"
+            return float(j[key]), "measured"
         except Exception:
             pass
-    return 6650.0, "fallback"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}[key], "fallback"
 
 
 class ClockSampler:
@@ -206,37 +212,81 @@ def run_reference(args, cfg):
     K = args.steps if args.steps is not None else 6
     W = args.warmup if args.warmup is not None else 3
     synth, adapters = build_inputs(cfg)
-    # bound the run to a few minutes whatever K is: past 40 steps, time 40 and report the per-step mean
-    k_run = min(K + W, 40)
-    tps, dt, desc = oracle_sample(cfg, synth, adapters, k_run)
+    if cfg.tree_nodes > 1:
+        # verify passes: a handful at most (a pass of the ~3B model is tens of seconds of CPU work)
+        k_run = min(K + W, 3 if cfg.d_model <= 2048 else 1)
+        val, dt, desc = oracle_verify_sample(cfg, synth, adapters, k_run)
+        metric, unit = "DS2D verify rows/s", "rows/s"
+    else:
+        # bound the run to a few minutes whatever K is: past 40 steps, time 40 and report the per-step mean
+        k_run = min(K + W, 40)
+        val, dt, desc = oracle_sample(cfg, synth, adapters, k_run)
+        metric, unit = "aggregate decode tokens/s over streams", "tokens/s"
     ms = 1000.0 * dt / k_run
     line = {
-        "impl": "reference", "metric": "aggregate decode tokens/s over streams", "value": tps, "unit": "tokens/s",
+        "impl": "reference", "metric": metric, "value": val, "unit": unit,
         "n_gpus": args.gpus, "steps": K, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": workload_name(cfg), "note": "CPU oracle on host cores; rank 0 only"},
-        "cpu_baseline": {"value": tps, "unit": "tokens/s", "cores": cores_used(), "kind": "oracle", "sample": desc},
-        "e2e": {"value": tps, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "cpu_baseline": {"value": val, "unit": unit, "cores": cores_used(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
 
 
+def oracle_verify_sample(cfg, synth, adapters, n_rounds):
+    """Times the CPU oracle, as it stands, on n_rounds DS2D verify passes (all streams' trees in one pass) after a
+    short prefill.  Returns (rows_per_s, seconds, description)."""
+    import gen
+    from oracle import ref
+    orc = ref.OracleModel.from_synth(synth, dtype=np.float32)
+    for a, (A, B) in enumerate(adapters):
+        orc.set_adapter(a, A, B, cfg.alpha)
+    n, T = cfg.n_streams, cfg.tree_nodes
+    orc.prefill_shared(gen.make_prompt_ids(cfg, 0, ORACLE_PREFIX), n_streams=n)
+    ad = list(range(n))
+    parents = np.stack([gen.build_tree(cfg.branch, T)] * n)
+    cand = gen.make_candidates(cfg, n_rounds + 1, n, T, 0)
+    tt = np.empty((n, T), dtype=np.int32)
+    nxt = np.arange(n, dtype=np.int32) + 1
+    dt = 0.0
+    for i in range(n_rounds + 1):                   # the first, untimed pass also pays the lazy dequantisation
+        tt[:, 0] = nxt
+        tt[:, 1:] = cand[i]
+        t0 = time.perf_counter()
+        nxt = orc.verify_tree(ad, parents, tt)["next"]
+        if i:
+            dt += time.perf_counter() - t0
+    desc = (f"{n_rounds} verify passes of {n} streams x {T}-node trees of {cfg.name} after a {ORACLE_PREFIX}-token "
+            f"prefill (numpy fp32, dense dequantised weights)")
+    return n * T * n_rounds / dt, dt, desc
+
+
 def run_verify(args, cfg):
-    """Side measurement: DS2D verify rounds (8 streams x tree_nodes rows per pass, uniform-random draft ids, so about
-    one token is accepted per stream and round).  One JSON line: rows/s verified and tokens/s emitted."""
+    """DS2D verify rounds (Sec. 3.5): 8 streams x tree_nodes rows per pass, uniform-random draft ids (so about one
+    token is accepted per stream and round).  One step = one verify pass + accept walk + KV compaction.  One JSON line
+    of the same shape as the decode benchmark's: rows/s verified, with the tokens/s emitted beside it."""
     import torch
     import gen
     from paper_2604_18655_b200 import binding as mb
     from paper_2604_18655_b200.runtime import MloraModel
     K = args.steps if args.steps is not None else 64
     W = max(args.warmup if args.warmup is not None else 8, 3)
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
     side = torch.cuda.Stream()
     synth, adapters = build_inputs(cfg)
     n, T = cfg.n_streams, cfg.tree_nodes
+    Ke = min(K, 64)
+    ROUNDS_PER_GEN = 32                              # streams restart (own segments emptied) every so many rounds
     with torch.cuda.stream(side):
-        model = MloraModel(synth, max_suffix=(K + W + 8) * 4 + 8, max_tree=T)
+        model = MloraModel(synth, max_suffix=ROUNDS_PER_GEN * T + 8, max_tree=T)
         for a, (A, B) in enumerate(adapters):
             model.set_adapter(a, A, B, cfg.alpha)
         ctx = model.ctx
@@ -248,47 +298,272 @@ def run_verify(args, cfg):
         tt = torch.empty(n, T, dtype=torch.int32, device=dev)
         acc_len = torch.empty(n, dtype=torch.int32, device=dev)
         acc_idx = torch.empty(n, T, dtype=torch.int32, device=dev)
-        nxt = torch.topk(last, n).indices.to(torch.int32)
+        first = torch.topk(last, n).indices.to(torch.int32)
+        nxt = first.clone()
         ad = torch.arange(n, dtype=torch.int32, device=dev)
         emitted = torch.zeros(1, dtype=torch.int64, device=dev)
 
         def round_(i):
+            if i % ROUNDS_PER_GEN == 0:
+                mb.mlora_reset_streams(ctx)
+                nxt.copy_(first)
             tt[:, 0] = nxt
             tt[:, 1:] = cand[i % 64]
             mb.mlora_verify_tree(ctx, ad, tt, parent, acc_len, acc_idx, nxt, None)
             emitted.add_(acc_len.sum())
 
+        def barrier():
+            if world > 1:
+                torch.distributed.barrier()
+            torch.cuda.synchronize()
+
         for i in range(W):
             round_(i)
         emitted.zero_()
+        sampler = ClockSampler(local)
+        sampler.start()
+        barrier()
+        l0 = mb.mlora_launch_count(ctx)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        side.synchronize()
+        t0 = time.time()
         e0.record(side)
         for i in range(K):
             round_(W + i)
         e1.record(side)
-        side.synchronize()
-        ms = e0.elapsed_time(e1) / K
+        barrier()
+        clocks = sampler.stop(t0, time.time())
+        ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / K
+        launches = mb.mlora_launch_count(ctx) - l0
         tokens = int(emitted.item())
-        mb.mlora_profile_begin(ctx)
+
+        # ---- end to end: the round's trees come from pinned host memory, its results go back to the host
+        h_tt = torch.empty(n, T, dtype=torch.int32).pin_memory()
+        h_cand = cand.cpu()
+        h_len = torch.empty(n, dtype=torch.int32).pin_memory()
+        h_idx = torch.empty(n, T, dtype=torch.int32).pin_memory()
+        h_next = torch.empty(n, dtype=torch.int32).pin_memory()
+        h_next.copy_(first.cpu())
+        h_first = first.cpu()
+
+        def e2e_round(i):
+            if i % ROUNDS_PER_GEN == 0:
+                mb.mlora_reset_streams(ctx)
+                h_next.copy_(h_first)
+            h_tt[:, 0] = h_next
+            h_tt[:, 1:] = h_cand[i % 64]
+            tt.copy_(h_tt, non_blocking=True)
+            mb.mlora_verify_tree(ctx, ad, tt, parent, acc_len, acc_idx, nxt, None)
+            h_len.copy_(acc_len, non_blocking=True)
+            h_idx.copy_(acc_idx, non_blocking=True)
+            h_next.copy_(nxt, non_blocking=True)
+            side.synchronize()                       # the host reads the accepted path before it drafts the next tree
+
         for i in range(4):
-            round_(W + K + i)
+            e2e_round(i)
+        barrier()
+        e0.record(side)
+        for i in range(Ke):
+            e2e_round(4 + i)
+        e1.record(side)
+        barrier()
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev) / Ke
+
+        mb.mlora_profile_begin(ctx)
+        prof_rounds = 4
+        for i in range(prof_rounds):
+            round_(1 + i)
         prof = mb.mlora_profile_end(ctx)
         mb.mlora_sync_status(ctx)
+    rows = n * T
     params = sum(gen.proj_shape(cfg, p)[0] * gen.proj_shape(cfg, p)[1] for p in gen.PROJ_NAMES) * cfg.n_layers + \
         cfg.d_model * cfg.vocab
+    flops_pass = 2.0 * rows * params                 # the projections' dense contraction (LoRA terms and attention not counted)
+    gemm_ms, gemm_launches = prof["gemm"]
+    peak, peak_kind = peaks("bf16_tflops_sustained")
+    achieved = flops_pass * prof_rounds / (gemm_ms / 1e3) / 1e12
+    attn_ms = prof["attn"][0] + prof["attn_merge"][0]
+    attn_flops = 4.0 * rows * cfg.n_q_heads * cfg.head_dim * (cfg.prompt_len + T) * cfg.n_layers
     line = {
-        "metric": "DS2D verify rows/s", "value": n * T / (ms / 1e3), "unit": "rows/s", "n_gpus": 1, "steps": K, "warmup": W,
-        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
+        "metric": "DS2D verify rows/s", "value": world * rows / (ms / 1e3), "unit": "rows/s", "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
         "data": "synthetic",
-        "config": {"workload": f"{cfg.name}: {n} streams x {T}-node trees {cfg.branch}, prompt {cfg.prompt_len}, "
-                               f"rank-{cfg.lora_rank} LoRA, uniform-random drafts", "rows_per_pass": n * T},
-        "tokens_per_s": tokens / (ms * K / 1e3), "tokens_per_round": tokens / K,
-        "gemm_tflops": 2.0 * n * T * params / (ms / 1e3) / 1e12,
-        "family_us_per_step": {k: 1e3 * v[0] / 4 for k, v in prof.items()},
+        "config": {"workload": f"{cfg.name}: d{cfg.d_model} L{cfg.n_layers} hd{cfg.head_dim} int4-g{cfg.group_size}; {n} streams x "
+                               f"{T}-node trees {cfg.branch}, shared prompt {cfg.prompt_len}, rank-{cfg.lora_rank} LoRA, "
+                               f"uniform-random drafts, streams restart every {ROUNDS_PER_GEN} rounds",
+                   "rows_per_pass": rows, "l2": "inputs larger than L2 (weights alone: %.0f MB)" % (params / 2e6),
+                   "launch": "CUDA-graph replay per pass", "multi_gpu": "replicas only"},
+        "clocks": clocks,
+        "e2e": {"value": world * rows / (ms_e2e / 1e3), "unit": "rows/s", "h2d_bytes_per_step": rows * 4,
+                "d2h_bytes_per_step": (n + rows + n) * 4, "steps": Ke, "ms_per_step": ms_e2e},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "kernel": "w4_gemm_tc_kernel (tcgen05 INT4 projection with its split-K epilogue), "
+                     "all launches of a pass", "achieved": achieved, "peak": peak,
+                     "peak_kind": "of " + peak_kind + " (bf16 sustained; fp16 has the same nominal rate)", "unit": "TFLOP/s",
+                     "frac": achieved / peak, "traffic": None, "flops_per_pass": flops_pass,
+                     "launches_per_pass": gemm_launches / prof_rounds, "us_per_pass": 1e3 * gemm_ms / prof_rounds},
+        "roofline_attention": {"bound": "tensor", "kernel": "tree attention (+ merge)", "achieved": attn_flops * prof_rounds / (attn_ms / 1e3) / 1e12
+                               if attn_ms > 0 else None, "peak": peak, "unit": "TFLOP/s",
+                               "frac": (attn_flops * prof_rounds / (attn_ms / 1e3) / 1e12 / peak) if attn_ms > 0 else None,
+                               "us_per_pass": 1e3 * attn_ms / prof_rounds},
+        "tokens_per_s": world * tokens / (ms * K / 1e3), "tokens_per_round": tokens / K,
+        "family_us_per_step": {k: 1e3 * v[0] / prof_rounds for k, v in prof.items()},
     }
-    print(json.dumps(line), flush=True)
+    if rank == 0 and not args.no_cpu_baseline:
+        n_or = 3 if cfg.d_model <= 2048 else 1
+        rps, dt, desc = oracle_verify_sample(cfg, synth, adapters, n_or)
+        line["cpu_baseline"] = {"value": rps, "unit": "rows/s", "cores": cores_used(), "kind": "oracle", "sample": desc,
+                                "seconds": dt}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
     model.close()
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def time_graph(stream, body, reps):
+    """Captures body() once into a CUDA graph on `stream`, replays it `reps` times; returns ms per replay."""
+    import torch
+    body()                                   # direct run first (first-use set-up stays out of the capture)
+    stream.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        body()
+    for _ in range(3):
+        g.replay()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    stream.synchronize()
+    e0.record(stream)
+    for _ in range(reps):
+        g.replay()
+    e1.record(stream)
+    stream.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def sweep_linear(stream, shapes, Ms, combos, peak):
+    """mlora_linear over K x N, rows and (adapters, rank): each point a graph of back-to-back launches that cycle
+    through enough copies of the weights to exceed the L2.  Algorithmic bytes: every nibble, scale, referenced adapter
+    element, activation and result once."""
+    import torch
+    import gen
+    from paper_2604_18655_b200 import binding as mb
+    pts = []
+    rng = np.random.default_rng(0)
+    for K, N in shapes:
+        G = 128
+        w_bytes = K * N // 2 + (K // G) * N * 2
+        n_copies = int(L2_BYTES // w_bytes) + 2
+        qb, sc = gen.quantize_int4(rng.standard_normal((K, N)).astype(np.float32) * 0.02, G)
+        dq, ds = torch.from_numpy(qb).cuda(), torch.from_numpy(sc).cuda()
+        ws_ = [mb.mlora_weight_create(dq, ds, K, N, G) for _ in range(n_copies)]
+        for n_ad, rank in combos:
+            A = [torch.randn(rank, K, device="cuda", dtype=torch.float16) / rank for _ in range(n_ad)]
+            B = [torch.randn(rank, N, device="cuda", dtype=torch.float16) * 0.05 for _ in range(n_ad)]
+            pa = torch.tensor([t.data_ptr() for t in A], dtype=torch.int64, device="cuda")
+            pb = torch.tensor([t.data_ptr() for t in B], dtype=torch.int64, device="cuda")
+            scale = torch.full((max(n_ad, 1),), 16.0 / max(rank, 1), device="cuda")
+            for M in Ms:
+                x = torch.randn(M, K, device="cuda", dtype=torch.float16)
+                y = torch.empty(M, N, device="cuda", dtype=torch.float32)
+                ra = torch.from_numpy(rng.integers(0, n_ad, size=M).astype(np.int32)).cuda() if n_ad else None
+                work = torch.zeros(mb.mlora_linear_workspace_bytes(ws_[0], M, max(rank, 1)), dtype=torch.uint8, device="cuda")
+
+                def body():
+                    for w in ws_:
+                        if n_ad:
+                            mb.mlora_linear(w, x, y, work, ra, pa, pb, scale, rank)
+                        else:
+                            mb.mlora_linear(w, x, y, work)
+                ms = time_graph(stream, body, 20) / n_copies
+                used = len(set(ra.cpu().tolist())) if n_ad else 0
+                bytes_ = w_bytes + used * rank * (K + N) * 2 + M * (K * 2 + N * 4)
+                pts.append({"op": "linear", "KxN": f"{K}x{N}", "rows": M, "adapters": n_ad, "rank": rank, "us": ms * 1e3,
+                            "gbs": bytes_ / ms / 1e6, "frac_hbm": bytes_ / ms / 1e6 / peak, "tflops": 2.0 * M * K * N / ms / 1e9})
+        for w in ws_:
+            mb.mlora_weight_destroy(w)
+    return pts
+
+
+def sweep_attention(stream, Ps, Ts, peak):
+    """mlora_attention with 8 streams, 32 query / 8 kv heads of 128, 64 own rows per stream; K/V counted once."""
+    import torch
+    import gen
+    from paper_2604_18655_b200 import binding as mb
+    pts = []
+    n, Hq, Hkv, hd, suf = 8, 32, 8, 128, 64
+    for P in Ps:
+        for T in Ts:
+            branch = {1: (), 16: (4, 2, 2), 64: (4, 4, 4)}[T]
+            parent = gen.build_tree(branch, T) if T > 1 else np.array([-1], dtype=np.int32)
+            parents = torch.from_numpy(np.stack([parent] * n).astype(np.int32)).cuda()
+            cap = suf + T
+            kv_bytes = 2 * Hkv * hd * 2 * (P + n * cap)
+            n_copies = int(L2_BYTES // kv_bytes) + 2
+            q = torch.randn(n * T, Hq, hd, device="cuda", dtype=torch.float16)
+            pk = [torch.randn(Hkv, P, hd, device="cuda", dtype=torch.float16) for _ in range(n_copies)]
+            pv = [torch.randn(Hkv, P, hd, device="cuda", dtype=torch.float16) for _ in range(n_copies)]
+            ok = [torch.randn(n, Hkv, cap, hd, device="cuda", dtype=torch.float16) for _ in range(n_copies)]
+            ov = [torch.randn(n, Hkv, cap, hd, device="cuda", dtype=torch.float16) for _ in range(n_copies)]
+            out = torch.empty(n * T, Hq, hd, device="cuda", dtype=torch.float16)
+            sl = torch.full((n,), suf, dtype=torch.int32, device="cuda")
+            ws = torch.empty(mb.mlora_attention_workspace_bytes(n, T, Hq, Hkv, hd, P, cap), dtype=torch.uint8, device="cuda")
+            status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+            def body():
+                for i in range(n_copies):
+                    mb.mlora_attention(q, pk[i], pv[i], ok[i], ov[i], sl, suf, parents, out, ws, status)
+            ms = time_graph(stream, body, 20) / n_copies
+            bytes_ = kv_bytes + 2 * n * T * Hq * hd * 2
+            flops = 2.0 * 2 * n * T * Hq * hd * (P + suf + T)
+            pts.append({"op": "attention", "prefix": P, "tree_nodes": T, "us": ms * 1e3, "gbs": bytes_ / ms / 1e6,
+                        "frac_hbm": bytes_ / ms / 1e6 / peak, "tflops": flops / ms / 1e9})
+    return pts
+
+
+def run_sweep(args):
+    """Kernel-level sweep (single projection and single attention pass through the C ABI).  One JSON line: `value` is
+    the 8-row, 8-adapter, rank-16 projection of 4096 x 4096 in microseconds; every point sits in `points`."""
+    import torch
+    peak, kind = peaks()
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        if args.quick:
+            shapes, Ms, combos = [(4096, 4096)], [1, 8, 128], [(0, 0), (8, 16)]
+            Ps, Ts = [512, 8192], [1, 16]
+        else:
+            shapes = [(4096, 4096), (4096, 14336), (14336, 4096)]
+            Ms = [1, 4, 8, 32, 128, 256]
+            combos = [(0, 0), (1, 16), (8, 16), (32, 8), (64, 64)]
+            Ps, Ts = [512, 2048, 8192], [1, 16, 64]
+        sampler = ClockSampler(0)
+        sampler.start()
+        t0 = time.time()
+        lin = sweep_linear(stream, shapes, Ms, combos, peak)
+        att = sweep_attention(stream, Ps, Ts, peak)
+        clocks = sampler.stop(t0, time.time())
+    if args.markdown:
+        print(f"HBM peak {peak:.0f} GB/s ({kind}); clocks {clocks}\n")
+        print("| K x N | rows | adapters | rank | us/launch | GB/s (algorithmic) | of peak | TFLOP/s |")
+        print("|---|---|---|---|---|---|---|---|")
+        for r in lin:
+            print(f"| {r['KxN']} | {r['rows']} | {r['adapters']} | {r['rank']} | {r['us']:.2f} | {r['gbs']:.0f} | "
+                  f"{r['frac_hbm']:.3f} | {r['tflops']:.1f} |")
+        print("\n| prefix | tree nodes | us/launch | GB/s (KV once) | of peak | TFLOP/s |")
+        print("|---|---|---|---|---|---|")
+        for r in att:
+            print(f"| {r['prefix']} | {r['tree_nodes']} | {r['us']:.2f} | {r['gbs']:.0f} | {r['frac_hbm']:.3f} | {r['tflops']:.1f} |")
+        return
+    head = next(r for r in lin if r["KxN"] == "4096x4096" and r["rows"] == 8 and r["adapters"] == 8)
+    line = {"metric": "fused INT4 + LoRA projection latency (4096x4096, 8 rows, 8 adapters, rank 16)", "value": head["us"],
+            "unit": "us", "n_gpus": 1, "steps": 20, "warmup": 3, "ms_per_step": head["us"] / 1e3, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+            "config": {"workload": "single-projection and single-attention sweep", "l2": "each point cycles through copies of "
+                       "its weights / KV that together exceed the L2", "launch": "CUDA graph of back-to-back launches"},
+            "clocks": clocks,
+            "roofline": {"bound": "hbm", "achieved": head["gbs"], "peak": peak, "peak_kind": "of " + kind, "unit": "GB/s",
+                         "frac": head["frac_hbm"], "traffic": None},
+            "points": lin + att}
+    print(json.dumps(line), flush=True)
 
 
 def print_timeline(tl, cfg, sm_mhz):
@@ -322,14 +597,22 @@ def print_timeline(tl, cfg, sm_mhz):
 
 
 def workload_name(cfg):
+    what = (f"{cfg.tree_nodes}-node draft trees {cfg.branch}, one verify pass per step" if cfg.tree_nodes > 1
+            else f"{GEN_STEPS} greedy decode steps per generation")
     return (f"{cfg.name}: d{cfg.d_model} L{cfg.n_layers} {cfg.n_q_heads}q/{cfg.n_kv_heads}kv hd{cfg.head_dim} "
             f"ffn{cfg.d_ffn} vocab{cfg.vocab} int4-g{cfg.group_size}; {cfg.n_streams} streams x rank-{cfg.lora_rank} "
-            f"LoRA; shared prompt {cfg.prompt_len}; {GEN_STEPS} greedy decode steps per generation")
+            f"LoRA; shared prompt {cfg.prompt_len}; {what}")
 
 
 def main():
     args = parse_args()
     import gen
+    if args.config == "cfg4":
+        if args.impl == "reference":
+            print(json.dumps({"impl": "reference", "unavailable": "the kernel-level sweep has no CPU arm"}), flush=True)
+        else:
+            run_sweep(args)
+        return
     cfg = {"cfg0": gen.CFG0, "cfg1": gen.CFG1, "cfg2": gen.CFG2, "cfg3": gen.CFG3}[args.config]
     if args.layers is not None:
         cfg = cfg.small(n_layers=args.layers, name=f"{cfg.name}-cut{args.layers}L")
@@ -478,6 +761,25 @@ def main():
         ms_e2e = max_over_ranks(ms_e2e, world, dev)
         e2e_value = aggregate_tokens_per_s(world, n, Ke, ms_e2e)
 
+        # ---- the same steps through the single-kernel decode step (one cooperative launch per step), for comparison
+        step_kernel_ms = None
+        if not hidden_io:
+            mb.mlora_debug_set(ctx, 6, 2)
+            Ks = min(K, 1024)
+            for i in range(GEN_STEPS):
+                generation_step(i)
+            barrier()
+            l1 = mb.mlora_launch_count(ctx)
+            e0.record(side)
+            for i in range(Ks):
+                generation_step(i)
+            e1.record(side)
+            barrier()
+            per_step = (mb.mlora_launch_count(ctx) - l1) / Ks
+            # (a model outside the single kernel's limits keeps running the per-layer kernels: then nothing to report)
+            step_kernel_ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / Ks if per_step < 2.5 else None
+            mb.mlora_debug_set(ctx, 6, 0)
+
         # ---- per-family device time of the same steps (direct launches, an event pair around every kernel)
         mb.mlora_reset_streams(ctx)
         if not hidden_io:
@@ -497,6 +799,11 @@ def main():
     peak, peak_kind = peaks()
     step_bytes = step_algorithmic_bytes(cfg, n, GEN_STEPS / 2)
     ms_step = ms_total / K
+    # decode attention: the shared prefix's and every stream's own K/V once per layer, q in and o out
+    attn_ms = prof["attn"][0] + prof["attn_merge"][0]
+    attn_bytes_step = cfg.n_layers * (2 * cfg.n_kv_heads * cfg.head_dim * 2 * (cfg.prompt_len + n * (4 + prof_steps / 2))
+                                      + 2 * n * cfg.n_q_heads * cfg.head_dim * 2)
+    attn_gbs = attn_bytes_step * prof_steps / (attn_ms / 1e3) / 1e9 if attn_ms > 0 else None
     line = {
         "metric": "aggregate decode tokens/s over streams", "value": value, "unit": "tokens/s", "n_gpus": world,
         "steps": K, "warmup": W, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -510,9 +817,17 @@ def main():
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "decode_chain_kernel (persistent INT4 GEMM + LoRA shrink/expand + norm), all launches of a step",
                      "achieved": achieved, "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH if args.config == "cfg1" and args.layers is None else None,
+                     "frac": achieved / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(args.config) if args.layers is None else None,
                      "bytes_per_launch": gemm_bytes_step / gemm_per_step, "launches_per_step": gemm_per_step,
                      "us_per_launch": 1e3 * gemm_ms / max(gemm_launches, 1)},
+        "roofline_attention": {"bound": "hbm", "kernel": "decode attention over the shared prefix and the streams' own segments "
+                               "(+ merge of the key chunks), all launches of a step", "achieved": attn_gbs, "peak": peak,
+                               "unit": "GB/s", "frac": attn_gbs / peak if attn_gbs else None, "traffic": None,
+                               "bytes_per_step": attn_bytes_step, "us_per_step": 1e3 * attn_ms / prof_steps,
+                               "launches_per_step": (prof["attn"][1] + prof["attn_merge"][1]) / prof_steps},
+        "single_kernel_step": None if step_kernel_ms is None else
+            {"ms_per_step": step_kernel_ms, "tokens_per_s": world * n / (step_kernel_ms / 1e3),
+             "note": "the whole step as one cooperative launch (selectable; the per-layer kernels are the default)"},
         "step_roofline": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_bytes / (ms_step / 1e3) / 1e9,
                           "frac": step_bytes / (ms_step / 1e3) / 1e9 / peak},
         "family_us_per_step": {k: 1e3 * v[0] / prof_steps for k, v in prof.items()},

@@ -57,8 +57,9 @@ typedef struct {
   int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn;
   int32_t vocab;             /* 0: hidden-state input/output, no embedding and no lm_head */
   int32_t group_size;        /* 64 or 128 (any multiple of 64 dividing every K) */
-  float rope_theta;          /* RoPE base; pairing is (i, i + head_dim/2) */
+  float rope_theta;          /* RoPE base */
   float rms_eps;
+  int32_t rope_style;        /* 0 = half-split pairs (i, i + head_dim/2); anything else: MLORA_ERR_UNSUPPORTED */
   int32_t lora_rank;         /* one rank for all adapters (Sec. 6: all LoRAs have identical shape) */
   int32_t lora_targets;      /* OR of MLORA_Q.. */
   int32_t max_adapters;      /* adapter slots */
@@ -137,6 +138,11 @@ const char* mlora_last_error(mlora_ctx* ctx);   /* text of the last host-side er
  * stream == -1 reads the shared segment (suffix_len receives the prefix length).  Synchronises. */
 int mlora_export_kv(mlora_ctx* ctx, int32_t layer, int32_t stream, int32_t first, int32_t count,
                     int32_t* suffix_len, void* k_out, void* v_out);
+/* The whole own segment of one stream in one layer (Sec. 3.4: the stream's private KV segment; the check of the KV
+ * compaction of Sec. 3.5 reads it): writes the stream's suffix length to *suffix_len (host) and its first suffix_len
+ * rows to k_out/v_out (dev fp16 [suffix_len][n_kv_heads][head_dim]; the buffers must hold max_suffix + max_tree rows).
+ * Synchronises.  Errors: ARG, CUDA. */
+int mlora_export_state(mlora_ctx* ctx, int32_t layer, int32_t stream, int32_t* suffix_len, void* k_out, void* v_out);
 /* Writes the dequantised weights of (layer, proj) as the GEMM kernel's own unpack path produces them:
  * out dev fp16 [K][N].  proj 0..6 = q,k,v,o,gate,up,down; layer == n_layers, proj == 0 = lm_head. */
 int mlora_debug_dequant(mlora_ctx* ctx, int32_t layer, int32_t proj, void* out_fp16);
@@ -187,7 +193,9 @@ size_t mlora_linear_workspace_bytes(const mlora_weight* w, int32_t M, int32_t ra
  * x dev fp16 [M][K]; row_adapter dev int32 [M] (-1 = base) or NULL for no LoRA; A, B: DEV arrays of
  * n_adapters device pointers (fp16 [rank][K], fp16 [rank][N]); scale dev fp32 [n_adapters] (= alpha/r);
  * y dev fp32 [M][N]; workspace dev, zero-filled before first use (the call leaves it zeroed where it matters).
- * Errors: ARG, CAPACITY (workspace too small), UNSUPPORTED (M > 4096). */
+ * x, y, workspace and every A[a], B[a] must be 16-byte aligned (the kernels use 128-bit loads and bulk copies).
+ * Errors: ARG (null or misaligned pointer), CAPACITY (workspace too small), UNSUPPORTED (M > 4096).  A bounded wait
+ * that runs out on the device is reported by mlora_linear_status. */
 int mlora_linear(mlora_weight* w, const void* x, int32_t M, const int32_t* row_adapter, const void* const* A,
                  const void* const* B, const float* scale, int32_t n_adapters, int32_t rank, float* y,
                  void* workspace, size_t workspace_bytes);
@@ -202,14 +210,22 @@ int mlora_linear(mlora_weight* w, const void* x, int32_t M, const int32_t* row_a
  * beforehand, does allocate.)
  * Limits: 1 <= M <= 8, rank <= 64, and an input width K small enough for the single-kernel path (K <= 8192
  * on a B200); anything beyond returns MLORA_ERR_CAPACITY and runs nothing -- use mlora_linear there.
+ * The array used is the one on the weight's device, which must be the current device (else MLORA_ERR_ARG).
  * The first call on a device looks up the array's device address; make that call outside any stream capture.
  * All calls on a device share the one array: two calls that overlap on the GPU (different streams) race;
  * calls on the weight's own stream, or otherwise ordered, are fine.
- * Errors: ARG, CAPACITY, UNSUPPORTED, CUDA. */
+ * A bounded wait that runs out on the device (e.g. after such a race) leaves garbage in y: mlora_linear_status(w, NULL)
+ * reports and clears it.  Errors: ARG (null or misaligned pointer, wrong device), CAPACITY, UNSUPPORTED, CUDA. */
 int mlora_linear_noalloc(mlora_weight* w, const void* x, int32_t M, const int32_t* row_adapter, const void* const* A,
                          const void* const* B, const float* scale, int32_t n_adapters, int32_t rank, float* y);
 
-/* Bytes of scratch for mlora_attention. */
+/* Device status of the mlora_linear calls made with `workspace` (workspace == NULL: of the mlora_linear_noalloc calls
+ * on the weight's device, which must be current).  Synchronises the weight's stream; returns MLORA_OK, or the status
+ * (MLORA_ERR_TIMEOUT: a bounded wait ran out and the last result is garbage) after clearing it together with the
+ * kernel's barrier words, so that the next call starts afresh.  Allocates nothing.  Errors: ARG, CUDA, TIMEOUT. */
+int mlora_linear_status(mlora_weight* w, void* workspace);
+
+/* Bytes of scratch for mlora_attention (the largest need over every suffix_bound up to own_capacity - n_nodes). */
 size_t mlora_attention_workspace_bytes(int32_t n_streams, int32_t n_nodes, int32_t n_q_heads, int32_t n_kv_heads,
                                        int32_t head_dim, int32_t prefix_len, int32_t own_capacity);
 /* Shared-prefix + own-segment + tree-ancestor attention (Sec. 3.4/3.5, App. A.1/A.2) for

@@ -27,7 +27,7 @@ class ModelDesc(C.Structure):
     _fields_ = [
         ("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
         ("head_dim", C.c_int32), ("d_ffn", C.c_int32), ("vocab", C.c_int32), ("group_size", C.c_int32),
-        ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("lora_rank", C.c_int32), ("lora_targets", C.c_int32),
+        ("rope_theta", C.c_float), ("rms_eps", C.c_float), ("rope_style", C.c_int32), ("lora_rank", C.c_int32), ("lora_targets", C.c_int32),
         ("max_adapters", C.c_int32), ("max_streams", C.c_int32), ("max_prefix", C.c_int32),
         ("max_suffix", C.c_int32), ("max_tree", C.c_int32),
         ("embed", C.c_void_p), ("qweight", C.POINTER(C.c_void_p)), ("scales", C.POINTER(C.c_void_p)),
@@ -54,6 +54,7 @@ _SIGS = {
     "mlora_last_error": (C.c_char_p, [C.c_void_p]),
     "mlora_export_kv": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_int32),
                                   C.c_void_p, C.c_void_p]),
+    "mlora_export_state": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int32), C.c_void_p, C.c_void_p]),
     "mlora_debug_dequant": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "mlora_debug_set": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32]),
     "mlora_profile_begin": (C.c_int, [C.c_void_p]),
@@ -69,6 +70,7 @@ _SIGS = {
                                C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_size_t]),
     "mlora_linear_noalloc": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                        C.c_int32, C.c_int32, C.c_void_p]),
+    "mlora_linear_status": (C.c_int, [C.c_void_p, C.c_void_p]),
     "mlora_attention_workspace_bytes": (C.c_size_t, [C.c_int32] * 7),
     "mlora_attention": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
                                   C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
@@ -125,6 +127,7 @@ def mlora_create(cfg, qweight, scales, rms_attn, rms_ffn, rms_final=None, embed=
     for f in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab", "group_size"):
         setattr(d, f, int(getattr(cfg, f)))
     d.rope_theta, d.rms_eps = float(cfg.rope_theta), float(cfg.rms_eps)
+    d.rope_style = int(getattr(cfg, "rope_style", 0))
     d.lora_rank = int(cfg.lora_rank if lora_rank is None else lora_rank)
     d.lora_targets = int(cfg.lora_targets if lora_targets is None else lora_targets)
     d.max_adapters, d.max_streams, d.max_prefix = max_adapters, max_streams, max_prefix
@@ -196,6 +199,13 @@ def mlora_export_kv(ctx, layer, stream, first, count, k_out=None, v_out=None):
     return s.value
 
 
+def mlora_export_state(ctx, layer, stream, k_out, v_out):
+    """The stream's whole own segment of one layer into k_out / v_out; returns its suffix length."""
+    s = C.c_int32(0)
+    _check(lib().mlora_export_state(ctx, layer, stream, C.byref(s), _ptr(k_out), _ptr(v_out)))
+    return s.value
+
+
 def mlora_debug_dequant(ctx, layer, proj, out_fp16):
     _check(lib().mlora_debug_dequant(ctx, layer, proj, _ptr(out_fp16)))
 
@@ -261,6 +271,11 @@ def mlora_linear_noalloc(w, x, y, row_adapter=None, A_ptrs=None, B_ptrs=None, sc
     n_ad = 0 if A_ptrs is None else A_ptrs.numel()
     _check(lib().mlora_linear_noalloc(w, _ptr(x), x.shape[0], _ptr(row_adapter), _ptr(A_ptrs), _ptr(B_ptrs),
                                       _ptr(scale), n_ad, rank, _ptr(y)))
+
+
+def mlora_linear_status(w, workspace=None):
+    """Raises MloraError if a bounded wait ran out in an mlora_linear / mlora_linear_noalloc call (None: the latter)."""
+    _check(lib().mlora_linear_status(w, _ptr(workspace)))
 
 
 def mlora_attention_workspace_bytes(n, T, Hq, Hkv, hd, P, own_capacity):

@@ -100,36 +100,6 @@ struct PhaseDerived {
   int item_sm[CH_MAX_ITEMS];         // their segment | row << 8
 };
 
-// ----------------------------------------------------------------------------- optional timeline (trace builds only)
-// With -DCHAIN_TRACE thread 0 of the first and the last CTA stamp the global nanosecond timer at the section
-// boundaries of every phase; mlora_trace_read copies the stamps out.  Compiled out otherwise.
-#ifdef CHAIN_TRACE
-constexpr int TR_PER_PHASE = 64, TR_PHASES = 160;
-__device__ long long g_trace[2 * TR_PHASES * TR_PER_PHASE * 3];
-#define STAMP(id)                                                                                          \
-  do {                                                                                                     \
-    if (tid == 0 && tr_slot >= 0 && tr_n < TR_PER_PHASE && p < TR_PHASES) {                                \
-      long long tns;                                                                                       \
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tns));                                              \
-      long long* e_ = g_trace + (((size_t)tr_slot * TR_PHASES + p) * TR_PER_PHASE + tr_n) * 3;             \
-      e_[0] = (id); e_[1] = tns; e_[2] = clock64(); ++tr_n;                                                \
-    }                                                                                                      \
-  } while (0)
-// the same from lane 0 of the first shrink warp (second half of the phase's record)
-#define STAMPS(id)                                                                                         \
-  do {                                                                                                     \
-    if (shr_id == 0 && lane == 0 && tr_slot >= 0 && tr_n2 < TR_PER_PHASE / 2 && p < TR_PHASES) {           \
-      long long tns;                                                                                       \
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tns));                                              \
-      long long* e_ = g_trace + (((size_t)tr_slot * TR_PHASES + p) * TR_PER_PHASE + TR_PER_PHASE / 2 + tr_n2) * 3; \
-      e_[0] = (id); e_[1] = tns; e_[2] = clock64(); ++tr_n2;                                               \
-    }                                                                                                      \
-  } while (0)
-#else
-#define STAMP(id) do { } while (0)
-#define STAMPS(id) do { } while (0)
-#endif
-
 // ----------------------------------------------------------------------------- the ring schedule
 // Everything immutable and bulky that a CTA needs flows through the ring in one fixed order, known to the
 // producer and to the consumers alike.  Per phase:
@@ -459,9 +429,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
   unsigned long long n_bar = 0;                       // barriers passed in this launch
   unsigned n_shr = 0;                                 // LoRA phases passed in this launch
   float* redf = reinterpret_cast<float*>(red);
-#ifdef CHAIN_TRACE
-  const int tr_slot = blockIdx.x == 0 ? 0 : (blockIdx.x == G - 1 ? 1 : -1);
-#endif
   for (int p = a.p0; p < a.p1; ++p) {
     const int slot = (p - a.p0) & 1;
     const ChainPhase& ph = s_ph[slot];
@@ -470,10 +437,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
     const PhaseDerived& pd = s_pd[slot];
     const WLayout L = pd.L;
     const int nseg = lora_on ? ph.lora_nseg : 0;
-#ifdef CHAIN_TRACE
-    int tr_n = 0, tr_n2 = 0;
-#endif
-    STAMP(0);
     const int tpu = pd.tpu, ipt = pd.ipt, gshift = pd.gshift, my_units = pd.my_units, teams = pd.teams;
     const int shr_warps = pd.shr_warps, gemm_warps = pd.gemm_warps;
     // the teams are formed anew for every round of units: the last round may have fewer units than teams, and
@@ -560,7 +523,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
       }
     }
     consumer_sync();
-    STAMP(1);
 
     // ---- 2. next phase's descriptor and adapter pointers (immutable) while this phase runs: warp 0 issues the
     // loads here and stores what they return further down, so neither round trip holds anything up
@@ -579,7 +541,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
       // to the shrink warps, so that a long row (K = 5632: six halves) does not sit on one warp; the partial sums
       // are added in order by the first shrink warp, which also tells the grid that the CTA's share of T is written.
       if (shr_id >= 0) {
-        STAMPS(10);
         const int hp = 2 * np;                                            // half pieces per item
         const int n_half = pd.n_valid * hp;
         const int st0 = pos_stage(pos, nstages);
@@ -594,7 +555,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
           uint32_t par = par0;
           if (st >= nstages) { st -= nstages; par ^= 1u; }
           const bool ok = wait_mbar(smem_u32(full_bar + st), par, wc, 2, p);
-          STAMPS(11);
           const int k0 = q * CH_A_PIECE + hf * (CH_A_PIECE / 2);
           const unsigned char* sb = ring + (size_t)st * CH_STAGE_BYTES + hf * CH_A_PIECE;   // bytes: half a piece
           const __half* hrow = hs + (size_t)m * hs_stride + k0;
@@ -621,7 +581,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
           if (lane < CH_ITEMS_PER_CHUNK / 2) mbar_arrive(smem_u32(empty_bar + st));   // the two halves free the stage
           const float acc = warp_sum((acc4[0] + acc4[1]) + (acc4[2] + acc4[3]));
           if (lane == 0) s_shr_part[kk][hq] = acc;
-          STAMPS(12);
         }
         asm volatile("bar.sync 11, %0;" ::"r"(shr_warps * 32) : "memory");
         if (shr_id == 0) {
@@ -633,7 +592,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
           // the warp barrier orders the lanes' stores before lane 0's release, which is cumulative over them
           __syncwarp();
           if (lane == 0) red_release_add_u64(a.sync + 1, 1ull);
-          STAMPS(13);
           // This warp has nothing else to do in the phase: it watches for the other CTAs' shares and brings all of
           // T into shared memory as soon as it is complete, so that the GEMM teams, when their main loop ends, find
           // it there instead of paying a counter poll and a load round trip each.
@@ -648,7 +606,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
       pos += np * pd.n_valid;
       ++n_shr;
     }
-    STAMP(2);
     if (prep_next) {
       reinterpret_cast<int*>(&s_ph[nslot])[lane] = prep_word;
       __syncwarp();
@@ -735,7 +692,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
           red[(size_t)(tu * CH_CWARPS + warp) * 32 + lane] =
               make_float4(acc0[0] + acc1[0], acc0[1] + acc1[1], acc0[2] + acc1[2], acc0[3] + acc1[3]);
         }
-        STAMP(3);
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         team_sync();
         if (nseg > 0 && !t_loaded) {
@@ -751,7 +707,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
           }
           team_sync();
           t_loaded = true;
-          STAMP(4);
         }
         // ---- epilogue of the unit: one thread per (row, column)
         for (int o = tt; o < CHAIN_MAX_ROWS * TILE_N; o += team_threads) {
@@ -798,7 +753,6 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
             ph.out_f16[(size_t)m * (ph.N / 2) + colv[1]] = __float2half_rn(v);
           }
         }
-        STAMP(5);
         team_sync();                                   // the team's partial sums and B slices may be rewritten
       }
     }
@@ -808,13 +762,11 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
       s_pA[nslot][lane / CHAIN_MAX_ROWS][lane % CHAIN_MAX_ROWS] = prep_pa;
       s_pB[nslot][lane / CHAIN_MAX_ROWS][lane % CHAIN_MAX_ROWS] = prep_pb;
     }
-    STAMP(6);
 
     // ---- 5. grid barrier: the next phase reads what every CTA wrote
     if (p + 1 < a.p1) {
       ++n_bar;
       consumer_sync();
-      STAMP(7);
       if (tid == 0) {
         // the release is cumulative over what the CTA's threads wrote before the named barrier above; the
         // acquire load inside wait_counter orders the next phase's reads after the other CTAs' writes
@@ -827,23 +779,9 @@ __global__ void __launch_bounds__(CH_THREADS, 1) decode_chain_kernel(const Chain
       if (tid == 32) derive_phase(p + 1);
       consumer_sync();
     }
-    STAMP(8);
   }
 }
 
-#ifdef CHAIN_TRACE
-extern "C" int mlora_trace_read(long long* host_out, int n_longs) {
-  const size_t total = sizeof(g_trace) / sizeof(long long);
-  const size_t n = (size_t)n_longs < total ? (size_t)n_longs : total;
-  return (int)cudaMemcpyFromSymbol(host_out, g_trace, n * sizeof(long long));
-}
-extern "C" int mlora_trace_clear() {
-  void* ptr = nullptr;
-  cudaError_t e = cudaGetSymbolAddress(&ptr, g_trace);
-  if (e != cudaSuccess) return (int)e;
-  return (int)cudaMemset(ptr, 0, sizeof(g_trace));
-}
-#endif
 
 // ----------------------------------------------------------------------------- host side
 cudaError_t init_chain() {

@@ -34,7 +34,7 @@ void free_packed(PackedWeight& w) {
 }
 
 struct GraphKey {
-  int kind, n, T, prefix_chunk, n_prefix_chunks, own_chunk, n_own_chunks, flags;
+  int kind, n, T, prefix_chunk, n_prefix_chunks, own_chunk, n_own_chunks, flags, suffix_bound, pad_;
   const void* p[8];
   bool operator==(const GraphKey& o) const { return std::memcmp(this, &o, sizeof(GraphKey)) == 0; }
 };
@@ -53,6 +53,7 @@ struct GraphEntry { cudaGraphExec_t exec; int nodes; };
 struct mlora_weight {
   PackedWeight w;
   cudaStream_t stream;
+  int device = 0;                  // the device the packed weights live on
   ChainPhase* phase = nullptr;     // dev: descriptor of this projection for the persistent kernel
   int sm_count = 0;
 };
@@ -492,7 +493,14 @@ int ensure_capacity(mlora_ctx* c, int T) {
 }
 
 int init_kernels() {
-  static bool done = false;
+  // the opt-in shared-memory sizes are per device: once for every device a context or weight is created on
+  static bool done_on[64] = {};
+  static std::mutex mu;
+  int dev = 0;
+  CK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(MLORA_ERR_UNSUPPORTED, "device ordinal out of range");
+  std::lock_guard<std::mutex> lock(mu);
+  bool& done = done_on[dev];
   if (done) return MLORA_OK;
   CK(init_gemm());
   CK(init_shrink());
@@ -565,6 +573,7 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
   if (!d.qweight || !d.scales || !d.rms_attn || !d.rms_ffn) return fail(MLORA_ERR_ARG, "null weight table");
   if (d.vocab > 0 && (!d.embed || !d.rms_final)) return fail(MLORA_ERR_ARG, "vocab > 0 needs embed and rms_final");
   if (d.head_dim != 64 && d.head_dim != 128) return fail(MLORA_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
+  if (d.rope_style != 0) return fail(MLORA_ERR_UNSUPPORTED, "rope_style must be 0 (half-split pairs)");
   if (d.n_q_heads % d.n_kv_heads) return fail(MLORA_ERR_ARG, "n_q_heads must be a multiple of n_kv_heads");
   if (!wlayout_group_ok(d.group_size))
     return fail(MLORA_ERR_UNSUPPORTED, "group_size must be 64, 128, 256 or a multiple of 512");
@@ -976,6 +985,7 @@ static int decode_impl(mlora_ctx* c, int n, const int32_t* adapter_idx, const in
   key.prefix_chunk = io.plan.prefix_chunk; key.n_prefix_chunks = io.plan.n_prefix_chunks;
   key.own_chunk = io.plan.own_chunk; key.n_own_chunks = io.plan.n_own_chunks;
   key.flags = c->P * 4 + c->dbg_inject_stall * 2 + c->dbg_no_chain;
+  key.suffix_bound = io.plan.suffix_bound;     // (rounded up by plan_pass: the kernels' launch shape and prefetch extents)
   key.p[0] = adapter_idx; key.p[1] = tokens; key.p[2] = hidden; key.p[3] = out_next; key.p[4] = out_logits; key.p[5] = hidden_out;
   rc = replay_or_run(c, key, [&]() -> int {
     int r = forward(c, io);
@@ -1049,6 +1059,7 @@ int mlora_verify_tree(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_id
   key.prefix_chunk = io.plan.prefix_chunk; key.n_prefix_chunks = io.plan.n_prefix_chunks;
   key.own_chunk = io.plan.own_chunk; key.n_own_chunks = io.plan.n_own_chunks;
   key.flags = c->P * 8 + c->dbg_no_tc * 4 + c->dbg_skip_compact * 2 + c->dbg_no_chain;
+  key.suffix_bound = io.plan.suffix_bound;
   key.p[0] = adapter_idx; key.p[1] = tree_tokens; key.p[2] = tree_parent; key.p[3] = out_accept_len;
   key.p[4] = out_accept_idx; key.p[5] = out_next; key.p[6] = out_logits;
   rc = replay_or_run(c, key, [&]() -> int {
@@ -1151,6 +1162,15 @@ int mlora_export_kv(mlora_ctx* c, int32_t layer, int32_t stream, int32_t first, 
   return MLORA_OK;
 }
 
+int mlora_export_state(mlora_ctx* c, int32_t layer, int32_t stream, int32_t* suffix_len, void* k_out, void* v_out) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (!suffix_len) return fail(MLORA_ERR_ARG, "export_state: suffix_len is null");
+  if (stream < 0) return fail(MLORA_ERR_ARG, "export_state: stream out of range");
+  int rc = mlora_export_kv(c, layer, stream, 0, 0, suffix_len, nullptr, nullptr);
+  if (rc != MLORA_OK || *suffix_len == 0) return rc;
+  return mlora_export_kv(c, layer, stream, 0, *suffix_len, suffix_len, k_out, v_out);
+}
+
 int mlora_debug_dequant(mlora_ctx* c, int32_t layer, int32_t proj, void* out_fp16) {
   if (check_ctx(c)) return MLORA_ERR_ARG;
   if (!out_fp16) return fail(MLORA_ERR_ARG, "null output");
@@ -1239,6 +1259,7 @@ int mlora_weight_create(const void* qweight, const void* scales, int32_t K, int3
   if (e == cudaSuccess) {
     int dev = 0;
     e = cudaGetDevice(&dev);
+    w->device = dev;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&w->sm_count, cudaDevAttrMultiProcessorCount, dev);
   }
   if (e == cudaSuccess) e = cudaMalloc(&w->phase, sizeof(ChainPhase));
@@ -1290,6 +1311,7 @@ int mlora_linear(mlora_weight* w, const void* x, int32_t M, const int32_t* row_a
                  size_t workspace_bytes) {
   if (!w || !x || !y || !workspace) return fail(MLORA_ERR_ARG, "null argument");
   if (M <= 0 || M > 4096) return fail(MLORA_ERR_UNSUPPORTED, "M must be in 1..4096");
+  if (((uintptr_t)x | (uintptr_t)y | (uintptr_t)workspace) & 15) return fail(MLORA_ERR_ARG, "x, y and workspace must be 16-byte aligned");
   const bool lora = row_adapter != nullptr;
   if (lora && (!A || !B || !scale || n_adapters <= 0 || rank <= 0)) return fail(MLORA_ERR_ARG, "incomplete adapter arguments");
   const size_t fixed = LIN_COUNTER_BYTES + lin_T_bytes(M, rank);
@@ -1353,6 +1375,7 @@ int mlora_linear_noalloc(mlora_weight* w, const void* x, int32_t M, const int32_
   if (!w || !x || !y) return fail(MLORA_ERR_ARG, "null argument");
   const bool lora = row_adapter != nullptr;
   if (lora && (!A || !B || !scale || n_adapters <= 0 || rank <= 0)) return fail(MLORA_ERR_ARG, "incomplete adapter arguments");
+  if (((uintptr_t)x | (uintptr_t)y) & 15) return fail(MLORA_ERR_ARG, "x and y must be 16-byte aligned");
   if (M < 1 || M > CHAIN_MAX_ROWS) return fail(MLORA_ERR_CAPACITY, "mlora_linear_noalloc takes 1..8 rows");
   if (lora && rank > CHAIN_MAX_RANK) return fail(MLORA_ERR_CAPACITY, "mlora_linear_noalloc takes LoRA ranks up to 64");
   if (NOALLOC_HEAD_BYTES + (size_t)M * (lora ? rank : 1) * sizeof(float) > NOALLOC_SCRATCH_BYTES)
@@ -1360,8 +1383,11 @@ int mlora_linear_noalloc(mlora_weight* w, const void* x, int32_t M, const int32_
   const int stages = chain_pick_stages(w->w.K, lora ? rank : 0);
   if (stages <= 0 || !chain_phase_fits(w->w.K, MODE_PLAIN, lora ? 1 : 0, rank, stages, w->sm_count))
     return fail(MLORA_ERR_CAPACITY, "input width too large for the built-in scratch path: use mlora_linear");
+  // the array is looked up on the device the weight lives on; that device must be the current one (the address
+  // query below and the launch both go to the current device)
   int dev = 0;
   CK(cudaGetDevice(&dev));
+  if (dev != w->device) return fail(MLORA_ERR_ARG, "the weight's device is not the current device");
   if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return fail(MLORA_ERR_UNSUPPORTED, "device ordinal out of range");
   void* scratch = nullptr;
   {
@@ -1393,6 +1419,28 @@ int mlora_linear_noalloc(mlora_weight* w, const void* x, int32_t M, const int32_
   return MLORA_OK;
 }
 
+int mlora_linear_status(mlora_weight* w, void* workspace) {
+  if (!w) return fail(MLORA_ERR_ARG, "null weight");
+  unsigned char* ws = (unsigned char*)workspace;
+  if (ws == nullptr) {                                   // the built-in array of mlora_linear_noalloc
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev != w->device) return fail(MLORA_ERR_ARG, "the weight's device is not the current device");
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (dev < 0 || dev >= NOALLOC_MAX_DEVICES || g_noalloc_ptr[dev] == nullptr) return MLORA_OK;   // never used: nothing to report
+    ws = (unsigned char*)g_noalloc_ptr[dev];
+  }
+  CK(cudaStreamSynchronize(w->stream));
+  int st = 0;
+  CK(cudaMemcpy(&st, ws + 32, sizeof(int), cudaMemcpyDeviceToHost));
+  if (st != 0) {
+    // the barrier words, the abort flag and the status start afresh
+    CK(cudaMemset(ws, 0, LIN_SYNC_BYTES));
+    return fail(st, st == MLORA_ERR_TIMEOUT ? "device status: a bounded wait of the projection kernel ran out" : "device status");
+  }
+  return MLORA_OK;
+}
+
 static void attn_fill(AttnArgs& a, int n, int T, int Hq, int Hkv, int hd, int P, int suffix_bound) {
   a = AttnArgs{};
   a.P = P; a.n = n; a.T = T; a.Hq = Hq; a.Hkv = Hkv; a.hd = hd;
@@ -1403,10 +1451,17 @@ static void attn_fill(AttnArgs& a, int n, int T, int Hq, int Hkv, int hd, int P,
 size_t mlora_attention_workspace_bytes(int32_t n, int32_t T, int32_t Hq, int32_t Hkv, int32_t hd, int32_t P,
                                        int32_t own_capacity) {
   if (n <= 0 || T <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv) return 0;
-  AttnArgs a;
-  attn_fill(a, n, T, Hq, Hkv, hd, P, own_capacity > T ? own_capacity - T : 0);
+  // the chunking, and with it the scratch, depends on the suffix bound of the call (not monotonically): take the
+  // largest need over every bound the capacity allows
+  size_t floats = 0;
+  for (int sb = 0; sb <= (own_capacity > T ? own_capacity - T : 0); ++sb) {
+    AttnArgs a;
+    attn_fill(a, n, T, Hq, Hkv, hd, P, sb);
+    const size_t f = attn_workspace_floats(a);
+    floats = f > floats ? f : floats;
+  }
   const size_t rows = (size_t)n * T;
-  return rows * (sizeof(unsigned long long) + sizeof(int32_t)) + 256 + attn_workspace_floats(a) * sizeof(float);
+  return rows * (sizeof(unsigned long long) + sizeof(int32_t)) + 256 + floats * sizeof(float);
 }
 
 int mlora_attention(const void* q, const void* prefix_k, const void* prefix_v, int32_t P, const void* own_k,

@@ -47,3 +47,18 @@ def test_host_side_argument_errors_need_no_gpu(libpath):
     assert L.mlora_destroy(None) == 0
     assert L.mlora_linear_workspace_bytes(None, 8, 16) == 0
     assert L.mlora_attention_workspace_bytes(8, 1, 32, 8, 128, 512, 65) > 0
+
+
+def test_unsupported_rope_style_is_refused_on_the_host(libpath):
+    """rope_style other than 0 (half-split pairs) is rejected before anything touches a device."""
+    from paper_2604_18655_b200 import binding as mb
+    L = mb.lib()
+    d = mb.ModelDesc()
+    d.n_layers, d.d_model, d.n_q_heads, d.n_kv_heads, d.head_dim, d.d_ffn = 1, 64, 1, 1, 64, 64
+    d.group_size, d.max_tree, d.max_streams, d.max_prefix, d.max_suffix = 64, 1, 1, 1, 1
+    arr = (ctypes.c_void_p * 8)(*([1] * 8))
+    d.qweight, d.scales, d.rms_attn, d.rms_ffn = arr, arr, arr, arr
+    d.rope_style = 1
+    out = ctypes.c_void_p()
+    assert L.mlora_create(ctypes.byref(d), ctypes.byref(out)) == -6
+    assert b"rope_style" in L.mlora_last_error(None)

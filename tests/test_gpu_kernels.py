@@ -103,6 +103,31 @@ def test_linear_lora_matches_oracle(mb, K, N, G, M, n_ad, rank):
     compare(got, want, f"linear lora K{K} N{N} M{M} ad{n_ad} r{rank}")
 
 
+@pytest.mark.parametrize("K,N", [(14336, 4096), (4096, 14336)])
+@pytest.mark.parametrize("M", [8, 256])
+def test_linear_lora_at_the_sweep_shapes(mb, K, N, M):
+    """The widest shapes of the single-projection workload (inputs or outputs of 14336 features), 8 adapters of rank 16
+    picked per row at random: the few-row kernels and the tensor-core path with its widest row block."""
+    got, want = run_linear(mb, K, N, 128, M, 8, 16, seed=K + M)
+    compare(got, want, f"linear lora K{K} N{N} M{M}")
+
+
+def test_linear_status_call_reports_nothing_after_clean_calls(mb):
+    rng = np.random.default_rng(2)
+    qb, sc = gen.quantize_int4(rng.standard_normal((256, 64)).astype(np.float32), 64)
+    w = mb.mlora_weight_create(dev(qb), dev(sc), 256, 64, 64)
+    x = dev(rng.standard_normal((4, 256)).astype(np.float16))
+    y = torch.empty(4, 64, dtype=torch.float32, device="cuda")
+    ws = torch.zeros(mb.mlora_linear_workspace_bytes(w, 4, 1), dtype=torch.uint8, device="cuda")
+    mb.mlora_linear(w, x, y, ws)
+    mb.mlora_linear_status(w, ws)                       # raises if the device status is set
+    mb.mlora_linear_status(w, None)                     # the built-in array (possibly never used yet)
+    with pytest.raises(mb.MloraError) as e:             # a misaligned input is refused on the host, not faulted on
+        mb.mlora_linear(w, x.view(-1)[4:4 + 3 * 256].view(3, 256), y[:3], ws)
+    assert e.value.code == -1
+    mb.mlora_weight_destroy(w)
+
+
 def test_linear_base_wide_ragged_output(mb):
     """Enough 16 x 32 output tiles for the warp-per-tile epilogue, with a width that is not a multiple of 32 and a row
     count that is not a multiple of 16: the ragged last tiles of both directions."""
@@ -176,6 +201,22 @@ def run_attention(mb, n, T, Hq, Hkv, hd, P, suf, branch, seed, cap=None):
 def test_attention_matches_oracle(mb, hd, n, T, branch, P, suf):
     got, want = run_attention(mb, n, T, 8, 2, hd, P, suf, branch, seed=hd + n + T + P)
     compare(got, want, f"attention hd{hd} n{n} T{T} P{P}")
+
+
+@pytest.mark.parametrize("n,T,branch,P,suf", [
+    (2, 32, (4, 4, 2), 2048, [64, 5]),       # the 3B verify shape: 32-node trees over a 2048-token prompt
+    (2, 16, (4, 2, 2), 8192, [64, 0]),       # the longest prefix of the attention sweep
+])
+def test_attention_tree_passes_at_long_prefixes(mb, n, T, branch, P, suf):
+    got, want = run_attention(mb, n, T, 32, 8, 128, P, suf, branch, seed=P + T)
+    compare(got, want, f"attention hd128 32q/8kv n{n} T{T} P{P}")
+
+
+def test_attention_workspace_covers_every_suffix_bound(mb):
+    """The documented workspace size must do for any suffix bound the capacity allows (the chunking, and with it the
+    scratch, is not monotone in the bound): capacity 129 with bound 127 once needed more than the size planned at 128."""
+    got, want = run_attention(mb, 8, 1, 32, 8, 64, 512, [127, 0, 5, 64, 100, 127, 1, 90], (), seed=9, cap=129)
+    compare(got, want, "attention cap129 bound127")
 
 
 def test_attention_long_prefix_split(mb):

@@ -391,6 +391,48 @@ def test_decode_paths_agree(GpuModel):
         compare(res[i][2], res[2][2], "V across paths")
 
 
+def test_debug_dequant_of_fused_projections_is_bit_exact(GpuModel):
+    """The context's own weights -- q, k, v packed into one fused matrix, gate and up interleaved by tiles, and the
+    plain ones -- unpacked by the kernels' dequantisation and compared bit for bit with the oracle's."""
+    from paper_2604_18655_b200 import binding as mb
+    cfg = TINYV
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=8)
+    for layer in (0, cfg.n_layers - 1):
+        for p, name in enumerate(gen.PROJ_NAMES):
+            K, N = gen.proj_shape(cfg, name)
+            out = torch.empty(K, N, dtype=torch.float16, device="cuda")
+            mb.mlora_debug_dequant(gm.ctx, layer, p, out)
+            torch.cuda.synchronize()
+            want = ref.dequant(m.qweight[layer * 7 + p], m.scales[layer * 7 + p], cfg.group_size)
+            assert np.array_equal(out.cpu().numpy().view(np.uint16), want.view(np.uint16)), (layer, name)
+    K, N = gen.proj_shape(cfg, "lm_head")
+    out = torch.empty(K, N, dtype=torch.float16, device="cuda")
+    mb.mlora_debug_dequant(gm.ctx, cfg.n_layers, 0, out)
+    torch.cuda.synchronize()
+    want = ref.dequant(m.qweight[cfg.n_layers * 7], m.scales[cfg.n_layers * 7], cfg.group_size)
+    assert np.array_equal(out.cpu().numpy().view(np.uint16), want.view(np.uint16))
+    gm.close()
+
+
+def test_export_state_gives_the_whole_own_segment(GpuModel):
+    from paper_2604_18655_b200 import binding as mb
+    cfg = TINYV
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+    ids = gen.make_prompt_ids(cfg, 0)
+    gm.prefill(ids)
+    orc.prefill_shared(ids)
+    toks = np.array([5, 6, 7], dtype=np.int32)
+    for _ in range(3):
+        toks, _ = gm.decode([0, 1, -1], toks)
+    k = torch.zeros(17, cfg.n_kv_heads, cfg.head_dim, dtype=torch.float16, device="cuda")
+    v = torch.zeros_like(k)
+    S = mb.mlora_export_state(gm.ctx, 1, 2, k, v)
+    assert S == 3
+    _, k2, v2 = gm.export_kv(1, 2, 0, 3)
+    assert np.array_equal(k.cpu().numpy()[:3], k2) and np.array_equal(v.cpu().numpy()[:3], v2)
+    gm.close()
+
+
 def test_host_buffer_step_matches_device_step(GpuModel):
     """mlora_decode_step_host (host arrays in and out) gives the tokens of mlora_decode_step."""
     from paper_2604_18655_b200 import binding as mb
