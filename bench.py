@@ -659,7 +659,8 @@ def main():
             last = torch.empty(cfg.vocab, dtype=torch.float32, device=dev)
             mb.mlora_prefill_shared(ctx, ids, last)
             # stream i starts from the (i+1)-th most likely first token (App. A.1: n distinct first tokens)
-            first = torch.topk(last, n).indices.to(torch.int32)
+            first = torch.empty(n, dtype=torch.int32, device=dev)
+            mb.mlora_sample_first(ctx, last, first)
         tok = [torch.empty(n, dtype=torch.int32, device=dev) for _ in range(2)]
 
         def generation_step(i):
@@ -674,6 +675,18 @@ def main():
                 mb.mlora_reset_streams(ctx)
                 tok[0].copy_(first)
             mb.mlora_decode_step(ctx, ad, tok[j & 1], tok[(j + 1) & 1], None)
+
+        gen_out = None if hidden_io else torch.empty(GEN_STEPS, n, dtype=torch.int32, device=dev)
+
+        def run_steps(count):
+            """`count` decode steps as whole generations: per generation one call, one CUDA graph of GEN_STEPS steps with
+            the tokens fed back on the device (the last generation may be shorter)."""
+            done = 0
+            while done < count:
+                k = min(GEN_STEPS, count - done)
+                mb.mlora_reset_streams(ctx)
+                mb.mlora_generate(ctx, ad, first, gen_out[:k])
+                done += k
 
         def barrier():
             if world > 1:
@@ -697,6 +710,10 @@ def main():
             print_timeline(mb.mlora_step_timeline(ctx), cfg, mhz)
             model.close()
             return
+        if not hidden_io:
+            run_steps(min(K, 2 * GEN_STEPS))         # builds the generation graphs (full length and remainder)
+            if K % GEN_STEPS:
+                run_steps(K % GEN_STEPS)
         sampler = ClockSampler(local)
         sampler.start()
         barrier()
@@ -704,8 +721,11 @@ def main():
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0 = time.time()
         e0.record(side)
-        for i in range(K):
-            generation_step(W + i)
+        if hidden_io:
+            for i in range(K):
+                generation_step(W + i)
+        else:
+            run_steps(K)
         e1.record(side)
         barrier()
         t1 = time.time()
@@ -715,64 +735,94 @@ def main():
         ms_total = max_over_ranks(ms_total, world, dev)
         value = aggregate_tokens_per_s(world, n, K, ms_total)
 
-        # ---- end to end through the C ABI with HOST buffers: H2D of the step's inputs, D2H of its result
-        Ke = min(K, 512)
-        h_tok = torch.empty(n, dtype=torch.int32).pin_memory()
+        # ---- the same K steps as one graph replay per step (the single-step call a server with its own loop makes)
+        for i in range(GEN_STEPS):
+            generation_step(i)
+        barrier()
+        e0.record(side)
+        for i in range(K):
+            generation_step(i)
+        e1.record(side)
+        barrier()
+        ms_per_step_call = max_over_ranks(e0.elapsed_time(e1), world, dev) / K
+
+        # ---- end to end through the C ABI with HOST buffers: H2D of the inputs, D2H of the results, inside the call
+        Ke = min(K, 1024)
         h_ad = torch.arange(n, dtype=torch.int32).pin_memory()
-        h_next = torch.empty(n, dtype=torch.int32).pin_memory()
-        d_tok = torch.empty(n, dtype=torch.int32, device=dev)
-        d_ad = torch.empty(n, dtype=torch.int32, device=dev)
-        d_next = torch.empty(n, dtype=torch.int32, device=dev)
         if hidden_io:
             h_hin = torch.from_numpy(gen.make_hidden(cfg, n, 0, 1)).pin_memory()
             h_hout = torch.empty(n, cfg.d_model, dtype=torch.float32).pin_memory()
+            d_ad = torch.empty(n, dtype=torch.int32, device=dev)
             h2d, d2h = h_hin.numel() * 2 + n * 4, h_hout.numel() * 4
+
+            def e2e_run(count):
+                for i in range(count):
+                    if i % GEN_STEPS == 0:
+                        mb.mlora_reset_streams(ctx)
+                    d_ad.copy_(h_ad, non_blocking=True)
+                    hin.copy_(h_hin, non_blocking=True)
+                    mb.mlora_decode_step_h(ctx, d_ad, hin, hout)
+                    h_hout.copy_(hout, non_blocking=True)
+                    side.synchronize()              # the host reads the step's result
         else:
-            h_tok.copy_(first.cpu())
-            h2d, d2h = 2 * n * 4, n * 4
+            h_first = torch.empty(n, dtype=torch.int32).pin_memory()
+            h_first.copy_(first.cpu())
+            h_out = torch.empty(GEN_STEPS, n, dtype=torch.int32).pin_memory()
+            # per generation: adapter ids and first tokens in, all tokens of the generation out
+            h2d, d2h = 2 * n * 4 / GEN_STEPS, n * 4
 
-        def e2e_step(i):
-            j = i % GEN_STEPS
-            if j == 0:
-                mb.mlora_reset_streams(ctx)
-                if not hidden_io:
-                    h_tok.copy_(first_host)
-            if hidden_io:
-                d_ad.copy_(h_ad, non_blocking=True)
-                hin.copy_(h_hin, non_blocking=True)
-                mb.mlora_decode_step_h(ctx, d_ad, hin, hout)
-                h_hout.copy_(hout, non_blocking=True)
-                side.synchronize()                  # the host reads the step's result
-            else:
-                # host arrays in, host array out: the copies and the synchronisation happen inside the call
-                mb.mlora_decode_step_host(ctx, h_ad, h_tok, h_next)
-                h_tok.copy_(h_next)
+            def e2e_run(count):
+                done = 0
+                while done < count:
+                    k = min(GEN_STEPS, count - done)
+                    mb.mlora_reset_streams(ctx)
+                    mb.mlora_generate_host(ctx, h_ad, h_first, h_out[:k])     # copies in, runs, copies out, synchronises
+                    done += k
 
-        first_host = None if hidden_io else first.cpu()
-        for i in range(8):
-            e2e_step(i)
+        e2e_run(min(Ke, GEN_STEPS))
         barrier()
         e0.record(side)
-        for i in range(Ke):
-            e2e_step(8 + i)
+        e2e_run(Ke)
         e1.record(side)
         barrier()
         ms_e2e = e0.elapsed_time(e1)
         ms_e2e = max_over_ranks(ms_e2e, world, dev)
         e2e_value = aggregate_tokens_per_s(world, n, Ke, ms_e2e)
 
+        # ---- the single-step host-array call (one step per call, the host sees every token before the next step)
+        ms_e2e_step = None
+        if not hidden_io:
+            h_tok = torch.empty(n, dtype=torch.int32).pin_memory()
+            h_next = torch.empty(n, dtype=torch.int32).pin_memory()
+            Ks1 = min(K, 512)
+
+            def e2e_steps(count):
+                for i in range(count):
+                    if i % GEN_STEPS == 0:
+                        mb.mlora_reset_streams(ctx)
+                        h_tok.copy_(h_first)
+                    mb.mlora_decode_step_host(ctx, h_ad, h_tok, h_next)
+                    h_tok.copy_(h_next)
+            e2e_steps(8)
+            barrier()
+            e0.record(side)
+            e2e_steps(Ks1)
+            e1.record(side)
+            barrier()
+            ms_e2e_step = max_over_ranks(e0.elapsed_time(e1), world, dev) / Ks1
+
         # ---- the same steps through the single-kernel decode step (one cooperative launch per step), for comparison
         step_kernel_ms = None
         if not hidden_io:
             mb.mlora_debug_set(ctx, 6, 2)
             Ks = min(K, 1024)
-            for i in range(GEN_STEPS):
-                generation_step(i)
+            run_steps(GEN_STEPS)
+            if Ks % GEN_STEPS:
+                run_steps(Ks % GEN_STEPS)
             barrier()
             l1 = mb.mlora_launch_count(ctx)
             e0.record(side)
-            for i in range(Ks):
-                generation_step(i)
+            run_steps(Ks)
             e1.record(side)
             barrier()
             per_step = (mb.mlora_launch_count(ctx) - l1) / Ks
@@ -809,11 +859,16 @@ def main():
         "steps": K, "warmup": W, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f16", "data": "synthetic",
         "config": {"workload": workload_name(cfg), "streams": n, "l2": "inputs larger than L2: %.0f MB of weights, "
-                   "adapters and KV stream per step" % (step_bytes / 1e6), "launch": "CUDA-graph replay per step",
+                   "adapters and KV stream per step" % (step_bytes / 1e6), "launch": "CUDA-graph replay per step" if hidden_io else
+                   f"one call and one CUDA graph per generation of {GEN_STEPS} steps, tokens fed back on the device",
                    "multi_gpu": "replicas only"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": Ke, "ms_per_step": ms_e2e / Ke},
+                "steps": Ke, "ms_per_step": ms_e2e / Ke,
+                "call": "mlora_decode_step_h on device copies of pinned host arrays" if hidden_io else
+                "mlora_generate_host: host arrays in, the generation's tokens out, once per generation",
+                "single_step_call_ms_per_step": ms_e2e_step},
+        "per_step_graph_replay_ms_per_step": ms_per_step_call,
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "decode_chain_kernel (persistent INT4 GEMM + LoRA shrink/expand + norm), all launches of a step",
                      "achieved": achieved, "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",

@@ -110,6 +110,25 @@ int mlora_decode_step(mlora_ctx* ctx, int32_t n_streams, const int32_t* adapter_
  * returning.  Errors: as mlora_decode_step. */
 int mlora_decode_step_host(mlora_ctx* ctx, int32_t n_streams, const int32_t* adapter_idx_host,
                            const int32_t* tokens_host, int32_t* out_next_host);
+/* First tokens of the streams (App. A.1: after the single prefill a sampler picks n distinct tokens, one per stream).
+ * logits: dev fp32 [vocab] (the prefill's out_last_logits); out_tokens: dev int32 [n] = the ids of the n largest
+ * logits in order of falling logit, equal logits in order of rising id; NaN counts as the smallest value.
+ * 1 <= n <= vocab.  Enqueued on the context's stream.  Errors: ARG, STATE (no vocabulary), CUDA. */
+int mlora_sample_first(mlora_ctx* ctx, const float* logits, int32_t n, int32_t* out_tokens);
+/* A whole generation without host round trips (App. A.1 flowsheet: first tokens, then the n-fold generative model
+ * step after step): k_steps greedy decode steps of n_streams streams; step 0 consumes first_tokens, step j the tokens
+ * step j - 1 produced, read on the device.  out_tokens: dev int32 [k_steps][n_streams], row j = the tokens produced by
+ * step j (row k_steps - 1 is not yet in the cache, like out_next of mlora_decode_step).  Gives exactly the tokens
+ * and the cache that k_steps calls of mlora_decode_step give.  On a capturable stream the k_steps steps are ONE CUDA
+ * graph, cached by (pointers, k_steps, state of the own segments at the start).  adapter_idx, first_tokens: dev int32
+ * [n_streams].  Errors: ARG, STATE, CAPACITY (own segments cannot take k_steps more rows), CUDA. */
+int mlora_generate(mlora_ctx* ctx, int32_t n_streams, const int32_t* adapter_idx, const int32_t* first_tokens,
+                   int32_t k_steps, int32_t* out_tokens);
+/* The same with HOST arrays (adapter_idx_host, first_tokens_host: [n_streams]; out_tokens_host: [k_steps][n_streams]):
+ * copies in, runs, copies out and synchronises.  The device buffer behind out_tokens_host is allocated at the
+ * first call of a larger k_steps * n_streams than any before. */
+int mlora_generate_host(mlora_ctx* ctx, int32_t n_streams, const int32_t* adapter_idx_host,
+                        const int32_t* first_tokens_host, int32_t k_steps, int32_t* out_tokens_host);
 /* Hidden-state variant: hidden_in dev fp16 [n_streams][d_model]; hidden_out dev fp32 [n_streams][d_model]
  * (residual stream after the last layer). */
 int mlora_decode_step_h(mlora_ctx* ctx, int32_t n_streams, const int32_t* adapter_idx, const void* hidden_in,

@@ -17,6 +17,9 @@ What follows which passage:
     a node sees the cached context plus its own ancestors               -- Sec. 3.5, App. A.2 (DS2D mask)
   * accepted drafts form one root path ("1-3-5"); first emitted token is
     the frozen model's own token (lossless)                              -- Sec. 3.5
+  * after the single prefill a sampler gives the n streams n distinct
+    first tokens (here: the n most probable, by falling logit, ties by
+    rising id), then the n-fold model runs step after step              -- App. A.1 (flowsheet)
 
 Arithmetic: everything after dequantisation is carried in ``dtype`` (float64 by default; float32
 for the 1B/3B shapes where the dense weights would not fit twice in memory).  No blocking, no
@@ -30,7 +33,8 @@ decode of each root path; shared-prefix attention against plain causal attention
 concatenated sequence; RoPE/RMSNorm/SiLU closed forms; accept walk against brute force on every
 small tree; the (3,2) -> 9/10/30 node counts and the 32-row budgets of Table 7; the wiring of a decoder block
 (norm placement, residuals, gate/up roles, final norm) against scalar loops written from the definitions
-(tests/test_oracle_wiring_pin.py).
+(tests/test_oracle_wiring_pin.py); the first-token sampler against exhaustive selection on small rows with ties and
+against argmax for n = 1 (tests/test_oracle_generate.py).
 Parity unpinned by the paper: absolute activation values of a forward pass of ITS model (it prints none).
 """
 import numpy as np
@@ -208,6 +212,18 @@ def accept_walk(tokens, parent, argmax):
         path.append(c)
 
 
+def first_tokens(logits, n):
+    """The n distinct first tokens of the streams (App. A.1): the ids of the n largest logits, listed by
+    falling logit, equal logits by rising id.  NaN ranks below every number."""
+    vals = [float(v) for v in np.asarray(logits).reshape(-1)]
+    vals = [float("-inf") if v != v else v for v in vals]
+    nan_ids = {i for i, v in enumerate(np.asarray(logits).reshape(-1)) if v != v}
+    # a NaN ranks below a true -inf: second sort key
+    order = sorted(range(len(vals)), key=lambda i: (-vals[i], i in nan_ids, i))
+    assert 1 <= n <= len(vals)
+    return np.array(order[:n], dtype=np.int32)
+
+
 # ----------------------------------------------------------------------------- the model
 class OracleModel:
     """Dense CPU model with a shared-prefix KV segment and one private KV segment per stream."""
@@ -373,6 +389,17 @@ class OracleModel:
                     self.suf_k[l][s] = np.concatenate([self.suf_k[l][s], new_k[l][rows]], axis=0)
                     self.suf_v[l][s] = np.concatenate([self.suf_v[l][s], new_v[l][rows]], axis=0)
         return out
+
+    def generate(self, adapter_idx, first, k_steps):
+        """k greedy decode steps, every stream fed its own previous token (App. A.1: the n-fold generative model run
+        step after step).  Returns (tokens [k][n]: row j = produced by step j, logits [k][n][vocab])."""
+        toks, out, lg = np.asarray(first, dtype=np.int32), [], []
+        for _ in range(k_steps):
+            r = self.decode_step(adapter_idx, tokens=toks)
+            toks = np.asarray(r["next"], dtype=np.int32)
+            out.append(toks)
+            lg.append(r["logits"])
+        return np.stack(out), np.stack(lg)
 
     def decode_step(self, adapter_idx, tokens=None, hidden=None, follow_argmax=None):
         """One token per stream: a verify pass whose tree is the root alone."""

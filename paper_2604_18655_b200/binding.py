@@ -54,6 +54,9 @@ _SIGS = {
     "mlora_last_error": (C.c_char_p, [C.c_void_p]),
     "mlora_export_kv": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_int32),
                                   C.c_void_p, C.c_void_p]),
+    "mlora_sample_first": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]),
+    "mlora_generate": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]),
+    "mlora_generate_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]),
     "mlora_export_state": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int32), C.c_void_p, C.c_void_p]),
     "mlora_debug_dequant": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "mlora_debug_set": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32]),
@@ -183,6 +186,25 @@ def mlora_verify_tree(ctx, adapter_idx, tree_tokens, tree_parent, out_accept_len
     n, T = tree_tokens.shape
     _check(lib().mlora_verify_tree(ctx, n, _ptr(adapter_idx), T, _ptr(tree_tokens), _ptr(tree_parent),
                                    _ptr(out_accept_len), _ptr(out_accept_idx), _ptr(out_next), _ptr(out_logits)))
+
+
+def mlora_sample_first(ctx, logits, out_tokens):
+    _check(lib().mlora_sample_first(ctx, _ptr(logits), out_tokens.numel(), _ptr(out_tokens)))
+
+
+def mlora_generate(ctx, adapter_idx, first_tokens, out_tokens):
+    """out_tokens: device int32 [k_steps][n_streams]"""
+    k, n = out_tokens.shape
+    _check(lib().mlora_generate(ctx, n, _ptr(adapter_idx), _ptr(first_tokens), k, _ptr(out_tokens)))
+
+
+def mlora_generate_host(ctx, adapter_idx, first_tokens, out_tokens):
+    """host (CPU) int32 tensors: adapter_idx, first_tokens [n_streams]; out_tokens [k_steps][n_streams]"""
+    k, n = out_tokens.shape
+    for t in (adapter_idx, first_tokens, out_tokens):
+        assert not t.is_cuda and t.is_contiguous() and t.dtype == torch.int32
+    _check(lib().mlora_generate_host(ctx, n, C.c_void_p(adapter_idx.data_ptr()), C.c_void_p(first_tokens.data_ptr()), k,
+                                     C.c_void_p(out_tokens.data_ptr())))
 
 
 def mlora_reset_streams(ctx):

@@ -292,6 +292,7 @@ bool attn_single_pass(const AttnArgs& a);          // one kernel does the whole 
 cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st);
 cudaError_t launch_attention_merge(const AttnArgs& a, cudaStream_t st);
 cudaError_t launch_argmax(const float* logits, int M, int V, int32_t* out, cudaStream_t st);
+cudaError_t launch_topn(const float* logits, int V, int n, int32_t* out, cudaStream_t st);
 cudaError_t launch_accept(const int32_t* tokens, const int32_t* parent, const int32_t* argmax, int n, int T,
                           int32_t* acc_len, int32_t* acc_idx, int32_t* next, cudaStream_t st);
 cudaError_t launch_compact(__half* own_k, __half* own_v, size_t layer_stride, size_t stream_stride,

@@ -99,6 +99,8 @@ struct mlora_ctx {
   int dbg_skip_compact = 0, dbg_no_graph = 0, dbg_no_chain = 0, dbg_no_tc = 0, dbg_inject_stall = 0;
   int step_mode = 0;                 // decode steps: 0 = the library's choice, 1 = per-layer kernels, 2 = the single-kernel step
   int32_t* host_io = nullptr;        // dev [3][max_streams]: adapter_idx, tokens, next of the host-buffer step
+  int32_t* gen_tokens = nullptr;     // dev [k][n]: the tokens of a host-buffer generation (grown on demand)
+  size_t gen_capacity = 0;
   // persistent projection chain (rows <= 8)
   ChainPhase* phases = nullptr;      // dev [4*L (+1)]: qkv, o, gate/up, down per layer; then lm_head
   int n_phases = 0;
@@ -886,7 +888,7 @@ int mlora_destroy(mlora_ctx* c) {
                       c->h, c->attn16, c->act16, c->counters, c->anc, c->depth, c->argmax, c->suffix_len,
                       c->zero_len, c->chain_parent, c->root_parent, c->status, c->cs_table, (void*)c->tabA,
                       (void*)c->tabB, c->ad_scale, c->phases, c->chain_sync, c->host_io, c->step_phases, c->xg_attn, c->xg_ffn,
-                      c->step_tacc, c->step_ssq, c->step_amax, c->step_trace, c->tmapA, c->tmapB};
+                      c->step_tacc, c->step_ssq, c->step_amax, c->step_trace, c->tmapA, c->tmapB, c->gen_tokens};
   for (void* p : dev_ptrs) if (p) cudaFree(p);
   if (c->stageA) cudaFreeHost((void*)c->stageA);
   if (c->stageB) cudaFreeHost((void*)c->stageB);
@@ -1027,6 +1029,90 @@ int mlora_decode_step_host(mlora_ctx* c, int32_t n_streams, const int32_t* adapt
   int rc = decode_impl(c, n_streams, d_ad, d_tok, nullptr, d_next, nullptr, nullptr);
   if (rc != MLORA_OK) return rc;
   CK(cudaMemcpyAsync(out_next_host, d_next, bytes, cudaMemcpyDeviceToHost, c->stream));
+  CK(cudaStreamSynchronize(c->stream));
+  return MLORA_OK;
+}
+
+int mlora_sample_first(mlora_ctx* c, const float* logits, int32_t n, int32_t* out_tokens) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (c->d.vocab == 0) return fail(MLORA_ERR_STATE, "context has no vocabulary");
+  if (!logits || !out_tokens) return fail(MLORA_ERR_ARG, "logits/out_tokens is null");
+  if (n < 1 || n > c->d.vocab) return fail(MLORA_ERR_ARG, "n must be between 1 and the vocabulary size");
+  CK(run(c, MLORA_PROF_MISC, [&] { return launch_topn(logits, c->d.vocab, n, out_tokens, c->stream); }));
+  return MLORA_OK;
+}
+
+// k decode steps enqueued back to back (captured as ONE graph where the stream allows it): step j reads the tokens that
+// step j - 1 wrote, on the device
+static int generate_impl(mlora_ctx* c, int n, const int32_t* adapter_idx, const int32_t* first, int k, int32_t* out) {
+  int rc = step_common_checks(c, n, adapter_idx, 1);
+  if (rc != MLORA_OK) return rc;
+  if (k > 1) { rc = ensure_capacity(c, k); if (rc != MLORA_OK) return rc; }
+  const int bound0 = c->suffix_bound;
+  GraphKey key{};
+  key.kind = 4; key.n = n; key.T = k;
+  key.flags = c->P * 16 + c->step_mode * 4 + c->dbg_inject_stall * 2 + c->dbg_no_chain;
+  key.suffix_bound = bound0;                           // every step's launch shapes follow from the bound at the start
+  key.p[0] = adapter_idx; key.p[1] = first; key.p[2] = out;
+  rc = replay_or_run(c, key, [&]() -> int {
+    for (int j = 0; j < k; ++j) {
+      const int32_t* tok = j ? out + (size_t)(j - 1) * n : first;
+      int32_t* next = out + (size_t)j * n;
+      if (step_eligible(c, n, 1)) {
+        int r = forward_step(c, n, adapter_idx, tok, nullptr, next, nullptr, nullptr);
+        if (r != MLORA_OK) return r;
+        continue;
+      }
+      PassIO io;
+      io.n = n; io.T = 1; io.tokens = tok; io.adapter_idx = adapter_idx;
+      io.parent = c->root_parent; io.pos_base = c->P; io.suffix_len = c->suffix_len; io.suffix_bound = bound0 + j;
+      io.logits = c->logits;
+      plan_pass(c, io);
+      int r = forward(c, io);
+      if (r != MLORA_OK) return r;
+      CK(run(c, MLORA_PROF_MISC, [&] { return launch_argmax(io.logits, n, c->d.vocab, next, c->stream); }));
+      CK(run(c, MLORA_PROF_MISC, [&] { return launch_advance(c->suffix_len, nullptr, n, 1, c->stream); }));
+    }
+    return MLORA_OK;
+  });
+  if (rc != MLORA_OK) return rc;
+  c->suffix_bound += k;
+  if (c->snap_pending) c->snap_inc += k;
+  return MLORA_OK;
+}
+
+int mlora_generate(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_idx, const int32_t* first_tokens, int32_t k_steps,
+                   int32_t* out_tokens) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (c->d.vocab == 0) return fail(MLORA_ERR_STATE, "context has no vocabulary");
+  if (!first_tokens || !out_tokens) return fail(MLORA_ERR_ARG, "first_tokens/out_tokens is null");
+  if (k_steps < 1) return fail(MLORA_ERR_ARG, "k_steps must be at least 1");
+  return generate_impl(c, n_streams, adapter_idx, first_tokens, k_steps, out_tokens);
+}
+
+int mlora_generate_host(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_idx_host, const int32_t* first_tokens_host,
+                        int32_t k_steps, int32_t* out_tokens_host) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (c->d.vocab == 0) return fail(MLORA_ERR_STATE, "context has no vocabulary");
+  if (!adapter_idx_host || !first_tokens_host || !out_tokens_host) return fail(MLORA_ERR_ARG, "null host buffer");
+  if (n_streams <= 0 || n_streams > c->d.max_streams) return fail(MLORA_ERR_ARG, "n_streams out of range");
+  if (k_steps < 1) return fail(MLORA_ERR_ARG, "k_steps must be at least 1");
+  const size_t need = (size_t)k_steps * n_streams;
+  if (need > c->gen_capacity) {                        // (grown outside any timed loop: the first call of a new size)
+    CK(cudaStreamSynchronize(c->stream));
+    if (c->gen_tokens) cudaFree(c->gen_tokens);
+    c->gen_tokens = nullptr; c->gen_capacity = 0;
+    CK(cudaMalloc(&c->gen_tokens, need * sizeof(int32_t)));
+    c->gen_capacity = need;
+  }
+  int32_t* d_ad = c->host_io;
+  int32_t* d_tok = c->host_io + c->d.max_streams;
+  const size_t bytes = (size_t)n_streams * sizeof(int32_t);
+  CK(cudaMemcpyAsync(d_ad, adapter_idx_host, bytes, cudaMemcpyHostToDevice, c->stream));
+  CK(cudaMemcpyAsync(d_tok, first_tokens_host, bytes, cudaMemcpyHostToDevice, c->stream));
+  int rc = generate_impl(c, n_streams, d_ad, d_tok, k_steps, c->gen_tokens);
+  if (rc != MLORA_OK) return rc;
+  CK(cudaMemcpyAsync(out_tokens_host, c->gen_tokens, need * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
   CK(cudaStreamSynchronize(c->stream));
   return MLORA_OK;
 }

@@ -1,6 +1,6 @@
 // Small kernels around the projections: embedding gather, draft-tree preparation (ancestor masks and
-// depths, Sec. 3.5 / App. A.2), row argmax, the greedy longest-accepted-path walk and the KV compaction that
-// follows it (Sec. 3.5).  (RoPE and the KV append of a pass happen inside the attention kernel.)
+// depths, Sec. 3.5 / App. A.2), row argmax, the streams' first tokens (App. A.1), the greedy longest-accepted-path
+// walk and the KV compaction that follows it (Sec. 3.5).  (RoPE and the KV append of a pass happen inside the attention kernel.)
 #include "common.cuh"
 
 namespace mlora {
@@ -122,6 +122,58 @@ __global__ void argmax_kernel(const float* __restrict__ logits, int V, int32_t* 
 
 cudaError_t launch_argmax(const float* logits, int M, int V, int32_t* out, cudaStream_t st) {
   argmax_kernel<<<M, 1024, 0, st>>>(logits, V, out);
+  return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------- first tokens of the streams (App. A.1)
+// After the shared prefill a sampler hands every stream a different first token: the n most probable ids of the
+// prefill's last logits, in order of falling logit, equal logits by rising id.  One CTA; round i finds the largest
+// key below round i-1's winner.  Key = order-preserving image of the float in the high word (NaN lowest), the
+// complemented id in the low word: one unsigned compare gives both rules.  The n rounds re-read the row from L2.
+__device__ __forceinline__ unsigned long long topn_key(float v, int i) {
+  if (v == 0.f) v = 0.f;                                // -0 and +0 are equal logits: one image for both
+  const unsigned b = __float_as_uint(v);
+  const unsigned ord = (v != v) ? 0u : ((b & 0x80000000u) ? ~b : (b | 0x80000000u));
+  return ((unsigned long long)ord << 32) | (unsigned)(0xffffffffu - (unsigned)i);
+}
+
+__global__ void __launch_bounds__(1024) topn_kernel(const float* __restrict__ logits, int V, int n, int32_t* __restrict__ out) {
+  __shared__ unsigned long long sb[32];
+  __shared__ unsigned long long s_prev;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  unsigned long long prev = ~0ull;
+  for (int r = 0; r < n; ++r) {
+    unsigned long long best = 0ull;                     // below every key (ids are below 2^31: a key's low word is not 0)
+    for (int i = threadIdx.x; i < V; i += blockDim.x) {
+      const unsigned long long k = topn_key(logits[i], i);
+      if (k < prev && k > best) best = k;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+      best = ob > best ? ob : best;
+    }
+    if (lane == 0) sb[warp] = best;
+    __syncthreads();
+    if (warp == 0) {
+      best = sb[lane];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+        best = ob > best ? ob : best;
+      }
+      if (lane == 0) {
+        s_prev = best;
+        out[r] = (int32_t)(0xffffffffu - (unsigned)(best & 0xffffffffull));
+      }
+    }
+    __syncthreads();
+    prev = s_prev;
+  }
+}
+
+cudaError_t launch_topn(const float* logits, int V, int n, int32_t* out, cudaStream_t st) {
+  topn_kernel<<<1, 1024, 0, st>>>(logits, V, n, out);
   return cudaGetLastError();
 }
 

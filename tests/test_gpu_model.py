@@ -433,6 +433,86 @@ def test_export_state_gives_the_whole_own_segment(GpuModel):
     gm.close()
 
 
+def test_sample_first_matches_oracle(GpuModel):
+    """The n distinct first tokens (App. A.1): integer work, exact -- with ties, infinities, signed zeros and NaN."""
+    from paper_2604_18655_b200 import binding as mb
+    cfg = TINYV
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=8)
+    rng = np.random.default_rng(3)
+    rows = [np.round(rng.standard_normal(cfg.vocab) * 2) / 2, rng.standard_normal(cfg.vocab), np.zeros(cfg.vocab)]
+    special = rng.standard_normal(cfg.vocab)
+    special[[5, 9]] = np.nan
+    special[[7, 70]] = np.inf
+    special[[1, 100]] = -np.inf
+    special[[30, 31]] = [-0.0, 0.0]
+    rows.append(special)
+    for row in rows:
+        row = row.astype(np.float32)
+        for n in (1, 3, 8, cfg.vocab):
+            out = torch.full((n,), -7, dtype=torch.int32, device="cuda")
+            mb.mlora_sample_first(gm.ctx, torch.from_numpy(row).cuda(), out)
+            torch.cuda.synchronize()
+            assert np.array_equal(out.cpu().numpy(), ref.first_tokens(row, n))
+    with pytest.raises(mb.MloraError):
+        mb.mlora_sample_first(gm.ctx, torch.zeros(cfg.vocab, device="cuda"), torch.zeros(cfg.vocab + 1, dtype=torch.int32, device="cuda"))
+    gm.close()
+
+
+@pytest.mark.parametrize("step_path", STEP_PATHS)
+def test_generation_in_one_call_matches_step_by_step(GpuModel, step_path):
+    """prefill -> sampler -> k steps with the tokens fed back on the device: the same tokens and the same cache, bit for
+    bit, as k single-step calls; the tokens are the oracle's wherever its margin decides; twice (the second call
+    replays the graph of the first)."""
+    from paper_2604_18655_b200 import binding as mb
+    cfg, k = TINYV, 12
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        m, orc, gm = make_pair(GpuModel, cfg, step_path=step_path, max_suffix=16)
+        ids = gen.make_prompt_ids(cfg, 0)
+        last = torch.from_numpy(gm.prefill(ids)).cuda()
+        want_last = orc.prefill_shared(ids, n_streams=cfg.n_streams)
+        n = cfg.n_streams
+        first = torch.empty(n, dtype=torch.int32, device="cuda")
+        mb.mlora_sample_first(gm.ctx, last, first)
+        assert np.array_equal(first.cpu().numpy(), ref.first_tokens(last.cpu().numpy(), n))
+        ad = [1, -1, 0]
+        d_ad = torch.tensor(ad, dtype=torch.int32, device="cuda")
+        # step by step
+        toks, steps = first.cpu().numpy(), []
+        for _ in range(k):
+            toks, _ = gm.decode(ad, toks, want_logits=False)
+            steps.append(toks)
+        steps = np.stack(steps)
+        kv = [gm.export_kv(l, s, 0, k) for l in range(cfg.n_layers) for s in range(n)]
+        for rep in range(2):
+            mb.mlora_reset_streams(gm.ctx)
+            out = torch.full((k, n), -1, dtype=torch.int32, device="cuda")
+            mb.mlora_generate(gm.ctx, d_ad, first, out)
+            side.synchronize()
+            assert np.array_equal(out.cpu().numpy(), steps), f"call {rep}"
+            kv2 = [gm.export_kv(l, s, 0, k) for l in range(cfg.n_layers) for s in range(n)]
+            for (s1, k1, v1), (s2, k2, v2) in zip(kv, kv2):
+                assert s1 == s2 == k
+                assert np.array_equal(k1.view(np.uint16), k2.view(np.uint16)) and np.array_equal(v1.view(np.uint16), v2.view(np.uint16))
+        # host-array form
+        mb.mlora_reset_streams(gm.ctx)
+        h_out = torch.empty(k, n, dtype=torch.int32).pin_memory()
+        mb.mlora_generate_host(gm.ctx, torch.tensor(ad, dtype=torch.int32), first.cpu(), h_out)
+        assert np.array_equal(h_out.numpy(), steps)
+        # the oracle, walked along the GPU's tokens
+        toks = first.cpu().numpy()
+        for j in range(k):
+            r = orc.decode_step(ad, tokens=toks)
+            check_argmax(steps[j], r["logits"], f"generation step {j}")
+            toks = steps[j]
+        # the own segments cannot take another k rows on top: CAPACITY, nothing enqueued
+        with pytest.raises(mb.MloraError) as e:
+            mb.mlora_generate(gm.ctx, d_ad, first, out)
+        assert e.value.code == -3
+        mb.mlora_sync_status(gm.ctx)
+        gm.close()
+
+
 def test_host_buffer_step_matches_device_step(GpuModel):
     """mlora_decode_step_host (host arrays in and out) gives the tokens of mlora_decode_step."""
     from paper_2604_18655_b200 import binding as mb

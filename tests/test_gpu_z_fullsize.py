@@ -102,17 +102,25 @@ def test_llama1b_full_prompt_sixteen_steps(step_path):
         n = cfg.n_streams
         ad = list(range(n))
         toks = np.argsort(-want_last)[:n].astype(np.int32)
+        first, produced = toks, []
         for step in range(16):
             nxt, logits = gm.decode(ad, toks)
             r = orc.decode_step(ad, tokens=toks)
             compare(logits, r["logits"], f"llama1b full-prompt decode logits step {step}")
             check_argmax(nxt, r["logits"], f"llama1b full-prompt decode step {step}")
             toks = nxt
+            produced.append(nxt)
         for s in (0, n - 1):
             got_s, k, v = gm.export_kv(cfg.n_layers - 1, s, 0, 16)
             assert got_s == 16
             compare(k, orc.suf_k[cfg.n_layers - 1][s], f"suffix K stream {s}")
             compare(v, orc.suf_v[cfg.n_layers - 1][s], f"suffix V stream {s}")
+        # the same generation as ONE call (one graph of 16 steps, tokens fed back on the device): the same tokens
+        mb.mlora_reset_streams(gm.ctx)
+        out = torch.empty(16, n, dtype=torch.int32, device="cuda")
+        mb.mlora_generate(gm.ctx, torch.tensor(ad, dtype=torch.int32, device="cuda"), torch.from_numpy(first).cuda(), out)
+        side.synchronize()
+        assert np.array_equal(out.cpu().numpy(), np.stack(produced))
         mb.mlora_sync_status(gm.ctx)
         gm.close()
 
