@@ -30,9 +30,12 @@ sys.path.insert(0, ROOT)
 GEN_STEPS = 128          # decode steps per generation (per stream) before the streams are reset
 ORACLE_PREFIX = 64       # prompt length used for the CPU-baseline sample (the 512-token prefill is not timed work)
 L2_BYTES = 126e6
-# DRAM bytes (read + write counters of one ncu capture) per launch of the dominant kernel, by workload; None where
-# no capture of the kernel as it stands exists
-NCU_DRAM_BYTES_PER_LAUNCH = {"cfg1": None}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture) per launch of the dominant kernel, by
+# workload; None where no capture of the kernel as it stands exists.  cfg1: decode_chain_kernel captured on a 4-layer
+# cut of the model (the launches of a layer are the same at any depth): 7.86 MB for the first launch of a step
+# (q,k,v only), 34.87 MB for each per-layer launch, the last launch (with the lm_head) taken at its algorithmic
+# 60 MB, averaged over the 17 launches of a full-model step
+NCU_DRAM_BYTES_PER_LAUNCH = {"cfg1": 34.8e6}
 
 
 def parse_args():
@@ -736,7 +739,7 @@ def main():
         value = aggregate_tokens_per_s(world, n, K, ms_total)
 
         # ---- the same K steps as one graph replay per step (the single-step call a server with its own loop makes)
-        for i in range(GEN_STEPS):
+        for i in range(min(GEN_STEPS, K)):
             generation_step(i)
         barrier()
         e0.record(side)
@@ -816,7 +819,7 @@ def main():
         if not hidden_io:
             mb.mlora_debug_set(ctx, 6, 2)
             Ks = min(K, 1024)
-            run_steps(GEN_STEPS)
+            run_steps(min(GEN_STEPS, Ks))
             if Ks % GEN_STEPS:
                 run_steps(Ks % GEN_STEPS)
             barrier()
