@@ -9,7 +9,10 @@
 // streams and all query heads of the kv head; an own-segment chunk is used by that stream's rows.
 // QK^T and PV run on the tensor cores (mma.sync m16n8k16, fp32 accumulate), K/V tiles are staged through
 // shared memory with a two-stage cp.async pipeline.
-#include "common.cuh"
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include "pipe.cuh"
 
 namespace mlora {
 
@@ -304,45 +307,51 @@ __device__ __forceinline__ void attn_partial_body(const AttnArgs& p, const int r
 // log-sum-exp merge of the chunks of virtual row v (row m, query head hq) of kv head kh by one warp.  The lanes
 // take the chunks' (max, sum) pairs side by side; the weighted sum over chunks runs in chunk order with
 // independent loads.
+template <int FAST>
+__device__ __forceinline__ void merge_row_fast(const AttnArgs& p, size_t base, int n_valid, __half* out, int lane) {
+  // one round trip: every load is issued before the first use; the partial outputs of FAST chunks sit in registers
+  const int hd = p.hd;
+  float2 ml = make_float2(-INFINITY, 0.f);
+  if (lane < n_valid) ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (base + lane) * 2));
+  float po[FAST][4];
+#pragma unroll
+  for (int i = 0; i < FAST; ++i)
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      po[i][e] = (i < n_valid && e * 32 + lane < hd) ? __ldcg(p.part_o + (base + i) * hd + e * 32 + lane) : 0.f;
+  float mmax = ml.x;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, o));
+  const float wgt = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - mmax);
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  float L = 0.f;
+#pragma unroll
+  for (int i = 0; i < FAST; ++i) {                                     // fixed order: chunk 0, 1, ...
+    const float wi = __shfl_sync(0xffffffffu, wgt, i);
+    L = fmaf(wi, __shfl_sync(0xffffffffu, ml.y, i), L);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) acc[e] = fmaf(wi, po[i][e], acc[e]);
+  }
+  const float inv = 1.f / L;
+#pragma unroll
+  for (int e = 0; e < 4; ++e)
+    if (e * 32 + lane < hd) out[e * 32 + lane] = __float2half_rn(acc[e] * inv);
+}
+
 __device__ __forceinline__ void merge_row(const AttnArgs& p, int kh, int v, int m, int hq, int lane) {
   const int g_heads = p.Hq / p.Hkv;
   const int R_all = p.n * p.T * g_heads;
   const int slots = p.n_prefix_chunks + p.n_own_chunks;
   const int s = m / p.T;
-  const int own_valid = min(p.n_own_chunks, (p.suffix_len[s] + p.T + p.own_chunk - 1) / p.own_chunk);
+  // (a single own chunk always holds the pass's own rows: no need to wait for the suffix length)
+  const int own_valid = p.n_own_chunks == 1 ? 1 : min(p.n_own_chunks, (p.suffix_len[s] + p.T + p.own_chunk - 1) / p.own_chunk);
   const int n_valid = p.n_prefix_chunks + own_valid;
   const size_t base = ((size_t)kh * R_all + v) * slots;
   const int hd = p.hd;
   __half* out = p.out + ((size_t)m * p.Hq + hq) * hd;
-  constexpr int FAST = 12;                             // chunks whose partial outputs fit in registers
-  if (n_valid <= FAST && hd <= 128) {
-    // one round trip: every load is issued before the first use
-    float2 ml = make_float2(-INFINITY, 0.f);
-    if (lane < n_valid) ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (base + lane) * 2));
-    float po[FAST][4];
-#pragma unroll
-    for (int i = 0; i < FAST; ++i)
-#pragma unroll
-      for (int e = 0; e < 4; ++e)
-        po[i][e] = (i < n_valid && e * 32 + lane < hd) ? __ldcg(p.part_o + (base + i) * hd + e * 32 + lane) : 0.f;
-    float mmax = ml.x;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, o));
-    const float wgt = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - mmax);
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    float L = 0.f;
-#pragma unroll
-    for (int i = 0; i < FAST; ++i) {                                     // fixed order: chunk 0, 1, ...
-      const float wi = __shfl_sync(0xffffffffu, wgt, i);
-      L = fmaf(wi, __shfl_sync(0xffffffffu, ml.y, i), L);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) acc[e] = fmaf(wi, po[i][e], acc[e]);
-    }
-    const float inv = 1.f / L;
-#pragma unroll
-    for (int e = 0; e < 4; ++e)
-      if (e * 32 + lane < hd) out[e * 32 + lane] = __float2half_rn(acc[e] * inv);
-    return;
+  if (hd <= 128) {
+    if (n_valid <= 12) { merge_row_fast<12>(p, base, n_valid, out, lane); return; }
+    if (n_valid <= 24) { merge_row_fast<24>(p, base, n_valid, out, lane); return; }
   }
   float mmax = -INFINITY;
   for (int i = lane; i < n_valid; i += 32) mmax = fmaxf(mmax, __ldcg(p.part_ml + (base + i) * 2));
@@ -667,13 +676,381 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+
+// ----------------------------------------------------------------------------- streaming decode attention
+// One decode row per stream and a LONG shared prefix (Sec. 3.4, App. A.1: every stream's row attends to the same
+// prefill segment): the prefix is cut into one chunk per SM and kv head, and the CTA of a chunk serves the rows of ALL
+// streams and all query heads of the kv head (at most 32 rows = two m16 tiles), so the prefix crosses HBM and L2 once.
+// A producer warp streams 64-key K and V tiles through a 4-stage ring with tiled TMA copies (tensor maps over the
+// prefix, 128-byte swizzle, rows past the prefix zero-filled, completion on mbarriers); eight consumer warps take
+// (row tile, 16 keys of the tile) each, with their own online softmax, and are combined by log-sum-exp in shared
+// memory at the end of the chunk.  The first n * Hkv CTAs also do one (stream, kv head) own segment each: its first
+// two tiles are fetched with cp.async into the same swizzled layout while the prefix streams (the new row is built
+// from the projections, rotated, and appended).  Partial results per (row, chunk) go to the scratch that
+// attn_merge_kernel combines.
+constexpr int STR_KEYS = 64;
+constexpr int STR_CWARPS = 8;
+constexpr int STR_THREADS = (STR_CWARPS + 1) * 32;
+constexpr int STR_STAGES = 4;
+constexpr int STR_ROWS = 32;
+constexpr int STR_OWN_TILES = 2;                          // own tiles fetched ahead, in shared memory of their own
+constexpr long long STR_WAIT_CYCLES = 2000000000ll;       // ~1 s
+__host__ __device__ constexpr size_t str_stage_bytes(int hd) { return (size_t)2 * STR_KEYS * hd * 2; }
+__host__ __device__ constexpr size_t str_smem_bytes(int hd) {
+  return 1024 + (STR_STAGES + STR_OWN_TILES) * str_stage_bytes(hd) + (size_t)(STR_ROWS + 16) * (hd + 8) * 2 + 128;
+}
+
+__device__ __forceinline__ void tma_tile_3d(uint32_t dst, const void* tmap, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+// byte offset of the 16-byte piece `piece` (0 .. hd/8 - 1) of row `row` in a [64][hd] tile stored as hd/64 column
+// halves of [64 rows][128 bytes], each with the 128-byte swizzle (piece index xor row mod 8)
+__device__ __forceinline__ uint32_t str_off(int row, int piece) {
+  return (uint32_t)((piece >> 3) * (STR_KEYS * 128) + row * 128 + (((piece & 7) ^ (row & 7)) << 4));
+}
+// bounded mbarrier wait: false once the CTA has given up (the flag is shared; the first to run out sets the status)
+__device__ __forceinline__ bool str_wait(uint32_t bar, uint32_t parity, volatile int* s_abort, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (int it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 127) == 127) {
+      if (*s_abort) return false;
+      if (clock64() - t0 > STR_WAIT_CYCLES) {
+        *s_abort = 1;
+        if (status) atomicCAS(status, 0, MLORA_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+// one warp: 16 query rows (fragments qf) against 16 keys (rows key16 .. key16+15 of the K and V tiles at kt / vt),
+// online softmax update of (o, mrow, lrow).  n_valid = number of valid keys among the 16.
+template <int HD>
+__device__ __forceinline__ void str_tile16(const uint32_t (&qf)[HD / 16][4], uint32_t kt, uint32_t vt, int key16, int n_valid,
+                                           float scale_log2, float (&o)[HD / 8][4], float (&mrow)[2], float (&lrow)[2]) {
+  constexpr int KSTEPS = HD / 16, DT = HD / 8;
+  const int lane = threadIdx.x & 31, t = lane & 3, mi = lane >> 3, r = lane & 7;
+  float sacc[2][4];
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
+    const int row = key16 + nt * 8 + r;
+#pragma unroll
+    for (int ks = 0; ks < KSTEPS; ks += 2) {
+      uint32_t kb[4];
+      asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                   : "=r"(kb[0]), "=r"(kb[1]), "=r"(kb[2]), "=r"(kb[3]) : "r"(kt + str_off(row, ks * 2 + mi)));
+      mma_16816(sacc[nt], qf[ks], kb[0], kb[1]);
+      mma_16816(sacc[nt], qf[ks + 1], kb[2], kb[3]);
+    }
+  }
+  float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int key = nt * 8 + 2 * t + (e & 1);
+      const float v = key < n_valid ? sacc[nt][e] * scale_log2 : -INFINITY;
+      sacc[nt][e] = v;
+      mx[e >> 1] = fmaxf(mx[e >> 1], v);
+    }
+  }
+  float corr[2], msafe[2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+    mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
+    const float mnew = fmaxf(mrow[h], mx[h]);
+    msafe[h] = (mnew == -INFINITY) ? 0.f : mnew;
+    corr[h] = exp2f(mrow[h] - msafe[h]);
+    mrow[h] = mnew;
+  }
+  uint32_t pf[4];
+  float ls[2] = {0.f, 0.f};
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    const float p0 = exp2f(sacc[nt][0] - msafe[0]), p1 = exp2f(sacc[nt][1] - msafe[0]);
+    const float p2 = exp2f(sacc[nt][2] - msafe[1]), p3 = exp2f(sacc[nt][3] - msafe[1]);
+    ls[0] += p0 + p1;
+    ls[1] += p2 + p3;
+    pf[nt * 2 + 0] = h2_as_u32(__floats2half2_rn(p0, p1));
+    pf[nt * 2 + 1] = h2_as_u32(__floats2half2_rn(p2, p3));
+  }
+#pragma unroll
+  for (int h = 0; h < 2; ++h) lrow[h] = lrow[h] * corr[h] + ls[h];
+#pragma unroll
+  for (int dt = 0; dt < DT; ++dt) {
+    o[dt][0] *= corr[0]; o[dt][1] *= corr[0];
+    o[dt][2] *= corr[1]; o[dt][3] *= corr[1];
+  }
+#pragma unroll
+  for (int dt = 0; dt < DT; dt += 2) {
+    uint32_t vb[4];
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(vb[0]), "=r"(vb[1]), "=r"(vb[2]), "=r"(vb[3])
+                 : "r"(vt + str_off(key16 + (mi & 1) * 8 + r, dt + (mi >> 1))));
+    mma_16816(o[dt], pf, vb[0], vb[1]);
+    mma_16816(o[dt + 1], pf, vb[2], vb[3]);
+  }
+}
+
+// the consumer warps' partial results -> one (max, sum, numerator) per row, written to the scratch slot.
+// Warp cw = row tile + 2 * key quarter; comb: [8 warps][16 rows][HD + 2] floats.
+template <int HD>
+__device__ __forceinline__ void str_combine_write(const AttnArgs& p, float* comb, int cw, const float (&o)[HD / 8][4],
+                                                  const float (&mrow)[2], float (&lrow)[2], int kh, int v0, int n_rows,
+                                                  int slot, int ctid) {
+  constexpr int DT = HD / 8, CS = HD + 2;
+  const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int g_heads = p.Hq / p.Hkv, R_all = p.n * g_heads, slots = p.n_prefix_chunks + p.n_own_chunks;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    lrow[h] += __shfl_xor_sync(0xffffffffu, lrow[h], 1);
+    lrow[h] += __shfl_xor_sync(0xffffffffu, lrow[h], 2);
+  }
+  float* mine = comb + (size_t)cw * 16 * CS;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    float* row = mine + (size_t)(g + 8 * h) * CS;
+#pragma unroll
+    for (int dt = 0; dt < DT; ++dt) *reinterpret_cast<float2*>(row + dt * 8 + 2 * t) = make_float2(o[dt][2 * h], o[dt][2 * h + 1]);
+    if (t == 0) { row[HD] = mrow[h]; row[HD + 1] = lrow[h]; }
+  }
+  asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");
+  for (int i = ctid; i < n_rows * (HD / 4); i += STR_CWARPS * 32) {
+    const int r = i / (HD / 4), d = (i % (HD / 4)) * 4;
+    const float* base = comb + (size_t)((r >> 4) * 16 + (r & 15)) * CS;   // key quarter 0 of the row's tile; quarter q: + 2 q warps
+    float M = -INFINITY;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) M = fmaxf(M, base[(size_t)(2 * q) * 16 * CS + HD]);
+    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+    float den = 0.f;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {                                          // fixed order
+      const float* w = base + (size_t)(2 * q) * 16 * CS;
+      const float mq = w[HD];
+      const float f = (mq == -INFINITY) ? 0.f : exp2f(mq - M);
+      num.x = fmaf(f, w[d], num.x); num.y = fmaf(f, w[d + 1], num.y);
+      num.z = fmaf(f, w[d + 2], num.z); num.w = fmaf(f, w[d + 3], num.w);
+      den = fmaf(f, w[HD + 1], den);
+    }
+    const size_t idx = ((size_t)kh * R_all + v0 + r) * slots + slot;
+    *reinterpret_cast<float4*>(p.part_o + idx * HD + d) = num;
+    if (d == 0) *reinterpret_cast<float2*>(p.part_ml + idx * 2) = make_float2(M, den);
+  }
+  asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");
+}
+
+template <int HD>
+__global__ void __launch_bounds__(STR_THREADS, 1)
+attn_stream_kernel(const AttnArgs p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                   const float scale_log2) {
+  constexpr int KSTEPS = HD / 16, DT = HD / 8, VPR = HD / 8, QSTRIDE = HD + 8;
+  constexpr uint32_t TILE_BYTES = STR_KEYS * HD * 2;                      // one K (or V) tile
+  constexpr uint32_t STAGE_BYTES = 2 * TILE_BYTES;
+  extern __shared__ unsigned char smem_raw_[];
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw_) + 1023) & ~(uintptr_t)1023);
+  unsigned char* ring = base;                                              // [STAGES][K tile, V tile]
+  unsigned char* own_tiles_mem = ring + STR_STAGES * STAGE_BYTES;          // [OWN_TILES][K tile, V tile]
+  __half* Qs = reinterpret_cast<__half*>(own_tiles_mem + STR_OWN_TILES * STAGE_BYTES);   // [32 + 16][QSTRIDE]
+  __half* Qown = Qs + (size_t)STR_ROWS * QSTRIDE;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(Qs) + (size_t)(STR_ROWS + 16) * QSTRIDE * 2);
+  float* comb = reinterpret_cast<float*>(ring);                            // after the prefix loop: [8 warps][16][HD + 2]
+  __shared__ int s_abort;
+  const uint32_t ring_u = smem_u32(ring), own_u = smem_u32(own_tiles_mem);
+  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STR_STAGES);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kh = blockIdx.x % p.Hkv, chunk = blockIdx.x / p.Hkv;
+  const int g_heads = p.Hq / p.Hkv, R_all = p.n * g_heads;
+  const bool fused = p.qkv_f32 != nullptr;
+  const int NT = (p.P + STR_KEYS - 1) / STR_KEYS;
+  const int t0 = (int)((long long)chunk * NT / p.n_prefix_chunks), t1 = (int)((long long)(chunk + 1) * NT / p.n_prefix_chunks);
+  const int n_tiles = t1 - t0;
+  const int s = chunk;                                                     // blockIdx.x = s * Hkv + kh: the CTA's own segment
+  const bool has_own = s < p.n;
+  const int S = has_own ? p.suffix_len[s] : 0;                             // (asked for early: used after the set-up)
+
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int i = 0; i < STR_STAGES; ++i) { mbar_init(full0 + 8 * i, 1); mbar_init(empty0 + 8 * i, STR_CWARPS); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp == STR_CWARPS) {
+    // ---- producer: one thread issues the tiled copies of the chunk's tiles
+    if (lane == 0) {
+      for (int i = 0; i < n_tiles; ++i) {
+        const int st = i % STR_STAGES;
+        if (i >= STR_STAGES && !str_wait(empty0 + 8 * st, (uint32_t)((i / STR_STAGES - 1) & 1), &s_abort, p.status)) break;
+        const uint32_t kd = ring_u + st * STAGE_BYTES, vd = kd + TILE_BYTES, bar = full0 + 8 * st;
+        mbar_expect_tx(bar, STAGE_BYTES);
+        const int key0 = (t0 + i) * STR_KEYS;
+#pragma unroll
+        for (int half = 0; half < HD / 64; ++half) {
+          tma_tile_3d(kd + half * (STR_KEYS * 128), &map_k, half * 64, key0, kh, bar);
+          tma_tile_3d(vd + half * (STR_KEYS * 128), &map_v, half * 64, key0, kh, bar);
+        }
+      }
+    }
+    return;                                                                 // (the consumers wait for every copy issued)
+  }
+
+  // ---- consumers
+  const int ctid = threadIdx.x;                                             // 0 .. 255
+  const int rt = warp & 1, kq = warp >> 1;                                  // row tile, key quarter of a tile
+  const int key_end = S + 1;                                                // own keys: cached rows + this pass's row
+  __half* ok_ = const_cast<__half*>(p.own_k) + (size_t)(has_own ? s : 0) * p.own_stream_stride + (size_t)kh * p.own_head_stride;
+  __half* ov_ = const_cast<__half*>(p.own_v) + (size_t)(has_own ? s : 0) * p.own_stream_stride + (size_t)kh * p.own_head_stride;
+  // own tile i into (kd, vd): cached rows by cp.async, the pass's row built here, rows past the end zero
+  auto fetch_own_tile = [&](int i, uint32_t kd, uint32_t vd, unsigned char* kd_g, unsigned char* vd_g) {
+    for (int j = ctid; j < STR_KEYS * VPR; j += STR_CWARPS * 32) {
+      const int r = j / VPR, piece = j % VPR, key = i * STR_KEYS + r;
+      const uint32_t off = str_off(r, piece);
+      if (key < key_end && !(fused && key == S)) {
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(kd + off), "l"(ok_ + (size_t)key * HD + piece * 8) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(vd + off), "l"(ov_ + (size_t)key * HD + piece * 8) : "memory");
+      } else {
+        uint4 kv8 = make_uint4(0, 0, 0, 0), vv8 = make_uint4(0, 0, 0, 0);
+        if (key < key_end) {
+          // this pass's row: built from the projections (k rotated), used, and appended to the stream's own segment
+          const float* row = p.qkv_f32 + (size_t)s * (size_t)((p.Hq + 2 * p.Hkv) * HD);
+          const float2* cs = p.cs_table + (size_t)(p.pos_base + S + p.depth[s]) * (HD / 2);
+          kv8 = head_piece_f16(row + (size_t)(p.Hq + kh) * HD, piece * 8, HD, cs);
+          vv8 = head_piece_f16(row + (size_t)(p.Hq + p.Hkv + kh) * HD, piece * 8, HD, nullptr);
+          *reinterpret_cast<uint4*>(ok_ + (size_t)key * HD + piece * 8) = kv8;
+          *reinterpret_cast<uint4*>(ov_ + (size_t)key * HD + piece * 8) = vv8;
+        }
+        *reinterpret_cast<uint4*>(kd_g + off) = kv8;
+        *reinterpret_cast<uint4*>(vd_g + off) = vv8;
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  const int own_tiles = has_own ? (key_end + STR_KEYS - 1) / STR_KEYS : 0;
+  for (int i = 0; i < own_tiles && i < STR_OWN_TILES; ++i)
+    fetch_own_tile(i, own_u + i * STAGE_BYTES, own_u + i * STAGE_BYTES + TILE_BYTES, own_tiles_mem + (size_t)i * STAGE_BYTES,
+                   own_tiles_mem + (size_t)i * STAGE_BYTES + TILE_BYTES);
+
+  // query rows v0 .. v0 + n_rows - 1 of the kv head's virtual rows (v = stream * g_heads + head in group) into dst
+  auto build_q = [&](__half* dst, int rows_cap, int v0, int n_rows) {
+    for (int i = ctid; i < rows_cap * VPR; i += STR_CWARPS * 32) {
+      const int r = i / VPR, c = (i % VPR) * 8;
+      uint4 val = make_uint4(0, 0, 0, 0);
+      if (r < n_rows) {
+        const int v = v0 + r, m = v / g_heads, j = v % g_heads;
+        if (fused) {
+          const float* row = p.qkv_f32 + (size_t)m * (size_t)((p.Hq + 2 * p.Hkv) * HD);
+          const float2* cs = p.cs_table + (size_t)(p.pos_base + p.suffix_len[m] + p.depth[m]) * (HD / 2);
+          val = head_piece_f16(row + (size_t)(kh * g_heads + j) * HD, c, HD, cs);
+        } else {
+          val = *reinterpret_cast<const uint4*>(p.q + ((size_t)m * p.Hq + kh * g_heads + j) * HD + c);
+        }
+      }
+      *reinterpret_cast<uint4*>(dst + (size_t)r * QSTRIDE + c) = val;
+    }
+  };
+  build_q(Qs, STR_ROWS, 0, R_all);
+  if (has_own) build_q(Qown, 16, s * g_heads, g_heads);
+  asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");
+  uint32_t qf[KSTEPS][4];
+  auto load_qf = [&](const __half* src, int row0) {
+#pragma unroll
+    for (int ks = 0; ks < KSTEPS; ++ks) {
+      const int mi = lane >> 3, r = lane & 7;
+      ldmatrix_x4(qf[ks], src + (size_t)(row0 + (mi & 1) * 8 + r) * QSTRIDE + ks * 16 + (mi >> 1) * 8);
+    }
+  };
+  float o[DT][4];
+  float mrow[2], lrow[2];
+  auto reset_acc = [&]() {
+#pragma unroll
+    for (int i = 0; i < DT; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+    mrow[0] = mrow[1] = -INFINITY;
+    lrow[0] = lrow[1] = 0.f;
+  };
+
+  // ---- the shared-prefix chunk, for the rows of all streams
+  load_qf(Qs, rt * 16);
+  reset_acc();
+  const bool rows_live = rt * 16 < R_all;
+  for (int i = 0; i < n_tiles; ++i) {
+    const int st = i % STR_STAGES;
+    const bool ok = str_wait(full0 + 8 * st, (uint32_t)((i / STR_STAGES) & 1), &s_abort, p.status);
+    if (ok && rows_live) {
+      const uint32_t kt = ring_u + st * STAGE_BYTES, vt = kt + TILE_BYTES;
+      const int key0 = (t0 + i) * STR_KEYS + kq * 16;
+      str_tile16<HD>(qf, kt, vt, kq * 16, min(16, p.P - key0), scale_log2, o, mrow, lrow);
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty0 + 8 * st);
+    if (!ok) break;
+  }
+  asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");         // every tile consumed: the ring is free
+  if (n_tiles > 0 && !s_abort) str_combine_write<HD>(p, comb, warp, o, mrow, lrow, kh, 0, R_all, chunk, ctid);
+
+  // ---- the CTA's own segment (stream s, this kv head): 4..16 rows in row tile 0
+  if (!has_own || s_abort) return;
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");
+  load_qf(Qown, 0);
+  reset_acc();
+  for (int i = 0; i < own_tiles; ++i) {
+    uint32_t kt = own_u + i * STAGE_BYTES;
+    if (i >= STR_OWN_TILES) {
+      // a long own segment: the further tiles one at a time through the start of the ring (its combine buffer has
+      // been read: str_combine_write ends with a barrier)
+      kt = ring_u;
+      fetch_own_tile(i, ring_u, ring_u + TILE_BYTES, ring, ring + TILE_BYTES);
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");
+    }
+    if (rt == 0) {
+      const int key0 = i * STR_KEYS + kq * 16;
+      if (key0 < key_end) str_tile16<HD>(qf, kt, kt + TILE_BYTES, kq * 16, min(16, key_end - key0), scale_log2, o, mrow, lrow);
+    }
+    if (i >= STR_OWN_TILES) asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");
+  }
+  // (the combine buffer is the start of the ring; own tiles beyond the first two were read from there: barrier above)
+  str_combine_write<HD>(p, comb, warp, o, mrow, lrow, kh, s * g_heads, g_heads, p.n_prefix_chunks, ctid);
+}
+
 // one decode row per stream, a context short enough for one CTA per (kv head, stream), at most 16 query heads per
 // kv head
 bool attn_single_pass(const AttnArgs& a) {
   return a.T == 1 && a.Hq / a.Hkv <= 16 && a.P + a.suffix_bound + 1 <= 2048 && (a.hd == 64 || a.hd == 128);
 }
 
+// one decode row per stream over a long shared prefix: the streaming kernel (one chunk of the prefix per SM and kv
+// head, all streams' rows per CTA).  Shapes only: the launch checks the pointers' alignment.
+static bool attn_stream_shape(const AttnArgs& a, int sm_count) {
+  if (a.T != 1 || attn_single_pass(a) || (a.hd != 64 && a.hd != 128)) return false;
+  const int g_heads = a.Hq / a.Hkv;
+  const int chunks = sm_count / a.Hkv;                    // CTAs per kv head
+  return a.n * g_heads <= STR_ROWS && g_heads <= 16 && a.P >= STR_KEYS && chunks >= a.n && a.suffix_bound + 1 <= 1024;
+}
+
 void attn_plan(AttnArgs& a, int sm_count) {
+  a.stream_mode = 0;
+  if (attn_stream_shape(a, sm_count)) {
+    const int NT = (a.P + STR_KEYS - 1) / STR_KEYS;
+    int chunks = sm_count / a.Hkv;
+    if (chunks > NT) chunks = NT;
+    if (chunks < a.n) chunks = a.n;                       // the first n CTAs of a kv head also take an own segment
+    if (chunks <= NT) {
+      a.stream_mode = 1;
+      a.n_prefix_chunks = chunks;
+      a.prefix_chunk = (NT + chunks - 1) / chunks * STR_KEYS;
+      a.n_own_chunks = 1;
+      a.own_chunk = (a.suffix_bound + 1 + STR_KEYS - 1) / STR_KEYS * STR_KEYS;
+      return;
+    }
+  }
   const int g_heads = a.Hq / a.Hkv;
   const int R_all = a.n * a.T * g_heads;
   const int rb_all = (R_all + ATT_ROWS - 1) / ATT_ROWS;
@@ -727,11 +1104,61 @@ cudaError_t init_attention() {
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(attn_decode_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem_bytes(128));
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attn_stream_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)str_smem_bytes(64));
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attn_stream_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)str_smem_bytes(128));
+  if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(attn_partial_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)((ATT_ROWS + 4 * ATT_KEYS) * (128 + 8) * sizeof(__half)));
 }
 
+static PFN_cuTensorMapEncodeTiled_v12000 attn_map_encoder() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = []() -> PFN_cuTensorMapEncodeTiled_v12000 {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    return reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(sym);
+  }();
+  return fn;
+}
+
+// rank-3 fp16 map over one side (K or V) of the shared prefix: (head_dim, P keys, kv heads); box = 64 features x 64 keys
+// of one head, 128-byte swizzle; keys past P read as zeros
+static cudaError_t attn_prefix_map(const __half* base, int hd, int P, int Hkv, size_t head_stride, CUtensorMap* out) {
+  PFN_cuTensorMapEncodeTiled_v12000 enc = attn_map_encoder();
+  if (enc == nullptr) return cudaErrorNotSupported;
+  const cuuint64_t dims[3] = {(cuuint64_t)hd, (cuuint64_t)P, (cuuint64_t)Hkv};
+  const cuuint64_t strides[2] = {(cuuint64_t)hd * sizeof(__half), (cuuint64_t)head_stride * sizeof(__half)};
+  const cuuint32_t box[3] = {64, (cuuint32_t)STR_KEYS, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult rc = enc(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<__half*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+static cudaError_t launch_attention_stream(const AttnArgs& a, cudaStream_t st) {
+  // the tiled copies and the 16-byte copies of the own rows need aligned bases and strides
+  if ((reinterpret_cast<uintptr_t>(a.prefix_k) & 15) || (reinterpret_cast<uintptr_t>(a.prefix_v) & 15) ||
+      (reinterpret_cast<uintptr_t>(a.own_k) & 15) || (reinterpret_cast<uintptr_t>(a.own_v) & 15) ||
+      (a.prefix_head_stride * sizeof(__half)) % 16 != 0)
+    return cudaErrorMisalignedAddress;
+  CUtensorMap mk, mv;
+  cudaError_t e = attn_prefix_map(a.prefix_k, a.hd, a.P, a.Hkv, a.prefix_head_stride, &mk);
+  if (e != cudaSuccess) return e;
+  e = attn_prefix_map(a.prefix_v, a.hd, a.P, a.Hkv, a.prefix_head_stride, &mv);
+  if (e != cudaSuccess) return e;
+  const float scale_log2 = 1.4426950408889634f / sqrtf((float)a.hd);
+  const dim3 grid((unsigned)(a.Hkv * a.n_prefix_chunks));
+  if (a.hd == 64) attn_stream_kernel<64><<<grid, STR_THREADS, str_smem_bytes(64), st>>>(a, mk, mv, scale_log2);
+  else attn_stream_kernel<128><<<grid, STR_THREADS, str_smem_bytes(128), st>>>(a, mk, mv, scale_log2);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st) {
+  if (a.stream_mode) return launch_attention_stream(a, st);
   if (attn_single_pass(a)) {
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)a.hd);
     cudaLaunchConfig_t cfg{};

@@ -132,6 +132,8 @@ struct AttnArgs {
   const float2* cs_table;         // cos/sin of pos * theta^(-2i/hd): [pos][hd/2]
   int pos_base;                   // position of a row = pos_base + suffix_len[s] + depth[row]
   const int32_t* depth;           // dev [rows]
+  int stream_mode;                // set by attn_plan: the streaming kernel for one row per stream over a long prefix
+  int* status;                    // dev status word for bounded waits that run out (may be null)
 };
 
 // ----------------------------------------------------------------------------- persistent projection chain

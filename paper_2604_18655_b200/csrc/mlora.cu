@@ -229,7 +229,7 @@ int launch_attention_block(mlora_ctx* c, const PassIO& io, int l) {
   a.prefix_head_stride = c->prefix_head_stride;
   a.own_k = kd; a.own_v = vd; a.own_stream_stride = sstride; a.own_head_stride = hstride;
   a.suffix_len = io.suffix_len; a.anc = c->anc; a.causal = io.prefill ? 1 : 0;
-  a.out = c->attn16;
+  a.out = c->attn16; a.status = c->status;
   if (attn_workspace_floats(a) > c->att_ws_floats) return fail(MLORA_ERR_CAPACITY, "attention scratch too small");
   a.part_o = c->att_ws;
   a.part_ml = c->att_ws + (attn_workspace_floats(a) / (a.hd + 2)) * a.hd;
@@ -1575,7 +1575,7 @@ int mlora_attention(const void* q, const void* prefix_k, const void* prefix_v, i
   a.prefix_k = (const __half*)prefix_k; a.prefix_v = (const __half*)prefix_v; a.prefix_head_stride = (size_t)P * hd;
   a.own_k = (const __half*)own_k; a.own_v = (const __half*)own_v;
   a.own_head_stride = (size_t)own_capacity * hd; a.own_stream_stride = a.own_head_stride * Hkv;
-  a.suffix_len = suffix_len; a.anc = anc; a.out = (__half*)out;
+  a.suffix_len = suffix_len; a.anc = anc; a.out = (__half*)out; a.status = status; a.depth = depth;
   a.part_o = (float*)(ws + head);
   a.part_ml = a.part_o + (attn_workspace_floats(a) / (hd + 2)) * hd;
   CK(launch_attention(a, st));

@@ -219,6 +219,21 @@ def test_attention_workspace_covers_every_suffix_bound(mb):
     compare(got, want, "attention cap129 bound127")
 
 
+@pytest.mark.parametrize("n,Hq,Hkv,hd,P,suf", [
+    (8, 32, 8, 128, 8192, [0, 63, 64, 65, 200, 1, 17, 128]),     # the sweep's longest prefix: 18 chunks per kv head
+    (8, 32, 8, 64, 2048, [5, 0, 64, 100, 127, 128, 129, 300]),   # two tiles per chunk at most
+    (3, 24, 8, 128, 2100, [0, 40, 90]),                          # three query heads per kv head, ragged last tile
+    (1, 8, 2, 64, 4099, [7]),                                    # one stream; 65 tiles on 65 chunks
+    (5, 8, 8, 128, 1990, [100, 3, 64, 0, 77]),                   # just past the single-kernel limit, one head per group
+    (8, 32, 8, 64, 2500, [1000, 0, 1, 2, 3, 4, 5, 6]),           # a long own segment: 16 tiles of it on one CTA
+])
+def test_attention_one_row_per_stream_over_long_prefix(mb, n, Hq, Hkv, hd, P, suf):
+    """One decode row per stream over a prefix too long for the single-kernel path: the streaming kernel (prefix chunks
+    shared by all streams' rows, tiled TMA copies) plus the merge."""
+    got, want = run_attention(mb, n, 1, Hq, Hkv, hd, P, suf, (), seed=P + n)
+    compare(got, want, f"attention stream hd{hd} {Hq}q/{Hkv}kv n{n} P{P}")
+
+
 def test_attention_long_prefix_split(mb):
     got, want = run_attention(mb, 2, 1, 8, 2, 128, 3000, [64, 10], (), seed=3)
     compare(got, want, "attention P3000")

@@ -433,6 +433,24 @@ def test_export_state_gives_the_whole_own_segment(GpuModel):
     gm.close()
 
 
+def test_decode_over_a_long_shared_prompt(GpuModel):
+    """Decode steps over a 2100-token shared prompt: past the single-kernel attention's limit, so the layers' attention
+    runs in the streaming kernel with q, k rotated on load and the new K/V row appended by it."""
+    cfg = gen.ModelCfg("tinylong", 2, 128, 4, 2, 64, 192, 160, 64, 4, 127, 3, 3, 2100, b_std=0.05)
+    m, orc, gm = make_pair(GpuModel, cfg, max_suffix=8)
+    ids = gen.make_prompt_ids(cfg, 0)
+    compare(gm.prefill(ids), orc.prefill_shared(ids, n_streams=3), "long prompt prefill logits")
+    ad, toks = [0, -1, 2], np.array([3, 4, 5], dtype=np.int32)
+    for step in range(4):
+        nxt, logits = gm.decode(ad, toks)
+        r = orc.decode_step(ad, tokens=toks)
+        compare(logits, r["logits"], f"long prompt decode logits step {step}")
+        check_argmax(nxt, r["logits"], f"long prompt step {step}")
+        toks = nxt
+    compare_kv(gm, orc, cfg, 3)
+    gm.close()
+
+
 def test_sample_first_matches_oracle(GpuModel):
     """The n distinct first tokens (App. A.1): integer work, exact -- with ties, infinities, signed zeros and NaN."""
     from paper_2604_18655_b200 import binding as mb
