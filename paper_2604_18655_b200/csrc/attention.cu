@@ -343,8 +343,8 @@ __device__ __forceinline__ void merge_row(const AttnArgs& p, int kh, int v, int 
   const int R_all = p.n * p.T * g_heads;
   const int slots = p.n_prefix_chunks + p.n_own_chunks;
   const int s = m / p.T;
-  // (a single own chunk always holds the pass's own rows: no need to wait for the suffix length)
-  const int own_valid = p.n_own_chunks == 1 ? 1 : min(p.n_own_chunks, (p.suffix_len[s] + p.T + p.own_chunk - 1) / p.own_chunk);
+  // (no or a single own chunk: no need to wait for the suffix length)
+  const int own_valid = p.n_own_chunks <= 1 ? p.n_own_chunks : min(p.n_own_chunks, (p.suffix_len[s] + p.T + p.own_chunk - 1) / p.own_chunk);
   const int n_valid = p.n_prefix_chunks + own_valid;
   const size_t base = ((size_t)kh * R_all + v) * slots;
   const int hd = p.hd;
@@ -684,10 +684,10 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
 // A producer warp streams 64-key K and V tiles through a 4-stage ring with tiled TMA copies (tensor maps over the
 // prefix, 128-byte swizzle, rows past the prefix zero-filled, completion on mbarriers); eight consumer warps take
 // (row tile, 16 keys of the tile) each, with their own online softmax, and are combined by log-sum-exp in shared
-// memory at the end of the chunk.  The first n * Hkv CTAs also do one (stream, kv head) own segment each: its first
-// two tiles are fetched with cp.async into the same swizzled layout while the prefix streams (the new row is built
-// from the projections, rotated, and appended).  Partial results per (row, chunk) go to the scratch that
-// attn_merge_kernel combines.
+// memory at the end of the chunk.  The first n * Hkv CTAs also take one (stream, kv head) own segment each, as further
+// keys of their partial that only that stream's rows may see: its first two tiles are fetched with cp.async into the
+// same swizzled layout while the prefix streams (the new row is built from the projections, rotated, and appended).
+// Partial results per (row, chunk) go to the scratch that attn_merge_kernel combines.
 constexpr int STR_KEYS = 64;
 constexpr int STR_CWARPS = 8;
 constexpr int STR_THREADS = (STR_CWARPS + 1) * 32;
@@ -697,7 +697,7 @@ constexpr int STR_OWN_TILES = 2;                          // own tiles fetched a
 constexpr long long STR_WAIT_CYCLES = 2000000000ll;       // ~1 s
 __host__ __device__ constexpr size_t str_stage_bytes(int hd) { return (size_t)2 * STR_KEYS * hd * 2; }
 __host__ __device__ constexpr size_t str_smem_bytes(int hd) {
-  return 1024 + (STR_STAGES + STR_OWN_TILES) * str_stage_bytes(hd) + (size_t)(STR_ROWS + 16) * (hd + 8) * 2 + 128;
+  return 1024 + (STR_STAGES + STR_OWN_TILES) * str_stage_bytes(hd) + (size_t)STR_ROWS * (hd + 8) * 2 + 128;
 }
 
 __device__ __forceinline__ void tma_tile_3d(uint32_t dst, const void* tmap, int x, int y, int z, uint32_t bar) {
@@ -731,7 +731,8 @@ __device__ __forceinline__ bool str_wait(uint32_t bar, uint32_t parity, volatile
 // online softmax update of (o, mrow, lrow).  n_valid = number of valid keys among the 16.
 template <int HD>
 __device__ __forceinline__ void str_tile16(const uint32_t (&qf)[HD / 16][4], uint32_t kt, uint32_t vt, int key16, int n_valid,
-                                           float scale_log2, float (&o)[HD / 8][4], float (&mrow)[2], float (&lrow)[2]) {
+                                           bool row_lo_ok, bool row_hi_ok, float scale_log2, float (&o)[HD / 8][4],
+                                           float (&mrow)[2], float (&lrow)[2]) {
   constexpr int KSTEPS = HD / 16, DT = HD / 8;
   const int lane = threadIdx.x & 31, t = lane & 3, mi = lane >> 3, r = lane & 7;
   float sacc[2][4];
@@ -754,7 +755,7 @@ __device__ __forceinline__ void str_tile16(const uint32_t (&qf)[HD / 16][4], uin
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const int key = nt * 8 + 2 * t + (e & 1);
-      const float v = key < n_valid ? sacc[nt][e] * scale_log2 : -INFINITY;
+      const float v = (key < n_valid && ((e & 2) ? row_hi_ok : row_lo_ok)) ? sacc[nt][e] * scale_log2 : -INFINITY;
       sacc[nt][e] = v;
       mx[e >> 1] = fmaxf(mx[e >> 1], v);
     }
@@ -766,7 +767,7 @@ __device__ __forceinline__ void str_tile16(const uint32_t (&qf)[HD / 16][4], uin
     mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
     const float mnew = fmaxf(mrow[h], mx[h]);
     msafe[h] = (mnew == -INFINITY) ? 0.f : mnew;
-    corr[h] = exp2f(mrow[h] - msafe[h]);
+    corr[h] = exp2f(mrow[h] - msafe[h]);                               // both -inf: exp2(-inf) = 0 on zeros, harmless
     mrow[h] = mnew;
   }
   uint32_t pf[4];
@@ -856,9 +857,8 @@ attn_stream_kernel(const AttnArgs p, const __grid_constant__ CUtensorMap map_k, 
   unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw_) + 1023) & ~(uintptr_t)1023);
   unsigned char* ring = base;                                              // [STAGES][K tile, V tile]
   unsigned char* own_tiles_mem = ring + STR_STAGES * STAGE_BYTES;          // [OWN_TILES][K tile, V tile]
-  __half* Qs = reinterpret_cast<__half*>(own_tiles_mem + STR_OWN_TILES * STAGE_BYTES);   // [32 + 16][QSTRIDE]
-  __half* Qown = Qs + (size_t)STR_ROWS * QSTRIDE;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(Qs) + (size_t)(STR_ROWS + 16) * QSTRIDE * 2);
+  __half* Qs = reinterpret_cast<__half*>(own_tiles_mem + STR_OWN_TILES * STAGE_BYTES);   // [32][QSTRIDE]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(Qs) + (size_t)STR_ROWS * QSTRIDE * 2);
   float* comb = reinterpret_cast<float*>(ring);                            // after the prefix loop: [8 warps][16][HD + 2]
   __shared__ int s_abort;
   const uint32_t ring_u = smem_u32(ring), own_u = smem_u32(own_tiles_mem);
@@ -956,7 +956,6 @@ attn_stream_kernel(const AttnArgs p, const __grid_constant__ CUtensorMap map_k, 
     }
   };
   build_q(Qs, STR_ROWS, 0, R_all);
-  if (has_own) build_q(Qown, 16, s * g_heads, g_heads);
   asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");
   uint32_t qf[KSTEPS][4];
   auto load_qf = [&](const __half* src, int row0) {
@@ -985,39 +984,40 @@ attn_stream_kernel(const AttnArgs p, const __grid_constant__ CUtensorMap map_k, 
     if (ok && rows_live) {
       const uint32_t kt = ring_u + st * STAGE_BYTES, vt = kt + TILE_BYTES;
       const int key0 = (t0 + i) * STR_KEYS + kq * 16;
-      str_tile16<HD>(qf, kt, vt, kq * 16, min(16, p.P - key0), scale_log2, o, mrow, lrow);
+      str_tile16<HD>(qf, kt, vt, kq * 16, min(16, p.P - key0), true, true, scale_log2, o, mrow, lrow);
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(empty0 + 8 * st);
     if (!ok) break;
   }
-  asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");         // every tile consumed: the ring is free
-  if (n_tiles > 0 && !s_abort) str_combine_write<HD>(p, comb, warp, o, mrow, lrow, kh, 0, R_all, chunk, ctid);
 
-  // ---- the CTA's own segment (stream s, this kv head): 4..16 rows in row tile 0
-  if (!has_own || s_abort) return;
-  asm volatile("cp.async.wait_group 0;" ::: "memory");
-  asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");
-  load_qf(Qown, 0);
-  reset_acc();
-  for (int i = 0; i < own_tiles; ++i) {
-    uint32_t kt = own_u + i * STAGE_BYTES;
-    if (i >= STR_OWN_TILES) {
-      // a long own segment: the further tiles one at a time through the start of the ring (its combine buffer has
-      // been read: str_combine_write ends with a barrier)
-      kt = ring_u;
-      fetch_own_tile(i, ring_u, ring_u + TILE_BYTES, ring, ring + TILE_BYTES);
-      asm volatile("cp.async.wait_group 0;" ::: "memory");
-      asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");
-    }
-    if (rt == 0) {
+  // ---- the CTA's own segment (stream s, this kv head): more keys for the rows of stream s alone (a softmax partial
+  // may cover any set of keys: these join the chunk's), masked for every other row
+  if (has_own && !s_abort) {
+    const int g = lane >> 2;
+    const int r_lo = rt * 16 + g, r_hi = r_lo + 8;
+    const bool lo_ok = r_lo / g_heads == s && r_lo < R_all, hi_ok = r_hi / g_heads == s && r_hi < R_all;
+    const bool tile_has = (s * g_heads) / 16 == rt || (s * g_heads + g_heads - 1) / 16 == rt;   // warp-uniform
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");
+    for (int i = 0; i < own_tiles; ++i) {
+      uint32_t kt = own_u + i * STAGE_BYTES;
+      if (i >= STR_OWN_TILES) {
+        // a long own segment: the further tiles one at a time through the start of the ring (every prefix tile has
+        // been consumed by all warps: barrier above)
+        kt = ring_u;
+        fetch_own_tile(i, ring_u, ring_u + TILE_BYTES, ring, ring + TILE_BYTES);
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");
+      }
       const int key0 = i * STR_KEYS + kq * 16;
-      if (key0 < key_end) str_tile16<HD>(qf, kt, kt + TILE_BYTES, kq * 16, min(16, key_end - key0), scale_log2, o, mrow, lrow);
+      if (tile_has && key0 < key_end)
+        str_tile16<HD>(qf, kt, kt + TILE_BYTES, kq * 16, min(16, key_end - key0), lo_ok, hi_ok, scale_log2, o, mrow, lrow);
+      if (i >= STR_OWN_TILES) asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");
     }
-    if (i >= STR_OWN_TILES) asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");
   }
-  // (the combine buffer is the start of the ring; own tiles beyond the first two were read from there: barrier above)
-  str_combine_write<HD>(p, comb, warp, o, mrow, lrow, kh, s * g_heads, g_heads, p.n_prefix_chunks, ctid);
+  asm volatile("bar.sync 1, %0;" ::"n"(STR_CWARPS * 32) : "memory");         // every tile consumed: the ring is free
+  if (!s_abort) str_combine_write<HD>(p, comb, warp, o, mrow, lrow, kh, 0, R_all, chunk, ctid);
 }
 
 // one decode row per stream, a context short enough for one CTA per (kv head, stream), at most 16 query heads per
@@ -1046,7 +1046,7 @@ void attn_plan(AttnArgs& a, int sm_count) {
       a.stream_mode = 1;
       a.n_prefix_chunks = chunks;
       a.prefix_chunk = (NT + chunks - 1) / chunks * STR_KEYS;
-      a.n_own_chunks = 1;
+      a.n_own_chunks = 0;                                 // the own segments' keys join the first n chunks' partials
       a.own_chunk = (a.suffix_bound + 1 + STR_KEYS - 1) / STR_KEYS * STR_KEYS;
       return;
     }
