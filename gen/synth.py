@@ -15,7 +15,7 @@ import numpy as np
 from .configs import ModelCfg, PROJ_NAMES, PROJ_BITS, proj_shape
 
 _KIND = {"w": 0, "A": 1, "B": 2, "rms_attn": 3, "rms_ffn": 4, "rms_final": 5, "embed": 6,
-         "prompt": 7, "hidden": 8, "cand": 9}
+         "prompt": 7, "hidden": 8, "cand": 9, "forecast": 10}
 _LM_HEAD = 7  # projection index of lm_head in the per-model list (after the 7 per-layer ones)
 
 
@@ -135,6 +135,45 @@ def build_tree(branch, n_nodes: int = None) -> np.ndarray:
     if n_nodes is not None:
         assert len(parent) == n_nodes, "branch configuration gives fewer nodes than requested"
     return np.asarray(parent, dtype=np.int32)
+
+
+def ds2d_template(branch, n_token_nodes: int = None) -> dict:
+    """Row layout of one DS2D pass that verifies a draft tree AND drafts the next one (one stream's rows).
+
+    Rows 0 .. T-1 are the tree's token nodes (build_tree order; node 0 = the last accepted token).  Every token node t
+    is followed, further down, by its m = len(branch) forecast rows T + t*m + (j-1), j = 1..m, chained under it
+    (forecast j sees node t's root path and forecasts 1..j of the same node).  Returns int32 arrays over the
+    R = T * (1 + m) rows: parent; level (0 root, d >= 1 draft node of depth d, -j forecast row j); rank (a draft
+    node's position among its parent's children); forecast_of (a token node's first forecast row, -1 otherwise);
+    and widths[d-1] = children per node at depth d."""
+    tok_parent = build_tree(branch, n_token_nodes)
+    T, m = len(tok_parent), len(branch)
+    R = T * (1 + m)
+    parent = np.full(R, -1, dtype=np.int32)
+    level = np.zeros(R, dtype=np.int32)
+    rank = np.zeros(R, dtype=np.int32)
+    forecast_of = np.full(R, -1, dtype=np.int32)
+    parent[:T] = tok_parent
+    depth = tree_depths(tok_parent)
+    seen = {}
+    for t in range(T):
+        level[t] = depth[t]
+        if t:
+            rank[t] = seen.get(int(tok_parent[t]), 0)
+            seen[int(tok_parent[t])] = rank[t] + 1
+        forecast_of[t] = T + t * m
+        for j in range(1, m + 1):
+            r = T + t * m + (j - 1)
+            parent[r] = t if j == 1 else r - 1
+            level[r] = -j
+    widths = np.array([max([rank[t] + 1 for t in range(T) if level[t] == d] or [0]) for d in range(1, m + 1)], dtype=np.int32)
+    return dict(parent=parent, level=level, rank=rank, forecast_of=forecast_of, widths=widths, T=T, m=m, R=R)
+
+
+def make_forecast(cfg: ModelCfg, m: int, seed: int = 0) -> np.ndarray:
+    """m synthetic forecast embeddings fp16 [m][d_model] (stand-ins for the prefix-tuned ones: untrained, so the
+    drafts they produce are rarely accepted; shapes and data flow are what they exercise)."""
+    return _normal(_rng(seed, 0, 0, "forecast"), (m, cfg.d_model), 0.02).astype(np.float16)
 
 
 def tree_depths(parent) -> np.ndarray:

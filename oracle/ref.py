@@ -20,6 +20,9 @@ What follows which passage:
   * after the single prefill a sampler gives the n streams n distinct
     first tokens (here: the n most probable, by falling logit, ties by
     rising id), then the n-fold model runs step after step              -- App. A.1 (flowsheet)
+  * m forecast embeddings ride along with every token node of the pass
+    as further rows chained under it; the top-b_j ids of forecast row j
+    of the last accepted node become the next tree's depth-j drafts     -- Sec. 3.5 (inference steps 1-2), App. A.2
 
 Arithmetic: everything after dequantisation is carried in ``dtype`` (float64 by default; float32
 for the 1B/3B shapes where the dense weights would not fit twice in memory).  No blocking, no
@@ -34,7 +37,9 @@ concatenated sequence; RoPE/RMSNorm/SiLU closed forms; accept walk against brute
 small tree; the (3,2) -> 9/10/30 node counts and the 32-row budgets of Table 7; the wiring of a decoder block
 (norm placement, residuals, gate/up roles, final norm) against scalar loops written from the definitions
 (tests/test_oracle_wiring_pin.py); the first-token sampler against exhaustive selection on small rows with ties and
-against argmax for n = 1 (tests/test_oracle_generate.py).
+against argmax for n = 1 (tests/test_oracle_generate.py); DS2D drafting: the printed row counts of the (3,2) example,
+forecast rows against the same vectors planted as ordinary embedding rows, draft placement by explicit loops, and
+losslessness of whole drafting rounds against plain greedy decoding (tests/test_oracle_ds2d_draft.py).
 Parity unpinned by the paper: absolute activation values of a forward pass of ITS model (it prints none).
 """
 import numpy as np
@@ -286,8 +291,19 @@ class OracleModel:
         self.suf_k = [[z() for _ in range(n_streams)] for _ in range(c.n_layers)]
         self.suf_v = [[z() for _ in range(n_streams)] for _ in range(c.n_layers)]
 
+    def set_forecast(self, forecast):
+        """m forecast embeddings [m][d_model] (Sec. 3.5): an input id vocab + j - 1 stands for forecast row j."""
+        self.forecast = None if forecast is None else np.asarray(forecast)
+
     def _embed(self, tokens):
-        return self.embed[np.asarray(tokens).reshape(-1)].astype(self.dt)
+        tokens = np.asarray(tokens).reshape(-1)
+        fc = getattr(self, "forecast", None)
+        if fc is None:
+            return self.embed[tokens].astype(self.dt)
+        V = self.cfg.vocab
+        assert tokens.max() < V + len(fc)
+        table = np.concatenate([self.embed, fc.astype(self.embed.dtype)], axis=0)
+        return table[tokens].astype(self.dt)
 
     def _mlp(self, l, X, row_adapter):
         c = self.cfg
@@ -388,6 +404,39 @@ class OracleModel:
                     rows = [s * T + int(u) for u in acc_idx[s, :acc_len[s]]]
                     self.suf_k[l][s] = np.concatenate([self.suf_k[l][s], new_k[l][rows]], axis=0)
                     self.suf_v[l][s] = np.concatenate([self.suf_v[l][s], new_v[l][rows]], axis=0)
+        return out
+
+    def ds2d_round(self, adapter_idx, template, tree_tokens, follow_argmax=None):
+        """One DS2D inference step (Sec. 3.5 steps 1-2, App. A.2): the pass verifies the draft tree in `tree_tokens`
+        AND, from the forecast rows chained under every token node, drafts the next tree.
+
+        template: row layout of one stream (parent, level, rank, forecast_of, widths; every stream uses the same).
+        tree_tokens [n][R]: token ids at the token nodes, vocab + j - 1 at forecast rows j.
+        After the accept walk, the drafts hang off the LAST ACCEPTED node: the next tree's nodes of depth d all carry,
+        by sibling rank, the widths[d-1] most probable ids of that node's forecast row d (ties by rising id); the next
+        root is the bonus token.  Returns verify_tree's dict plus next_tree_tokens [n][R] and drafts [n][m][max width]."""
+        n = len(adapter_idx)
+        R, m, V = len(template["parent"]), len(template["widths"]), self.cfg.vocab
+        tree_tokens = np.asarray(tree_tokens).reshape(n, R)
+        out = self.verify_tree(adapter_idx, np.stack([template["parent"]] * n), tree_tokens, follow_argmax=follow_argmax)
+        wmax = int(max(template["widths"]))
+        drafts = np.full((n, m, wmax), -1, dtype=np.int32)
+        nxt = np.empty((n, R), dtype=np.int32)
+        for s in range(n):
+            leaf = int(out["accept_idx"][s][out["accept_len"][s] - 1])
+            for j in range(1, m + 1):
+                row = s * R + int(template["forecast_of"][leaf]) + (j - 1)
+                w = int(template["widths"][j - 1])
+                drafts[s, j - 1, :w] = first_tokens(out["logits"][row], w)
+            for i in range(R):
+                lv = int(template["level"][i])
+                if lv == 0:
+                    nxt[s, i] = out["next"][s]
+                elif lv > 0:
+                    nxt[s, i] = drafts[s, lv - 1, int(template["rank"][i])]
+                else:
+                    nxt[s, i] = V + (-lv) - 1
+        out["next_tree_tokens"], out["drafts"] = nxt, drafts
         return out
 
     def generate(self, adapter_idx, first, k_steps):
