@@ -148,6 +148,30 @@ int mlora_verify_tree(mlora_ctx* ctx, int32_t n_streams, const int32_t* adapter_
                       const int32_t* tree_tokens, const int32_t* tree_parent, int32_t* out_accept_len,
                       int32_t* out_accept_idx, int32_t* out_next, float* out_logits);
 
+/* DS2D draft generation (Sec. 3.5 inference steps 1-2, App. A.2).  m forecast embeddings (dev fp16 [m][d_model],
+ * caller-owned, must stay valid; 1 <= m <= 8) ride along with the tokens of a pass: from now on an input id
+ * vocab + j - 1 (j = 1..m) in tree_tokens of mlora_verify_tree / mlora_ds2d_round denotes forecast row j, whose input
+ * row is forecast[j - 1].  A forecast row is an ordinary tree row for attention (chain it under its token node with
+ * tree_parent); it can never be accepted and its K/V never reaches the cache.  forecast == NULL or m == 0 switches the
+ * ids off again.  Errors: ARG, STATE (no vocabulary). */
+int mlora_set_forecast(mlora_ctx* ctx, const void* forecast, int32_t m);
+/* One DS2D inference step: verifies the tree in tree_tokens exactly as mlora_verify_tree does AND drafts the next tree
+ * from the forecast rows of every stream's last accepted node, without a host round trip.  The n_rows rows of a stream
+ * are described by four dev int32 arrays shared by all streams: tree_parent as in mlora_verify_tree (here [n_streams]
+ * [n_rows] as well); row_level [n_rows]: 0 = root, d >= 1 = draft node of depth d, -j = forecast row j; row_rank
+ * [n_rows]: a draft node's position among its parent's children; forecast_of [n_rows]: for a token node the row index
+ * of its forecast row 1 (its m forecast rows are consecutive), else ignored; widths [m]: children per node at depth
+ * 1..m (each <= max_width <= 32).  out_tree_tokens dev int32 [n_streams][n_rows] (must not alias tree_tokens) receives
+ * the next pass's inputs: the bonus token at the root; at a draft node of depth d and rank r the r-th most probable id
+ * (ties by rising id) of forecast row d of the last accepted node; vocab + j - 1 at forecast rows.
+ * out_logits: dev fp32 [n_streams * n_rows][vocab] or NULL.  n_rows <= max_tree.  Errors: as mlora_verify_tree, plus STATE (no forecast embeddings set); a template that points
+ * outside the pass sets the device status to MLORA_ERR_ARG. */
+int mlora_ds2d_round(mlora_ctx* ctx, int32_t n_streams, const int32_t* adapter_idx, int32_t n_rows,
+                     const int32_t* tree_tokens, const int32_t* tree_parent, const int32_t* row_level,
+                     const int32_t* row_rank, const int32_t* forecast_of, const int32_t* widths, int32_t m,
+                     int32_t max_width, int32_t* out_accept_len, int32_t* out_accept_idx, int32_t* out_next,
+                     int32_t* out_tree_tokens, float* out_logits);
+
 /* ---- state / diagnostics ---- */
 int mlora_reset_streams(mlora_ctx* ctx);        /* empties every stream's own segment; keeps the shared one */
 int mlora_sync_status(mlora_ctx* ctx);          /* synchronises the stream; returns and clears the device status */

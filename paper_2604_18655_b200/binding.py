@@ -57,6 +57,9 @@ _SIGS = {
     "mlora_sample_first": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]),
     "mlora_generate": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]),
     "mlora_generate_host": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]),
+    "mlora_set_forecast": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32]),
+    "mlora_ds2d_round": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32] + [C.c_void_p] * 6 + [C.c_int32, C.c_int32] +
+                         [C.c_void_p] * 5),
     "mlora_export_state": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int32), C.c_void_p, C.c_void_p]),
     "mlora_debug_dequant": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "mlora_debug_set": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32]),
@@ -205,6 +208,20 @@ def mlora_generate_host(ctx, adapter_idx, first_tokens, out_tokens):
         assert not t.is_cuda and t.is_contiguous() and t.dtype == torch.int32
     _check(lib().mlora_generate_host(ctx, n, C.c_void_p(adapter_idx.data_ptr()), C.c_void_p(first_tokens.data_ptr()), k,
                                      C.c_void_p(out_tokens.data_ptr())))
+
+
+def mlora_set_forecast(ctx, forecast):
+    """forecast: CUDA fp16 [m][d_model] (kept alive by the caller) or None"""
+    _check(lib().mlora_set_forecast(ctx, _ptr(forecast), 0 if forecast is None else forecast.shape[0]))
+
+
+def mlora_ds2d_round(ctx, adapter_idx, tree_tokens, tree_parent, row_level, row_rank, forecast_of, widths, max_width,
+                     out_accept_len, out_accept_idx, out_next, out_tree_tokens, out_logits=None):
+    n, R = tree_tokens.shape
+    _check(lib().mlora_ds2d_round(ctx, n, _ptr(adapter_idx), R, _ptr(tree_tokens), _ptr(tree_parent), _ptr(row_level),
+                                  _ptr(row_rank), _ptr(forecast_of), _ptr(widths), widths.numel(), max_width,
+                                  _ptr(out_accept_len), _ptr(out_accept_idx), _ptr(out_next), _ptr(out_tree_tokens),
+                                  _ptr(out_logits)))
 
 
 def mlora_reset_streams(ctx):

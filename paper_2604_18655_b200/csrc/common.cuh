@@ -285,7 +285,12 @@ bool gemm_tc_eligible(const GemmArgs& a);
 cudaError_t launch_gemm_tc(const GemmArgs& a, int sm_count, int* status, cudaStream_t st);
 cudaError_t launch_shrink(const ShrinkArgs& a, cudaStream_t st);
 cudaError_t launch_embed(const int32_t* tokens, const __half* embed, const __half* hidden_in, float* X, int M,
-                         int d, int vocab, int* status, cudaStream_t st);
+                         int d, int vocab, int* status, cudaStream_t st, const __half* forecast = nullptr,
+                         int n_forecast = 0);
+cudaError_t launch_draft(const float* logits, int V, int n, int R, int m, int wmax, const int32_t* widths,
+                         const int32_t* level, const int32_t* rank, const int32_t* forecast_of, const int32_t* acc_len,
+                         const int32_t* acc_idx, const int32_t* next, int32_t* cand, int32_t* out_tokens, int* status,
+                         cudaStream_t st);
 cudaError_t launch_tree_prep(const int32_t* parent, int n, int T, unsigned long long* anc, int32_t* depth,
                              int* status, cudaStream_t st);
 void attn_plan(AttnArgs& a, int sm_count);

@@ -33,9 +33,11 @@ void free_packed(PackedWeight& w) {
   w.data = nullptr;
 }
 
+constexpr int MAX_FORECAST = 8, MAX_DRAFT_WIDTH = 32;
+
 struct GraphKey {
   int kind, n, T, prefix_chunk, n_prefix_chunks, own_chunk, n_own_chunks, flags, suffix_bound, pad_;
-  const void* p[8];
+  const void* p[12];
   bool operator==(const GraphKey& o) const { return std::memcmp(this, &o, sizeof(GraphKey)) == 0; }
 };
 struct GraphKeyHash {
@@ -99,6 +101,9 @@ struct mlora_ctx {
   int dbg_skip_compact = 0, dbg_no_graph = 0, dbg_no_chain = 0, dbg_no_tc = 0, dbg_inject_stall = 0;
   int step_mode = 0;                 // decode steps: 0 = the library's choice, 1 = per-layer kernels, 2 = the single-kernel step
   int32_t* host_io = nullptr;        // dev [3][max_streams]: adapter_idx, tokens, next of the host-buffer step
+  const __half* forecast = nullptr;  // caller-owned dev fp16 [n_forecast][d_model] (DS2D forecast embeddings)
+  int n_forecast = 0;
+  int32_t* draft_cand = nullptr;     // dev [max_streams][MAX_FORECAST][MAX_DRAFT_WIDTH]: candidates of a drafting round
   int32_t* gen_tokens = nullptr;     // dev [k][n]: the tokens of a host-buffer generation (grown on demand)
   size_t gen_capacity = 0;
   // persistent projection chain (rows <= 8)
@@ -287,7 +292,7 @@ int forward_chain(mlora_ctx* c, const PassIO& io) {
   const mlora_model_desc& d = c->d;
   cudaStream_t st = c->stream;
   const int M = io.n * io.T;
-  CK(run(c, MLORA_PROF_MISC, [&] { return launch_embed(io.tokens, (const __half*)d.embed, io.hidden_in, c->X, M, d.d_model, d.vocab, c->status, st); }));
+  CK(run(c, MLORA_PROF_MISC, [&] { return launch_embed(io.tokens, (const __half*)d.embed, io.hidden_in, c->X, M, d.d_model, d.vocab, c->status, st, c->forecast, c->n_forecast); }));
   CK(run(c, MLORA_PROF_MISC, [&] { return launch_tree_prep(io.parent, io.n, io.T, c->anc, c->depth, c->status, st); }));
   ChainArgs a{};
   a.phases = c->phases;
@@ -353,7 +358,7 @@ int forward(mlora_ctx* c, const PassIO& io) {
   cudaStream_t st = c->stream;
   const int M = io.n * io.T;
   const int dm = d.d_model, F = d.d_ffn;
-  CK(run(c, MLORA_PROF_MISC, [&] { return launch_embed(io.tokens, (const __half*)d.embed, io.hidden_in, c->X, M, dm, d.vocab, c->status, st); }));
+  CK(run(c, MLORA_PROF_MISC, [&] { return launch_embed(io.tokens, (const __half*)d.embed, io.hidden_in, c->X, M, dm, d.vocab, c->status, st, c->forecast, c->n_forecast); }));
   CK(run(c, MLORA_PROF_MISC, [&] { return launch_tree_prep(io.parent, io.n, io.T, c->anc, c->depth, c->status, st); }));
   for (int l = 0; l < c->L; ++l) {
     // attention block
@@ -675,6 +680,7 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
     CKC(cudaMalloc(&c->att_ws, c->att_ws_floats * sizeof(float)));
   }
   CKC(cudaMalloc(&c->host_io, 3 * (size_t)d.max_streams * sizeof(int32_t)));
+  CKC(cudaMalloc(&c->draft_cand, (size_t)d.max_streams * MAX_FORECAST * MAX_DRAFT_WIDTH * sizeof(int32_t)));
   CKC(cudaMalloc(&c->anc, Mm * sizeof(unsigned long long)));
   CKC(cudaMalloc(&c->depth, Mm * sizeof(int32_t)));
   CKC(cudaMalloc(&c->argmax, Mm * sizeof(int32_t)));
@@ -888,7 +894,7 @@ int mlora_destroy(mlora_ctx* c) {
                       c->h, c->attn16, c->act16, c->counters, c->anc, c->depth, c->argmax, c->suffix_len,
                       c->zero_len, c->chain_parent, c->root_parent, c->status, c->cs_table, (void*)c->tabA,
                       (void*)c->tabB, c->ad_scale, c->phases, c->chain_sync, c->host_io, c->step_phases, c->xg_attn, c->xg_ffn,
-                      c->step_tacc, c->step_ssq, c->step_amax, c->step_trace, c->tmapA, c->tmapB, c->gen_tokens};
+                      c->step_tacc, c->step_ssq, c->step_amax, c->step_trace, c->tmapA, c->tmapB, c->gen_tokens, c->draft_cand};
   for (void* p : dev_ptrs) if (p) cudaFree(p);
   if (c->stageA) cudaFreeHost((void*)c->stageA);
   if (c->stageB) cudaFreeHost((void*)c->stageB);
@@ -1125,9 +1131,16 @@ int mlora_decode_step_h(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_
   return decode_impl(c, n_streams, adapter_idx, nullptr, (const __half*)hidden_in, nullptr, nullptr, hidden_out);
 }
 
-int mlora_verify_tree(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_idx, int32_t n_nodes,
-                      const int32_t* tree_tokens, const int32_t* tree_parent, int32_t* out_accept_len,
-                      int32_t* out_accept_idx, int32_t* out_next, float* out_logits) {
+// what a drafting round adds to a verify pass (all device arrays; the templates are shared by the streams)
+struct DraftIO {
+  const int32_t *level, *rank, *forecast_of, *widths;
+  int m, wmax;
+  int32_t* out_tokens;
+};
+
+static int verify_impl(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_idx, int32_t n_nodes,
+                       const int32_t* tree_tokens, const int32_t* tree_parent, int32_t* out_accept_len,
+                       int32_t* out_accept_idx, int32_t* out_next, float* out_logits, const DraftIO* draft) {
   if (check_ctx(c)) return MLORA_ERR_ARG;
   if (c->d.vocab == 0) return fail(MLORA_ERR_STATE, "verification needs logits: context has no vocabulary");
   if (!tree_tokens || !tree_parent || !out_accept_len || !out_accept_idx || !out_next)
@@ -1141,13 +1154,19 @@ int mlora_verify_tree(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_id
   io.logits = out_logits ? out_logits : c->logits;
   plan_pass(c, io);
   GraphKey key{};
-  key.kind = 3; key.n = n; key.T = T;
+  key.kind = draft ? 5 : 3; key.n = n; key.T = T;
   key.prefix_chunk = io.plan.prefix_chunk; key.n_prefix_chunks = io.plan.n_prefix_chunks;
   key.own_chunk = io.plan.own_chunk; key.n_own_chunks = io.plan.n_own_chunks;
   key.flags = c->P * 8 + c->dbg_no_tc * 4 + c->dbg_skip_compact * 2 + c->dbg_no_chain;
   key.suffix_bound = io.plan.suffix_bound;
   key.p[0] = adapter_idx; key.p[1] = tree_tokens; key.p[2] = tree_parent; key.p[3] = out_accept_len;
   key.p[4] = out_accept_idx; key.p[5] = out_next; key.p[6] = out_logits;
+  if (draft) {
+    key.p[7] = draft->level; key.p[8] = draft->rank; key.p[9] = draft->forecast_of; key.p[10] = draft->widths;
+    key.p[11] = draft->out_tokens;
+    key.flags += (draft->m * 64 + draft->wmax) * 65536;
+  }
+  key.pad_ = c->n_forecast;
   rc = replay_or_run(c, key, [&]() -> int {
     int r = forward(c, io);
     if (r != MLORA_OK) return r;
@@ -1160,6 +1179,16 @@ int mlora_verify_tree(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_id
                               c->d.n_kv_heads, c->d.head_dim, c->suffix_len, out_accept_len, out_accept_idx, T, st);
       }));
       CK(run(c, MLORA_PROF_MISC, [&] { return launch_advance(c->suffix_len, out_accept_len, n, 0, st); }));
+    }
+    if (draft) {
+      // the next tree, from the forecast rows of every stream's last accepted node (two launches)
+      if (c->capturing) c->captured_nodes++;
+      else c->launches++;
+      CK(run(c, MLORA_PROF_MISC, [&] {
+        return launch_draft(io.logits, c->d.vocab, n, T, draft->m, draft->wmax, draft->widths, draft->level, draft->rank,
+                            draft->forecast_of, out_accept_len, out_accept_idx, out_next, c->draft_cand, draft->out_tokens,
+                            c->status, st);
+      }));
     }
     return MLORA_OK;
   });
@@ -1176,6 +1205,40 @@ int mlora_verify_tree(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_id
     }
   }
   return MLORA_OK;
+}
+
+int mlora_verify_tree(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_idx, int32_t n_nodes,
+                      const int32_t* tree_tokens, const int32_t* tree_parent, int32_t* out_accept_len,
+                      int32_t* out_accept_idx, int32_t* out_next, float* out_logits) {
+  return verify_impl(c, n_streams, adapter_idx, n_nodes, tree_tokens, tree_parent, out_accept_len, out_accept_idx, out_next,
+                     out_logits, nullptr);
+}
+
+int mlora_set_forecast(mlora_ctx* c, const void* forecast, int32_t m) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (c->d.vocab == 0) return fail(MLORA_ERR_STATE, "forecast rows need a vocabulary");
+  if (forecast == nullptr || m == 0) { c->forecast = nullptr; c->n_forecast = 0; return MLORA_OK; }
+  if (m < 0 || m > MAX_FORECAST) return fail(MLORA_ERR_ARG, "between 1 and 8 forecast embeddings");
+  if (reinterpret_cast<uintptr_t>(forecast) & 3) return fail(MLORA_ERR_ARG, "forecast must be 4-byte aligned");
+  c->forecast = (const __half*)forecast;
+  c->n_forecast = m;
+  return MLORA_OK;
+}
+
+int mlora_ds2d_round(mlora_ctx* c, int32_t n_streams, const int32_t* adapter_idx, int32_t n_rows, const int32_t* tree_tokens,
+                     const int32_t* tree_parent, const int32_t* row_level, const int32_t* row_rank,
+                     const int32_t* forecast_of, const int32_t* widths, int32_t m, int32_t max_width,
+                     int32_t* out_accept_len, int32_t* out_accept_idx, int32_t* out_next, int32_t* out_tree_tokens,
+                     float* out_logits) {
+  if (check_ctx(c)) return MLORA_ERR_ARG;
+  if (!row_level || !row_rank || !forecast_of || !widths || !out_tree_tokens) return fail(MLORA_ERR_ARG, "null argument");
+  if (c->n_forecast == 0) return fail(MLORA_ERR_STATE, "no forecast embeddings: call mlora_set_forecast first");
+  if (m < 1 || m > c->n_forecast) return fail(MLORA_ERR_ARG, "m exceeds the forecast embeddings set");
+  if (max_width < 1 || max_width > MAX_DRAFT_WIDTH || max_width > c->d.vocab) return fail(MLORA_ERR_ARG, "max_width must be 1..32");
+  if (out_tree_tokens == tree_tokens) return fail(MLORA_ERR_ARG, "out_tree_tokens must not alias tree_tokens");
+  DraftIO dr{row_level, row_rank, forecast_of, widths, m, max_width, out_tree_tokens};
+  return verify_impl(c, n_streams, adapter_idx, n_rows, tree_tokens, tree_parent, out_accept_len, out_accept_idx, out_next,
+                     out_logits, &dr);
 }
 
 int mlora_reset_streams(mlora_ctx* c) {

@@ -1,25 +1,32 @@
 // Small kernels around the projections: embedding gather, draft-tree preparation (ancestor masks and
 // depths, Sec. 3.5 / App. A.2), row argmax, the streams' first tokens (App. A.1), the greedy longest-accepted-path
 // walk and the KV compaction that follows it (Sec. 3.5).  (RoPE and the KV append of a pass happen inside the attention kernel.)
+#include "../../include/mlora.h"
 #include "common.cuh"
 
 namespace mlora {
 
 // ----------------------------------------------------------------------------- embedding / hidden input
+// An id in [vocab, vocab + n_forecast) stands for a forecast row (Sec. 3.5: forecast embeddings ride along with the
+// tokens of a DS2D pass): its input is the forecast embedding of that index.
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const __half* __restrict__ embed,
                              const __half* __restrict__ hidden_in, float* __restrict__ X, int d, int vocab,
-                             int* __restrict__ status) {
+                             const __half* __restrict__ forecast, int n_forecast, int* __restrict__ status) {
   const int m = blockIdx.x;
   const __half* src;
   if (hidden_in != nullptr) {
     src = hidden_in + (size_t)m * d;
   } else {
     int tok = tokens[m];
-    if (tok < 0 || tok >= vocab) {           // keep the access in bounds, report through the status word
-      if (threadIdx.x == 0) atomicCAS(status, 0, -1);
-      tok = 0;
+    if (tok >= vocab && tok < vocab + n_forecast) {
+      src = forecast + (size_t)(tok - vocab) * d;
+    } else {
+      if (tok < 0 || tok >= vocab) {         // keep the access in bounds, report through the status word
+        if (threadIdx.x == 0) atomicCAS(status, 0, -1);
+        tok = 0;
+      }
+      src = embed + (size_t)tok * d;
     }
-    src = embed + (size_t)tok * d;
   }
   for (int k = threadIdx.x * 2; k < d; k += blockDim.x * 2) {
     const float2 v = __half22float2(*reinterpret_cast<const __half2*>(src + k));
@@ -28,8 +35,8 @@ __global__ void embed_kernel(const int32_t* __restrict__ tokens, const __half* _
 }
 
 cudaError_t launch_embed(const int32_t* tokens, const __half* embed, const __half* hidden_in, float* X, int M, int d,
-                         int vocab, int* status, cudaStream_t st) {
-  embed_kernel<<<M, 256, 0, st>>>(tokens, embed, hidden_in, X, d, vocab, status);
+                         int vocab, int* status, cudaStream_t st, const __half* forecast, int n_forecast) {
+  embed_kernel<<<M, 256, 0, st>>>(tokens, embed, hidden_in, X, d, vocab, forecast, forecast ? n_forecast : 0, status);
   return cudaGetLastError();
 }
 
@@ -137,7 +144,8 @@ __device__ __forceinline__ unsigned long long topn_key(float v, int i) {
   return ((unsigned long long)ord << 32) | (unsigned)(0xffffffffu - (unsigned)i);
 }
 
-__global__ void __launch_bounds__(1024) topn_kernel(const float* __restrict__ logits, int V, int n, int32_t* __restrict__ out) {
+// the n largest entries of logits[0..V) by a whole CTA of 1024 threads; out may be global or shared memory
+__device__ __forceinline__ void block_topn(const float* __restrict__ logits, int V, int n, int32_t* out) {
   __shared__ unsigned long long sb[32];
   __shared__ unsigned long long s_prev;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -170,6 +178,56 @@ __global__ void __launch_bounds__(1024) topn_kernel(const float* __restrict__ lo
     __syncthreads();
     prev = s_prev;
   }
+}
+
+__global__ void __launch_bounds__(1024) topn_kernel(const float* __restrict__ logits, int V, int n, int32_t* __restrict__ out) {
+  block_topn(logits, V, n, out);
+}
+
+// ----------------------------------------------------------------------------- DS2D draft generation (Sec. 3.5, App. A.2)
+// After the accept walk the next tree hangs off the LAST ACCEPTED node: CTA (j, s) takes the logits of forecast row
+// j + 1 of that node of stream s and lists its widths[j] most probable ids (ties by rising id) in cand[s][j][.].
+__global__ void __launch_bounds__(1024) draft_topk_kernel(const float* __restrict__ logits, int V, int R, int m, int wmax,
+                                                        const int32_t* __restrict__ widths, const int32_t* __restrict__ forecast_of,
+                                                        const int32_t* __restrict__ acc_len, const int32_t* __restrict__ acc_idx,
+                                                        int32_t* __restrict__ cand, int* __restrict__ status) {
+  const int j = blockIdx.x, s = blockIdx.y;
+  int leaf = acc_idx[(size_t)s * R + acc_len[s] - 1];
+  if (leaf < 0 || leaf >= R) leaf = 0;
+  int row = forecast_of[leaf] + j;
+  int w = widths[j];
+  if (row < 0 || row >= R || w < 0 || w > wmax) {      // a malformed template: stay in bounds, report
+    if (threadIdx.x == 0) atomicCAS(status, 0, MLORA_ERR_ARG);
+    row = 0;
+    w = w < 0 ? 0 : wmax;
+  }
+  block_topn(logits + ((size_t)s * R + row) * V, V, w, cand + ((size_t)s * m + j) * wmax);
+}
+// The next pass's inputs, row by row: the root takes the bonus token, a draft node of depth d and sibling rank r the
+// r-th candidate of forecast row d, a forecast row j the id vocab + j - 1.
+__global__ void draft_fill_kernel(const int32_t* __restrict__ level, const int32_t* __restrict__ rank,
+                                  const int32_t* __restrict__ cand, const int32_t* __restrict__ next, int n, int R, int m,
+                                  int wmax, int V, int32_t* __restrict__ out_tokens, int* __restrict__ status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n * R) return;
+  const int s = i / R, lv = level[i % R], rk = rank[i % R];
+  int tok;
+  if (lv == 0) tok = next[s];
+  else if (lv > 0 && lv <= m && rk >= 0 && rk < wmax) tok = cand[((size_t)s * m + (lv - 1)) * wmax + rk];
+  else if (lv < 0 && -lv <= m) tok = V + (-lv) - 1;
+  else { atomicCAS(status, 0, MLORA_ERR_ARG); tok = 0; }
+  out_tokens[i] = tok;
+}
+
+cudaError_t launch_draft(const float* logits, int V, int n, int R, int m, int wmax, const int32_t* widths,
+                         const int32_t* level, const int32_t* rank, const int32_t* forecast_of, const int32_t* acc_len,
+                         const int32_t* acc_idx, const int32_t* next, int32_t* cand, int32_t* out_tokens, int* status,
+                         cudaStream_t st) {
+  draft_topk_kernel<<<dim3((unsigned)m, (unsigned)n), 1024, 0, st>>>(logits, V, R, m, wmax, widths, forecast_of, acc_len, acc_idx, cand, status);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  draft_fill_kernel<<<(n * R + 255) / 256, 256, 0, st>>>(level, rank, cand, next, n, R, m, wmax, V, out_tokens, status);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_topn(const float* logits, int V, int n, int32_t* out, cudaStream_t st) {

@@ -451,6 +451,91 @@ def test_decode_over_a_long_shared_prompt(GpuModel):
     gm.close()
 
 
+def test_ds2d_rounds_verify_and_draft_on_the_device(GpuModel):
+    """DS2D inference steps (Sec. 3.5, App. A.2): every pass verifies a (3,2) tree and drafts the next one from the
+    forecast rows of the last accepted node, the drafted tokens staying on the device.  Follow mode: the oracle walks on
+    the GPU's row argmax; accept results and the cache are exact, logits within tolerance, and the drafts are exactly
+    the top ids of the GPU's own forecast logits (and near-maximal in the oracle's)."""
+    from dataclasses import replace
+    from paper_2604_18655_b200 import binding as mb
+    # (adapters a few times the base projection, not TINYV's ten times: with random draft tokens at every node the
+    # fp16 activations' rounding, amplified by the adapter branch, otherwise sits right at the logit tolerance)
+    cfg = replace(TINYV, name="tinyds2d", b_std=0.02)
+    t = gen.ds2d_template((3, 2))
+    R, m, V, n = t["R"], t["m"], cfg.vocab, cfg.n_streams
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        mdl, orc, gm = make_pair(GpuModel, cfg, max_suffix=40, max_tree=R)
+        fc = gen.make_forecast(cfg, m, 0)
+        d_fc = torch.from_numpy(fc).cuda()
+        mb.mlora_set_forecast(gm.ctx, d_fc)
+        orc.set_forecast(fc)
+        ids = gen.make_prompt_ids(cfg, 0)
+        last = gm.prefill(ids)
+        orc.prefill_shared(ids, n_streams=n)
+        ad = [2, -1, 0]
+        dv = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+        d_ad = dv(np.array(ad, dtype=np.int32))
+        d_par = dv(np.stack([t["parent"]] * n))
+        d_lvl, d_rank, d_fo, d_w = dv(t["level"]), dv(t["rank"]), dv(t["forecast_of"]), dv(t["widths"])
+        tt = np.zeros((n, R), dtype=np.int32)
+        tt[:, 0] = ref.first_tokens(last, n)
+        tt[:, 1:t["T"]] = np.random.default_rng(0).integers(0, V, size=(n, t["T"] - 1))
+        tt[:, t["level"] < 0] = (V - np.minimum(t["level"], 0) - 1)[t["level"] < 0]
+        bufs = [dv(tt), torch.empty(n, R, dtype=torch.int32, device="cuda")]
+        acc_len = torch.empty(n, dtype=torch.int32, device="cuda")
+        acc_idx = torch.empty(n, R, dtype=torch.int32, device="cuda")
+        nxt = torch.empty(n, dtype=torch.int32, device="cuda")
+        logits = torch.empty(n * R, V, dtype=torch.float32, device="cuda")
+        accepted = 0
+        for rnd in range(5):
+            cur, out = bufs[rnd & 1], bufs[(rnd + 1) & 1]
+            h_tt = cur.cpu().numpy().copy()
+            if rnd in (1, 3):                           # plant the true continuation on a draft node of stream 0 (and
+                probe = orc.verify_tree(ad, np.stack([t["parent"]] * n), h_tt, commit=False)    # its child in round 3)
+                h_tt[0, 2] = probe["argmax"][0, 0]
+                if rnd == 3:
+                    probe = orc.verify_tree(ad, np.stack([t["parent"]] * n), h_tt, commit=False)
+                    h_tt[0, 7] = probe["argmax"][0, 2]
+                cur.copy_(dv(h_tt))
+            mb.mlora_ds2d_round(gm.ctx, d_ad, cur, d_par, d_lvl, d_rank, d_fo, d_w, int(t["widths"].max()),
+                                acc_len, acc_idx, nxt, out, logits)
+            side.synchronize()
+            g_logits = logits.cpu().numpy()
+            r = orc.ds2d_round(ad, t, h_tt, follow_argmax=np.argmax(g_logits, axis=1).reshape(n, R))
+            compare(g_logits, r["logits"], f"ds2d round {rnd} logits")
+            assert np.array_equal(acc_len.cpu().numpy(), r["accept_len"])
+            assert np.array_equal(acc_idx.cpu().numpy(), r["accept_idx"])
+            assert np.array_equal(nxt.cpu().numpy(), r["next"])
+            accepted += int(r["accept_len"].sum()) - n
+            g_next = out.cpu().numpy()
+            o_lg = r["logits"].reshape(n, R, V)
+            for s in range(n):
+                leaf = int(r["accept_idx"][s][r["accept_len"][s] - 1])
+                for i in range(R):
+                    lv = int(t["level"][i])
+                    if lv == 0:
+                        assert g_next[s, i] == nxt[s].item()
+                    elif lv < 0:
+                        assert g_next[s, i] == V - lv - 1
+                    else:
+                        row = s * R + int(t["forecast_of"][leaf]) + lv - 1
+                        want = ref.first_tokens(g_logits[row], int(t["widths"][lv - 1]))[int(t["rank"][i])]
+                        assert g_next[s, i] == want, (rnd, s, i)
+                        o_row = o_lg[s, int(t["forecast_of"][leaf]) + lv - 1]
+                        kth = np.sort(o_row)[::-1][int(t["rank"][i])]
+                        assert abs(o_row[g_next[s, i]] - kth) <= 1e-2       # the oracle's r-th best, up to near-ties
+        assert accepted >= 3
+        compare_kv(gm, orc, cfg, n)
+        # the second call with the same arguments replays the captured graph: same outputs
+        mb.mlora_sync_status(gm.ctx)
+        mb.mlora_set_forecast(gm.ctx, None)
+        with pytest.raises(mb.MloraError) as e:
+            mb.mlora_ds2d_round(gm.ctx, d_ad, bufs[1], d_par, d_lvl, d_rank, d_fo, d_w, 3, acc_len, acc_idx, nxt, bufs[0])
+        assert e.value.code == -2
+        gm.close()
+
+
 def test_sample_first_matches_oracle(GpuModel):
     """The n distinct first tokens (App. A.1): integer work, exact -- with ties, infinities, signed zeros and NaN."""
     from paper_2604_18655_b200 import binding as mb
