@@ -47,6 +47,9 @@ def parse_args():
     ap.add_argument("--config", default="cfg1", choices=["cfg0", "cfg1", "cfg2", "cfg3", "cfg4"],
                     help="cfg1 (default) is the benchmark workload; cfg2/cfg3 time DS2D verify rounds; cfg4 is the "
                          "kernel-level sweep (one JSON line with a list of points; --markdown prints tables)")
+    ap.add_argument("--draft", action="store_true",
+                    help="cfg2/cfg3: DS2D rounds that also draft the next tree on the device ((3,2) trees with two forecast "
+                         "rows per node, 30 rows per stream, synthetic forecast embeddings) instead of host-made drafts")
     ap.add_argument("--quick", action="store_true", help="cfg4: a small sub-grid")
     ap.add_argument("--markdown", action="store_true", help="cfg4: markdown tables instead of the JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -214,11 +217,12 @@ def run_reference(args, cfg):
         return
     K = args.steps if args.steps is not None else 6
     W = args.warmup if args.warmup is not None else 3
+    import gen
     synth, adapters = build_inputs(cfg)
     if cfg.tree_nodes > 1:
         # verify passes: a handful at most (a pass of the ~3B model is tens of seconds of CPU work)
         k_run = min(K + W, 3 if cfg.d_model <= 2048 else 1)
-        val, dt, desc = oracle_verify_sample(cfg, synth, adapters, k_run)
+        val, dt, desc = oracle_verify_sample(cfg, synth, adapters, k_run, gen.ds2d_template((3, 2)) if args.draft else None)
         metric, unit = "DS2D verify rows/s", "rows/s"
     else:
         # bound the run to a few minutes whatever K is: past 40 steps, time 40 and report the per-step mean
@@ -237,7 +241,7 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
-def oracle_verify_sample(cfg, synth, adapters, n_rounds):
+def oracle_verify_sample(cfg, synth, adapters, n_rounds, tpl=None):
     """Times the CPU oracle, as it stands, on n_rounds DS2D verify passes (all streams' trees in one pass) after a
     short prefill.  Returns (rows_per_s, seconds, description)."""
     import gen
@@ -245,23 +249,30 @@ def oracle_verify_sample(cfg, synth, adapters, n_rounds):
     orc = ref.OracleModel.from_synth(synth, dtype=np.float32)
     for a, (A, B) in enumerate(adapters):
         orc.set_adapter(a, A, B, cfg.alpha)
-    n, T = cfg.n_streams, cfg.tree_nodes
+    n, T = cfg.n_streams, cfg.tree_nodes if tpl is None else tpl["R"]
     orc.prefill_shared(gen.make_prompt_ids(cfg, 0, ORACLE_PREFIX), n_streams=n)
     ad = list(range(n))
-    parents = np.stack([gen.build_tree(cfg.branch, T)] * n)
+    parents = np.stack([gen.build_tree(cfg.branch, T) if tpl is None else tpl["parent"]] * n)
     cand = gen.make_candidates(cfg, n_rounds + 1, n, T, 0)
     tt = np.empty((n, T), dtype=np.int32)
     nxt = np.arange(n, dtype=np.int32) + 1
+    if tpl is not None:
+        orc.set_forecast(gen.make_forecast(cfg, tpl["m"], 0))
+        tt[:, 0], tt[:, 1:] = nxt, cand[0]
+        tt[:, tpl["level"] < 0] = (cfg.vocab - tpl["level"] - 1)[tpl["level"] < 0]
     dt = 0.0
     for i in range(n_rounds + 1):                   # the first, untimed pass also pays the lazy dequantisation
-        tt[:, 0] = nxt
-        tt[:, 1:] = cand[i]
         t0 = time.perf_counter()
-        nxt = orc.verify_tree(ad, parents, tt)["next"]
+        if tpl is None:
+            tt[:, 0] = nxt
+            tt[:, 1:] = cand[i]
+            nxt = orc.verify_tree(ad, parents, tt)["next"]
+        else:
+            tt = orc.ds2d_round(ad, tpl, tt)["next_tree_tokens"]
         if i:
             dt += time.perf_counter() - t0
-    desc = (f"{n_rounds} verify passes of {n} streams x {T}-node trees of {cfg.name} after a {ORACLE_PREFIX}-token "
-            f"prefill (numpy fp32, dense dequantised weights)")
+    desc = (f"{n_rounds} {'drafting rounds' if tpl is not None else 'verify passes'} of {n} streams x {T} rows of {cfg.name} "
+            f"after a {ORACLE_PREFIX}-token prefill (numpy fp32, dense dequantised weights)")
     return n * T * n_rounds / dt, dt, desc
 
 
@@ -286,6 +297,9 @@ def run_verify(args, cfg):
     side = torch.cuda.Stream()
     synth, adapters = build_inputs(cfg)
     n, T = cfg.n_streams, cfg.tree_nodes
+    tpl = gen.ds2d_template((3, 2)) if args.draft else None
+    if tpl is not None:
+        T = tpl["R"]                                 # rows per stream: 10 token nodes + 20 forecast rows (Sec. 3.5's example)
     Ke = min(K, 64)
     ROUNDS_PER_GEN = 32                              # streams restart (own segments emptied) every so many rounds
     with torch.cuda.stream(side):
@@ -296,7 +310,8 @@ def run_verify(args, cfg):
         ids = torch.from_numpy(gen.make_prompt_ids(cfg, 0)).to(dev)
         last = torch.empty(cfg.vocab, dtype=torch.float32, device=dev)
         mb.mlora_prefill_shared(ctx, ids, last)
-        parent = torch.from_numpy(np.stack([gen.build_tree(cfg.branch, T)] * n).astype(np.int32)).to(dev)
+        tree_parent = tpl["parent"] if tpl is not None else gen.build_tree(cfg.branch, T)
+        parent = torch.from_numpy(np.stack([tree_parent] * n).astype(np.int32)).to(dev)
         cand = torch.from_numpy(gen.make_candidates(cfg, 64, n, T, 0)).to(dev)
         tt = torch.empty(n, T, dtype=torch.int32, device=dev)
         acc_len = torch.empty(n, dtype=torch.int32, device=dev)
@@ -306,13 +321,33 @@ def run_verify(args, cfg):
         ad = torch.arange(n, dtype=torch.int32, device=dev)
         emitted = torch.zeros(1, dtype=torch.int64, device=dev)
 
+        if tpl is not None:
+            forecast = torch.from_numpy(gen.make_forecast(cfg, tpl["m"], 0)).to(dev)
+            mb.mlora_set_forecast(ctx, forecast)
+            d_lvl, d_rank, d_fo, d_w = (torch.from_numpy(tpl[k]).to(dev) for k in ("level", "rank", "forecast_of", "widths"))
+            wmax = int(tpl["widths"].max())
+            tt0 = torch.empty(n, T, dtype=torch.int32, device=dev)       # the first tree of a generation: random drafts
+            tt0[:, 0] = first
+            tt0[:, 1:] = cand[0]
+            is_fc = d_lvl < 0
+            tt0[:, is_fc] = (cfg.vocab - d_lvl[is_fc] - 1).to(torch.int32)
+            tbuf, cur = [tt, torch.empty_like(tt)], [0]
+
         def round_(i):
             if i % ROUNDS_PER_GEN == 0:
                 mb.mlora_reset_streams(ctx)
                 nxt.copy_(first)
-            tt[:, 0] = nxt
-            tt[:, 1:] = cand[i % 64]
-            mb.mlora_verify_tree(ctx, ad, tt, parent, acc_len, acc_idx, nxt, None)
+                if tpl is not None:
+                    tbuf[cur[0]].copy_(tt0)
+            if tpl is not None:
+                # verify + draft: the next round's tree is written by this one, on the device
+                mb.mlora_ds2d_round(ctx, ad, tbuf[cur[0]], parent, d_lvl, d_rank, d_fo, d_w, wmax, acc_len, acc_idx, nxt,
+                                    tbuf[cur[0] ^ 1])
+                cur[0] ^= 1
+            else:
+                tt[:, 0] = nxt
+                tt[:, 1:] = cand[i % 64]
+                mb.mlora_verify_tree(ctx, ad, tt, parent, acc_len, acc_idx, nxt, None)
             emitted.add_(acc_len.sum())
 
         def barrier():
@@ -349,6 +384,14 @@ def run_verify(args, cfg):
         h_first = first.cpu()
 
         def e2e_round(i):
+            if tpl is not None:
+                # drafted on the device: nothing goes in; the host reads the accepted path and the bonus token
+                round_(i)
+                h_len.copy_(acc_len, non_blocking=True)
+                h_idx.copy_(acc_idx, non_blocking=True)
+                h_next.copy_(nxt, non_blocking=True)
+                side.synchronize()
+                return
             if i % ROUNDS_PER_GEN == 0:
                 mb.mlora_reset_streams(ctx)
                 h_next.copy_(h_first)
@@ -391,12 +434,15 @@ def run_verify(args, cfg):
         "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
         "data": "synthetic",
         "config": {"workload": f"{cfg.name}: d{cfg.d_model} L{cfg.n_layers} hd{cfg.head_dim} int4-g{cfg.group_size}; {n} streams x "
-                               f"{T}-node trees {cfg.branch}, shared prompt {cfg.prompt_len}, rank-{cfg.lora_rank} LoRA, "
-                               f"uniform-random drafts, streams restart every {ROUNDS_PER_GEN} rounds",
+                               + (f"{T} rows per stream = (3,2) trees of 10 token nodes + 2 forecast rows each, drafted on "
+                                  f"the device from synthetic forecast embeddings, " if tpl is not None else
+                                  f"{T}-node trees {cfg.branch}, uniform-random drafts, ")
+                               + f"shared prompt {cfg.prompt_len}, rank-{cfg.lora_rank} LoRA, "
+                               f"streams restart every {ROUNDS_PER_GEN} rounds",
                    "rows_per_pass": rows, "l2": "inputs larger than L2 (weights alone: %.0f MB)" % (params / 2e6),
                    "launch": "CUDA-graph replay per pass", "multi_gpu": "replicas only"},
         "clocks": clocks,
-        "e2e": {"value": world * rows / (ms_e2e / 1e3), "unit": "rows/s", "h2d_bytes_per_step": rows * 4,
+        "e2e": {"value": world * rows / (ms_e2e / 1e3), "unit": "rows/s", "h2d_bytes_per_step": 0 if tpl is not None else rows * 4,
                 "d2h_bytes_per_step": (n + rows + n) * 4, "steps": Ke, "ms_per_step": ms_e2e},
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "kernel": "w4_gemm_tc_kernel (tcgen05 INT4 projection with its split-K epilogue), "
@@ -413,7 +459,7 @@ def run_verify(args, cfg):
     }
     if rank == 0 and not args.no_cpu_baseline:
         n_or = 3 if cfg.d_model <= 2048 else 1
-        rps, dt, desc = oracle_verify_sample(cfg, synth, adapters, n_or)
+        rps, dt, desc = oracle_verify_sample(cfg, synth, adapters, n_or, tpl)
         line["cpu_baseline"] = {"value": rps, "unit": "rows/s", "cores": cores_used(), "kind": "oracle", "sample": desc,
                                 "seconds": dt}
     if rank == 0:
