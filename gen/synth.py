@@ -50,6 +50,20 @@ def quantize_int4(w: np.ndarray, group: int):
     return pack_nibbles((q + 8).astype(np.uint8)), scale
 
 
+def quantize_int4_per_channel(w: np.ndarray):
+    """Symmetric per-output-channel INT4 quantiser (input preparation for the INT4 x INT8 regime of Sec. 3.3).
+
+    w [K][N]; scale[n] = fp16(max_k |w[k][n]| / 7) (1 where that is 0); q = clip(round_half_even(w / scale), -8, 7).
+    Returns (packed uint8 [N][K/2]: channel-major, nibble q + 8, even k in the low nibble; fp16 [N])."""
+    K, N = w.shape
+    assert K % 2 == 0
+    w = w.astype(np.float32)
+    scale = (np.abs(w).max(axis=0) / np.float32(7.0)).astype(np.float16)
+    scale = np.where(scale == 0, np.float16(1.0), scale).astype(np.float16)
+    q = np.clip(np.rint(w / scale.astype(np.float32)[None, :]), -8, 7).astype(np.int8)
+    return pack_nibbles(np.ascontiguousarray((q + 8).astype(np.uint8).T)), scale
+
+
 @dataclass
 class SynthModel:
     cfg: ModelCfg

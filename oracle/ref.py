@@ -17,6 +17,8 @@ What follows which passage:
     a node sees the cached context plus its own ancestors               -- Sec. 3.5, App. A.2 (DS2D mask)
   * accepted drafts form one root path ("1-3-5"); first emitted token is
     the frozen model's own token (lossless)                              -- Sec. 3.5
+  * the paper's own precision regime: activations per-tensor INT8, weights
+    per-channel INT4, integer contraction (single projection)            -- Sec. 3.3 "LLM Quantization"
   * after the single prefill a sampler gives the n streams n distinct
     first tokens (here: the n most probable, by falling logit, ties by
     rising id), then the n-fold model runs step after step              -- App. A.1 (flowsheet)
@@ -39,7 +41,9 @@ small tree; the (3,2) -> 9/10/30 node counts and the 32-row budgets of Table 7; 
 (tests/test_oracle_wiring_pin.py); the first-token sampler against exhaustive selection on small rows with ties and
 against argmax for n = 1 (tests/test_oracle_generate.py); DS2D drafting: the printed row counts of the (3,2) example,
 forecast rows against the same vectors planted as ordinary embedding rows, draft placement by explicit loops, and
-losslessness of whole drafting rounds against plain greedy decoding (tests/test_oracle_ds2d_draft.py).
+losslessness of whole drafting rounds against plain greedy decoding (tests/test_oracle_ds2d_draft.py); the INT4 x INT8
+projection against Python-integer brute force, the float product of the dequantised operands and the quantisation error
+bound (tests/test_oracle_w4a8.py).
 Parity unpinned by the paper: absolute activation values of a forward pass of ITS model (it prints none).
 """
 import numpy as np
@@ -69,6 +73,28 @@ def dequant(qbytes: np.ndarray, scales: np.ndarray, group: int) -> np.ndarray:
     assert s.shape == q.shape
     with np.errstate(over="ignore"):
         return (q * s).astype(np.float16)
+
+
+# ----------------------------------------------------------------------------- the INT4 x INT8 regime (Sec. 3.3)
+def quantize_act_int8(x, scale):
+    """Per-tensor symmetric INT8 activations: q = clip(round_half_even(x / scale), -127, 127), the division carried in
+    float32 (the precision the kernel takes this decision in)."""
+    q = np.rint(np.asarray(x, dtype=np.float32) / np.float32(scale))
+    return np.clip(q, -127, 127).astype(np.int8)
+
+
+def linear_w4a8(qx, x_scale, qw_bytes, w_scale):
+    """Projection with per-channel INT4 weights and per-tensor INT8 activations (Sec. 3.3 "LLM Quantization":
+    activations per-tensor to Int8, weights per-channel to Int4).
+
+    qx int8 [M][K]; qw_bytes uint8 [N][K/2] (channel-major, nibble q + 8, even k low); w_scale fp16 [N].
+    The contraction is exact integer arithmetic; y[m][n] = float32(acc) * (float32(x_scale) * float32(w_scale[n])),
+    both products in float32 (the format fixes this precision, so the result is reproducible bit for bit)."""
+    qw = unpack_int4(np.asarray(qw_bytes)).astype(np.int64)            # [N][K]
+    acc = np.asarray(qx).astype(np.int64) @ qw.T                        # exact
+    assert np.abs(acc).max() < 2 ** 31
+    f = np.float32(x_scale) * np.asarray(w_scale).astype(np.float32)    # [N], float32
+    return acc.astype(np.float32) * f[None, :]
 
 
 # ----------------------------------------------------------------------------- elementwise pieces (Sec. 3.1)
