@@ -268,6 +268,20 @@ int mlora_linear_noalloc(mlora_weight* w, const void* x, int32_t M, const int32_
  * kernel's barrier words, so that the next call starts afresh.  Allocates nothing.  Errors: ARG, CUDA, TIMEOUT. */
 int mlora_linear_status(mlora_weight* w, void* workspace);
 
+/* ---- the paper's own precision regime, single projection (Sec. 3.3 "LLM Quantization": activations quantised per
+ * tensor to Int8, weights per channel to Int4) ----
+ * mlora_quantize_act_int8: out[i] = clip(round_half_even(x[i] / scale), -127, 127) with the division in float32.
+ * x dev fp16 [count], out dev int8 [count], scale > 0 (host).  Enqueued on cuda_stream.  Errors: ARG, CUDA.
+ * mlora_linear_w4a8: y[m][n] = float32(sum_k qx[m][k] * qw[n][k]) * (x_scale * float32(w_scale[n])): the sum in exact
+ * integer arithmetic (tensor cores, s8 x s8 -> s32), the two products in float32, so the result is reproducible bit
+ * for bit.  qweight dev uint8 [N][K/2] (channel-major; the nibble of input k is q + 8, even k in the low nibble);
+ * w_scale dev fp16 [N]; qx dev int8 [M][K]; y dev fp32 [M][N].  qweight and qx 16-byte aligned.  1 <= M <= 64,
+ * K a multiple of 256, N a multiple of 16 (UNSUPPORTED otherwise).  No adapter term, no scratch memory.
+ * Errors: ARG, UNSUPPORTED, CUDA. */
+int mlora_quantize_act_int8(const void* x_fp16, int64_t count, float scale, void* out_int8, void* cuda_stream);
+int mlora_linear_w4a8(const void* qweight, const void* w_scale, const void* qx, float x_scale, int32_t M, int32_t K,
+                      int32_t N, float* y, void* cuda_stream);
+
 /* Bytes of scratch for mlora_attention (the largest need over every suffix_bound up to own_capacity - n_nodes). */
 size_t mlora_attention_workspace_bytes(int32_t n_streams, int32_t n_nodes, int32_t n_q_heads, int32_t n_kv_heads,
                                        int32_t head_dim, int32_t prefix_len, int32_t own_capacity);

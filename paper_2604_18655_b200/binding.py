@@ -60,6 +60,9 @@ _SIGS = {
     "mlora_set_forecast": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32]),
     "mlora_ds2d_round": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32] + [C.c_void_p] * 6 + [C.c_int32, C.c_int32] +
                          [C.c_void_p] * 5),
+    "mlora_quantize_act_int8": (C.c_int, [C.c_void_p, C.c_int64, C.c_float, C.c_void_p, C.c_void_p]),
+    "mlora_linear_w4a8": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                    C.c_void_p]),
     "mlora_export_state": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_int32), C.c_void_p, C.c_void_p]),
     "mlora_debug_dequant": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "mlora_debug_set": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32]),
@@ -222,6 +225,17 @@ def mlora_ds2d_round(ctx, adapter_idx, tree_tokens, tree_parent, row_level, row_
                                   _ptr(row_rank), _ptr(forecast_of), _ptr(widths), widths.numel(), max_width,
                                   _ptr(out_accept_len), _ptr(out_accept_idx), _ptr(out_next), _ptr(out_tree_tokens),
                                   _ptr(out_logits)))
+
+
+def mlora_quantize_act_int8(x_fp16, scale, out_int8):
+    _check(lib().mlora_quantize_act_int8(_ptr(x_fp16), x_fp16.numel(), scale, _ptr(out_int8), _stream()))
+
+
+def mlora_linear_w4a8(qweight, w_scale, qx, x_scale, y):
+    """qweight uint8 [N][K/2], w_scale fp16 [N], qx int8 [M][K], y fp32 [M][N] (CUDA tensors)"""
+    M, K = qx.shape
+    _check(lib().mlora_linear_w4a8(_ptr(qweight), _ptr(w_scale), _ptr(qx), x_scale, M, K, qweight.shape[0], _ptr(y),
+                                   _stream()))
 
 
 def mlora_reset_streams(ctx):

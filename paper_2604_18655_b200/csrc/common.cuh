@@ -306,6 +306,10 @@ cudaError_t launch_compact(__half* own_k, __half* own_v, size_t layer_stride, si
                            size_t head_stride, int L, int n, int Hkv, int hd, const int32_t* suffix_len,
                            const int32_t* acc_len, const int32_t* acc_idx, int T, cudaStream_t st);
 cudaError_t launch_advance(int32_t* suffix_len, const int32_t* acc_len, int n, int fixed, cudaStream_t st);
+cudaError_t launch_quant_act(const __half* x, long long count, float scale, signed char* out, cudaStream_t st);
+bool w4a8_shape_ok(int M, int K, int N);
+cudaError_t launch_w4a8(const unsigned char* w, const __half* ws, const signed char* x, float x_scale, int M, int K, int N,
+                        float* y, cudaStream_t st);
 cudaError_t launch_copy_rows_f32(const float* src, float* dst, size_t count, cudaStream_t st);
 
 // ----------------------------------------------------------------------------- device helpers

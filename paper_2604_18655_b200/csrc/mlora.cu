@@ -1646,4 +1646,25 @@ int mlora_attention(const void* q, const void* prefix_k, const void* prefix_v, i
   return MLORA_OK;
 }
 
+int mlora_quantize_act_int8(const void* x_fp16, int64_t count, float scale, void* out_int8, void* cuda_stream) {
+  if (!x_fp16 || !out_int8 || count < 0) return fail(MLORA_ERR_ARG, "quantize_act_int8: null buffer or negative count");
+  if (!(scale > 0.f)) return fail(MLORA_ERR_ARG, "quantize_act_int8: scale must be positive");
+  if (count == 0) return MLORA_OK;
+  CK(launch_quant_act((const __half*)x_fp16, (long long)count, scale, (signed char*)out_int8, (cudaStream_t)cuda_stream));
+  return MLORA_OK;
+}
+
+int mlora_linear_w4a8(const void* qweight, const void* w_scale, const void* qx, float x_scale, int32_t M, int32_t K,
+                      int32_t N, float* y, void* cuda_stream) {
+  if (!qweight || !w_scale || !qx || !y) return fail(MLORA_ERR_ARG, "linear_w4a8: null argument");
+  if (M < 1 || K < 1 || N < 1) return fail(MLORA_ERR_ARG, "linear_w4a8: non-positive size");
+  if (!w4a8_shape_ok(M, K, N))
+    return fail(MLORA_ERR_UNSUPPORTED, "linear_w4a8: needs M <= 64, K a multiple of 256 (below 2^31 / 1016), N a multiple of 16");
+  if ((reinterpret_cast<uintptr_t>(qweight) & 15) || (reinterpret_cast<uintptr_t>(qx) & 15))
+    return fail(MLORA_ERR_ARG, "linear_w4a8: qweight and qx must be 16-byte aligned");
+  CK(launch_w4a8((const unsigned char*)qweight, (const __half*)w_scale, (const signed char*)qx, x_scale, M, K, N, y,
+                 (cudaStream_t)cuda_stream));
+  return MLORA_OK;
+}
+
 }  // extern "C"

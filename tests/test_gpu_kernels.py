@@ -234,6 +234,46 @@ def test_attention_one_row_per_stream_over_long_prefix(mb, n, Hq, Hkv, hd, P, su
     compare(got, want, f"attention stream hd{hd} {Hq}q/{Hkv}kv n{n} P{P}")
 
 
+@pytest.mark.parametrize("K,N", [(2048, 2048), (4096, 4096), (5632, 2048), (14336, 4096), (256, 16)])
+@pytest.mark.parametrize("M", [1, 3, 8, 9, 16, 31, 64])
+def test_w4a8_projection_is_bit_exact(mb, K, N, M):
+    """The paper's own regime (Sec. 3.3): per-channel INT4 weights x per-tensor INT8 activations.  Integer contraction and
+    float32 scaling in a fixed order on both sides: compared bit for bit, the activation quantiser too."""
+    rng = np.random.default_rng(K + N + M)
+    qb, sc = gen.quantize_int4_per_channel(rng.standard_normal((K, N)).astype(np.float32) * 0.02)
+    x = rng.standard_normal((M, K)).astype(np.float16)
+    sx = float(np.float32(np.abs(x.astype(np.float32)).max() / np.float32(127)))
+    d_qx = torch.empty(M, K, dtype=torch.int8, device="cuda")
+    mb.mlora_quantize_act_int8(dev(x), sx, d_qx)
+    qx = ref.quantize_act_int8(x, sx)
+    assert np.array_equal(d_qx.cpu().numpy(), qx)
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    mb.mlora_linear_w4a8(dev(qb), dev(sc), d_qx, sx, y)
+    torch.cuda.synchronize()
+    want = ref.linear_w4a8(qx, sx, qb, sc)
+    assert np.array_equal(y.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
+def test_w4a8_extreme_values_and_limits(mb):
+    """Every product at its largest magnitude (-8 x -127 and -8 x 127 over K = 14336 inputs stays inside 32 bits), and
+    the shapes outside the kernel's limits are refused on the host."""
+    K, N, M = 14336, 16, 2
+    qb = np.zeros((N, K // 2), dtype=np.uint8)                       # nibble 0 = q -8 everywhere
+    sc = np.full(N, 1.0, dtype=np.float16)
+    qx = np.stack([np.full(K, -127, dtype=np.int8), np.full(K, 127, dtype=np.int8)])
+    y = torch.empty(M, N, dtype=torch.float32, device="cuda")
+    mb.mlora_linear_w4a8(dev(qb), dev(sc), dev(qx), 1.0, y)
+    torch.cuda.synchronize()
+    assert np.array_equal(y.cpu().numpy(), ref.linear_w4a8(qx, 1.0, qb, sc))
+    assert y[0, 0].item() == float(np.float32(8 * 127 * K))
+    for bad in [(65, 256, 16), (1, 300, 16), (1, 256, 24)]:
+        Mb, Kb, Nb = bad
+        with pytest.raises(mb.MloraError) as e:
+            mb.mlora_linear_w4a8(torch.zeros(Nb, Kb // 2, dtype=torch.uint8, device="cuda"), torch.ones(Nb, dtype=torch.float16, device="cuda"),
+                                 torch.zeros(Mb, Kb, dtype=torch.int8, device="cuda"), 1.0, torch.empty(Mb, Nb, device="cuda"))
+        assert e.value.code == -6
+
+
 def test_attention_long_prefix_split(mb):
     got, want = run_attention(mb, 2, 1, 8, 2, 128, 3000, [64, 10], (), seed=3)
     compare(got, want, "attention P3000")
