@@ -569,6 +569,34 @@ def sweep_attention(stream, Ps, Ts, peak):
     return pts
 
 
+def sweep_w4a8(stream, shapes, Ms, peak):
+    """mlora_linear_w4a8 (per-channel INT4 weights x per-tensor INT8 activations, Sec. 3.3): bytes = nibbles + channel
+    scales + int8 activations + fp32 results."""
+    import torch
+    import gen
+    from paper_2604_18655_b200 import binding as mb
+    pts = []
+    rng = np.random.default_rng(0)
+    for K, N in shapes:
+        w_bytes = K * N // 2 + N * 2
+        n_copies = int(L2_BYTES // w_bytes) + 2
+        qb, sc = gen.quantize_int4_per_channel(rng.standard_normal((K, N)).astype(np.float32) * 0.02)
+        ws_ = [torch.from_numpy(qb).cuda() for _ in range(n_copies)]
+        dsc = torch.from_numpy(sc).cuda()
+        for M in Ms:
+            qx = torch.randint(-127, 128, (M, K), dtype=torch.int8, device="cuda")
+            y = torch.empty(M, N, device="cuda", dtype=torch.float32)
+
+            def body():
+                for w in ws_:
+                    mb.mlora_linear_w4a8(w, dsc, qx, 0.01, y)
+            ms = time_graph(stream, body, 20) / n_copies
+            bytes_ = w_bytes + M * (K + N * 4)
+            pts.append({"op": "linear_w4a8", "KxN": f"{K}x{N}", "rows": M, "us": ms * 1e3, "gbs": bytes_ / ms / 1e6,
+                        "frac_hbm": bytes_ / ms / 1e6 / peak, "tops": 2.0 * M * K * N / ms / 1e9})
+    return pts
+
+
 def run_sweep(args):
     """Kernel-level sweep (single projection and single attention pass through the C ABI).  One JSON line: `value` is
     the 8-row, 8-adapter, rank-16 projection of 4096 x 4096 in microseconds; every point sits in `points`."""
@@ -589,6 +617,7 @@ def run_sweep(args):
         t0 = time.time()
         lin = sweep_linear(stream, shapes, Ms, combos, peak)
         att = sweep_attention(stream, Ps, Ts, peak)
+        wa = sweep_w4a8(stream, shapes, [m for m in Ms if m <= 64] + ([64] if 64 not in Ms and not args.quick else []), peak)
         clocks = sampler.stop(t0, time.time())
     if args.markdown:
         print(f"HBM peak {peak:.0f} GB/s ({kind}); clocks {clocks}\n")
@@ -601,6 +630,11 @@ def run_sweep(args):
         print("|---|---|---|---|---|---|")
         for r in att:
             print(f"| {r['prefix']} | {r['tree_nodes']} | {r['us']:.2f} | {r['gbs']:.0f} | {r['frac_hbm']:.3f} | {r['tflops']:.1f} |")
+        print("\nINT4 x INT8 projection (per-channel weights, per-tensor activations, integer tensor cores)\n")
+        print("| K x N | rows | us/launch | GB/s (algorithmic) | of peak | TOP/s |")
+        print("|---|---|---|---|---|---|")
+        for r in wa:
+            print(f"| {r['KxN']} | {r['rows']} | {r['us']:.2f} | {r['gbs']:.0f} | {r['frac_hbm']:.3f} | {r['tops']:.1f} |")
         return
     head = next(r for r in lin if r["KxN"] == "4096x4096" and r["rows"] == 8 and r["adapters"] == 8)
     line = {"metric": "fused INT4 + LoRA projection latency (4096x4096, 8 rows, 8 adapters, rank 16)", "value": head["us"],
@@ -611,7 +645,7 @@ def run_sweep(args):
             "clocks": clocks,
             "roofline": {"bound": "hbm", "achieved": head["gbs"], "peak": peak, "peak_kind": "of " + kind, "unit": "GB/s",
                          "frac": head["frac_hbm"], "traffic": None},
-            "points": lin + att}
+            "points": lin + att + wa}
     print(json.dumps(line), flush=True)
 
 

@@ -5,7 +5,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-SOURCES = ["w4_gemm.cu", "lora_shrink.cu", "step_misc.cu", "attention.cu", "decode_chain.cu", "decode_step.cu", "w4_gemm_tc.cu", "w4a8_gemm.cu", "mlora.cu"]
+SOURCES = ["w4_gemm.cu", "lora_shrink.cu", "step_misc.cu", "attention.cu", "decode_chain.cu", "decode_step.cu", "decode_lean.cu", "w4_gemm_tc.cu", "w4a8_gemm.cu", "mlora.cu"]
 LIB = os.path.join(HERE, "libmlora.so")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]

@@ -421,6 +421,10 @@ __host__ __device__ constexpr size_t dec_smem_bytes(int hd) {
 template <int HD>
 __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const AttnArgs p, const float scale_log2) {
   constexpr int W = dec_warps(HD), STRIDE = HD + 8, KSTEPS = HD / 16, DT = HD / 8, VPR = HD / 8;
+  // (programmatic launches around this kernel: the kernel after it may start its own independent loads now; nothing
+  // here is read before the kernel ahead has finished -- both are no-ops in ordinary launches)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __half* Qs = reinterpret_cast<__half*>(smem_raw);                       // [16][STRIDE]
   __half* tiles = Qs + 16 * STRIDE;                                       // [W][2 buffers][K, V][DEC_KEYS][STRIDE]
@@ -669,7 +673,35 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
         den = f0 * den + f1 * den1;
         M = Mn;
       }
-      p.out[((size_t)m * p.Hq + kh * g_heads + r) * HD + d] = __float2half_rn(den > 0.f ? num / den : 0.f);
+      const __half hv = __float2half_rn(den > 0.f ? num / den : 0.f);
+      p.out[((size_t)m * p.Hq + kh * g_heads + r) * HD + d] = hv;
+      Qs[(size_t)r * STRIDE + d] = hv;                     // (the query tile is long since in registers)
+    }
+    if (p.o_tacc != nullptr) {
+      // partial shrink of the o projection's adapter (Eq. 1-4) over this kv head's output features of row m: rank
+      // index j by warp; integer atomics on fixed-point sums, so the total does not depend on the arrival order
+      const int ad = p.o_adapter_idx[s];
+      const __half* A = (ad >= 0 && ad < p.o_n_slots) ? p.o_tabA[(size_t)ad * p.o_tab_stride + p.o_proj_index] : nullptr;
+      __syncthreads();
+      if (A != nullptr) {
+        const int feats = g_heads * HD, ld = p.Hq * HD;
+        for (int j = warp; j < p.o_rank; j += W) {
+          const __half* arow = A + (size_t)j * ld + (size_t)kh * feats;
+          float sum = 0.f;
+          for (int i = lane * 2; i < feats; i += 64) {
+            const float2 av = __half22float2(__ldg(reinterpret_cast<const __half2*>(arow + i)));
+            const float2 xv = __half22float2(*reinterpret_cast<const __half2*>(Qs + (size_t)(i / HD) * STRIDE + (i % HD)));
+            sum = fmaf(xv.x, av.x, sum);
+            sum = fmaf(xv.y, av.y, sum);
+          }
+#pragma unroll
+          for (int o2 = 16; o2 > 0; o2 >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o2);
+          if (lane == 0) {
+            const unsigned long long q = (unsigned long long)__float2ll_rn(sum * 4294967296.f);
+            asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p.o_tacc + ((size_t)m * 3 + 0) * p.o_rank + j), "l"(q) : "memory");
+          }
+        }
+      }
     }
   }
   // the peer's shared memory must outlive the reads above

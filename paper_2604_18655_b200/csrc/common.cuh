@@ -134,6 +134,12 @@ struct AttnArgs {
   const int32_t* depth;           // dev [rows]
   int stream_mode;                // set by attn_plan: the streaming kernel for one row per stream over a long prefix
   int* status;                    // dev status word for bounded waits that run out (may be null)
+  // single-kernel decode attention only: partial LoRA shrink of the o projection over the (kv head, stream)'s output
+  // features, added to 64-bit fixed-point sums (o_tacc == nullptr: not wanted)
+  unsigned long long* o_tacc;     // [8 rows][3][o_rank] of the o projection's group
+  const __half* const* o_tabA;    // adapter A pointers [slot][o_tab_stride]
+  const int32_t* o_adapter_idx;   // dev [n]
+  int o_proj_index, o_rank, o_tab_stride, o_n_slots;
 };
 
 // ----------------------------------------------------------------------------- persistent projection chain
@@ -306,6 +312,26 @@ cudaError_t launch_compact(__half* own_k, __half* own_v, size_t layer_stride, si
                            size_t head_stride, int L, int n, int Hkv, int hd, const int32_t* suffix_len,
                            const int32_t* acc_len, const int32_t* acc_idx, int T, cudaStream_t st);
 cudaError_t launch_advance(int32_t* suffix_len, const int32_t* acc_len, int n, int fixed, cudaStream_t st);
+// ---- decode step as one small kernel per projection group (decode_lean.cu)
+struct LeanArgs {
+  const StepPhase* ph;            // dev: this kernel's phase
+  int M;
+  float eps;
+  const int32_t* adapter_idx;     // dev [M] or nullptr
+  const __half* const* tabA;
+  const __half* const* tabB;
+  const float* scale;
+  int tab_stride, n_slots, rank;
+  float* X;                       // residual stream fp32 [M][d_model]
+  float* logits;                  // destination of a phase whose out_f32 is null
+  unsigned long long* tacc;       // [n_tacc][8][3][rank]
+  unsigned long long* ssq;        // [n_ssq][8]
+};
+cudaError_t init_lean();
+bool lean_shapes_ok(int d_model, int d_ffn, int Nq, int Nkv, int rank);
+cudaError_t launch_lean_embed(const LeanArgs& a, const int32_t* tokens, const __half* embed, int vocab,
+                              const __half* hidden_in, int d_model, int* status, cudaStream_t st);
+cudaError_t launch_lean_gemm(const LeanArgs& a, const StepPhase& ph, cudaStream_t st);
 cudaError_t launch_quant_act(const __half* x, long long count, float scale, signed char* out, cudaStream_t st);
 bool w4a8_shape_ok(int M, int K, int N);
 cudaError_t launch_w4a8(const unsigned char* w, const __half* ws, const signed char* x, float x_scale, int M, int K, int N,

@@ -1,0 +1,394 @@
+// Decode step (at most 8 rows) as one small kernel per projection group, with nothing between them but the kernel
+// boundary: no normalisation pass, no shrink pass, no exchange of intermediate sums through waits.
+//
+//  * A projection kernel reads its input rows as fp16 (x * gain of the RMSNorm ahead of it, not yet normalised; or
+//    the attention / SwiGLU output), streams its 16 output columns' INT4 weights straight from global memory into
+//    registers (one 16-byte load per lane and k-tile in the fragment-major layout; eight warps split K), dequantises
+//    in registers (exactly fp16(q * scale)) and multiplies on the tensor cores (mma.sync m16n8k16, weights as the
+//    16-wide operand, the rows as the 8-wide one).  The rows' 1/rms factor multiplies the finished sums: RMSNorm
+//    (Sec. 3.1) is linear up to that factor.
+//  * LoRA (Eq. 1-4): the expand y += T B happens in the epilogue; the shrink T = s x A^T of the NEXT projection is
+//    computed by the kernel that PRODUCES x -- every CTA multiplies its 16 fresh columns with the matching columns of
+//    A and adds the partial sums into 64-bit fixed-point accumulators with integer atomics (integer addition is
+//    associative: the total is bit-reproducible), as it does for the rows' sums of squares.  By the time the next
+//    kernel starts, T and the norm factors are complete.
+//  * The accumulators of a whole step are zeroed by one memset at its start.
+#include "../../include/mlora.h"
+#include "common.cuh"
+
+namespace mlora {
+
+constexpr int LN_WARPS = 8;
+constexpr int LN_THREADS = LN_WARPS * 32;
+constexpr float LN_FIX = 4294967296.f, LN_UNFIX = 1.f / 4294967296.f;
+
+__device__ __forceinline__ unsigned long long ln_fix(float v) { return (unsigned long long)__float2ll_rn(v * LN_FIX); }
+__device__ __forceinline__ float ln_unfix(unsigned long long q) { return __ll2float_rn((long long)q) * LN_UNFIX; }
+__device__ __forceinline__ void ln_red_add(unsigned long long* p, unsigned long long v) {
+  asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ uint4 ln_ldg_stream(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ void ln_cp_async16(void* smem, const void* gmem, bool valid) {
+  const uint32_t sa = (uint32_t)__cvta_generic_to_shared(smem);
+  const int sz = valid ? 16 : 0;                          // 0: the 16 bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(sa), "l"(gmem), "r"(sz) : "memory");
+}
+
+// The adapter slices a CTA needs at its end, asked for at its start (cp.async, behind the main loop):
+//   sB [NTILE][M][r][16]: rows of B of this group for the CTA's columns (the expand);
+//   sA [M][next_nseg][r][16]: rows of A of the consuming group for the CTA's output columns (its partial shrink).
+// A missing adapter or matrix gives zeros.
+template <int NTILE>
+__device__ __forceinline__ void lean_prefetch_slices(const LeanArgs& a, const StepPhase& ph, int tile0, int n_out0, bool lora,
+                                                     __half* sB, __half* sA) {
+  const int r = a.rank, M = a.M;
+  if (lora) {
+    for (int it = threadIdx.x; it < NTILE * M * r * 2; it += LN_THREADS) {
+      const int hf = it & 1, j = (it >> 1) % r, m = ((it >> 1) / r) % M, u = (it >> 1) / (r * M);
+      const int ad = a.adapter_idx[m];
+      int seg, col;
+      map_col(ph.mode, (tile0 + u) * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
+      const __half* B = (ad >= 0 && ad < a.n_slots) ? a.tabB[(size_t)ad * a.tab_stride + ph.lora_proj[seg]] : nullptr;
+      ln_cp_async16(sB + (((size_t)u * M + m) * r + j) * 16 + hf * 8, B ? B + (size_t)j * ph.lora_n[seg] + col + hf * 8 : (const __half*)a.X,
+                    B != nullptr);
+    }
+  }
+  if (ph.next_nseg > 0 && a.adapter_idx != nullptr) {
+    for (int it = threadIdx.x; it < M * ph.next_nseg * r * 2; it += LN_THREADS) {
+      const int hf = it & 1, j = (it >> 1) % r, seg = ((it >> 1) / r) % ph.next_nseg, m = (it >> 1) / (r * ph.next_nseg);
+      const int ad = a.adapter_idx[m];
+      const __half* A = (ad >= 0 && ad < a.n_slots) ? a.tabA[(size_t)ad * a.tab_stride + ph.next_proj[seg]] : nullptr;
+      ln_cp_async16(sA + (((size_t)m * ph.next_nseg + seg) * r + j) * 16 + hf * 8,
+                    A ? A + (size_t)j * ph.next_ld + n_out0 + hf * 8 : (const __half*)a.X, A != nullptr);
+    }
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// partial shrink of the consuming group over this CTA's fresh fp16 outputs vals[8][16]: one item per (row, segment,
+// rank index), the A slices in shared memory
+__device__ __forceinline__ void lean_shrink_partial(const LeanArgs& a, const StepPhase& ph, const __half (*vals)[16], const __half* sA) {
+  if (ph.next_nseg == 0 || a.adapter_idx == nullptr) return;
+  const int r = a.rank;
+  for (int it = threadIdx.x; it < a.M * ph.next_nseg * r; it += LN_THREADS) {
+    const int j = it % r, seg = (it / r) % ph.next_nseg, m = it / (r * ph.next_nseg);
+    const __half2* av = reinterpret_cast<const __half2*>(sA + (size_t)it * 16);
+    const __half2* xv = reinterpret_cast<const __half2*>(vals[m]);
+    float s = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const float2 x = __half22float2(xv[q]), w = __half22float2(av[q]);
+      s = fmaf(x.x, w.x, s); s = fmaf(x.y, w.y, s);
+    }
+    ln_red_add(a.tacc + ((size_t)ph.t_out * CHAIN_MAX_ROWS + m) * 3 * r + seg * r + j, ln_fix(s));
+  }
+}
+
+// NTILE = 1: 16 physical columns per CTA; NTILE = 2: a gate tile and its up tile (SwiGLU pair)
+// Launched with programmatic stream serialisation: everything ahead of pdl_wait() -- the first weights, the adapter
+// slices -- depends on no earlier kernel and is in flight while the kernel before this one finishes.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <int NTILE>
+__global__ void __launch_bounds__(LN_THREADS) lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
+  __shared__ float red[LN_WARPS][NTILE][32][4];
+  __shared__ float s_inv[CHAIN_MAX_ROWS];
+  __shared__ float s_T[CHAIN_MAX_ROWS][3 * 64];
+  __shared__ float s_y[NTILE][CHAIN_MAX_ROWS][16];
+  __shared__ __align__(16) __half s_vals[CHAIN_MAX_ROWS][16];
+  __shared__ float s_sq[CHAIN_MAX_ROWS][16];
+  extern __shared__ __align__(16) unsigned char ln_dyn[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  pdl_launch_dependents();
+  const int M = a.M, K = ph.K, r = a.rank;
+  const WLayout L = make_wlayout(K, ph.N, ph.G);
+  const int tile0 = blockIdx.x * NTILE;
+  // ---- ahead of the wait: adapter slices and the first weights (immutable data)
+  const bool lora = ph.lora_nseg > 0 && a.adapter_idx != nullptr;
+  __half* sB = reinterpret_cast<__half*>(ln_dyn);                          // [NTILE][M][r][16]
+  __half* sA = sB + (size_t)NTILE * CHAIN_MAX_ROWS * r * 16;               // [M][next_nseg][r][16]
+  const int n_out0 = ph.epi == EPI_SWIGLU ? (tile0 >> 1) * TILE_N : tile0 * TILE_N;   // first column the CTA produces
+  lean_prefetch_slices<NTILE>(a, ph, tile0, n_out0, lora, sB, sA);
+  const int kt0 = (L.KT * warp) / LN_WARPS, kt1 = (L.KT * (warp + 1)) / LN_WARPS;
+  const unsigned char* unit[NTILE];
+#pragma unroll
+  for (int u = 0; u < NTILE; ++u) unit[u] = ph.w + (size_t)(tile0 + u) * L.unit_bytes;
+  constexpr int PF = 4;
+  uint4 wv[PF][NTILE];
+  uint32_t sv[PF][NTILE];
+  auto load_weights = [&](int kb) {
+#pragma unroll
+    for (int i = 0; i < PF; ++i) {
+      const int kt = kb + i;
+      if (kt < kt1) {
+#pragma unroll
+        for (int u = 0; u < NTILE; ++u) {
+          wv[i][u] = ln_ldg_stream(unit[u] + wl_tile_off(L, kt) + lane * 16);
+          sv[i][u] = __ldg(reinterpret_cast<const uint32_t*>(unit[u] + wl_scale_off(L, kt)) + g);
+        }
+      }
+    }
+  };
+  load_weights(kt0);
+  pdl_wait();
+  // ---- what earlier kernels produced: the old residual, norm factors, T of this group, the input rows
+  float x_old = 0.f, gain_nx = 1.f;
+  if (ph.epi == EPI_RESID && threadIdx.x < 128 && (threadIdx.x >> 4) < M) {
+    x_old = __ldcg(a.X + (size_t)(threadIdx.x >> 4) * ph.N + n_out0 + (threadIdx.x & 15));
+    if (ph.gain_next != nullptr) gain_nx = __half2float(__ldg(ph.gain_next + n_out0 + (threadIdx.x & 15)));
+  }
+  if (threadIdx.x < CHAIN_MAX_ROWS) {
+    float inv = 1.f;
+    if (ph.norm_in >= 0 && threadIdx.x < M)
+      inv = rsqrtf(ln_unfix(__ldcg(a.ssq + (size_t)ph.norm_in * CHAIN_MAX_ROWS + threadIdx.x)) / (float)K + a.eps);
+    s_inv[threadIdx.x] = inv;
+  }
+  if (lora) {
+    for (int i = threadIdx.x; i < M * ph.lora_nseg * r; i += LN_THREADS) {
+      const int m = i / (ph.lora_nseg * r), rest = i % (ph.lora_nseg * r);
+      const int ad = a.adapter_idx[m];
+      float v = 0.f;
+      if (ad >= 0 && ad < a.n_slots)
+        v = ln_unfix(__ldcg(a.tacc + ((size_t)ph.t_in * CHAIN_MAX_ROWS + m) * 3 * r + rest)) * a.scale[ad];
+      s_T[m][rest] = v;
+    }
+  }
+  // ---- main loop: warp w takes the k-tiles [kt0, kt1)
+  float acc[NTILE][4];
+#pragma unroll
+  for (int u = 0; u < NTILE; ++u) acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0.f;
+  const __half* xrow = ph.in16 + (size_t)g * K + 16 * t;
+  const bool row_live = g < M;
+#pragma unroll 1
+  for (int kb = kt0; kb < kt1; kb += PF) {
+    uint4 x0[PF], x1[PF];
+#pragma unroll
+    for (int i = 0; i < PF; ++i) {
+      const int kt = kb + i;
+      if (kt < kt1 && row_live) {
+        x0[i] = __ldcg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * TILE_K));
+        x1[i] = __ldcg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * TILE_K) + 1);
+      } else {
+        x0[i] = make_uint4(0, 0, 0, 0);
+        x1[i] = make_uint4(0, 0, 0, 0);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < PF; ++i) {
+      if (kb + i < kt1) {
+#pragma unroll
+        for (int u = 0; u < NTILE; ++u) {
+          __half2 s_lo, s_hi;
+          split_scales(sv[i][u], s_lo, s_hi);
+          uint32_t af[4][4];
+          dequant8(wv[i][u].x, s_lo, s_hi, af[0]);
+          dequant8(wv[i][u].y, s_lo, s_hi, af[1]);
+          dequant8(wv[i][u].z, s_lo, s_hi, af[2]);
+          dequant8(wv[i][u].w, s_lo, s_hi, af[3]);
+          mma_16816(acc[u], af[0], x0[i].x, x0[i].y);
+          mma_16816(acc[u], af[1], x0[i].z, x0[i].w);
+          mma_16816(acc[u], af[2], x1[i].x, x1[i].y);
+          mma_16816(acc[u], af[3], x1[i].z, x1[i].w);
+        }
+      }
+    }
+    if (kb + PF < kt1) load_weights(kb + PF);
+  }
+#pragma unroll
+  for (int u = 0; u < NTILE; ++u)
+    *reinterpret_cast<float4*>(red[warp][u][lane]) = make_float4(acc[u][0], acc[u][1], acc[u][2], acc[u][3]);
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+
+  // ---- one thread per (tile, row, column): sum of the warps' parts in warp order, LoRA expand, norm factor
+  for (int o = threadIdx.x; o < NTILE * 128; o += LN_THREADS) {
+    const int u = o >> 7, m = (o >> 4) & 7, c = o & 15;
+    // accumulator layout of m16n8k16: lane (g,t) holds (out g, row 2t), (g, 2t+1), (g+8, 2t), (g+8, 2t+1)
+    const int src_lane = (c & 7) * 4 + (m >> 1), e = (c >> 3) * 2 + (m & 1);
+    float y = 0.f;
+    if (m < M) {
+#pragma unroll
+      for (int w = 0; w < LN_WARPS; ++w) y += red[w][u][src_lane][e];
+      if (lora) {
+        int seg, col;
+        map_col(ph.mode, (tile0 + u) * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
+        const float* T = s_T[m] + seg * r;
+        const __half* Bs = sB + ((size_t)u * M + m) * r * 16 + c;           // (zeros where the row has no adapter)
+        float ex = 0.f;
+        for (int j = 0; j < r; ++j) ex = fmaf(T[j], __half2float(Bs[(size_t)j * 16]), ex);
+        y += ex;
+      }
+      y *= s_inv[m];
+    }
+    s_y[u][m][c] = y;
+  }
+  __syncthreads();
+
+  const int n0 = tile0 * TILE_N;                                            // first physical column (NTILE = 1)
+  if (ph.epi == EPI_F32) {
+    float* out = ph.out_f32 != nullptr ? ph.out_f32 : a.logits;
+    for (int o = threadIdx.x; o < NTILE * 128; o += LN_THREADS) {
+      const int u = o >> 7, m = (o >> 4) & 7, c = o & 15;
+      if (m < M) out[(size_t)m * ph.ldo + (tile0 + u) * TILE_N + c] = s_y[u][m][c];
+    }
+    return;
+  }
+  if (ph.epi == EPI_RESID) {
+    // new residual; x * gain for the norm that follows; the rows' sums of squares; the next group's partial shrink
+    if (threadIdx.x < 128) {
+      const int m = threadIdx.x >> 4, c = threadIdx.x & 15;
+      float xn = 0.f;
+      __half hv = __float2half_rn(0.f);
+      if (m < M) {
+        xn = x_old + s_y[0][m][c];
+        a.X[(size_t)m * ph.N + n0 + c] = xn;
+        if (ph.gain_next != nullptr) {
+          hv = __float2half_rn(xn * gain_nx);
+          ph.out16[(size_t)m * ph.N + n0 + c] = hv;
+        }
+      }
+      s_vals[m][c] = hv;
+      s_sq[m][c] = xn * xn;
+    }
+    __syncthreads();
+    if (ph.ssq_out >= 0 && threadIdx.x < M) {
+      float sq = 0.f;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) sq += s_sq[threadIdx.x][c];
+      ln_red_add(a.ssq + (size_t)ph.ssq_out * CHAIN_MAX_ROWS + threadIdx.x, ln_fix(sq));
+    }
+    lean_shrink_partial(a, ph, s_vals, sA);
+    return;
+  }
+  // EPI_SWIGLU: tile0 is the gate tile, tile0 + 1 the up tile of 16 features
+  if (NTILE == 2) {
+    const int f0 = (tile0 >> 1) * TILE_N, F = ph.N / 2;
+    if (threadIdx.x < 128) {
+      const int m = threadIdx.x >> 4, c = threadIdx.x & 15;
+      __half hv = __float2half_rn(0.f);
+      if (m < M) {
+        const float gt = s_y[0][m][c], up = s_y[NTILE - 1][m][c];
+        hv = __float2half_rn(gt / (1.f + __expf(-gt)) * up);
+        ph.out16[(size_t)m * F + f0 + c] = hv;
+      }
+      s_vals[m][c] = hv;
+    }
+    __syncthreads();
+    lean_shrink_partial(a, ph, s_vals, sA);
+  }
+}
+
+// Embedding (or hidden-state input) of the step's rows: residual fp32, x * gain of the first norm as fp16, the rows'
+// sums of squares, and the shrink sums of the first q,k,v group.  CTA (m, part): row m; part 0 also writes the row.
+__global__ void __launch_bounds__(LN_THREADS) lean_embed_kernel(const LeanArgs a, const int32_t* __restrict__ tokens,
+                                                               const __half* __restrict__ embed, int vocab,
+                                                               const __half* __restrict__ hidden_in, int* __restrict__ status) {
+  extern __shared__ __align__(16) unsigned char ln_smem[];
+  __half* xg = reinterpret_cast<__half*>(ln_smem);                         // [d]
+  __shared__ float s_part[LN_WARPS];
+  pdl_launch_dependents();
+  const StepPhase& ph = *a.ph;
+  const int m = blockIdx.x, part = blockIdx.y, d = ph.N;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const __half* src;
+  if (hidden_in != nullptr) src = hidden_in + (size_t)m * d;
+  else {
+    int tok = tokens[m];
+    if (tok < 0 || tok >= vocab) {
+      if (threadIdx.x == 0 && part == 0) atomicCAS(status, 0, -1);
+      tok = 0;
+    }
+    src = embed + (size_t)tok * d;
+  }
+  float sq = 0.f;
+  for (int k = threadIdx.x * 2; k < d; k += LN_THREADS * 2) {
+    const float2 v = __half22float2(*reinterpret_cast<const __half2*>(src + k));
+    const float2 gn = ph.gain_next ? __half22float2(*reinterpret_cast<const __half2*>(ph.gain_next + k)) : make_float2(1.f, 1.f);
+    const __half2 hv = __floats2half2_rn(v.x * gn.x, v.y * gn.y);
+    *reinterpret_cast<__half2*>(xg + k) = hv;
+    sq += v.x * v.x + v.y * v.y;
+    if (part == 0) {
+      *reinterpret_cast<float2*>(a.X + (size_t)m * d + k) = v;
+      if (ph.out16) *reinterpret_cast<__half2*>(ph.out16 + (size_t)m * d + k) = hv;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+  if (lane == 0) s_part[warp] = sq;
+  __syncthreads();
+  if (part == 0 && threadIdx.x == 0 && ph.ssq_out >= 0) {
+    float tot = 0.f;
+    for (int w = 0; w < LN_WARPS; ++w) tot += s_part[w];
+    ln_red_add(a.ssq + (size_t)ph.ssq_out * CHAIN_MAX_ROWS + m, ln_fix(tot));
+  }
+  if (ph.next_nseg == 0 || a.adapter_idx == nullptr) return;
+  const int ad = a.adapter_idx[m];
+  if (ad < 0 || ad >= a.n_slots) return;
+  const int r = a.rank, items = ph.next_nseg * r;
+  // the CTA's share of the (segment, rank index) dot products, a warp each
+  for (int it = part * LN_WARPS + warp; it < items; it += gridDim.y * LN_WARPS) {
+    const int seg = it / r, j = it % r;
+    const __half* A = a.tabA[(size_t)ad * a.tab_stride + ph.next_proj[seg]];
+    if (A == nullptr) continue;
+    const __half* arow = A + (size_t)j * ph.next_ld;
+    float s = 0.f;
+    for (int k = lane * 8; k < d; k += 32 * 8) {
+      const uint4 av = __ldg(reinterpret_cast<const uint4*>(arow + k));
+      const uint4 xv = *reinterpret_cast<const uint4*>(xg + k);
+      const __half2* ap = reinterpret_cast<const __half2*>(&av);
+      const __half2* xp = reinterpret_cast<const __half2*>(&xv);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float2 x = __half22float2(xp[q]), w = __half22float2(ap[q]);
+        s = fmaf(x.x, w.x, s); s = fmaf(x.y, w.y, s);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) ln_red_add(a.tacc + ((size_t)ph.t_out * CHAIN_MAX_ROWS + m) * 3 * r + seg * r + j, ln_fix(s));
+  }
+}
+
+bool lean_shapes_ok(int d_model, int d_ffn, int Nq, int Nkv, int rank) {
+  // whole 16-column tiles, rows cut into 8-element pieces, T of a row within the kernels' shared arrays
+  return d_model % 64 == 0 && d_ffn % 64 == 0 && Nq % 64 == 0 && Nkv % 16 == 0 && rank <= 64 && d_model <= 16384;
+}
+
+cudaError_t launch_lean_embed(const LeanArgs& a, const int32_t* tokens, const __half* embed, int vocab,
+                              const __half* hidden_in, int d_model, int* status, cudaStream_t st) {
+  lean_embed_kernel<<<dim3((unsigned)a.M, 6), LN_THREADS, (size_t)d_model * sizeof(__half), st>>>(a, tokens, embed, vocab, hidden_in, status);
+  return cudaGetLastError();
+}
+
+cudaError_t init_lean() {
+  // room for the adapter slices at rank 64: 5 x 16 KB
+  cudaError_t e = cudaFuncSetAttribute(lean_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(lean_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
+}
+
+cudaError_t launch_lean_gemm(const LeanArgs& a, const StepPhase& ph, cudaStream_t st) {
+  const int tiles = ph.N / TILE_N, mode = ph.mode;
+  // B slices of up to two tiles and A slices of up to three consuming segments, 8 rows x rank x 16 columns each
+  const size_t slice = (size_t)CHAIN_MAX_ROWS * (a.rank > 0 ? a.rank : 1) * 16 * sizeof(__half);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)(mode == MODE_GATEUP ? tiles / 2 : tiles));
+  cfg.blockDim = dim3(LN_THREADS);
+  cfg.dynamicSmemBytes = (mode == MODE_GATEUP ? 5 : 4) * slice;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start while the kernel before it drains
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (mode == MODE_GATEUP) return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<2>, a, ph);
+  return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<1>, a, ph);
+}
+
+}  // namespace mlora

@@ -112,6 +112,9 @@ struct mlora_ctx {
   unsigned long long* chain_sync = nullptr;   // dev [4]
   int chain_stages = 0, chain_kmax = 0;
   // whole decode step in one kernel (one row per stream, rows <= 8)
+  std::vector<StepPhase> step_phases_host;
+  size_t step_acc_bytes = 0;         // step_tacc and step_ssq, contiguous
+  bool lean_ok = false;              // the per-projection decode kernels take this model's shapes
   StepPhase* step_phases = nullptr;  // dev [5*L + 3]: embed; qkv, attention, o, gate/up, down per layer; lm_head; end
   int n_step_phases = 0, step_stages = 0, step_own_tiles = 0;
   unsigned char *tmapA = nullptr, *tmapB = nullptr;           // dev [max_adapters][L*7] tensor maps over the adapters' matrices
@@ -352,7 +355,58 @@ cudaError_t launch_projection(mlora_ctx* c, const GemmArgs& g, cudaStream_t st) 
 }
 
 // the launch sequence of one pass over M = n*T rows (Sec. 3.1 decoder, Eq. 1-4 projections)
+// decode-sized pass as one small kernel per projection group (decode_lean.cu), attention between them
+bool lean_eligible(const mlora_ctx* c, const PassIO& io) {
+  return c->step_mode == 3 && c->lean_ok && c->step_phases != nullptr && !io.prefill && io.T == 1 &&
+         io.n <= CHAIN_MAX_ROWS && io.parent == c->root_parent && attn_single_pass(io.plan);
+}
+
+int forward_lean(mlora_ctx* c, const PassIO& io) {
+  const mlora_model_desc& d = c->d;
+  cudaStream_t st = c->stream;
+  CK(cudaMemsetAsync(c->step_tacc, 0, c->step_acc_bytes, st));   // the step's accumulators (a memset node, not a kernel)
+  LeanArgs a{};
+  a.M = io.n; a.eps = d.rms_eps;
+  const bool lora = io.adapter_idx != nullptr && d.lora_rank > 0 && d.max_adapters > 0 && d.lora_targets != 0;
+  if (lora) {
+    a.adapter_idx = io.adapter_idx; a.tabA = c->tabA; a.tabB = c->tabB; a.scale = c->ad_scale;
+    a.tab_stride = c->L * 7; a.n_slots = d.max_adapters;
+  }
+  a.rank = (d.max_adapters > 0 && d.lora_targets != 0) ? d.lora_rank : 0;
+  a.X = c->X; a.logits = io.logits; a.tacc = c->step_tacc; a.ssq = c->step_ssq;
+  for (size_t p = 0; p < c->step_phases_host.size(); ++p) {
+    const StepPhase& ph = c->step_phases_host[p];
+    a.ph = c->step_phases + p;
+    if (ph.kind == SK_EMBED) {
+      CK(run(c, MLORA_PROF_MISC, [&] {
+        return launch_lean_embed(a, io.tokens, (const __half*)d.embed, d.vocab, io.hidden_in, d.d_model, c->status, st);
+      }));
+    } else if (ph.kind == SK_GEMM) {
+      if (ph.epi == EPI_F32 && ph.out_f32 == nullptr && io.logits == nullptr) continue;   // lm_head not wanted
+      CK(run(c, MLORA_PROF_GEMM, [&] { return launch_lean_gemm(a, ph, st); }));
+    } else if (ph.kind == SK_ATTN) {
+      const int l = ph.layer;
+      AttnArgs at = io.plan;
+      at.qkv_f32 = c->qkv; at.cs_table = c->cs_table; at.pos_base = io.pos_base; at.depth = c->zero_len;   // one row per stream: depth 0
+      at.prefix_k = c->prefix_k + (size_t)l * c->prefix_layer_stride;
+      at.prefix_v = c->prefix_v + (size_t)l * c->prefix_layer_stride;
+      at.prefix_head_stride = c->prefix_head_stride;
+      at.own_k = c->own_k + (size_t)l * c->own_layer_stride; at.own_v = c->own_v + (size_t)l * c->own_layer_stride;
+      at.own_stream_stride = c->own_stream_stride; at.own_head_stride = c->own_head_stride;
+      at.suffix_len = io.suffix_len; at.anc = c->anc; at.causal = 0; at.out = c->attn16; at.status = c->status;
+      if (lora && ph.next_nseg > 0) {
+        at.o_tacc = c->step_tacc + (size_t)ph.t_out * CHAIN_MAX_ROWS * 3 * a.rank;
+        at.o_tabA = c->tabA; at.o_adapter_idx = io.adapter_idx; at.o_proj_index = ph.next_proj[0]; at.o_rank = a.rank;
+        at.o_tab_stride = c->L * 7; at.o_n_slots = d.max_adapters;
+      }
+      CK(run(c, MLORA_PROF_ATTN, [&] { return launch_attention(at, st); }));
+    }
+  }
+  return MLORA_OK;
+}
+
 int forward(mlora_ctx* c, const PassIO& io) {
+  if (lean_eligible(c, io)) return forward_lean(c, io);
   if (chain_eligible(c, io)) return forward_chain(c, io);
   const mlora_model_desc& d = c->d;
   cudaStream_t st = c->stream;
@@ -512,6 +566,7 @@ int init_kernels() {
   CK(init_gemm());
   CK(init_shrink());
   CK(init_attention());
+  CK(init_lean());
   CK(init_chain());
   CK(init_step());
   CK(init_gemm_tc());
@@ -788,16 +843,19 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
   {
     const int tg = d.lora_rank > 0 && d.max_adapters > 0 ? d.lora_targets : 0;
     c->step_stages = step_plan(dm, F, Nq, Nkv, hd, d.lora_rank, tg, c->sm_count, &c->step_own_tiles);
-    if (d.max_streams > 0 && c->step_stages > 0) {
+    c->lean_ok = lean_shapes_ok(dm, F, Nq, Nkv, tg ? d.lora_rank : 0);
+    if (d.max_streams > 0 && (c->step_stages > 0 || c->lean_ok)) {
       const int rr = tg ? d.lora_rank : 0;
       c->n_tacc = 4 * L; c->n_ssq = 2 * L + 1;
       CKC(cudaMalloc(&c->xg_attn, (size_t)CHAIN_MAX_ROWS * dm * sizeof(__half)));
       CKC(cudaMalloc(&c->xg_ffn, (size_t)CHAIN_MAX_ROWS * dm * sizeof(__half)));
       const size_t tacc_bytes = (size_t)c->n_tacc * CHAIN_MAX_ROWS * 3 * (rr > 0 ? rr : 1) * sizeof(unsigned long long);
-      CKC(cudaMalloc(&c->step_tacc, tacc_bytes));
-      CKC(cudaMemsetAsync(c->step_tacc, 0, tacc_bytes, st));
-      CKC(cudaMalloc(&c->step_ssq, (size_t)c->n_ssq * CHAIN_MAX_ROWS * sizeof(unsigned long long)));
-      CKC(cudaMemsetAsync(c->step_ssq, 0, (size_t)c->n_ssq * CHAIN_MAX_ROWS * sizeof(unsigned long long), st));
+      // (one allocation for both kinds of accumulators: one memset clears a step's worth)
+      const size_t ssq_bytes = (size_t)c->n_ssq * CHAIN_MAX_ROWS * sizeof(unsigned long long);
+      CKC(cudaMalloc(&c->step_tacc, tacc_bytes + ssq_bytes));
+      CKC(cudaMemsetAsync(c->step_tacc, 0, tacc_bytes + ssq_bytes, st));
+      c->step_ssq = c->step_tacc + tacc_bytes / sizeof(unsigned long long);
+      c->step_acc_bytes = tacc_bytes + ssq_bytes;
       CKC(cudaMalloc(&c->step_amax, (size_t)c->sm_count * CHAIN_MAX_ROWS * sizeof(unsigned long long)));
       CKC(cudaMemsetAsync(c->step_amax, 0, (size_t)c->sm_count * CHAIN_MAX_ROWS * sizeof(unsigned long long), st));
       std::vector<StepPhase> sp;
@@ -871,6 +929,7 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
       CKC(cudaMemsetAsync(c->step_trace, 0, sp.size() * 2 * 12 * sizeof(long long), st));
       CKC(cudaMalloc(&c->step_phases, sp.size() * sizeof(StepPhase)));
       CKC(cudaMemcpy(c->step_phases, sp.data(), sp.size() * sizeof(StepPhase), cudaMemcpyHostToDevice));
+      c->step_phases_host = sp;
     }
   }
   CKC(cudaMallocHost(&c->snap, d.max_streams * sizeof(int32_t)));
@@ -894,7 +953,7 @@ int mlora_destroy(mlora_ctx* c) {
                       c->h, c->attn16, c->act16, c->counters, c->anc, c->depth, c->argmax, c->suffix_len,
                       c->zero_len, c->chain_parent, c->root_parent, c->status, c->cs_table, (void*)c->tabA,
                       (void*)c->tabB, c->ad_scale, c->phases, c->chain_sync, c->host_io, c->step_phases, c->xg_attn, c->xg_ffn,
-                      c->step_tacc, c->step_ssq, c->step_amax, c->step_trace, c->tmapA, c->tmapB, c->gen_tokens, c->draft_cand};
+                      c->step_tacc, c->step_amax, c->step_trace, c->tmapA, c->tmapB, c->gen_tokens, c->draft_cand};
   for (void* p : dev_ptrs) if (p) cudaFree(p);
   if (c->stageA) cudaFreeHost((void*)c->stageA);
   if (c->stageB) cudaFreeHost((void*)c->stageB);
@@ -992,7 +1051,7 @@ static int decode_impl(mlora_ctx* c, int n, const int32_t* adapter_idx, const in
   key.kind = hidden ? 2 : 1; key.n = n; key.T = 1;
   key.prefix_chunk = io.plan.prefix_chunk; key.n_prefix_chunks = io.plan.n_prefix_chunks;
   key.own_chunk = io.plan.own_chunk; key.n_own_chunks = io.plan.n_own_chunks;
-  key.flags = c->P * 4 + c->dbg_inject_stall * 2 + c->dbg_no_chain;
+  key.flags = (c->P * 4 + c->dbg_inject_stall * 2 + c->dbg_no_chain) * 4 + c->step_mode;
   key.suffix_bound = io.plan.suffix_bound;     // (rounded up by plan_pass: the kernels' launch shape and prefetch extents)
   key.p[0] = adapter_idx; key.p[1] = tokens; key.p[2] = hidden; key.p[3] = out_next; key.p[4] = out_logits; key.p[5] = hidden_out;
   rc = replay_or_run(c, key, [&]() -> int {
@@ -1350,7 +1409,7 @@ int mlora_debug_set(mlora_ctx* c, int32_t key, int32_t value) {
   else if (key == 3) c->dbg_no_chain = value ? 1 : 0;
   else if (key == 4) c->dbg_no_tc = value ? 1 : 0;
   else if (key == 5) c->dbg_inject_stall = value ? 1 : 0;
-  else if (key == 6) c->step_mode = (value >= 0 && value <= 2) ? value : 0;
+  else if (key == 6) c->step_mode = (value >= 0 && value <= 3) ? value : 0;
   else if (key == 7) c->dbg_trace = value ? 1 : 0;
   else return fail(MLORA_ERR_ARG, "unknown debug key");
   return MLORA_OK;

@@ -22,7 +22,8 @@ def GpuModel():
 
 
 # decode-step paths of the library (debug switch 6): per-layer kernels, or one kernel for the whole step
-STEP_PATHS = [pytest.param(1, id="per_layer_kernels"), pytest.param(2, id="single_kernel_step")]
+STEP_PATHS = [pytest.param(1, id="per_layer_kernels"), pytest.param(2, id="single_kernel_step"),
+              pytest.param(3, id="kernel_per_projection")]
 
 
 def make_pair(GpuModel, cfg, seed=0, step_path=0, **kw):
@@ -642,7 +643,7 @@ def test_host_buffer_step_matches_device_step(GpuModel):
     assert np.array_equal(outs[0], outs[1])
 
 
-@pytest.mark.parametrize("step_path", STEP_PATHS)
+@pytest.mark.parametrize("step_path", STEP_PATHS[:2])       # (the kernel-per-projection path has no device-side wait)
 def test_bounded_wait_runs_out_and_context_recovers(GpuModel, step_path):
     """Failure detection without a fault: a grid barrier of the persistent kernel is made to wait (limit ~0.1 s) for an
     arrival nobody makes.  The kernel must return, the device status must say TIMEOUT and name the wait, and after

@@ -83,7 +83,7 @@ def test_llama1b_full_depth_single_kernel_step():
     run_decode_and_verify(gen.CFG1, n_decode=3, branch=(4, 2, 2), T=16, step_path=2)
 
 
-@pytest.mark.parametrize("step_path", [1, 2])
+@pytest.mark.parametrize("step_path", [1, 2, 3])
 def test_llama1b_full_prompt_sixteen_steps(step_path):
     """The benchmark workload itself: the full 512-token shared prompt, 8 streams, 16 greedy decode steps in follow
     mode (the oracle walks on the GPU's tokens), logits of every step against the oracle, own-segment KV at the end."""
