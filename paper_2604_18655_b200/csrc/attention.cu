@@ -424,7 +424,6 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   // (programmatic launches around this kernel: the kernel after it may start its own independent loads now; nothing
   // here is read before the kernel ahead has finished -- both are no-ops in ordinary launches)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __half* Qs = reinterpret_cast<__half*>(smem_raw);                       // [16][STRIDE]
   __half* tiles = Qs + 16 * STRIDE;                                       // [W][2 buffers][K, V][DEC_KEYS][STRIDE]
@@ -494,6 +493,7 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   };
   // a warp whose first tile lies in the shared prefix starts it before anything that depends on the stream
   if (tile_of(warp) < n_ptiles) load_tile(tile_of(warp), 0);
+  asm volatile("griddepcontrol.wait;" ::: "memory");                       // (the shared prefix does not change in decode)
   S = p.suffix_len[s];
   own_keys = S + 1;                                                       // cached rows + this pass's row
   n_tiles = n_ptiles + (own_keys + DEC_KEYS - 1) / DEC_KEYS;
@@ -1198,11 +1198,13 @@ cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st) {
     cfg.blockDim = dim3((unsigned)dec_warps(a.hd) * 32);
     cfg.dynamicSmemBytes = dec_smem_bytes(a.hd);
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;      // the DEC_SPLIT CTAs of a (kv head, stream) form a cluster
     attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = DEC_SPLIT;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // its first prefix tiles may be in flight while
+    attr[1].val.programmaticStreamSerializationAllowed = 1;            // the kernel ahead of it drains
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = a.pdl ? 2 : 1;
     if (a.hd == 64) return cudaLaunchKernelEx(&cfg, attn_decode_kernel<64>, a, scale_log2);
     return cudaLaunchKernelEx(&cfg, attn_decode_kernel<128>, a, scale_log2);
   }

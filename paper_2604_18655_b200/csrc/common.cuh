@@ -140,6 +140,7 @@ struct AttnArgs {
   const __half* const* o_tabA;    // adapter A pointers [slot][o_tab_stride]
   const int32_t* o_adapter_idx;   // dev [n]
   int o_proj_index, o_rank, o_tab_stride, o_n_slots;
+  int pdl;                        // launch the single-kernel decode attention with programmatic stream serialisation
 };
 
 // ----------------------------------------------------------------------------- persistent projection chain

@@ -48,7 +48,7 @@ __device__ __forceinline__ void lean_prefetch_slices(const LeanArgs& a, const St
                                                      __half* sB, __half* sA) {
   const int r = a.rank, M = a.M;
   if (lora) {
-    for (int it = threadIdx.x; it < NTILE * M * r * 2; it += LN_THREADS) {
+    for (int it = threadIdx.x; it < NTILE * M * r * 2; it += blockDim.x) {
       const int hf = it & 1, j = (it >> 1) % r, m = ((it >> 1) / r) % M, u = (it >> 1) / (r * M);
       const int ad = a.adapter_idx[m];
       int seg, col;
@@ -59,7 +59,7 @@ __device__ __forceinline__ void lean_prefetch_slices(const LeanArgs& a, const St
     }
   }
   if (ph.next_nseg > 0 && a.adapter_idx != nullptr) {
-    for (int it = threadIdx.x; it < M * ph.next_nseg * r * 2; it += LN_THREADS) {
+    for (int it = threadIdx.x; it < M * ph.next_nseg * r * 2; it += blockDim.x) {
       const int hf = it & 1, j = (it >> 1) % r, seg = ((it >> 1) / r) % ph.next_nseg, m = (it >> 1) / (r * ph.next_nseg);
       const int ad = a.adapter_idx[m];
       const __half* A = (ad >= 0 && ad < a.n_slots) ? a.tabA[(size_t)ad * a.tab_stride + ph.next_proj[seg]] : nullptr;
@@ -75,7 +75,7 @@ __device__ __forceinline__ void lean_prefetch_slices(const LeanArgs& a, const St
 __device__ __forceinline__ void lean_shrink_partial(const LeanArgs& a, const StepPhase& ph, const __half (*vals)[16], const __half* sA) {
   if (ph.next_nseg == 0 || a.adapter_idx == nullptr) return;
   const int r = a.rank;
-  for (int it = threadIdx.x; it < a.M * ph.next_nseg * r; it += LN_THREADS) {
+  for (int it = threadIdx.x; it < a.M * ph.next_nseg * r; it += blockDim.x) {
     const int j = it % r, seg = (it / r) % ph.next_nseg, m = it / (r * ph.next_nseg);
     const __half2* av = reinterpret_cast<const __half2*>(sA + (size_t)it * 16);
     const __half2* xv = reinterpret_cast<const __half2*>(vals[m]);
@@ -95,9 +95,11 @@ __device__ __forceinline__ void lean_shrink_partial(const LeanArgs& a, const Ste
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-template <int NTILE>
-__global__ void __launch_bounds__(LN_THREADS) lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
-  __shared__ float red[LN_WARPS][NTILE][32][4];
+template <int NTILE, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, NTILE == 2 ? 3 : (WARPS == 8 ? 2 : 1))
+lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
+  constexpr int THREADS = WARPS * 32;
+  __shared__ float red[WARPS][NTILE][32][4];
   __shared__ float s_inv[CHAIN_MAX_ROWS];
   __shared__ float s_T[CHAIN_MAX_ROWS][3 * 64];
   __shared__ float s_y[NTILE][CHAIN_MAX_ROWS][16];
@@ -114,12 +116,11 @@ __global__ void __launch_bounds__(LN_THREADS) lean_gemm_kernel(const LeanArgs a,
   __half* sB = reinterpret_cast<__half*>(ln_dyn);                          // [NTILE][M][r][16]
   __half* sA = sB + (size_t)NTILE * CHAIN_MAX_ROWS * r * 16;               // [M][next_nseg][r][16]
   const int n_out0 = ph.epi == EPI_SWIGLU ? (tile0 >> 1) * TILE_N : tile0 * TILE_N;   // first column the CTA produces
-  lean_prefetch_slices<NTILE>(a, ph, tile0, n_out0, lora, sB, sA);
-  const int kt0 = (L.KT * warp) / LN_WARPS, kt1 = (L.KT * (warp + 1)) / LN_WARPS;
+  const int kt0 = (L.KT * warp) / WARPS, kt1 = (L.KT * (warp + 1)) / WARPS;
   const unsigned char* unit[NTILE];
 #pragma unroll
   for (int u = 0; u < NTILE; ++u) unit[u] = ph.w + (size_t)(tile0 + u) * L.unit_bytes;
-  constexpr int PF = 4;
+  constexpr int PF = 4;                                                    // k-tiles in flight per warp
   uint4 wv[PF][NTILE];
   uint32_t sv[PF][NTILE];
   auto load_weights = [&](int kb) {
@@ -135,7 +136,8 @@ __global__ void __launch_bounds__(LN_THREADS) lean_gemm_kernel(const LeanArgs a,
       }
     }
   };
-  load_weights(kt0);
+  load_weights(kt0);                                                       // (first: the longest latency)
+  lean_prefetch_slices<NTILE>(a, ph, tile0, n_out0, lora, sB, sA);
   pdl_wait();
   // ---- what earlier kernels produced: the old residual, norm factors, T of this group, the input rows
   float x_old = 0.f, gain_nx = 1.f;
@@ -150,7 +152,7 @@ __global__ void __launch_bounds__(LN_THREADS) lean_gemm_kernel(const LeanArgs a,
     s_inv[threadIdx.x] = inv;
   }
   if (lora) {
-    for (int i = threadIdx.x; i < M * ph.lora_nseg * r; i += LN_THREADS) {
+    for (int i = threadIdx.x; i < M * ph.lora_nseg * r; i += THREADS) {
       const int m = i / (ph.lora_nseg * r), rest = i % (ph.lora_nseg * r);
       const int ad = a.adapter_idx[m];
       float v = 0.f;
@@ -207,14 +209,14 @@ __global__ void __launch_bounds__(LN_THREADS) lean_gemm_kernel(const LeanArgs a,
   __syncthreads();
 
   // ---- one thread per (tile, row, column): sum of the warps' parts in warp order, LoRA expand, norm factor
-  for (int o = threadIdx.x; o < NTILE * 128; o += LN_THREADS) {
+  for (int o = threadIdx.x; o < NTILE * 128; o += THREADS) {
     const int u = o >> 7, m = (o >> 4) & 7, c = o & 15;
     // accumulator layout of m16n8k16: lane (g,t) holds (out g, row 2t), (g, 2t+1), (g+8, 2t), (g+8, 2t+1)
     const int src_lane = (c & 7) * 4 + (m >> 1), e = (c >> 3) * 2 + (m & 1);
     float y = 0.f;
     if (m < M) {
 #pragma unroll
-      for (int w = 0; w < LN_WARPS; ++w) y += red[w][u][src_lane][e];
+      for (int w = 0; w < WARPS; ++w) y += red[w][u][src_lane][e];
       if (lora) {
         int seg, col;
         map_col(ph.mode, (tile0 + u) * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
@@ -233,7 +235,7 @@ __global__ void __launch_bounds__(LN_THREADS) lean_gemm_kernel(const LeanArgs a,
   const int n0 = tile0 * TILE_N;                                            // first physical column (NTILE = 1)
   if (ph.epi == EPI_F32) {
     float* out = ph.out_f32 != nullptr ? ph.out_f32 : a.logits;
-    for (int o = threadIdx.x; o < NTILE * 128; o += LN_THREADS) {
+    for (int o = threadIdx.x; o < NTILE * 128; o += THREADS) {
       const int u = o >> 7, m = (o >> 4) & 7, c = o & 15;
       if (m < M) out[(size_t)m * ph.ldo + (tile0 + u) * TILE_N + c] = s_y[u][m][c];
     }
@@ -368,9 +370,11 @@ cudaError_t launch_lean_embed(const LeanArgs& a, const int32_t* tokens, const __
 
 cudaError_t init_lean() {
   // room for the adapter slices at rank 64: 5 x 16 KB
-  cudaError_t e = cudaFuncSetAttribute(lean_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(lean_gemm_kernel<1, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(lean_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
+  e = cudaFuncSetAttribute(lean_gemm_kernel<1, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(lean_gemm_kernel<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
 }
 
 cudaError_t launch_lean_gemm(const LeanArgs& a, const StepPhase& ph, cudaStream_t st) {
@@ -379,7 +383,8 @@ cudaError_t launch_lean_gemm(const LeanArgs& a, const StepPhase& ph, cudaStream_
   const size_t slice = (size_t)CHAIN_MAX_ROWS * (a.rank > 0 ? a.rank : 1) * 16 * sizeof(__half);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(mode == MODE_GATEUP ? tiles / 2 : tiles));
-  cfg.blockDim = dim3(LN_THREADS);
+  const bool wide = mode != MODE_GATEUP && ph.K >= 4096;    // a long K on few tiles: sixteen warps split it
+  cfg.blockDim = dim3(wide ? 512 : LN_THREADS);
   cfg.dynamicSmemBytes = (mode == MODE_GATEUP ? 5 : 4) * slice;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -387,8 +392,9 @@ cudaError_t launch_lean_gemm(const LeanArgs& a, const StepPhase& ph, cudaStream_
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (mode == MODE_GATEUP) return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<2>, a, ph);
-  return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<1>, a, ph);
+  if (mode == MODE_GATEUP) return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<2, 8>, a, ph);
+  if (wide) return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<1, 16>, a, ph);
+  return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<1, 8>, a, ph);
 }
 
 }  // namespace mlora

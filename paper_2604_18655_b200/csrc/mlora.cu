@@ -394,6 +394,7 @@ int forward_lean(mlora_ctx* c, const PassIO& io) {
       at.own_k = c->own_k + (size_t)l * c->own_layer_stride; at.own_v = c->own_v + (size_t)l * c->own_layer_stride;
       at.own_stream_stride = c->own_stream_stride; at.own_head_stride = c->own_head_stride;
       at.suffix_len = io.suffix_len; at.anc = c->anc; at.causal = 0; at.out = c->attn16; at.status = c->status;
+      at.pdl = 1;
       if (lora && ph.next_nseg > 0) {
         at.o_tacc = c->step_tacc + (size_t)ph.t_out * CHAIN_MAX_ROWS * 3 * a.rank;
         at.o_tabA = c->tabA; at.o_adapter_idx = io.adapter_idx; at.o_proj_index = ph.next_proj[0]; at.o_rank = a.rank;
