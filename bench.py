@@ -31,11 +31,10 @@ GEN_STEPS = 128          # decode steps per generation (per stream) before the s
 ORACLE_PREFIX = 64       # prompt length used for the CPU-baseline sample (the 512-token prefill is not timed work)
 L2_BYTES = 126e6
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture) per launch of the dominant kernel, by
-# workload; None where no capture of the kernel as it stands exists.  cfg1: decode_chain_kernel captured on a 4-layer
-# cut of the model (the launches of a layer are the same at any depth): 7.86 MB for the first launch of a step
-# (q,k,v only), 34.87 MB for each per-layer launch, the last launch (with the lm_head) taken at its algorithmic
-# 60 MB, averaged over the 17 launches of a full-model step
-NCU_DRAM_BYTES_PER_LAUNCH = {"cfg1": 34.8e6}
+# workload; None where no capture of the kernel as it stands exists.  cfg1: the 17 lean_gemm_kernel launches of a step
+# of a 4-layer cut of the model (the launches of a layer are the same at any depth): 4.10 MB q,k,v + 3.88 MB o +
+# 16.31 MB gate/up + 8.25 MB down = 32.54 MB per layer, 33.86 MB for the lm_head; (16 x 32.54 + 33.86) / 65 launches
+NCU_DRAM_BYTES_PER_LAUNCH = {"cfg1": 8.53e6}
 
 
 def parse_args():
@@ -953,7 +952,9 @@ def main():
                 "single_step_call_ms_per_step": ms_e2e_step},
         "per_step_graph_replay_ms_per_step": ms_per_step_call,
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "decode_chain_kernel (persistent INT4 GEMM + LoRA shrink/expand + norm), all launches of a step",
+        "roofline": {"bound": "hbm", "kernel": "lean_gemm_kernel (INT4 projection group + LoRA expand + epilogue + next group's partial shrink), all "
+                     "launches of a step; durations from direct launches with an event pair around each, which serialises "
+                     "the programmatic launches the timed graph overlaps: an upper bound on the time",
                      "achieved": achieved, "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(args.config) if args.layers is None else None,
                      "bytes_per_launch": gemm_bytes_step / gemm_per_step, "launches_per_step": gemm_per_step,
@@ -965,7 +966,7 @@ def main():
                                "launches_per_step": (prof["attn"][1] + prof["attn_merge"][1]) / prof_steps},
         "single_kernel_step": None if step_kernel_ms is None else
             {"ms_per_step": step_kernel_ms, "tokens_per_s": world * n / (step_kernel_ms / 1e3),
-             "note": "the whole step as one cooperative launch (selectable; the per-layer kernels are the default)"},
+             "note": "the whole step as one cooperative launch (selectable; one kernel per projection group is the default)"},
         "step_roofline": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_bytes / (ms_step / 1e3) / 1e9,
                           "frac": step_bytes / (ms_step / 1e3) / 1e9 / peak},
         "family_us_per_step": {k: 1e3 * v[0] / prof_steps for k, v in prof.items()},

@@ -192,11 +192,14 @@ int mlora_debug_dequant(mlora_ctx* ctx, int32_t layer, int32_t proj, void* out_f
 /* Debug switches: key 1 = skip KV compaction and suffix growth in mlora_verify_tree (tree rows stay where
  * the pass wrote them: rows suffix_len .. suffix_len + n_nodes - 1 of the own segment).
  * key 2 = 1 disables CUDA-graph replay of steps (every kernel launched directly).
- * key 3 = 1 runs decode-sized passes through the one-kernel-per-projection path instead of the persistent kernels.
+ * key 3 = 1 runs decode-sized passes through the general split-K kernels (one per operation: norm + shrink, projection,
+ *         attention, ...) instead of any of the decode paths of key 6.
  * key 6 picks the path of decode steps (one row per stream, at most 8 streams): 1 = the per-layer persistent projection
- *         kernel plus attention kernels, replayed from a CUDA graph; 2 = ONE kernel that does the whole step (embedding to
- *         greedy token; where the model's shapes allow it, else the per-layer path); 0 = the library's choice
- *         (currently the per-layer path, the faster of the two at the 1B / 8-stream shapes).
+ *         kernel plus attention kernels; 2 = ONE kernel that does the whole step (embedding to greedy token; where the
+ *         model's shapes allow it, else the per-layer path); 3 = one small kernel per projection group, launched
+ *         programmatically so that each one's weights are in flight while the one before it drains (contexts up to
+ *         2047 keys; longer ones take the per-layer path); 0 = the library's choice (3 where it applies: the fastest of
+ *         the three at the 1B / 8-stream shapes).  All are replayed from CUDA graphs.
  * key 7 = 1 makes the single-kernel decode step record a timeline (see mlora_step_timeline). */
 int mlora_debug_set(mlora_ctx* ctx, int32_t key, int32_t value);
 /* Timeline of the LAST decode step that ran with debug key 7 set (Sec. 3.1 decoder: the step's phases are the

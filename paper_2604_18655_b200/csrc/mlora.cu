@@ -357,7 +357,8 @@ cudaError_t launch_projection(mlora_ctx* c, const GemmArgs& g, cudaStream_t st) 
 // the launch sequence of one pass over M = n*T rows (Sec. 3.1 decoder, Eq. 1-4 projections)
 // decode-sized pass as one small kernel per projection group (decode_lean.cu), attention between them
 bool lean_eligible(const mlora_ctx* c, const PassIO& io) {
-  return c->step_mode == 3 && c->lean_ok && c->step_phases != nullptr && !io.prefill && io.T == 1 &&
+  // (the library's own choice where it applies: the fastest of the three decode paths at the measured shapes)
+  return (c->step_mode == 3 || c->step_mode == 0) && !c->dbg_no_chain && c->lean_ok && c->step_phases != nullptr && !io.prefill && io.T == 1 &&
          io.n <= CHAIN_MAX_ROWS && io.parent == c->root_parent && attn_single_pass(io.plan);
 }
 
