@@ -493,8 +493,10 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   };
   // a warp whose first tile lies in the shared prefix starts it before anything that depends on the stream
   if (tile_of(warp) < n_ptiles) load_tile(tile_of(warp), 0);
-  asm volatile("griddepcontrol.wait;" ::: "memory");                       // (the shared prefix does not change in decode)
+  // (programmatic launch: the shared prefix does not change in decode, and the suffix lengths were last written by the
+  // step before this one, which an ordinary launch at the start of this step has waited for)
   S = p.suffix_len[s];
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   own_keys = S + 1;                                                       // cached rows + this pass's row
   n_tiles = n_ptiles + (own_keys + DEC_KEYS - 1) / DEC_KEYS;
   if (fused) cs = p.cs_table + (size_t)(p.pos_base + S + p.depth[m]) * (HD / 2);

@@ -96,7 +96,7 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 template <int NTILE, int WARPS>
-__global__ void __launch_bounds__(WARPS * 32, NTILE == 2 ? 3 : (WARPS == 8 ? 2 : 1))
+__global__ void __launch_bounds__(WARPS * 32, WARPS == 8 ? 3 : 1)
 lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
   constexpr int THREADS = WARPS * 32;
   __shared__ float red[WARPS][NTILE][32][4];
