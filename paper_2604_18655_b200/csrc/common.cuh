@@ -315,7 +315,6 @@ cudaError_t launch_compact(__half* own_k, __half* own_v, size_t layer_stride, si
 cudaError_t launch_advance(int32_t* suffix_len, const int32_t* acc_len, int n, int fixed, cudaStream_t st);
 // ---- decode step as one small kernel per projection group (decode_lean.cu)
 struct LeanArgs {
-  const StepPhase* ph;            // dev: this kernel's phase
   int M;
   float eps;
   const int32_t* adapter_idx;     // dev [M] or nullptr
@@ -327,11 +326,12 @@ struct LeanArgs {
   float* logits;                  // destination of a phase whose out_f32 is null
   unsigned long long* tacc;       // [n_tacc][8][3][rank]
   unsigned long long* ssq;        // [n_ssq][8]
+  int late_wait;                  // the kernel ahead produces only T: wait for it after the main loop, not before
 };
 cudaError_t init_lean();
 bool lean_shapes_ok(int d_model, int d_ffn, int Nq, int Nkv, int rank);
-cudaError_t launch_lean_embed(const LeanArgs& a, const int32_t* tokens, const __half* embed, int vocab,
-                              const __half* hidden_in, int d_model, int* status, cudaStream_t st);
+cudaError_t launch_lean_embed(const LeanArgs& a, const StepPhase& ph, const int32_t* tokens, const __half* embed, int vocab,
+                              const __half* hidden_in, int* status, cudaStream_t st);
 cudaError_t launch_lean_gemm(const LeanArgs& a, const StepPhase& ph, cudaStream_t st);
 cudaError_t launch_quant_act(const __half* x, long long count, float scale, signed char* out, cudaStream_t st);
 bool w4a8_shape_ok(int M, int K, int N);

@@ -54,7 +54,7 @@ __device__ __forceinline__ void lean_prefetch_slices(const LeanArgs& a, const St
       int seg, col;
       map_col(ph.mode, (tile0 + u) * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
       const __half* B = (ad >= 0 && ad < a.n_slots) ? a.tabB[(size_t)ad * a.tab_stride + ph.lora_proj[seg]] : nullptr;
-      ln_cp_async16(sB + (((size_t)u * M + m) * r + j) * 16 + hf * 8, B ? B + (size_t)j * ph.lora_n[seg] + col + hf * 8 : (const __half*)a.X,
+      ln_cp_async16(sB + (((size_t)u * M + m) * r + j) * 16 + hf * 8, B ? B + (size_t)j * ph.lora_n[seg] + col + hf * 8 : (const __half*)ph.w,
                     B != nullptr);
     }
   }
@@ -64,7 +64,7 @@ __device__ __forceinline__ void lean_prefetch_slices(const LeanArgs& a, const St
       const int ad = a.adapter_idx[m];
       const __half* A = (ad >= 0 && ad < a.n_slots) ? a.tabA[(size_t)ad * a.tab_stride + ph.next_proj[seg]] : nullptr;
       ln_cp_async16(sA + (((size_t)m * ph.next_nseg + seg) * r + j) * 16 + hf * 8,
-                    A ? A + (size_t)j * ph.next_ld + n_out0 + hf * 8 : (const __half*)a.X, A != nullptr);
+                    A ? A + (size_t)j * ph.next_ld + n_out0 + hf * 8 : (const __half*)ph.w, A != nullptr);
     }
   }
   asm volatile("cp.async.commit_group;" ::: "memory");
@@ -151,7 +151,7 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
       inv = rsqrtf(ln_unfix(__ldcg(a.ssq + (size_t)ph.norm_in * CHAIN_MAX_ROWS + threadIdx.x)) / (float)K + a.eps);
     s_inv[threadIdx.x] = inv;
   }
-  if (lora) {
+  auto load_T = [&]() {
     for (int i = threadIdx.x; i < M * ph.lora_nseg * r; i += THREADS) {
       const int m = i / (ph.lora_nseg * r), rest = i % (ph.lora_nseg * r);
       const int ad = a.adapter_idx[m];
@@ -160,7 +160,8 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
         v = ln_unfix(__ldcg(a.tacc + ((size_t)ph.t_in * CHAIN_MAX_ROWS + m) * 3 * r + rest)) * a.scale[ad];
       s_T[m][rest] = v;
     }
-  }
+  };
+  if (lora && !a.late_wait) load_T();
   // ---- main loop: warp w takes the k-tiles [kt0, kt1)
   float acc[NTILE][4];
 #pragma unroll
@@ -201,6 +202,10 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
       }
     }
     if (kb + PF < kt1) load_weights(kb + PF);
+  }
+  if (a.late_wait) {
+    pdl_wait();
+    if (lora) load_T();
   }
 #pragma unroll
   for (int u = 0; u < NTILE; ++u)
@@ -288,14 +293,14 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
 
 // Embedding (or hidden-state input) of the step's rows: residual fp32, x * gain of the first norm as fp16, the rows'
 // sums of squares, and the shrink sums of the first q,k,v group.  CTA (m, part): row m; part 0 also writes the row.
-__global__ void __launch_bounds__(LN_THREADS) lean_embed_kernel(const LeanArgs a, const int32_t* __restrict__ tokens,
+__global__ void __launch_bounds__(LN_THREADS) lean_embed_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph,
+                                                               const int32_t* __restrict__ tokens,
                                                                const __half* __restrict__ embed, int vocab,
                                                                const __half* __restrict__ hidden_in, int* __restrict__ status) {
   extern __shared__ __align__(16) unsigned char ln_smem[];
   __half* xg = reinterpret_cast<__half*>(ln_smem);                         // [d]
   __shared__ float s_part[LN_WARPS];
   pdl_launch_dependents();
-  const StepPhase& ph = *a.ph;
   const int m = blockIdx.x, part = blockIdx.y, d = ph.N;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const __half* src;
@@ -316,7 +321,7 @@ __global__ void __launch_bounds__(LN_THREADS) lean_embed_kernel(const LeanArgs a
     *reinterpret_cast<__half2*>(xg + k) = hv;
     sq += v.x * v.x + v.y * v.y;
     if (part == 0) {
-      *reinterpret_cast<float2*>(a.X + (size_t)m * d + k) = v;
+      if (a.X) *reinterpret_cast<float2*>(a.X + (size_t)m * d + k) = v;
       if (ph.out16) *reinterpret_cast<__half2*>(ph.out16 + (size_t)m * d + k) = hv;
     }
   }
@@ -332,15 +337,21 @@ __global__ void __launch_bounds__(LN_THREADS) lean_embed_kernel(const LeanArgs a
   if (ph.next_nseg == 0 || a.adapter_idx == nullptr) return;
   const int ad = a.adapter_idx[m];
   if (ad < 0 || ad >= a.n_slots) return;
-  const int r = a.rank, items = ph.next_nseg * r;
-  // the CTA's share of the (segment, rank index) dot products, a warp each
+  const int r = a.rank;
+  // the CTA's share of the (segment, rank index, 1024-element piece of the row) partial dot products, a warp each
+  // (ph.pad_ = 1: whole dot products, stored: the sums need no zeroing then -- the single-projection call)
+  const int KC = ph.pad_ ? 1 : (d + 1023) / 1024, items = ph.next_nseg * r * KC;
   for (int it = part * LN_WARPS + warp; it < items; it += gridDim.y * LN_WARPS) {
-    const int seg = it / r, j = it % r;
+    const int kc = it % KC, j = (it / KC) % r, seg = it / (KC * r);
     const __half* A = a.tabA[(size_t)ad * a.tab_stride + ph.next_proj[seg]];
-    if (A == nullptr) continue;
+    if (A == nullptr) {
+      if (ph.pad_ && lane == 0) a.tacc[((size_t)ph.t_out * CHAIN_MAX_ROWS + m) * 3 * r + seg * r + j] = 0ull;
+      continue;
+    }
     const __half* arow = A + (size_t)j * ph.next_ld;
+    const int k1 = ph.pad_ ? d : min(d, (kc + 1) * 1024);
     float s = 0.f;
-    for (int k = lane * 8; k < d; k += 32 * 8) {
+    for (int k = kc * 1024 + lane * 8; k < k1; k += 32 * 8) {
       const uint4 av = __ldg(reinterpret_cast<const uint4*>(arow + k));
       const uint4 xv = *reinterpret_cast<const uint4*>(xg + k);
       const __half2* ap = reinterpret_cast<const __half2*>(&av);
@@ -353,7 +364,11 @@ __global__ void __launch_bounds__(LN_THREADS) lean_embed_kernel(const LeanArgs a
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    if (lane == 0) ln_red_add(a.tacc + ((size_t)ph.t_out * CHAIN_MAX_ROWS + m) * 3 * r + seg * r + j, ln_fix(s));
+    if (lane == 0) {
+      unsigned long long* dst = a.tacc + ((size_t)ph.t_out * CHAIN_MAX_ROWS + m) * 3 * r + seg * r + j;
+      if (ph.pad_) *dst = ln_fix(s);
+      else ln_red_add(dst, ln_fix(s));
+    }
   }
 }
 
@@ -362,9 +377,12 @@ bool lean_shapes_ok(int d_model, int d_ffn, int Nq, int Nkv, int rank) {
   return d_model % 64 == 0 && d_ffn % 64 == 0 && Nq % 64 == 0 && Nkv % 16 == 0 && rank <= 64 && d_model <= 16384;
 }
 
-cudaError_t launch_lean_embed(const LeanArgs& a, const int32_t* tokens, const __half* embed, int vocab,
-                              const __half* hidden_in, int d_model, int* status, cudaStream_t st) {
-  lean_embed_kernel<<<dim3((unsigned)a.M, 6), LN_THREADS, (size_t)d_model * sizeof(__half), st>>>(a, tokens, embed, vocab, hidden_in, status);
+cudaError_t launch_lean_embed(const LeanArgs& a, const StepPhase& ph, const int32_t* tokens, const __half* embed, int vocab,
+                              const __half* hidden_in, int* status, cudaStream_t st) {
+  // a warp per (segment, rank index, 1024-element piece): enough CTAs per row to give every item its own warp
+  const int items = (a.adapter_idx != nullptr ? ph.next_nseg * a.rank : 0) * (ph.pad_ ? 1 : (ph.N + 1023) / 1024);
+  const int gy = items <= LN_WARPS ? 1 : (items + LN_WARPS - 1) / LN_WARPS > 32 ? 32 : (items + LN_WARPS - 1) / LN_WARPS;
+  lean_embed_kernel<<<dim3((unsigned)a.M, (unsigned)gy), LN_THREADS, (size_t)ph.N * sizeof(__half), st>>>(a, ph, tokens, embed, vocab, hidden_in, status);
   return cudaGetLastError();
 }
 
@@ -383,7 +401,7 @@ cudaError_t launch_lean_gemm(const LeanArgs& a, const StepPhase& ph, cudaStream_
   const size_t slice = (size_t)CHAIN_MAX_ROWS * (a.rank > 0 ? a.rank : 1) * 16 * sizeof(__half);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(mode == MODE_GATEUP ? tiles / 2 : tiles));
-  const bool wide = mode != MODE_GATEUP && ph.K >= 4096;    // a long K on few tiles: sixteen warps split it
+  const bool wide = mode != MODE_GATEUP && ph.K >= 4096 && tiles <= 148;   // a long K on few tiles: sixteen warps split it
   cfg.blockDim = dim3(wide ? 512 : LN_THREADS);
   cfg.dynamicSmemBytes = (mode == MODE_GATEUP ? 5 : 4) * slice;
   cfg.stream = st;
