@@ -953,8 +953,9 @@ def main():
         "per_step_graph_replay_ms_per_step": ms_per_step_call,
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "lean_gemm_kernel (INT4 projection group + LoRA expand + epilogue + next group's partial shrink), all "
-                     "launches of a step; durations from direct launches with an event pair around each, which serialises "
-                     "the programmatic launches the timed graph overlaps: an upper bound on the time",
+                     "launches of a step; durations from direct launches with an event pair around every run of consecutive "
+                     "projection kernels (o, gate/up, down, next q,k,v): the run's first kernel loses the overlap with the "
+                     "attention kernel ahead of it that the timed graph has, so an upper bound on the time",
                      "achieved": achieved, "peak": peak, "peak_kind": "of " + peak_kind, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(args.config) if args.layers is None else None,
                      "bytes_per_launch": gemm_bytes_step / gemm_per_step, "launches_per_step": gemm_per_step,

@@ -214,7 +214,8 @@ int mlora_debug_set(mlora_ctx* ctx, int32_t key, int32_t value);
  * Synchronises.  Errors: ARG, STATE, CAPACITY, CUDA. */
 int mlora_step_timeline(mlora_ctx* ctx, int64_t* host_out, int32_t capacity, int32_t* n_phases);
 /* Per-kernel-family device time of the NEXT steps, measured with CUDA events on the context's stream.
- * mlora_profile_begin switches to direct launches with an event pair around every kernel; mlora_profile_end
+ * mlora_profile_begin switches to direct launches with an event pair around every run of consecutive launches of one
+ * family (kernels of a run keep whatever overlap they have among themselves); mlora_profile_end
  * synchronises, switches back, and fills ms[family] / launches[family] (host arrays of MLORA_PROF_FAMILIES). */
 enum { MLORA_PROF_GEMM = 0, MLORA_PROF_SHRINK = 1, MLORA_PROF_ATTN = 2, MLORA_PROF_ATTN_MERGE = 3,
        MLORA_PROF_ROPE_KV = 4 /* unused: RoPE and the KV append run inside the attention kernel */, MLORA_PROF_MISC = 5,

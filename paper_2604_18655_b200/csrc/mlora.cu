@@ -129,7 +129,7 @@ struct mlora_ctx {
   bool capturing = false;
   // profiling
   bool profiling = false;
-  struct Ev { cudaEvent_t a, b; int fam; };
+  struct Ev { cudaEvent_t a, b; int fam, count; bool open; };   // one interval per run of consecutive launches of a family
   std::vector<Ev> evs;
   std::vector<cudaEvent_t> ev_pool;
   int64_t launches = 0;
@@ -149,23 +149,34 @@ int fail(int code, const std::string& msg) {
       return fail(MLORA_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e__));            \
   } while (0)
 
-// wraps one kernel launch: counts it and, when profiling, brackets it with an event pair
+// ends the open profiling interval, if any
+void prof_close(mlora_ctx* c) {
+  if (!c->evs.empty() && c->evs.back().open) {
+    cudaEventRecord(c->evs.back().b, c->stream);
+    c->evs.back().open = false;
+  }
+}
+
+// wraps one kernel launch: counts it and, when profiling, keeps it inside an event pair.  Consecutive launches of one
+// family share a pair, so that what they overlap among themselves (programmatic launches) stays overlapped.
 template <class F>
 cudaError_t run(mlora_ctx* c, int fam, F&& f) {
   if (c->capturing) c->captured_nodes++;
   else c->launches++;
   if (!c->profiling) return f();
-  mlora_ctx::Ev ev;
-  for (cudaEvent_t* e : {&ev.a, &ev.b}) {
-    if (!c->ev_pool.empty()) { *e = c->ev_pool.back(); c->ev_pool.pop_back(); }
-    else { cudaError_t r = cudaEventCreate(e); if (r != cudaSuccess) return r; }
+  if (c->evs.empty() || !c->evs.back().open || c->evs.back().fam != fam) {
+    prof_close(c);
+    mlora_ctx::Ev ev;
+    for (cudaEvent_t* e : {&ev.a, &ev.b}) {
+      if (!c->ev_pool.empty()) { *e = c->ev_pool.back(); c->ev_pool.pop_back(); }
+      else { cudaError_t r = cudaEventCreate(e); if (r != cudaSuccess) return r; }
+    }
+    ev.fam = fam; ev.count = 0; ev.open = true;
+    cudaEventRecord(ev.a, c->stream);
+    c->evs.push_back(ev);
   }
-  ev.fam = fam;
-  cudaEventRecord(ev.a, c->stream);
-  cudaError_t r = f();
-  cudaEventRecord(ev.b, c->stream);
-  c->evs.push_back(ev);
-  return r;
+  c->evs.back().count++;
+  return f();
 }
 
 struct PassIO {
@@ -1425,6 +1436,7 @@ int mlora_profile_begin(mlora_ctx* c) {
 
 int mlora_profile_end(mlora_ctx* c, float* ms, int32_t* launches) {
   if (check_ctx(c)) return MLORA_ERR_ARG;
+  prof_close(c);
   CK(cudaStreamSynchronize(c->stream));
   c->profiling = false;
   for (int i = 0; i < MLORA_PROF_FAMILIES; ++i) { if (ms) ms[i] = 0.f; if (launches) launches[i] = 0; }
@@ -1432,7 +1444,7 @@ int mlora_profile_end(mlora_ctx* c, float* ms, int32_t* launches) {
     float t = 0.f;
     cudaEventElapsedTime(&t, e.a, e.b);
     if (ms) ms[e.fam] += t;
-    if (launches) launches[e.fam] += 1;
+    if (launches) launches[e.fam] += e.count;
     c->ev_pool.push_back(e.a);
     c->ev_pool.push_back(e.b);
   }
