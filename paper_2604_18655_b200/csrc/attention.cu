@@ -430,6 +430,7 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   float* part_o = reinterpret_cast<float*>(tiles + (size_t)W * 4 * DEC_KEYS * STRIDE);   // [W][16][HD]
   float* part_ml = part_o + (size_t)W * 16 * HD;                          // [W][16][2]
   float* xch = part_ml + (size_t)W * 16 * 2;                              // [16][HD + 2]: this CTA's result for its peer
+  __half* a_sl = reinterpret_cast<__half*>(xch + 16 * (HD + 2));          // [o_rank][g_heads * HD]: the o adapter's A rows
   const int rank = blockIdx.z;                                            // position in the cluster (1, 1, DEC_SPLIT)
   auto tile_of = [&](int li) { return li * DEC_SPLIT + rank; };          // the CTA's li-th tile
 
@@ -491,6 +492,21 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
     }
     cp_async_commit();
   };
+  // the o projection's adapter rows over this kv head's features (first CTA of the cluster; immutable: asked for
+  // ahead of everything; its cp.async group is the oldest, so every later wait covers it)
+  const __half* oA = nullptr;
+  if (p.o_tacc != nullptr && rank == 0) {
+    const int ad = p.o_adapter_idx[s];
+    oA = (ad >= 0 && ad < p.o_n_slots) ? p.o_tabA[(size_t)ad * p.o_tab_stride + p.o_proj_index] : nullptr;
+    if (oA != nullptr) {
+      const int feats = g_heads * HD, ld = p.Hq * HD, pieces = feats / 8;
+      for (int i = threadIdx.x; i < p.o_rank * pieces; i += W * 32) {
+        const int j = i / pieces, c = (i % pieces) * 8;
+        cp_async16(a_sl + (size_t)j * feats + c, oA + (size_t)j * ld + (size_t)kh * feats + c);
+      }
+    }
+    cp_async_commit();
+  }
   // a warp whose first tile lies in the shared prefix starts it before anything that depends on the stream
   if (tile_of(warp) < n_ptiles) load_tile(tile_of(warp), 0);
   // (programmatic launch: the shared prefix does not change in decode, and the suffix lengths were last written by the
@@ -682,16 +698,15 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
     if (p.o_tacc != nullptr) {
       // partial shrink of the o projection's adapter (Eq. 1-4) over this kv head's output features of row m: rank
       // index j by warp; integer atomics on fixed-point sums, so the total does not depend on the arrival order
-      const int ad = p.o_adapter_idx[s];
-      const __half* A = (ad >= 0 && ad < p.o_n_slots) ? p.o_tabA[(size_t)ad * p.o_tab_stride + p.o_proj_index] : nullptr;
+      cp_async_wait<0>();
       __syncthreads();
-      if (A != nullptr) {
-        const int feats = g_heads * HD, ld = p.Hq * HD;
+      if (oA != nullptr) {
+        const int feats = g_heads * HD;
         for (int j = warp; j < p.o_rank; j += W) {
-          const __half* arow = A + (size_t)j * ld + (size_t)kh * feats;
+          const __half* arow = a_sl + (size_t)j * feats;
           float sum = 0.f;
           for (int i = lane * 2; i < feats; i += 64) {
-            const float2 av = __half22float2(__ldg(reinterpret_cast<const __half2*>(arow + i)));
+            const float2 av = __half22float2(*reinterpret_cast<const __half2*>(arow + i));
             const float2 xv = __half22float2(*reinterpret_cast<const __half2*>(Qs + (size_t)(i / HD) * STRIDE + (i % HD)));
             sum = fmaf(xv.x, av.x, sum);
             sum = fmaf(xv.y, av.y, sum);
@@ -1054,6 +1069,11 @@ attn_stream_kernel(const AttnArgs p, const __grid_constant__ CUtensorMap map_k, 
   if (!s_abort) str_combine_write<HD>(p, comb, warp, o, mrow, lrow, kh, 0, R_all, chunk, ctid);
 }
 
+// the o adapter's A rows over a kv head's features sit in shared memory beside the decode kernel's tiles
+bool attn_decode_o_slice_fits(int hd, int g_heads, int rank) {
+  return dec_smem_bytes(hd) + (size_t)rank * g_heads * hd * sizeof(__half) <= (size_t)227 * 1024;
+}
+
 // one decode row per stream, a context short enough for one CTA per (kv head, stream), at most 16 query heads per
 // kv head
 bool attn_single_pass(const AttnArgs& a) {
@@ -1134,9 +1154,10 @@ cudaError_t init_attention() {
   cudaError_t e = cudaFuncSetAttribute(attn_partial_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)((ATT_ROWS + 4 * ATT_KEYS) * (64 + 8) * sizeof(__half)));
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(attn_decode_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem_bytes(64));
+  // (+ room for the o adapter's rows over a kv head's features, up to the limit of a CTA)
+  e = cudaFuncSetAttribute(attn_decode_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(attn_decode_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem_bytes(128));
+  e = cudaFuncSetAttribute(attn_decode_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(attn_stream_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)str_smem_bytes(64));
   if (e != cudaSuccess) return e;
@@ -1198,7 +1219,7 @@ cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)a.Hkv, (unsigned)a.n, DEC_SPLIT);
     cfg.blockDim = dim3((unsigned)dec_warps(a.hd) * 32);
-    cfg.dynamicSmemBytes = dec_smem_bytes(a.hd);
+    cfg.dynamicSmemBytes = dec_smem_bytes(a.hd) + (a.o_tacc ? (size_t)a.o_rank * (a.Hq / a.Hkv) * a.hd * sizeof(__half) : 0);
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;      // the DEC_SPLIT CTAs of a (kv head, stream) form a cluster

@@ -302,6 +302,7 @@ cudaError_t launch_tree_prep(const int32_t* parent, int n, int T, unsigned long 
                              int* status, cudaStream_t st);
 void attn_plan(AttnArgs& a, int sm_count);
 size_t attn_workspace_floats(const AttnArgs& a);
+bool attn_decode_o_slice_fits(int hd, int g_heads, int rank);
 bool attn_single_pass(const AttnArgs& a);          // one kernel does the whole softmax: no merge launch follows
 cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st);
 cudaError_t launch_attention_merge(const AttnArgs& a, cudaStream_t st);

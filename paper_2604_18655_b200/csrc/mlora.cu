@@ -855,7 +855,8 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
   {
     const int tg = d.lora_rank > 0 && d.max_adapters > 0 ? d.lora_targets : 0;
     c->step_stages = step_plan(dm, F, Nq, Nkv, hd, d.lora_rank, tg, c->sm_count, &c->step_own_tiles);
-    c->lean_ok = lean_shapes_ok(dm, F, Nq, Nkv, tg ? d.lora_rank : 0);
+    c->lean_ok = lean_shapes_ok(dm, F, Nq, Nkv, tg ? d.lora_rank : 0) &&
+                 attn_decode_o_slice_fits(hd, d.n_q_heads / d.n_kv_heads, (tg & MLORA_O) ? d.lora_rank : 0);
     if (d.max_streams > 0 && (c->step_stages > 0 || c->lean_ok)) {
       const int rr = tg ? d.lora_rank : 0;
       c->n_tacc = 4 * L; c->n_ssq = 2 * L + 1;
