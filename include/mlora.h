@@ -100,7 +100,8 @@ int mlora_prefill_shared_h(mlora_ctx* ctx, const void* hidden, int32_t n, float*
 /* One decode step for n_streams streams (Sec. 3.4): stream s feeds tokens[s] with adapter
  * adapter_idx[s] (-1 = base weights), attends to the shared segment and its own segment, appends its
  * K/V to its own segment and returns the greedy next token.
- * adapter_idx, tokens, out_next: dev int32 [n_streams]; out_logits: dev fp32 [n_streams][vocab] or NULL.
+ * adapter_idx, tokens, out_next: dev int32 [n_streams]; out_logits: dev fp32 [n_streams][vocab] or NULL (then no
+ * logits are formed anywhere: the lm_head keeps only each row's running maximum, lowest id on ties).
  * Errors: ARG, STATE (no prefill yet), CAPACITY (own segment full). */
 int mlora_decode_step(mlora_ctx* ctx, int32_t n_streams, const int32_t* adapter_idx, const int32_t* tokens,
                       int32_t* out_next, float* out_logits);

@@ -328,7 +328,10 @@ struct LeanArgs {
   unsigned long long* tacc;       // [n_tacc][8][3][rank]
   unsigned long long* ssq;        // [n_ssq][8]
   int late_wait;                  // the kernel ahead produces only T: wait for it after the main loop, not before
+  unsigned long long* amax;       // [8]: row maxima of the lm_head as (ordered value, complemented column) keys, zero at
+                                  // the start of a step; non-null = no logits are written, the greedy tokens come from here
 };
+cudaError_t launch_lean_finish(const unsigned long long* amax, int32_t* out_next, int32_t* suffix_len, int n, cudaStream_t st);
 cudaError_t init_lean();
 bool lean_shapes_ok(int d_model, int d_ffn, int Nq, int Nkv, int rank);
 cudaError_t launch_lean_embed(const LeanArgs& a, const StepPhase& ph, const int32_t* tokens, const __half* embed, int vocab,

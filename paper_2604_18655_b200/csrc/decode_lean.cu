@@ -238,6 +238,27 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
   __syncthreads();
 
   const int n0 = tile0 * TILE_N;                                            // first physical column (NTILE = 1)
+  if (ph.epi == EPI_F32 && ph.out_f32 == nullptr && a.amax != nullptr) {
+    // lm_head without a logits destination: the row argmax (Sec. 3.5: greedy tokens; lowest column on ties) is all that
+    // is wanted.  Key = order-preserving image of the value (NaN lowest) over the complemented column: the CTA's best
+    // per row goes to a global maximum -- tried only when it beats what is there already.
+    if (threadIdx.x < M) {
+      const int m = threadIdx.x;
+      unsigned long long best = 0ull;
+#pragma unroll
+      for (int u = 0; u < NTILE; ++u)
+        for (int c = 0; c < 16; ++c) {
+          float v = s_y[u][m][c];
+          if (v == 0.f) v = 0.f;
+          const unsigned b = __float_as_uint(v);
+          const unsigned ord = (v != v) ? 0u : ((b & 0x80000000u) ? ~b : (b | 0x80000000u));
+          const unsigned long long k = ((unsigned long long)ord << 32) | (unsigned)(0xffffffffu - (unsigned)((tile0 + u) * TILE_N + c));
+          best = k > best ? k : best;
+        }
+      if (best > __ldcg(a.amax + m)) atomicMax(a.amax + m, best);
+    }
+    return;
+  }
   if (ph.epi == EPI_F32) {
     float* out = ph.out_f32 != nullptr ? ph.out_f32 : a.logits;
     for (int o = threadIdx.x; o < NTILE * 128; o += THREADS) {
@@ -370,6 +391,21 @@ __global__ void __launch_bounds__(LN_THREADS) lean_embed_kernel(const LeanArgs a
       else ln_red_add(dst, ln_fix(s));
     }
   }
+}
+
+// the greedy tokens from the lm_head's row maxima, and the suffix lengths one further
+__global__ void lean_finish_kernel(const unsigned long long* __restrict__ amax, int32_t* __restrict__ out_next,
+                                   int32_t* __restrict__ suffix_len, int n) {
+  const int m = threadIdx.x;
+  if (m >= n) return;
+  const unsigned long long k = amax[m];
+  out_next[m] = k == 0ull ? 0 : (int32_t)(0xffffffffu - (unsigned)(k & 0xffffffffull));
+  suffix_len[m] += 1;
+}
+
+cudaError_t launch_lean_finish(const unsigned long long* amax, int32_t* out_next, int32_t* suffix_len, int n, cudaStream_t st) {
+  lean_finish_kernel<<<1, 32, 0, st>>>(amax, out_next, suffix_len, n);
+  return cudaGetLastError();
 }
 
 bool lean_shapes_ok(int d_model, int d_ffn, int Nq, int Nkv, int rank) {

@@ -190,6 +190,9 @@ struct PassIO {
   const int32_t* suffix_len = nullptr;
   int suffix_bound = 0;
   float* logits = nullptr;                 // [M][vocab] destination, nullptr: skip lm_head
+  int32_t* fused_next = nullptr;           // decode passes that want no logits: greedy tokens straight from the lm_head,
+                                           // suffix lengths advanced (set by forward when its path did both)
+  bool fused_done = false;
   AttnArgs plan;                           // chunking, filled by plan_pass
 };
 
@@ -373,7 +376,7 @@ bool lean_eligible(const mlora_ctx* c, const PassIO& io) {
          io.n <= CHAIN_MAX_ROWS && io.parent == c->root_parent && attn_single_pass(io.plan);
 }
 
-int forward_lean(mlora_ctx* c, const PassIO& io) {
+int forward_lean(mlora_ctx* c, PassIO& io) {
   const mlora_model_desc& d = c->d;
   cudaStream_t st = c->stream;
   CK(cudaMemsetAsync(c->step_tacc, 0, c->step_acc_bytes, st));   // the step's accumulators (a memset node, not a kernel)
@@ -386,6 +389,8 @@ int forward_lean(mlora_ctx* c, const PassIO& io) {
   }
   a.rank = (d.max_adapters > 0 && d.lora_targets != 0) ? d.lora_rank : 0;
   a.X = c->X; a.logits = io.logits; a.tacc = c->step_tacc; a.ssq = c->step_ssq;
+  const bool fused = io.fused_next != nullptr && d.vocab > 0;
+  if (fused) { a.logits = nullptr; a.amax = c->step_ssq + (size_t)c->n_ssq * CHAIN_MAX_ROWS; }
   for (size_t p = 0; p < c->step_phases_host.size(); ++p) {
     const StepPhase& ph = c->step_phases_host[p];
     if (ph.kind == SK_EMBED) {
@@ -393,7 +398,7 @@ int forward_lean(mlora_ctx* c, const PassIO& io) {
         return launch_lean_embed(a, ph, io.tokens, (const __half*)d.embed, d.vocab, io.hidden_in, c->status, st);
       }));
     } else if (ph.kind == SK_GEMM) {
-      if (ph.epi == EPI_F32 && ph.out_f32 == nullptr && io.logits == nullptr) continue;   // lm_head not wanted
+      if (ph.epi == EPI_F32 && ph.out_f32 == nullptr && io.logits == nullptr && !fused) continue;   // lm_head not wanted
       CK(run(c, MLORA_PROF_GEMM, [&] { return launch_lean_gemm(a, ph, st); }));
     } else if (ph.kind == SK_ATTN) {
       const int l = ph.layer;
@@ -414,10 +419,14 @@ int forward_lean(mlora_ctx* c, const PassIO& io) {
       CK(run(c, MLORA_PROF_ATTN, [&] { return launch_attention(at, st); }));
     }
   }
+  if (fused) {
+    CK(run(c, MLORA_PROF_MISC, [&] { return launch_lean_finish(a.amax, io.fused_next, c->suffix_len, io.n, st); }));
+    io.fused_done = true;
+  }
   return MLORA_OK;
 }
 
-int forward(mlora_ctx* c, const PassIO& io) {
+int forward(mlora_ctx* c, PassIO& io) {
   if (lean_eligible(c, io)) return forward_lean(c, io);
   if (chain_eligible(c, io)) return forward_chain(c, io);
   const mlora_model_desc& d = c->d;
@@ -865,10 +874,11 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
       const size_t tacc_bytes = (size_t)c->n_tacc * CHAIN_MAX_ROWS * 3 * (rr > 0 ? rr : 1) * sizeof(unsigned long long);
       // (one allocation for both kinds of accumulators: one memset clears a step's worth)
       const size_t ssq_bytes = (size_t)c->n_ssq * CHAIN_MAX_ROWS * sizeof(unsigned long long);
-      CKC(cudaMalloc(&c->step_tacc, tacc_bytes + ssq_bytes));
-      CKC(cudaMemsetAsync(c->step_tacc, 0, tacc_bytes + ssq_bytes, st));
+      const size_t amax_bytes = CHAIN_MAX_ROWS * sizeof(unsigned long long);   // row maxima of the lm_head (lean path)
+      CKC(cudaMalloc(&c->step_tacc, tacc_bytes + ssq_bytes + amax_bytes));
+      CKC(cudaMemsetAsync(c->step_tacc, 0, tacc_bytes + ssq_bytes + amax_bytes, st));
       c->step_ssq = c->step_tacc + tacc_bytes / sizeof(unsigned long long);
-      c->step_acc_bytes = tacc_bytes + ssq_bytes;
+      c->step_acc_bytes = tacc_bytes + ssq_bytes + amax_bytes;
       CKC(cudaMalloc(&c->step_amax, (size_t)c->sm_count * CHAIN_MAX_ROWS * sizeof(unsigned long long)));
       CKC(cudaMemsetAsync(c->step_amax, 0, (size_t)c->sm_count * CHAIN_MAX_ROWS * sizeof(unsigned long long), st));
       std::vector<StepPhase> sp;
@@ -1059,6 +1069,7 @@ static int decode_impl(mlora_ctx* c, int n, const int32_t* adapter_idx, const in
   io.n = n; io.T = 1; io.tokens = tokens; io.hidden_in = hidden; io.adapter_idx = adapter_idx;
   io.parent = c->root_parent; io.pos_base = c->P; io.suffix_len = c->suffix_len; io.suffix_bound = c->suffix_bound;
   io.logits = c->d.vocab > 0 ? (out_logits ? out_logits : c->logits) : nullptr;
+  if (c->d.vocab > 0 && out_logits == nullptr) io.fused_next = out_next;     // (taken up by the path that can)
   plan_pass(c, io);
   GraphKey key{};
   key.kind = hidden ? 2 : 1; key.n = n; key.T = 1;
@@ -1070,6 +1081,7 @@ static int decode_impl(mlora_ctx* c, int n, const int32_t* adapter_idx, const in
   rc = replay_or_run(c, key, [&]() -> int {
     int r = forward(c, io);
     if (r != MLORA_OK) return r;
+    if (io.fused_done) return MLORA_OK;               // tokens written, suffix lengths advanced
     if (c->d.vocab > 0) {
       CK(run(c, MLORA_PROF_MISC, [&] { return launch_argmax(io.logits, n, c->d.vocab, out_next, c->stream); }));
     } else {
@@ -1145,9 +1157,11 @@ static int generate_impl(mlora_ctx* c, int n, const int32_t* adapter_idx, const 
       io.n = n; io.T = 1; io.tokens = tok; io.adapter_idx = adapter_idx;
       io.parent = c->root_parent; io.pos_base = c->P; io.suffix_len = c->suffix_len; io.suffix_bound = bound0 + j;
       io.logits = c->logits;
+      io.fused_next = next;
       plan_pass(c, io);
       int r = forward(c, io);
       if (r != MLORA_OK) return r;
+      if (io.fused_done) continue;
       CK(run(c, MLORA_PROF_MISC, [&] { return launch_argmax(io.logits, n, c->d.vocab, next, c->stream); }));
       CK(run(c, MLORA_PROF_MISC, [&] { return launch_advance(c->suffix_len, nullptr, n, 1, c->stream); }));
     }
