@@ -10,6 +10,8 @@ constexpr int SHRINK_THREADS = 256;
 constexpr int SHRINK_JCHUNK = 8;   // rank indices per CTA
 
 __global__ void __launch_bounds__(SHRINK_THREADS) norm_shrink_kernel(const ShrinkArgs p, const int jchunks) {
+  // (the tensor-core projection launched after this kernel may start streaming its weights now)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __half* hrow = reinterpret_cast<__half*>(smem_raw);          // [K]
   __shared__ float red[SHRINK_THREADS / 32];
@@ -91,6 +93,8 @@ __global__ void __launch_bounds__(SHRINK_THREADS) norm_shrink_kernel(const Shrin
 // GEMM reads (written by the norm pass before), so the A matrix of a stream is fetched once per 16 rows.
 constexpr int SHRINK_MMA_WARPS = 16;
 __global__ void __launch_bounds__(SHRINK_MMA_WARPS * 32) shrink_mma_kernel(const ShrinkArgs p, const __half* __restrict__ h) {
+  // (the tensor-core projection launched after this kernel may start streaming its weights now)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   __shared__ float red[SHRINK_MMA_WARPS][32][4];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int m0 = blockIdx.x * 16, r = p.lora.rank, K = p.K;

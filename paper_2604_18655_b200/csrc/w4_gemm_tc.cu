@@ -118,6 +118,9 @@ w4_gemm_tc_kernel(const GemmArgs p, const int kts_per_split, int* status, const 
     // ---- activation producer (one thread).  Step j's tile: 64 features (x = kt * 64 elements: a multiple of 128
     // bytes) of NROWS rows from m0, rows >= M filled with zero; tile j % NSTB is refilled once step j - NSTB is done
     if (lane == 0) {
+      // programmatic launch: set-up, tensor memory and the dequantising warps' first weight tiles (immutable data) run
+      // while the kernel ahead of this one finishes; the activations are that kernel's output
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       int issued = 0;
       for (int j = 0; j < nk; ++j) {
         if (j >= NSTB) wait_step(j - NSTB);
@@ -518,8 +521,14 @@ static cudaError_t tc_launch(const GemmArgs& a, int slabs, int ksplit, int kts_p
   CUtensorMap map;
   const cudaError_t e = encode_act_map(a, NROWS, &map);
   if (e != cudaSuccess) return e;
-  w4_gemm_tc_kernel<NROWS><<<grid, TC_THREADS, smem, st>>>(a, kts_per_split, status, map);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = dim3(TC_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, w4_gemm_tc_kernel<NROWS>, a, kts_per_split, status, map);
 }
 
 cudaError_t init_gemm_tc() {
