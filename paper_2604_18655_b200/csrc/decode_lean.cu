@@ -175,8 +175,10 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
     for (int i = 0; i < PF; ++i) {
       const int kt = kb + i;
       if (kt < kt1 && row_live) {
-        x0[i] = __ldcg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * TILE_K));
-        x1[i] = __ldcg(reinterpret_cast<const uint4*>(xrow + (size_t)kt * TILE_K) + 1);
+        // (ordinary cached loads: the CTAs that share an SM read the same rows, and loads behind the wait see what
+        // the kernel ahead wrote)
+        x0[i] = *(reinterpret_cast<const uint4*>(xrow + (size_t)kt * TILE_K));
+        x1[i] = *(reinterpret_cast<const uint4*>(xrow + (size_t)kt * TILE_K) + 1);
       } else {
         x0[i] = make_uint4(0, 0, 0, 0);
         x1[i] = make_uint4(0, 0, 0, 0);
