@@ -195,6 +195,9 @@ int mlora_debug_dequant(mlora_ctx* ctx, int32_t layer, int32_t proj, void* out_f
  * key 2 = 1 disables CUDA-graph replay of steps (every kernel launched directly).
  * key 3 = 1 runs decode-sized passes through the general split-K kernels (one per operation: norm + shrink, projection,
  *         attention, ...) instead of any of the decode paths of key 6.
+ * key 4 = 1 runs passes of 32 rows and more through the split-K mma.sync kernels instead of the tcgen05 projection kernel.
+ * key 5 = 1 makes the first wait of the next decode step (paths 1 and 2 of key 6) run out, on a flag nothing sets: the
+ *         step returns the timeout status instead of hanging (the test of the bounded waits).
  * key 6 picks the path of decode steps (one row per stream, at most 8 streams): 1 = the per-layer persistent projection
  *         kernel plus attention kernels; 2 = ONE kernel that does the whole step (embedding to greedy token; where the
  *         model's shapes allow it, else the per-layer path); 3 = one small kernel per projection group, launched
