@@ -496,7 +496,7 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   // ahead of everything; its cp.async group is the oldest, so every later wait covers it)
   const __half* oA = nullptr;
   if (p.o_tacc != nullptr && rank == 0) {
-    const int ad = p.o_adapter_idx[s];
+    const int ad = p.o_direct ? s : p.o_adapter_idx[s];
     oA = (ad >= 0 && ad < p.o_n_slots) ? p.o_tabA[(size_t)ad * p.o_tab_stride + p.o_proj_index] : nullptr;
     if (oA != nullptr) {
       const int feats = g_heads * HD, ld = p.Hq * HD, pieces = feats / 8;

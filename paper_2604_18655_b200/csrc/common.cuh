@@ -29,6 +29,16 @@ struct WLayout {
   uint32_t chunk_full, chunk_last;             // bytes
   size_t unit_bytes;
 };
+// log2 of a power of two (group sizes below a chunk's 512 inputs are 64, 128 or 256: wlayout_group_ok)
+__host__ __device__ inline int wl_log2(int v) {
+#ifdef __CUDA_ARCH__
+  return 31 - __clz(v);
+#else
+  int s = 0;
+  while ((1 << (s + 1)) <= v) ++s;
+  return s;
+#endif
+}
 __host__ __device__ inline WLayout make_wlayout(int K, int N, int G) {
   WLayout L;
   L.K = K; L.N = N; L.G = G;
@@ -36,8 +46,9 @@ __host__ __device__ inline WLayout make_wlayout(int K, int N, int G) {
   L.nchunks = (L.KT + CHUNK_KT - 1) / CHUNK_KT;
   L.kc_last = L.KT - (L.nchunks - 1) * CHUNK_KT;
   const int ck = CHUNK_KT * TILE_K;
-  L.gpc = G >= ck ? 1 : ck / G;
-  L.g_last = G >= ck ? 1 : (L.kc_last * TILE_K + G - 1) / G;
+  // (G < ck: a power of two, so the divisions are shifts -- these run at the start of every kernel)
+  L.gpc = G >= ck ? 1 : ck >> wl_log2(G);
+  L.g_last = G >= ck ? 1 : (L.kc_last * TILE_K + G - 1) >> wl_log2(G);
   L.chunk_full = CHUNK_KT * 512 + L.gpc * 32;
   L.chunk_last = L.kc_last * 512 + L.g_last * 32;
   L.unit_bytes = (size_t)(L.nchunks - 1) * L.chunk_full + L.chunk_last;
@@ -54,7 +65,7 @@ __host__ __device__ inline size_t wl_tile_off(const WLayout& L, int kt) {
 __host__ __device__ inline size_t wl_scale_off(const WLayout& L, int kt) {
   const int c = kt / CHUNK_KT;
   const int kc = (c == L.nchunks - 1) ? L.kc_last : CHUNK_KT;
-  const int gi = (L.G >= CHUNK_KT * TILE_K) ? 0 : ((kt % CHUNK_KT) * TILE_K) / L.G;
+  const int gi = (L.G >= CHUNK_KT * TILE_K) ? 0 : ((kt % CHUNK_KT) * TILE_K) >> wl_log2(L.G);
   return (size_t)c * L.chunk_full + (size_t)kc * 512 + (size_t)gi * 32;
 }
 
@@ -140,6 +151,7 @@ struct AttnArgs {
   const __half* const* o_tabA;    // adapter A pointers [slot][o_tab_stride]
   const int32_t* o_adapter_idx;   // dev [n]
   int o_proj_index, o_rank, o_tab_stride, o_n_slots;
+  int o_direct;                   // o_tabA is indexed by stream (looked up once per call): o_adapter_idx is not read
   int pdl;                        // launch the single-kernel decode attention with programmatic stream serialisation
 };
 
@@ -205,6 +217,7 @@ cudaError_t launch_chain(const ChainArgs& a, int sm_count, cudaStream_t st);
 // projection group, the attention of every layer, lm_head, row argmax and the suffix-length update are phases
 // separated by grid barriers.
 enum StepKind { SK_EMBED = 0, SK_GEMM = 1, SK_ATTN = 2, SK_FIN = 3 };
+constexpr unsigned long long LEAN_PF_MAX_BYTES = 16ull << 20;   // at most this much of the next group's weights is asked for in L2
 struct StepPhase {
   int kind, layer;
   const unsigned char* w;         // SK_GEMM: packed weights
@@ -228,6 +241,8 @@ struct StepPhase {
   int t_out;                      // where the partial shrink sums over this phase's outputs are accumulated
   int last;                       // the residual rows this phase writes are the call's hidden-state output
   int pad_;
+  const unsigned char* pf_w;      // kernel-per-projection path: packed weights of the projection group that runs next,
+  unsigned long long pf_bytes;    // asked for in L2 by this phase's CTAs (a share each); 0: nothing
 };
 struct StepArgs {
   const StepPhase* phases;        // dev
@@ -327,10 +342,21 @@ struct LeanArgs {
   float* logits;                  // destination of a phase whose out_f32 is null
   unsigned long long* tacc;       // [n_tacc][8][3][rank]
   unsigned long long* ssq;        // [n_ssq][8]
+  int rank_log2;                  // log2(rank) when the rank is a power of two, else -1 (index arithmetic by shifts)
+  int rows_direct;                // tabA / tabB / scale are indexed by ROW (looked up once per call): adapter_idx is not read
   int late_wait;                  // the kernel ahead produces only T: wait for it after the main loop, not before
   unsigned long long* amax;       // [8]: row maxima of the lm_head as (ordered value, complemented column) keys, zero at
                                   // the start of a step; non-null = no logits are written, the greedy tokens come from here
 };
+inline int lean_rank_log2(int r) {                     // LeanArgs::rank_log2
+  if (r <= 0 || (r & (r - 1)) != 0) return -1;
+  int s = 0;
+  while ((1 << s) < r) ++s;
+  return s;
+}
+cudaError_t launch_lean_rowptr(const int32_t* adapter_idx, const __half* const* tabA, const __half* const* tabB, const float* scale,
+                               int n_slots, int tab_stride, int M, const __half** rowA, const __half** rowB, float* rowscale,
+                               cudaStream_t st);
 cudaError_t launch_lean_finish(const unsigned long long* amax, int32_t* out_next, int32_t* suffix_len, int n, cudaStream_t st);
 cudaError_t init_lean();
 bool lean_shapes_ok(int d_model, int d_ffn, int Nq, int Nkv, int rank);

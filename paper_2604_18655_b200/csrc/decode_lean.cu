@@ -43,29 +43,42 @@ __device__ __forceinline__ void ln_cp_async16(void* smem, const void* gmem, bool
 //   sB [NTILE][M][r][16]: rows of B of this group for the CTA's columns (the expand);
 //   sA [M][next_nseg][r][16]: rows of A of the consuming group for the CTA's output columns (its partial shrink).
 // A missing adapter or matrix gives zeros.
+// x = q * rank + j by shifts where the rank is a power of two (runtime divisions cost tens of instructions each, and
+// these index computations sit at the start of every CTA and behind its main loop)
+__device__ __forceinline__ void ln_divmod_rank(const LeanArgs& a, int x, int& q, int& j) {
+  if (a.rank_log2 >= 0) { q = x >> a.rank_log2; j = x & (a.rank - 1); }
+  else { q = x / a.rank; j = x - q * a.rank; }
+}
+
+// Items run over all CHAIN_MAX_ROWS rows (row = low three bits of the quotient; rows past M are skipped), so that no
+// index needs a division by the row count.
 template <int NTILE>
 __device__ __forceinline__ void lean_prefetch_slices(const LeanArgs& a, const StepPhase& ph, int tile0, int n_out0, bool lora,
                                                      __half* sB, __half* sA) {
   const int r = a.rank, M = a.M;
-  if (lora) {
-    for (int it = threadIdx.x; it < NTILE * M * r * 2; it += blockDim.x) {
-      const int hf = it & 1, j = (it >> 1) % r, m = ((it >> 1) / r) % M, u = (it >> 1) / (r * M);
-      const int ad = a.adapter_idx[m];
-      int seg, col;
-      map_col(ph.mode, (tile0 + u) * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
-      const __half* B = (ad >= 0 && ad < a.n_slots) ? a.tabB[(size_t)ad * a.tab_stride + ph.lora_proj[seg]] : nullptr;
-      ln_cp_async16(sB + (((size_t)u * M + m) * r + j) * 16 + hf * 8, B ? B + (size_t)j * ph.lora_n[seg] + col + hf * 8 : (const __half*)ph.w,
-                    B != nullptr);
-    }
+  const int nB = lora ? NTILE * CHAIN_MAX_ROWS * r * 2 : 0;
+  const int nA = (ph.next_nseg > 0 && a.adapter_idx != nullptr) ? ph.next_nseg * CHAIN_MAX_ROWS * r * 2 : 0;
+  for (int it = threadIdx.x; it < nB; it += blockDim.x) {
+    int q, j;
+    ln_divmod_rank(a, it >> 1, q, j);
+    const int hf = it & 1, m = q & (CHAIN_MAX_ROWS - 1), u = q >> 3;
+    if (m >= M) continue;
+    const int ad = a.rows_direct ? m : a.adapter_idx[m];
+    int seg, col;
+    map_col(ph.mode, (tile0 + u) * TILE_N, ph.seg_n0, ph.seg_n1, seg, col);
+    const __half* B = (ad >= 0 && ad < a.n_slots) ? a.tabB[(size_t)ad * a.tab_stride + ph.lora_proj[seg]] : nullptr;
+    ln_cp_async16(sB + (((size_t)u * M + m) * r + j) * 16 + hf * 8, B ? B + (size_t)j * ph.lora_n[seg] + col + hf * 8 : (const __half*)ph.w,
+                  B != nullptr);
   }
-  if (ph.next_nseg > 0 && a.adapter_idx != nullptr) {
-    for (int it = threadIdx.x; it < M * ph.next_nseg * r * 2; it += blockDim.x) {
-      const int hf = it & 1, j = (it >> 1) % r, seg = ((it >> 1) / r) % ph.next_nseg, m = (it >> 1) / (r * ph.next_nseg);
-      const int ad = a.adapter_idx[m];
-      const __half* A = (ad >= 0 && ad < a.n_slots) ? a.tabA[(size_t)ad * a.tab_stride + ph.next_proj[seg]] : nullptr;
-      ln_cp_async16(sA + (((size_t)m * ph.next_nseg + seg) * r + j) * 16 + hf * 8,
-                    A ? A + (size_t)j * ph.next_ld + n_out0 + hf * 8 : (const __half*)ph.w, A != nullptr);
-    }
+  for (int it = threadIdx.x; it < nA; it += blockDim.x) {
+    int q, j;
+    ln_divmod_rank(a, it >> 1, q, j);
+    const int hf = it & 1, m = q & (CHAIN_MAX_ROWS - 1), seg = q >> 3;
+    if (m >= M) continue;
+    const int ad = a.rows_direct ? m : a.adapter_idx[m];
+    const __half* A = (ad >= 0 && ad < a.n_slots) ? a.tabA[(size_t)ad * a.tab_stride + ph.next_proj[seg]] : nullptr;
+    ln_cp_async16(sA + (((size_t)m * ph.next_nseg + seg) * r + j) * 16 + hf * 8,
+                  A ? A + (size_t)j * ph.next_ld + n_out0 + hf * 8 : (const __half*)ph.w, A != nullptr);
   }
   asm volatile("cp.async.commit_group;" ::: "memory");
 }
@@ -75,14 +88,17 @@ __device__ __forceinline__ void lean_prefetch_slices(const LeanArgs& a, const St
 __device__ __forceinline__ void lean_shrink_partial(const LeanArgs& a, const StepPhase& ph, const __half (*vals)[16], const __half* sA) {
   if (ph.next_nseg == 0 || a.adapter_idx == nullptr) return;
   const int r = a.rank;
-  for (int it = threadIdx.x; it < a.M * ph.next_nseg * r; it += blockDim.x) {
-    const int j = it % r, seg = (it / r) % ph.next_nseg, m = it / (r * ph.next_nseg);
-    const __half2* av = reinterpret_cast<const __half2*>(sA + (size_t)it * 16);
+  for (int it = threadIdx.x; it < ph.next_nseg * CHAIN_MAX_ROWS * r; it += blockDim.x) {
+    int q, j;
+    ln_divmod_rank(a, it, q, j);
+    const int m = q & (CHAIN_MAX_ROWS - 1), seg = q >> 3;
+    if (m >= a.M) continue;
+    const __half2* av = reinterpret_cast<const __half2*>(sA + (((size_t)m * ph.next_nseg + seg) * r + j) * 16);
     const __half2* xv = reinterpret_cast<const __half2*>(vals[m]);
     float s = 0.f;
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      const float2 x = __half22float2(xv[q]), w = __half22float2(av[q]);
+    for (int q2 = 0; q2 < 8; ++q2) {
+      const float2 x = __half22float2(xv[q2]), w = __half22float2(av[q2]);
       s = fmaf(x.x, w.x, s); s = fmaf(x.y, w.y, s);
     }
     ln_red_add(a.tacc + ((size_t)ph.t_out * CHAIN_MAX_ROWS + m) * 3 * r + seg * r + j, ln_fix(s));
@@ -137,6 +153,16 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
     }
   };
   load_weights(kt0);                                                       // (first: the longest latency)
+  // this CTA's share of the next projection group's weights, asked for in L2: that kernel's CTAs mostly start only
+  // when this kernel's leave their SMs, and then find their weights a short trip away
+  if (threadIdx.x == 32 && ph.pf_bytes != 0) {
+    const unsigned long long per = ((ph.pf_bytes / gridDim.x) + 15ull) & ~15ull;
+    const unsigned long long b0 = per * blockIdx.x, b1 = b0 + per < ph.pf_bytes ? b0 + per : (ph.pf_bytes & ~15ull);
+    for (unsigned long long o = b0; o < b1; o += 16384ull) {
+      const uint32_t n = (uint32_t)(b1 - o < 16384ull ? b1 - o : 16384ull);
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(ph.pf_w + o), "r"(n) : "memory");
+    }
+  }
   lean_prefetch_slices<NTILE>(a, ph, tile0, n_out0, lora, sB, sA);
   pdl_wait();
   // ---- what earlier kernels produced: the old residual, norm factors, T of this group, the input rows
@@ -152,9 +178,12 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
     s_inv[threadIdx.x] = inv;
   }
   auto load_T = [&]() {
-    for (int i = threadIdx.x; i < M * ph.lora_nseg * r; i += THREADS) {
-      const int m = i / (ph.lora_nseg * r), rest = i % (ph.lora_nseg * r);
-      const int ad = a.adapter_idx[m];
+    for (int i = threadIdx.x; i < ph.lora_nseg * CHAIN_MAX_ROWS * r; i += THREADS) {
+      int q, j;
+      ln_divmod_rank(a, i, q, j);
+      const int m = q & (CHAIN_MAX_ROWS - 1), rest = (q >> 3) * r + j;
+      if (m >= M) continue;
+      const int ad = a.rows_direct ? m : a.adapter_idx[m];
       float v = 0.f;
       if (ad >= 0 && ad < a.n_slots)
         v = ln_unfix(__ldcg(a.tacc + ((size_t)ph.t_in * CHAIN_MAX_ROWS + m) * 3 * r + rest)) * a.scale[ad];
@@ -358,7 +387,7 @@ __global__ void __launch_bounds__(LN_THREADS) lean_embed_kernel(const LeanArgs a
     ln_red_add(a.ssq + (size_t)ph.ssq_out * CHAIN_MAX_ROWS + m, ln_fix(tot));
   }
   if (ph.next_nseg == 0 || a.adapter_idx == nullptr) return;
-  const int ad = a.adapter_idx[m];
+  const int ad = a.rows_direct ? m : a.adapter_idx[m];
   if (ad < 0 || ad >= a.n_slots) return;
   const int r = a.rank;
   // the CTA's share of the (segment, rank index, 1024-element piece of the row) partial dot products, a warp each
@@ -407,6 +436,30 @@ __global__ void lean_finish_kernel(const unsigned long long* __restrict__ amax, 
 
 cudaError_t launch_lean_finish(const unsigned long long* amax, int32_t* out_next, int32_t* suffix_len, int n, cudaStream_t st) {
   lean_finish_kernel<<<1, 32, 0, st>>>(amax, out_next, suffix_len, n);
+  return cudaGetLastError();
+}
+
+// The adapter matrices of every row, looked up once per call: rowA/rowB[m][p] = A/B of row m's adapter for
+// projection p (nullptr: none), rowscale[m] its scale.  The per-projection kernels then index by row and skip the
+// adapter-index load that every pointer lookup would otherwise wait for.
+__global__ void lean_rowptr_kernel(const int32_t* __restrict__ adapter_idx, const __half* const* __restrict__ tabA,
+                                   const __half* const* __restrict__ tabB, const float* __restrict__ scale, int n_slots,
+                                   int tab_stride, int M, const __half** rowA, const __half** rowB, float* rowscale) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= CHAIN_MAX_ROWS * tab_stride) return;
+  const int m = i / tab_stride, p = i % tab_stride;
+  const int ad = (m < M && adapter_idx != nullptr) ? adapter_idx[m] : -1;
+  const bool ok = ad >= 0 && ad < n_slots;
+  rowA[i] = ok ? tabA[(size_t)ad * tab_stride + p] : nullptr;
+  rowB[i] = ok ? tabB[(size_t)ad * tab_stride + p] : nullptr;
+  if (p == 0) rowscale[m] = ok ? scale[ad] : 0.f;
+}
+
+cudaError_t launch_lean_rowptr(const int32_t* adapter_idx, const __half* const* tabA, const __half* const* tabB, const float* scale,
+                               int n_slots, int tab_stride, int M, const __half** rowA, const __half** rowB, float* rowscale,
+                               cudaStream_t st) {
+  const int total = CHAIN_MAX_ROWS * tab_stride;
+  lean_rowptr_kernel<<<(total + 255) / 256, 256, 0, st>>>(adapter_idx, tabA, tabB, scale, n_slots, tab_stride, M, rowA, rowB, rowscale);
   return cudaGetLastError();
 }
 

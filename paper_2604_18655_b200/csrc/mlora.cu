@@ -115,6 +115,9 @@ struct mlora_ctx {
   std::vector<StepPhase> step_phases_host;
   size_t step_acc_bytes = 0;         // step_tacc and step_ssq, contiguous
   bool lean_ok = false;              // the per-projection decode kernels take this model's shapes
+  const __half** step_rowA = nullptr;   // dev [8][L*7]: the rows' adapter matrices, looked up once per call (lean path)
+  const __half** step_rowB = nullptr;
+  float* step_rowscale = nullptr;    // dev [8]
   StepPhase* step_phases = nullptr;  // dev [5*L + 3]: embed; qkv, attention, o, gate/up, down per layer; lm_head; end
   int n_step_phases = 0, step_stages = 0, step_own_tiles = 0;
   unsigned char *tmapA = nullptr, *tmapB = nullptr;           // dev [max_adapters][L*7] tensor maps over the adapters' matrices
@@ -193,6 +196,7 @@ struct PassIO {
   int32_t* fused_next = nullptr;           // decode passes that want no logits: greedy tokens straight from the lm_head,
                                            // suffix lengths advanced (set by forward when its path did both)
   bool fused_done = false;
+  bool rows_resolved = false;              // the rows' adapter pointers were looked up earlier in this call (same adapter_idx)
   AttnArgs plan;                           // chunking, filled by plan_pass
 };
 
@@ -384,10 +388,18 @@ int forward_lean(mlora_ctx* c, PassIO& io) {
   a.M = io.n; a.eps = d.rms_eps;
   const bool lora = io.adapter_idx != nullptr && d.lora_rank > 0 && d.max_adapters > 0 && d.lora_targets != 0;
   if (lora) {
-    a.adapter_idx = io.adapter_idx; a.tabA = c->tabA; a.tabB = c->tabB; a.scale = c->ad_scale;
-    a.tab_stride = c->L * 7; a.n_slots = d.max_adapters;
+    // the rows' adapter matrices by row: one small kernel per call, ordinary launch (everything behind it sees the table)
+    if (!io.rows_resolved)
+      CK(run(c, MLORA_PROF_MISC, [&] {
+        return launch_lean_rowptr(io.adapter_idx, c->tabA, c->tabB, c->ad_scale, d.max_adapters, c->L * 7, io.n, c->step_rowA,
+                                  c->step_rowB, c->step_rowscale, st);
+      }));
+    a.adapter_idx = io.adapter_idx; a.rows_direct = 1;
+    a.tabA = c->step_rowA; a.tabB = c->step_rowB; a.scale = c->step_rowscale;
+    a.tab_stride = c->L * 7; a.n_slots = CHAIN_MAX_ROWS;
   }
   a.rank = (d.max_adapters > 0 && d.lora_targets != 0) ? d.lora_rank : 0;
+  a.rank_log2 = lean_rank_log2(a.rank);
   a.X = c->X; a.logits = io.logits; a.tacc = c->step_tacc; a.ssq = c->step_ssq;
   const bool fused = io.fused_next != nullptr && d.vocab > 0;
   if (fused) { a.logits = nullptr; a.amax = c->step_ssq + (size_t)c->n_ssq * CHAIN_MAX_ROWS; }
@@ -413,8 +425,8 @@ int forward_lean(mlora_ctx* c, PassIO& io) {
       at.pdl = 1;
       if (lora && ph.next_nseg > 0) {
         at.o_tacc = c->step_tacc + (size_t)ph.t_out * CHAIN_MAX_ROWS * 3 * a.rank;
-        at.o_tabA = c->tabA; at.o_adapter_idx = io.adapter_idx; at.o_proj_index = ph.next_proj[0]; at.o_rank = a.rank;
-        at.o_tab_stride = c->L * 7; at.o_n_slots = d.max_adapters;
+        at.o_tabA = c->step_rowA; at.o_adapter_idx = io.adapter_idx; at.o_direct = 1; at.o_proj_index = ph.next_proj[0]; at.o_rank = a.rank;
+        at.o_tab_stride = c->L * 7; at.o_n_slots = CHAIN_MAX_ROWS;
       }
       CK(run(c, MLORA_PROF_ATTN, [&] { return launch_attention(at, st); }));
     }
@@ -879,6 +891,9 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
       CKC(cudaMemsetAsync(c->step_tacc, 0, tacc_bytes + ssq_bytes + amax_bytes, st));
       c->step_ssq = c->step_tacc + tacc_bytes / sizeof(unsigned long long);
       c->step_acc_bytes = tacc_bytes + ssq_bytes + amax_bytes;
+      CKC(cudaMalloc(&c->step_rowA, (size_t)CHAIN_MAX_ROWS * L * 7 * sizeof(__half*)));
+      CKC(cudaMalloc(&c->step_rowB, (size_t)CHAIN_MAX_ROWS * L * 7 * sizeof(__half*)));
+      CKC(cudaMalloc(&c->step_rowscale, CHAIN_MAX_ROWS * sizeof(float)));
       CKC(cudaMalloc(&c->step_amax, (size_t)c->sm_count * CHAIN_MAX_ROWS * sizeof(unsigned long long)));
       CKC(cudaMemsetAsync(c->step_amax, 0, (size_t)c->sm_count * CHAIN_MAX_ROWS * sizeof(unsigned long long), st));
       std::vector<StepPhase> sp;
@@ -947,6 +962,19 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
       StepPhase fin{};
       fin.kind = SK_FIN; fin.norm_in = -1; fin.ssq_out = -1;
       sp.push_back(fin);
+      // each projection phase names the weights of the next one (the step after the lm_head starts with layer 0 again):
+      // its CTAs ask for them in L2 while they run (kernel-per-projection path)
+      {
+        std::vector<int> gi;
+        for (size_t i = 0; i < sp.size(); ++i) if (sp[i].kind == SK_GEMM) gi.push_back((int)i);
+        for (size_t k = 0; k < gi.size(); ++k) {
+          const StepPhase& nx = sp[gi[(k + 1) % gi.size()]];
+          const WLayout nl = make_wlayout(nx.K, nx.N, nx.G);
+          const unsigned long long bytes = (unsigned long long)nl.NT * nl.unit_bytes;
+          sp[gi[k]].pf_w = nx.w;
+          sp[gi[k]].pf_bytes = bytes < LEAN_PF_MAX_BYTES ? bytes : LEAN_PF_MAX_BYTES;
+        }
+      }
       c->n_step_phases = (int)sp.size();
       CKC(cudaMalloc(&c->step_trace, sp.size() * 2 * 12 * sizeof(long long)));
       CKC(cudaMemsetAsync(c->step_trace, 0, sp.size() * 2 * 12 * sizeof(long long), st));
@@ -976,7 +1004,8 @@ int mlora_destroy(mlora_ctx* c) {
                       c->h, c->attn16, c->act16, c->counters, c->anc, c->depth, c->argmax, c->suffix_len,
                       c->zero_len, c->chain_parent, c->root_parent, c->status, c->cs_table, (void*)c->tabA,
                       (void*)c->tabB, c->ad_scale, c->phases, c->chain_sync, c->host_io, c->step_phases, c->xg_attn, c->xg_ffn,
-                      c->step_tacc, c->step_amax, c->step_trace, c->tmapA, c->tmapB, c->gen_tokens, c->draft_cand};
+                      c->step_tacc, c->step_amax, c->step_trace, c->tmapA, c->tmapB, c->gen_tokens, c->draft_cand,
+                      (void*)c->step_rowA, (void*)c->step_rowB, c->step_rowscale};
   for (void* p : dev_ptrs) if (p) cudaFree(p);
   if (c->stageA) cudaFreeHost((void*)c->stageA);
   if (c->stageB) cudaFreeHost((void*)c->stageB);
@@ -1158,6 +1187,7 @@ static int generate_impl(mlora_ctx* c, int n, const int32_t* adapter_idx, const 
       io.parent = c->root_parent; io.pos_base = c->P; io.suffix_len = c->suffix_len; io.suffix_bound = bound0 + j;
       io.logits = c->logits;
       io.fused_next = next;
+      io.rows_resolved = j > 0;
       plan_pass(c, io);
       int r = forward(c, io);
       if (r != MLORA_OK) return r;
@@ -1566,7 +1596,7 @@ int mlora_linear(mlora_weight* w, const void* x, int32_t M, const int32_t* row_a
     ph.in16 = (const __half*)x; ph.norm_in = -1; ph.out_f32 = y; ph.ldo = w->w.N; ph.ssq_out = -1;
     if (lora) {
       a.adapter_idx = row_adapter; a.tabA = (const __half* const*)A; a.tabB = (const __half* const*)B; a.scale = scale;
-      a.tab_stride = 1; a.n_slots = n_adapters; a.rank = rank;
+      a.tab_stride = 1; a.n_slots = n_adapters; a.rank = rank; a.rank_log2 = lean_rank_log2(rank);
       a.tacc = (unsigned long long*)(ws + LIN_COUNTER_BYTES + lin_T_bytes(M, rank));
       ph.lora_nseg = 1; ph.lora_proj[0] = 0; ph.lora_n[0] = w->w.N; ph.t_in = 0;
       StepPhase sh{};
