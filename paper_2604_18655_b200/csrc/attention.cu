@@ -424,6 +424,8 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   // (programmatic launches around this kernel: the kernel after it may start its own independent loads now; nothing
   // here is read before the kernel ahead has finished -- both are no-ops in ordinary launches)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // first phase of the cluster barrier: "this CTA runs" (waited for before the peer's shared memory is written)
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __half* Qs = reinterpret_cast<__half*>(smem_raw);                       // [16][STRIDE]
   __half* tiles = Qs + 16 * STRIDE;                                       // [W][2 buffers][K, V][DEC_KEYS][STRIDE]
@@ -512,10 +514,17 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   // (programmatic launch: the shared prefix does not change in decode, and the suffix lengths were last written by the
   // step before this one, which an ordinary launch at the start of this step has waited for)
   S = p.suffix_len[s];
+  if (fused && p.depth == nullptr) {
+    // rows without a tree depth (plain decode): the rotation table row of the new position is known already -- asked
+    // for now, so that the rotation behind the wait waits only for the projections
+    cs = p.cs_table + (size_t)(p.pos_base + S) * (HD / 2);
+    if (threadIdx.x < (HD / 2) * (int)sizeof(float2) / 128)
+      asm volatile("prefetch.global.L1 [%0];" ::"l"(reinterpret_cast<const char*>(cs) + threadIdx.x * 128) : "memory");
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");
   own_keys = S + 1;                                                       // cached rows + this pass's row
   n_tiles = n_ptiles + (own_keys + DEC_KEYS - 1) / DEC_KEYS;
-  if (fused) cs = p.cs_table + (size_t)(p.pos_base + S + p.depth[m]) * (HD / 2);
+  if (fused && p.depth != nullptr) cs = p.cs_table + (size_t)(p.pos_base + S + p.depth[m]) * (HD / 2);
   if (tile_of(warp) >= n_ptiles && tile_of(warp) < n_tiles) load_tile(tile_of(warp), 0);
   if (tile_of(warp + W) < n_tiles) load_tile(tile_of(warp + W), 1);
   // the warp's later tiles: ask for them in L2 now, so that their copies two iterations on do not wait for HBM
@@ -660,36 +669,42 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
       den += f * part_ml[((size_t)w * 16 + r) * 2 + 1];
     }
   };
+  // The second CTA of the cluster PUSHES its result into the first one's exchange area (distributed shared memory),
+  // so that after the barrier the first CTA combines from its own shared memory and nothing of the second CTA's is
+  // read any more: no barrier at the end.  Every thread of both CTAs takes both barrier phases (no early exit above).
+  static_assert(DEC_SPLIT == 2, "one exchange area: one peer");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");       // (phase 1: the peer runs)
+  float M_own = -INFINITY, num_own = 0.f, den_own = 0.f;                   // this thread's first element, ahead of the barrier
   if (rank != 0) {
+    uint32_t dst;                                                          // rank 0's xch in the cluster's shared window
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"((uint32_t)__cvta_generic_to_shared(xch)), "r"(0));
+    auto push = [&](int idx, float v) { asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(dst + 4u * (uint32_t)idx), "f"(v) : "memory"); };
     for (int i = threadIdx.x; i < g_heads * HD; i += W * 32) {
       const int r = i / HD, d = i % HD;
       float M, num, den;
       cta_result(r, d, M, num, den);
-      xch[r * (HD + 2) + d] = num;
-      if (d == 0) { xch[r * (HD + 2) + HD] = M; xch[r * (HD + 2) + HD + 1] = den; }
+      push(r * (HD + 2) + d, num);
+      if (d == 0) { push(r * (HD + 2) + HD, M); push(r * (HD + 2) + HD + 1, den); }
     }
+  } else if (threadIdx.x < g_heads * HD) {
+    cta_result(threadIdx.x / HD, threadIdx.x % HD, M_own, num_own, den_own);
   }
-  // every thread of both CTAs gets here (no early exit above): the peer's result is complete and visible
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
   if (rank == 0) {
-    const uint32_t mine = (uint32_t)__cvta_generic_to_shared(xch);
     for (int i = threadIdx.x; i < g_heads * HD; i += W * 32) {
       const int r = i / HD, d = i % HD;
-      float M, num, den;
-      cta_result(r, d, M, num, den);
+      float M = M_own, num = num_own, den = den_own;
+      if (i != (int)threadIdx.x) cta_result(r, d, M, num, den);
       if (M == -INFINITY) { num = 0.f; den = 0.f; }
-#pragma unroll
-      for (int pr = 1; pr < DEC_SPLIT; ++pr) {             // peer order: fixed
-        uint32_t peer;                                     // the peer's xch in the cluster's shared window
-        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(peer) : "r"(mine), "r"(pr));
-        auto peer_f32 = [&](int idx) { float v; asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(peer + 4u * (uint32_t)idx) : "memory"); return v; };
-        const float num1 = peer_f32(r * (HD + 2) + d), M1 = peer_f32(r * (HD + 2) + HD), den1 = peer_f32(r * (HD + 2) + HD + 1);
-        if (M1 == -INFINITY) continue;                     // a peer without tiles
-        const float Mn = fmaxf(M, M1);
-        const float f0 = (M == -INFINITY) ? 0.f : exp2f(M - Mn), f1 = exp2f(M1 - Mn);
-        num = f0 * num + f1 * num1;
-        den = f0 * den + f1 * den1;
-        M = Mn;
+      {
+        const float num1 = xch[r * (HD + 2) + d], M1 = xch[r * (HD + 2) + HD], den1 = xch[r * (HD + 2) + HD + 1];
+        if (M1 != -INFINITY) {                             // (a peer without tiles contributes nothing)
+          const float Mn = fmaxf(M, M1);
+          const float f0 = (M == -INFINITY) ? 0.f : exp2f(M - Mn), f1 = exp2f(M1 - Mn);
+          num = f0 * num + f1 * num1;
+          den = f0 * den + f1 * den1;
+          M = Mn;
+        }
       }
       const __half hv = __float2half_rn(den > 0.f ? num / den : 0.f);
       p.out[((size_t)m * p.Hq + kh * g_heads + r) * HD + d] = hv;
@@ -721,8 +736,6 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
       }
     }
   }
-  // the peer's shared memory must outlive the reads above
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 

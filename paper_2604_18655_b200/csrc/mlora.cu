@@ -415,7 +415,7 @@ int forward_lean(mlora_ctx* c, PassIO& io) {
     } else if (ph.kind == SK_ATTN) {
       const int l = ph.layer;
       AttnArgs at = io.plan;
-      at.qkv_f32 = c->qkv; at.cs_table = c->cs_table; at.pos_base = io.pos_base; at.depth = c->zero_len;   // one row per stream: depth 0
+      at.qkv_f32 = c->qkv; at.cs_table = c->cs_table; at.pos_base = io.pos_base; at.depth = nullptr;   // one row per stream: depth 0, nothing to read
       at.prefix_k = c->prefix_k + (size_t)l * c->prefix_layer_stride;
       at.prefix_v = c->prefix_v + (size_t)l * c->prefix_layer_stride;
       at.prefix_head_stride = c->prefix_head_stride;
