@@ -415,7 +415,7 @@ constexpr int DEC_SPLIT = 2;                 // CTAs (one cluster) that share th
 __host__ __device__ constexpr int dec_warps(int hd) { return hd == 64 ? 8 : 4; }
 __host__ __device__ constexpr size_t dec_smem_bytes(int hd) {
   return (size_t)16 * (hd + 8) * 2 + (size_t)dec_warps(hd) * 4 * DEC_KEYS * (hd + 8) * 2 +
-         (size_t)dec_warps(hd) * 16 * (hd + 2) * 4 + (size_t)16 * (hd + 2) * 4;
+         (size_t)dec_warps(hd) * 16 * (hd + 2) * 4 + (size_t)16 * (hd + 2) * 4 + (size_t)2 * hd * 2;
 }
 
 template <int HD>
@@ -432,7 +432,8 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   float* part_o = reinterpret_cast<float*>(tiles + (size_t)W * 4 * DEC_KEYS * STRIDE);   // [W][16][HD]
   float* part_ml = part_o + (size_t)W * 16 * HD;                          // [W][16][2]
   float* xch = part_ml + (size_t)W * 16 * 2;                              // [16][HD + 2]: this CTA's result for its peer
-  __half* a_sl = reinterpret_cast<__half*>(xch + 16 * (HD + 2));          // [o_rank][g_heads * HD]: the o adapter's A rows
+  __half (*newkv)[HD] = reinterpret_cast<__half (*)[HD]>(xch + 16 * (HD + 2));   // [2][HD]: the pass's new K (rotated) and V rows
+  __half* a_sl = reinterpret_cast<__half*>(xch + 16 * (HD + 2)) + 2 * HD;  // [o_rank][g_heads * HD]: the o adapter's A rows
   const int rank = blockIdx.z;                                            // position in the cluster (1, 1, DEC_SPLIT)
   auto tile_of = [&](int li) { return li * DEC_SPLIT + rank; };          // the CTA's li-th tile
 
@@ -451,7 +452,8 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   const float2* cs = nullptr;
 
   __half* my_tiles = tiles + (size_t)warp * 4 * DEC_KEYS * STRIDE;
-  auto load_tile = [&](int ti, int buf) {
+  // (new_row_later: the pass's new row is not there yet -- the caller puts it in with fill_new_row)
+  auto load_tile = [&](int ti, int buf, bool new_row_later = false) {
     __half* kd = my_tiles + (size_t)buf * 2 * DEC_KEYS * STRIDE;
     __half* vd = kd + DEC_KEYS * STRIDE;
     const bool own = ti >= n_ptiles;
@@ -481,12 +483,11 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
         *reinterpret_cast<uint4*>(kd + (size_t)r * STRIDE + c) = make_uint4(0, 0, 0, 0);
         *reinterpret_cast<uint4*>(vd + (size_t)r * STRIDE + c) = make_uint4(0, 0, 0, 0);
       } else if (fused && own && key == S) {
-        const uint4 kv8 = head_piece_f16(prow + (size_t)(p.Hq + kh) * HD, c, HD, cs);
-        const uint4 vv8 = head_piece_f16(prow + (size_t)(p.Hq + p.Hkv + kh) * HD, c, HD, nullptr);
-        *reinterpret_cast<uint4*>(kd + (size_t)r * STRIDE + c) = kv8;
-        *reinterpret_cast<uint4*>(vd + (size_t)r * STRIDE + c) = vv8;
-        *reinterpret_cast<uint4*>(ok + (size_t)key * HD + c) = kv8;
-        *reinterpret_cast<uint4*>(ov + (size_t)key * HD + c) = vv8;
+        // the pass's new row: built (rotated, appended to the cache) next to the query rows, copied from there
+        if (!new_row_later) {
+          *reinterpret_cast<uint4*>(kd + (size_t)r * STRIDE + c) = *reinterpret_cast<const uint4*>(&newkv[0][c]);
+          *reinterpret_cast<uint4*>(vd + (size_t)r * STRIDE + c) = *reinterpret_cast<const uint4*>(&newkv[1][c]);
+        }
       } else {
         cp_async16(kd + (size_t)r * STRIDE + c, kb + (size_t)key * HD + c);
         cp_async16(vd + (size_t)r * STRIDE + c, vb + (size_t)key * HD + c);
@@ -525,8 +526,11 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
   own_keys = S + 1;                                                       // cached rows + this pass's row
   n_tiles = n_ptiles + (own_keys + DEC_KEYS - 1) / DEC_KEYS;
   if (fused && p.depth != nullptr) cs = p.cs_table + (size_t)(p.pos_base + S + p.depth[m]) * (HD / 2);
-  if (tile_of(warp) >= n_ptiles && tile_of(warp) < n_tiles) load_tile(tile_of(warp), 0);
-  if (tile_of(warp + W) < n_tiles) load_tile(tile_of(warp + W), 1);
+  // (the tile that holds the new row gets its cached rows now and the new row once that has been built: below, with
+  // the query rows, so that the loads of all of them are in flight together)
+  const int s_tile = fused ? n_ptiles + S / DEC_KEYS : -1;
+  if (tile_of(warp) >= n_ptiles && tile_of(warp) < n_tiles) load_tile(tile_of(warp), 0, true);
+  if (tile_of(warp + W) < n_tiles) load_tile(tile_of(warp + W), 1, true);
   // the warp's later tiles: ask for them in L2 now, so that their copies two iterations on do not wait for HBM
   if (lane == 0) {
     for (int li = warp + 2 * W; tile_of(li) < n_tiles; li += W) {
@@ -551,7 +555,27 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
     }
     *reinterpret_cast<uint4*>(Qs + (size_t)r * STRIDE + c) = val;
   }
+  // the new K and V rows of this kv head, by the CTA whose tile they fall into (threads the query rows leave idle,
+  // where there are any): rotated, appended to the stream's cache, kept for the tile
+  if (fused && s_tile % DEC_SPLIT == rank) {
+    const int base = (16 * VPR) % (W * 32);                              // first thread without a query piece in the last pass
+    for (int i = (threadIdx.x - base + W * 32) % (W * 32); i < 2 * VPR; i += W * 32) {
+      const int which = i / VPR, c = (i % VPR) * 8;
+      const uint4 v8 = which == 0 ? head_piece_f16(prow + (size_t)(p.Hq + kh) * HD, c, HD, cs)
+                                  : head_piece_f16(prow + (size_t)(p.Hq + p.Hkv + kh) * HD, c, HD, nullptr);
+      *reinterpret_cast<uint4*>(&newkv[which][c]) = v8;
+      *reinterpret_cast<uint4*>((which == 0 ? ok : ov) + (size_t)S * HD + c) = v8;
+    }
+  }
   __syncthreads();
+  if (tile_of(warp) == s_tile || tile_of(warp + W) == s_tile) {
+    __half* kd = my_tiles + (size_t)(tile_of(warp) == s_tile ? 0 : 1) * 2 * DEC_KEYS * STRIDE;
+    const int r = S % DEC_KEYS;
+    if (lane < 2 * VPR) {
+      const int which = lane / VPR, c = (lane % VPR) * 8;
+      *reinterpret_cast<uint4*>(kd + (size_t)which * DEC_KEYS * STRIDE + (size_t)r * STRIDE + c) = *reinterpret_cast<const uint4*>(&newkv[which][c]);
+    }
+  }
   uint32_t qf[KSTEPS][4];
 #pragma unroll
   for (int ks = 0; ks < KSTEPS; ++ks) {
