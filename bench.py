@@ -31,10 +31,10 @@ GEN_STEPS = 128          # decode steps per generation (per stream) before the s
 ORACLE_PREFIX = 64       # prompt length used for the CPU-baseline sample (the 512-token prefill is not timed work)
 L2_BYTES = 126e6
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture) per launch of the dominant kernel, by
-# workload; None where no capture of the kernel as it stands exists.  cfg1: the 17 lean_gemm_kernel launches of a step
-# of a 4-layer cut of the model (the launches of a layer are the same at any depth): 4.10 MB q,k,v + 3.88 MB o +
-# 16.31 MB gate/up + 8.25 MB down = 32.54 MB per layer, 33.86 MB for the lm_head; (16 x 32.54 + 33.86) / 65 launches
-NCU_DRAM_BYTES_PER_LAUNCH = {"cfg1": 8.53e6}
+# workload; None where no capture of the kernel as it stands exists.  cfg1: the 132 lean_gemm_kernel launches of two
+# consecutive steps of the full model, one pass, caches not flushed between launches (every projection kernel asks for
+# the next one's weights in L2, so a capture that flushes counts them twice): 1105.7 MB read + 23 MB written
+NCU_DRAM_BYTES_PER_LAUNCH = {"cfg1": 8.55e6}
 
 
 def parse_args():
