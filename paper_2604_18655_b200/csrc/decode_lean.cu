@@ -343,6 +343,150 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
   }
 }
 
+// The lm_head (or any wide projection without adapters: EPI_F32, K of at most LM_PF k-tiles per warp) as a persistent
+// loop: a CTA takes the column tiles b, b + grid, b + 2 grid, ...; the input rows' fragments are fetched once and stay in
+// registers; the packed weights of the CTA's next LM_DEPTH tiles are always in flight (cp.async into a shared-memory
+// ring in which every thread owns the slots it copies into and reads back only those: no barrier); the cross-warp sums
+// go through two alternating buffers (one barrier per tile); in row-maxima mode every thread keeps the best key of its
+// (row, column of the tile) across its tiles: one atomic per row and CTA at the end.  2000 short-lived CTAs of the
+// one-tile kernel took 20 us for the 33 MB of a 32000 x 2048 lm_head (4.5 waves, each paying the trip to HBM).
+constexpr int LM_PF = 4;
+constexpr int LM_DEPTH = 4;
+constexpr size_t lm_smem_bytes(int threads) { return (size_t)LM_DEPTH * LM_PF * threads * (16 + 4); }
+template <int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, 2) lean_lmhead_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
+  constexpr int THREADS = WARPS * 32;
+  extern __shared__ __align__(16) unsigned char lm_dyn[];
+  uint4* const wring = reinterpret_cast<uint4*>(lm_dyn);                                  // [LM_DEPTH][LM_PF][THREADS]
+  uint32_t* const sring = reinterpret_cast<uint32_t*>(wring + (size_t)LM_DEPTH * LM_PF * THREADS);   // the same shape
+  __shared__ float red[2][WARPS][32][4];
+  __shared__ float s_inv[CHAIN_MAX_ROWS];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  pdl_launch_dependents();
+  const int M = a.M, K = ph.K;
+  const WLayout L = make_wlayout(K, ph.N, ph.G);
+  const int kt0 = (L.KT * warp) / WARPS, kt1 = (L.KT * (warp + 1)) / WARPS;   // at most LM_PF k-tiles (the launcher checks)
+  // this thread's pieces of a tile: offsets inside the tile's unit and slots inside a ring stage, fixed for the kernel
+  uint32_t woff[LM_PF], soff[LM_PF];
+#pragma unroll
+  for (int i = 0; i < LM_PF; ++i) {
+    const int kt = kt0 + i < kt1 ? kt0 + i : kt0;
+    woff[i] = (uint32_t)wl_tile_off(L, kt) + lane * 16;
+    soff[i] = (uint32_t)wl_scale_off(L, kt) + g * 4;
+  }
+  const uint32_t wslot = (uint32_t)__cvta_generic_to_shared(wring + threadIdx.x), sslot = (uint32_t)__cvta_generic_to_shared(sring + threadIdx.x);
+  // one cp.async group per tile (an empty one past the last tile, so that the group count stays in step)
+  auto issue = [&](int stage, int tile) {
+    if (tile < L.NT) {
+      const unsigned char* unit = ph.w + (size_t)tile * L.unit_bytes;
+#pragma unroll
+      for (int i = 0; i < LM_PF; ++i) {
+        if (kt0 + i < kt1) {
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(wslot + (uint32_t)((stage * LM_PF + i) * THREADS * 16)), "l"(unit + woff[i]) : "memory");
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sslot + (uint32_t)((stage * LM_PF + i) * THREADS * 4)), "l"(unit + soff[i]) : "memory");
+        }
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  int tile = blockIdx.x;
+#pragma unroll
+  for (int d = 0; d < LM_DEPTH; ++d) issue(d, tile + d * (int)gridDim.x);
+  if (threadIdx.x == 32 && ph.pf_bytes != 0) {               // the next projection group's weights, a share per CTA
+    const unsigned long long per = ((ph.pf_bytes / gridDim.x) + 15ull) & ~15ull;
+    const unsigned long long b0 = per * blockIdx.x, b1 = b0 + per < ph.pf_bytes ? b0 + per : (ph.pf_bytes & ~15ull);
+    for (unsigned long long o = b0; o < b1; o += 16384ull) {
+      const uint32_t n = (uint32_t)(b1 - o < 16384ull ? b1 - o : 16384ull);
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(ph.pf_w + o), "r"(n) : "memory");
+    }
+  }
+  pdl_wait();
+  if (threadIdx.x < CHAIN_MAX_ROWS) {
+    float inv = 1.f;
+    if (ph.norm_in >= 0 && threadIdx.x < M)
+      inv = rsqrtf(ln_unfix(__ldcg(a.ssq + (size_t)ph.norm_in * CHAIN_MAX_ROWS + threadIdx.x)) / (float)K + a.eps);
+    s_inv[threadIdx.x] = inv;
+  }
+  uint4 x0[LM_PF], x1[LM_PF];
+  {
+    const __half* xrow = ph.in16 + (size_t)g * K + 16 * t;
+#pragma unroll
+    for (int i = 0; i < LM_PF; ++i) {
+      const int kt = kt0 + i;
+      if (kt < kt1 && g < M) {
+        x0[i] = *(reinterpret_cast<const uint4*>(xrow + (size_t)kt * TILE_K));
+        x1[i] = *(reinterpret_cast<const uint4*>(xrow + (size_t)kt * TILE_K) + 1);
+      } else {
+        x0[i] = make_uint4(0, 0, 0, 0);
+        x1[i] = make_uint4(0, 0, 0, 0);
+      }
+    }
+  }
+  __syncthreads();                                            // s_inv
+  const bool maxima = ph.out_f32 == nullptr && a.amax != nullptr;
+  float* const out = ph.out_f32 != nullptr ? ph.out_f32 : a.logits;
+  // this thread's (row, column of the tile) in the epilogue, and where that sum sits in the warps' accumulators
+  const int em = (threadIdx.x >> 4) & 7, ec = threadIdx.x & 15;
+  const int src_lane = (ec & 7) * 4 + (em >> 1), e = (ec >> 3) * 2 + (em & 1);
+  const float inv_m = s_inv[em];
+  unsigned long long best = 0ull;
+  int par = 0, stage = 0;
+#pragma unroll 1
+  for (; tile < L.NT; tile += gridDim.x) {
+    asm volatile("cp.async.wait_group %0;" ::"n"(LM_DEPTH - 1) : "memory");   // this thread's pieces of the oldest tile are there
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < LM_PF; ++i) {
+      if (kt0 + i < kt1) {
+        const uint4 wv = wring[((size_t)stage * LM_PF + i) * THREADS + threadIdx.x];
+        const uint32_t sv = sring[((size_t)stage * LM_PF + i) * THREADS + threadIdx.x];
+        __half2 s_lo, s_hi;
+        split_scales(sv, s_lo, s_hi);
+        uint32_t af[4][4];
+        dequant8(wv.x, s_lo, s_hi, af[0]);
+        dequant8(wv.y, s_lo, s_hi, af[1]);
+        dequant8(wv.z, s_lo, s_hi, af[2]);
+        dequant8(wv.w, s_lo, s_hi, af[3]);
+        mma_16816(acc, af[0], x0[i].x, x0[i].y);
+        mma_16816(acc, af[1], x0[i].z, x0[i].w);
+        mma_16816(acc, af[2], x1[i].x, x1[i].y);
+        mma_16816(acc, af[3], x1[i].z, x1[i].w);
+      }
+    }
+    issue(stage, tile + LM_DEPTH * (int)gridDim.x);          // refills the slots just read (this thread's own)
+    stage = stage + 1 == LM_DEPTH ? 0 : stage + 1;
+    *reinterpret_cast<float4*>(red[par][warp][lane]) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    __syncthreads();
+    if (threadIdx.x < 128 && em < M) {
+      float y = 0.f;
+#pragma unroll
+      for (int w = 0; w < WARPS; ++w) y += red[par][w][src_lane][e];
+      y *= inv_m;
+      const int col = tile * TILE_N + ec;
+      if (maxima) {
+        if (y == 0.f) y = 0.f;
+        const unsigned b = __float_as_uint(y);
+        const unsigned ord = (y != y) ? 0u : ((b & 0x80000000u) ? ~b : (b | 0x80000000u));
+        const unsigned long long key = ((unsigned long long)ord << 32) | (unsigned)(0xffffffffu - (unsigned)col);
+        best = key > best ? key : best;
+      } else {
+        out[(size_t)em * ph.ldo + col] = y;
+      }
+    }
+    par ^= 1;
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  if (maxima && threadIdx.x < 128) {
+    // the best key of a row: over its 16 columns' threads (half a warp), then one atomic per row and CTA
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) {
+      const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+      best = other > best ? other : best;
+    }
+    if (ec == 0 && em < M && best > __ldcg(a.amax + em)) atomicMax(a.amax + em, best);
+  }
+}
+
 // Embedding (or hidden-state input) of the step's rows: residual fp32, x * gain of the first norm as fp16, the rows'
 // sums of squares, and the shrink sums of the first q,k,v group.  CTA (m, part): row m; part 0 also writes the row.
 __global__ void __launch_bounds__(LN_THREADS) lean_embed_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph,
@@ -483,6 +627,8 @@ cudaError_t init_lean() {
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(lean_gemm_kernel<1, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
   if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(lean_lmhead_kernel<LN_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lm_smem_bytes(LN_THREADS));
+  if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(lean_gemm_kernel<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
 }
 
@@ -501,6 +647,15 @@ cudaError_t launch_lean_gemm(const LeanArgs& a, const StepPhase& ph, cudaStream_
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  // wide projections without adapters (the lm_head): persistent CTAs, two per SM, that loop over the column tiles
+  static const int sms = [] { int d = 0, n = 0; cudaGetDevice(&d); cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, d); return n; }();
+  if (mode == MODE_PLAIN && ph.epi == EPI_F32 && ph.lora_nseg == 0 && tiles >= 4 * sms && sms > 0 &&
+      (ph.K / TILE_K + LN_WARPS - 1) / LN_WARPS <= LM_PF) {
+    cfg.gridDim = dim3((unsigned)(2 * sms < tiles ? 2 * sms : tiles));
+    cfg.blockDim = dim3(LN_THREADS);
+    cfg.dynamicSmemBytes = lm_smem_bytes(LN_THREADS);
+    return cudaLaunchKernelEx(&cfg, lean_lmhead_kernel<LN_WARPS>, a, ph);
+  }
   if (mode == MODE_GATEUP) return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<2, 8>, a, ph);
   if (wide) return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<1, 16>, a, ph);
   return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<1, 8>, a, ph);
