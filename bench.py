@@ -9,7 +9,7 @@ decoding in generations of 128 steps per stream.  One "step" = one mlora_decode_
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
   python bench.py --config cfg2|cfg3        DS2D verify rounds (8 streams x 16- or 32-node trees), same line shape
   python bench.py --config cfg4 [--quick]   kernel-level sweep of the single projection and of tree attention
-  python bench.py --timeline                phase timeline of the single-kernel decode step (markdown)
+  python bench.py --timeline                timelines of a traced decode step: default path and single-kernel step (markdown)
 
 With N > 1 (torchrun) every rank runs an independent replica of the same job: the path has no exchange
 step, so there is no collective on the data path ("replicas only").
@@ -678,6 +678,31 @@ def print_timeline(tl, cfg, sm_mhz):
     print(f"\nstep (global timer, first CTA): {(tl[0][-1][11] - tl[0][0][11]) / 1e3:.1f} us")
 
 
+def print_timeline_lean(tl, cfg):
+    """Markdown table of one traced decode step of the kernel-per-projection path: global-timer stamps per launch,
+    microseconds after the latest end of the launch before it, averaged over the layers (first layer left out)."""
+    kinds = ["embed"] + ["qkv", "attention", "o", "gate_up", "down"] * cfg.n_layers + (["lm_head"] if cfg.vocab else []) + ["end"]
+    agg, prev_end = {}, None
+    for p, k in enumerate(kinds):
+        a, b = tl[0][p], tl[1][p]
+        if a[0] == 0:
+            continue
+        end = int(a[4])
+        if prev_end is not None and p > 6:
+            rel = lambda v: (int(v) - prev_end) / 1e3 if v else float("nan")
+            agg.setdefault(k, []).append([rel(a[0]), rel(a[1]), rel(a[2]), rel(a[3]), rel(b[0]), rel(b[1]), rel(b[3]), rel(end)])
+        prev_end = end
+    print("| kernel | n | first CTA: start | wait returned | main loop done | end | last CTA: start | wait returned | end | latest end of all CTAs |")
+    print("|---|---|---|---|---|---|---|---|---|---|")
+    for k, rows in agg.items():
+        m = np.nanmean(np.array(rows, dtype=np.float64), axis=0)
+        print(f"| {k} | {len(rows)} | " + " | ".join("-" if np.isnan(v) else f"{v:.2f}" for v in m) + " |")
+    ends = [int(tl[0][p][4]) for p in range(len(kinds)) if tl[0][p][0]]
+    starts = [int(tl[0][p][1]) for p in range(len(kinds)) if tl[0][p][0]]
+    print(f"\n(us after the latest end of the launch before; first projection's wait returned -> last launch's end: "
+          f"{(max(ends) - min(starts)) / 1e3:.1f} us; the traced kernels run a few per cent slower than the untraced ones)")
+
+
 def workload_name(cfg):
     what = (f"{cfg.tree_nodes}-node draft trees {cfg.branch}, one verify pass per step" if cfg.tree_nodes > 1
             else f"{GEN_STEPS} greedy decode steps per generation")
@@ -779,6 +804,15 @@ def main():
         for i in range(W):
             generation_step(i)
         if args.timeline:
+            # the default path (one kernel per projection group) first: global-timer stamps of a traced step
+            mb.mlora_debug_set(ctx, 6, 0)
+            mb.mlora_debug_set(ctx, 7, 1)
+            for i in range(3):
+                generation_step(W + i)
+            side.synchronize()
+            print("## kernel-per-projection path (default)\n")
+            print_timeline_lean(mb.mlora_step_timeline(ctx), cfg)
+            print("\n## single-kernel step\n")
             mb.mlora_debug_set(ctx, 6, 2)
             mb.mlora_debug_set(ctx, 7, 1)
             generation_step(W)

@@ -204,7 +204,8 @@ int mlora_debug_dequant(mlora_ctx* ctx, int32_t layer, int32_t proj, void* out_f
  *         programmatically so that each one's weights are in flight while the one before it drains (contexts up to
  *         2047 keys; longer ones take the per-layer path); 0 = the library's choice (3 where it applies: the fastest of
  *         the three at the 1B / 8-stream shapes).  All are replayed from CUDA graphs.
- * key 7 = 1 makes the single-kernel decode step record a timeline (see mlora_step_timeline). */
+ * key 7 = 1 makes decode steps of paths 2 and 3 (key 6) record a timeline (see mlora_step_timeline); path 3 then runs
+ *         instantiations of its kernels that carry the stamps (the untraced ones carry none). */
 int mlora_debug_set(mlora_ctx* ctx, int32_t key, int32_t value);
 /* Timeline of the LAST decode step that ran with debug key 7 set (Sec. 3.1 decoder: the step's phases are the
  * embedding, then q,k,v projection / attention / o projection / gate,up projection / down projection per layer,
@@ -214,7 +215,12 @@ int mlora_debug_set(mlora_ctx* ctx, int32_t key, int32_t value);
  * multiplied, 10 all tiles of the first batch multiplied, 1 main loop (attention: the row's q,k,v in shared memory) done, 2 partial sums parked (attention: all
  * key tiles done), 3 epilogue done, 4 phase work done, 5 CTA at the grid barrier, 6 barrier passed; 0 where a point
  * does not apply.  Slot 11 of the first phase / of the last phase holds the GPU's global nanosecond timer at the
- * step's start / end.  capacity = values host_out holds (>= 24 * n_phases); *n_phases receives the phase count.
+ * step's start / end.
+ * Path 3 (one kernel per projection group; the embedding and closing phases are not stamped): every slot is a reading of
+ * the GPU's GLOBAL nanosecond timer, comparable across CTAs and kernels: 0 kernel start, 1 its wait for the kernel ahead
+ * returned, 2 main loop (attention: key tiles) done, 3 end, for thread 0 of the launch's first CTA (index 0) and of its
+ * last CTA (index 1; not for attention); slot 4 of index 0 = the latest end over ALL CTAs of the launch.
+ * capacity = values host_out holds (>= 24 * n_phases); *n_phases receives the phase count.
  * Synchronises.  Errors: ARG, STATE, CAPACITY, CUDA. */
 int mlora_step_timeline(mlora_ctx* ctx, int64_t* host_out, int32_t capacity, int32_t* n_phases);
 /* Per-kernel-family device time of the NEXT steps, measured with CUDA events on the context's stream.

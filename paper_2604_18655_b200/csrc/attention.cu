@@ -418,11 +418,25 @@ __host__ __device__ constexpr size_t dec_smem_bytes(int hd) {
          (size_t)dec_warps(hd) * 16 * (hd + 2) * 4 + (size_t)16 * (hd + 2) * 4 + (size_t)2 * hd * 2;
 }
 
-template <int HD>
+// (TRACE: the instantiation that stamps a traced step's timeline -- thread 0 of the first CTA writes the GPU's global
+// nanosecond timer to slots 0 start, 1 wait returned, 2 key tiles done, 3 end of its launch's row; every CTA's thread 0
+// raises slot 4 to its own end)
+__device__ __forceinline__ long long attn_now() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+template <bool TRACE>
+__device__ __forceinline__ void attn_stamp(const AttnArgs& p, int slot) {
+  if constexpr (TRACE) {
+    if (threadIdx.x == 0) {
+      if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) p.trace0[slot] = attn_now();
+      if (slot == 3) atomicMax(reinterpret_cast<unsigned long long*>(p.trace0 + 4), (unsigned long long)attn_now());
+    }
+  }
+}
+template <int HD, bool TRACE>
 __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const AttnArgs p, const float scale_log2) {
   constexpr int W = dec_warps(HD), STRIDE = HD + 8, KSTEPS = HD / 16, DT = HD / 8, VPR = HD / 8;
   // (programmatic launches around this kernel: the kernel after it may start its own independent loads now; nothing
   // here is read before the kernel ahead has finished -- both are no-ops in ordinary launches)
+  attn_stamp<TRACE>(p, 0);
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // first phase of the cluster barrier: "this CTA runs" (waited for before the peer's shared memory is written)
   asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
@@ -523,6 +537,7 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
       asm volatile("prefetch.global.L1 [%0];" ::"l"(reinterpret_cast<const char*>(cs) + threadIdx.x * 128) : "memory");
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  attn_stamp<TRACE>(p, 1);
   own_keys = S + 1;                                                       // cached rows + this pass's row
   n_tiles = n_ptiles + (own_keys + DEC_KEYS - 1) / DEC_KEYS;
   if (fused && p.depth != nullptr) cs = p.cs_table + (size_t)(p.pos_base + S + p.depth[m]) * (HD / 2);
@@ -665,6 +680,7 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
     if (tile_of(li + 2 * W) < n_tiles) load_tile(tile_of(li + 2 * W), buf);
   }
 
+  attn_stamp<TRACE>(p, 2);
   // this warp's un-normalised output, running max (log2 domain) and sum for the group's rows
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
@@ -760,6 +776,7 @@ __global__ void __launch_bounds__(dec_warps(HD) * 32) attn_decode_kernel(const A
       }
     }
   }
+  attn_stamp<TRACE>(p, 3);
 }
 
 
@@ -1192,9 +1209,13 @@ cudaError_t init_attention() {
                                        (int)((ATT_ROWS + 4 * ATT_KEYS) * (64 + 8) * sizeof(__half)));
   if (e != cudaSuccess) return e;
   // (+ room for the o adapter's rows over a kv head's features, up to the limit of a CTA)
-  e = cudaFuncSetAttribute(attn_decode_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  e = cudaFuncSetAttribute(attn_decode_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(attn_decode_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  e = cudaFuncSetAttribute(attn_decode_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attn_decode_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attn_decode_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(attn_stream_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)str_smem_bytes(64));
   if (e != cudaSuccess) return e;
@@ -1265,8 +1286,12 @@ cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st) {
     attr[1].val.programmaticStreamSerializationAllowed = 1;            // the kernel ahead of it drains
     cfg.attrs = attr;
     cfg.numAttrs = a.pdl ? 2 : 1;
-    if (a.hd == 64) return cudaLaunchKernelEx(&cfg, attn_decode_kernel<64>, a, scale_log2);
-    return cudaLaunchKernelEx(&cfg, attn_decode_kernel<128>, a, scale_log2);
+    if (a.trace0 != nullptr) {                              // (the instantiations that stamp the step's timeline)
+      if (a.hd == 64) return cudaLaunchKernelEx(&cfg, attn_decode_kernel<64, true>, a, scale_log2);
+      return cudaLaunchKernelEx(&cfg, attn_decode_kernel<128, true>, a, scale_log2);
+    }
+    if (a.hd == 64) return cudaLaunchKernelEx(&cfg, attn_decode_kernel<64, false>, a, scale_log2);
+    return cudaLaunchKernelEx(&cfg, attn_decode_kernel<128, false>, a, scale_log2);
   }
   if (a.hd == 64) return launch_attn_hd<64>(a, st);
   if (a.hd == 128) return launch_attn_hd<128>(a, st);

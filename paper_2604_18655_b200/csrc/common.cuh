@@ -151,6 +151,7 @@ struct AttnArgs {
   const __half* const* o_tabA;    // adapter A pointers [slot][o_tab_stride]
   const int32_t* o_adapter_idx;   // dev [n]
   int o_proj_index, o_rank, o_tab_stride, o_n_slots;
+  long long* trace0;              // timeline of a traced step (nullptr otherwise): this launch's 12 slots
   int o_direct;                   // o_tabA is indexed by stream (looked up once per call): o_adapter_idx is not read
   int pdl;                        // launch the single-kernel decode attention with programmatic stream serialisation
 };
@@ -342,6 +343,8 @@ struct LeanArgs {
   float* logits;                  // destination of a phase whose out_f32 is null
   unsigned long long* tacc;       // [n_tacc][8][3][rank]
   unsigned long long* ssq;        // [n_ssq][8]
+  long long* trace0;              // timeline of a traced step (nullptr otherwise): 12 slots of this launch for its first CTA
+  long long* trace1;              // ... and for its last CTA
   int rank_log2;                  // log2(rank) when the rank is a power of two, else -1 (index arithmetic by shifts)
   int rows_direct;                // tabA / tabB / scale are indexed by ROW (looked up once per call): adapter_idx is not read
   int late_wait;                  // the kernel ahead produces only T: wait for it after the main loop, not before

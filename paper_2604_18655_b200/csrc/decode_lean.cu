@@ -108,10 +108,26 @@ __device__ __forceinline__ void lean_shrink_partial(const LeanArgs& a, const Ste
 // NTILE = 1: 16 physical columns per CTA; NTILE = 2: a gate tile and its up tile (SwiGLU pair)
 // Launched with programmatic stream serialisation: everything ahead of pdl_wait() -- the first weights, the adapter
 // slices -- depends on no earlier kernel and is in flight while the kernel before this one finishes.
+// Timeline of a traced step (the TRACE instantiations of the kernels; the others carry none of it): thread 0 of the
+// first and of the last CTA stamp the GPU's global nanosecond timer into their launch's slots -- 0 start, 1 wait
+// returned, 2 main loop done, 3 end -- and every CTA's thread 0 raises slot 4 of the first CTA's row to its own end.
+__device__ __forceinline__ long long ln_now() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+template <bool TRACE>
+__device__ __forceinline__ void ln_stamp(const LeanArgs& a, int slot) {
+  if constexpr (TRACE) {
+    if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1)) {
+      const long long now = ln_now();
+      if (blockIdx.x == 0) a.trace0[slot] = now;
+      if (blockIdx.x == gridDim.x - 1) a.trace1[slot] = now;
+    }
+    if (slot == 3 && threadIdx.x == 0) atomicMax(reinterpret_cast<unsigned long long*>(a.trace0 + 4), (unsigned long long)ln_now());
+  }
+}
+
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-template <int NTILE, int WARPS>
+template <int NTILE, int WARPS, bool TRACE>
 __global__ void __launch_bounds__(WARPS * 32, WARPS == 8 ? 3 : 1)
 lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
   constexpr int THREADS = WARPS * 32;
@@ -123,6 +139,7 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
   __shared__ float s_sq[CHAIN_MAX_ROWS][16];
   extern __shared__ __align__(16) unsigned char ln_dyn[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  ln_stamp<TRACE>(a, 0);
   pdl_launch_dependents();
   const int M = a.M, K = ph.K, r = a.rank;
   const WLayout L = make_wlayout(K, ph.N, ph.G);
@@ -165,6 +182,7 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
   }
   lean_prefetch_slices<NTILE>(a, ph, tile0, n_out0, lora, sB, sA);
   pdl_wait();
+  ln_stamp<TRACE>(a, 1);
   // ---- what earlier kernels produced: the old residual, norm factors, T of this group, the input rows
   float x_old = 0.f, gain_nx = 1.f;
   if (ph.epi == EPI_RESID && threadIdx.x < 128 && (threadIdx.x >> 4) < M) {
@@ -238,6 +256,7 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
     pdl_wait();
     if (lora) load_T();
   }
+  ln_stamp<TRACE>(a, 2);
 #pragma unroll
   for (int u = 0; u < NTILE; ++u)
     *reinterpret_cast<float4*>(red[warp][u][lane]) = make_float4(acc[u][0], acc[u][1], acc[u][2], acc[u][3]);
@@ -288,6 +307,7 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
         }
       if (best > __ldcg(a.amax + m)) atomicMax(a.amax + m, best);
     }
+    ln_stamp<TRACE>(a, 3);
     return;
   }
   if (ph.epi == EPI_F32) {
@@ -296,6 +316,7 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
       const int u = o >> 7, m = (o >> 4) & 7, c = o & 15;
       if (m < M) out[(size_t)m * ph.ldo + (tile0 + u) * TILE_N + c] = s_y[u][m][c];
     }
+    ln_stamp<TRACE>(a, 3);
     return;
   }
   if (ph.epi == EPI_RESID) {
@@ -323,6 +344,7 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
       ln_red_add(a.ssq + (size_t)ph.ssq_out * CHAIN_MAX_ROWS + threadIdx.x, ln_fix(sq));
     }
     lean_shrink_partial(a, ph, s_vals, sA);
+    ln_stamp<TRACE>(a, 3);
     return;
   }
   // EPI_SWIGLU: tile0 is the gate tile, tile0 + 1 the up tile of 16 features
@@ -341,6 +363,7 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
     __syncthreads();
     lean_shrink_partial(a, ph, s_vals, sA);
   }
+  ln_stamp<TRACE>(a, 3);
 }
 
 // The lm_head (or any wide projection without adapters: EPI_F32, K of at most LM_PF k-tiles per warp) as a persistent
@@ -353,7 +376,7 @@ lean_gemm_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
 constexpr int LM_PF = 4;
 constexpr int LM_DEPTH = 4;
 constexpr size_t lm_smem_bytes(int threads) { return (size_t)LM_DEPTH * LM_PF * threads * (16 + 4); }
-template <int WARPS>
+template <int WARPS, bool TRACE>
 __global__ void __launch_bounds__(WARPS * 32, 2) lean_lmhead_kernel(const LeanArgs a, const __grid_constant__ StepPhase ph) {
   constexpr int THREADS = WARPS * 32;
   extern __shared__ __align__(16) unsigned char lm_dyn[];
@@ -362,6 +385,7 @@ __global__ void __launch_bounds__(WARPS * 32, 2) lean_lmhead_kernel(const LeanAr
   __shared__ float red[2][WARPS][32][4];
   __shared__ float s_inv[CHAIN_MAX_ROWS];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  ln_stamp<TRACE>(a, 0);
   pdl_launch_dependents();
   const int M = a.M, K = ph.K;
   const WLayout L = make_wlayout(K, ph.N, ph.G);
@@ -401,6 +425,7 @@ __global__ void __launch_bounds__(WARPS * 32, 2) lean_lmhead_kernel(const LeanAr
     }
   }
   pdl_wait();
+  ln_stamp<TRACE>(a, 1);
   if (threadIdx.x < CHAIN_MAX_ROWS) {
     float inv = 1.f;
     if (ph.norm_in >= 0 && threadIdx.x < M)
@@ -476,6 +501,7 @@ __global__ void __launch_bounds__(WARPS * 32, 2) lean_lmhead_kernel(const LeanAr
     par ^= 1;
   }
   asm volatile("cp.async.wait_group 0;" ::: "memory");
+  ln_stamp<TRACE>(a, 2);
   if (maxima && threadIdx.x < 128) {
     // the best key of a row: over its 16 columns' threads (half a warp), then one atomic per row and CTA
 #pragma unroll
@@ -485,6 +511,7 @@ __global__ void __launch_bounds__(WARPS * 32, 2) lean_lmhead_kernel(const LeanAr
     }
     if (ec == 0 && em < M && best > __ldcg(a.amax + em)) atomicMax(a.amax + em, best);
   }
+  ln_stamp<TRACE>(a, 3);
 }
 
 // Embedding (or hidden-state input) of the step's rows: residual fp32, x * gain of the first norm as fp16, the rows'
@@ -621,18 +648,24 @@ cudaError_t launch_lean_embed(const LeanArgs& a, const StepPhase& ph, const int3
   return cudaGetLastError();
 }
 
-cudaError_t init_lean() {
+template <bool TRACE>
+static cudaError_t init_lean_variant() {
   // room for the adapter slices at rank 64: 5 x 16 KB
-  cudaError_t e = cudaFuncSetAttribute(lean_gemm_kernel<1, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(lean_gemm_kernel<1, 8, TRACE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(lean_gemm_kernel<1, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
+  e = cudaFuncSetAttribute(lean_gemm_kernel<1, 16, TRACE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(lean_lmhead_kernel<LN_WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lm_smem_bytes(LN_THREADS));
+  e = cudaFuncSetAttribute(lean_lmhead_kernel<LN_WARPS, TRACE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lm_smem_bytes(LN_THREADS));
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(lean_gemm_kernel<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
+  return cudaFuncSetAttribute(lean_gemm_kernel<2, 8, TRACE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
+}
+cudaError_t init_lean() {
+  const cudaError_t e = init_lean_variant<false>();
+  return e != cudaSuccess ? e : init_lean_variant<true>();
 }
 
-cudaError_t launch_lean_gemm(const LeanArgs& a, const StepPhase& ph, cudaStream_t st) {
+template <bool TRACE>
+static cudaError_t launch_lean_gemm_variant(const LeanArgs& a, const StepPhase& ph, cudaStream_t st) {
   const int tiles = ph.N / TILE_N, mode = ph.mode;
   // B slices of up to two tiles and A slices of up to three consuming segments, 8 rows x rank x 16 columns each
   const size_t slice = (size_t)CHAIN_MAX_ROWS * (a.rank > 0 ? a.rank : 1) * 16 * sizeof(__half);
@@ -654,11 +687,16 @@ cudaError_t launch_lean_gemm(const LeanArgs& a, const StepPhase& ph, cudaStream_
     cfg.gridDim = dim3((unsigned)(2 * sms < tiles ? 2 * sms : tiles));
     cfg.blockDim = dim3(LN_THREADS);
     cfg.dynamicSmemBytes = lm_smem_bytes(LN_THREADS);
-    return cudaLaunchKernelEx(&cfg, lean_lmhead_kernel<LN_WARPS>, a, ph);
+    return cudaLaunchKernelEx(&cfg, lean_lmhead_kernel<LN_WARPS, TRACE>, a, ph);
   }
-  if (mode == MODE_GATEUP) return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<2, 8>, a, ph);
-  if (wide) return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<1, 16>, a, ph);
-  return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<1, 8>, a, ph);
+  if (mode == MODE_GATEUP) return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<2, 8, TRACE>, a, ph);
+  if (wide) return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<1, 16, TRACE>, a, ph);
+  return cudaLaunchKernelEx(&cfg, lean_gemm_kernel<1, 8, TRACE>, a, ph);
+}
+
+// (a.trace0 set: the instantiations that stamp the step's timeline)
+cudaError_t launch_lean_gemm(const LeanArgs& a, const StepPhase& ph, cudaStream_t st) {
+  return a.trace0 != nullptr ? launch_lean_gemm_variant<true>(a, ph, st) : launch_lean_gemm_variant<false>(a, ph, st);
 }
 
 }  // namespace mlora

@@ -403,8 +403,14 @@ int forward_lean(mlora_ctx* c, PassIO& io) {
   a.X = c->X; a.logits = io.logits; a.tacc = c->step_tacc; a.ssq = c->step_ssq;
   const bool fused = io.fused_next != nullptr && d.vocab > 0;
   if (fused) { a.logits = nullptr; a.amax = c->step_ssq + (size_t)c->n_ssq * CHAIN_MAX_ROWS; }
+  const bool trace = c->dbg_trace && c->step_trace != nullptr;
+  if (trace) CK(cudaMemsetAsync(c->step_trace, 0, (size_t)c->n_step_phases * 2 * 12 * sizeof(long long), st));
   for (size_t p = 0; p < c->step_phases_host.size(); ++p) {
     const StepPhase& ph = c->step_phases_host[p];
+    if (trace) {                                       // this launch's rows of the timeline: first CTA, last CTA
+      a.trace0 = c->step_trace + p * 12;
+      a.trace1 = c->step_trace + ((size_t)c->n_step_phases + p) * 12;
+    }
     if (ph.kind == SK_EMBED) {
       CK(run(c, MLORA_PROF_MISC, [&] {
         return launch_lean_embed(a, ph, io.tokens, (const __half*)d.embed, d.vocab, io.hidden_in, c->status, st);
@@ -423,6 +429,7 @@ int forward_lean(mlora_ctx* c, PassIO& io) {
       at.own_stream_stride = c->own_stream_stride; at.own_head_stride = c->own_head_stride;
       at.suffix_len = io.suffix_len; at.anc = c->anc; at.causal = 0; at.out = c->attn16; at.status = c->status;
       at.pdl = 1;
+      at.trace0 = trace ? c->step_trace + p * 12 : nullptr;
       if (lora && ph.next_nseg > 0) {
         at.o_tacc = c->step_tacc + (size_t)ph.t_out * CHAIN_MAX_ROWS * 3 * a.rank;
         at.o_tabA = c->step_rowA; at.o_adapter_idx = io.adapter_idx; at.o_direct = 1; at.o_proj_index = ph.next_proj[0]; at.o_rank = a.rank;
@@ -1104,7 +1111,7 @@ static int decode_impl(mlora_ctx* c, int n, const int32_t* adapter_idx, const in
   key.kind = hidden ? 2 : 1; key.n = n; key.T = 1;
   key.prefix_chunk = io.plan.prefix_chunk; key.n_prefix_chunks = io.plan.n_prefix_chunks;
   key.own_chunk = io.plan.own_chunk; key.n_own_chunks = io.plan.n_own_chunks;
-  key.flags = (c->P * 4 + c->dbg_inject_stall * 2 + c->dbg_no_chain) * 4 + c->step_mode;
+  key.flags = ((c->P * 4 + c->dbg_inject_stall * 2 + c->dbg_no_chain) * 4 + c->step_mode) * 2 + c->dbg_trace;
   key.suffix_bound = io.plan.suffix_bound;     // (rounded up by plan_pass: the kernels' launch shape and prefetch extents)
   key.p[0] = adapter_idx; key.p[1] = tokens; key.p[2] = hidden; key.p[3] = out_next; key.p[4] = out_logits; key.p[5] = hidden_out;
   rc = replay_or_run(c, key, [&]() -> int {
@@ -1170,7 +1177,7 @@ static int generate_impl(mlora_ctx* c, int n, const int32_t* adapter_idx, const 
   const int bound0 = c->suffix_bound;
   GraphKey key{};
   key.kind = 4; key.n = n; key.T = k;
-  key.flags = c->P * 16 + c->step_mode * 4 + c->dbg_inject_stall * 2 + c->dbg_no_chain;
+  key.flags = (c->P * 16 + c->step_mode * 4 + c->dbg_inject_stall * 2 + c->dbg_no_chain) * 2 + c->dbg_trace;
   key.suffix_bound = bound0;                           // every step's launch shapes follow from the bound at the start
   key.p[0] = adapter_idx; key.p[1] = first; key.p[2] = out;
   rc = replay_or_run(c, key, [&]() -> int {

@@ -367,6 +367,38 @@ def test_step_kernel_is_one_launch_and_bit_reproducible(GpuModel):
     assert np.array_equal(res[0].view(np.uint32), res[1].view(np.uint32))
 
 
+def test_step_timeline_of_the_default_decode_path(GpuModel):
+    """Debug switch 7 on the kernel-per-projection path: the traced instantiations give the same tokens and logits as
+    the untraced kernels, and every stamped launch reads start <= wait returned <= main loop done <= end <= latest end
+    of all its CTAs, the launches in step order."""
+    from paper_2604_18655_b200 import binding as mb
+    cfg = TINYV
+    res = []
+    for trace in (0, 1):
+        m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+        mb.mlora_debug_set(gm.ctx, 6, 3)
+        mb.mlora_debug_set(gm.ctx, 7, trace)
+        gm.prefill(gen.make_prompt_ids(cfg, 0))
+        toks = np.array([1, 2, 3], dtype=np.int32)
+        hist = []
+        for _ in range(3):
+            toks, logits = gm.decode([0, 1, -1], toks)
+            hist.append(logits)
+        res.append(np.stack(hist))
+        if trace:
+            tl = mb.mlora_step_timeline(gm.ctx)
+            rows = [r for r in tl[0] if r[0]]
+            assert len(rows) >= 5 * cfg.n_layers                  # q,k,v / attention / o / gate,up / down per layer (+ lm_head)
+            prev = 0
+            for r in rows:
+                assert r[0] <= r[1] <= r[2] <= r[3] <= r[4], r
+                assert r[4] >= prev                                   # a launch ends after the one before it
+                prev = r[4]
+        mb.mlora_sync_status(gm.ctx)
+        gm.close()
+    assert np.array_equal(res[0].view(np.uint32), res[1].view(np.uint32))
+
+
 def test_decode_paths_agree(GpuModel):
     """The single-kernel step against the per-layer persistent projection kernel (debug switch 6) and the
     one-kernel-per-projection form of the same arithmetic (debug switch 3): logits and KV within the parity tolerance."""
