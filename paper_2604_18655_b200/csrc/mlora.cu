@@ -33,6 +33,7 @@ void free_packed(PackedWeight& w) {
   w.data = nullptr;
 }
 
+constexpr int PREFILL_ROWS = 1024;                 // rows of one causal prefill pass
 constexpr int MAX_FORECAST = 8, MAX_DRAFT_WIDTH = 32;
 
 struct GraphKey {
@@ -196,6 +197,8 @@ struct PassIO {
   int32_t* fused_next = nullptr;           // decode passes that want no logits: greedy tokens straight from the lm_head,
                                            // suffix lengths advanced (set by forward when its path did both)
   bool fused_done = false;
+  bool last_row_logits = false;            // prefill: only the pass's last row goes through the final norm and lm_head
+                                           // (io.logits receives that one row)
   bool rows_resolved = false;              // the rows' adapter pointers were looked up earlier in this call (same adapter_idx)
   AttnArgs plan;                           // chunking, filled by plan_pass
 };
@@ -524,12 +527,13 @@ int forward(mlora_ctx* c, PassIO& io) {
     }
   }
   if (d.vocab > 0 && io.logits != nullptr) {
+    const int Ml = io.last_row_logits ? 1 : M;           // rows that get logits: the last Ml of the pass
     ShrinkArgs s{};
-    s.x_f32 = c->X; s.gain = (const __half*)d.rms_final; s.eps = d.rms_eps; s.h_out = c->h; s.M = M; s.K = dm;
+    s.x_f32 = c->X + (size_t)(M - Ml) * dm; s.gain = (const __half*)d.rms_final; s.eps = d.rms_eps; s.h_out = c->h; s.M = Ml; s.K = dm;
     CK(run(c, MLORA_PROF_SHRINK, [&] { return launch_shrink(s, st); }));
     GemmArgs g{};
     const PackedWeight& w = c->w_lm;
-    g.w = w.data; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->h; g.M = M;
+    g.w = w.data; g.K = w.K; g.N = w.N; g.G = w.G; g.h = c->h; g.M = Ml;
     g.mode = MODE_PLAIN; g.epi = EPI_F32; g.out_f32 = io.logits; g.ldo = d.vocab;
     g.partial = c->partial; g.partial_capacity = c->partial_floats; g.counters = c->counters;
     CK(run(c, MLORA_PROF_GEMM, [&] { return launch_projection(c, g, st); }));
@@ -619,8 +623,9 @@ int check_ctx(mlora_ctx* c) { return c ? MLORA_OK : fail(MLORA_ERR_ARG, "null co
 int prefill_impl(mlora_ctx* c, const int32_t* ids, const __half* hidden, int n, float* out_last) {
   if (n <= 0) return fail(MLORA_ERR_ARG, "prefill needs at least one position");
   if (n > c->d.max_prefix) return fail(MLORA_ERR_CAPACITY, "prompt longer than max_prefix");
-  // a chunk of the prompt is one causal pass: 256 rows keep the tensor-core GEMMs at their largest row block
-  const int chunk = c->Mmax >= 256 ? 256 : c->Mmax / 64 * 64;
+  // a chunk of the prompt is one causal pass of up to PREFILL_ROWS rows (row blocks of 256 in the tensor-core GEMMs: the
+  // weights are unpacked once per pass and slab, whatever the number of row blocks)
+  const int chunk = c->Mmax >= PREFILL_ROWS ? PREFILL_ROWS : c->Mmax / 64 * 64;
   const int dm = c->d.d_model;
   for (int p0 = 0; p0 < n; p0 += chunk) {
     PassIO io;
@@ -635,11 +640,12 @@ int prefill_impl(mlora_ctx* c, const int32_t* ids, const __half* hidden, int n, 
     io.suffix_bound = 0;
     const bool last = (p0 + io.T >= n);
     io.logits = (last && c->d.vocab > 0 && out_last) ? c->logits : nullptr;
+    io.last_row_logits = true;
     plan_pass(c, io);
     int rc = forward(c, io);
     if (rc != MLORA_OK) return rc;
     if (last && out_last) {
-      const float* src = c->d.vocab > 0 ? c->logits + (size_t)(io.T - 1) * c->d.vocab : c->X + (size_t)(io.T - 1) * dm;
+      const float* src = c->d.vocab > 0 ? c->logits : c->X + (size_t)(io.T - 1) * dm;
       const size_t cnt = c->d.vocab > 0 ? (size_t)c->d.vocab : (size_t)dm;
       CK(run(c, MLORA_PROF_MISC, [&] { return launch_copy_rows_f32(src, out_last, cnt, c->stream); }));
     }
@@ -695,7 +701,7 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
   c->L = d.n_layers; c->Nq = Nq; c->Nkv = Nkv; c->Nqkv = Nq + 2 * Nkv;
   c->cap = d.max_suffix + d.max_tree;
   c->Mmax = d.max_streams * d.max_tree;
-  if (c->Mmax < 256) c->Mmax = 256;        // prefill passes have up to 256 rows
+  if (c->Mmax < PREFILL_ROWS) c->Mmax = PREFILL_ROWS;        // prefill passes have up to this many rows
 #define CKC(call)                                                                                  \
   do {                                                                                             \
     cudaError_t e__ = (call);                                                                      \
@@ -760,7 +766,7 @@ int mlora_create(const mlora_model_desc* desc, mlora_ctx** out) {
   CKC(cudaMalloc(&c->h, Mm * maxK * sizeof(__half)));
   CKC(cudaMalloc(&c->attn16, Mm * Nq * sizeof(__half)));
   CKC(cudaMalloc(&c->act16, Mm * F * sizeof(__half)));
-  if (d.vocab > 0) CKC(cudaMalloc(&c->logits, Mm * d.vocab * sizeof(float)));
+  if (d.vocab > 0) CKC(cudaMalloc(&c->logits, (size_t)d.max_streams * d.max_tree * d.vocab * sizeof(float)));   // (prefill: one row)
   CKC(cudaMalloc(&c->T, Mm * 3 * (d.lora_rank > 0 ? d.lora_rank : 1) * sizeof(float)));
   c->partial_floats = (size_t)16 << 20;               // 64 MB of split-K scratch
   CKC(cudaMalloc(&c->partial, c->partial_floats * sizeof(float)));
