@@ -1479,7 +1479,13 @@ int mlora_debug_set(mlora_ctx* c, int32_t key, int32_t value) {
   else if (key == 3) c->dbg_no_chain = value ? 1 : 0;
   else if (key == 4) c->dbg_no_tc = value ? 1 : 0;
   else if (key == 5) c->dbg_inject_stall = value ? 1 : 0;
-  else if (key == 6) c->step_mode = (value >= 0 && value <= 3) ? value : 0;
+  else if (key == 6) {
+    c->step_mode = (value >= 0 && value <= 3) ? value : 0;
+    // the single-kernel step expects the step's accumulators zero when it starts (it clears them on its way out); the
+    // kernel-per-projection path clears them when a step starts and leaves them used: clear them at every switch
+    if (c->step_tacc != nullptr) CK(cudaMemsetAsync(c->step_tacc, 0, c->step_acc_bytes, c->stream));
+    if (c->step_amax != nullptr) CK(cudaMemsetAsync(c->step_amax, 0, (size_t)c->sm_count * CHAIN_MAX_ROWS * sizeof(unsigned long long), c->stream));
+  }
   else if (key == 7) c->dbg_trace = value ? 1 : 0;
   else return fail(MLORA_ERR_ARG, "unknown debug key");
   return MLORA_OK;
