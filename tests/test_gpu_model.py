@@ -399,6 +399,32 @@ def test_step_timeline_of_the_default_decode_path(GpuModel):
     assert np.array_equal(res[0].view(np.uint32), res[1].view(np.uint32))
 
 
+def test_switching_decode_paths_in_one_context(GpuModel):
+    """Debug switch 6 in the middle of a context's life: steps of the single-kernel path that follow steps of the
+    kernel-per-projection path give, bit for bit, what a context that only ever ran the single-kernel path gives (the
+    step's accumulators are cleared at the switch)."""
+    from paper_2604_18655_b200 import binding as mb
+    cfg = TINYV
+    res = []
+    for warm_path in (2, 3):
+        m, orc, gm = make_pair(GpuModel, cfg, max_suffix=16)
+        gm.prefill(gen.make_prompt_ids(cfg, 0))
+        mb.mlora_debug_set(gm.ctx, 6, warm_path)
+        toks = np.array([1, 2, 3], dtype=np.int32)
+        for _ in range(2):
+            gm.decode([0, 1, -1], toks)
+        mb.mlora_reset_streams(gm.ctx)
+        mb.mlora_debug_set(gm.ctx, 6, 2)
+        hist = []
+        for _ in range(3):
+            toks, logits = gm.decode([0, 1, -1], toks)
+            hist.append(logits)
+        res.append(np.stack(hist))
+        mb.mlora_sync_status(gm.ctx)
+        gm.close()
+    assert np.array_equal(res[0].view(np.uint32), res[1].view(np.uint32))
+
+
 def test_decode_paths_agree(GpuModel):
     """The single-kernel step against the per-layer persistent projection kernel (debug switch 6) and the
     one-kernel-per-projection form of the same arithmetic (debug switch 3): logits and KV within the parity tolerance."""
